@@ -1,0 +1,268 @@
+/*
+ * ckpt_b200 - checkpointed CNN training step for one B200 (sm_100a), C ABI.
+ *
+ * Two halves:
+ *   - host planners: given the data sizes d_0..d_n of a layer chain, choose the checkpoint set that
+ *     minimises peak activation memory under one of the paper's two memory models;
+ *   - device executor: run one training step of a chain of layer units (forward keeping only the
+ *     checkpoints, backward that recomputes each segment from its nearest checkpoint) inside a
+ *     caller-provided activation arena, returning weight gradients and the arena's high-water mark.
+ *
+ * Conventions
+ *   - every function returns CKPT_OK (0) or a negative CKPT_E_* code; nothing throws or aborts;
+ *     ckpt_last_error() returns a thread-local, human-readable message for the last failure.
+ *   - "host" / "device" is stated for every pointer.  The library never allocates device memory:
+ *     arena, workspace, parameters and gradients are caller-owned (for example torch tensors).
+ *   - activations are NHWC; convolution matrices are [C_out][k][k][C_in]; fully connected matrices
+ *     are [out][in] with `in` enumerating the NHWC-flattened input.
+ *   - d_i is the byte size of unit i's output for the whole batch, rounded up to 256 bytes so that
+ *     every arena offset is aligned for vector and bulk-tensor access; d_0 is the input batch.
+ *   - checkpoint sets are byte masks is_ckpt[0..n]; indices 0 and n are always checkpoints
+ *     (Section 3.1 of the paper).
+ */
+#ifndef CKPT_B200_H
+#define CKPT_B200_H
+
+#include <stdint.h>
+
+#if defined(__GNUC__)
+#define CKPT_API __attribute__((visibility("default")))
+#else
+#define CKPT_API
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* ---------------------------------------------------------------- status codes */
+#define CKPT_OK 0
+#define CKPT_E_NULL (-1)           /* a required pointer is null                                  */
+#define CKPT_E_BAD_N (-2)          /* n < 1                                                       */
+#define CKPT_E_BAD_SIZE (-3)       /* some d_i < 1                                                */
+#define CKPT_E_OVERFLOW (-4)       /* 2 * sum(d) does not fit in int64                            */
+#define CKPT_E_BAD_PLAN (-5)       /* is_ckpt[0] or is_ckpt[n] is 0                               */
+#define CKPT_E_BAD_ARG (-6)        /* unknown enum value, inconsistent shapes, ...                */
+#define CKPT_E_ARENA_OOM (-7)      /* arena smaller than the plan's peak; nothing was launched    */
+#define CKPT_E_WORKSPACE (-8)      /* workspace smaller than ckpt_chain_workspace_bytes()         */
+#define CKPT_E_CUDA (-9)           /* a CUDA runtime/driver call failed (see ckpt_last_error)     */
+#define CKPT_E_DEVICE_TIMEOUT (-10)/* a bounded device-side wait gave up; results are invalid     */
+#define CKPT_E_UNSUPPORTED (-11)   /* shape/dtype combination has no kernel                       */
+#define CKPT_E_NO_DEVICE (-12)     /* no CUDA device / driver available                           */
+
+CKPT_API const char* ckpt_last_error(void);
+
+/* ---------------------------------------------------------------- host planners
+ *
+ * Algorithms (numbered as in the paper):
+ *   CKPT_ALGO_STATIC_N3  - Algorithm 3, "Checkpoint Selection" (Section 3.2): minimises Eq. (cost),
+ *                          sum of checkpoints + largest segment sum, in O(n^3).
+ *   CKPT_ALGO_DYNAMIC_N2 - Algorithm 5 (Section 4.1): minimises max_i m(i) of Eq. (memory) by the
+ *                          O(n^2) recursion Eq. (T-rec).
+ *   CKPT_ALGO_DYNAMIC_N  - Algorithm 6 (Section 4.2): same optimum by the monotone-queue /
+ *                          two-pointer search.
+ * Readings of the printed algorithms: data are d_0..d_n and the dynamic recursion runs down to
+ * i = 0 (answer M(0)); j ranges up to n inclusive; M(n) = d_n is the base case; Algorithm 3 forces
+ * d_n as a checkpoint (answer min_s s + d_n + M(n-1,s)) and inserts candidate i before reading the
+ * queue head, as Eq. (T) requires.  Ties: dynamic - the smallest next checkpoint attaining the
+ * minimum; static - the smallest segment cap, then the smallest previous checkpoint.
+ */
+#define CKPT_ALGO_STATIC_N3 0
+#define CKPT_ALGO_DYNAMIC_N2 1
+#define CKPT_ALGO_DYNAMIC_N 2
+
+/* d: host, n+1 sizes (>= 1).  is_ckpt: host, n+1 bytes, written (0/1).  peak_bytes: host, written:
+ * the objective value of the returned set under the algorithm's own memory model. */
+CKPT_API int ckpt_plan(int algo, int64_t n, const int64_t* d, uint8_t* is_ckpt, int64_t* peak_bytes);
+
+/* Same as ckpt_plan, also reporting how many inner-loop steps the search took (queue pushes, pops
+ * and pointer moves for the queue-based algorithms; (i,j) pairs for Algorithm 5). work: host. */
+CKPT_API int ckpt_plan_counted(int algo, int64_t n, const int64_t* d, uint8_t* is_ckpt,
+                      int64_t* peak_bytes, int64_t* work);
+
+/* Objective of an arbitrary checkpoint set.
+ *   CKPT_MODEL_STATIC  - Eq. (cost) (Section 3.1).
+ *   CKPT_MODEL_DYNAMIC - Eq. (memory)/(memory-simple) with s(h,i) of Eq. (s) (Section 4).
+ *   CKPT_MODEL_STORE_ALL - Algorithm 1: sum of d_0..d_n (is_ckpt ignored, may be null). */
+#define CKPT_MODEL_STATIC 0
+#define CKPT_MODEL_DYNAMIC 1
+#define CKPT_MODEL_STORE_ALL 2
+CKPT_API int ckpt_eval(int model, int64_t n, const int64_t* d, const uint8_t* is_ckpt, int64_t* peak_bytes);
+
+/* ---------------------------------------------------------------- arena schedule (host only)
+ *
+ * Execution policies = the paper's three memory schedules:
+ *   CKPT_POLICY_STORE_ALL - Algorithm 1: every d_i allocated and kept.
+ *   CKPT_POLICY_STATIC    - Algorithm 2: forward keeps checkpoints; backward frees the finished
+ *                           segment and recomputes the previous one; checkpoints are never freed.
+ *   CKPT_POLICY_DYNAMIC   - Algorithm 4: d_i released right after backward step i; one output-
+ *                           gradient buffer of size max(d_h..d_{i-1}) per segment, the old buffer
+ *                           being released before the next segment is recomputed, so that the
+ *                           high-water mark is exactly Eq. (memory).
+ *
+ * ckpt_arena_dry_run replays the allocation events of one step without touching a device.
+ * events (host, may be null): up to max_events records of 4 int64:
+ *   {kind (1 = alloc, 0 = free), tensor id (0..n = d_i, n+1 = gradient buffer), offset, size}.
+ * n_events / high_water_bytes / extent_bytes: host, written.  extent_bytes = highest arena offset
+ * ever occupied; the placement rule guarantees extent_bytes == high_water_bytes == ckpt_eval(). */
+#define CKPT_POLICY_STORE_ALL 0
+#define CKPT_POLICY_STATIC 1
+#define CKPT_POLICY_DYNAMIC 2
+CKPT_API int ckpt_arena_dry_run(int policy, int64_t n, const int64_t* d, const uint8_t* is_ckpt,
+                       int64_t* events, int64_t max_events, int64_t* n_events,
+                       int64_t* high_water_bytes, int64_t* extent_bytes);
+
+/* ---------------------------------------------------------------- layer-chain description
+ *
+ * A chain is Eq. (1): d_i = f_i(d_{i-1}, w_i), i = 1..n, followed by a loss.  Unit kinds:
+ *   CKPT_UNIT_CONV_BN_RELU - k x k cross-correlation (stride, zero padding, no bias), batch
+ *       normalisation in training mode (biased variance, eps 1e-5), ReLU.
+ *       parameters: w [c_out][k][k][c_in] (activation dtype), gamma [c_out] f32, beta [c_out] f32.
+ *   CKPT_UNIT_MAXPOOL      - k x k max pooling (stride, padding); the first maximum in row-major
+ *       window order receives the gradient.  No parameters.
+ *   CKPT_UNIT_FC           - fully connected on the flattened input, bias, optional ReLU
+ *       (flags & 1).  parameters: w [c_out][c_in] (activation dtype), b [c_out] f32.
+ *   CKPT_UNIT_AVGPOOL      - global average over H and W.  No parameters.
+ *   CKPT_UNIT_BOTTLENECK   - ResNet v1.5 bottleneck: 1x1 (c_in -> mid), 3x3 carrying the stride
+ *       (mid -> mid), 1x1 (mid -> c_out), each with batch norm; projection shortcut when
+ *       (flags & 2); ReLU after the residual add.  parameters: w1,g1,b1,w2,g2,b2,w3,g3,b3
+ *       [,wp,gp,bp].
+ * Parameter tensors are numbered consecutively over the chain in the order listed above.
+ * Gradients are always float32 with the parameter's shape.
+ */
+#define CKPT_UNIT_CONV_BN_RELU 0
+#define CKPT_UNIT_MAXPOOL 1
+#define CKPT_UNIT_FC 2
+#define CKPT_UNIT_AVGPOOL 3
+#define CKPT_UNIT_BOTTLENECK 4
+
+#define CKPT_DTYPE_F32 0   /* float32 storage and arithmetic (no tensor cores)                    */
+#define CKPT_DTYPE_BF16 1  /* bfloat16 storage, float32 accumulation                              */
+
+#define CKPT_LOSS_SUM 0        /* L = sum of every element of d_n                                 */
+#define CKPT_LOSS_SOFTMAX_CE 1 /* softmax cross-entropy over d_n's channels, mean over the batch  */
+
+typedef struct ckpt_unit_desc {
+    int32_t kind;
+    int32_t c_in;    /* FC: input features (must equal H*W*C of the incoming tensor)              */
+    int32_t c_out;
+    int32_t k;       /* filter / window size                                                      */
+    int32_t stride;
+    int32_t pad;
+    int32_t mid;     /* bottleneck width                                                          */
+    int32_t flags;   /* FC: bit 0 = ReLU; bottleneck: bit 1 = projection shortcut                 */
+} ckpt_unit_desc;
+
+typedef struct ckpt_chain ckpt_chain;  /* opaque, host memory owned by the library */
+
+/* units: host array of n descriptors (copied).  Shapes are checked unit by unit. */
+CKPT_API int ckpt_chain_create(const ckpt_unit_desc* units, int64_t n, int64_t batch, int32_t in_h,
+                      int32_t in_w, int32_t in_c, int dtype, int loss, ckpt_chain** out);
+CKPT_API void ckpt_chain_destroy(ckpt_chain* chain);
+
+/* d: host, n+1 entries written (bytes, 256-aligned).  shapes (host, may be null): 3*(n+1) int32
+ * {H, W, C} of d_0..d_n. */
+CKPT_API int ckpt_chain_sizes(const ckpt_chain* chain, int64_t* d, int32_t* shapes);
+CKPT_API int ckpt_chain_num_params(const ckpt_chain* chain, int64_t* count);
+/* unit (1-based index of the owning unit), elems (element count), dtype (CKPT_DTYPE_* of the
+ * parameter's storage; its gradient is always f32): host, written. */
+CKPT_API int ckpt_chain_param_info(const ckpt_chain* chain, int64_t p, int64_t* unit, int64_t* elems,
+                          int32_t* dtype);
+/* Plan-independent scratch the executor needs besides the arena: gradient carry buffers, the
+ * pre-normalisation buffer that each unit's backward re-derives, split-K partial sums, saved
+ * batch statistics.  bytes: host, written. */
+CKPT_API int ckpt_chain_workspace_bytes(const ckpt_chain* chain, int64_t* bytes);
+/* Kernel selection for dense contractions: 0 = automatic (tensor cores where a kernel exists),
+ * 1 = plain CUDA-core kernels only. */
+CKPT_API int ckpt_chain_set_impl(ckpt_chain* chain, int impl);
+
+/* ---------------------------------------------------------------- the training step
+ *
+ * One pass of Algorithm 1, 2 or 4 (policy) over one batch.  Follows the paper's "Require: weights
+ * w_1..w_n, input x (d_0), ground truth G", except that the weight update is left to the caller:
+ * the step *returns* g_i (Eq. (5)) for every parameter.
+ *
+ * batch:   host or device, d_0 payload (batch*H*W*C elements of the chain dtype); copied into the
+ *          arena at the start of the step, on `stream`.
+ * labels:  host or device int32[batch] (ignored for CKPT_LOSS_SUM, may be null).
+ * params:  host array of device pointers, one per parameter tensor.
+ * grads:   host array of device pointers (float32), written.
+ * arena:   device, arena_bytes >= ckpt_eval(model of policy) or CKPT_E_ARENA_OOM is returned before
+ *          anything is launched.  Contents on return are unspecified.
+ * workspace: device, ws_bytes >= ckpt_chain_workspace_bytes().
+ * stream:  a cudaStream_t (null = default stream).  The call returns after the stream has drained.
+ * report:  host, written.
+ * Determinism: every reduction has a fixed order, so gradients are bit-identical across policies
+ * and checkpoint sets for the same inputs.
+ */
+typedef struct ckpt_step_report {
+    int64_t peak_bytes;      /* arena high-water mark: max over time of live bytes               */
+    int64_t extent_bytes;    /* highest arena offset occupied                                    */
+    int64_t predicted_bytes; /* ckpt_eval() of (policy's model, is_ckpt)                         */
+    int64_t workspace_bytes; /* workspace actually required                                      */
+    int64_t launches;        /* kernels launched by this step                                    */
+    int64_t recomputed_units;/* unit forwards re-run during the backward phase                   */
+    double loss;
+    int32_t device_status;   /* 0, or the code written by a kernel whose bounded wait gave up    */
+    int32_t reserved;
+} ckpt_step_report;
+
+CKPT_API int ckpt_train_step(ckpt_chain* chain, const uint8_t* is_ckpt, int policy, const void* batch,
+                    const int32_t* labels, void* const* params, void* const* grads, void* arena,
+                    int64_t arena_bytes, void* workspace, int64_t ws_bytes, void* stream,
+                    ckpt_step_report* report);
+
+/* ---------------------------------------------------------------- single operations
+ *
+ * The kernels the step is made of, callable one at a time (used by the parity tests and for
+ * profiling).  All tensor pointers are device pointers; scratch is device memory of at least the
+ * size returned by the matching *_scratch_bytes call (may be null when that size is 0).
+ * impl: 0 = automatic, 1 = CUDA-core kernel, 2 = tensor-core kernel (CKPT_E_UNSUPPORTED if the
+ * shape has none).  Calls are asynchronous on `stream`.
+ *
+ * ckpt_conv2d_forward : z[n,ho,wo,co] = sum_{r,s,ci} x[n, ho*stride-pad+r, wo*stride-pad+s, ci] *
+ *                       w[co,r,s,ci]                                    (Eq. (1) for a conv unit)
+ * ckpt_conv2d_dgrad   : dx = (d z / d x)^T dz                           (Eq. (3))
+ * ckpt_conv2d_wgrad   : dw[co,r,s,ci] (f32) = sum_{n,ho,wo} dz * x      (Eq. (5))
+ */
+typedef struct ckpt_conv_shape {
+    int32_t n, h, w, c_in, c_out, k, stride, pad;
+} ckpt_conv_shape;
+
+CKPT_API int ckpt_conv2d_scratch_bytes(const ckpt_conv_shape* s, int dtype, int64_t* bytes);
+CKPT_API int ckpt_conv2d_forward(const ckpt_conv_shape* s, int dtype, int impl, const void* x, const void* w,
+                        void* z, void* scratch, int64_t scratch_bytes, void* stream);
+CKPT_API int ckpt_conv2d_dgrad(const ckpt_conv_shape* s, int dtype, int impl, const void* dz, const void* w,
+                      void* dx, void* scratch, int64_t scratch_bytes, void* stream);
+CKPT_API int ckpt_conv2d_wgrad(const ckpt_conv_shape* s, int dtype, int impl, const void* dz, const void* x,
+                      float* dw, void* scratch, int64_t scratch_bytes, void* stream);
+
+/* Batch normalisation (training mode) + ReLU over rows x channels (rows = N*H*W).
+ * forward : stats[0..c) = mean, [c..2c) = 1/sqrt(var+eps), [2c..3c) = scale, [3c..4c) = shift
+ *           (y = max(z*scale + shift, 0) when relu != 0, else z*scale+shift).
+ * backward: given dy and the same z/stats, writes dz (may alias dy), dgamma, dbeta.
+ * scratch: ckpt_bn_scratch_bytes(). */
+CKPT_API int ckpt_bn_scratch_bytes(int64_t rows, int32_t c, int64_t* bytes);
+CKPT_API int ckpt_bn_relu_forward(int dtype, int64_t rows, int32_t c, const void* z, const float* gamma,
+                         const float* beta, int relu, void* y, float* stats, void* scratch,
+                         void* stream);
+CKPT_API int ckpt_bn_relu_backward(int dtype, int64_t rows, int32_t c, const void* dy, const void* z,
+                          const float* gamma, const float* stats, int relu, void* dz, float* dgamma,
+                          float* dbeta, void* scratch, void* stream);
+
+/* Max pooling, NHWC.  backward recomputes the arg-max from x. */
+CKPT_API int ckpt_maxpool_forward(int dtype, int32_t n, int32_t h, int32_t w, int32_t c, int32_t k,
+                         int32_t stride, int32_t pad, const void* x, void* y, void* stream);
+CKPT_API int ckpt_maxpool_backward(int dtype, int32_t n, int32_t h, int32_t w, int32_t c, int32_t k,
+                          int32_t stride, int32_t pad, const void* x, const void* dy, void* dx,
+                          void* stream);
+
+/* Softmax cross-entropy, mean over the batch: loss (device float, written), dlogits (chain dtype).
+ * labels: device int32. */
+CKPT_API int ckpt_softmax_ce(int dtype, int32_t batch, int32_t classes, const void* logits,
+                    const int32_t* labels, float* loss, void* dlogits, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* CKPT_B200_H */

@@ -1,0 +1,509 @@
+// Layer-chain description, workspace layout and the step executor (Algorithms 1, 2 and 4).
+//
+// The executor is host control flow only: it walks the units, asks the arena where each d_i lives,
+// and launches kernels.  The same walk with launches disabled is the arena dry run.
+#include <cuda_runtime.h>
+
+#include <algorithm>
+#include <cstring>
+
+#include "internal.h"
+
+namespace ckpt {
+
+struct Shape { int h, w, c; };
+
+struct Unit {
+    ckpt_unit_desc desc;
+    Shape in, out;
+    int param_first = 0, n_params = 0;
+    int64_t stats_off = 0;       // float offset of this unit's saved batch statistics
+    ConvGeom geom;               // conv / fc as a convolution
+};
+
+struct ParamInfo { int64_t unit, elems; int32_t dtype; };
+
+}  // namespace ckpt
+
+struct ckpt_chain {
+    std::vector<ckpt::Unit> units;       // units[0] is unit 1
+    std::vector<int64_t> d;              // d_0..d_n, bytes
+    std::vector<ckpt::Shape> shapes;
+    std::vector<ckpt::ParamInfo> params;
+    int64_t batch = 0;
+    int dtype = 0, loss = 0, impl = 0;
+    // workspace layout (byte offsets)
+    int64_t max_d = 0, off_g0 = 0, off_g1 = 0, off_z = 0, off_scr = 0, scr_bytes = 0, off_stats = 0,
+            off_misc = 0, ws_bytes = 0;
+};
+
+namespace ckpt {
+
+static int out_size(int h, int k, int stride, int pad) { return (h + 2 * pad - k) / stride + 1; }
+
+static int check_conv(const ckpt_unit_desc& u, const Shape& in, int64_t idx) {
+    if (u.k < 1 || u.stride < 1 || u.pad < 0 || u.c_out < 1) { set_error("unit %lld: bad conv parameters", (long long)idx); return CKPT_E_BAD_ARG; }
+    if (u.c_in != in.c) { set_error("unit %lld: c_in %d != incoming channels %d", (long long)idx, u.c_in, in.c); return CKPT_E_BAD_ARG; }
+    if (in.h + 2 * u.pad < u.k || in.w + 2 * u.pad < u.k) { set_error("unit %lld: window larger than input", (long long)idx); return CKPT_E_BAD_ARG; }
+    return CKPT_OK;
+}
+
+static bool use_tc(const ckpt_chain* ch, const ConvGeom& g) {
+    return ch->impl == 0 && tc_conv_supported(ch->dtype, g);
+}
+
+// ------------------------------------------------------------------------------------------------
+// executor
+// ------------------------------------------------------------------------------------------------
+struct StepCtx {
+    ckpt_chain* ch;
+    const uint8_t* is_ckpt;
+    int policy;
+    bool dry;
+    char* arena_base;
+    char* ws;
+    void* const* params;
+    void* const* grads;
+    const void* batch;
+    const int32_t* labels;
+    cudaStream_t stream;
+    Arena* arena;
+    int64_t recomputed = 0;
+    int* status() const { return (int*)(ws + ch->off_misc + 64); }
+};
+
+static const int64_t kGradId = 1000000007;   // arena id of the per-segment gradient buffer
+
+static int conv_forward_any(StepCtx& c, const ConvGeom& g, const void* x, const void* w, void* z,
+                            const float* bias, int relu) {
+    if (!bias && use_tc(c.ch, g))
+        return tc_conv_fwd(g, x, w, z, c.ws + c.ch->off_scr, c.ch->scr_bytes, c.status(), c.stream);
+    return simt_conv_fwd(c.ch->dtype, g, x, w, z, bias, relu, c.stream);
+}
+static int conv_dgrad_any(StepCtx& c, const ConvGeom& g, const void* dz, const void* w, void* dx) {
+    if (use_tc(c.ch, g))
+        return tc_conv_dgrad(g, dz, w, dx, c.ws + c.ch->off_scr, c.ch->scr_bytes, c.status(), c.stream);
+    return simt_conv_dgrad(c.ch->dtype, g, dz, w, dx, c.stream);
+}
+static int conv_wgrad_any(StepCtx& c, const ConvGeom& g, const void* dz, const void* x, float* dw) {
+    if (use_tc(c.ch, g))
+        return tc_conv_wgrad(g, dz, x, dw, c.ws + c.ch->off_scr, c.ch->scr_bytes, c.status(), c.stream);
+    return simt_conv_wgrad(c.ch->dtype, g, dz, x, dw, c.ws + c.ch->off_scr, c.ch->scr_bytes, c.stream);
+}
+
+// d_i = f_i(d_{i-1}, w_i)  (Eq. (1)); i is 1-based.
+static int unit_forward(StepCtx& c, int64_t i, const void* x, void* y) {
+    if (c.dry) return CKPT_OK;
+    const Unit& u = c.ch->units[i - 1];
+    const int dt = c.ch->dtype;
+    const int64_t rows = c.ch->batch * u.out.h * u.out.w;
+    void* const* p = c.params + u.param_first;
+    char* ws = c.ws;
+    switch (u.desc.kind) {
+        case CKPT_UNIT_CONV_BN_RELU: {
+            void* z = ws + c.ch->off_z;
+            int rc = conv_forward_any(c, u.geom, x, p[0], z, nullptr, 0);
+            if (rc) return rc;
+            float* stats = (float*)(ws + c.ch->off_stats) + u.stats_off;
+            return bn_relu_forward(dt, rows, u.out.c, z, (const float*)p[1], (const float*)p[2], 1, y,
+                                   stats, ws + c.ch->off_scr, c.stream);
+        }
+        case CKPT_UNIT_MAXPOOL:
+            return maxpool_forward(dt, (int)c.ch->batch, u.in.h, u.in.w, u.in.c, u.desc.k, u.desc.stride,
+                                   u.desc.pad, x, y, c.stream);
+        case CKPT_UNIT_AVGPOOL:
+            return avgpool_forward(dt, (int)c.ch->batch, u.in.h, u.in.w, u.in.c, x, y, c.stream);
+        case CKPT_UNIT_FC:
+            return conv_forward_any(c, u.geom, x, p[0], y, (const float*)p[1], u.desc.flags & 1);
+    }
+    set_error("unit kind %d has no forward kernel", u.desc.kind);
+    return CKPT_E_UNSUPPORTED;
+}
+
+// r_i and g_i (Eqs. (3) and (5)): g_in = dL/dd_i (may be overwritten), g_out = dL/dd_{i-1} or null.
+static int unit_backward(StepCtx& c, int64_t i, const void* x, const void* y, void* g_in, void* g_out) {
+    if (c.dry) return CKPT_OK;
+    const Unit& u = c.ch->units[i - 1];
+    const int dt = c.ch->dtype;
+    const int64_t rows = c.ch->batch * u.out.h * u.out.w;
+    void* const* p = c.params + u.param_first;
+    void* const* g = c.grads + u.param_first;
+    char* ws = c.ws;
+    int rc;
+    switch (u.desc.kind) {
+        case CKPT_UNIT_CONV_BN_RELU: {
+            // The pre-normalisation tensor is not part of the chain's stored data: derive it again.
+            void* z = ws + c.ch->off_z;
+            if ((rc = conv_forward_any(c, u.geom, x, p[0], z, nullptr, 0))) return rc;
+            float* stats = (float*)(ws + c.ch->off_stats) + u.stats_off;
+            if ((rc = bn_relu_backward(dt, rows, u.out.c, g_in, z, (const float*)p[1], stats, 1, g_in,
+                                       (float*)g[1], (float*)g[2], ws + c.ch->off_scr, c.stream))) return rc;
+            if ((rc = conv_wgrad_any(c, u.geom, g_in, x, (float*)g[0]))) return rc;
+            if (g_out) return conv_dgrad_any(c, u.geom, g_in, p[0], g_out);
+            return CKPT_OK;
+        }
+        case CKPT_UNIT_MAXPOOL:
+            if (!g_out) return CKPT_OK;
+            return maxpool_backward(dt, (int)c.ch->batch, u.in.h, u.in.w, u.in.c, u.desc.k, u.desc.stride,
+                                    u.desc.pad, x, g_in, g_out, c.stream);
+        case CKPT_UNIT_AVGPOOL:
+            if (!g_out) return CKPT_OK;
+            return avgpool_backward(dt, (int)c.ch->batch, u.in.h, u.in.w, u.in.c, g_in, g_out, c.stream);
+        case CKPT_UNIT_FC: {
+            const int64_t elems = c.ch->batch * u.out.c;
+            if (u.desc.flags & 1)
+                if ((rc = relu_mask_inplace(dt, elems, g_in, y, c.stream))) return rc;
+            if ((rc = column_sums(dt, c.ch->batch, u.out.c, g_in, (float*)g[1], c.stream))) return rc;
+            if ((rc = conv_wgrad_any(c, u.geom, g_in, x, (float*)g[0]))) return rc;
+            if (g_out) return conv_dgrad_any(c, u.geom, g_in, p[0], g_out);
+            return CKPT_OK;
+        }
+    }
+    set_error("unit kind %d has no backward kernel", u.desc.kind);
+    return CKPT_E_UNSUPPORTED;
+}
+
+static int run_step(StepCtx& c, double* loss_out) {
+    ckpt_chain* ch = c.ch;
+    const int64_t n = (int64_t)ch->units.size();
+    const std::vector<int64_t>& d = ch->d;
+    Arena& A = *c.arena;
+    const bool store_all = c.policy == CKPT_POLICY_STORE_ALL;
+    auto ck = [&](int64_t i) { return store_all || c.is_ckpt[i] != 0; };
+    auto ptr = [&](int64_t id) -> void* {
+        int64_t off = A.offset_of(id);
+        return (c.dry || off < 0) ? nullptr : (void*)(c.arena_base + off);
+    };
+    int rc;
+    int64_t off;
+
+    // ---------------- forward phase
+    if ((rc = A.alloc_stack(0, d[0], &off))) return rc;
+    if (!c.dry) {
+        const int64_t payload = ch->batch * ch->shapes[0].h * ch->shapes[0].w * ch->shapes[0].c * dtype_size(ch->dtype);
+        cudaError_t e = cudaMemcpyAsync(c.arena_base + off, c.batch, payload, cudaMemcpyDefault, c.stream);
+        if (e != cudaSuccess) return cuda_fail(e, "copy of the input batch into the arena");
+    }
+    // Side of each forward temporary: the one just before a checkpoint sits at the top of the slab,
+    // the one before it on the stack, and so on alternately.
+    std::vector<uint8_t> top_side(n + 1, 0);
+    for (int64_t i = n, dist = 0; i >= 1; --i) {
+        if (ck(i)) dist = 0; else { top_side[i] = (dist % 2 == 0); ++dist; }
+    }
+    if (store_all) {
+        for (int64_t i = 1; i <= n; ++i) if ((rc = A.alloc_stack(i, d[i], &off))) return rc;
+    }
+    for (int64_t i = 1; i <= n; ++i) {
+        if (!store_all) {
+            if (ck(i) || !top_side[i]) rc = A.alloc_stack(i, d[i], &off);
+            else rc = A.alloc_top(i, d[i], &off);
+            if (rc) return rc;
+        }
+        if ((rc = unit_forward(c, i, ptr(i - 1), ptr(i)))) return rc;
+        if (!ck(i - 1)) if ((rc = A.release(i - 1))) return rc;
+    }
+
+    // ---------------- loss and dL/dd_n
+    char* gbuf[2] = {c.dry ? nullptr : c.ws + ch->off_g0, c.dry ? nullptr : c.ws + ch->off_g1};
+    void* g_cur = gbuf[0];
+    if (!c.dry) {
+        const Shape& so = ch->shapes[n];
+        if (ch->loss == CKPT_LOSS_SOFTMAX_CE) {
+            const int32_t* lab = (const int32_t*)(c.ws + ch->off_misc + 128 + 256);
+            cudaError_t e = cudaMemcpyAsync((void*)lab, c.labels, ch->batch * sizeof(int32_t), cudaMemcpyDefault, c.stream);
+            if (e != cudaSuccess) return cuda_fail(e, "copy of the labels");
+            rc = softmax_ce(ch->dtype, (int)ch->batch, so.h * so.w * so.c, ptr(n), lab,
+                            (float*)(c.ws + ch->off_misc), g_cur, (float*)(c.ws + ch->off_scr), c.stream);
+        } else {
+            rc = sum_loss(ch->dtype, ch->batch * so.h * so.w * so.c, ptr(n), (double*)(c.ws + ch->off_misc),
+                          g_cur, (double*)(c.ws + ch->off_scr), c.stream);
+        }
+        if (rc) return rc;
+    }
+
+    // ---------------- backward phase
+    bool have_r = false;            // Algorithm 4: a per-segment gradient buffer is live in the arena
+    bool g_in_r = false;            // the current gradient lives in that buffer
+    std::vector<int64_t> live_segment;
+    for (int64_t i = n; i >= 1; --i) {
+        if (!store_all && c.is_ckpt[i]) {
+            int64_t h = i - 1;
+            while (!c.is_ckpt[h]) --h;
+            if (c.policy == CKPT_POLICY_DYNAMIC) {
+                if (have_r) {
+                    if (g_in_r) {
+                        // the gradient entering the next segment must outlive the buffer it sits in
+                        if (!c.dry && (rc = device_copy(gbuf[0], g_cur, d[i], c.stream))) return rc;
+                        g_cur = gbuf[0];
+                        g_in_r = false;
+                    }
+                    if ((rc = A.release(kGradId))) return rc;
+                }
+            } else {
+                for (int64_t k : live_segment) if ((rc = A.release(k))) return rc;
+                live_segment.clear();
+            }
+            for (int64_t k = h + 1; k < i; ++k) {
+                if ((rc = A.alloc_stack(k, d[k], &off))) return rc;
+                if ((rc = unit_forward(c, k, ptr(k - 1), ptr(k)))) return rc;
+                ++c.recomputed;
+                if (c.policy == CKPT_POLICY_STATIC) live_segment.push_back(k);
+            }
+            if (c.policy == CKPT_POLICY_DYNAMIC) {
+                int64_t r = 0;
+                for (int64_t k = h; k < i; ++k) r = std::max(r, d[k]);
+                if ((rc = A.alloc_stack(kGradId, r, &off))) return rc;
+                have_r = true;
+            }
+        }
+        // where the outgoing gradient goes: the segment's buffer (Algorithm 4) or the other carry buffer
+        void* g_next;
+        bool next_in_r = false;
+        if (c.policy == CKPT_POLICY_DYNAMIC && !g_in_r) { g_next = ptr(kGradId); next_in_r = true; }
+        else if (c.policy == CKPT_POLICY_DYNAMIC) g_next = gbuf[0];
+        else g_next = (g_cur == gbuf[0]) ? gbuf[1] : gbuf[0];
+        const bool need_dx = i > 1;   // the gradient w.r.t. the input batch is never used
+        if ((rc = unit_backward(c, i, ptr(i - 1), ptr(i), g_cur, need_dx ? g_next : nullptr))) return rc;
+        if (need_dx) { g_cur = g_next; g_in_r = next_in_r; }
+        if (c.policy == CKPT_POLICY_DYNAMIC) if ((rc = A.release(i))) return rc;
+    }
+
+    if (!c.dry) {
+        int status = 0;
+        cudaError_t e;
+        if (ch->loss == CKPT_LOSS_SOFTMAX_CE) {
+            float l = 0;
+            e = cudaMemcpyAsync(&l, c.ws + ch->off_misc, sizeof(float), cudaMemcpyDeviceToHost, c.stream);
+            if (e == cudaSuccess) e = cudaMemcpyAsync(&status, c.status(), sizeof(int), cudaMemcpyDeviceToHost, c.stream);
+            if (e == cudaSuccess) e = cudaStreamSynchronize(c.stream);
+            *loss_out = l;
+        } else {
+            double l = 0;
+            e = cudaMemcpyAsync(&l, c.ws + ch->off_misc, sizeof(double), cudaMemcpyDeviceToHost, c.stream);
+            if (e == cudaSuccess) e = cudaMemcpyAsync(&status, c.status(), sizeof(int), cudaMemcpyDeviceToHost, c.stream);
+            if (e == cudaSuccess) e = cudaStreamSynchronize(c.stream);
+            *loss_out = l;
+        }
+        if (e != cudaSuccess) return cuda_fail(e, "end-of-step synchronisation");
+        if (status != 0) { set_error("a device-side wait gave up (status %d)", status); return CKPT_E_DEVICE_TIMEOUT; }
+    }
+    return CKPT_OK;
+}
+
+static int policy_model(int policy) {
+    return policy == CKPT_POLICY_STORE_ALL ? CKPT_MODEL_STORE_ALL
+         : policy == CKPT_POLICY_STATIC ? CKPT_MODEL_STATIC : CKPT_MODEL_DYNAMIC;
+}
+
+}  // namespace ckpt
+
+using namespace ckpt;
+
+extern "C" {
+
+int ckpt_arena_dry_run(int policy, int64_t n, const int64_t* d, const uint8_t* is_ckpt, int64_t* events,
+                       int64_t max_events, int64_t* n_events, int64_t* high_water_bytes, int64_t* extent_bytes) {
+    if (policy < 0 || policy > 2) { set_error("unknown policy %d", policy); return CKPT_E_BAD_ARG; }
+    int64_t predicted = 0;
+    int rc = eval_model(policy_model(policy), n, d, is_ckpt, &predicted);
+    if (rc) return rc;
+    ckpt_chain fake;
+    fake.units.resize(n);
+    fake.d.assign(d, d + n + 1);
+    fake.shapes.resize(n + 1);
+    Arena arena(predicted);
+    StepCtx c{};
+    c.ch = &fake; c.is_ckpt = is_ckpt; c.policy = policy; c.dry = true; c.arena = &arena;
+    double loss = 0;
+    rc = run_step(c, &loss);
+    if (rc) return rc;
+    if (n_events) *n_events = (int64_t)arena.events.size();
+    if (events) {
+        int64_t m = std::min<int64_t>(max_events, (int64_t)arena.events.size());
+        for (int64_t e = 0; e < m; ++e) {
+            const ArenaEvent& ev = arena.events[e];
+            events[4 * e + 0] = ev.kind;
+            events[4 * e + 1] = ev.id == kGradId ? n + 1 : ev.id;
+            events[4 * e + 2] = ev.offset;
+            events[4 * e + 3] = ev.size;
+        }
+    }
+    if (high_water_bytes) *high_water_bytes = arena.high_water();
+    if (extent_bytes) *extent_bytes = arena.extent();
+    return CKPT_OK;
+}
+
+int ckpt_chain_create(const ckpt_unit_desc* units, int64_t n, int64_t batch, int32_t in_h, int32_t in_w,
+                      int32_t in_c, int dtype, int loss, ckpt_chain** out) {
+    if (!units || !out) { set_error("null pointer"); return CKPT_E_NULL; }
+    if (n < 1) { set_error("n < 1"); return CKPT_E_BAD_N; }
+    if (batch < 1 || in_h < 1 || in_w < 1 || in_c < 1) { set_error("bad input shape"); return CKPT_E_BAD_ARG; }
+    if (dtype != CKPT_DTYPE_F32 && dtype != CKPT_DTYPE_BF16) { set_error("unknown dtype %d", dtype); return CKPT_E_BAD_ARG; }
+    if (loss != CKPT_LOSS_SUM && loss != CKPT_LOSS_SOFTMAX_CE) { set_error("unknown loss %d", loss); return CKPT_E_BAD_ARG; }
+    ckpt_chain* ch = new ckpt_chain();
+    ch->batch = batch; ch->dtype = dtype; ch->loss = loss;
+    const int64_t es = dtype_size(dtype);
+    Shape cur{in_h, in_w, in_c};
+    ch->shapes.push_back(cur);
+    ch->d.push_back(align_up(batch * cur.h * cur.w * cur.c * es, 256));
+    int64_t stats_floats = 0, max_z = 0, scr = 256;
+    for (int64_t i = 1; i <= n; ++i) {
+        Unit u;
+        u.desc = units[i - 1];
+        u.in = cur;
+        u.param_first = (int)ch->params.size();
+        int rc = CKPT_OK;
+        switch (u.desc.kind) {
+            case CKPT_UNIT_CONV_BN_RELU: {
+                rc = check_conv(u.desc, cur, i);
+                if (rc) break;
+                u.out = {out_size(cur.h, u.desc.k, u.desc.stride, u.desc.pad),
+                         out_size(cur.w, u.desc.k, u.desc.stride, u.desc.pad), u.desc.c_out};
+                u.geom = {(int)batch, cur.h, cur.w, cur.c, u.out.h, u.out.w, u.out.c, u.desc.k, u.desc.stride, u.desc.pad};
+                ch->params.push_back({i, (int64_t)u.desc.c_out * u.desc.k * u.desc.k * u.desc.c_in, dtype});
+                ch->params.push_back({i, u.desc.c_out, CKPT_DTYPE_F32});
+                ch->params.push_back({i, u.desc.c_out, CKPT_DTYPE_F32});
+                u.stats_off = stats_floats;
+                stats_floats += 4 * (int64_t)u.desc.c_out;
+                const int64_t rows = batch * u.out.h * u.out.w;
+                max_z = std::max(max_z, align_up(rows * u.out.c * es, 256));
+                scr = std::max(scr, bn_scratch_bytes(rows, u.out.c));
+                scr = std::max(scr, simt_wgrad_scratch_bytes(u.geom));
+                if (tc_conv_supported(dtype, u.geom)) scr = std::max(scr, tc_conv_scratch_bytes(u.geom));
+                break;
+            }
+            case CKPT_UNIT_MAXPOOL:
+                if (u.desc.k < 1 || u.desc.stride < 1 || u.desc.pad < 0 || 2 * u.desc.pad > u.desc.k ||
+                    cur.h + 2 * u.desc.pad < u.desc.k || cur.w + 2 * u.desc.pad < u.desc.k) {
+                    set_error("unit %lld: bad pooling parameters", (long long)i); rc = CKPT_E_BAD_ARG; break;
+                }
+                u.out = {out_size(cur.h, u.desc.k, u.desc.stride, u.desc.pad),
+                         out_size(cur.w, u.desc.k, u.desc.stride, u.desc.pad), cur.c};
+                break;
+            case CKPT_UNIT_AVGPOOL:
+                u.out = {1, 1, cur.c};
+                break;
+            case CKPT_UNIT_FC: {
+                if (u.desc.c_in != cur.h * cur.w * cur.c || u.desc.c_out < 1) {
+                    set_error("unit %lld: fc c_in %d != flattened input %d", (long long)i, u.desc.c_in, cur.h * cur.w * cur.c);
+                    rc = CKPT_E_BAD_ARG; break;
+                }
+                u.out = {1, 1, u.desc.c_out};
+                u.geom = {(int)batch, 1, 1, u.desc.c_in, 1, 1, u.desc.c_out, 1, 1, 0};
+                ch->params.push_back({i, (int64_t)u.desc.c_out * u.desc.c_in, dtype});
+                ch->params.push_back({i, u.desc.c_out, CKPT_DTYPE_F32});
+                scr = std::max(scr, simt_wgrad_scratch_bytes(u.geom));
+                if (tc_conv_supported(dtype, u.geom)) scr = std::max(scr, tc_conv_scratch_bytes(u.geom));
+                break;
+            }
+            default:
+                set_error("unit %lld: kind %d is not implemented", (long long)i, u.desc.kind);
+                rc = CKPT_E_UNSUPPORTED;
+        }
+        if (rc) { delete ch; return rc; }
+        u.n_params = (int)ch->params.size() - u.param_first;
+        cur = u.out;
+        ch->shapes.push_back(cur);
+        ch->d.push_back(align_up(batch * cur.h * cur.w * cur.c * es, 256));
+        ch->units.push_back(u);
+    }
+    scr = std::max<int64_t>(scr, std::max<int64_t>(sum_loss_scratch_bytes(), batch * (int64_t)sizeof(float)));
+    ch->max_d = *std::max_element(ch->d.begin(), ch->d.end());
+    int64_t o = 0;
+    ch->off_g0 = o; o += ch->max_d;
+    ch->off_g1 = o; o += ch->max_d;
+    ch->off_z = o; o += std::max<int64_t>(max_z, 256);
+    ch->off_scr = o; ch->scr_bytes = align_up(scr, 256); o += ch->scr_bytes;
+    ch->off_stats = o; o += align_up(std::max<int64_t>(stats_floats, 1) * 4, 256);
+    ch->off_misc = o; o += align_up(128 + 256 + batch * 4, 256);
+    ch->ws_bytes = o;
+    *out = ch;
+    return CKPT_OK;
+}
+
+void ckpt_chain_destroy(ckpt_chain* chain) { delete chain; }
+
+int ckpt_chain_sizes(const ckpt_chain* chain, int64_t* d, int32_t* shapes) {
+    if (!chain || !d) { set_error("null pointer"); return CKPT_E_NULL; }
+    for (size_t i = 0; i < chain->d.size(); ++i) {
+        d[i] = chain->d[i];
+        if (shapes) { shapes[3 * i] = chain->shapes[i].h; shapes[3 * i + 1] = chain->shapes[i].w; shapes[3 * i + 2] = chain->shapes[i].c; }
+    }
+    return CKPT_OK;
+}
+
+int ckpt_chain_num_params(const ckpt_chain* chain, int64_t* count) {
+    if (!chain || !count) { set_error("null pointer"); return CKPT_E_NULL; }
+    *count = (int64_t)chain->params.size();
+    return CKPT_OK;
+}
+
+int ckpt_chain_param_info(const ckpt_chain* chain, int64_t p, int64_t* unit, int64_t* elems, int32_t* dtype) {
+    if (!chain) { set_error("null pointer"); return CKPT_E_NULL; }
+    if (p < 0 || p >= (int64_t)chain->params.size()) { set_error("parameter index out of range"); return CKPT_E_BAD_ARG; }
+    if (unit) *unit = chain->params[p].unit;
+    if (elems) *elems = chain->params[p].elems;
+    if (dtype) *dtype = chain->params[p].dtype;
+    return CKPT_OK;
+}
+
+int ckpt_chain_workspace_bytes(const ckpt_chain* chain, int64_t* bytes) {
+    if (!chain || !bytes) { set_error("null pointer"); return CKPT_E_NULL; }
+    *bytes = chain->ws_bytes;
+    return CKPT_OK;
+}
+
+int ckpt_chain_set_impl(ckpt_chain* chain, int impl) {
+    if (!chain) { set_error("null pointer"); return CKPT_E_NULL; }
+    if (impl != 0 && impl != 1) { set_error("impl must be 0 or 1"); return CKPT_E_BAD_ARG; }
+    chain->impl = impl;
+    return CKPT_OK;
+}
+
+int ckpt_train_step(ckpt_chain* chain, const uint8_t* is_ckpt, int policy, const void* batch,
+                    const int32_t* labels, void* const* params, void* const* grads, void* arena,
+                    int64_t arena_bytes, void* workspace, int64_t ws_bytes, void* stream,
+                    ckpt_step_report* report) {
+    if (!chain || !batch || !params || !grads || !arena || !workspace || !report) { set_error("null pointer"); return CKPT_E_NULL; }
+    if (policy < 0 || policy > 2) { set_error("unknown policy %d", policy); return CKPT_E_BAD_ARG; }
+    if (policy != CKPT_POLICY_STORE_ALL && !is_ckpt) { set_error("is_ckpt is null"); return CKPT_E_NULL; }
+    if (chain->loss == CKPT_LOSS_SOFTMAX_CE && !labels) { set_error("labels are null"); return CKPT_E_NULL; }
+    for (size_t p = 0; p < chain->params.size(); ++p)
+        if (!params[p] || !grads[p]) { set_error("parameter or gradient pointer %zu is null", p); return CKPT_E_NULL; }
+    const int64_t n = (int64_t)chain->units.size();
+    memset(report, 0, sizeof(*report));
+    int64_t predicted = 0;
+    int rc = eval_model(policy_model(policy), n, chain->d.data(), is_ckpt, &predicted);
+    if (rc) return rc;
+    report->predicted_bytes = predicted;
+    report->workspace_bytes = chain->ws_bytes;
+    if (arena_bytes < predicted) {
+        set_error("arena of %lld bytes is smaller than the plan's peak of %lld bytes", (long long)arena_bytes, (long long)predicted);
+        return CKPT_E_ARENA_OOM;
+    }
+    if (ws_bytes < chain->ws_bytes) {
+        set_error("workspace of %lld bytes, %lld needed", (long long)ws_bytes, (long long)chain->ws_bytes);
+        return CKPT_E_WORKSPACE;
+    }
+    int ndev = 0;
+    if (cudaGetDeviceCount(&ndev) != cudaSuccess || ndev == 0) { set_error("no CUDA device"); return CKPT_E_NO_DEVICE; }
+    Arena ar(predicted);
+    StepCtx c{};
+    c.ch = chain; c.is_ckpt = is_ckpt; c.policy = policy; c.dry = false;
+    c.arena_base = (char*)arena; c.ws = (char*)workspace; c.params = params; c.grads = grads;
+    c.batch = batch; c.labels = labels; c.stream = (cudaStream_t)stream; c.arena = &ar;
+    cudaError_t e = cudaMemsetAsync(c.ws + chain->off_misc, 0, 128, c.stream);
+    if (e != cudaSuccess) return cuda_fail(e, "clearing the status words");
+    const int64_t launches0 = g_launches;
+    double loss = 0;
+    rc = run_step(c, &loss);
+    report->peak_bytes = ar.high_water();
+    report->extent_bytes = ar.extent();
+    report->launches = g_launches - launches0;
+    report->recomputed_units = c.recomputed;
+    report->loss = loss;
+    if (rc == CKPT_E_DEVICE_TIMEOUT) report->device_status = 1;
+    return rc;
+}
+
+}  // extern "C"

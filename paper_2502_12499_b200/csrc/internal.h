@@ -1,0 +1,104 @@
+// Internal declarations shared by the translation units of libckpt_b200 (not part of the C ABI).
+#pragma once
+#include <cstdint>
+#include <cstddef>
+#include <string>
+#include <vector>
+
+#include "../../include/ckpt_b200.h"
+
+namespace ckpt {
+
+void set_error(const char* fmt, ...);
+int cuda_fail(int err, const char* what);   // records the CUDA error string, returns CKPT_E_CUDA
+
+inline int64_t align_up(int64_t v, int64_t a) { return (v + a - 1) / a * a; }
+inline int64_t dtype_size(int dtype) { return dtype == CKPT_DTYPE_BF16 ? 2 : 4; }
+
+// Number of kernels launched since the library was loaded (incremented by every launcher).
+extern int64_t g_launches;
+
+// ------------------------------------------------------------------ host planners (planner.cpp)
+int validate_sizes(int64_t n, const int64_t* d);
+int plan_static_n3(int64_t n, const int64_t* d, uint8_t* is_ckpt, int64_t* peak, int64_t* work);
+int plan_dynamic_n2(int64_t n, const int64_t* d, uint8_t* is_ckpt, int64_t* peak, int64_t* work);
+int plan_dynamic_n(int64_t n, const int64_t* d, uint8_t* is_ckpt, int64_t* peak, int64_t* work);
+int eval_model(int model, int64_t n, const int64_t* d, const uint8_t* is_ckpt, int64_t* peak);
+
+// ------------------------------------------------------------------ arena bookkeeping (arena.cpp)
+struct ArenaEvent { int64_t kind, id, offset, size; };
+
+// Offsets inside one slab of `capacity` bytes.  Checkpoints and recomputed segments form a stack
+// that grows from offset 0; forward-phase temporaries alternate between the top of the slab and
+// the top of the stack so that two consecutive temporaries never fragment the slab.
+class Arena {
+public:
+    explicit Arena(int64_t capacity) : capacity_(capacity) {}
+    int alloc_stack(int64_t id, int64_t size, int64_t* offset);
+    int alloc_top(int64_t id, int64_t size, int64_t* offset);
+    int release(int64_t id);
+    bool is_live(int64_t id) const;
+    int64_t offset_of(int64_t id) const;
+    int64_t high_water() const { return high_water_; }
+    int64_t extent() const { return extent_; }
+    std::vector<ArenaEvent> events;
+private:
+    struct Block { int64_t id, off, size; bool top; };
+    int64_t stack_top() const;
+    int64_t top_floor() const;
+    void account(int64_t id, int64_t off, int64_t size, bool top);
+    std::vector<Block> live_;
+    int64_t capacity_, live_bytes_ = 0, high_water_ = 0, extent_ = 0;
+};
+
+// ------------------------------------------------------------------ kernel launchers (kernels_simt.cu)
+struct ConvGeom {
+    int n, h, w, cin, ho, wo, cout, k, stride, pad;
+};
+ConvGeom make_geom(const ckpt_conv_shape& s);
+
+// CUDA-core implicit-GEMM kernels (any k / stride / pad / channel count).
+int simt_conv_fwd(int dtype, const ConvGeom& g, const void* x, const void* w, void* z,
+                  const float* bias, int relu, void* stream);
+int simt_conv_dgrad(int dtype, const ConvGeom& g, const void* dz, const void* w, void* dx, void* stream);
+int64_t simt_wgrad_scratch_bytes(const ConvGeom& g);
+int simt_conv_wgrad(int dtype, const ConvGeom& g, const void* dz, const void* x, float* dw,
+                    void* scratch, int64_t scratch_bytes, void* stream);
+
+// Tensor-core (tcgen05) implicit-GEMM kernels; *_supported tells whether the shape has one.
+bool tc_conv_supported(int dtype, const ConvGeom& g);
+int64_t tc_conv_scratch_bytes(const ConvGeom& g);
+int tc_conv_fwd(const ConvGeom& g, const void* x, const void* w, void* z, void* scratch,
+                int64_t scratch_bytes, int* device_status, void* stream);
+int tc_conv_dgrad(const ConvGeom& g, const void* dz, const void* w, void* dx, void* scratch,
+                  int64_t scratch_bytes, int* device_status, void* stream);
+int tc_conv_wgrad(const ConvGeom& g, const void* dz, const void* x, float* dw, void* scratch,
+                  int64_t scratch_bytes, int* device_status, void* stream);
+
+int64_t bn_scratch_bytes(int64_t rows, int c);
+int bn_relu_forward(int dtype, int64_t rows, int c, const void* z, const float* gamma, const float* beta,
+                    int relu, void* y, float* stats, void* scratch, void* stream);
+int bn_relu_backward(int dtype, int64_t rows, int c, const void* dy, const void* z, const float* gamma,
+                     const float* stats, int relu, void* dz, float* dgamma, float* dbeta, void* scratch,
+                     void* stream);
+
+int maxpool_forward(int dtype, int n, int h, int w, int c, int k, int stride, int pad, const void* x,
+                    void* y, void* stream);
+int maxpool_backward(int dtype, int n, int h, int w, int c, int k, int stride, int pad, const void* x,
+                     const void* dy, void* dx, void* stream);
+int avgpool_forward(int dtype, int n, int h, int w, int c, const void* x, void* y, void* stream);
+int avgpool_backward(int dtype, int n, int h, int w, int c, const void* dy, void* dx, void* stream);
+
+// g <- g * (y > 0), elementwise over `elems`.
+int relu_mask_inplace(int dtype, int64_t elems, void* g, const void* y, void* stream);
+// out[c] (f32) = sum over rows of g[row][c], rows summed in index order.
+int column_sums(int dtype, int64_t rows, int c, const void* g, float* out, void* stream);
+int softmax_ce(int dtype, int batch, int classes, const void* logits, const int32_t* labels,
+               float* loss, void* dlogits, float* row_scratch, void* stream);
+// loss (device double) = sum of all elements; grad filled with ones.
+int sum_loss(int dtype, int64_t elems, const void* y, double* loss, void* grad, double* scratch,
+             void* stream);
+int64_t sum_loss_scratch_bytes();
+int device_copy(void* dst, const void* src, int64_t bytes, void* stream);
+
+}  // namespace ckpt

@@ -1,0 +1,747 @@
+// CUDA-core kernels: general implicit-GEMM convolution (forward, dgrad, wgrad; any filter size,
+// stride, padding and channel count; float32 or bfloat16 storage with float32 accumulation),
+// batch normalisation, pooling, losses and small element-wise helpers.
+//
+// Every reduction has a fixed summation order (no floating-point atomics), so repeated runs and
+// recomputation give bit-identical results.
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include <algorithm>
+#include <cstdio>
+
+#include "internal.h"
+
+namespace ckpt {
+
+int cuda_fail(int err, const char* what) {
+    set_error("CUDA error during %s: %s", what, cudaGetErrorString((cudaError_t)err));
+    return CKPT_E_CUDA;
+}
+
+#define CKPT_LAUNCH_CHECK(what)                                   \
+    do {                                                          \
+        ++g_launches;                                             \
+        cudaError_t e__ = cudaGetLastError();                     \
+        if (e__ != cudaSuccess) return cuda_fail(e__, what);      \
+    } while (0)
+
+ConvGeom make_geom(const ckpt_conv_shape& s) {
+    ConvGeom g;
+    g.n = s.n; g.h = s.h; g.w = s.w; g.cin = s.c_in; g.cout = s.c_out; g.k = s.k; g.stride = s.stride; g.pad = s.pad;
+    g.ho = (s.h + 2 * s.pad - s.k) / s.stride + 1;
+    g.wo = (s.w + 2 * s.pad - s.k) / s.stride + 1;
+    return g;
+}
+
+template <typename T> __device__ __forceinline__ float ld(const T* p);
+template <> __device__ __forceinline__ float ld<float>(const float* p) { return *p; }
+template <> __device__ __forceinline__ float ld<__nv_bfloat16>(const __nv_bfloat16* p) { return __bfloat162float(*p); }
+template <typename T> __device__ __forceinline__ T cvt(float v);
+template <> __device__ __forceinline__ float cvt<float>(float v) { return v; }
+template <> __device__ __forceinline__ __nv_bfloat16 cvt<__nv_bfloat16>(float v) { return __float2bfloat16_rn(v); }
+
+// ================================================================================================
+// Implicit GEMM  C[M][N] = sum_k A(m,k) * B(k,n), 64x64 tile, 16-deep k slices, 4x4 per thread.
+//   MODE 0 forward: M = pixels out, N = c_out, K = k*k*c_in
+//   MODE 1 dgrad  : M = pixels in,  N = c_in,  K = k*k*c_out
+//   MODE 2 wgrad  : M = c_out,      N = k*k*c_in, K = pixels out, split over gridDim.z
+// ================================================================================================
+constexpr int TM = 64, TN = 64, TK = 16;
+
+template <typename T, int MODE>
+__device__ __forceinline__ float load_a(const ConvGeom& g, const T* A, int m, int kk, int M, int K) {
+    if (m >= M || kk >= K) return 0.f;
+    if (MODE == 0) {
+        int ci = kk % g.cin, tap = kk / g.cin, r = tap / g.k, s = tap % g.k;
+        int ow = m % g.wo, t = m / g.wo, oh = t % g.ho, n = t / g.ho;
+        int ih = oh * g.stride - g.pad + r, iw = ow * g.stride - g.pad + s;
+        if (ih < 0 || ih >= g.h || iw < 0 || iw >= g.w) return 0.f;
+        return ld(A + (((size_t)n * g.h + ih) * g.w + iw) * g.cin + ci);
+    } else if (MODE == 1) {
+        int co = kk % g.cout, tap = kk / g.cout, r = tap / g.k, s = tap % g.k;
+        int iw = m % g.w, t = m / g.w, ih = t % g.h, n = t / g.h;
+        int th = ih + g.pad - r, tw = iw + g.pad - s;
+        if (th < 0 || tw < 0 || th % g.stride || tw % g.stride) return 0.f;
+        int oh = th / g.stride, ow = tw / g.stride;
+        if (oh >= g.ho || ow >= g.wo) return 0.f;
+        return ld(A + (((size_t)n * g.ho + oh) * g.wo + ow) * g.cout + co);
+    } else {
+        return ld(A + (size_t)kk * g.cout + m);              // dz[pixel][c_out]
+    }
+}
+
+template <typename T, int MODE>
+__device__ __forceinline__ float load_b(const ConvGeom& g, const T* B, int kk, int n, int K, int N) {
+    if (kk >= K || n >= N) return 0.f;
+    if (MODE == 0) {
+        return ld(B + (size_t)n * K + kk);                   // w[c_out][k][k][c_in]
+    } else if (MODE == 1) {
+        int co = kk % g.cout, tap = kk / g.cout;
+        return ld(B + ((size_t)co * g.k * g.k + tap) * g.cin + n);
+    } else {
+        int ci = n % g.cin, tap = n / g.cin, r = tap / g.k, s = tap % g.k;
+        int ow = kk % g.wo, t = kk / g.wo, oh = t % g.ho, img = t / g.ho;
+        int ih = oh * g.stride - g.pad + r, iw = ow * g.stride - g.pad + s;
+        if (ih < 0 || ih >= g.h || iw < 0 || iw >= g.w) return 0.f;
+        return ld(B + (((size_t)img * g.h + ih) * g.w + iw) * g.cin + ci);
+    }
+}
+
+template <typename T, int MODE>
+__global__ void __launch_bounds__(256) conv_gemm_kernel(ConvGeom g, const T* __restrict__ A, const T* __restrict__ B,
+                                                        void* __restrict__ out, const float* __restrict__ bias,
+                                                        int relu, int M, int N, int K, int k_per_slice) {
+    __shared__ float As[TK][TM + 1];
+    __shared__ float Bs[TK][TN + 1];
+    const int tid = threadIdx.x;
+    const int m0 = blockIdx.x * TM, n0 = blockIdx.y * TN;
+    const int k_begin = blockIdx.z * k_per_slice;
+    const int k_end = min(K, k_begin + k_per_slice);
+    const int tx = tid % 16, ty = tid / 16;
+    float acc[4][4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
+
+    for (int k0 = k_begin; k0 < k_end; k0 += TK) {
+        // operand tiles; the index that is contiguous in memory varies fastest across threads
+#pragma unroll
+        for (int p = 0; p < 4; ++p) {
+            if (MODE == 2) {
+                int mm = tid % TM, kk = tid / TM + 4 * p;
+                As[kk][mm] = (k0 + kk < k_end) ? load_a<T, MODE>(g, A, m0 + mm, k0 + kk, M, K) : 0.f;
+            } else {
+                int kk = tid % TK, mm = tid / TK + 16 * p;
+                As[kk][mm] = (k0 + kk < k_end) ? load_a<T, MODE>(g, A, m0 + mm, k0 + kk, M, K) : 0.f;
+            }
+            if (MODE == 0) {
+                int kk = tid % TK, nn = tid / TK + 16 * p;
+                Bs[kk][nn] = (k0 + kk < k_end) ? load_b<T, MODE>(g, B, k0 + kk, n0 + nn, K, N) : 0.f;
+            } else {
+                int nn = tid % TN, kk = tid / TN + 4 * p;
+                Bs[kk][nn] = (k0 + kk < k_end) ? load_b<T, MODE>(g, B, k0 + kk, n0 + nn, K, N) : 0.f;
+            }
+        }
+        __syncthreads();
+#pragma unroll
+        for (int kk = 0; kk < TK; ++kk) {
+            float a[4], b[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) a[i] = As[kk][ty * 4 + i];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) b[j] = Bs[kk][tx * 4 + j];
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+#pragma unroll
+                for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(a[i], b[j], acc[i][j]);
+        }
+        __syncthreads();
+    }
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        int m = m0 + ty * 4 + i;
+        if (m >= M) continue;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            int n = n0 + tx * 4 + j;
+            if (n >= N) continue;
+            float v = acc[i][j];
+            if (MODE == 2) {
+                ((float*)out)[((size_t)blockIdx.z * M + m) * N + n] = v;
+            } else {
+                if (bias) v += bias[n];
+                if (relu) v = fmaxf(v, 0.f);
+                ((T*)out)[(size_t)m * N + n] = cvt<T>(v);
+            }
+        }
+    }
+}
+
+// out[e] = sum over slices (in slice order) of partial[slice][e]
+__global__ void slice_sum_kernel(const float* __restrict__ partial, float* __restrict__ out, int64_t elems, int slices) {
+    int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (e >= elems) return;
+    float s = 0.f;
+    for (int z = 0; z < slices; ++z) s += partial[(size_t)z * elems + e];
+    out[e] = s;
+}
+
+template <typename T>
+static int launch_fwd(const ConvGeom& g, const void* x, const void* w, void* z, const float* bias, int relu, cudaStream_t st) {
+    int M = g.n * g.ho * g.wo, N = g.cout, K = g.k * g.k * g.cin;
+    dim3 grid((M + TM - 1) / TM, (N + TN - 1) / TN, 1);
+    conv_gemm_kernel<T, 0><<<grid, 256, 0, st>>>(g, (const T*)x, (const T*)w, z, bias, relu, M, N, K, K);
+    CKPT_LAUNCH_CHECK("conv forward (CUDA cores)");
+    return CKPT_OK;
+}
+template <typename T>
+static int launch_dgrad(const ConvGeom& g, const void* dz, const void* w, void* dx, cudaStream_t st) {
+    int M = g.n * g.h * g.w, N = g.cin, K = g.k * g.k * g.cout;
+    dim3 grid((M + TM - 1) / TM, (N + TN - 1) / TN, 1);
+    conv_gemm_kernel<T, 1><<<grid, 256, 0, st>>>(g, (const T*)dz, (const T*)w, dx, nullptr, 0, M, N, K, K);
+    CKPT_LAUNCH_CHECK("conv dgrad (CUDA cores)");
+    return CKPT_OK;
+}
+
+static void wgrad_split(const ConvGeom& g, int* slices, int* k_per_slice) {
+    int M = g.cout, N = g.k * g.k * g.cin;
+    int64_t K = (int64_t)g.n * g.ho * g.wo;
+    int64_t tiles = (int64_t)((M + TM - 1) / TM) * ((N + TN - 1) / TN);
+    int64_t want = std::max<int64_t>(1, (148 * 4 + tiles - 1) / tiles);      // about four tiles per SM
+    int64_t max_by_k = std::max<int64_t>(1, K / 256);                        // at least 256 deep per slice
+    int64_t s = std::min<int64_t>(std::min<int64_t>(want, max_by_k), 512);
+    int64_t per = ((K + s - 1) / s + TK - 1) / TK * TK;
+    *slices = (int)((K + per - 1) / per);
+    *k_per_slice = (int)per;
+}
+
+int64_t simt_wgrad_scratch_bytes(const ConvGeom& g) {
+    int slices, per;
+    wgrad_split(g, &slices, &per);
+    if (slices <= 1) return 0;
+    return (int64_t)slices * g.cout * g.k * g.k * g.cin * (int64_t)sizeof(float);
+}
+
+template <typename T>
+static int launch_wgrad(const ConvGeom& g, const void* dz, const void* x, float* dw, void* scratch, int64_t scratch_bytes, cudaStream_t st) {
+    int M = g.cout, N = g.k * g.k * g.cin, K = g.n * g.ho * g.wo;
+    int slices, per;
+    wgrad_split(g, &slices, &per);
+    if (slices > 1 && scratch_bytes < simt_wgrad_scratch_bytes(g)) { set_error("wgrad scratch too small"); return CKPT_E_WORKSPACE; }
+    dim3 grid((M + TM - 1) / TM, (N + TN - 1) / TN, slices);
+    float* target = slices > 1 ? (float*)scratch : dw;
+    conv_gemm_kernel<T, 2><<<grid, 256, 0, st>>>(g, (const T*)dz, (const T*)x, target, nullptr, 0, M, N, K, per);
+    CKPT_LAUNCH_CHECK("conv wgrad (CUDA cores)");
+    if (slices > 1) {
+        int64_t elems = (int64_t)M * N;
+        slice_sum_kernel<<<(unsigned)((elems + 255) / 256), 256, 0, st>>>((const float*)scratch, dw, elems, slices);
+        CKPT_LAUNCH_CHECK("wgrad slice sum");
+    }
+    return CKPT_OK;
+}
+
+int simt_conv_fwd(int dtype, const ConvGeom& g, const void* x, const void* w, void* z, const float* bias, int relu, void* stream) {
+    return dtype == CKPT_DTYPE_BF16 ? launch_fwd<__nv_bfloat16>(g, x, w, z, bias, relu, (cudaStream_t)stream)
+                                    : launch_fwd<float>(g, x, w, z, bias, relu, (cudaStream_t)stream);
+}
+int simt_conv_dgrad(int dtype, const ConvGeom& g, const void* dz, const void* w, void* dx, void* stream) {
+    return dtype == CKPT_DTYPE_BF16 ? launch_dgrad<__nv_bfloat16>(g, dz, w, dx, (cudaStream_t)stream)
+                                    : launch_dgrad<float>(g, dz, w, dx, (cudaStream_t)stream);
+}
+int simt_conv_wgrad(int dtype, const ConvGeom& g, const void* dz, const void* x, float* dw, void* scratch, int64_t scratch_bytes, void* stream) {
+    return dtype == CKPT_DTYPE_BF16 ? launch_wgrad<__nv_bfloat16>(g, dz, x, dw, scratch, scratch_bytes, (cudaStream_t)stream)
+                                    : launch_wgrad<float>(g, dz, x, dw, scratch, scratch_bytes, (cudaStream_t)stream);
+}
+
+// ================================================================================================
+// Batch normalisation (training mode) + ReLU over a [rows][c] matrix, c contiguous.
+// Each thread owns VEC consecutive channels (one 16-byte load when the channel count allows it) and
+// walks down the rows of its block's slab; partial sums are combined in a fixed order.
+// ================================================================================================
+constexpr int BN_THREADS = 256;
+constexpr int BN_MAX_BLOCKS = 148 * 8;
+constexpr float BN_EPS = 1e-5f;
+
+template <typename T, int VEC>
+__device__ __forceinline__ void load_vec(const T* p, float (&v)[VEC]) {
+    if constexpr (VEC == 1) {
+        v[0] = ld(p);
+    } else if constexpr (sizeof(T) == 4) {
+        float4 t = *reinterpret_cast<const float4*>(p);
+        v[0] = t.x; v[1] = t.y; v[2] = t.z; v[3] = t.w;
+    } else {
+        uint4 t = *reinterpret_cast<const uint4*>(p);
+        const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&t);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) { float2 f = __bfloat1622float2(h[i]); v[2 * i] = f.x; v[2 * i + 1] = f.y; }
+    }
+}
+template <typename T, int VEC>
+__device__ __forceinline__ void store_vec(T* p, const float (&v)[VEC]) {
+    if constexpr (VEC == 1) {
+        *p = cvt<T>(v[0]);
+    } else if constexpr (sizeof(T) == 4) {
+        *reinterpret_cast<float4*>(p) = make_float4(v[0], v[1], v[2], v[3]);
+    } else {
+        uint4 t;
+        __nv_bfloat162* h = reinterpret_cast<__nv_bfloat162*>(&t);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) h[i] = __floats2bfloat162_rn(v[2 * i], v[2 * i + 1]);
+        *reinterpret_cast<uint4*>(p) = t;
+    }
+}
+
+struct BnLayout {
+    int lanes;          // threads across the channel dimension (c / VEC)
+    int rows_per_iter;  // rows covered by one sweep of a block
+    int blocks;         // row slabs
+    int64_t rows_per_block;
+};
+static BnLayout bn_layout(int64_t rows, int c, int vec) {
+    BnLayout L;
+    L.lanes = c / vec;
+    int lanes_in_block = std::min(L.lanes, BN_THREADS);
+    L.rows_per_iter = std::max(1, BN_THREADS / lanes_in_block);
+    int64_t want = (rows + (int64_t)L.rows_per_iter * 8 - 1) / ((int64_t)L.rows_per_iter * 8);   // >= 8 sweeps each
+    L.blocks = (int)std::max<int64_t>(1, std::min<int64_t>(BN_MAX_BLOCKS, want));
+    L.rows_per_block = (rows + L.blocks - 1) / L.blocks;
+    L.blocks = (int)((rows + L.rows_per_block - 1) / L.rows_per_block);
+    return L;
+}
+static int bn_vec(int dtype, int c) {
+    if (dtype == CKPT_DTYPE_BF16) return (c % 8 == 0) ? 8 : 1;
+    return (c % 4 == 0) ? 4 : 1;
+}
+int64_t bn_scratch_bytes(int64_t rows, int c) {
+    (void)rows;
+    return (int64_t)BN_MAX_BLOCKS * c * 2 * (int64_t)sizeof(float) + 4 * (int64_t)c * sizeof(float);
+}
+
+// Two running sums per channel over a slab of rows.  WHAT 0: (z, z^2).  WHAT 1: (g, g*xhat) with
+// g = dy masked by the ReLU of the forward output.
+template <typename T, int VEC, int WHAT>
+__global__ void __launch_bounds__(BN_THREADS) bn_partial_kernel(const T* __restrict__ z, const T* __restrict__ dy,
+                                                                const float* __restrict__ stats, int relu, int64_t rows,
+                                                                int c, int lanes, int rows_per_iter, int64_t rows_per_block,
+                                                                float* __restrict__ partial) {
+    extern __shared__ float red[];          // [BN_THREADS][2*VEC]
+    const int lanes_here = min(lanes, BN_THREADS);
+    const int64_t row_begin = (int64_t)blockIdx.x * rows_per_block;
+    const int64_t row_end = min(rows, row_begin + rows_per_block);
+    for (int lane0 = 0; lane0 < lanes; lane0 += lanes_here) {
+        const int lane = lane0 + threadIdx.x % lanes_here;
+        const int r = threadIdx.x / lanes_here;
+        float s0[VEC], s1[VEC];
+#pragma unroll
+        for (int i = 0; i < VEC; ++i) { s0[i] = 0.f; s1[i] = 0.f; }
+        const bool active = r < rows_per_iter && lane < lanes;
+        if (active) {
+            const int ch = lane * VEC;
+            float mean[VEC], inv[VEC], sc[VEC], sh[VEC];
+            if (WHAT == 1) {
+#pragma unroll
+                for (int i = 0; i < VEC; ++i) { mean[i] = stats[ch + i]; inv[i] = stats[c + ch + i]; sc[i] = stats[2 * c + ch + i]; sh[i] = stats[3 * c + ch + i]; }
+            }
+            for (int64_t row = row_begin + r; row < row_end; row += rows_per_iter) {
+                float v[VEC];
+                load_vec<T, VEC>(z + row * c + ch, v);
+                if (WHAT == 0) {
+#pragma unroll
+                    for (int i = 0; i < VEC; ++i) { s0[i] += v[i]; s1[i] = fmaf(v[i], v[i], s1[i]); }
+                } else {
+                    float g[VEC];
+                    load_vec<T, VEC>(dy + row * c + ch, g);
+#pragma unroll
+                    for (int i = 0; i < VEC; ++i) {
+                        float yv = fmaf(v[i], sc[i], sh[i]);
+                        bool pass = !relu || (float)cvt<T>(fmaxf(yv, 0.f)) > 0.f;
+                        float gi = pass ? g[i] : 0.f;
+                        float xh = (v[i] - mean[i]) * inv[i];
+                        s0[i] += gi;
+                        s1[i] = fmaf(gi, xh, s1[i]);
+                    }
+                }
+            }
+        }
+        float* mine = red + ((size_t)(threadIdx.x / lanes_here) * lanes_here + threadIdx.x % lanes_here) * 2 * VEC;
+#pragma unroll
+        for (int i = 0; i < VEC; ++i) { mine[i] = s0[i]; mine[VEC + i] = s1[i]; }
+        __syncthreads();
+        if (r == 0 && lane < lanes) {
+            const int ch = lane * VEC;
+#pragma unroll
+            for (int i = 0; i < VEC; ++i) {
+                float a = 0.f, b = 0.f;
+                for (int rr = 0; rr < rows_per_iter; ++rr) {
+                    const float* o = red + ((size_t)rr * lanes_here + threadIdx.x % lanes_here) * 2 * VEC;
+                    a += o[i];
+                    b += o[VEC + i];
+                }
+                partial[((size_t)blockIdx.x * 2 + 0) * c + ch + i] = a;
+                partial[((size_t)blockIdx.x * 2 + 1) * c + ch + i] = b;
+            }
+        }
+        __syncthreads();
+    }
+}
+
+// mean, 1/sqrt(var+eps), scale = gamma*inv, shift = beta - mean*scale
+__global__ void bn_finalize_fwd_kernel(const float* __restrict__ partial, int blocks, int c, double inv_rows,
+                                       const float* __restrict__ gamma, const float* __restrict__ beta, float* __restrict__ stats) {
+    int ch = blockIdx.x * blockDim.x + threadIdx.x;
+    if (ch >= c) return;
+    double s = 0.0, q = 0.0;
+    for (int b = 0; b < blocks; ++b) { s += partial[((size_t)b * 2) * c + ch]; q += partial[((size_t)b * 2 + 1) * c + ch]; }
+    double mean = s * inv_rows;
+    double var = q * inv_rows - mean * mean;
+    if (var < 0.0) var = 0.0;
+    float inv = (float)(1.0 / sqrt(var + (double)BN_EPS));
+    float scale = gamma[ch] * inv;
+    stats[ch] = (float)mean;
+    stats[c + ch] = inv;
+    stats[2 * c + ch] = scale;
+    stats[3 * c + ch] = beta[ch] - (float)mean * scale;
+}
+
+// dbeta, dgamma and the two per-channel coefficients of the input gradient:
+//   dz = scale*g - k1 - xhat*k2,  k1 = scale*dbeta/rows, k2 = scale*dgamma/rows
+__global__ void bn_finalize_bwd_kernel(const float* __restrict__ partial, int blocks, int c, double inv_rows,
+                                       const float* __restrict__ stats, float* __restrict__ dgamma, float* __restrict__ dbeta,
+                                       float* __restrict__ coef) {
+    int ch = blockIdx.x * blockDim.x + threadIdx.x;
+    if (ch >= c) return;
+    double s = 0.0, q = 0.0;
+    for (int b = 0; b < blocks; ++b) { s += partial[((size_t)b * 2) * c + ch]; q += partial[((size_t)b * 2 + 1) * c + ch]; }
+    dbeta[ch] = (float)s;
+    dgamma[ch] = (float)q;
+    double scale = stats[2 * c + ch];
+    coef[ch] = (float)(scale * s * inv_rows);
+    coef[c + ch] = (float)(scale * q * inv_rows);
+}
+
+template <typename T, int VEC>
+__global__ void __launch_bounds__(256) bn_apply_kernel(const T* __restrict__ z, const float* __restrict__ stats, int relu,
+                                                       int64_t vecs, int lanes, int c, T* __restrict__ y) {
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < vecs; i += (int64_t)gridDim.x * blockDim.x) {
+        const int ch = (int)(i % lanes) * VEC;
+        float v[VEC], o[VEC];
+        load_vec<T, VEC>(z + i * VEC, v);
+#pragma unroll
+        for (int k = 0; k < VEC; ++k) {
+            float t = fmaf(v[k], stats[2 * c + ch + k], stats[3 * c + ch + k]);
+            o[k] = relu ? fmaxf(t, 0.f) : t;
+        }
+        store_vec<T, VEC>(y + i * VEC, o);
+    }
+}
+
+template <typename T, int VEC>
+__global__ void __launch_bounds__(256) bn_bwd_apply_kernel(const T* __restrict__ dy, const T* __restrict__ z,
+                                                           const float* __restrict__ stats, const float* __restrict__ coef,
+                                                           int relu, int64_t vecs, int lanes, int c, T* __restrict__ dz) {
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < vecs; i += (int64_t)gridDim.x * blockDim.x) {
+        const int ch = (int)(i % lanes) * VEC;
+        float v[VEC], g[VEC], o[VEC];
+        load_vec<T, VEC>(z + i * VEC, v);
+        load_vec<T, VEC>(dy + i * VEC, g);
+#pragma unroll
+        for (int k = 0; k < VEC; ++k) {
+            float sc = stats[2 * c + ch + k];
+            float yv = fmaf(v[k], sc, stats[3 * c + ch + k]);
+            bool pass = !relu || (float)cvt<T>(fmaxf(yv, 0.f)) > 0.f;
+            float gi = pass ? g[k] : 0.f;
+            float xh = (v[k] - stats[ch + k]) * stats[c + ch + k];
+            o[k] = sc * gi - coef[ch + k] - xh * coef[c + ch + k];
+        }
+        store_vec<T, VEC>(dz + i * VEC, o);
+    }
+}
+
+static unsigned elementwise_grid(int64_t items) {
+    int64_t b = (items + 255) / 256;
+    return (unsigned)std::max<int64_t>(1, std::min<int64_t>(b, 148 * 16));
+}
+
+template <typename T, int VEC>
+static int bn_forward_t(int64_t rows, int c, const void* z, const float* gamma, const float* beta, int relu, void* y,
+                        float* stats, void* scratch, cudaStream_t st) {
+    BnLayout L = bn_layout(rows, c, VEC);
+    float* partial = (float*)scratch;
+    size_t smem = (size_t)BN_THREADS * 2 * VEC * sizeof(float);
+    bn_partial_kernel<T, VEC, 0><<<L.blocks, BN_THREADS, smem, st>>>((const T*)z, nullptr, nullptr, 0, rows, c, L.lanes,
+                                                                      L.rows_per_iter, L.rows_per_block, partial);
+    CKPT_LAUNCH_CHECK("batch-norm statistics");
+    bn_finalize_fwd_kernel<<<(c + 127) / 128, 128, 0, st>>>(partial, L.blocks, c, 1.0 / (double)rows, gamma, beta, stats);
+    CKPT_LAUNCH_CHECK("batch-norm finalize");
+    int64_t vecs = rows * c / VEC;
+    bn_apply_kernel<T, VEC><<<elementwise_grid(vecs), 256, 0, st>>>((const T*)z, stats, relu, vecs, L.lanes, c, (T*)y);
+    CKPT_LAUNCH_CHECK("batch-norm apply");
+    return CKPT_OK;
+}
+
+template <typename T, int VEC>
+static int bn_backward_t(int64_t rows, int c, const void* dy, const void* z, const float* stats, int relu, void* dz,
+                         float* dgamma, float* dbeta, void* scratch, cudaStream_t st) {
+    BnLayout L = bn_layout(rows, c, VEC);
+    float* partial = (float*)scratch;
+    float* coef = partial + (size_t)BN_MAX_BLOCKS * c * 2;
+    size_t smem = (size_t)BN_THREADS * 2 * VEC * sizeof(float);
+    bn_partial_kernel<T, VEC, 1><<<L.blocks, BN_THREADS, smem, st>>>((const T*)z, (const T*)dy, stats, relu, rows, c, L.lanes,
+                                                                      L.rows_per_iter, L.rows_per_block, partial);
+    CKPT_LAUNCH_CHECK("batch-norm backward sums");
+    bn_finalize_bwd_kernel<<<(c + 127) / 128, 128, 0, st>>>(partial, L.blocks, c, 1.0 / (double)rows, stats, dgamma, dbeta, coef);
+    CKPT_LAUNCH_CHECK("batch-norm backward finalize");
+    int64_t vecs = rows * c / VEC;
+    bn_bwd_apply_kernel<T, VEC><<<elementwise_grid(vecs), 256, 0, st>>>((const T*)dy, (const T*)z, stats, coef, relu, vecs,
+                                                                         L.lanes, c, (T*)dz);
+    CKPT_LAUNCH_CHECK("batch-norm backward apply");
+    return CKPT_OK;
+}
+
+int bn_relu_forward(int dtype, int64_t rows, int c, const void* z, const float* gamma, const float* beta, int relu, void* y,
+                    float* stats, void* scratch, void* stream) {
+    cudaStream_t st = (cudaStream_t)stream;
+    int vec = bn_vec(dtype, c);
+    if (dtype == CKPT_DTYPE_BF16)
+        return vec == 8 ? bn_forward_t<__nv_bfloat16, 8>(rows, c, z, gamma, beta, relu, y, stats, scratch, st)
+                        : bn_forward_t<__nv_bfloat16, 1>(rows, c, z, gamma, beta, relu, y, stats, scratch, st);
+    return vec == 4 ? bn_forward_t<float, 4>(rows, c, z, gamma, beta, relu, y, stats, scratch, st)
+                    : bn_forward_t<float, 1>(rows, c, z, gamma, beta, relu, y, stats, scratch, st);
+}
+
+int bn_relu_backward(int dtype, int64_t rows, int c, const void* dy, const void* z, const float* gamma, const float* stats,
+                     int relu, void* dz, float* dgamma, float* dbeta, void* scratch, void* stream) {
+    (void)gamma;   // scale = gamma * inv_std is part of the saved statistics
+    cudaStream_t st = (cudaStream_t)stream;
+    int vec = bn_vec(dtype, c);
+    if (dtype == CKPT_DTYPE_BF16)
+        return vec == 8 ? bn_backward_t<__nv_bfloat16, 8>(rows, c, dy, z, stats, relu, dz, dgamma, dbeta, scratch, st)
+                        : bn_backward_t<__nv_bfloat16, 1>(rows, c, dy, z, stats, relu, dz, dgamma, dbeta, scratch, st);
+    return vec == 4 ? bn_backward_t<float, 4>(rows, c, dy, z, stats, relu, dz, dgamma, dbeta, scratch, st)
+                    : bn_backward_t<float, 1>(rows, c, dy, z, stats, relu, dz, dgamma, dbeta, scratch, st);
+}
+
+// ================================================================================================
+// Pooling
+// ================================================================================================
+template <typename T>
+__global__ void maxpool_fwd_kernel(const T* __restrict__ x, T* __restrict__ y, int n, int h, int w, int c, int ho, int wo,
+                                   int k, int stride, int pad) {
+    int64_t total = (int64_t)n * ho * wo * c;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+        int ch = (int)(i % c);
+        int64_t t = i / c;
+        int ow = (int)(t % wo); t /= wo;
+        int oh = (int)(t % ho);
+        int img = (int)(t / ho);
+        float best = -INFINITY;
+        for (int r = 0; r < k; ++r) {
+            int ih = oh * stride - pad + r;
+            if (ih < 0 || ih >= h) continue;
+            for (int s = 0; s < k; ++s) {
+                int iw = ow * stride - pad + s;
+                if (iw < 0 || iw >= w) continue;
+                best = fmaxf(best, ld(x + (((size_t)img * h + ih) * w + iw) * c + ch));
+            }
+        }
+        y[i] = cvt<T>(best);
+    }
+}
+
+// Gather form: every input element looks at the windows that contain it and takes the gradient of
+// those in which it is the first maximum (row-major window order).
+template <typename T>
+__global__ void maxpool_bwd_kernel(const T* __restrict__ x, const T* __restrict__ dy, T* __restrict__ dx, int n, int h, int w,
+                                   int c, int ho, int wo, int k, int stride, int pad) {
+    int64_t total = (int64_t)n * h * w * c;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+        int ch = (int)(i % c);
+        int64_t t = i / c;
+        int iw = (int)(t % w); t /= w;
+        int ih = (int)(t % h);
+        int img = (int)(t / h);
+        const float mine = ld(x + i);
+        float acc = 0.f;
+        int oh_lo = max(0, (ih + pad - k + stride) / stride), oh_hi = min(ho - 1, (ih + pad) / stride);
+        int ow_lo = max(0, (iw + pad - k + stride) / stride), ow_hi = min(wo - 1, (iw + pad) / stride);
+        for (int oh = oh_lo; oh <= oh_hi; ++oh) {
+            for (int ow = ow_lo; ow <= ow_hi; ++ow) {
+                // am I the first maximum of window (oh, ow)?
+                bool first = true;
+                for (int r = 0; r < k && first; ++r) {
+                    int yy = oh * stride - pad + r;
+                    if (yy < 0 || yy >= h) continue;
+                    for (int s = 0; s < k; ++s) {
+                        int xx = ow * stride - pad + s;
+                        if (xx < 0 || xx >= w) continue;
+                        float v = ld(x + (((size_t)img * h + yy) * w + xx) * c + ch);
+                        bool before = (yy < ih) || (yy == ih && xx < iw);
+                        if (v > mine || (before && v == mine)) { first = false; break; }
+                    }
+                }
+                if (first) acc += ld(dy + (((size_t)img * ho + oh) * wo + ow) * c + ch);
+            }
+        }
+        dx[i] = cvt<T>(acc);
+    }
+}
+
+int maxpool_forward(int dtype, int n, int h, int w, int c, int k, int stride, int pad, const void* x, void* y, void* stream) {
+    int ho = (h + 2 * pad - k) / stride + 1, wo = (w + 2 * pad - k) / stride + 1;
+    unsigned grid = elementwise_grid((int64_t)n * ho * wo * c);
+    if (dtype == CKPT_DTYPE_BF16)
+        maxpool_fwd_kernel<__nv_bfloat16><<<grid, 256, 0, (cudaStream_t)stream>>>((const __nv_bfloat16*)x, (__nv_bfloat16*)y, n, h, w, c, ho, wo, k, stride, pad);
+    else
+        maxpool_fwd_kernel<float><<<grid, 256, 0, (cudaStream_t)stream>>>((const float*)x, (float*)y, n, h, w, c, ho, wo, k, stride, pad);
+    CKPT_LAUNCH_CHECK("max-pool forward");
+    return CKPT_OK;
+}
+
+int maxpool_backward(int dtype, int n, int h, int w, int c, int k, int stride, int pad, const void* x, const void* dy, void* dx, void* stream) {
+    int ho = (h + 2 * pad - k) / stride + 1, wo = (w + 2 * pad - k) / stride + 1;
+    unsigned grid = elementwise_grid((int64_t)n * h * w * c);
+    if (dtype == CKPT_DTYPE_BF16)
+        maxpool_bwd_kernel<__nv_bfloat16><<<grid, 256, 0, (cudaStream_t)stream>>>((const __nv_bfloat16*)x, (const __nv_bfloat16*)dy, (__nv_bfloat16*)dx, n, h, w, c, ho, wo, k, stride, pad);
+    else
+        maxpool_bwd_kernel<float><<<grid, 256, 0, (cudaStream_t)stream>>>((const float*)x, (const float*)dy, (float*)dx, n, h, w, c, ho, wo, k, stride, pad);
+    CKPT_LAUNCH_CHECK("max-pool backward");
+    return CKPT_OK;
+}
+
+template <typename T>
+__global__ void avgpool_fwd_kernel(const T* __restrict__ x, T* __restrict__ y, int n, int hw, int c) {
+    int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n * c) return;
+    int ch = i % c, img = i / c;
+    float s = 0.f;
+    for (int p = 0; p < hw; ++p) s += ld(x + ((size_t)img * hw + p) * c + ch);
+    y[i] = cvt<T>(s / (float)hw);
+}
+template <typename T>
+__global__ void avgpool_bwd_kernel(const T* __restrict__ dy, T* __restrict__ dx, int64_t total, int hw, int c) {
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+        int ch = (int)(i % c);
+        int64_t img = i / ((int64_t)hw * c);
+        dx[i] = cvt<T>(ld(dy + img * c + ch) / (float)hw);
+    }
+}
+int avgpool_forward(int dtype, int n, int h, int w, int c, const void* x, void* y, void* stream) {
+    unsigned grid = (unsigned)((n * c + 255) / 256);
+    if (dtype == CKPT_DTYPE_BF16) avgpool_fwd_kernel<__nv_bfloat16><<<grid, 256, 0, (cudaStream_t)stream>>>((const __nv_bfloat16*)x, (__nv_bfloat16*)y, n, h * w, c);
+    else avgpool_fwd_kernel<float><<<grid, 256, 0, (cudaStream_t)stream>>>((const float*)x, (float*)y, n, h * w, c);
+    CKPT_LAUNCH_CHECK("average-pool forward");
+    return CKPT_OK;
+}
+int avgpool_backward(int dtype, int n, int h, int w, int c, const void* dy, void* dx, void* stream) {
+    int64_t total = (int64_t)n * h * w * c;
+    if (dtype == CKPT_DTYPE_BF16) avgpool_bwd_kernel<__nv_bfloat16><<<elementwise_grid(total), 256, 0, (cudaStream_t)stream>>>((const __nv_bfloat16*)dy, (__nv_bfloat16*)dx, total, h * w, c);
+    else avgpool_bwd_kernel<float><<<elementwise_grid(total), 256, 0, (cudaStream_t)stream>>>((const float*)dy, (float*)dx, total, h * w, c);
+    CKPT_LAUNCH_CHECK("average-pool backward");
+    return CKPT_OK;
+}
+
+// ================================================================================================
+// Small helpers for the fully connected units and the losses
+// ================================================================================================
+template <typename T>
+__global__ void relu_mask_kernel(T* __restrict__ g, const T* __restrict__ y, int64_t elems) {
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < elems; i += (int64_t)gridDim.x * blockDim.x)
+        if (!(ld(y + i) > 0.f)) g[i] = cvt<T>(0.f);
+}
+int relu_mask_inplace(int dtype, int64_t elems, void* g, const void* y, void* stream) {
+    if (dtype == CKPT_DTYPE_BF16) relu_mask_kernel<__nv_bfloat16><<<elementwise_grid(elems), 256, 0, (cudaStream_t)stream>>>((__nv_bfloat16*)g, (const __nv_bfloat16*)y, elems);
+    else relu_mask_kernel<float><<<elementwise_grid(elems), 256, 0, (cudaStream_t)stream>>>((float*)g, (const float*)y, elems);
+    CKPT_LAUNCH_CHECK("ReLU mask");
+    return CKPT_OK;
+}
+
+template <typename T>
+__global__ void column_sum_kernel(const T* __restrict__ g, float* __restrict__ out, int64_t rows, int c) {
+    int ch = blockIdx.x * blockDim.x + threadIdx.x;
+    if (ch >= c) return;
+    float s = 0.f;
+    for (int64_t r = 0; r < rows; ++r) s += ld(g + r * c + ch);
+    out[ch] = s;
+}
+int column_sums(int dtype, int64_t rows, int c, const void* g, float* out, void* stream) {
+    if (dtype == CKPT_DTYPE_BF16) column_sum_kernel<__nv_bfloat16><<<(c + 127) / 128, 128, 0, (cudaStream_t)stream>>>((const __nv_bfloat16*)g, out, rows, c);
+    else column_sum_kernel<float><<<(c + 127) / 128, 128, 0, (cudaStream_t)stream>>>((const float*)g, out, rows, c);
+    CKPT_LAUNCH_CHECK("column sums");
+    return CKPT_OK;
+}
+
+// One block per sample: max, sum of exponentials, loss term, gradient (softmax - onehot)/batch.
+template <typename T>
+__global__ void __launch_bounds__(256) softmax_ce_kernel(const T* __restrict__ logits, const int32_t* __restrict__ labels,
+                                                         int classes, float inv_batch, float* __restrict__ row_loss,
+                                                         T* __restrict__ dlogits) {
+    __shared__ float red[256];
+    const T* row = logits + (size_t)blockIdx.x * classes;
+    float m = -INFINITY;
+    for (int i = threadIdx.x; i < classes; i += 256) m = fmaxf(m, ld(row + i));
+    red[threadIdx.x] = m;
+    __syncthreads();
+    for (int s = 128; s > 0; s >>= 1) { if (threadIdx.x < s) red[threadIdx.x] = fmaxf(red[threadIdx.x], red[threadIdx.x + s]); __syncthreads(); }
+    m = red[0];
+    __syncthreads();
+    float sum = 0.f;
+    for (int i = threadIdx.x; i < classes; i += 256) sum += expf(ld(row + i) - m);
+    red[threadIdx.x] = sum;
+    __syncthreads();
+    for (int s = 128; s > 0; s >>= 1) { if (threadIdx.x < s) red[threadIdx.x] += red[threadIdx.x + s]; __syncthreads(); }
+    sum = red[0];
+    const int label = labels[blockIdx.x];
+    const float inv_sum = 1.f / sum;
+    for (int i = threadIdx.x; i < classes; i += 256) {
+        float p = expf(ld(row + i) - m) * inv_sum;
+        dlogits[(size_t)blockIdx.x * classes + i] = cvt<T>((p - (i == label ? 1.f : 0.f)) * inv_batch);
+    }
+    if (threadIdx.x == 0) row_loss[blockIdx.x] = logf(sum) + m - ld(row + label);
+}
+__global__ void mean_rows_kernel(const float* __restrict__ row_loss, int batch, float* __restrict__ loss) {
+    if (threadIdx.x == 0 && blockIdx.x == 0) {
+        double s = 0.0;
+        for (int i = 0; i < batch; ++i) s += row_loss[i];
+        *loss = (float)(s / batch);
+    }
+}
+int softmax_ce(int dtype, int batch, int classes, const void* logits, const int32_t* labels, float* loss, void* dlogits,
+               float* row_scratch, void* stream) {
+    cudaStream_t st = (cudaStream_t)stream;
+    if (dtype == CKPT_DTYPE_BF16)
+        softmax_ce_kernel<__nv_bfloat16><<<batch, 256, 0, st>>>((const __nv_bfloat16*)logits, labels, classes, 1.f / batch, row_scratch, (__nv_bfloat16*)dlogits);
+    else
+        softmax_ce_kernel<float><<<batch, 256, 0, st>>>((const float*)logits, labels, classes, 1.f / batch, row_scratch, (float*)dlogits);
+    CKPT_LAUNCH_CHECK("softmax cross-entropy");
+    mean_rows_kernel<<<1, 32, 0, st>>>(row_scratch, batch, loss);
+    CKPT_LAUNCH_CHECK("loss mean");
+    return CKPT_OK;
+}
+
+constexpr int SUM_BLOCKS = 256;
+template <typename T>
+__global__ void __launch_bounds__(256) sum_partial_kernel(const T* __restrict__ y, int64_t elems, double* __restrict__ partial,
+                                                          T* __restrict__ grad) {
+    __shared__ double red[256];
+    double s = 0.0;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < elems; i += (int64_t)gridDim.x * blockDim.x) {
+        s += (double)ld(y + i);
+        grad[i] = cvt<T>(1.f);
+    }
+    red[threadIdx.x] = s;
+    __syncthreads();
+    for (int k = 128; k > 0; k >>= 1) { if (threadIdx.x < k) red[threadIdx.x] += red[threadIdx.x + k]; __syncthreads(); }
+    if (threadIdx.x == 0) partial[blockIdx.x] = red[0];
+}
+__global__ void sum_final_kernel(const double* __restrict__ partial, int blocks, double* __restrict__ loss) {
+    if (threadIdx.x == 0 && blockIdx.x == 0) {
+        double s = 0.0;
+        for (int i = 0; i < blocks; ++i) s += partial[i];
+        *loss = s;
+    }
+}
+int64_t sum_loss_scratch_bytes() { return SUM_BLOCKS * (int64_t)sizeof(double); }
+int sum_loss(int dtype, int64_t elems, const void* y, double* loss, void* grad, double* scratch, void* stream) {
+    cudaStream_t st = (cudaStream_t)stream;
+    if (dtype == CKPT_DTYPE_BF16) sum_partial_kernel<__nv_bfloat16><<<SUM_BLOCKS, 256, 0, st>>>((const __nv_bfloat16*)y, elems, scratch, (__nv_bfloat16*)grad);
+    else sum_partial_kernel<float><<<SUM_BLOCKS, 256, 0, st>>>((const float*)y, elems, scratch, (float*)grad);
+    CKPT_LAUNCH_CHECK("sum loss");
+    sum_final_kernel<<<1, 32, 0, st>>>(scratch, SUM_BLOCKS, loss);
+    CKPT_LAUNCH_CHECK("sum loss final");
+    return CKPT_OK;
+}
+
+__global__ void copy_kernel(uint4* __restrict__ dst, const uint4* __restrict__ src, int64_t vecs) {
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < vecs; i += (int64_t)gridDim.x * blockDim.x) dst[i] = src[i];
+}
+int device_copy(void* dst, const void* src, int64_t bytes, void* stream) {
+    // sizes and offsets inside the arena and the workspace are multiples of 256 bytes
+    int64_t vecs = bytes / 16;
+    copy_kernel<<<elementwise_grid(vecs), 256, 0, (cudaStream_t)stream>>>((uint4*)dst, (const uint4*)src, vecs);
+    CKPT_LAUNCH_CHECK("gradient carry copy");
+    return CKPT_OK;
+}
+
+}  // namespace ckpt

@@ -1,0 +1,285 @@
+// Host planners: checkpoint selection under the paper's two memory models, in exact int64.
+//
+//   plan_static_n3  - Algorithm 3 (Section 3.2), objective Eq. (cost)
+//   plan_dynamic_n2 - Algorithm 5 (Section 4.1), objective Eq. (memory)
+//   plan_dynamic_n  - Algorithm 6 (Section 4.2), same objective, monotone queue + pointer walk
+//   eval_model      - Eq. (cost) / Eq. (memory) / Algorithm 1 total for a given set
+#include <algorithm>
+#include <cstdarg>
+#include <cstdio>
+#include <limits>
+
+#include "internal.h"
+
+namespace ckpt {
+
+static thread_local char g_error[512] = "";
+int64_t g_launches = 0;
+
+void set_error(const char* fmt, ...) {
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(g_error, sizeof(g_error), fmt, ap);
+    va_end(ap);
+}
+
+int validate_sizes(int64_t n, const int64_t* d) {
+    if (!d) { set_error("d is null"); return CKPT_E_NULL; }
+    if (n < 1) { set_error("n = %lld < 1", (long long)n); return CKPT_E_BAD_N; }
+    const int64_t limit = std::numeric_limits<int64_t>::max() / 2;
+    int64_t sum = 0;
+    for (int64_t i = 0; i <= n; ++i) {
+        if (d[i] < 1) { set_error("d[%lld] = %lld < 1", (long long)i, (long long)d[i]); return CKPT_E_BAD_SIZE; }
+        if (d[i] > limit - sum) { set_error("2*sum(d) overflows int64"); return CKPT_E_OVERFLOW; }
+        sum += d[i];
+    }
+    return CKPT_OK;
+}
+
+static int validate_plan(int64_t n, const uint8_t* is_ckpt) {
+    if (!is_ckpt) { set_error("is_ckpt is null"); return CKPT_E_NULL; }
+    if (!is_ckpt[0] || !is_ckpt[n]) { set_error("d_0 and d_n must be checkpoints"); return CKPT_E_BAD_PLAN; }
+    return CKPT_OK;
+}
+
+// ------------------------------------------------------------------------------------------------
+// Objectives
+// ------------------------------------------------------------------------------------------------
+int eval_model(int model, int64_t n, const int64_t* d, const uint8_t* is_ckpt, int64_t* peak) {
+    if (!peak) { set_error("peak_bytes is null"); return CKPT_E_NULL; }
+    int rc = validate_sizes(n, d);
+    if (rc) return rc;
+    if (model == CKPT_MODEL_STORE_ALL) {
+        int64_t s = 0;
+        for (int64_t i = 0; i <= n; ++i) s += d[i];
+        *peak = s;
+        return CKPT_OK;
+    }
+    rc = validate_plan(n, is_ckpt);
+    if (rc) return rc;
+    if (model == CKPT_MODEL_STATIC) {
+        // Eq. (cost): checkpoint memory + largest segment memory.
+        int64_t ckpt_mem = 0, seg = 0, seg_max = 0;
+        for (int64_t i = 0; i <= n; ++i) {
+            if (is_ckpt[i]) { ckpt_mem += d[i]; seg_max = std::max(seg_max, seg); seg = 0; }
+            else seg += d[i];
+        }
+        *peak = ckpt_mem + seg_max;
+        return CKPT_OK;
+    }
+    if (model == CKPT_MODEL_DYNAMIC) {
+        // Eq. (memory): at every checkpoint i (previous checkpoint h):
+        //   sum of checkpoints <= i  +  sum d_{h+1..i-1}  +  max d_{h..i-1}.
+        int64_t ckpt_mem = d[0], seg = 0, run_max = d[0], worst = 0;
+        for (int64_t i = 1; i <= n; ++i) {
+            if (is_ckpt[i]) {
+                ckpt_mem += d[i];
+                worst = std::max(worst, ckpt_mem + seg + run_max);
+                seg = 0;
+                run_max = d[i];
+            } else {
+                seg += d[i];
+                run_max = std::max(run_max, d[i]);
+            }
+        }
+        *peak = worst;
+        return CKPT_OK;
+    }
+    set_error("unknown memory model %d", model);
+    return CKPT_E_BAD_ARG;
+}
+
+// ------------------------------------------------------------------------------------------------
+// Algorithm 3: for every candidate segment cap s, M(i,s) = min_{l(i)<=j<=i} d_j + M(j-1,s) with a
+// sliding-window minimum; answer min_s s + d_n + M(n-1,s).
+// ------------------------------------------------------------------------------------------------
+namespace {
+struct StaticTable {
+    int64_t n;
+    const int64_t* d;
+    std::vector<int64_t> prefix, key, M, arg, queue;
+    StaticTable(int64_t n_, const int64_t* d_) : n(n_), d(d_), prefix(n_ + 1), key(n_), M(n_), arg(n_), queue(n_) {
+        prefix[0] = 0;
+        for (int64_t i = 1; i <= n; ++i) prefix[i] = prefix[i - 1] + d[i];
+    }
+    // Fills M[0..n-1] (and arg) for one cap; returns M(n-1, s).
+    int64_t run(int64_t s, int64_t* work) {
+        int64_t head = 0, tail = 0;   // queue[head..tail)
+        int64_t lo = 0;               // l(i): smallest j with d_{j+1} + ... + d_i <= s
+        int64_t steps = 0;
+        for (int64_t i = 0; i < n; ++i) {
+            key[i] = d[i] + (i >= 1 ? M[i - 1] : 0);          // M(-1,s) = 0
+            while (tail > head && key[queue[tail - 1]] > key[i]) { --tail; ++steps; }
+            queue[tail++] = i;
+            while (prefix[i] - prefix[lo] > s) ++lo;
+            while (queue[head] < lo) { ++head; ++steps; }
+            M[i] = key[queue[head]];
+            arg[i] = queue[head];
+            ++steps;
+        }
+        if (work) *work += steps;
+        return M[n - 1];
+    }
+};
+}  // namespace
+
+int plan_static_n3(int64_t n, const int64_t* d, uint8_t* is_ckpt, int64_t* peak, int64_t* work) {
+    std::vector<int64_t> caps;
+    caps.push_back(0);
+    for (int64_t a = 1; a <= n - 1; ++a) {
+        int64_t acc = 0;
+        for (int64_t b = a; b <= n - 1; ++b) { acc += d[b]; caps.push_back(acc); }
+    }
+    std::sort(caps.begin(), caps.end());
+    caps.erase(std::unique(caps.begin(), caps.end()), caps.end());
+
+    StaticTable t(n, d);
+    int64_t best = -1, best_s = 0;
+    for (int64_t s : caps) {
+        // M(n-1,s) >= d_0, so no larger cap can do strictly better once this bound is reached.
+        if (best >= 0 && s + d[n] + d[0] >= best) break;
+        int64_t total = s + d[n] + t.run(s, work);
+        if (best < 0 || total < best) { best = total; best_s = s; }
+    }
+    t.run(best_s, nullptr);
+    for (int64_t i = 0; i <= n; ++i) is_ckpt[i] = 0;
+    is_ckpt[n] = 1;
+    for (int64_t i = n - 1; i >= 0;) {
+        int64_t j = t.arg[i];
+        is_ckpt[j] = 1;
+        i = j - 1;
+    }
+    *peak = best;
+    return CKPT_OK;
+}
+
+// ------------------------------------------------------------------------------------------------
+// Algorithm 5: M(n) = d_n; M(i) = min_{i<j<=n} max(d_i + M(j), d_i + s(i,j) + d_j).
+// ------------------------------------------------------------------------------------------------
+static void walk_next(int64_t n, const std::vector<int64_t>& nxt, uint8_t* is_ckpt) {
+    for (int64_t i = 0; i <= n; ++i) is_ckpt[i] = 0;
+    for (int64_t i = 0; i != n; i = nxt[i]) is_ckpt[i] = 1;
+    is_ckpt[n] = 1;
+}
+
+int plan_dynamic_n2(int64_t n, const int64_t* d, uint8_t* is_ckpt, int64_t* peak, int64_t* work) {
+    std::vector<int64_t> M(n + 1), nxt(n + 1, -1);
+    M[n] = d[n];
+    int64_t steps = 0;
+    for (int64_t i = n - 1; i >= 0; --i) {
+        int64_t seg_sum = 0, seg_max = d[i], best = -1, best_j = -1;
+        for (int64_t j = i + 1; j <= n; ++j) {
+            int64_t u = seg_sum + seg_max + d[j];              // U(i,j) = s(i,j) + d_j
+            int64_t v = d[i] + std::max(M[j], u);
+            if (best < 0 || v < best) { best = v; best_j = j; }
+            seg_sum += d[j];
+            seg_max = std::max(seg_max, d[j]);
+            ++steps;
+        }
+        M[i] = best;
+        nxt[i] = best_j;
+    }
+    walk_next(n, nxt, is_ckpt);
+    *peak = M[0];
+    if (work) *work += steps;
+    return CKPT_OK;
+}
+
+// ------------------------------------------------------------------------------------------------
+// Algorithm 6.  Q holds indices with strictly decreasing M as the index grows (Lemma 2); only Q has
+// to be searched (Lemma 3); U(i,.) increases along Q while M decreases, so max(M(j),U(i,j)) is
+// unimodal along Q and its minimum sits at the crossover; the crossover only moves towards smaller
+// j as i decreases (Lemma 4), so a pointer that walks along Q finds it in amortised O(1) moves.
+// U(i,j) is evaluated exactly from prefix sums and a range maximum: the record-maxima stack of the
+// suffix d_i, d_{i+1}, ... (maintained as i decreases) searched by bisection, O(log n) per value.
+// ------------------------------------------------------------------------------------------------
+int plan_dynamic_n(int64_t n, const int64_t* d, uint8_t* is_ckpt, int64_t* peak, int64_t* work) {
+    std::vector<int64_t> prefix(n + 1), M(n + 1), nxt(n + 1, -1), q(n + 1), rec(n + 1);
+    prefix[0] = 0;
+    for (int64_t i = 1; i <= n; ++i) prefix[i] = prefix[i - 1] + d[i];
+    int64_t steps = 0;
+
+    // rec[0..nrec): indices k with d_k larger than every d between the current i and k; stored with
+    // the largest index first, so indices decrease and values decrease along the array.
+    int64_t nrec = 0;
+    int64_t cur_i = 0;
+    auto range_max = [&](int64_t last) -> int64_t {   // max d[cur_i..last], last >= cur_i
+        // first position (from the front) whose index <= last
+        int64_t lo = 0, hi = nrec - 1;
+        while (lo < hi) {
+            int64_t mid = (lo + hi) / 2;
+            if (rec[mid] <= last) hi = mid; else lo = mid + 1;
+        }
+        return d[rec[lo]];
+    };
+    auto U = [&](int64_t j) -> int64_t {               // U(cur_i, j), j > cur_i
+        return prefix[j - 1] - prefix[cur_i] + range_max(j - 1) + d[j];
+    };
+
+    M[n] = d[n];
+    int64_t top = 0;      // q[0..top]: q[0] = n (largest index), q[top] = head (smallest index)
+    q[0] = n;
+    int64_t p = 0;        // position in q of the current minimiser
+    for (int64_t i = n - 1; i >= 0; --i) {
+        cur_i = i;
+        while (nrec > 0 && d[rec[nrec - 1]] <= d[i]) --nrec;
+        rec[nrec++] = i;
+
+        auto f = [&](int64_t t) -> int64_t { ++steps; return std::max(M[q[t]], U(q[t])); };
+        if (p > top) p = top;
+        int64_t fp = f(p);
+        // towards the head (smaller j) while not worse: on a tie the smaller j wins
+        while (p < top) {
+            int64_t fn = f(p + 1);
+            if (fn <= fp) { ++p; fp = fn; } else break;
+        }
+        // towards larger j only if strictly better (never needed when Lemma 4 holds)
+        while (p > 0) {
+            int64_t fn = f(p - 1);
+            if (fn < fp) { --p; fp = fn; } else break;
+        }
+        M[i] = d[i] + fp;
+        nxt[i] = q[p];
+        while (top >= 0 && M[q[top]] >= M[i]) { --top; ++steps; }
+        q[++top] = i;
+        ++steps;
+    }
+    walk_next(n, nxt, is_ckpt);
+    *peak = M[0];
+    if (work) *work += steps;
+    return CKPT_OK;
+}
+
+}  // namespace ckpt
+
+// ------------------------------------------------------------------------------------------------
+// C ABI
+// ------------------------------------------------------------------------------------------------
+extern "C" {
+
+const char* ckpt_last_error(void) { return ckpt::g_error; }
+
+int ckpt_plan_counted(int algo, int64_t n, const int64_t* d, uint8_t* is_ckpt, int64_t* peak_bytes,
+                      int64_t* work) {
+    int rc = ckpt::validate_sizes(n, d);
+    if (rc) return rc;
+    if (!is_ckpt || !peak_bytes) { ckpt::set_error("output pointer is null"); return CKPT_E_NULL; }
+    if (work) *work = 0;
+    switch (algo) {
+        case CKPT_ALGO_STATIC_N3: return ckpt::plan_static_n3(n, d, is_ckpt, peak_bytes, work);
+        case CKPT_ALGO_DYNAMIC_N2: return ckpt::plan_dynamic_n2(n, d, is_ckpt, peak_bytes, work);
+        case CKPT_ALGO_DYNAMIC_N: return ckpt::plan_dynamic_n(n, d, is_ckpt, peak_bytes, work);
+    }
+    ckpt::set_error("unknown algorithm %d", algo);
+    return CKPT_E_BAD_ARG;
+}
+
+int ckpt_plan(int algo, int64_t n, const int64_t* d, uint8_t* is_ckpt, int64_t* peak_bytes) {
+    return ckpt_plan_counted(algo, n, d, is_ckpt, peak_bytes, nullptr);
+}
+
+int ckpt_eval(int model, int64_t n, const int64_t* d, const uint8_t* is_ckpt, int64_t* peak_bytes) {
+    return ckpt::eval_model(model, n, d, is_ckpt, peak_bytes);
+}
+
+}  // extern "C"
