@@ -1,0 +1,300 @@
+"""Benchmark: checkpointed training-step throughput (images/s) of the VGG-16-shaped chain on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--config 2]
+
+One "step" = one full pass of the hot path over one synthetic batch: forward keeping the planned
+checkpoints, loss, backward with segment recomputation, all weight gradients.  The plan is the
+O(n) dynamic planner's (Algorithm 6) and the schedule is Algorithm 4.  With N > 1 (torchrun) every
+rank runs an independent replica on its own batch: the step has no exchange between GPUs.
+
+Prints one JSON line (rank 0).  `--impl reference` times the CPU oracle instead, on rank 0 only.
+"""
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2502_12499_b200 import workloads as wl  # noqa: E402
+
+METRIC = "checkpointed_train_step_images_per_s"
+UNIT = "images/s"
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return dict(hbm_gbs=p["hbm_gbs"], tflops_burst=p["bf16_tflops"], tflops_sustained=p["bf16_tflops_sustained"],
+                    source="measured")
+    return dict(hbm_gbs=6650.0, tflops_burst=1590.0, tflops_sustained=1400.0, source="fallback")
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    QUERY = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index = index
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.QUERY,
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            threading.Thread(target=self._pump, daemon=True).start()
+        except OSError:
+            self.proc = None
+
+    def _pump(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return dict(sm_mhz=None, sm_max_mhz=None, reasons=["nvidia-smi unavailable"])
+        time.sleep(0.15)
+        self.proc.terminate()
+        sm, smax, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in self.lines:
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 6:
+                continue
+            try:
+                sm.append(float(parts[0])); smax.append(float(parts[1]))
+            except ValueError:
+                continue
+            for name, flag in zip(names, parts[2:6]):
+                if flag.lower().startswith("active"):
+                    reasons.add(name)
+        return dict(sm_mhz=float(np.median(sm)) if sm else None, sm_max_mhz=max(smax) if smax else None,
+                    reasons=sorted(reasons), samples=len(sm))
+
+
+def conv_flops(spec, plan_mask, shapes):
+    """Algorithmic FLOPs of one step: 2*MAC x (forward + recompute of non-checkpoints + backward
+    re-derivation of the pre-normalisation tensor + dgrad (units 2..n) + wgrad)."""
+    fwd = []
+    h, w, c = spec["input_hwc"]
+    for u, (ho, wo, co) in zip(spec["units"], shapes[1:]):
+        if u["kind"] == "conv_bn_relu":
+            fwd.append(2.0 * spec["batch"] * ho * wo * co * u["k"] * u["k"] * u["cin"])
+        elif u["kind"] == "fc":
+            fwd.append(2.0 * spec["batch"] * u["cin"] * u["cout"])
+        else:
+            fwd.append(0.0)
+    total = 0.0
+    for i, f in enumerate(fwd, start=1):
+        conv = spec["units"][i - 1]["kind"] == "conv_bn_relu"
+        total += f                                   # forward
+        if not plan_mask[i]:
+            total += f                               # segment recompute
+        if conv:
+            total += f                               # backward re-derives the conv output
+        total += f                                   # wgrad
+        if i > 1:
+            total += f                               # dgrad
+    return total, fwd
+
+
+def run_reference(args, spec):
+    """The CPU oracle, as it stands, on a bounded sample of the same workload."""
+    from oracle import numeric_oracle as no
+    try:
+        from threadpoolctl import threadpool_info
+        cores = max([p.get("num_threads", 1) for p in threadpool_info()] + [1])
+    except Exception:
+        cores = os.cpu_count()
+    sample_batch = min(spec["batch"], args.cpu_batch)
+    small = dict(spec, batch=sample_batch)
+    params = wl.make_params(small, seed=0)
+    x, labels = wl.make_batch(small, seed=1)
+    times = []
+    for it in range(args.warmup_cpu + args.steps_cpu):
+        t0 = time.perf_counter()
+        no.chain_forward_backward(small, params, x, labels)
+        dt = time.perf_counter() - t0
+        if it >= args.warmup_cpu:
+            times.append(dt)
+    t = float(np.mean(times))
+    return dict(value=sample_batch / t, unit=UNIT, cores=int(cores), kind="oracle",
+                sample="store-all step of the same chain on a batch of %d of %d images, float64 numpy, %d timed step(s)"
+                       % (sample_batch, spec["batch"], len(times)), seconds_per_step=t)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours")
+    ap.add_argument("--config", type=int, default=2)
+    ap.add_argument("--batch", type=int, default=0, help="override the batch size (debugging only)")
+    ap.add_argument("--cpu-batch", type=int, default=4)
+    ap.add_argument("--steps-cpu", type=int, default=1)
+    ap.add_argument("--warmup-cpu", type=int, default=0)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    spec = wl.config(args.config)
+    if args.batch:
+        spec = dict(spec, batch=args.batch)
+    config = {"workload": "%s: %d units, batch %d of %dx%dx%d %s, plan = Algorithm 6, schedule = Algorithm 4"
+                          % (spec["name"], len(spec["units"]), spec["batch"], *spec["input_hwc"], spec["dtype"]),
+              "l2": "inputs larger than L2 (every step streams > 1 GB of activations)",
+              "parallelism": "replicas x%d" % world if world > 1 else "single GPU"}
+
+    if args.impl == "reference":
+        if rank != 0:
+            return
+        cpu = run_reference(args, spec)
+        line = {"impl": "reference", "metric": METRIC, "value": cpu["value"], "unit": UNIT, "n_gpus": args.gpus,
+                "steps": args.steps_cpu, "warmup": args.warmup_cpu, "ms_per_step": 1e3 * cpu["seconds_per_step"],
+                "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+                "config": config, "cpu_baseline": cpu,
+                "e2e": {"value": cpu["value"], "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+                "gpu_launches": 0}
+        print(json.dumps(line))
+        return
+
+    import torch
+    import torch.distributed as dist
+    from paper_2502_12499_b200 import binding as ck
+
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl")
+
+    chain = ck.Chain(spec)
+    d = chain.sizes()
+    shapes = [tuple(int(v) for v in s) for s in chain.shapes()]
+    t0 = time.perf_counter()
+    mask, peak = ck.plan(ck.ALGO_DYNAMIC_N, d)
+    plan_us = 1e6 * (time.perf_counter() - t0)
+    store_all = ck.eval(ck.MODEL_STORE_ALL, d, None)
+
+    params_h = wl.make_params(spec, seed=0)
+    params, grads, _ = ck.upload_params(chain, params_h)
+    del params_h
+    x_h, labels_h = wl.make_batch(spec, seed=1 + rank)
+    tdt = torch.bfloat16 if spec["dtype"] == "bf16" else torch.float32
+    x_pinned = torch.from_numpy(x_h).to(tdt).pin_memory()
+    labels_pinned = torch.from_numpy(labels_h).pin_memory()
+    x_dev = x_pinned.cuda()
+    labels_dev = labels_pinned.cuda()
+    arena = torch.empty(peak, dtype=torch.uint8, device="cuda")
+    workspace = torch.empty(chain.workspace_bytes(), dtype=torch.uint8, device="cuda")
+    stream = torch.cuda.current_stream()
+
+    def step(batch, labels):
+        return ck.train_step(chain, mask, ck.POLICY_DYNAMIC, batch, labels, params, grads, arena, workspace, stream)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def timed(batch, labels, steps):
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        rep = None
+        for _ in range(steps):
+            rep = step(batch, labels)
+        e1.record(stream)
+        barrier()
+        ms = e0.elapsed_time(e1)
+        if world > 1:
+            t = torch.tensor([ms], device="cuda")
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms = t.item()
+        return ms, rep
+
+    for _ in range(max(args.warmup, 3)):
+        rep = step(x_dev, labels_dev)
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+    ms, rep = timed(x_dev, labels_dev, args.steps)
+    ms_e2e, rep_e2e = timed(x_pinned, labels_pinned, args.steps)
+    clocks = sampler.stop() if rank == 0 else None
+
+    images = spec["batch"] * world * args.steps
+    value = images / (ms * 1e-3)
+    e2e_value = images / (ms_e2e * 1e-3)
+
+    if rank == 0:
+        peaks = measured_peaks()
+        flops, _ = conv_flops(spec, mask, shapes)
+        roofline = dominant_kernel_roofline(ck, spec, shapes, peaks, torch, stream)
+        line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+                "warmup": max(args.warmup, 3), "ms_per_step": ms / args.steps, "higher_is_better": True,
+                "scaling": "weak", "vs_baseline": None, "dtype": spec["dtype"], "data": "synthetic", "config": config,
+                "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": int(x_pinned.numel() * x_pinned.element_size() + labels_pinned.numel() * 4),
+                        "d2h_bytes_per_step": 12},
+                "gpu_launches": int(rep["launches"]) * args.steps, "clocks": clocks, "roofline": roofline,
+                "peak_bytes": int(rep["peak_bytes"]), "predicted_bytes": int(peak), "store_all_bytes": int(store_all),
+                "peak_gib": rep["peak_bytes"] / 2 ** 30, "workspace_gib": chain.workspace_bytes() / 2 ** 30,
+                "recomputed_units": int(rep["recomputed_units"]), "plan_us": plan_us, "loss": rep["loss"],
+                "step_tflops": flops / (ms / args.steps * 1e-3) / 1e12,
+                "step_tensor_frac_of_sustained": flops / (ms / args.steps * 1e-3) / 1e12 / peaks["tflops_sustained"],
+                "peaks": peaks}
+        if not args.no_cpu_baseline and world == 1:
+            line["cpu_baseline"] = run_reference(args, spec)
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def dominant_kernel_roofline(ck, spec, shapes, peaks, torch, stream):
+    """Times the convolution-forward kernel on every conv layer shape of the workload (it runs in
+    the forward phase, in segment recomputation and at the start of every unit's backward) and
+    reports the launch-weighted throughput against the measured tensor-core peak."""
+    dtype = ck.DTYPE_BF16 if spec["dtype"] == "bf16" else ck.DTYPE_F32
+    tdt = torch.bfloat16 if spec["dtype"] == "bf16" else torch.float32
+    total_flops, total_ms, launches = 0.0, 0.0, 0
+    per_layer = []
+    for u, (hi, wi, ci), (ho, wo, co) in zip(spec["units"], shapes[:-1], shapes[1:]):
+        if u["kind"] != "conv_bn_relu" or u["cin"] < 16:
+            continue
+        shape = ck.ConvShape(spec["batch"], hi, wi, ci, co, u["k"], u["stride"], u["pad"])
+        x = torch.randn(spec["batch"], hi, wi, ci, device="cuda").to(tdt)
+        w = (torch.randn(co, u["k"], u["k"], ci, device="cuda") * 0.05).to(tdt)
+        z = torch.empty(spec["batch"], ho, wo, co, device="cuda", dtype=tdt)
+        scratch = torch.empty(max(256, ck.conv2d_scratch_bytes(shape, dtype)), dtype=torch.uint8, device="cuda")
+        reps = 3
+        ck.conv2d_forward(shape, dtype, 0, x, w, z, scratch, stream)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        e0.record(stream)
+        for _ in range(reps):
+            ck.conv2d_forward(shape, dtype, 0, x, w, z, scratch, stream)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1) / reps
+        fl = 2.0 * spec["batch"] * ho * wo * co * u["k"] * u["k"] * ci
+        total_flops += fl; total_ms += ms; launches += 1
+        per_layer.append({"shape": "%dx%dx%d->%d" % (hi, wi, ci, co), "ms": ms, "tflops": fl / ms / 1e9})
+        del x, w, z, scratch
+    achieved = total_flops / (total_ms * 1e-3) / 1e12 if total_ms > 0 else 0.0
+    return {"kernel": "conv forward (implicit GEMM)", "bound": "tensor", "achieved": achieved, "peak": peaks["tflops_burst"],
+            "unit": "TFLOP/s", "frac": achieved / peaks["tflops_burst"], "peak_source": peaks["source"], "traffic": None,
+            "launch_shapes": launches, "per_layer": per_layer}
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,139 @@
+"""GPU parity of the single operations against the float64 oracle, through the C ABI.
+
+Tolerances (max |err| / max |ref| per tensor): 1e-3 for float32 storage (plain FMA arithmetic, no
+TF32), 3e-2 for bfloat16 storage with float32 accumulation.  Inputs handed to both sides are
+already rounded to the storage type, so the only differences are accumulation order and the final
+rounding of each output element."""
+import numpy as np
+import pytest
+
+from oracle import numeric_oracle as no
+from paper_2502_12499_b200 import binding as ck
+from paper_2502_12499_b200 import workloads as wl
+from tests.gpu_util import max_rel_err, to_dev, to_host
+
+pytestmark = pytest.mark.gpu
+TOL = {ck.DTYPE_F32: 1e-3, ck.DTYPE_BF16: 3e-2}
+# pure rounding of one bf16 output is 2^-9 relative; anything above a few of those is a bug
+TIGHT = {ck.DTYPE_F32: 2e-5, ck.DTYPE_BF16: 6e-3}
+
+CONV_CASES = [
+    # n, h, w, cin, cout, k, stride, pad
+    (2, 9, 7, 3, 5, 3, 1, 1),        # ragged everything, tiny channels
+    (4, 32, 32, 3, 16, 3, 1, 1),     # first layer of the 8-unit chain
+    (4, 32, 32, 16, 16, 3, 1, 1),
+    (3, 17, 13, 24, 40, 3, 2, 1),    # stride 2
+    (2, 14, 14, 64, 96, 1, 1, 0),    # 1x1
+    (2, 15, 15, 32, 64, 1, 2, 0),    # 1x1 stride 2 (projection shortcut)
+    (2, 23, 19, 3, 16, 7, 2, 3),     # stem-like
+    (3, 28, 28, 64, 64, 3, 1, 1),    # several 64-wide tiles with a tail
+    (5, 1, 1, 200, 70, 1, 1, 0),     # fully connected as a 1x1 convolution
+]
+
+
+def rounded(a, dtype):
+    a = a.astype(np.float32)
+    return wl.to_bf16_representable(a) if dtype == ck.DTYPE_BF16 else a
+
+
+@pytest.mark.parametrize("dtype", [ck.DTYPE_F32, ck.DTYPE_BF16])
+@pytest.mark.parametrize("case", CONV_CASES)
+def test_conv_cuda_core_kernels(case, dtype):
+    import torch
+    n, h, w, cin, cout, k, stride, pad = case
+    rng = np.random.default_rng(hash(case) % 2 ** 31)
+    x = rounded(rng.standard_normal((n, h, w, cin)), dtype)
+    wt = rounded(rng.standard_normal((cout, k, k, cin)) / np.sqrt(k * k * cin), dtype)
+    z_ref = no.conv2d_fwd(x.astype(np.float64), wt.astype(np.float64), stride, pad)
+    dz = rounded(rng.standard_normal(z_ref.shape), dtype)
+    dx_ref, dw_ref = no.conv2d_bwd(x.astype(np.float64), wt.astype(np.float64), dz.astype(np.float64), stride, pad)
+
+    shape = ck.ConvShape(n, h, w, cin, cout, k, stride, pad)
+    xd, wd, dzd = to_dev(x, dtype), to_dev(wt, dtype), to_dev(dz, dtype)
+    z = torch.full(z_ref.shape, float("nan"), device="cuda").to(xd.dtype)
+    dx = torch.full(x.shape, float("nan"), device="cuda").to(xd.dtype)
+    dw = torch.full(wt.shape, float("nan"), device="cuda", dtype=torch.float32)
+    sb = ck.conv2d_scratch_bytes(shape, dtype)
+    scratch = torch.empty(max(sb, 256), dtype=torch.uint8, device="cuda")
+    ck.conv2d_forward(shape, dtype, 1, xd, wd, z, scratch)
+    ck.conv2d_dgrad(shape, dtype, 1, dzd, wd, dx, scratch)
+    ck.conv2d_wgrad(shape, dtype, 1, dzd, xd, dw, scratch)
+    torch.cuda.synchronize()
+    assert max_rel_err(to_host(z), z_ref) <= TIGHT[dtype]
+    assert max_rel_err(to_host(dx), dx_ref) <= TIGHT[dtype]
+    assert max_rel_err(to_host(dw), dw_ref) <= 2e-5        # gradients are float32 in both modes
+    assert TIGHT[dtype] <= TOL[dtype]
+
+
+@pytest.mark.parametrize("dtype", [ck.DTYPE_F32, ck.DTYPE_BF16])
+@pytest.mark.parametrize("rows,c,relu", [(37, 3, 1), (4096, 16, 1), (5000, 64, 1), (777, 40, 0), (64, 1000, 0), (3001, 24, 1)])
+def test_batchnorm_relu(rows, c, relu, dtype):
+    import torch
+    rng = np.random.default_rng(rows * 7 + c)
+    z = rounded(rng.standard_normal((1, 1, rows, c)) * 2 + 0.5, dtype)
+    gamma = rng.uniform(0.5, 1.5, c).astype(np.float32)
+    beta = (rng.standard_normal(c) * 0.3).astype(np.float32)
+    dy = rounded(rng.standard_normal(z.shape), dtype)
+    y_ref, cache = no.bn_fwd(z.astype(np.float64), gamma.astype(np.float64), beta.astype(np.float64))
+    if relu:
+        y_ref = np.maximum(y_ref, 0)
+    g_ref = dy.astype(np.float64) * ((y_ref > 0) if relu else 1.0)
+    dz_ref, dgamma_ref, dbeta_ref = no.bn_bwd(g_ref, cache, gamma.astype(np.float64))
+
+    zd, dyd = to_dev(z, dtype), to_dev(dy, dtype)
+    gd, bd = torch.from_numpy(gamma).cuda(), torch.from_numpy(beta).cuda()
+    y = torch.empty_like(zd)
+    stats = torch.empty(4 * c, device="cuda", dtype=torch.float32)
+    scratch = torch.empty(ck.bn_scratch_bytes(rows, c), dtype=torch.uint8, device="cuda")
+    ck.bn_relu_forward(dtype, rows, c, zd, gd, bd, relu, y, stats, scratch)
+    dz = torch.empty_like(zd)
+    dgamma = torch.empty(c, device="cuda"); dbeta = torch.empty(c, device="cuda")
+    ck.bn_relu_backward(dtype, rows, c, dyd, zd, gd, stats, relu, dz, dgamma, dbeta, scratch)
+    torch.cuda.synchronize()
+    xhat, inv_std = cache
+    assert max_rel_err(to_host(stats[c:2 * c]), inv_std) <= 1e-5
+    assert max_rel_err(to_host(y), y_ref) <= TIGHT[dtype]
+    # elements whose forward output rounds to exactly zero in bf16 may flip the mask; none here
+    assert max_rel_err(to_host(dbeta), dbeta_ref) <= 1e-4
+    assert max_rel_err(to_host(dgamma), dgamma_ref) <= 1e-4
+    assert max_rel_err(to_host(dz), dz_ref) <= TIGHT[dtype]
+    # in-place variant (dz aliases dy) gives the same bits
+    ck.bn_relu_backward(dtype, rows, c, dyd, zd, gd, stats, relu, dyd, dgamma, dbeta, scratch)
+    torch.cuda.synchronize()
+    assert torch.equal(dyd, dz)
+
+
+@pytest.mark.parametrize("dtype", [ck.DTYPE_F32, ck.DTYPE_BF16])
+@pytest.mark.parametrize("n,h,w,c,k,stride,pad", [(2, 8, 6, 5, 2, 2, 0), (3, 13, 11, 8, 3, 2, 1), (2, 32, 32, 16, 2, 2, 0)])
+def test_maxpool(n, h, w, c, k, stride, pad, dtype):
+    import torch
+    rng = np.random.default_rng(h * w)
+    x = rng.integers(-3, 4, size=(n, h, w, c)).astype(np.float32)          # many exact ties
+    y_ref, arg = no.maxpool_fwd(x.astype(np.float64), k, stride, pad)
+    dy = rounded(rng.standard_normal(y_ref.shape), dtype)
+    dx_ref = no.maxpool_bwd(dy.astype(np.float64), arg, x.shape, k, stride, pad)
+    xd, dyd = to_dev(x, dtype), to_dev(dy, dtype)
+    y = torch.empty(y_ref.shape, device="cuda").to(xd.dtype)
+    dx = torch.empty_like(xd)
+    ck.maxpool_forward(dtype, n, h, w, c, k, stride, pad, xd, y)
+    ck.maxpool_backward(dtype, n, h, w, c, k, stride, pad, xd, dyd, dx)
+    torch.cuda.synchronize()
+    assert np.array_equal(to_host(y), y_ref)
+    assert max_rel_err(to_host(dx), dx_ref) <= TIGHT[dtype]
+
+
+@pytest.mark.parametrize("dtype", [ck.DTYPE_F32, ck.DTYPE_BF16])
+def test_softmax_cross_entropy(dtype):
+    import torch
+    rng = np.random.default_rng(5)
+    logits = rounded(rng.standard_normal((64, 1, 1, 1000)) * 3, dtype)
+    labels = rng.integers(0, 1000, 64).astype(np.int32)
+    loss_ref, g_ref = no.softmax_ce(logits.astype(np.float64), labels)
+    ld = to_dev(logits, dtype)
+    lab = torch.from_numpy(labels).cuda()
+    loss = torch.zeros(1, device="cuda")
+    g = torch.empty_like(ld)
+    ck.softmax_ce(dtype, 64, 1000, ld, lab, loss, g)
+    torch.cuda.synchronize()
+    assert abs(loss.item() - loss_ref) <= 1e-5 * abs(loss_ref)
+    assert max_rel_err(to_host(g), g_ref) <= TIGHT[dtype]

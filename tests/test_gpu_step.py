@@ -1,0 +1,128 @@
+"""GPU parity of the whole training step (ckpt_train_step) against the oracle's store-all step.
+
+Checked for every case: weight gradients within tolerance of the float64 oracle; gradients of every
+checkpointed run bit-identical to the GPU's own store-all run; arena high-water mark == highest
+offset used == the planner's predicted peak, with an arena of exactly that many bytes."""
+import random
+
+import numpy as np
+import pytest
+
+from oracle import numeric_oracle as no
+from oracle import planner_oracle as po
+from paper_2502_12499_b200 import binding as ck
+from paper_2502_12499_b200 import workloads as wl
+from tests.gpu_util import StepRunner, max_rel_err
+
+pytestmark = pytest.mark.gpu
+TOL = {"f32": 1e-3, "bf16": 3e-2}
+
+
+def mini_vgg(dtype, batch=4):
+    return wl.vgg16_chain(batch, hw=(32, 32), dtype=dtype, widths=(8, 16, 24, 32, 32), fc_width=48, classes=10,
+                          name="mini_vgg_" + dtype)
+
+
+def oracle_step(spec, params, x, labels):
+    p64 = [{k: v.astype(np.float64) for k, v in p.items()} for p in params]
+    return no.chain_forward_backward(spec, p64, x.astype(np.float64), labels)
+
+
+def compare_with_oracle(runner, grads, ref, tol):
+    worst = 0.0
+    for (ui, name, _), g in zip(runner.flat, grads):
+        want = ref["grads"][ui][name]
+        assert np.all(np.isfinite(g)), (ui, name)
+        err = max_rel_err(g.reshape(want.shape), want)
+        assert err <= tol, (ui, name, err)
+        worst = max(worst, err)
+    return worst
+
+
+def all_policies_agree(runner, x, labels, masks_dynamic, masks_static):
+    rep0, g0 = runner.run(ck.POLICY_STORE_ALL, None, x, labels)
+    assert rep0["peak_bytes"] == rep0["extent_bytes"] == rep0["predicted_bytes"] == int(sum(runner.d))
+    assert rep0["recomputed_units"] == 0 and rep0["launches"] > 0 and rep0["device_status"] == 0
+    for policy, masks in ((ck.POLICY_DYNAMIC, masks_dynamic), (ck.POLICY_STATIC, masks_static)):
+        for mask in masks:
+            rep, g = runner.run(policy, mask, x, labels)
+            C = [int(i) for i in np.nonzero(mask)[0]]
+            want = (po.eval_dynamic if policy == ck.POLICY_DYNAMIC else po.eval_static)([int(v) for v in runner.d], C)
+            assert rep["peak_bytes"] == rep["extent_bytes"] == rep["predicted_bytes"] == want
+            assert rep["recomputed_units"] == runner.n + 1 - len(C)
+            assert rep["loss"] == rep0["loss"]
+            for a, b in zip(g, g0):
+                assert np.array_equal(a, b)            # bit-identical to the store-all run
+    return rep0, g0
+
+
+def test_config1_plain8_fp32_all_masks():
+    spec = wl.config(1)
+    params = wl.make_params(spec, seed=0)
+    x, _ = wl.make_batch(spec, seed=1)
+    runner = StepRunner(spec, params)
+    d = [int(v) for v in runner.d]
+    assert d == [49152] + [262144] * 8
+    # the planners' sets (checked against brute force over all 256 masks on the CPU side)
+    m6, peak6 = ck.plan(ck.ALGO_DYNAMIC_N, d)
+    m3, peak3 = ck.plan(ck.ALGO_STATIC_N3, d)
+    assert peak6 == po.brute_force_dynamic(d)["value"] and peak3 == po.brute_force_static(d)["value"]
+    masks = [m6, m3]
+    rng = random.Random(0)
+    every = [ck.mask_from_set(8, [0] + [i for i in range(1, 8) if (bits >> (i - 1)) & 1] + [8]) for bits in range(128)]
+    masks += rng.sample(every, 12)
+    rep0, g0 = all_policies_agree(runner, x, None, masks, masks)
+    ref = oracle_step(spec, params, x, None)
+    assert abs(rep0["loss"] - ref["loss"]) <= 1e-5 * abs(ref["loss"])
+    compare_with_oracle(runner, g0, ref, TOL["f32"])
+    # the high-water mark of all 128 feasible masks equals Eq. (memory) (arena of exactly that size)
+    for mask in every:
+        rep, _ = runner.run(ck.POLICY_DYNAMIC, mask, x, None)
+        assert rep["peak_bytes"] == rep["need"] == rep["extent_bytes"]
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_mini_vgg_against_oracle(dtype):
+    spec = mini_vgg(dtype)
+    params = wl.make_params(spec, seed=3, bn_affine="random")
+    x, labels = wl.make_batch(spec, seed=4)
+    runner = StepRunner(spec, params)
+    d = [int(v) for v in runner.d]
+    n = runner.n
+    m6, _ = ck.plan(ck.ALGO_DYNAMIC_N, d)
+    m3, _ = ck.plan(ck.ALGO_STATIC_N3, d)
+    rng = random.Random(1)
+    extra = [ck.mask_from_set(n, [0] + [i for i in range(1, n) if rng.random() < 0.4] + [n]) for _ in range(4)]
+    extra.append(ck.mask_from_set(n, [0, n]))
+    extra.append(ck.mask_from_set(n, range(n + 1)))
+    rep0, g0 = all_policies_agree(runner, x, labels, [m6] + extra, [m3] + extra)
+    ref = oracle_step(spec, params, x, labels)
+    assert abs(rep0["loss"] - ref["loss"]) <= (1e-5 if dtype == "f32" else 2e-2) * abs(ref["loss"])
+    compare_with_oracle(runner, g0, ref, TOL[dtype])
+
+
+def test_ragged_chain_fp32():
+    # odd spatial sizes and channel counts: nothing is a multiple of a tile or a vector width
+    units = [wl.conv_unit(3, 7), wl.conv_unit(7, 13, k=3, stride=2, pad=1), {"kind": "maxpool", "k": 3, "stride": 2, "pad": 1},
+             wl.conv_unit(13, 10, k=1, stride=1, pad=0), {"kind": "avgpool"}, {"kind": "fc", "cin": 10, "cout": 6, "relu": False}]
+    spec = dict(units=units, input_hwc=(19, 23, 3), batch=3, dtype="f32", loss="softmax_ce", name="ragged")
+    params = wl.make_params(spec, seed=5, bn_affine="random")
+    x, labels = wl.make_batch(spec, seed=6)
+    runner = StepRunner(spec, params)
+    n = runner.n
+    masks = [ck.mask_from_set(n, [0, n]), ck.mask_from_set(n, [0, 2, 4, n]), ck.plan(ck.ALGO_DYNAMIC_N, runner.d)[0]]
+    rep0, g0 = all_policies_agree(runner, x, labels, masks, masks)
+    ref = oracle_step(spec, params, x, labels)
+    compare_with_oracle(runner, g0, ref, TOL["f32"])
+
+
+def test_arena_too_small_is_rejected_before_any_launch():
+    spec = wl.config(1)
+    runner = StepRunner(spec, wl.make_params(spec, seed=0))
+    x, _ = wl.make_batch(spec, seed=1)
+    mask, peak = ck.plan(ck.ALGO_DYNAMIC_N, runner.d)
+    with pytest.raises(ck.CkptError) as e:
+        runner.run(ck.POLICY_DYNAMIC, mask, x, None, arena_bytes=peak - 256)
+    assert e.value.code == -7
+    rep, _ = runner.run(ck.POLICY_DYNAMIC, mask, x, None, arena_bytes=peak)
+    assert rep["peak_bytes"] == peak
