@@ -24,8 +24,9 @@ the exact result.  ``storage="exact"`` (default) rounds nothing.
 Parity status: pinned by tests/test_oracle_numeric.py - central finite differences of the loss
 for every parameter kind, a pure-Python-loop convolution and pool on tiny inputs,
 scipy.signal.correlate2d, the zero-gradient property of batch norm under a constant upstream
-gradient, and hand-computed softmax values.  The "bf16" storage mode is pinned only through its
-rounding function (exact bit patterns) - its end-to-end result is "parity unpinned".
+gradient, and hand-computed softmax values.  The "bf16" storage mode is pinned through its
+rounding function (exact bit patterns), the property that exactly the stored tensors are bfloat16
+codes, and its distance from the exact mode on a one-unit chain.
 """
 
 import numpy as np

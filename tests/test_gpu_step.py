@@ -23,9 +23,9 @@ def mini_vgg(dtype, batch=4):
                           name="mini_vgg_" + dtype)
 
 
-def oracle_step(spec, params, x, labels):
+def oracle_step(spec, params, x, labels, storage="exact"):
     p64 = [{k: v.astype(np.float64) for k, v in p.items()} for p in params]
-    return no.chain_forward_backward(spec, p64, x.astype(np.float64), labels)
+    return no.chain_forward_backward(spec, p64, x.astype(np.float64), labels, storage=storage)
 
 
 def compare_with_oracle(runner, grads, ref, tol):
@@ -83,6 +83,13 @@ def test_config1_plain8_fp32_all_masks():
 
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
 def test_mini_vgg_against_oracle(dtype):
+    """16 units deep.  float32: against the exact oracle.  bfloat16: every stored tensor is a
+    quantised code and every ReLU mask / pooling arg-max is a discrete decision taken on those
+    codes, so the oracle takes them in the kernel's precision too (storage="bf16": float64
+    arithmetic, tensors rounded to bfloat16 where the executor stores them).  Against the exact
+    oracle a 16-unit bfloat16 chain differs by tens of percent for purely mathematical reasons
+    (the oracle's own two modes differ by that much), which is why that comparison is made on the
+    one-unit-deep chains below instead."""
     spec = mini_vgg(dtype)
     params = wl.make_params(spec, seed=3, bn_affine="random")
     x, labels = wl.make_batch(spec, seed=4)
@@ -96,9 +103,39 @@ def test_mini_vgg_against_oracle(dtype):
     extra.append(ck.mask_from_set(n, [0, n]))
     extra.append(ck.mask_from_set(n, range(n + 1)))
     rep0, g0 = all_policies_agree(runner, x, labels, [m6] + extra, [m3] + extra)
-    ref = oracle_step(spec, params, x, labels)
-    assert abs(rep0["loss"] - ref["loss"]) <= (1e-5 if dtype == "f32" else 2e-2) * abs(ref["loss"])
+    ref = oracle_step(spec, params, x, labels, storage="exact" if dtype == "f32" else "bf16")
+    assert abs(rep0["loss"] - ref["loss"]) <= 1e-5 * abs(ref["loss"])
     compare_with_oracle(runner, g0, ref, TOL[dtype])
+    if dtype == "bf16":
+        exact = oracle_step(spec, params, x, labels)
+        assert abs(rep0["loss"] - exact["loss"]) <= 2e-2 * abs(exact["loss"])
+
+
+def shallow_chains():
+    s = wl.plain_chain(1, 32, 16, (24, 20), 16, "bf16", "softmax_ce", name="conv+fc")
+    s["units"].append({"kind": "fc", "cin": 24 * 20 * 32, "cout": 10, "relu": False})
+    yield s
+    s = wl.plain_chain(1, 24, 8, (16, 16), 32, "bf16", "softmax_ce", name="conv+pool+fc")
+    s["units"] += [{"kind": "maxpool", "k": 2, "stride": 2, "pad": 0}, {"kind": "fc", "cin": 8 * 8 * 24, "cout": 10, "relu": False}]
+    yield s
+    s = dict(units=[{"kind": "fc", "cin": 6 * 6 * 8, "cout": 40, "relu": True}, {"kind": "fc", "cin": 40, "cout": 12, "relu": False}],
+             input_hwc=(6, 6, 8), batch=16, dtype="bf16", loss="softmax_ce", name="fc+fc")
+    yield s
+
+
+@pytest.mark.parametrize("spec", list(shallow_chains()), ids=lambda s: s["name"])
+def test_shallow_bf16_chains_against_exact_oracle(spec):
+    """bfloat16 storage against the *exact* float64 oracle, on chains one parametrised unit deep
+    below the classifier, where one rounding per stored tensor is the only difference."""
+    params = wl.make_params(spec, seed=11, bn_affine="random")
+    x, labels = wl.make_batch(spec, seed=12)
+    runner = StepRunner(spec, params)
+    n = runner.n
+    masks = [ck.mask_from_set(n, [0, n]), ck.plan(ck.ALGO_DYNAMIC_N, runner.d)[0]]
+    rep0, g0 = all_policies_agree(runner, x, labels, masks, masks)
+    ref = oracle_step(spec, params, x, labels)
+    assert abs(rep0["loss"] - ref["loss"]) <= 5e-3 * abs(ref["loss"])
+    compare_with_oracle(runner, g0, ref, TOL["bf16"])
 
 
 def test_ragged_chain_fp32():

@@ -173,3 +173,26 @@ def test_output_shapes_match_forward():
         x, _ = wl.make_batch(chain, seed=2)
         d, _, _ = no.chain_forward(chain, params, x)
         assert [t.shape[1:] for t in d] == no.output_shapes(chain)
+
+
+def test_bf16_storage_mode_rounds_stored_tensors_only():
+    """storage="bf16": every stored tensor is a bfloat16 code, the arithmetic stays float64, and on
+    a one-unit chain the result stays within a few roundings of the exact one."""
+    spec = wl.plain_chain(1, 8, 4, (6, 6), 8, "bf16", "softmax_ce")
+    spec["units"].append({"kind": "fc", "cin": 6 * 6 * 8, "cout": 5, "relu": False})
+    params = wl.make_params(spec, seed=1, bn_affine="random")
+    params = [{k: v.astype(np.float64) for k, v in p.items()} for p in params]
+    x, labels = wl.make_batch(spec, seed=2)
+    exact = no.chain_forward_backward(spec, params, x.astype(np.float64), labels)
+    stored = no.chain_forward_backward(spec, params, x.astype(np.float64), labels, storage="bf16")
+    for t in stored["d"]:
+        assert np.array_equal(t, no.round_bf16(t))
+    assert not np.array_equal(exact["d"][1], no.round_bf16(exact["d"][1]))
+    # conv output of unit 1: stored = round(exact conv), nothing else
+    z_exact = no.conv2d_fwd(x.astype(np.float64), params[0]["w"], 1, 1)
+    y_stored, _ = no.bn_fwd(no.round_bf16(z_exact), params[0]["gamma"], params[0]["beta"])
+    assert np.array_equal(stored["d"][1], no.round_bf16(np.maximum(y_stored, 0)))
+    for ge, gs in zip(exact["grads"], stored["grads"]):
+        for k in ge:
+            assert np.abs(ge[k] - gs[k]).max() <= 3e-2 * np.abs(ge[k]).max()
+    assert abs(exact["loss"] - stored["loss"]) <= 5e-3 * abs(exact["loss"])
