@@ -250,6 +250,25 @@ CKPT_API int ckpt_bn_relu_backward(int dtype, int64_t rows, int32_t c, const voi
                           const float* gamma, const float* stats, int relu, void* dz, float* dgamma,
                           float* dbeta, void* scratch, void* stream);
 
+/* Same result as ckpt_bn_relu_forward, for callers that cannot allocate device memory and therefore
+ * have no scratch buffer to pass: code embedded in a framework that owns the whole memory budget,
+ * latency-critical loops that must avoid the device-wide synchronisation of cudaMalloc/cudaFree,
+ * or callers that were themselves only given input and output buffers.  (The paper has no
+ * counterpart to this call; it exists for deployment only.)
+ *   - The partial sums live in an array built into the library image (4,857,856 bytes, resident on
+ *     every GPU that loads the library until the process exits), enough for
+ *     c <= CKPT_BN_STATIC_MAX_CHANNELS and any row count; a larger c returns CKPT_E_UNSUPPORTED.
+ *   - The call performs no cudaMalloc/cudaFree and calls no allocating routine.
+ *   - The first call on each device looks up the array's device address; make that first call
+ *     before starting any stream capture on that device.
+ *   - All calls share the one array, which keeps whatever the previous call left in it (nothing in
+ *     it needs clearing: each call overwrites what it reads).  Two calls that may run on the GPU at
+ *     the same time - different streams, or different host threads - race on it: serialise them.
+ * Pointers as for ckpt_bn_relu_forward (all device); asynchronous on `stream`. */
+#define CKPT_BN_STATIC_MAX_CHANNELS 512
+CKPT_API int ckpt_bn_relu_forward_noalloc(int dtype, int64_t rows, int32_t c, const void* z, const float* gamma,
+                                 const float* beta, int relu, void* y, float* stats, void* stream);
+
 /* Max pooling, NHWC.  backward recomputes the arg-max from x. */
 CKPT_API int ckpt_maxpool_forward(int dtype, int32_t n, int32_t h, int32_t w, int32_t c, int32_t k,
                          int32_t stride, int32_t pad, const void* x, void* y, void* stream);

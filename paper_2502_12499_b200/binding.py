@@ -299,6 +299,12 @@ def bn_relu_forward(dtype, rows, c, z, gamma, beta, relu, y, stats, scratch, str
                                       C.c_int(relu), _dev(y), _dev(stats), _dev(scratch), _stream(stream)))
 
 
+def bn_relu_forward_noalloc(dtype, rows, c, z, gamma, beta, relu, y, stats, stream=None):
+    """ckpt_bn_relu_forward_noalloc: same arguments as bn_relu_forward minus the scratch buffer."""
+    _check(lib().ckpt_bn_relu_forward_noalloc(C.c_int(dtype), C.c_int64(rows), C.c_int32(c), _dev(z), _dev(gamma), _dev(beta),
+                                              C.c_int(relu), _dev(y), _dev(stats), _stream(stream)))
+
+
 def bn_relu_backward(dtype, rows, c, dy, z, gamma, stats, relu, dz, dgamma, dbeta, scratch, stream=None):
     _check(lib().ckpt_bn_relu_backward(C.c_int(dtype), C.c_int64(rows), C.c_int32(c), _dev(dy), _dev(z), _dev(gamma),
                                        _dev(stats), C.c_int(relu), _dev(dz), _dev(dgamma), _dev(dbeta), _dev(scratch),
