@@ -1,9 +1,625 @@
-// Tensor-core implicit-GEMM convolution (placeholder until the tcgen05 kernels land).
+// Tensor-core implicit-GEMM convolution for sm_100a: tcgen05.mma with the accumulator in tensor
+// memory, operands staged in shared memory by TMA (cp.async.bulk.tensor) with the 128-byte swizzle,
+// bf16 operands, f32 accumulation.
+//
+//   forward : D[pixel][c_out] = sum over taps (r,s) and 64-channel blocks of
+//             X[pixel shifted by (r,s)][c_in block] * W[c_out][(r,s)][c_in block]^T
+//             A = one TMA box of the NHWC input per (tap, block): 128 pixels x 64 channels; the
+//             hardware zero-fills coordinates outside the image, which is the padding.
+//             B = one TMA box of the [c_out][k*k*c_in] matrix.  Both operands K-major.
+//   dgrad   : the same kernel on dz with the matrix transposed and the taps reversed (stride 1).
+//   wgrad   : D[c_out][(tap, c_in)] = sum over pixels of dz[pixel][c_out] * x[pixel shifted][c_in]
+//             Both operands are pixel-major in memory, i.e. MN-major for the tensor core; the
+//             pixel range is split over CTAs and the partial results are added in a fixed order.
+//
+// One CTA = 6 warps: warp 0 issues TMA, warp 1 owns tensor memory and issues the MMAs, warps 2-5
+// read the accumulator back and store it.  Every wait on an mbarrier is bounded: when it gives
+// up it records a code in the status word, the CTA drains its outstanding copies (bounded too),
+// frees its tensor memory and returns.
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include <algorithm>
+#include <cstring>
+
 #include "internal.h"
+
 namespace ckpt {
-bool tc_conv_supported(int, const ConvGeom&) { return false; }
-int64_t tc_conv_scratch_bytes(const ConvGeom&) { return 0; }
-int tc_conv_fwd(const ConvGeom&, const void*, const void*, void*, void*, int64_t, int*, void*) { set_error("no tensor-core kernel"); return CKPT_E_UNSUPPORTED; }
-int tc_conv_dgrad(const ConvGeom&, const void*, const void*, void*, void*, int64_t, int*, void*) { set_error("no tensor-core kernel"); return CKPT_E_UNSUPPORTED; }
-int tc_conv_wgrad(const ConvGeom&, const void*, const void*, float*, void*, int64_t, int*, void*) { set_error("no tensor-core kernel"); return CKPT_E_UNSUPPORTED; }
+
+#define CKPT_LAUNCH_CHECK(what)                                   \
+    do {                                                          \
+        ++g_launches;                                             \
+        cudaError_t e__ = cudaGetLastError();                     \
+        if (e__ != cudaSuccess) return cuda_fail(e__, what);      \
+    } while (0)
+
+namespace {
+
+constexpr int kThreads = 192;
+constexpr int kMaxStages = 8;
+constexpr uint32_t kSmemBudget = 200 * 1024;          // operand stages; barriers live behind them
+constexpr long long kWaitCycles = 4000000000LL;       // ~2 s at 2 GHz: far beyond any legitimate wait
+constexpr long long kDrainCycles = 200000000LL;
+
+// ------------------------------------------------------------------------------------------------
+// PTX wrappers
+// ------------------------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
 }
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+// Bounded wait.  `failed` is a CTA-wide flag in shared memory: once any role gave up, every other
+// wait returns at once so that the whole CTA reaches its tear-down.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* failed, int* status, int code,
+                                          long long limit = kWaitCycles) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    while (true) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if (*failed) return false;
+        if (clock64() - t0 > limit) {
+            *failed = 1;
+            atomicCAS(status, 0, code);
+            return false;
+        }
+    }
+}
+// After a failure: give copies that are still in flight a bounded time to land.
+__device__ __forceinline__ void mbar_drain(uint32_t bar, uint32_t parity) {
+    const long long t0 = clock64();
+    while (!mbar_try_wait(bar, parity) && clock64() - t0 < kDrainCycles) {}
+}
+__device__ __forceinline__ void fence_barrier_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
+__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2, int c3) {
+    asm volatile(
+        "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+        ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+        ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1) : "memory");
+}
+__device__ __forceinline__ void tma_prefetch_desc(const CUtensorMap* map) {
+    asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
+}
+
+__device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t cols) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(cols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t cols) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+// The mbarrier is signalled once every MMA issued so far by this thread has completed.
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+// 32 lanes x 32 consecutive columns: thread t of the warp receives lane (base lane + t).
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr) : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+// Shared-memory matrix descriptor, 128-byte swizzle.  Rows of 128 bytes; 8-row groups of 1024 bytes
+// `sbo` bytes apart.  K-major operands ignore `lbo`; MN-major operands use it as the distance
+// between consecutive 64-element blocks along M/N.
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo, uint32_t sbo) {
+    uint64_t d = 0;
+    d |= (uint64_t)((addr >> 4) & 0x3FFF);
+    d |= (uint64_t)((lbo >> 4) & 0x3FFF) << 16;
+    d |= (uint64_t)((sbo >> 4) & 0x3FFF) << 32;
+    d |= (uint64_t)1 << 46;     // descriptor version of this architecture
+    d |= (uint64_t)2 << 61;     // 128-byte swizzle
+    return d;
+}
+// Instruction descriptor: f32 accumulator, bf16 A and B, M x N tile, operand majors (0 = K, 1 = MN).
+__host__ __device__ inline uint32_t instr_desc(int M, int N, int a_mn_major, int b_mn_major) {
+    uint32_t d = 0;
+    d |= 1u << 4;                       // accumulator format: f32
+    d |= 1u << 7;                       // A format: bf16
+    d |= 1u << 10;                      // B format: bf16
+    d |= (uint32_t)a_mn_major << 15;
+    d |= (uint32_t)b_mn_major << 16;
+    d |= (uint32_t)(N >> 3) << 17;
+    d |= (uint32_t)(M >> 4) << 24;
+    return d;
+}
+
+// ------------------------------------------------------------------------------------------------
+// Forward / dgrad kernel
+// ------------------------------------------------------------------------------------------------
+struct FwdParams {
+    int H, W, N;                 // spatial size (same for input and output: stride 1) and batch
+    int c_red, c_out;            // reduction channels (multiple of 64) and output channels
+    int k, pad;                  // filter size and padding
+    int tw, th, tn;              // pixel tile, tw*th*tn = 128
+    int tiles_w, tiles_h, tiles_n;
+    int bn, n_tiles;             // output-channel tile and their count
+    int stages;
+};
+
+__global__ void __launch_bounds__(kThreads, 1)
+tc_conv_fwd_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w,
+                   __nv_bfloat16* __restrict__ out, FwdParams p, int* status) {
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    const uint32_t a_bytes = 128 * 128, b_bytes = (uint32_t)p.bn * 128, stage_bytes = a_bytes + b_bytes;
+    const uint32_t bars = base + (uint32_t)p.stages * stage_bytes;           // full[s], empty[s], accum
+    __shared__ uint32_t tmem_base_slot;
+    __shared__ int failed_flag;
+    volatile int* failed = &failed_flag;
+
+    const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
+    const int n_tile = blockIdx.x % p.n_tiles;
+    int mt = blockIdx.x / p.n_tiles;
+    const int tile_w = mt % p.tiles_w; mt /= p.tiles_w;
+    const int tile_h = mt % p.tiles_h;
+    const int tile_n = mt / p.tiles_h;
+    const int w0 = tile_w * p.tw, h0 = tile_h * p.th, n0 = tile_n * p.tn;
+    const int blocks = p.c_red / 64;
+    const int iters = p.k * p.k * blocks;
+    const uint32_t tmem_cols = p.bn < 32 ? 32 : p.bn;
+
+    auto full_bar = [&](int s) { return bars + 8u * s; };
+    auto empty_bar = [&](int s) { return bars + 8u * (kMaxStages + s); };
+    const uint32_t accum_bar = bars + 8u * (2 * kMaxStages);
+
+    if (threadIdx.x == 0) {
+        failed_flag = 0;
+        for (int s = 0; s < p.stages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+        mbar_init(accum_bar, 1);
+        fence_barrier_init();
+        tma_prefetch_desc(&map_x);
+        tma_prefetch_desc(&map_w);
+    }
+    if (warp == 1) tmem_alloc(smem_u32(&tmem_base_slot), tmem_cols);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = tmem_base_slot;
+
+    if (warp == 0 && lane == 0) {
+        // ---------------- TMA producer
+        int issued = 0;
+        for (int it = 0; it < iters; ++it) {
+            const int s = it % p.stages;
+            const uint32_t phase = (uint32_t)(it / p.stages) & 1u;
+            if (!mbar_wait(empty_bar(s), phase ^ 1u, failed, status, 101)) break;
+            const int tap = it / blocks, blk = it % blocks;
+            const int r = tap / p.k, q = tap % p.k;
+            mbar_expect_tx(full_bar(s), stage_bytes);
+            const uint32_t a_dst = base + (uint32_t)s * stage_bytes;
+            tma_load_4d(a_dst, &map_x, full_bar(s), blk * 64, w0 + q - p.pad, h0 + r - p.pad, n0);
+            tma_load_2d(a_dst + a_bytes, &map_w, full_bar(s), tap * p.c_red + blk * 64, n_tile * p.bn);
+            issued = it + 1;
+        }
+        if (*failed) {
+            // copies that were issued but never consumed must land before the CTA may exit
+            for (int it = max(0, issued - p.stages); it < issued; ++it)
+                mbar_drain(full_bar(it % p.stages), (uint32_t)(it / p.stages) & 1u);
+        }
+    } else if (warp == 1 && lane == 0) {
+        // ---------------- MMA issuer
+        const uint32_t idesc = instr_desc(128, p.bn, 0, 0);
+        bool ok = true;
+        for (int it = 0; it < iters && ok; ++it) {
+            const int s = it % p.stages;
+            const uint32_t phase = (uint32_t)(it / p.stages) & 1u;
+            if (!mbar_wait(full_bar(s), phase, failed, status, 102)) { ok = false; break; }
+            tc_fence_after();
+            const uint32_t a_addr = base + (uint32_t)s * stage_bytes;
+            const uint32_t b_addr = a_addr + a_bytes;
+#pragma unroll
+            for (int kk = 0; kk < 4; ++kk) {        // 4 x (K = 16 bf16 = 32 bytes) per 64-channel block
+                umma_bf16(tmem_base, smem_desc(a_addr + kk * 32, 0, 1024), smem_desc(b_addr + kk * 32, 0, 1024), idesc,
+                          (it > 0 || kk > 0) ? 1u : 0u);
+            }
+            umma_commit(empty_bar(s));              // frees the stage when these MMAs have read it
+        }
+        if (ok) umma_commit(accum_bar);             // accumulator complete
+    } else if (warp >= 2) {
+        // ---------------- epilogue: TMEM -> registers -> bf16 -> global
+        const int quarter = warp % 4;               // a warp may only touch its own 32 TMEM lanes
+        const int row = quarter * 32 + lane;
+        const int wl = row % p.tw, hl = (row / p.tw) % p.th, nl = row / (p.tw * p.th);
+        const bool valid = (w0 + wl < p.W) && (h0 + hl < p.H) && (n0 + nl < p.N);
+        __nv_bfloat16* dst = out + ((((size_t)(n0 + nl) * p.H + (h0 + hl)) * p.W + (w0 + wl)) * p.c_out + (size_t)n_tile * p.bn);
+        if (mbar_wait(accum_bar, 0, failed, status, 103)) {
+            tc_fence_after();
+            for (int c0 = 0; c0 < p.bn; c0 += 32) {
+                uint32_t v[32];
+                tmem_ld32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)c0, v);
+                if (valid) {
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        uint4 pk;
+                        __nv_bfloat162* h = reinterpret_cast<__nv_bfloat162*>(&pk);
+#pragma unroll
+                        for (int e = 0; e < 4; ++e)
+                            h[e] = __floats2bfloat162_rn(__uint_as_float(v[8 * j + 2 * e]), __uint_as_float(v[8 * j + 2 * e + 1]));
+                        *reinterpret_cast<uint4*>(dst + c0 + 8 * j) = pk;
+                    }
+                }
+            }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        __syncwarp();
+        tc_fence_after();
+        tmem_dealloc(tmem_base, tmem_cols);
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// wgrad kernel: D[c_out tile of 128][up to 4 blocks of 64 (tap, c_in) columns], K = pixels
+// ------------------------------------------------------------------------------------------------
+struct WgradParams {
+    int H, W, N;
+    int c_out, c_in;
+    int k, pad;
+    int tw, th, tn;              // pixel tile, tw*th*tn = 64
+    int tiles_w, tiles_h, tiles_n;
+    int nb;                      // column blocks per CTA (1..4)
+    int total_blocks;            // k*k*c_in/64
+    int tiles_per_slice;         // pixel tiles per CTA along the reduction
+    int total_tiles;
+    int stages;
+};
+
+__global__ void __launch_bounds__(kThreads, 1)
+tc_conv_wgrad_kernel(const __grid_constant__ CUtensorMap map_dz, const __grid_constant__ CUtensorMap map_x,
+                     float* __restrict__ partial, WgradParams p, int* status) {
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    constexpr uint32_t box_bytes = 64 * 128;                      // 64 pixels x 64 channels
+    const uint32_t stage_bytes = (2 + (uint32_t)p.nb) * box_bytes;
+    const uint32_t bars = base + (uint32_t)p.stages * stage_bytes;
+    __shared__ uint32_t tmem_base_slot;
+    __shared__ int failed_flag;
+    volatile int* failed = &failed_flag;
+
+    const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
+    const int slice = blockIdx.x, group = blockIdx.y, co_tile = blockIdx.z;
+    const int blk_begin = group * p.nb;
+    const int nb_here = min(p.nb, p.total_blocks - blk_begin);
+    const int cin_blocks = p.c_in / 64;
+    const int tile_begin = slice * p.tiles_per_slice;
+    const int tile_end = min(p.total_tiles, tile_begin + p.tiles_per_slice);
+    const int iters = tile_end - tile_begin;
+    const uint32_t n_cols = (uint32_t)nb_here * 64;
+    const uint32_t tmem_cols = n_cols <= 64 ? 64 : (n_cols <= 128 ? 128 : 256);
+
+    auto full_bar = [&](int s) { return bars + 8u * s; };
+    auto empty_bar = [&](int s) { return bars + 8u * (kMaxStages + s); };
+    const uint32_t accum_bar = bars + 8u * (2 * kMaxStages);
+
+    if (threadIdx.x == 0) {
+        failed_flag = 0;
+        for (int s = 0; s < p.stages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+        mbar_init(accum_bar, 1);
+        fence_barrier_init();
+        tma_prefetch_desc(&map_dz);
+        tma_prefetch_desc(&map_x);
+    }
+    if (warp == 1) tmem_alloc(smem_u32(&tmem_base_slot), tmem_cols);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = tmem_base_slot;
+
+    if (warp == 0 && lane == 0) {
+        int issued = 0;
+        for (int it = 0; it < iters; ++it) {
+            const int s = it % p.stages;
+            const uint32_t phase = (uint32_t)(it / p.stages) & 1u;
+            if (!mbar_wait(empty_bar(s), phase ^ 1u, failed, status, 201)) break;
+            int t = tile_begin + it;
+            const int w0 = (t % p.tiles_w) * p.tw; t /= p.tiles_w;
+            const int h0 = (t % p.tiles_h) * p.th;
+            const int n0 = (t / p.tiles_h) * p.tn;
+            mbar_expect_tx(full_bar(s), (2 + (uint32_t)nb_here) * box_bytes);
+            const uint32_t dst = base + (uint32_t)s * stage_bytes;
+            tma_load_4d(dst, &map_dz, full_bar(s), co_tile * 128, w0, h0, n0);
+            tma_load_4d(dst + box_bytes, &map_dz, full_bar(s), co_tile * 128 + 64, w0, h0, n0);
+            for (int j = 0; j < nb_here; ++j) {
+                const int b = blk_begin + j, tap = b / cin_blocks, cib = b % cin_blocks;
+                tma_load_4d(dst + (2 + j) * box_bytes, &map_x, full_bar(s), cib * 64, w0 + tap % p.k - p.pad, h0 + tap / p.k - p.pad, n0);
+            }
+            issued = it + 1;
+        }
+        if (*failed) {
+            for (int it = max(0, issued - p.stages); it < issued; ++it)
+                mbar_drain(full_bar(it % p.stages), (uint32_t)(it / p.stages) & 1u);
+        }
+    } else if (warp == 1 && lane == 0) {
+        const uint32_t idesc = instr_desc(128, (int)n_cols, 1, 1);
+        bool ok = true;
+        for (int it = 0; it < iters && ok; ++it) {
+            const int s = it % p.stages;
+            const uint32_t phase = (uint32_t)(it / p.stages) & 1u;
+            if (!mbar_wait(full_bar(s), phase, failed, status, 202)) { ok = false; break; }
+            tc_fence_after();
+            const uint32_t a_addr = base + (uint32_t)s * stage_bytes;
+            const uint32_t b_addr = a_addr + 2 * box_bytes;
+#pragma unroll
+            for (int kk = 0; kk < 4; ++kk) {        // 4 x (K = 16 pixels = 2 groups of 8 rows = 2048 bytes)
+                umma_bf16(tmem_base, smem_desc(a_addr + kk * 2048, box_bytes, 1024), smem_desc(b_addr + kk * 2048, box_bytes, 1024),
+                          idesc, (it > 0 || kk > 0) ? 1u : 0u);
+            }
+            umma_commit(empty_bar(s));
+        }
+        if (ok) umma_commit(accum_bar);
+    } else if (warp >= 2) {
+        const int quarter = warp % 4;
+        const int co = co_tile * 128 + quarter * 32 + lane;
+        const bool valid = co < p.c_out;
+        const size_t row_elems = (size_t)p.k * p.k * p.c_in;
+        float* dst_row = partial + ((size_t)slice * p.c_out + (valid ? co : 0)) * row_elems;
+        if (iters > 0 && mbar_wait(accum_bar, 0, failed, status, 203)) {
+            tc_fence_after();
+            for (int j = 0; j < nb_here; ++j) {
+                float* dst = dst_row + (size_t)(blk_begin + j) * 64;     // column (tap, c_in) = block*64 + c
+                for (int c0 = 0; c0 < 64; c0 += 32) {
+                    uint32_t v[32];
+                    tmem_ld32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(j * 64 + c0), v);
+                    if (valid) {
+#pragma unroll
+                        for (int e = 0; e < 8; ++e)
+                            *reinterpret_cast<float4*>(dst + c0 + 4 * e) =
+                                make_float4(__uint_as_float(v[4 * e]), __uint_as_float(v[4 * e + 1]), __uint_as_float(v[4 * e + 2]), __uint_as_float(v[4 * e + 3]));
+                    }
+                }
+            }
+        } else if (iters == 0 && valid) {
+            for (int j = 0; j < nb_here; ++j)
+                for (int c = 0; c < 64; ++c) dst_row[(size_t)(blk_begin + j) * 64 + c] = 0.f;
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        __syncwarp();
+        tc_fence_after();
+        tmem_dealloc(tmem_base, tmem_cols);
+    }
+}
+
+// wt[ci][tap'][co] = w[co][taps-1-tap'][ci]: the matrix of the transposed convolution (stride 1).
+__global__ void transpose_flip_kernel(const __nv_bfloat16* __restrict__ w, __nv_bfloat16* __restrict__ wt, int c_out, int taps, int c_in) {
+    const int64_t total = (int64_t)c_out * taps * c_in;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+        const int co = (int)(i % c_out);
+        const int64_t t = i / c_out;
+        const int tap = (int)(t % taps), ci = (int)(t / taps);
+        wt[i] = w[((size_t)co * taps + (taps - 1 - tap)) * c_in + ci];
+    }
+}
+
+__global__ void slice_sum_tc_kernel(const float* __restrict__ partial, float* __restrict__ out, int64_t elems, int slices) {
+    int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (e >= elems) return;
+    float s = 0.f;
+    for (int z = 0; z < slices; ++z) s += partial[(size_t)z * elems + e];
+    out[e] = s;
+}
+
+// ------------------------------------------------------------------------------------------------
+// Host side
+// ------------------------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess && q == cudaDriverEntryPointSuccess)
+            fn = (EncodeTiledFn)p;
+    }
+    return fn;
+}
+
+// NHWC bf16 tensor as (C, W, H, N); box = 64 channels x tw x th x tn pixels, 128-byte swizzle.
+int make_act_map(CUtensorMap* map, const void* ptr, int N, int H, int W, int C, int tw, int th, int tn) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) { set_error("cuTensorMapEncodeTiled is not available from this driver"); return CKPT_E_CUDA; }
+    cuuint64_t dims[4] = {(cuuint64_t)C, (cuuint64_t)W, (cuuint64_t)H, (cuuint64_t)N};
+    cuuint64_t strides[3] = {(cuuint64_t)C * 2, (cuuint64_t)W * C * 2, (cuuint64_t)H * W * C * 2};
+    cuuint32_t box[4] = {64, (cuuint32_t)tw, (cuuint32_t)th, (cuuint32_t)tn};
+    cuuint32_t es[4] = {1, 1, 1, 1};
+    CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(ptr), dims, strides, box, es,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) { set_error("cuTensorMapEncodeTiled failed for an activation tensor (code %d)", (int)r); return CKPT_E_CUDA; }
+    return CKPT_OK;
+}
+
+// Row-major [rows][cols] bf16 matrix as (cols, rows); box = 64 columns x box_rows.
+int make_mat_map(CUtensorMap* map, const void* ptr, int64_t rows, int64_t cols, int box_rows) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) { set_error("cuTensorMapEncodeTiled is not available from this driver"); return CKPT_E_CUDA; }
+    cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+    cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
+    cuuint32_t box[2] = {64, (cuuint32_t)box_rows};
+    cuuint32_t es[2] = {1, 1};
+    CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, es,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) { set_error("cuTensorMapEncodeTiled failed for a weight matrix (code %d)", (int)r); return CKPT_E_CUDA; }
+    return CKPT_OK;
+}
+
+// Pixel tile of `pixels` = tw*th*tn (powers of two) that wastes the fewest padded pixels.
+void choose_tile(int pixels, int W, int H, int N, int* tw, int* th, int* tn) {
+    double best = 1e30;
+    for (int a = pixels; a >= 1; a /= 2) {
+        for (int b = pixels / a; b >= 1; b /= 2) {
+            const int c = pixels / (a * b);
+            const double padded = (double)((W + a - 1) / a * a) * ((H + b - 1) / b * b) * ((N + c - 1) / c * c);
+            if (padded < best) { best = padded; *tw = a; *th = b; *tn = c; }   // ties: widest, then tallest
+        }
+    }
+}
+
+int pick_bn(int c_out) { return c_out % 256 == 0 ? 256 : (c_out % 128 == 0 ? 128 : 64); }
+
+int launch_fwd_like(const void* x, const void* w_mat, void* out, int N, int H, int W, int c_red, int c_out, int k, int pad,
+                    int* status, cudaStream_t st, const char* what) {
+    FwdParams p;
+    p.H = H; p.W = W; p.N = N; p.c_red = c_red; p.c_out = c_out; p.k = k; p.pad = pad;
+    choose_tile(128, W, H, N, &p.tw, &p.th, &p.tn);
+    p.tiles_w = (W + p.tw - 1) / p.tw; p.tiles_h = (H + p.th - 1) / p.th; p.tiles_n = (N + p.tn - 1) / p.tn;
+    p.bn = pick_bn(c_out);
+    p.n_tiles = c_out / p.bn;
+    const uint32_t stage_bytes = 128 * 128 + p.bn * 128;
+    p.stages = std::min<int>(kMaxStages, kSmemBudget / stage_bytes);
+    CUtensorMap mx, mw;
+    int rc = make_act_map(&mx, x, N, H, W, c_red, p.tw, p.th, p.tn);
+    if (rc) return rc;
+    rc = make_mat_map(&mw, w_mat, c_out, (int64_t)k * k * c_red, p.bn);
+    if (rc) return rc;
+    const size_t smem = (size_t)p.stages * stage_bytes + 1024 + 256;
+    static bool attr_set = false;
+    if (!attr_set) {
+        cudaError_t e = cudaFuncSetAttribute(tc_conv_fwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget + 2048);
+        if (e != cudaSuccess) return cuda_fail(e, "raising the shared-memory limit");
+        attr_set = true;
+    }
+    const int64_t ctas = (int64_t)p.tiles_w * p.tiles_h * p.tiles_n * p.n_tiles;
+    tc_conv_fwd_kernel<<<(unsigned)ctas, kThreads, smem, st>>>(mx, mw, (__nv_bfloat16*)out, p, status);
+    CKPT_LAUNCH_CHECK(what);
+    return CKPT_OK;
+}
+
+void wgrad_plan(const ConvGeom& g, WgradParams* p, int* slices, int* groups, int* co_tiles) {
+    p->H = g.h; p->W = g.w; p->N = g.n; p->c_out = g.cout; p->c_in = g.cin; p->k = g.k; p->pad = g.pad;
+    choose_tile(64, g.w, g.h, g.n, &p->tw, &p->th, &p->tn);
+    p->tiles_w = (g.w + p->tw - 1) / p->tw; p->tiles_h = (g.h + p->th - 1) / p->th; p->tiles_n = (g.n + p->tn - 1) / p->tn;
+    p->total_tiles = p->tiles_w * p->tiles_h * p->tiles_n;
+    p->total_blocks = g.k * g.k * g.cin / 64;
+    // column blocks per CTA: 4 when that divides evenly or the remainder is small, else 3
+    p->nb = p->total_blocks % 4 == 0 ? 4 : (p->total_blocks % 3 == 0 ? 3 : (p->total_blocks >= 4 ? 4 : p->total_blocks));
+    *groups = (p->total_blocks + p->nb - 1) / p->nb;
+    *co_tiles = (g.cout + 127) / 128;
+    const int64_t base_ctas = (int64_t)*groups * *co_tiles;
+    int64_t want = std::max<int64_t>(1, (148 * 3 + base_ctas - 1) / base_ctas);
+    int64_t by_k = std::max<int64_t>(1, p->total_tiles / 8);          // at least 8 pixel tiles per slice
+    int64_t s = std::min<int64_t>(std::min<int64_t>(want, by_k), 256);
+    p->tiles_per_slice = (int)((p->total_tiles + s - 1) / s);
+    *slices = (p->total_tiles + p->tiles_per_slice - 1) / p->tiles_per_slice;
+    const uint32_t stage_bytes = (2 + p->nb) * 64 * 128;
+    p->stages = std::min<int>(kMaxStages, kSmemBudget / stage_bytes);
+}
+
+}  // namespace
+
+bool tc_conv_supported(int dtype, const ConvGeom& g) {
+    if (dtype != CKPT_DTYPE_BF16) return false;
+    if (g.stride != 1) return false;
+    if (!((g.k == 3 && g.pad == 1) || (g.k == 1 && g.pad == 0))) return false;
+    if (g.cin % 64 || g.cout % 64) return false;
+    if (g.ho != g.h || g.wo != g.w) return false;
+    return true;
+}
+
+int64_t tc_conv_scratch_bytes(const ConvGeom& g) {
+    WgradParams p;
+    int slices, groups, co_tiles;
+    wgrad_plan(g, &p, &slices, &groups, &co_tiles);
+    const int64_t elems = (int64_t)g.cout * g.k * g.k * g.cin;
+    const int64_t partial = slices > 1 ? (int64_t)slices * elems * 4 : 0;
+    return std::max<int64_t>(partial, elems * 2);
+}
+
+int tc_conv_fwd(const ConvGeom& g, const void* x, const void* w, void* z, void*, int64_t, int* device_status, void* stream) {
+    if (!device_status) { set_error("no status word"); return CKPT_E_NULL; }
+    return launch_fwd_like(x, w, z, g.n, g.h, g.w, g.cin, g.cout, g.k, g.pad, device_status, (cudaStream_t)stream,
+                           "conv forward (tensor cores)");
+}
+
+int tc_conv_dgrad(const ConvGeom& g, const void* dz, const void* w, void* dx, void* scratch, int64_t scratch_bytes,
+                  int* device_status, void* stream) {
+    if (!device_status) { set_error("no status word"); return CKPT_E_NULL; }
+    const int taps = g.k * g.k;
+    const int64_t elems = (int64_t)g.cout * taps * g.cin;
+    if (!scratch || scratch_bytes < elems * 2) { set_error("dgrad scratch too small"); return CKPT_E_WORKSPACE; }
+    cudaStream_t st = (cudaStream_t)stream;
+    const unsigned grid = (unsigned)std::min<int64_t>((elems + 255) / 256, 148 * 8);
+    transpose_flip_kernel<<<grid, 256, 0, st>>>((const __nv_bfloat16*)w, (__nv_bfloat16*)scratch, g.cout, taps, g.cin);
+    CKPT_LAUNCH_CHECK("dgrad matrix transpose");
+    return launch_fwd_like(dz, scratch, dx, g.n, g.h, g.w, g.cout, g.cin, g.k, g.k - 1 - g.pad, device_status, st,
+                           "conv dgrad (tensor cores)");
+}
+
+int tc_conv_wgrad(const ConvGeom& g, const void* dz, const void* x, float* dw, void* scratch, int64_t scratch_bytes,
+                  int* device_status, void* stream) {
+    if (!device_status) { set_error("no status word"); return CKPT_E_NULL; }
+    WgradParams p;
+    int slices, groups, co_tiles;
+    wgrad_plan(g, &p, &slices, &groups, &co_tiles);
+    const int64_t elems = (int64_t)g.cout * g.k * g.k * g.cin;
+    if (slices > 1 && (!scratch || scratch_bytes < (int64_t)slices * elems * 4)) { set_error("wgrad scratch too small"); return CKPT_E_WORKSPACE; }
+    CUtensorMap mdz, mx;
+    int rc = make_act_map(&mdz, dz, g.n, g.h, g.w, g.cout, p.tw, p.th, p.tn);
+    if (rc) return rc;
+    rc = make_act_map(&mx, x, g.n, g.h, g.w, g.cin, p.tw, p.th, p.tn);
+    if (rc) return rc;
+    cudaStream_t st = (cudaStream_t)stream;
+    static bool attr_set = false;
+    if (!attr_set) {
+        cudaError_t e = cudaFuncSetAttribute(tc_conv_wgrad_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget + 2048);
+        if (e != cudaSuccess) return cuda_fail(e, "raising the shared-memory limit");
+        attr_set = true;
+    }
+    const size_t smem = (size_t)p.stages * (2 + p.nb) * 64 * 128 + 1024 + 256;
+    float* target = slices > 1 ? (float*)scratch : dw;
+    dim3 grid(slices, groups, co_tiles);
+    tc_conv_wgrad_kernel<<<grid, kThreads, smem, st>>>(mdz, mx, target, p, device_status);
+    CKPT_LAUNCH_CHECK("conv wgrad (tensor cores)");
+    if (slices > 1) {
+        slice_sum_tc_kernel<<<(unsigned)((elems + 255) / 256), 256, 0, st>>>((const float*)scratch, dw, elems, slices);
+        CKPT_LAUNCH_CHECK("wgrad slice sum");
+    }
+    return CKPT_OK;
+}
+
+}  // namespace ckpt

@@ -31,6 +31,19 @@ CONV_CASES = [
 ]
 
 
+TC_CASES = [
+    # n, h, w, cin, cout, k, pad: shapes served by the tensor-core kernels (stride 1, channels % 64 == 0)
+    (2, 16, 16, 64, 64, 3, 1),       # one pixel tile per image pair
+    (3, 13, 19, 64, 128, 3, 1),      # ragged in every spatial dimension and in the batch
+    (4, 28, 28, 128, 256, 3, 1),     # two channel blocks, 256-wide output tile
+    (2, 14, 14, 192, 64, 3, 1),      # three channel blocks
+    (8, 7, 7, 64, 320, 1, 0),        # 1x1, output channels not a multiple of 128
+    (5, 30, 30, 128, 64, 1, 0),
+    (64, 1, 1, 512, 192, 1, 0),      # fully connected shape
+    (2, 56, 56, 64, 64, 3, 1),
+]
+
+
 def rounded(a, dtype):
     a = a.astype(np.float32)
     return wl.to_bf16_representable(a) if dtype == ck.DTYPE_BF16 else a
@@ -63,6 +76,44 @@ def test_conv_cuda_core_kernels(case, dtype):
     assert max_rel_err(to_host(dx), dx_ref) <= TIGHT[dtype]
     assert max_rel_err(to_host(dw), dw_ref) <= 2e-5        # gradients are float32 in both modes
     assert TIGHT[dtype] <= TOL[dtype]
+
+
+@pytest.mark.parametrize("case", TC_CASES)
+def test_conv_tensor_core_kernels(case):
+    """tcgen05 forward / dgrad / wgrad against the float64 oracle, and bit-reproducible."""
+    import torch
+    dtype = ck.DTYPE_BF16
+    n, h, w, cin, cout, k, pad = case
+    rng = np.random.default_rng(hash(case) % 2 ** 31)
+    x = rounded(rng.standard_normal((n, h, w, cin)), dtype)
+    wt = rounded(rng.standard_normal((cout, k, k, cin)) / np.sqrt(k * k * cin), dtype)
+    z_ref = no.conv2d_fwd(x.astype(np.float64), wt.astype(np.float64), 1, pad)
+    dz = rounded(rng.standard_normal(z_ref.shape), dtype)
+    dx_ref, dw_ref = no.conv2d_bwd(x.astype(np.float64), wt.astype(np.float64), dz.astype(np.float64), 1, pad)
+    shape = ck.ConvShape(n, h, w, cin, cout, k, 1, pad)
+    xd, wd, dzd = to_dev(x, dtype), to_dev(wt, dtype), to_dev(dz, dtype)
+    scratch = torch.empty(max(ck.conv2d_scratch_bytes(shape, dtype), 256), dtype=torch.uint8, device="cuda")
+    results = []
+    for rep in range(2):
+        z = torch.full(z_ref.shape, float("nan"), device="cuda").to(xd.dtype)
+        dx = torch.full(x.shape, float("nan"), device="cuda").to(xd.dtype)
+        dw = torch.full(wt.shape, float("nan"), device="cuda", dtype=torch.float32)
+        ck.conv2d_forward(shape, dtype, 2, xd, wd, z, scratch)
+        ck.conv2d_dgrad(shape, dtype, 2, dzd, wd, dx, scratch)
+        ck.conv2d_wgrad(shape, dtype, 2, dzd, xd, dw, scratch)
+        torch.cuda.synchronize()
+        results.append((z, dx, dw))
+    z, dx, dw = results[0]
+    assert max_rel_err(to_host(z), z_ref) <= TIGHT[dtype]
+    assert max_rel_err(to_host(dx), dx_ref) <= TIGHT[dtype]
+    assert max_rel_err(to_host(dw), dw_ref) <= 2e-5
+    for a, b in zip(results[0], results[1]):
+        assert torch.equal(a, b)
+    # and the CUDA-core kernels agree with them to rounding
+    z2 = torch.empty_like(z)
+    ck.conv2d_forward(shape, dtype, 1, xd, wd, z2, scratch)
+    torch.cuda.synchronize()
+    assert max_rel_err(to_host(z2), to_host(z)) <= TIGHT[dtype]
 
 
 @pytest.mark.parametrize("dtype", [ck.DTYPE_F32, ck.DTYPE_BF16])
