@@ -76,8 +76,8 @@ static const int64_t kGradId = 1000000007;   // arena id of the per-segment grad
 
 static int conv_forward_any(StepCtx& c, const ConvGeom& g, const void* x, const void* w, void* z,
                             const float* bias, int relu) {
-    if (!bias && use_tc(c.ch, g))
-        return tc_conv_fwd(g, x, w, z, c.ws + c.ch->off_scr, c.ch->scr_bytes, c.status(), c.stream);
+    if (use_tc(c.ch, g))
+        return tc_conv_fwd(g, x, w, z, bias, relu, c.ws + c.ch->off_scr, c.ch->scr_bytes, c.status(), c.stream);
     return simt_conv_fwd(c.ch->dtype, g, x, w, z, bias, relu, c.stream);
 }
 static int conv_dgrad_any(StepCtx& c, const ConvGeom& g, const void* dz, const void* w, void* dx) {

@@ -175,7 +175,7 @@ struct FwdParams {
 
 __global__ void __launch_bounds__(kThreads, 1)
 tc_conv_fwd_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w,
-                   __nv_bfloat16* __restrict__ out, FwdParams p, int* status) {
+                   __nv_bfloat16* __restrict__ out, const float* __restrict__ bias, int relu, FwdParams p, int* status) {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const uint32_t a_bytes = 128 * 128, b_bytes = (uint32_t)p.bn * 128, stage_bytes = a_bytes + b_bytes;
@@ -265,6 +265,14 @@ tc_conv_fwd_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_const
                 uint32_t v[32];
                 tmem_ld32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)c0, v);
                 if (valid) {
+                    if (bias) {
+#pragma unroll
+                        for (int e = 0; e < 32; ++e) v[e] = __float_as_uint(__uint_as_float(v[e]) + bias[n_tile * p.bn + c0 + e]);
+                    }
+                    if (relu) {
+#pragma unroll
+                        for (int e = 0; e < 32; ++e) v[e] = __float_as_uint(fmaxf(__uint_as_float(v[e]), 0.f));
+                    }
 #pragma unroll
                     for (int j = 0; j < 4; ++j) {
                         uint4 pk;
@@ -502,8 +510,8 @@ void choose_tile(int pixels, int W, int H, int N, int* tw, int* th, int* tn) {
 
 int pick_bn(int c_out) { return c_out % 256 == 0 ? 256 : (c_out % 128 == 0 ? 128 : 64); }
 
-int launch_fwd_like(const void* x, const void* w_mat, void* out, int N, int H, int W, int c_red, int c_out, int k, int pad,
-                    int* status, cudaStream_t st, const char* what) {
+int launch_fwd_like(const void* x, const void* w_mat, void* out, const float* bias, int relu, int N, int H, int W, int c_red,
+                    int c_out, int k, int pad, int* status, cudaStream_t st, const char* what) {
     FwdParams p;
     p.H = H; p.W = W; p.N = N; p.c_red = c_red; p.c_out = c_out; p.k = k; p.pad = pad;
     choose_tile(128, W, H, N, &p.tw, &p.th, &p.tn);
@@ -525,7 +533,7 @@ int launch_fwd_like(const void* x, const void* w_mat, void* out, int N, int H, i
         attr_set = true;
     }
     const int64_t ctas = (int64_t)p.tiles_w * p.tiles_h * p.tiles_n * p.n_tiles;
-    tc_conv_fwd_kernel<<<(unsigned)ctas, kThreads, smem, st>>>(mx, mw, (__nv_bfloat16*)out, p, status);
+    tc_conv_fwd_kernel<<<(unsigned)ctas, kThreads, smem, st>>>(mx, mw, (__nv_bfloat16*)out, bias, relu, p, status);
     CKPT_LAUNCH_CHECK(what);
     return CKPT_OK;
 }
@@ -570,9 +578,10 @@ int64_t tc_conv_scratch_bytes(const ConvGeom& g) {
     return std::max<int64_t>(partial, elems * 2);
 }
 
-int tc_conv_fwd(const ConvGeom& g, const void* x, const void* w, void* z, void*, int64_t, int* device_status, void* stream) {
+int tc_conv_fwd(const ConvGeom& g, const void* x, const void* w, void* z, const float* bias, int relu, void*, int64_t,
+                int* device_status, void* stream) {
     if (!device_status) { set_error("no status word"); return CKPT_E_NULL; }
-    return launch_fwd_like(x, w, z, g.n, g.h, g.w, g.cin, g.cout, g.k, g.pad, device_status, (cudaStream_t)stream,
+    return launch_fwd_like(x, w, z, bias, relu, g.n, g.h, g.w, g.cin, g.cout, g.k, g.pad, device_status, (cudaStream_t)stream,
                            "conv forward (tensor cores)");
 }
 
@@ -586,7 +595,7 @@ int tc_conv_dgrad(const ConvGeom& g, const void* dz, const void* w, void* dx, vo
     const unsigned grid = (unsigned)std::min<int64_t>((elems + 255) / 256, 148 * 8);
     transpose_flip_kernel<<<grid, 256, 0, st>>>((const __nv_bfloat16*)w, (__nv_bfloat16*)scratch, g.cout, taps, g.cin);
     CKPT_LAUNCH_CHECK("dgrad matrix transpose");
-    return launch_fwd_like(dz, scratch, dx, g.n, g.h, g.w, g.cout, g.cin, g.k, g.k - 1 - g.pad, device_status, st,
+    return launch_fwd_like(dz, scratch, dx, nullptr, 0, g.n, g.h, g.w, g.cout, g.cin, g.k, g.k - 1 - g.pad, device_status, st,
                            "conv dgrad (tensor cores)");
 }
 

@@ -68,8 +68,8 @@ int simt_conv_wgrad(int dtype, const ConvGeom& g, const void* dz, const void* x,
 // Tensor-core (tcgen05) implicit-GEMM kernels; *_supported tells whether the shape has one.
 bool tc_conv_supported(int dtype, const ConvGeom& g);
 int64_t tc_conv_scratch_bytes(const ConvGeom& g);
-int tc_conv_fwd(const ConvGeom& g, const void* x, const void* w, void* z, void* scratch,
-                int64_t scratch_bytes, int* device_status, void* stream);
+int tc_conv_fwd(const ConvGeom& g, const void* x, const void* w, void* z, const float* bias, int relu,
+                void* scratch, int64_t scratch_bytes, int* device_status, void* stream);
 int tc_conv_dgrad(const ConvGeom& g, const void* dz, const void* w, void* dx, void* scratch,
                   int64_t scratch_bytes, int* device_status, void* stream);
 int tc_conv_wgrad(const ConvGeom& g, const void* dz, const void* x, float* dw, void* scratch,

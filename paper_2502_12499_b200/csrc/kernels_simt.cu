@@ -240,6 +240,11 @@ int simt_conv_wgrad(int dtype, const ConvGeom& g, const void* dz, const void* x,
 // Each thread owns VEC consecutive channels (one 16-byte load when the channel count allows it) and
 // walks down the rows of its block's slab; partial sums are combined in a fixed order.
 // ================================================================================================
+static unsigned elementwise_grid(int64_t items) {
+    int64_t b = (items + 255) / 256;
+    return (unsigned)std::max<int64_t>(1, std::min<int64_t>(b, 148 * 16));
+}
+
 constexpr int BN_THREADS = 256;
 constexpr int BN_MAX_BLOCKS = 148 * 8;
 constexpr float BN_EPS = 1e-5f;
@@ -324,23 +329,33 @@ __global__ void __launch_bounds__(BN_THREADS) bn_partial_kernel(const T* __restr
 #pragma unroll
                 for (int i = 0; i < VEC; ++i) { mean[i] = stats[ch + i]; inv[i] = stats[c + ch + i]; sc[i] = stats[2 * c + ch + i]; sh[i] = stats[3 * c + ch + i]; }
             }
-            for (int64_t row = row_begin + r; row < row_end; row += rows_per_iter) {
-                float v[VEC];
-                load_vec<T, VEC>(z + row * c + ch, v);
-                if (WHAT == 0) {
+            // four rows in flight per thread; sums are still taken in row order
+            for (int64_t row = row_begin + r; row < row_end; row += 4 * (int64_t)rows_per_iter) {
+                float v[4][VEC], g[4][VEC];
 #pragma unroll
-                    for (int i = 0; i < VEC; ++i) { s0[i] += v[i]; s1[i] = fmaf(v[i], v[i], s1[i]); }
-                } else {
-                    float g[VEC];
-                    load_vec<T, VEC>(dy + row * c + ch, g);
+                for (int u = 0; u < 4; ++u) {
+                    const int64_t rr = row + (int64_t)u * rows_per_iter;
+                    if (rr < row_end) {
+                        load_vec<T, VEC>(z + rr * c + ch, v[u]);
+                        if (WHAT == 1) load_vec<T, VEC>(dy + rr * c + ch, g[u]);
+                    }
+                }
 #pragma unroll
-                    for (int i = 0; i < VEC; ++i) {
-                        float yv = fmaf(v[i], sc[i], sh[i]);
-                        bool pass = !relu || (float)cvt<T>(fmaxf(yv, 0.f)) > 0.f;
-                        float gi = pass ? g[i] : 0.f;
-                        float xh = (v[i] - mean[i]) * inv[i];
-                        s0[i] += gi;
-                        s1[i] = fmaf(gi, xh, s1[i]);
+                for (int u = 0; u < 4; ++u) {
+                    if (row + (int64_t)u * rows_per_iter >= row_end) break;
+                    if (WHAT == 0) {
+#pragma unroll
+                        for (int i = 0; i < VEC; ++i) { s0[i] += v[u][i]; s1[i] = fmaf(v[u][i], v[u][i], s1[i]); }
+                    } else {
+#pragma unroll
+                        for (int i = 0; i < VEC; ++i) {
+                            float yv = fmaf(v[u][i], sc[i], sh[i]);
+                            bool pass = !relu || (float)cvt<T>(fmaxf(yv, 0.f)) > 0.f;
+                            float gi = pass ? g[u][i] : 0.f;
+                            float xh = (v[u][i] - mean[i]) * inv[i];
+                            s0[i] += gi;
+                            s1[i] = fmaf(gi, xh, s1[i]);
+                        }
                     }
                 }
             }
@@ -367,13 +382,22 @@ __global__ void __launch_bounds__(BN_THREADS) bn_partial_kernel(const T* __restr
     }
 }
 
-// mean, 1/sqrt(var+eps), scale = gamma*inv, shift = beta - mean*scale
-__global__ void bn_finalize_fwd_kernel(const float* __restrict__ partial, int blocks, int c, double inv_rows,
+// Sum of the per-block partials of one channel by one warp: lane l adds blocks l, l+32, ... in order,
+// then the 32 lane sums are combined by a fixed butterfly.  Double precision throughout.
+__device__ __forceinline__ void warp_channel_sums(const float* __restrict__ partial, int blocks, int c, int ch, double& s, double& q) {
+    s = 0.0; q = 0.0;
+    for (int b = threadIdx.x; b < blocks; b += 32) { s += partial[((size_t)b * 2) * c + ch]; q += partial[((size_t)b * 2 + 1) * c + ch]; }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) { s += __shfl_xor_sync(0xffffffffu, s, o); q += __shfl_xor_sync(0xffffffffu, q, o); }
+}
+
+// mean, 1/sqrt(var+eps), scale = gamma*inv, shift = beta - mean*scale.  One warp per channel.
+__global__ void __launch_bounds__(32) bn_finalize_fwd_kernel(const float* __restrict__ partial, int blocks, int c, double inv_rows,
                                        const float* __restrict__ gamma, const float* __restrict__ beta, float* __restrict__ stats) {
-    int ch = blockIdx.x * blockDim.x + threadIdx.x;
-    if (ch >= c) return;
-    double s = 0.0, q = 0.0;
-    for (int b = 0; b < blocks; ++b) { s += partial[((size_t)b * 2) * c + ch]; q += partial[((size_t)b * 2 + 1) * c + ch]; }
+    const int ch = blockIdx.x;
+    double s, q;
+    warp_channel_sums(partial, blocks, c, ch, s, q);
+    if (threadIdx.x != 0) return;
     double mean = s * inv_rows;
     double var = q * inv_rows - mean * mean;
     if (var < 0.0) var = 0.0;
@@ -387,13 +411,13 @@ __global__ void bn_finalize_fwd_kernel(const float* __restrict__ partial, int bl
 
 // dbeta, dgamma and the two per-channel coefficients of the input gradient:
 //   dz = scale*g - k1 - xhat*k2,  k1 = scale*dbeta/rows, k2 = scale*dgamma/rows
-__global__ void bn_finalize_bwd_kernel(const float* __restrict__ partial, int blocks, int c, double inv_rows,
+__global__ void __launch_bounds__(32) bn_finalize_bwd_kernel(const float* __restrict__ partial, int blocks, int c, double inv_rows,
                                        const float* __restrict__ stats, float* __restrict__ dgamma, float* __restrict__ dbeta,
                                        float* __restrict__ coef) {
-    int ch = blockIdx.x * blockDim.x + threadIdx.x;
-    if (ch >= c) return;
-    double s = 0.0, q = 0.0;
-    for (int b = 0; b < blocks; ++b) { s += partial[((size_t)b * 2) * c + ch]; q += partial[((size_t)b * 2 + 1) * c + ch]; }
+    const int ch = blockIdx.x;
+    double s, q;
+    warp_channel_sums(partial, blocks, c, ch, s, q);
+    if (threadIdx.x != 0) return;
     dbeta[ch] = (float)s;
     dgamma[ch] = (float)q;
     double scale = stats[2 * c + ch];
@@ -401,10 +425,39 @@ __global__ void bn_finalize_bwd_kernel(const float* __restrict__ partial, int bl
     coef[c + ch] = (float)(scale * q * inv_rows);
 }
 
+// y = max(z*scale + shift, 0).  When the grid's thread count is a multiple of the number of channel
+// groups, every thread stays on one channel group: its coefficients live in registers and four
+// independent 16-byte loads are in flight per thread.
 template <typename T, int VEC>
 __global__ void __launch_bounds__(256) bn_apply_kernel(const T* __restrict__ z, const float* __restrict__ stats, int relu,
                                                        int64_t vecs, int lanes, int c, T* __restrict__ y) {
-    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < vecs; i += (int64_t)gridDim.x * blockDim.x) {
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    const int64_t first = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (stride % lanes == 0) {
+        const int ch = (int)(first % lanes) * VEC;
+        float sc[VEC], sh[VEC];
+#pragma unroll
+        for (int k = 0; k < VEC; ++k) { sc[k] = stats[2 * c + ch + k]; sh[k] = stats[3 * c + ch + k]; }
+        for (int64_t i = first; i < vecs; i += 4 * stride) {
+            float v[4][VEC];
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+                if (i + u * stride < vecs) load_vec<T, VEC>(z + (i + u * stride) * VEC, v[u]);
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                if (i + u * stride >= vecs) break;
+                float o[VEC];
+#pragma unroll
+                for (int k = 0; k < VEC; ++k) {
+                    float t = fmaf(v[u][k], sc[k], sh[k]);
+                    o[k] = relu ? fmaxf(t, 0.f) : t;
+                }
+                store_vec<T, VEC>(y + (i + u * stride) * VEC, o);
+            }
+        }
+        return;
+    }
+    for (int64_t i = first; i < vecs; i += stride) {
         const int ch = (int)(i % lanes) * VEC;
         float v[VEC], o[VEC];
         load_vec<T, VEC>(z + i * VEC, v);
@@ -418,30 +471,59 @@ __global__ void __launch_bounds__(256) bn_apply_kernel(const T* __restrict__ z, 
 }
 
 template <typename T, int VEC>
-__global__ void __launch_bounds__(256) bn_bwd_apply_kernel(const T* __restrict__ dy, const T* __restrict__ z,
-                                                           const float* __restrict__ stats, const float* __restrict__ coef,
-                                                           int relu, int64_t vecs, int lanes, int c, T* __restrict__ dz) {
-    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < vecs; i += (int64_t)gridDim.x * blockDim.x) {
-        const int ch = (int)(i % lanes) * VEC;
-        float v[VEC], g[VEC], o[VEC];
-        load_vec<T, VEC>(z + i * VEC, v);
-        load_vec<T, VEC>(dy + i * VEC, g);
+__device__ __forceinline__ void bn_bwd_point(const float (&v)[VEC], const float (&g)[VEC], const float (&mean)[VEC],
+                                             const float (&inv)[VEC], const float (&sc)[VEC], const float (&sh)[VEC],
+                                             const float (&k1)[VEC], const float (&k2)[VEC], int relu, float (&o)[VEC]) {
 #pragma unroll
-        for (int k = 0; k < VEC; ++k) {
-            float sc = stats[2 * c + ch + k];
-            float yv = fmaf(v[k], sc, stats[3 * c + ch + k]);
-            bool pass = !relu || (float)cvt<T>(fmaxf(yv, 0.f)) > 0.f;
-            float gi = pass ? g[k] : 0.f;
-            float xh = (v[k] - stats[ch + k]) * stats[c + ch + k];
-            o[k] = sc * gi - coef[ch + k] - xh * coef[c + ch + k];
-        }
-        store_vec<T, VEC>(dz + i * VEC, o);
+    for (int k = 0; k < VEC; ++k) {
+        float yv = fmaf(v[k], sc[k], sh[k]);
+        bool pass = !relu || (float)cvt<T>(fmaxf(yv, 0.f)) > 0.f;
+        float gi = pass ? g[k] : 0.f;
+        float xh = (v[k] - mean[k]) * inv[k];
+        o[k] = sc[k] * gi - k1[k] - xh * k2[k];
     }
 }
 
-static unsigned elementwise_grid(int64_t items) {
-    int64_t b = (items + 255) / 256;
-    return (unsigned)std::max<int64_t>(1, std::min<int64_t>(b, 148 * 16));
+template <typename T, int VEC>
+__global__ void __launch_bounds__(256) bn_bwd_apply_kernel(const T* __restrict__ dy, const T* __restrict__ z,
+                                                           const float* __restrict__ stats, const float* __restrict__ coef,
+                                                           int relu, int64_t vecs, int lanes, int c, T* __restrict__ dz) {
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    const int64_t first = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const bool fixed = stride % lanes == 0;
+    float mean[VEC], inv[VEC], sc[VEC], sh[VEC], k1[VEC], k2[VEC];
+    auto load_coef = [&](int ch) {
+#pragma unroll
+        for (int k = 0; k < VEC; ++k) {
+            mean[k] = stats[ch + k]; inv[k] = stats[c + ch + k]; sc[k] = stats[2 * c + ch + k]; sh[k] = stats[3 * c + ch + k];
+            k1[k] = coef[ch + k]; k2[k] = coef[c + ch + k];
+        }
+    };
+    if (fixed) {
+        load_coef((int)(first % lanes) * VEC);
+        for (int64_t i = first; i < vecs; i += 2 * stride) {
+            float v[2][VEC], g[2][VEC];
+#pragma unroll
+            for (int u = 0; u < 2; ++u)
+                if (i + u * stride < vecs) { load_vec<T, VEC>(z + (i + u * stride) * VEC, v[u]); load_vec<T, VEC>(dy + (i + u * stride) * VEC, g[u]); }
+#pragma unroll
+            for (int u = 0; u < 2; ++u) {
+                if (i + u * stride >= vecs) break;
+                float o[VEC];
+                bn_bwd_point<T, VEC>(v[u], g[u], mean, inv, sc, sh, k1, k2, relu, o);
+                store_vec<T, VEC>(dz + (i + u * stride) * VEC, o);
+            }
+        }
+        return;
+    }
+    for (int64_t i = first; i < vecs; i += stride) {
+        load_coef((int)(i % lanes) * VEC);
+        float v[VEC], g[VEC], o[VEC];
+        load_vec<T, VEC>(z + i * VEC, v);
+        load_vec<T, VEC>(dy + i * VEC, g);
+        bn_bwd_point<T, VEC>(v, g, mean, inv, sc, sh, k1, k2, relu, o);
+        store_vec<T, VEC>(dz + i * VEC, o);
+    }
 }
 
 template <typename T, int VEC>
@@ -453,7 +535,7 @@ static int bn_forward_t(int64_t rows, int c, const void* z, const float* gamma, 
     bn_partial_kernel<T, VEC, 0><<<L.blocks, BN_THREADS, smem, st>>>((const T*)z, nullptr, nullptr, 0, rows, c, L.lanes,
                                                                       L.rows_per_iter, L.rows_per_block, partial);
     CKPT_LAUNCH_CHECK("batch-norm statistics");
-    bn_finalize_fwd_kernel<<<(c + 127) / 128, 128, 0, st>>>(partial, L.blocks, c, 1.0 / (double)rows, gamma, beta, stats);
+    bn_finalize_fwd_kernel<<<c, 32, 0, st>>>(partial, L.blocks, c, 1.0 / (double)rows, gamma, beta, stats);
     CKPT_LAUNCH_CHECK("batch-norm finalize");
     int64_t vecs = rows * c / VEC;
     bn_apply_kernel<T, VEC><<<elementwise_grid(vecs), 256, 0, st>>>((const T*)z, stats, relu, vecs, L.lanes, c, (T*)y);
@@ -471,7 +553,7 @@ static int bn_backward_t(int64_t rows, int c, const void* dy, const void* z, con
     bn_partial_kernel<T, VEC, 1><<<L.blocks, BN_THREADS, smem, st>>>((const T*)z, (const T*)dy, stats, relu, rows, c, L.lanes,
                                                                       L.rows_per_iter, L.rows_per_block, partial);
     CKPT_LAUNCH_CHECK("batch-norm backward sums");
-    bn_finalize_bwd_kernel<<<(c + 127) / 128, 128, 0, st>>>(partial, L.blocks, c, 1.0 / (double)rows, stats, dgamma, dbeta, coef);
+    bn_finalize_bwd_kernel<<<c, 32, 0, st>>>(partial, L.blocks, c, 1.0 / (double)rows, stats, dgamma, dbeta, coef);
     CKPT_LAUNCH_CHECK("batch-norm backward finalize");
     int64_t vecs = rows * c / VEC;
     bn_bwd_apply_kernel<T, VEC><<<elementwise_grid(vecs), 256, 0, st>>>((const T*)dy, (const T*)z, stats, coef, relu, vecs,
@@ -568,8 +650,76 @@ __global__ void maxpool_bwd_kernel(const T* __restrict__ x, const T* __restrict_
     }
 }
 
+// 2x2 / stride 2 / no padding on even-sized images, VEC channels per thread (16-byte accesses):
+// the layout every pooling layer of the benchmark chains has.  One thread per output pixel group.
+template <typename T, int VEC>
+__global__ void __launch_bounds__(256) maxpool2x2_fwd_kernel(const T* __restrict__ x, T* __restrict__ y, int64_t items, int wo, int ho, int cv, int c) {
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < items; i += (int64_t)gridDim.x * blockDim.x) {
+        const int cg = (int)(i % cv);
+        int64_t t = i / cv;
+        const int ow = (int)(t % wo); t /= wo;
+        const int oh = (int)(t % ho);
+        const int64_t img = t / ho;
+        const T* p = x + (((img * (2 * ho) + 2 * oh) * (int64_t)(2 * wo) + 2 * ow) * c + cg * VEC);
+        float a[VEC], b[VEC], d[VEC], e[VEC], o[VEC];
+        load_vec<T, VEC>(p, a);
+        load_vec<T, VEC>(p + c, b);
+        load_vec<T, VEC>(p + (int64_t)2 * wo * c, d);
+        load_vec<T, VEC>(p + (int64_t)2 * wo * c + c, e);
+#pragma unroll
+        for (int k = 0; k < VEC; ++k) o[k] = fmaxf(fmaxf(a[k], b[k]), fmaxf(d[k], e[k]));
+        store_vec<T, VEC>(y + i * VEC, o);
+    }
+}
+
+// Backward of the same: the first maximum of the window in row-major order takes the gradient.
+template <typename T, int VEC>
+__global__ void __launch_bounds__(256) maxpool2x2_bwd_kernel(const T* __restrict__ x, const T* __restrict__ dy, T* __restrict__ dx,
+                                                             int64_t items, int wo, int ho, int cv, int c) {
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < items; i += (int64_t)gridDim.x * blockDim.x) {
+        const int cg = (int)(i % cv);
+        int64_t t = i / cv;
+        const int ow = (int)(t % wo); t /= wo;
+        const int oh = (int)(t % ho);
+        const int64_t img = t / ho;
+        const int64_t off = ((img * (2 * ho) + 2 * oh) * (int64_t)(2 * wo) + 2 * ow) * c + cg * VEC;
+        const int64_t down = (int64_t)2 * wo * c;
+        float a[VEC], b[VEC], d[VEC], e[VEC], g[VEC], oa[VEC], ob[VEC], od[VEC], oe[VEC];
+        load_vec<T, VEC>(x + off, a);
+        load_vec<T, VEC>(x + off + c, b);
+        load_vec<T, VEC>(x + off + down, d);
+        load_vec<T, VEC>(x + off + down + c, e);
+        load_vec<T, VEC>(dy + i * VEC, g);
+#pragma unroll
+        for (int k = 0; k < VEC; ++k) {
+            const float m = fmaxf(fmaxf(a[k], b[k]), fmaxf(d[k], e[k]));
+            const bool ta = a[k] == m, tb = !ta && b[k] == m, td = !ta && !tb && d[k] == m, te = !ta && !tb && !td;
+            oa[k] = ta ? g[k] : 0.f; ob[k] = tb ? g[k] : 0.f; od[k] = td ? g[k] : 0.f; oe[k] = te ? g[k] : 0.f;
+        }
+        store_vec<T, VEC>(dx + off, oa);
+        store_vec<T, VEC>(dx + off + c, ob);
+        store_vec<T, VEC>(dx + off + down, od);
+        store_vec<T, VEC>(dx + off + down + c, oe);
+    }
+}
+
+static bool pool_fast_path(int dtype, int h, int w, int c, int k, int stride, int pad) {
+    const int vec = dtype == CKPT_DTYPE_BF16 ? 8 : 4;
+    return k == 2 && stride == 2 && pad == 0 && h % 2 == 0 && w % 2 == 0 && c % vec == 0;
+}
+
 int maxpool_forward(int dtype, int n, int h, int w, int c, int k, int stride, int pad, const void* x, void* y, void* stream) {
     int ho = (h + 2 * pad - k) / stride + 1, wo = (w + 2 * pad - k) / stride + 1;
+    if (pool_fast_path(dtype, h, w, c, k, stride, pad)) {
+        const int vec = dtype == CKPT_DTYPE_BF16 ? 8 : 4;
+        const int64_t items = (int64_t)n * ho * wo * (c / vec);
+        if (dtype == CKPT_DTYPE_BF16)
+            maxpool2x2_fwd_kernel<__nv_bfloat16, 8><<<elementwise_grid(items), 256, 0, (cudaStream_t)stream>>>((const __nv_bfloat16*)x, (__nv_bfloat16*)y, items, wo, ho, c / vec, c);
+        else
+            maxpool2x2_fwd_kernel<float, 4><<<elementwise_grid(items), 256, 0, (cudaStream_t)stream>>>((const float*)x, (float*)y, items, wo, ho, c / vec, c);
+        CKPT_LAUNCH_CHECK("max-pool 2x2 forward");
+        return CKPT_OK;
+    }
     unsigned grid = elementwise_grid((int64_t)n * ho * wo * c);
     if (dtype == CKPT_DTYPE_BF16)
         maxpool_fwd_kernel<__nv_bfloat16><<<grid, 256, 0, (cudaStream_t)stream>>>((const __nv_bfloat16*)x, (__nv_bfloat16*)y, n, h, w, c, ho, wo, k, stride, pad);
@@ -581,6 +731,16 @@ int maxpool_forward(int dtype, int n, int h, int w, int c, int k, int stride, in
 
 int maxpool_backward(int dtype, int n, int h, int w, int c, int k, int stride, int pad, const void* x, const void* dy, void* dx, void* stream) {
     int ho = (h + 2 * pad - k) / stride + 1, wo = (w + 2 * pad - k) / stride + 1;
+    if (pool_fast_path(dtype, h, w, c, k, stride, pad)) {
+        const int vec = dtype == CKPT_DTYPE_BF16 ? 8 : 4;
+        const int64_t items = (int64_t)n * ho * wo * (c / vec);
+        if (dtype == CKPT_DTYPE_BF16)
+            maxpool2x2_bwd_kernel<__nv_bfloat16, 8><<<elementwise_grid(items), 256, 0, (cudaStream_t)stream>>>((const __nv_bfloat16*)x, (const __nv_bfloat16*)dy, (__nv_bfloat16*)dx, items, wo, ho, c / vec, c);
+        else
+            maxpool2x2_bwd_kernel<float, 4><<<elementwise_grid(items), 256, 0, (cudaStream_t)stream>>>((const float*)x, (const float*)dy, (float*)dx, items, wo, ho, c / vec, c);
+        CKPT_LAUNCH_CHECK("max-pool 2x2 backward");
+        return CKPT_OK;
+    }
     unsigned grid = elementwise_grid((int64_t)n * h * w * c);
     if (dtype == CKPT_DTYPE_BF16)
         maxpool_bwd_kernel<__nv_bfloat16><<<grid, 256, 0, (cudaStream_t)stream>>>((const __nv_bfloat16*)x, (const __nv_bfloat16*)dy, (__nv_bfloat16*)dx, n, h, w, c, ho, wo, k, stride, pad);

@@ -144,6 +144,9 @@ def shallow_chains():
     s = dict(units=[{"kind": "fc", "cin": 6 * 6 * 8, "cout": 40, "relu": True}, {"kind": "fc", "cin": 40, "cout": 12, "relu": False}],
              input_hwc=(6, 6, 8), batch=16, dtype="bf16", loss="softmax_ce", name="fc+fc")
     yield s
+    s = dict(units=[{"kind": "fc", "cin": 2 * 2 * 64, "cout": 128, "relu": True}, {"kind": "fc", "cin": 128, "cout": 64, "relu": False}],
+             input_hwc=(2, 2, 64), batch=24, dtype="bf16", loss="softmax_ce", name="fc+fc on tensor cores")
+    yield s
     s = wl.plain_chain(2, 64, 64, (12, 12), 8, "bf16", "softmax_ce", name="conv64+conv64+fc")
     s["units"].append({"kind": "fc", "cin": 12 * 12 * 64, "cout": 10, "relu": False})
     yield s
