@@ -7,7 +7,7 @@ from concurrent.futures import ThreadPoolExecutor
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libckpt_b200.so")
-SOURCES = ["planner.cpp", "arena.cpp", "chain.cu", "kernels_simt.cu", "conv_tc.cu", "capi.cu", "no_alloc.cu"]
+SOURCES = ["planner.cpp", "arena.cpp", "chain.cu", "kernels_simt.cu", "conv_tc.cu", "conv_small.cu", "capi.cu", "no_alloc.cu"]
 NVCC = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
 FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
          "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden", "-Xptxas", "-v"]

@@ -191,7 +191,7 @@ tc_conv_fwd_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_const
     const int tile_h = mt % p.tiles_h;
     const int tile_n = mt / p.tiles_h;
     const int w0 = tile_w * p.tw, h0 = tile_h * p.th, n0 = tile_n * p.tn;
-    const int blocks = p.c_red / 64;
+    const int blocks = (p.c_red + 63) / 64;      // a ragged last block is zero-filled by the TMA unit
     const int iters = p.k * p.k * blocks;
     const uint32_t tmem_cols = p.bn < 32 ? 32 : p.bn;
 
@@ -264,10 +264,12 @@ tc_conv_fwd_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_const
             for (int c0 = 0; c0 < p.bn; c0 += 32) {
                 uint32_t v[32];
                 tmem_ld32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)c0, v);
-                if (valid) {
+                const int col0 = n_tile * p.bn + c0;          // first output channel of this chunk
+                if (valid && col0 < p.c_out) {
                     if (bias) {
 #pragma unroll
-                        for (int e = 0; e < 32; ++e) v[e] = __float_as_uint(__uint_as_float(v[e]) + bias[n_tile * p.bn + c0 + e]);
+                        for (int e = 0; e < 32; ++e)
+                            if (col0 + e < p.c_out) v[e] = __float_as_uint(__uint_as_float(v[e]) + bias[col0 + e]);
                     }
                     if (relu) {
 #pragma unroll
@@ -280,7 +282,7 @@ tc_conv_fwd_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_const
 #pragma unroll
                         for (int e = 0; e < 4; ++e)
                             h[e] = __floats2bfloat162_rn(__uint_as_float(v[8 * j + 2 * e]), __uint_as_float(v[8 * j + 2 * e + 1]));
-                        *reinterpret_cast<uint4*>(dst + c0 + 8 * j) = pk;
+                        if (col0 + 8 * j + 8 <= p.c_out) *reinterpret_cast<uint4*>(dst + c0 + 8 * j) = pk;
                     }
                 }
             }
@@ -517,7 +519,7 @@ int launch_fwd_like(const void* x, const void* w_mat, void* out, const float* bi
     choose_tile(128, W, H, N, &p.tw, &p.th, &p.tn);
     p.tiles_w = (W + p.tw - 1) / p.tw; p.tiles_h = (H + p.th - 1) / p.th; p.tiles_n = (N + p.tn - 1) / p.tn;
     p.bn = pick_bn(c_out);
-    p.n_tiles = c_out / p.bn;
+    p.n_tiles = (c_out + p.bn - 1) / p.bn;
     const uint32_t stage_bytes = 128 * 128 + p.bn * 128;
     p.stages = std::min<int>(kMaxStages, kSmemBudget / stage_bytes);
     CUtensorMap mx, mw;
@@ -564,7 +566,10 @@ bool tc_conv_supported(int dtype, const ConvGeom& g) {
     if (dtype != CKPT_DTYPE_BF16) return false;
     if (g.stride != 1) return false;
     if (!((g.k == 3 && g.pad == 1) || (g.k == 1 && g.pad == 0))) return false;
-    if (g.cin % 64 || g.cout % 64) return false;
+    // the reduction runs over whole 64-channel blocks per tap; only a 1x1 filter may end in a ragged
+    // block (zero-filled), and stores are 8 channels wide
+    if (g.cin % 64) return false;
+    if (g.cout % 64 && !(g.k == 1 && g.cout % 8 == 0)) return false;
     if (g.ho != g.h || g.wo != g.w) return false;
     return true;
 }

@@ -65,6 +65,13 @@ int64_t simt_wgrad_scratch_bytes(const ConvGeom& g);
 int simt_conv_wgrad(int dtype, const ConvGeom& g, const void* dz, const void* x, float* dw,
                     void* scratch, int64_t scratch_bytes, void* stream);
 
+// First layer (3 input channels, 3x3, stride 1, padding 1, bf16): CUDA-core kernels of their own.
+bool small_conv_supported(int dtype, const ConvGeom& g);
+int64_t small_conv_scratch_bytes(const ConvGeom& g);
+int small_conv_fwd(const ConvGeom& g, const void* x, const void* w, void* z, void* stream);
+int small_conv_wgrad(const ConvGeom& g, const void* dz, const void* x, float* dw, void* scratch,
+                     int64_t scratch_bytes, void* stream);
+
 // Tensor-core (tcgen05) implicit-GEMM kernels; *_supported tells whether the shape has one.
 bool tc_conv_supported(int dtype, const ConvGeom& g);
 int64_t tc_conv_scratch_bytes(const ConvGeom& g);

@@ -198,6 +198,7 @@ static void wgrad_split(const ConvGeom& g, int* slices, int* k_per_slice) {
 }
 
 int64_t simt_wgrad_scratch_bytes(const ConvGeom& g) {
+    if (small_conv_supported(CKPT_DTYPE_BF16, g)) return small_conv_scratch_bytes(g);   // upper bound for both dtypes
     int slices, per;
     wgrad_split(g, &slices, &per);
     if (slices <= 1) return 0;
@@ -223,6 +224,7 @@ static int launch_wgrad(const ConvGeom& g, const void* dz, const void* x, float*
 }
 
 int simt_conv_fwd(int dtype, const ConvGeom& g, const void* x, const void* w, void* z, const float* bias, int relu, void* stream) {
+    if (!bias && !relu && small_conv_supported(dtype, g)) return small_conv_fwd(g, x, w, z, stream);
     return dtype == CKPT_DTYPE_BF16 ? launch_fwd<__nv_bfloat16>(g, x, w, z, bias, relu, (cudaStream_t)stream)
                                     : launch_fwd<float>(g, x, w, z, bias, relu, (cudaStream_t)stream);
 }
@@ -231,6 +233,7 @@ int simt_conv_dgrad(int dtype, const ConvGeom& g, const void* dz, const void* w,
                                     : launch_dgrad<float>(g, dz, w, dx, (cudaStream_t)stream);
 }
 int simt_conv_wgrad(int dtype, const ConvGeom& g, const void* dz, const void* x, float* dw, void* scratch, int64_t scratch_bytes, void* stream) {
+    if (small_conv_supported(dtype, g)) return small_conv_wgrad(g, dz, x, dw, scratch, scratch_bytes, stream);
     return dtype == CKPT_DTYPE_BF16 ? launch_wgrad<__nv_bfloat16>(g, dz, x, dw, scratch, scratch_bytes, (cudaStream_t)stream)
                                     : launch_wgrad<float>(g, dz, x, dw, scratch, scratch_bytes, (cudaStream_t)stream);
 }
@@ -304,14 +307,16 @@ int64_t bn_scratch_bytes(int64_t rows, int c) {
     return (int64_t)BN_MAX_BLOCKS * c * 2 * (int64_t)sizeof(float) + 4 * (int64_t)c * sizeof(float);
 }
 
-// Two running sums per channel over a slab of rows.  WHAT 0: (z, z^2).  WHAT 1: (g, g*xhat) with
-// g = dy masked by the ReLU of the forward output.
+// Two running sums per channel over a slab of rows.  WHAT 0: (z, z^2).  WHAT 1: (g, g*z) with
+// g = dy masked by the ReLU of the forward output (the normalised form g*xhat follows in the
+// finalize step: sum g*xhat = inv_std * (sum g*z - mean * sum g)).
 template <typename T, int VEC, int WHAT>
-__global__ void __launch_bounds__(BN_THREADS) bn_partial_kernel(const T* __restrict__ z, const T* __restrict__ dy,
-                                                                const float* __restrict__ stats, int relu, int64_t rows,
-                                                                int c, int lanes, int rows_per_iter, int64_t rows_per_block,
-                                                                float* __restrict__ partial) {
+__global__ void __launch_bounds__(BN_THREADS, 3) bn_partial_kernel(const T* __restrict__ z, const T* __restrict__ dy,
+                                                                   const float* __restrict__ stats, int relu, int64_t rows,
+                                                                   int c, int lanes, int rows_per_iter, int64_t rows_per_block,
+                                                                   float* __restrict__ partial) {
     extern __shared__ float red[];          // [BN_THREADS][2*VEC]
+    constexpr int U = WHAT == 0 ? 4 : 2;    // rows in flight per thread
     const int lanes_here = min(lanes, BN_THREADS);
     const int64_t row_begin = (int64_t)blockIdx.x * rows_per_block;
     const int64_t row_end = min(rows, row_begin + rows_per_block);
@@ -324,24 +329,24 @@ __global__ void __launch_bounds__(BN_THREADS) bn_partial_kernel(const T* __restr
         const bool active = r < rows_per_iter && lane < lanes;
         if (active) {
             const int ch = lane * VEC;
-            float mean[VEC], inv[VEC], sc[VEC], sh[VEC];
+            float sc[VEC], sh[VEC];
             if (WHAT == 1) {
 #pragma unroll
-                for (int i = 0; i < VEC; ++i) { mean[i] = stats[ch + i]; inv[i] = stats[c + ch + i]; sc[i] = stats[2 * c + ch + i]; sh[i] = stats[3 * c + ch + i]; }
+                for (int i = 0; i < VEC; ++i) { sc[i] = stats[2 * c + ch + i]; sh[i] = stats[3 * c + ch + i]; }
             }
-            // four rows in flight per thread; sums are still taken in row order
-            for (int64_t row = row_begin + r; row < row_end; row += 4 * (int64_t)rows_per_iter) {
-                float v[4][VEC], g[4][VEC];
+            // U rows in flight per thread; sums are still taken in row order
+            for (int64_t row = row_begin + r; row < row_end; row += U * (int64_t)rows_per_iter) {
+                float v[U][VEC], g[WHAT == 1 ? U : 1][VEC];
 #pragma unroll
-                for (int u = 0; u < 4; ++u) {
+                for (int u = 0; u < U; ++u) {
                     const int64_t rr = row + (int64_t)u * rows_per_iter;
                     if (rr < row_end) {
                         load_vec<T, VEC>(z + rr * c + ch, v[u]);
-                        if (WHAT == 1) load_vec<T, VEC>(dy + rr * c + ch, g[u]);
+                        if (WHAT == 1) load_vec<T, VEC>(dy + rr * c + ch, g[WHAT == 1 ? u : 0]);
                     }
                 }
 #pragma unroll
-                for (int u = 0; u < 4; ++u) {
+                for (int u = 0; u < U; ++u) {
                     if (row + (int64_t)u * rows_per_iter >= row_end) break;
                     if (WHAT == 0) {
 #pragma unroll
@@ -351,10 +356,9 @@ __global__ void __launch_bounds__(BN_THREADS) bn_partial_kernel(const T* __restr
                         for (int i = 0; i < VEC; ++i) {
                             float yv = fmaf(v[u][i], sc[i], sh[i]);
                             bool pass = !relu || (float)cvt<T>(fmaxf(yv, 0.f)) > 0.f;
-                            float gi = pass ? g[u][i] : 0.f;
-                            float xh = (v[u][i] - mean[i]) * inv[i];
+                            float gi = pass ? g[WHAT == 1 ? u : 0][i] : 0.f;
                             s0[i] += gi;
-                            s1[i] = fmaf(gi, xh, s1[i]);
+                            s1[i] = fmaf(gi, v[u][i], s1[i]);
                         }
                     }
                 }
@@ -418,11 +422,13 @@ __global__ void __launch_bounds__(32) bn_finalize_bwd_kernel(const float* __rest
     double s, q;
     warp_channel_sums(partial, blocks, c, ch, s, q);
     if (threadIdx.x != 0) return;
+    // q = sum g*z  ->  sum g*xhat = inv_std * (q - mean * sum g)
+    const double gx = (double)stats[c + ch] * (q - (double)stats[ch] * s);
     dbeta[ch] = (float)s;
-    dgamma[ch] = (float)q;
+    dgamma[ch] = (float)gx;
     double scale = stats[2 * c + ch];
     coef[ch] = (float)(scale * s * inv_rows);
-    coef[c + ch] = (float)(scale * q * inv_rows);
+    coef[c + ch] = (float)(scale * gx * inv_rows);
 }
 
 // y = max(z*scale + shift, 0).  When the grid's thread count is a multiple of the number of channel

@@ -28,6 +28,8 @@ CONV_CASES = [
     (2, 23, 19, 3, 16, 7, 2, 3),     # stem-like
     (3, 28, 28, 64, 64, 3, 1, 1),    # several 64-wide tiles with a tail
     (5, 1, 1, 200, 70, 1, 1, 0),     # fully connected as a 1x1 convolution
+    (3, 21, 18, 3, 64, 3, 1, 1),     # first-layer kernels (3 input channels, 64 outputs)
+    (2, 40, 40, 3, 128, 3, 1, 1),
 ]
 
 
@@ -40,6 +42,7 @@ TC_CASES = [
     (8, 7, 7, 64, 320, 1, 0),        # 1x1, output channels not a multiple of 128
     (5, 30, 30, 128, 64, 1, 0),
     (64, 1, 1, 512, 192, 1, 0),      # fully connected shape
+    (48, 1, 1, 256, 1000, 1, 0),     # classifier: output channels not a multiple of 64
     (2, 56, 56, 64, 64, 3, 1),
 ]
 

@@ -38,10 +38,10 @@ def test_noalloc_matches_ordinary_entry_point_twice(dtype):
         scratch = torch.empty(ck.bn_scratch_bytes(rows, c), dtype=torch.uint8, device="cuda")
         ck.bn_relu_forward(dtype, rows, c, zd, gd, bd, relu, y_ref, st_ref, scratch)
         torch.cuda.synchronize()
-        allocated = torch.cuda.memory_allocated()
+        free_before = torch.cuda.mem_get_info()[0]          # device-wide: sees any cudaMalloc, whoever makes it
         ck.bn_relu_forward_noalloc(dtype, rows, c, zd, gd, bd, relu, y_new, st_new)
         torch.cuda.synchronize()
-        assert torch.cuda.memory_allocated() == allocated
+        assert torch.cuda.mem_get_info()[0] >= free_before
         assert max_rel_err(to_host(st_new), to_host(st_ref)) <= 1e-6
         assert max_rel_err(to_host(y_new), to_host(y_ref)) <= TIGHT[dtype]
 
