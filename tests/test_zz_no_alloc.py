@@ -23,6 +23,12 @@ TIGHT = {ck.DTYPE_F32: 2e-5, ck.DTYPE_BF16: 6e-3}       # same bounds as tests/t
 def test_noalloc_matches_ordinary_entry_point_twice(dtype):
     import torch
     rng = np.random.default_rng(99)
+    # The first call on a device looks up the built-in array (and, with lazy module loading, makes
+    # the driver load the module that contains it): do it before watching the free-memory counter.
+    warm = torch.zeros(8, 8, device="cuda").to(torch.bfloat16 if dtype == ck.DTYPE_BF16 else torch.float32)
+    ones = torch.ones(8, device="cuda")
+    ck.bn_relu_forward_noalloc(dtype, 8, 8, warm, ones, ones, 0, torch.empty_like(warm), torch.empty(32, device="cuda"))
+    torch.cuda.synchronize()
     # first a large, wide case that fills much of the shared array, then a small one
     for rows, c, relu in ((20000, 512, 1), (333, 24, 0)):
         z = (rng.standard_normal((rows, c)) * 1.5 + 0.3).astype(np.float32)
