@@ -83,8 +83,8 @@ class ClockSampler:
 
 
 def conv_flops(spec, plan_mask, shapes):
-    """Algorithmic FLOPs of one step: 2*MAC x (forward + recompute of non-checkpoints + backward
-    re-derivation of the pre-normalisation tensor + dgrad (units 2..n) + wgrad)."""
+    """Algorithmic FLOPs of one step: 2*MAC x (forward + recompute of non-checkpoints + dgrad
+    (units 2..n) + wgrad)."""
     fwd = []
     h, w, c = spec["input_hwc"]
     for u, (ho, wo, co) in zip(spec["units"], shapes[1:]):
@@ -96,12 +96,9 @@ def conv_flops(spec, plan_mask, shapes):
             fwd.append(0.0)
     total = 0.0
     for i, f in enumerate(fwd, start=1):
-        conv = spec["units"][i - 1]["kind"] == "conv_bn_relu"
         total += f                                   # forward
         if not plan_mask[i]:
             total += f                               # segment recompute
-        if conv:
-            total += f                               # backward re-derives the conv output
         total += f                                   # wgrad
         if i > 1:
             total += f                               # dgrad

@@ -104,14 +104,14 @@ int ckpt_maxpool_forward(int dtype, int32_t n, int32_t h, int32_t w, int32_t c, 
                          const void* x, void* y, void* stream) {
     if (!x || !y) { set_error("null pointer"); return CKPT_E_NULL; }
     if (n < 1 || c < 1 || k < 1 || stride < 1 || pad < 0 || 2 * pad > k || h + 2 * pad < k || w + 2 * pad < k) { set_error("bad pooling shape"); return CKPT_E_BAD_ARG; }
-    return maxpool_forward(dtype, n, h, w, c, k, stride, pad, x, y, stream);
+    return maxpool_forward(dtype, n, h, w, c, k, stride, pad, x, y, nullptr, stream);
 }
 
 int ckpt_maxpool_backward(int dtype, int32_t n, int32_t h, int32_t w, int32_t c, int32_t k, int32_t stride, int32_t pad,
                           const void* x, const void* dy, void* dx, void* stream) {
     if (!x || !dy || !dx) { set_error("null pointer"); return CKPT_E_NULL; }
     if (n < 1 || c < 1 || k < 1 || stride < 1 || pad < 0 || 2 * pad > k || h + 2 * pad < k || w + 2 * pad < k) { set_error("bad pooling shape"); return CKPT_E_BAD_ARG; }
-    return maxpool_backward(dtype, n, h, w, c, k, stride, pad, x, dy, dx, stream);
+    return maxpool_backward(dtype, n, h, w, c, k, stride, pad, x, dy, dx, nullptr, stream);
 }
 
 int ckpt_softmax_ce(int dtype, int32_t batch, int32_t classes, const void* logits, const int32_t* labels, float* loss,

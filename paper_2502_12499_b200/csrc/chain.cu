@@ -91,76 +91,120 @@ static int conv_wgrad_any(StepCtx& c, const ConvGeom& g, const void* dz, const v
     return simt_conv_wgrad(c.ch->dtype, g, dz, x, dw, c.ws + c.ch->off_scr, c.ch->scr_bytes, c.stream);
 }
 
+// A conv+BN+ReLU unit stores its convolution output *before* normalisation as d_i; normalisation and
+// ReLU (fixed by the batch statistics saved next to the parameters) are applied by whoever reads
+// d_i.  The unit's backward then has everything it needs - its input, its own pre-normalisation
+// tensor - without re-running the convolution, and d_i keeps the size the planner was given.
+static bool pending_act(const ckpt_chain* ch, int64_t j) {
+    return j >= 1 && ch->units[j - 1].desc.kind == CKPT_UNIT_CONV_BN_RELU;
+}
+static float* stats_of(StepCtx& c, int64_t j) {
+    return (float*)(c.ws + c.ch->off_stats) + c.ch->units[j - 1].stats_off;
+}
+static int64_t rows_of(const ckpt_chain* ch, int64_t j) { return ch->batch * ch->shapes[j].h * ch->shapes[j].w; }
+
+// The activated form of d_j: d_j itself, or a materialised copy in the workspace.
+static int activated(StepCtx& c, int64_t j, const void* raw, const void** out) {
+    *out = raw;
+    if (!pending_act(c.ch, j)) return CKPT_OK;
+    void* xbuf = c.ws + c.ch->off_z;
+    *out = xbuf;
+    return bn_apply(c.ch->dtype, rows_of(c.ch, j), c.ch->shapes[j].c, raw, stats_of(c, j), 1, xbuf, c.stream);
+}
+
 // d_i = f_i(d_{i-1}, w_i)  (Eq. (1)); i is 1-based.
-static int unit_forward(StepCtx& c, int64_t i, const void* x, void* y) {
+static int unit_forward(StepCtx& c, int64_t i, const void* x_raw, void* y) {
     if (c.dry) return CKPT_OK;
     const Unit& u = c.ch->units[i - 1];
     const int dt = c.ch->dtype;
-    const int64_t rows = c.ch->batch * u.out.h * u.out.w;
     void* const* p = c.params + u.param_first;
     char* ws = c.ws;
+    const void* x = x_raw;
+    int rc;
     switch (u.desc.kind) {
-        case CKPT_UNIT_CONV_BN_RELU: {
-            void* z = ws + c.ch->off_z;
-            int rc = conv_forward_any(c, u.geom, x, p[0], z, nullptr, 0);
-            if (rc) return rc;
-            float* stats = (float*)(ws + c.ch->off_stats) + u.stats_off;
-            return bn_relu_forward(dt, rows, u.out.c, z, (const float*)p[1], (const float*)p[2], 1, y,
-                                   stats, ws + c.ch->off_scr, c.stream);
+        case CKPT_UNIT_CONV_BN_RELU:
+            if ((rc = activated(c, i - 1, x_raw, &x))) return rc;
+            if ((rc = conv_forward_any(c, u.geom, x, p[0], y, nullptr, 0))) return rc;
+            return bn_statistics(dt, rows_of(c.ch, i), u.out.c, y, (const float*)p[1], (const float*)p[2], stats_of(c, i),
+                                 ws + c.ch->off_scr, c.stream);
+        case CKPT_UNIT_MAXPOOL: {
+            const float* act = nullptr;
+            if (pending_act(c.ch, i - 1)) {
+                if (maxpool_fuses_activation(dt, u.in.h, u.in.w, u.in.c, u.desc.k, u.desc.stride, u.desc.pad)) act = stats_of(c, i - 1);
+                else if ((rc = activated(c, i - 1, x_raw, &x))) return rc;
+            }
+            return maxpool_forward(dt, (int)c.ch->batch, u.in.h, u.in.w, u.in.c, u.desc.k, u.desc.stride, u.desc.pad, x, y, act,
+                                   c.stream);
         }
-        case CKPT_UNIT_MAXPOOL:
-            return maxpool_forward(dt, (int)c.ch->batch, u.in.h, u.in.w, u.in.c, u.desc.k, u.desc.stride,
-                                   u.desc.pad, x, y, c.stream);
         case CKPT_UNIT_AVGPOOL:
+            if ((rc = activated(c, i - 1, x_raw, &x))) return rc;
             return avgpool_forward(dt, (int)c.ch->batch, u.in.h, u.in.w, u.in.c, x, y, c.stream);
         case CKPT_UNIT_FC:
+            if ((rc = activated(c, i - 1, x_raw, &x))) return rc;
             return conv_forward_any(c, u.geom, x, p[0], y, (const float*)p[1], u.desc.flags & 1);
     }
     set_error("unit kind %d has no forward kernel", u.desc.kind);
     return CKPT_E_UNSUPPORTED;
 }
 
+// Turns dL/d(activated d_j) into dL/d(d_j) in place when d_j carries a pending normalisation, and
+// writes the gradients of that normalisation's scale and shift.
+static int through_pending_act(StepCtx& c, int64_t j, const void* d_j, void* g) {
+    if (!pending_act(c.ch, j)) return CKPT_OK;
+    const Unit& uj = c.ch->units[j - 1];
+    void* const* p = c.params + uj.param_first;
+    void* const* gr = c.grads + uj.param_first;
+    return bn_relu_backward(c.ch->dtype, rows_of(c.ch, j), uj.out.c, g, d_j, (const float*)p[1], stats_of(c, j), 1, g,
+                            (float*)gr[1], (float*)gr[2], c.ws + c.ch->off_scr, c.stream);
+}
+
 // r_i and g_i (Eqs. (3) and (5)): g_in = dL/dd_i (may be overwritten), g_out = dL/dd_{i-1} or null.
-static int unit_backward(StepCtx& c, int64_t i, const void* x, const void* y, void* g_in, void* g_out) {
+static int unit_backward(StepCtx& c, int64_t i, const void* x_raw, const void* y, void* g_in, void* g_out) {
     if (c.dry) return CKPT_OK;
     const Unit& u = c.ch->units[i - 1];
     const int dt = c.ch->dtype;
-    const int64_t rows = c.ch->batch * u.out.h * u.out.w;
     void* const* p = c.params + u.param_first;
     void* const* g = c.grads + u.param_first;
-    char* ws = c.ws;
+    const void* x = x_raw;
     int rc;
     switch (u.desc.kind) {
-        case CKPT_UNIT_CONV_BN_RELU: {
-            // The pre-normalisation tensor is not part of the chain's stored data: derive it again.
-            void* z = ws + c.ch->off_z;
-            if ((rc = conv_forward_any(c, u.geom, x, p[0], z, nullptr, 0))) return rc;
-            float* stats = (float*)(ws + c.ch->off_stats) + u.stats_off;
-            if ((rc = bn_relu_backward(dt, rows, u.out.c, g_in, z, (const float*)p[1], stats, 1, g_in,
-                                       (float*)g[1], (float*)g[2], ws + c.ch->off_scr, c.stream))) return rc;
+        case CKPT_UNIT_CONV_BN_RELU:
+            if ((rc = activated(c, i - 1, x_raw, &x))) return rc;
             if ((rc = conv_wgrad_any(c, u.geom, g_in, x, (float*)g[0]))) return rc;
-            if (g_out) return conv_dgrad_any(c, u.geom, g_in, p[0], g_out);
-            return CKPT_OK;
+            if (g_out && (rc = conv_dgrad_any(c, u.geom, g_in, p[0], g_out))) return rc;
+            break;
+        case CKPT_UNIT_MAXPOOL: {
+            if (!g_out) break;
+            const float* act = nullptr;
+            if (pending_act(c.ch, i - 1)) {
+                if (maxpool_fuses_activation(dt, u.in.h, u.in.w, u.in.c, u.desc.k, u.desc.stride, u.desc.pad)) act = stats_of(c, i - 1);
+                else if ((rc = activated(c, i - 1, x_raw, &x))) return rc;
+            }
+            if ((rc = maxpool_backward(dt, (int)c.ch->batch, u.in.h, u.in.w, u.in.c, u.desc.k, u.desc.stride, u.desc.pad, x, g_in,
+                                       g_out, act, c.stream))) return rc;
+            break;
         }
-        case CKPT_UNIT_MAXPOOL:
-            if (!g_out) return CKPT_OK;
-            return maxpool_backward(dt, (int)c.ch->batch, u.in.h, u.in.w, u.in.c, u.desc.k, u.desc.stride,
-                                    u.desc.pad, x, g_in, g_out, c.stream);
         case CKPT_UNIT_AVGPOOL:
-            if (!g_out) return CKPT_OK;
-            return avgpool_backward(dt, (int)c.ch->batch, u.in.h, u.in.w, u.in.c, g_in, g_out, c.stream);
+            if (!g_out) break;
+            if ((rc = avgpool_backward(dt, (int)c.ch->batch, u.in.h, u.in.w, u.in.c, g_in, g_out, c.stream))) return rc;
+            break;
         case CKPT_UNIT_FC: {
             const int64_t elems = c.ch->batch * u.out.c;
+            if ((rc = activated(c, i - 1, x_raw, &x))) return rc;
             if (u.desc.flags & 1)
                 if ((rc = relu_mask_inplace(dt, elems, g_in, y, c.stream))) return rc;
             if ((rc = column_sums(dt, c.ch->batch, u.out.c, g_in, (float*)g[1], c.stream))) return rc;
             if ((rc = conv_wgrad_any(c, u.geom, g_in, x, (float*)g[0]))) return rc;
-            if (g_out) return conv_dgrad_any(c, u.geom, g_in, p[0], g_out);
-            return CKPT_OK;
+            if (g_out && (rc = conv_dgrad_any(c, u.geom, g_in, p[0], g_out))) return rc;
+            break;
         }
+        default:
+            set_error("unit kind %d has no backward kernel", u.desc.kind);
+            return CKPT_E_UNSUPPORTED;
     }
-    set_error("unit kind %d has no backward kernel", u.desc.kind);
-    return CKPT_E_UNSUPPORTED;
+    // the producer of d_{i-1} may have left its normalisation pending: finish the chain rule through it
+    if (g_out) return through_pending_act(c, i - 1, x_raw, g_out);
+    return CKPT_OK;
 }
 
 static int run_step(StepCtx& c, double* loss_out) {
@@ -208,17 +252,20 @@ static int run_step(StepCtx& c, double* loss_out) {
     void* g_cur = gbuf[0];
     if (!c.dry) {
         const Shape& so = ch->shapes[n];
+        const void* out_act = nullptr;
+        if ((rc = activated(c, n, ptr(n), &out_act))) return rc;
         if (ch->loss == CKPT_LOSS_SOFTMAX_CE) {
             const int32_t* lab = (const int32_t*)(c.ws + ch->off_misc + 128 + 256);
             cudaError_t e = cudaMemcpyAsync((void*)lab, c.labels, ch->batch * sizeof(int32_t), cudaMemcpyDefault, c.stream);
             if (e != cudaSuccess) return cuda_fail(e, "copy of the labels");
-            rc = softmax_ce(ch->dtype, (int)ch->batch, so.h * so.w * so.c, ptr(n), lab,
+            rc = softmax_ce(ch->dtype, (int)ch->batch, so.h * so.w * so.c, out_act, lab,
                             (float*)(c.ws + ch->off_misc), g_cur, (float*)(c.ws + ch->off_scr), c.stream);
         } else {
-            rc = sum_loss(ch->dtype, ch->batch * so.h * so.w * so.c, ptr(n), (double*)(c.ws + ch->off_misc),
+            rc = sum_loss(ch->dtype, ch->batch * so.h * so.w * so.c, out_act, (double*)(c.ws + ch->off_misc),
                           g_cur, (double*)(c.ws + ch->off_scr), c.stream);
         }
         if (rc) return rc;
+        if ((rc = through_pending_act(c, n, ptr(n), g_cur))) return rc;
     }
 
     // ---------------- backward phase

@@ -89,10 +89,18 @@ int bn_relu_backward(int dtype, int64_t rows, int c, const void* dy, const void*
                      const float* stats, int relu, void* dz, float* dgamma, float* dbeta, void* scratch,
                      void* stream);
 
+// stats = the 4*c floats written by bn_statistics (mean, 1/std, scale, shift).
+int bn_statistics(int dtype, int64_t rows, int c, const void* z, const float* gamma, const float* beta, float* stats,
+                  void* scratch, void* stream);
+int bn_apply(int dtype, int64_t rows, int c, const void* z, const float* stats, int relu, void* y, void* stream);
+
+// act (may be null): statistics block of the producing conv unit; when given, the pooling kernels
+// read x through its pending normalisation + ReLU.  Only the 2x2/stride-2 kernels can do that.
+bool maxpool_fuses_activation(int dtype, int h, int w, int c, int k, int stride, int pad);
 int maxpool_forward(int dtype, int n, int h, int w, int c, int k, int stride, int pad, const void* x,
-                    void* y, void* stream);
+                    void* y, const float* act, void* stream);
 int maxpool_backward(int dtype, int n, int h, int w, int c, int k, int stride, int pad, const void* x,
-                     const void* dy, void* dx, void* stream);
+                     const void* dy, void* dx, const float* act, void* stream);
 int avgpool_forward(int dtype, int n, int h, int w, int c, const void* x, void* y, void* stream);
 int avgpool_backward(int dtype, int n, int h, int w, int c, const void* dy, void* dx, void* stream);
 

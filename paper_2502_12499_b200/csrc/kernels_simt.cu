@@ -533,8 +533,8 @@ __global__ void __launch_bounds__(256) bn_bwd_apply_kernel(const T* __restrict__
 }
 
 template <typename T, int VEC>
-static int bn_forward_t(int64_t rows, int c, const void* z, const float* gamma, const float* beta, int relu, void* y,
-                        float* stats, void* scratch, cudaStream_t st) {
+static int bn_stats_t(int64_t rows, int c, const void* z, const float* gamma, const float* beta, float* stats, void* scratch,
+                      cudaStream_t st) {
     BnLayout L = bn_layout(rows, c, VEC);
     float* partial = (float*)scratch;
     size_t smem = (size_t)BN_THREADS * 2 * VEC * sizeof(float);
@@ -543,8 +543,13 @@ static int bn_forward_t(int64_t rows, int c, const void* z, const float* gamma, 
     CKPT_LAUNCH_CHECK("batch-norm statistics");
     bn_finalize_fwd_kernel<<<c, 32, 0, st>>>(partial, L.blocks, c, 1.0 / (double)rows, gamma, beta, stats);
     CKPT_LAUNCH_CHECK("batch-norm finalize");
+    return CKPT_OK;
+}
+
+template <typename T, int VEC>
+static int bn_apply_t(int64_t rows, int c, const void* z, const float* stats, int relu, void* y, cudaStream_t st) {
     int64_t vecs = rows * c / VEC;
-    bn_apply_kernel<T, VEC><<<elementwise_grid(vecs), 256, 0, st>>>((const T*)z, stats, relu, vecs, L.lanes, c, (T*)y);
+    bn_apply_kernel<T, VEC><<<elementwise_grid(vecs), 256, 0, st>>>((const T*)z, stats, relu, vecs, c / VEC, c, (T*)y);
     CKPT_LAUNCH_CHECK("batch-norm apply");
     return CKPT_OK;
 }
@@ -568,15 +573,30 @@ static int bn_backward_t(int64_t rows, int c, const void* dy, const void* z, con
     return CKPT_OK;
 }
 
-int bn_relu_forward(int dtype, int64_t rows, int c, const void* z, const float* gamma, const float* beta, int relu, void* y,
-                    float* stats, void* scratch, void* stream) {
+int bn_statistics(int dtype, int64_t rows, int c, const void* z, const float* gamma, const float* beta, float* stats,
+                  void* scratch, void* stream) {
     cudaStream_t st = (cudaStream_t)stream;
     int vec = bn_vec(dtype, c);
     if (dtype == CKPT_DTYPE_BF16)
-        return vec == 8 ? bn_forward_t<__nv_bfloat16, 8>(rows, c, z, gamma, beta, relu, y, stats, scratch, st)
-                        : bn_forward_t<__nv_bfloat16, 1>(rows, c, z, gamma, beta, relu, y, stats, scratch, st);
-    return vec == 4 ? bn_forward_t<float, 4>(rows, c, z, gamma, beta, relu, y, stats, scratch, st)
-                    : bn_forward_t<float, 1>(rows, c, z, gamma, beta, relu, y, stats, scratch, st);
+        return vec == 8 ? bn_stats_t<__nv_bfloat16, 8>(rows, c, z, gamma, beta, stats, scratch, st)
+                        : bn_stats_t<__nv_bfloat16, 1>(rows, c, z, gamma, beta, stats, scratch, st);
+    return vec == 4 ? bn_stats_t<float, 4>(rows, c, z, gamma, beta, stats, scratch, st)
+                    : bn_stats_t<float, 1>(rows, c, z, gamma, beta, stats, scratch, st);
+}
+
+int bn_apply(int dtype, int64_t rows, int c, const void* z, const float* stats, int relu, void* y, void* stream) {
+    cudaStream_t st = (cudaStream_t)stream;
+    int vec = bn_vec(dtype, c);
+    if (dtype == CKPT_DTYPE_BF16)
+        return vec == 8 ? bn_apply_t<__nv_bfloat16, 8>(rows, c, z, stats, relu, y, st) : bn_apply_t<__nv_bfloat16, 1>(rows, c, z, stats, relu, y, st);
+    return vec == 4 ? bn_apply_t<float, 4>(rows, c, z, stats, relu, y, st) : bn_apply_t<float, 1>(rows, c, z, stats, relu, y, st);
+}
+
+int bn_relu_forward(int dtype, int64_t rows, int c, const void* z, const float* gamma, const float* beta, int relu, void* y,
+                    float* stats, void* scratch, void* stream) {
+    int rc = bn_statistics(dtype, rows, c, z, gamma, beta, stats, scratch, stream);
+    if (rc) return rc;
+    return bn_apply(dtype, rows, c, z, stats, relu, y, stream);
 }
 
 int bn_relu_backward(int dtype, int64_t rows, int c, const void* dy, const void* z, const float* gamma, const float* stats,
@@ -658,8 +678,18 @@ __global__ void maxpool_bwd_kernel(const T* __restrict__ x, const T* __restrict_
 
 // 2x2 / stride 2 / no padding on even-sized images, VEC channels per thread (16-byte accesses):
 // the layout every pooling layer of the benchmark chains has.  One thread per output pixel group.
+// Optional pending activation of the producer: value = round_T(max(v*scale + shift, 0)), exactly what a
+// materialised copy of the activated tensor would hold.
 template <typename T, int VEC>
-__global__ void __launch_bounds__(256) maxpool2x2_fwd_kernel(const T* __restrict__ x, T* __restrict__ y, int64_t items, int wo, int ho, int cv, int c) {
+__device__ __forceinline__ void pending_act(float (&v)[VEC], const float* __restrict__ act, int c, int ch) {
+    if (!act) return;
+#pragma unroll
+    for (int k = 0; k < VEC; ++k) v[k] = (float)cvt<T>(fmaxf(fmaf(v[k], act[2 * c + ch + k], act[3 * c + ch + k]), 0.f));
+}
+
+template <typename T, int VEC>
+__global__ void __launch_bounds__(256) maxpool2x2_fwd_kernel(const T* __restrict__ x, T* __restrict__ y, int64_t items, int wo, int ho, int cv, int c,
+                                                             const float* __restrict__ act) {
     for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < items; i += (int64_t)gridDim.x * blockDim.x) {
         const int cg = (int)(i % cv);
         int64_t t = i / cv;
@@ -672,6 +702,8 @@ __global__ void __launch_bounds__(256) maxpool2x2_fwd_kernel(const T* __restrict
         load_vec<T, VEC>(p + c, b);
         load_vec<T, VEC>(p + (int64_t)2 * wo * c, d);
         load_vec<T, VEC>(p + (int64_t)2 * wo * c + c, e);
+        pending_act<T, VEC>(a, act, c, cg * VEC); pending_act<T, VEC>(b, act, c, cg * VEC);
+        pending_act<T, VEC>(d, act, c, cg * VEC); pending_act<T, VEC>(e, act, c, cg * VEC);
 #pragma unroll
         for (int k = 0; k < VEC; ++k) o[k] = fmaxf(fmaxf(a[k], b[k]), fmaxf(d[k], e[k]));
         store_vec<T, VEC>(y + i * VEC, o);
@@ -681,7 +713,7 @@ __global__ void __launch_bounds__(256) maxpool2x2_fwd_kernel(const T* __restrict
 // Backward of the same: the first maximum of the window in row-major order takes the gradient.
 template <typename T, int VEC>
 __global__ void __launch_bounds__(256) maxpool2x2_bwd_kernel(const T* __restrict__ x, const T* __restrict__ dy, T* __restrict__ dx,
-                                                             int64_t items, int wo, int ho, int cv, int c) {
+                                                             int64_t items, int wo, int ho, int cv, int c, const float* __restrict__ act) {
     for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < items; i += (int64_t)gridDim.x * blockDim.x) {
         const int cg = (int)(i % cv);
         int64_t t = i / cv;
@@ -696,6 +728,8 @@ __global__ void __launch_bounds__(256) maxpool2x2_bwd_kernel(const T* __restrict
         load_vec<T, VEC>(x + off + down, d);
         load_vec<T, VEC>(x + off + down + c, e);
         load_vec<T, VEC>(dy + i * VEC, g);
+        pending_act<T, VEC>(a, act, c, cg * VEC); pending_act<T, VEC>(b, act, c, cg * VEC);
+        pending_act<T, VEC>(d, act, c, cg * VEC); pending_act<T, VEC>(e, act, c, cg * VEC);
 #pragma unroll
         for (int k = 0; k < VEC; ++k) {
             const float m = fmaxf(fmaxf(a[k], b[k]), fmaxf(d[k], e[k]));
@@ -709,23 +743,24 @@ __global__ void __launch_bounds__(256) maxpool2x2_bwd_kernel(const T* __restrict
     }
 }
 
-static bool pool_fast_path(int dtype, int h, int w, int c, int k, int stride, int pad) {
+bool maxpool_fuses_activation(int dtype, int h, int w, int c, int k, int stride, int pad) {
     const int vec = dtype == CKPT_DTYPE_BF16 ? 8 : 4;
     return k == 2 && stride == 2 && pad == 0 && h % 2 == 0 && w % 2 == 0 && c % vec == 0;
 }
 
-int maxpool_forward(int dtype, int n, int h, int w, int c, int k, int stride, int pad, const void* x, void* y, void* stream) {
+int maxpool_forward(int dtype, int n, int h, int w, int c, int k, int stride, int pad, const void* x, void* y, const float* act, void* stream) {
     int ho = (h + 2 * pad - k) / stride + 1, wo = (w + 2 * pad - k) / stride + 1;
-    if (pool_fast_path(dtype, h, w, c, k, stride, pad)) {
+    if (maxpool_fuses_activation(dtype, h, w, c, k, stride, pad)) {
         const int vec = dtype == CKPT_DTYPE_BF16 ? 8 : 4;
         const int64_t items = (int64_t)n * ho * wo * (c / vec);
         if (dtype == CKPT_DTYPE_BF16)
-            maxpool2x2_fwd_kernel<__nv_bfloat16, 8><<<elementwise_grid(items), 256, 0, (cudaStream_t)stream>>>((const __nv_bfloat16*)x, (__nv_bfloat16*)y, items, wo, ho, c / vec, c);
+            maxpool2x2_fwd_kernel<__nv_bfloat16, 8><<<elementwise_grid(items), 256, 0, (cudaStream_t)stream>>>((const __nv_bfloat16*)x, (__nv_bfloat16*)y, items, wo, ho, c / vec, c, act);
         else
-            maxpool2x2_fwd_kernel<float, 4><<<elementwise_grid(items), 256, 0, (cudaStream_t)stream>>>((const float*)x, (float*)y, items, wo, ho, c / vec, c);
+            maxpool2x2_fwd_kernel<float, 4><<<elementwise_grid(items), 256, 0, (cudaStream_t)stream>>>((const float*)x, (float*)y, items, wo, ho, c / vec, c, act);
         CKPT_LAUNCH_CHECK("max-pool 2x2 forward");
         return CKPT_OK;
     }
+    if (act) { set_error("the general pooling kernel takes an activated input"); return CKPT_E_BAD_ARG; }
     unsigned grid = elementwise_grid((int64_t)n * ho * wo * c);
     if (dtype == CKPT_DTYPE_BF16)
         maxpool_fwd_kernel<__nv_bfloat16><<<grid, 256, 0, (cudaStream_t)stream>>>((const __nv_bfloat16*)x, (__nv_bfloat16*)y, n, h, w, c, ho, wo, k, stride, pad);
@@ -735,18 +770,19 @@ int maxpool_forward(int dtype, int n, int h, int w, int c, int k, int stride, in
     return CKPT_OK;
 }
 
-int maxpool_backward(int dtype, int n, int h, int w, int c, int k, int stride, int pad, const void* x, const void* dy, void* dx, void* stream) {
+int maxpool_backward(int dtype, int n, int h, int w, int c, int k, int stride, int pad, const void* x, const void* dy, void* dx, const float* act, void* stream) {
     int ho = (h + 2 * pad - k) / stride + 1, wo = (w + 2 * pad - k) / stride + 1;
-    if (pool_fast_path(dtype, h, w, c, k, stride, pad)) {
+    if (maxpool_fuses_activation(dtype, h, w, c, k, stride, pad)) {
         const int vec = dtype == CKPT_DTYPE_BF16 ? 8 : 4;
         const int64_t items = (int64_t)n * ho * wo * (c / vec);
         if (dtype == CKPT_DTYPE_BF16)
-            maxpool2x2_bwd_kernel<__nv_bfloat16, 8><<<elementwise_grid(items), 256, 0, (cudaStream_t)stream>>>((const __nv_bfloat16*)x, (const __nv_bfloat16*)dy, (__nv_bfloat16*)dx, items, wo, ho, c / vec, c);
+            maxpool2x2_bwd_kernel<__nv_bfloat16, 8><<<elementwise_grid(items), 256, 0, (cudaStream_t)stream>>>((const __nv_bfloat16*)x, (const __nv_bfloat16*)dy, (__nv_bfloat16*)dx, items, wo, ho, c / vec, c, act);
         else
-            maxpool2x2_bwd_kernel<float, 4><<<elementwise_grid(items), 256, 0, (cudaStream_t)stream>>>((const float*)x, (const float*)dy, (float*)dx, items, wo, ho, c / vec, c);
+            maxpool2x2_bwd_kernel<float, 4><<<elementwise_grid(items), 256, 0, (cudaStream_t)stream>>>((const float*)x, (const float*)dy, (float*)dx, items, wo, ho, c / vec, c, act);
         CKPT_LAUNCH_CHECK("max-pool 2x2 backward");
         return CKPT_OK;
     }
+    if (act) { set_error("the general pooling kernel takes an activated input"); return CKPT_E_BAD_ARG; }
     unsigned grid = elementwise_grid((int64_t)n * h * w * c);
     if (dtype == CKPT_DTYPE_BF16)
         maxpool_bwd_kernel<__nv_bfloat16><<<grid, 256, 0, (cudaStream_t)stream>>>((const __nv_bfloat16*)x, (const __nv_bfloat16*)dy, (__nv_bfloat16*)dx, n, h, w, c, ho, wo, k, stride, pad);
