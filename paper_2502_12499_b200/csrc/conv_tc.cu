@@ -298,6 +298,160 @@ tc_conv_fwd_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_const
 }
 
 // ------------------------------------------------------------------------------------------------
+// Forward / dgrad for 64 reduction channels, 3x3, padding 1 (first layers of VGG-like chains, the
+// whole 64-channel deep chain).  With K = 9*64 the generic kernel is bound by L2->SM traffic (every
+// tap re-fetches the pixel tile) and by the unhidden epilogue.  Here a persistent CTA
+//   - keeps the whole filter of its 64 output channels (9 taps x 64 x 64, 72 KiB) in shared memory,
+//   - fetches per tile three copies of the input patch, one per horizontal tap offset, each with a
+//     one-row halo above and below: a vertical tap offset is then a whole number of 1024-byte
+//     swizzle atoms (8 pixels x 128 B), so every tap is a plain, aligned descriptor into a copy,
+//   - double-buffers both the patches and the accumulator (2 x 64 TMEM columns), so the epilogue
+//     of one tile runs under the MMAs of the next.
+// Pixel tile: 8 wide x th high (th <= 16) of one image; accumulator row m = h_local*8 + w_local.
+// ------------------------------------------------------------------------------------------------
+struct C64Params {
+    int H, W, N, c_out;
+    int th;                      // tile height (tile width is 8)
+    int tiles_w, tiles_h;
+    int n_tiles;                 // c_out / 64
+    int m_tiles;                 // tiles_w * tiles_h * N
+    int ctas_per_n;              // persistent CTAs that share one output-channel tile
+    uint32_t box_stride;         // bytes between the three shifted copies of a patch
+};
+
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+
+__global__ void __launch_bounds__(kThreads, 1)
+tc_conv_c64_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w,
+                   __nv_bfloat16* __restrict__ out, C64Params p, int* status) {
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    constexpr uint32_t w_bytes = 9 * 64 * 128;                       // resident filter
+    const uint32_t stage_bytes = 3 * p.box_stride;
+    const uint32_t a_base = base + w_bytes;
+    const uint32_t bars = a_base + 2 * stage_bytes;
+    __shared__ uint32_t tmem_base_slot;
+    __shared__ int failed_flag;
+    volatile int* failed = &failed_flag;
+    const uint32_t w_full = bars, a_full0 = bars + 8, a_empty0 = bars + 24, acc_full0 = bars + 40, acc_empty0 = bars + 56;
+
+    const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
+    const int n_tile = blockIdx.x % p.n_tiles;
+    const int first = blockIdx.x / p.n_tiles;
+    const int my_tiles = first < p.m_tiles ? (p.m_tiles - first + p.ctas_per_n - 1) / p.ctas_per_n : 0;
+    const uint32_t patch_bytes = (uint32_t)(8 * (p.th + 2)) * 128;
+
+    if (threadIdx.x == 0) {
+        failed_flag = 0;
+        mbar_init(w_full, 1);
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(a_full0 + 8 * b, 1); mbar_init(a_empty0 + 8 * b, 1);
+            mbar_init(acc_full0 + 8 * b, 1); mbar_init(acc_empty0 + 8 * b, 128);
+        }
+        fence_barrier_init();
+        tma_prefetch_desc(&map_x);
+        tma_prefetch_desc(&map_w);
+    }
+    if (warp == 1) tmem_alloc(smem_u32(&tmem_base_slot), 128);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = tmem_base_slot;
+
+    auto tile_origin = [&](int j, int& w0, int& h0, int& img) {
+        int t = first + j * p.ctas_per_n;
+        w0 = (t % p.tiles_w) * 8; t /= p.tiles_w;
+        h0 = (t % p.tiles_h) * p.th;
+        img = t / p.tiles_h;
+    };
+
+    if (warp == 0 && lane == 0) {
+        // ---------------- producer: the filter once, then the patches
+        mbar_expect_tx(w_full, w_bytes);
+        for (int tap = 0; tap < 9; ++tap) tma_load_2d(base + tap * 8192, &map_w, w_full, tap * 64, n_tile * 64);
+        int issued = 0;
+        for (int j = 0; j < my_tiles; ++j) {
+            const int b = j & 1;
+            if (!mbar_wait(a_empty0 + 8 * b, ((uint32_t)(j >> 1) & 1u) ^ 1u, failed, status, 301)) break;
+            int w0, h0, img;
+            tile_origin(j, w0, h0, img);
+            mbar_expect_tx(a_full0 + 8 * b, 3 * patch_bytes);
+            for (int sft = 0; sft < 3; ++sft)
+                tma_load_4d(a_base + b * stage_bytes + sft * p.box_stride, &map_x, a_full0 + 8 * b, 0, w0 + sft - 1, h0 - 1, img);
+            issued = j + 1;
+        }
+        if (*failed) {
+            mbar_drain(w_full, 0);
+            for (int j = max(0, issued - 2); j < issued; ++j) mbar_drain(a_full0 + 8 * (j & 1), (uint32_t)(j >> 1) & 1u);
+        }
+    } else if (warp == 1 && lane == 0) {
+        // ---------------- MMA issuer
+        const uint32_t idesc = instr_desc(128, 64, 0, 0);
+        bool ok = mbar_wait(w_full, 0, failed, status, 302);
+        for (int j = 0; j < my_tiles && ok; ++j) {
+            const int b = j & 1;
+            const uint32_t ph = (uint32_t)(j >> 1) & 1u;
+            if (!mbar_wait(acc_empty0 + 8 * b, ph ^ 1u, failed, status, 303)) { ok = false; break; }
+            if (!mbar_wait(a_full0 + 8 * b, ph, failed, status, 304)) { ok = false; break; }
+            tc_fence_after();
+            const uint32_t acc = tmem_base + (uint32_t)b * 64;
+#pragma unroll 1
+            for (int tap = 0; tap < 9; ++tap) {
+                const uint32_t a_addr = a_base + b * stage_bytes + (tap % 3) * p.box_stride + (tap / 3) * 1024;
+                const uint32_t b_addr = base + tap * 8192;
+#pragma unroll
+                for (int kk = 0; kk < 4; ++kk)
+                    umma_bf16(acc, smem_desc(a_addr + kk * 32, 0, 1024), smem_desc(b_addr + kk * 32, 0, 1024), idesc,
+                              (tap > 0 || kk > 0) ? 1u : 0u);
+            }
+            umma_commit(a_empty0 + 8 * b);
+            umma_commit(acc_full0 + 8 * b);
+        }
+    } else if (warp >= 2) {
+        // ---------------- epilogue
+        const int quarter = warp % 4;
+        const int row = quarter * 32 + lane;
+        const int wl = row % 8, hl = row / 8;
+        for (int j = 0; j < my_tiles; ++j) {
+            const int b = j & 1;
+            if (!mbar_wait(acc_full0 + 8 * b, (uint32_t)(j >> 1) & 1u, failed, status, 305)) break;
+            tc_fence_after();
+            int w0, h0, img;
+            tile_origin(j, w0, h0, img);
+            const bool valid = hl < p.th && (h0 + hl) < p.H && (w0 + wl) < p.W;
+            __nv_bfloat16* dst = out + ((((size_t)img * p.H + (h0 + hl)) * p.W + (w0 + wl)) * p.c_out + (size_t)n_tile * 64);
+#pragma unroll
+            for (int c0 = 0; c0 < 64; c0 += 32) {
+                uint32_t v[32];
+                tmem_ld32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(b * 64 + c0), v);
+                if (valid) {
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        uint4 pk;
+                        __nv_bfloat162* h = reinterpret_cast<__nv_bfloat162*>(&pk);
+#pragma unroll
+                        for (int e = 0; e < 4; ++e)
+                            h[e] = __floats2bfloat162_rn(__uint_as_float(v[8 * q + 2 * e]), __uint_as_float(v[8 * q + 2 * e + 1]));
+                        *reinterpret_cast<uint4*>(dst + c0 + 8 * q) = pk;
+                    }
+                }
+            }
+            tc_fence_before();
+            mbar_arrive(acc_empty0 + 8 * b);
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        __syncwarp();
+        tc_fence_after();
+        tmem_dealloc(tmem_base, 128);
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
 // wgrad kernel: D[c_out tile of 128][up to 4 blocks of 64 (tap, c_in) columns], K = pixels
 // ------------------------------------------------------------------------------------------------
 struct WgradParams {
@@ -512,8 +666,43 @@ void choose_tile(int pixels, int W, int H, int N, int* tw, int* th, int* tn) {
 
 int pick_bn(int c_out) { return c_out % 256 == 0 ? 256 : (c_out % 128 == 0 ? 128 : 64); }
 
+int launch_c64(const void* x, const void* w_mat, void* out, int N, int H, int W, int c_out, int* status, cudaStream_t st,
+               const char* what) {
+    C64Params p;
+    p.H = H; p.W = W; p.N = N; p.c_out = c_out;
+    const int nt = (H + 15) / 16;
+    p.th = (H + nt - 1) / nt;
+    p.tiles_h = (H + p.th - 1) / p.th;
+    p.tiles_w = (W + 7) / 8;
+    p.n_tiles = c_out / 64;
+    p.m_tiles = p.tiles_w * p.tiles_h * N;
+    int sms = 148, dev = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    p.ctas_per_n = std::max(1, std::min(sms / p.n_tiles, p.m_tiles));
+    // a tap reads 128 rows starting up to 2 halo rows (16 pixels) into a copy: keep that inside the copy's slot
+    p.box_stride = (uint32_t)align_up((int64_t)std::max(8 * (p.th + 2), 16 + 128) * 128, 1024);
+    CUtensorMap mx, mw;
+    int rc = make_act_map(&mx, x, N, H, W, 64, 8, p.th + 2, 1);
+    if (rc) return rc;
+    rc = make_mat_map(&mw, w_mat, c_out, 9 * 64, 64);
+    if (rc) return rc;
+    const size_t smem = 9 * 64 * 128 + 2 * 3 * (size_t)p.box_stride + 1024 + 256;
+    static bool attr_set = false;
+    if (!attr_set) {
+        cudaError_t e = cudaFuncSetAttribute(tc_conv_c64_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024);
+        if (e != cudaSuccess) return cuda_fail(e, "raising the shared-memory limit");
+        attr_set = true;
+    }
+    tc_conv_c64_kernel<<<p.ctas_per_n * p.n_tiles, kThreads, smem, st>>>(mx, mw, (__nv_bfloat16*)out, p, status);
+    CKPT_LAUNCH_CHECK(what);
+    return CKPT_OK;
+}
+
 int launch_fwd_like(const void* x, const void* w_mat, void* out, const float* bias, int relu, int N, int H, int W, int c_red,
                     int c_out, int k, int pad, int* status, cudaStream_t st, const char* what) {
+    if (c_red == 64 && k == 3 && pad == 1 && c_out % 64 == 0 && !bias && !relu)
+        return launch_c64(x, w_mat, out, N, H, W, c_out, status, st, what);
     FwdParams p;
     p.H = H; p.W = W; p.N = N; p.c_red = c_red; p.c_out = c_out; p.k = k; p.pad = pad;
     choose_tile(128, W, H, N, &p.tw, &p.th, &p.tn);
