@@ -213,8 +213,9 @@ tc_conv_fwd_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_const
     tc_fence_after();
     const uint32_t tmem_base = tmem_base_slot;
 
-    if (warp == 0 && lane == 0) {
-        // ---------------- TMA producer
+    if (warp == 0) {
+        // ---------------- TMA producer: the whole warp walks the ring, each copy is issued by its own lane
+        // (issuing a bulk-tensor copy keeps a thread busy for a few hundred cycles)
         int issued = 0;
         for (int it = 0; it < iters; ++it) {
             const int s = it % p.stages;
@@ -222,13 +223,14 @@ tc_conv_fwd_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_const
             if (!mbar_wait(empty_bar(s), phase ^ 1u, failed, status, 101)) break;
             const int tap = it / blocks, blk = it % blocks;
             const int r = tap / p.k, q = tap % p.k;
-            mbar_expect_tx(full_bar(s), stage_bytes);
+            if (lane == 0) mbar_expect_tx(full_bar(s), stage_bytes);
+            __syncwarp();
             const uint32_t a_dst = base + (uint32_t)s * stage_bytes;
-            tma_load_4d(a_dst, &map_x, full_bar(s), blk * 64, w0 + q - p.pad, h0 + r - p.pad, n0);
-            tma_load_2d(a_dst + a_bytes, &map_w, full_bar(s), tap * p.c_red + blk * 64, n_tile * p.bn);
+            if (lane == 0) tma_load_4d(a_dst, &map_x, full_bar(s), blk * 64, w0 + q - p.pad, h0 + r - p.pad, n0);
+            if (lane == 1) tma_load_2d(a_dst + a_bytes, &map_w, full_bar(s), tap * p.c_red + blk * 64, n_tile * p.bn);
             issued = it + 1;
         }
-        if (*failed) {
+        if (*failed && lane == 0) {
             // copies that were issued but never consumed must land before the CTA may exit
             for (int it = max(0, issued - p.stages); it < issued; ++it)
                 mbar_drain(full_bar(it % p.stages), (uint32_t)(it / p.stages) & 1u);
@@ -367,22 +369,24 @@ tc_conv_c64_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_const
         img = t / p.tiles_h;
     };
 
-    if (warp == 0 && lane == 0) {
-        // ---------------- producer: the filter once, then the patches
-        mbar_expect_tx(w_full, w_bytes);
-        for (int tap = 0; tap < 9; ++tap) tma_load_2d(base + tap * 8192, &map_w, w_full, tap * 64, n_tile * 64);
+    if (warp == 0) {
+        // ---------------- producer: the filter once, then the patches; one lane per copy
+        if (lane == 0) mbar_expect_tx(w_full, w_bytes);
+        __syncwarp();
+        if (lane < 9) tma_load_2d(base + lane * 8192, &map_w, w_full, lane * 64, n_tile * 64);
         int issued = 0;
         for (int j = 0; j < my_tiles; ++j) {
             const int b = j & 1;
             if (!mbar_wait(a_empty0 + 8 * b, ((uint32_t)(j >> 1) & 1u) ^ 1u, failed, status, 301)) break;
             int w0, h0, img;
             tile_origin(j, w0, h0, img);
-            mbar_expect_tx(a_full0 + 8 * b, 3 * patch_bytes);
-            for (int sft = 0; sft < 3; ++sft)
-                tma_load_4d(a_base + b * stage_bytes + sft * p.box_stride, &map_x, a_full0 + 8 * b, 0, w0 + sft - 1, h0 - 1, img);
+            if (lane == 0) mbar_expect_tx(a_full0 + 8 * b, 3 * patch_bytes);
+            __syncwarp();
+            if (lane < 3)
+                tma_load_4d(a_base + b * stage_bytes + lane * p.box_stride, &map_x, a_full0 + 8 * b, 0, w0 + lane - 1, h0 - 1, img);
             issued = j + 1;
         }
-        if (*failed) {
+        if (*failed && lane == 0) {
             mbar_drain(w_full, 0);
             for (int j = max(0, issued - 2); j < issued; ++j) mbar_drain(a_full0 + 8 * (j & 1), (uint32_t)(j >> 1) & 1u);
         }
@@ -508,7 +512,8 @@ tc_conv_wgrad_kernel(const __grid_constant__ CUtensorMap map_dz, const __grid_co
     tc_fence_after();
     const uint32_t tmem_base = tmem_base_slot;
 
-    if (warp == 0 && lane == 0) {
+    if (warp == 0) {
+        // one lane per copy (see the forward kernel)
         int issued = 0;
         for (int it = 0; it < iters; ++it) {
             const int s = it % p.stages;
@@ -518,17 +523,19 @@ tc_conv_wgrad_kernel(const __grid_constant__ CUtensorMap map_dz, const __grid_co
             const int w0 = (t % p.tiles_w) * p.tw; t /= p.tiles_w;
             const int h0 = (t % p.tiles_h) * p.th;
             const int n0 = (t / p.tiles_h) * p.tn;
-            mbar_expect_tx(full_bar(s), (2 + (uint32_t)nb_here) * box_bytes);
+            if (lane == 0) mbar_expect_tx(full_bar(s), (2 + (uint32_t)nb_here) * box_bytes);
+            __syncwarp();
             const uint32_t dst = base + (uint32_t)s * stage_bytes;
-            tma_load_4d(dst, &map_dz, full_bar(s), co_tile * 128, w0, h0, n0);
-            tma_load_4d(dst + box_bytes, &map_dz, full_bar(s), co_tile * 128 + 64, w0, h0, n0);
-            for (int j = 0; j < nb_here; ++j) {
+            if (lane < 2) {
+                tma_load_4d(dst + lane * box_bytes, &map_dz, full_bar(s), co_tile * 128 + 64 * lane, w0, h0, n0);
+            } else if (lane < 2 + nb_here) {
+                const int j = lane - 2;
                 const int b = blk_begin + j, tap = b / cin_blocks, cib = b % cin_blocks;
                 tma_load_4d(dst + (2 + j) * box_bytes, &map_x, full_bar(s), cib * 64, w0 + tap % p.k - p.pad, h0 + tap / p.k - p.pad, n0);
             }
             issued = it + 1;
         }
-        if (*failed) {
+        if (*failed && lane == 0) {
             for (int it = max(0, issued - p.stages); it < issued; ++it)
                 mbar_drain(full_bar(it % p.stages), (uint32_t)(it / p.stages) & 1u);
         }
@@ -739,10 +746,22 @@ void wgrad_plan(const ConvGeom& g, WgradParams* p, int* slices, int* groups, int
     p->nb = p->total_blocks % 4 == 0 ? 4 : (p->total_blocks % 3 == 0 ? 3 : (p->total_blocks >= 4 ? 4 : p->total_blocks));
     *groups = (p->total_blocks + p->nb - 1) / p->nb;
     *co_tiles = (g.cout + 127) / 128;
+    // slices of the pixel range: fill the SMs with whole waves of equally long CTAs (2 to 4 waves),
+    // keeping at least 8 pixel tiles per slice
     const int64_t base_ctas = (int64_t)*groups * *co_tiles;
-    int64_t want = std::max<int64_t>(1, (148 * 3 + base_ctas - 1) / base_ctas);
-    int64_t by_k = std::max<int64_t>(1, p->total_tiles / 8);          // at least 8 pixel tiles per slice
-    int64_t s = std::min<int64_t>(std::min<int64_t>(want, by_k), 256);
+    int sms = 148, dev = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    int64_t by_k = std::max<int64_t>(1, p->total_tiles / 8);
+    int64_t s = 1;
+    double best_eff = -1.0;
+    for (int64_t cand = 1; cand <= std::min<int64_t>(by_k, 256); ++cand) {
+        const int64_t ctas = cand * base_ctas;
+        const int64_t waves = (ctas + sms - 1) / sms;
+        if (waves > 4 && cand > 1) break;
+        const double eff = (double)ctas / (double)(waves * sms) * (waves >= 2 ? 1.0 : 0.9);
+        if (eff > best_eff + 1e-9) { best_eff = eff; s = cand; }
+    }
     p->tiles_per_slice = (int)((p->total_tiles + s - 1) / s);
     *slices = (p->total_tiles + p->tiles_per_slice - 1) / p->tiles_per_slice;
     const uint32_t stage_bytes = (2 + p->nb) * 64 * 128;
