@@ -213,9 +213,8 @@ tc_conv_fwd_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_const
     tc_fence_after();
     const uint32_t tmem_base = tmem_base_slot;
 
-    if (warp == 0) {
-        // ---------------- TMA producer: the whole warp walks the ring, each copy is issued by its own lane
-        // (issuing a bulk-tensor copy keeps a thread busy for a few hundred cycles)
+    if (warp == 0 && lane == 0) {
+        // ---------------- TMA producer (two copies per stage: measured fastest from a single thread)
         int issued = 0;
         for (int it = 0; it < iters; ++it) {
             const int s = it % p.stages;
@@ -223,14 +222,13 @@ tc_conv_fwd_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_const
             if (!mbar_wait(empty_bar(s), phase ^ 1u, failed, status, 101)) break;
             const int tap = it / blocks, blk = it % blocks;
             const int r = tap / p.k, q = tap % p.k;
-            if (lane == 0) mbar_expect_tx(full_bar(s), stage_bytes);
-            __syncwarp();
+            mbar_expect_tx(full_bar(s), stage_bytes);
             const uint32_t a_dst = base + (uint32_t)s * stage_bytes;
-            if (lane == 0) tma_load_4d(a_dst, &map_x, full_bar(s), blk * 64, w0 + q - p.pad, h0 + r - p.pad, n0);
-            if (lane == 1) tma_load_2d(a_dst + a_bytes, &map_w, full_bar(s), tap * p.c_red + blk * 64, n_tile * p.bn);
+            tma_load_4d(a_dst, &map_x, full_bar(s), blk * 64, w0 + q - p.pad, h0 + r - p.pad, n0);
+            tma_load_2d(a_dst + a_bytes, &map_w, full_bar(s), tap * p.c_red + blk * 64, n_tile * p.bn);
             issued = it + 1;
         }
-        if (*failed && lane == 0) {
+        if (*failed) {
             // copies that were issued but never consumed must land before the CTA may exit
             for (int it = max(0, issued - p.stages); it < issued; ++it)
                 mbar_drain(full_bar(it % p.stages), (uint32_t)(it / p.stages) & 1u);
@@ -377,11 +375,14 @@ tc_conv_c64_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_const
         int issued = 0;
         for (int j = 0; j < my_tiles; ++j) {
             const int b = j & 1;
-            if (!mbar_wait(a_empty0 + 8 * b, ((uint32_t)(j >> 1) & 1u) ^ 1u, failed, status, 301)) break;
+            int go = 1;
+            if (lane == 0) {
+                go = mbar_wait(a_empty0 + 8 * b, ((uint32_t)(j >> 1) & 1u) ^ 1u, failed, status, 301) ? 1 : 0;
+                if (go) mbar_expect_tx(a_full0 + 8 * b, 3 * patch_bytes);
+            }
+            if (!__shfl_sync(0xffffffffu, go, 0)) break;
             int w0, h0, img;
             tile_origin(j, w0, h0, img);
-            if (lane == 0) mbar_expect_tx(a_full0 + 8 * b, 3 * patch_bytes);
-            __syncwarp();
             if (lane < 3)
                 tma_load_4d(a_base + b * stage_bytes + lane * p.box_stride, &map_x, a_full0 + 8 * b, 0, w0 + lane - 1, h0 - 1, img);
             issued = j + 1;
@@ -513,18 +514,19 @@ tc_conv_wgrad_kernel(const __grid_constant__ CUtensorMap map_dz, const __grid_co
     const uint32_t tmem_base = tmem_base_slot;
 
     if (warp == 0) {
-        // one lane per copy (see the forward kernel)
+        // six copies per stage: one lane each (issuing a bulk-tensor copy occupies a thread for a few hundred cycles)
         int issued = 0;
         for (int it = 0; it < iters; ++it) {
             const int s = it % p.stages;
             const uint32_t phase = (uint32_t)(it / p.stages) & 1u;
+            // every lane watches the barrier itself: measured faster than one lane polling for the warp
             if (!mbar_wait(empty_bar(s), phase ^ 1u, failed, status, 201)) break;
+            if (lane == 0) mbar_expect_tx(full_bar(s), (2 + (uint32_t)nb_here) * box_bytes);
+            __syncwarp();
             int t = tile_begin + it;
             const int w0 = (t % p.tiles_w) * p.tw; t /= p.tiles_w;
             const int h0 = (t % p.tiles_h) * p.th;
             const int n0 = (t / p.tiles_h) * p.tn;
-            if (lane == 0) mbar_expect_tx(full_bar(s), (2 + (uint32_t)nb_here) * box_bytes);
-            __syncwarp();
             const uint32_t dst = base + (uint32_t)s * stage_bytes;
             if (lane < 2) {
                 tma_load_4d(dst + lane * box_bytes, &map_dz, full_bar(s), co_tile * 128 + 64 * lane, w0, h0, n0);
