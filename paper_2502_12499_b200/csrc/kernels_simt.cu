@@ -427,8 +427,12 @@ __global__ void __launch_bounds__(32) bn_finalize_bwd_kernel(const float* __rest
     dbeta[ch] = (float)s;
     dgamma[ch] = (float)gx;
     double scale = stats[2 * c + ch];
-    coef[ch] = (float)(scale * s * inv_rows);
-    coef[c + ch] = (float)(scale * gx * inv_rows);
+    // dz = scale*g - k1 - xhat*k2 with k1 = scale*dbeta/rows, k2 = scale*dgamma/rows and
+    // xhat = (z - mean)*inv_std, regrouped as  dz = scale*g - A - z*B
+    const double k1 = scale * s * inv_rows, k2 = scale * gx * inv_rows;
+    const double mean = stats[ch], inv = stats[c + ch];
+    coef[ch] = (float)(k1 - mean * inv * k2);
+    coef[c + ch] = (float)(inv * k2);
 }
 
 // y = max(z*scale + shift, 0).  When the grid's thread count is a multiple of the number of channel
@@ -477,32 +481,31 @@ __global__ void __launch_bounds__(256) bn_apply_kernel(const T* __restrict__ z, 
 }
 
 template <typename T, int VEC>
-__device__ __forceinline__ void bn_bwd_point(const float (&v)[VEC], const float (&g)[VEC], const float (&mean)[VEC],
-                                             const float (&inv)[VEC], const float (&sc)[VEC], const float (&sh)[VEC],
-                                             const float (&k1)[VEC], const float (&k2)[VEC], int relu, float (&o)[VEC]) {
+__device__ __forceinline__ void bn_bwd_point(const float (&v)[VEC], const float (&g)[VEC], const float (&sc)[VEC],
+                                             const float (&sh)[VEC], const float (&ca)[VEC], const float (&cb)[VEC], int relu,
+                                             float (&o)[VEC]) {
 #pragma unroll
     for (int k = 0; k < VEC; ++k) {
         float yv = fmaf(v[k], sc[k], sh[k]);
         bool pass = !relu || (float)cvt<T>(fmaxf(yv, 0.f)) > 0.f;
         float gi = pass ? g[k] : 0.f;
-        float xh = (v[k] - mean[k]) * inv[k];
-        o[k] = sc[k] * gi - k1[k] - xh * k2[k];
+        o[k] = fmaf(-v[k], cb[k], fmaf(sc[k], gi, -ca[k]));
     }
 }
 
 template <typename T, int VEC>
-__global__ void __launch_bounds__(256) bn_bwd_apply_kernel(const T* __restrict__ dy, const T* __restrict__ z,
-                                                           const float* __restrict__ stats, const float* __restrict__ coef,
-                                                           int relu, int64_t vecs, int lanes, int c, T* __restrict__ dz) {
+__global__ void __launch_bounds__(256, 3) bn_bwd_apply_kernel(const T* __restrict__ dy, const T* __restrict__ z,
+                                                              const float* __restrict__ stats, const float* __restrict__ coef,
+                                                              int relu, int64_t vecs, int lanes, int c, T* __restrict__ dz) {
     const int64_t stride = (int64_t)gridDim.x * blockDim.x;
     const int64_t first = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     const bool fixed = stride % lanes == 0;
-    float mean[VEC], inv[VEC], sc[VEC], sh[VEC], k1[VEC], k2[VEC];
+    float sc[VEC], sh[VEC], ca[VEC], cb[VEC];
     auto load_coef = [&](int ch) {
 #pragma unroll
         for (int k = 0; k < VEC; ++k) {
-            mean[k] = stats[ch + k]; inv[k] = stats[c + ch + k]; sc[k] = stats[2 * c + ch + k]; sh[k] = stats[3 * c + ch + k];
-            k1[k] = coef[ch + k]; k2[k] = coef[c + ch + k];
+            sc[k] = stats[2 * c + ch + k]; sh[k] = stats[3 * c + ch + k];
+            ca[k] = coef[ch + k]; cb[k] = coef[c + ch + k];
         }
     };
     if (fixed) {
@@ -516,7 +519,7 @@ __global__ void __launch_bounds__(256) bn_bwd_apply_kernel(const T* __restrict__
             for (int u = 0; u < 2; ++u) {
                 if (i + u * stride >= vecs) break;
                 float o[VEC];
-                bn_bwd_point<T, VEC>(v[u], g[u], mean, inv, sc, sh, k1, k2, relu, o);
+                bn_bwd_point<T, VEC>(v[u], g[u], sc, sh, ca, cb, relu, o);
                 store_vec<T, VEC>(dz + (i + u * stride) * VEC, o);
             }
         }
@@ -527,9 +530,93 @@ __global__ void __launch_bounds__(256) bn_bwd_apply_kernel(const T* __restrict__
         float v[VEC], g[VEC], o[VEC];
         load_vec<T, VEC>(z + i * VEC, v);
         load_vec<T, VEC>(dy + i * VEC, g);
-        bn_bwd_point<T, VEC>(v, g, mean, inv, sc, sh, k1, k2, relu, o);
+        bn_bwd_point<T, VEC>(v, g, sc, sh, ca, cb, relu, o);
         store_vec<T, VEC>(dz + i * VEC, o);
     }
+}
+
+// Streaming form of the per-channel sums for channel counts whose vector lanes divide the block:
+// every thread keeps one channel group for the whole kernel (its stride through the tensor is a
+// multiple of the row length), holds U independent 16-byte loads in flight, and the block combines
+// its threads by a fixed tree.  Same two sums as bn_partial_kernel.
+constexpr int BNF_THREADS = 384;
+template <typename T, int VEC, int WHAT>
+__global__ void __launch_bounds__(BNF_THREADS, 2) bn_partial_stream_kernel(const T* __restrict__ z, const T* __restrict__ dy,
+                                                                           const float* __restrict__ stats, int relu,
+                                                                           int64_t vecs, int lanes, int c,
+                                                                           float* __restrict__ partial) {
+    __shared__ float red[BNF_THREADS][2 * VEC + 1];
+    constexpr int U = WHAT == 0 ? 4 : 2;
+    const int64_t stride = (int64_t)gridDim.x * BNF_THREADS;
+    const int64_t first = (int64_t)blockIdx.x * BNF_THREADS + threadIdx.x;
+    const int ch = (int)(first % lanes) * VEC;
+    float s0[VEC], s1[VEC], sc[VEC], sh[VEC];
+#pragma unroll
+    for (int k = 0; k < VEC; ++k) { s0[k] = 0.f; s1[k] = 0.f; }
+    if (WHAT == 1) {
+#pragma unroll
+        for (int k = 0; k < VEC; ++k) { sc[k] = stats[2 * c + ch + k]; sh[k] = stats[3 * c + ch + k]; }
+    }
+    for (int64_t i = first; i < vecs; i += U * stride) {
+        float v[U][VEC], g[WHAT == 1 ? U : 1][VEC];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            if (i + u * stride < vecs) {
+                load_vec<T, VEC>(z + (i + u * stride) * VEC, v[u]);
+                if (WHAT == 1) load_vec<T, VEC>(dy + (i + u * stride) * VEC, g[WHAT == 1 ? u : 0]);
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            if (i + u * stride >= vecs) break;
+#pragma unroll
+            for (int k = 0; k < VEC; ++k) {
+                if (WHAT == 0) {
+                    s0[k] += v[u][k];
+                    s1[k] = fmaf(v[u][k], v[u][k], s1[k]);
+                } else {
+                    float yv = fmaf(v[u][k], sc[k], sh[k]);
+                    bool pass = !relu || (float)cvt<T>(fmaxf(yv, 0.f)) > 0.f;
+                    float gi = pass ? g[WHAT == 1 ? u : 0][k] : 0.f;
+                    s0[k] += gi;
+                    s1[k] = fmaf(gi, v[u][k], s1[k]);
+                }
+            }
+        }
+    }
+#pragma unroll
+    for (int k = 0; k < VEC; ++k) { red[threadIdx.x][k] = s0[k]; red[threadIdx.x][VEC + k] = s1[k]; }
+    __syncthreads();
+    // 384 -> 128 partial rows, then halving down to one row per channel group; threads t and t + m*lanes
+    // always hold the same channel group because every step keeps the index modulo `lanes`
+    if (threadIdx.x < 128) {
+#pragma unroll
+        for (int k = 0; k < 2 * VEC; ++k) red[threadIdx.x][k] = (red[threadIdx.x][k] + red[threadIdx.x + 128][k]) + red[threadIdx.x + 256][k];
+    }
+    __syncthreads();
+    for (int off = 64; off >= lanes; off >>= 1) {
+        if ((int)threadIdx.x < off) {
+#pragma unroll
+            for (int k = 0; k < 2 * VEC; ++k) red[threadIdx.x][k] += red[threadIdx.x + off][k];
+        }
+        __syncthreads();
+    }
+    if ((int)threadIdx.x < lanes) {
+        const int chn = (int)(((int64_t)blockIdx.x * BNF_THREADS + threadIdx.x) % lanes) * VEC;
+#pragma unroll
+        for (int k = 0; k < VEC; ++k) {
+            partial[((size_t)blockIdx.x * 2 + 0) * c + chn + k] = red[threadIdx.x][k];
+            partial[((size_t)blockIdx.x * 2 + 1) * c + chn + k] = red[threadIdx.x][VEC + k];
+        }
+    }
+}
+
+// The streaming kernel needs: lanes a power of two between 8 and 128 (so that 128 and the block
+// size are multiples of it).
+static bool bn_stream_ok(int lanes) { return lanes >= 8 && lanes <= 128 && (lanes & (lanes - 1)) == 0; }
+static int bn_stream_blocks(int64_t vecs) {
+    int64_t b = (vecs + (int64_t)BNF_THREADS * 8 - 1) / ((int64_t)BNF_THREADS * 8);
+    return (int)std::max<int64_t>(1, std::min<int64_t>(b, 148 * 2));
 }
 
 template <typename T, int VEC>
@@ -537,11 +624,18 @@ static int bn_stats_t(int64_t rows, int c, const void* z, const float* gamma, co
                       cudaStream_t st) {
     BnLayout L = bn_layout(rows, c, VEC);
     float* partial = (float*)scratch;
-    size_t smem = (size_t)BN_THREADS * 2 * VEC * sizeof(float);
-    bn_partial_kernel<T, VEC, 0><<<L.blocks, BN_THREADS, smem, st>>>((const T*)z, nullptr, nullptr, 0, rows, c, L.lanes,
-                                                                      L.rows_per_iter, L.rows_per_block, partial);
+    int blocks = L.blocks;
+    if (VEC > 1 && bn_stream_ok(L.lanes)) {
+        const int64_t vecs = rows * c / VEC;
+        blocks = bn_stream_blocks(vecs);
+        bn_partial_stream_kernel<T, VEC, 0><<<blocks, BNF_THREADS, 0, st>>>((const T*)z, nullptr, nullptr, 0, vecs, L.lanes, c, partial);
+    } else {
+        size_t smem = (size_t)BN_THREADS * 2 * VEC * sizeof(float);
+        bn_partial_kernel<T, VEC, 0><<<L.blocks, BN_THREADS, smem, st>>>((const T*)z, nullptr, nullptr, 0, rows, c, L.lanes,
+                                                                          L.rows_per_iter, L.rows_per_block, partial);
+    }
     CKPT_LAUNCH_CHECK("batch-norm statistics");
-    bn_finalize_fwd_kernel<<<c, 32, 0, st>>>(partial, L.blocks, c, 1.0 / (double)rows, gamma, beta, stats);
+    bn_finalize_fwd_kernel<<<c, 32, 0, st>>>(partial, blocks, c, 1.0 / (double)rows, gamma, beta, stats);
     CKPT_LAUNCH_CHECK("batch-norm finalize");
     return CKPT_OK;
 }
@@ -560,11 +654,18 @@ static int bn_backward_t(int64_t rows, int c, const void* dy, const void* z, con
     BnLayout L = bn_layout(rows, c, VEC);
     float* partial = (float*)scratch;
     float* coef = partial + (size_t)BN_MAX_BLOCKS * c * 2;
-    size_t smem = (size_t)BN_THREADS * 2 * VEC * sizeof(float);
-    bn_partial_kernel<T, VEC, 1><<<L.blocks, BN_THREADS, smem, st>>>((const T*)z, (const T*)dy, stats, relu, rows, c, L.lanes,
-                                                                      L.rows_per_iter, L.rows_per_block, partial);
+    int blocks = L.blocks;
+    if (VEC > 1 && bn_stream_ok(L.lanes)) {
+        const int64_t nvecs = rows * c / VEC;
+        blocks = bn_stream_blocks(nvecs);
+        bn_partial_stream_kernel<T, VEC, 1><<<blocks, BNF_THREADS, 0, st>>>((const T*)z, (const T*)dy, stats, relu, nvecs, L.lanes, c, partial);
+    } else {
+        size_t smem = (size_t)BN_THREADS * 2 * VEC * sizeof(float);
+        bn_partial_kernel<T, VEC, 1><<<L.blocks, BN_THREADS, smem, st>>>((const T*)z, (const T*)dy, stats, relu, rows, c, L.lanes,
+                                                                          L.rows_per_iter, L.rows_per_block, partial);
+    }
     CKPT_LAUNCH_CHECK("batch-norm backward sums");
-    bn_finalize_bwd_kernel<<<c, 32, 0, st>>>(partial, L.blocks, c, 1.0 / (double)rows, stats, dgamma, dbeta, coef);
+    bn_finalize_bwd_kernel<<<c, 32, 0, st>>>(partial, blocks, c, 1.0 / (double)rows, stats, dgamma, dbeta, coef);
     CKPT_LAUNCH_CHECK("batch-norm backward finalize");
     int64_t vecs = rows * c / VEC;
     bn_bwd_apply_kernel<T, VEC><<<elementwise_grid(vecs), 256, 0, st>>>((const T*)dy, (const T*)z, stats, coef, relu, vecs,
