@@ -42,6 +42,7 @@ int ckpt_conv2d_scratch_bytes(const ckpt_conv_shape* s, int dtype, int64_t* byte
     ConvGeom g = make_geom(*s);
     int64_t b = simt_wgrad_scratch_bytes(g);
     if (tc_conv_supported(dtype, g)) b = b > tc_conv_scratch_bytes(g) ? b : tc_conv_scratch_bytes(g);
+    if (small_conv_supported(dtype, g)) b = b > small_conv_scratch_bytes(g) ? b : small_conv_scratch_bytes(g);
     *bytes = b;
     return CKPT_OK;
 }
@@ -74,6 +75,8 @@ int ckpt_conv2d_wgrad(const ckpt_conv_shape* s, int dtype, int impl, const void*
     if (rc) return rc;
     if (!dz || !x || !dw) { set_error("null tensor"); return CKPT_E_NULL; }
     ConvGeom g = make_geom(*s);
+    if (impl != 1 && small_conv_supported(dtype, g))
+        return small_conv_wgrad(g, dz, x, dw, scratch, scratch_bytes, op_status_word(), stream);
     if (want_tc(impl, dtype, g, &rc)) return tc_conv_wgrad(g, dz, x, dw, scratch, scratch_bytes, op_status_word(), stream);
     if (rc) return rc;
     return simt_conv_wgrad(dtype, g, dz, x, dw, scratch, scratch_bytes, stream);

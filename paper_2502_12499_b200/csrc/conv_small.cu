@@ -3,8 +3,8 @@
 // the layer is bound by writing its 64-channel output, so it runs on the CUDA cores:
 //   forward: one thread per output pixel, 64 output channels in registers, the filter in shared
 //            memory (read as broadcast float4), the pixel's 128-byte output row written as 8 x 16 B;
-//   wgrad  : each thread owns 4 output channels x all 9*c_in filter taps for a strided subset of
-//            the block's pixels; block partials are combined in a fixed order.
+//   wgrad  : the input is unfolded to [pixel][9*c_in padded to 64] and the gradient becomes a
+//            [c_out x 64] contraction over pixels on the tensor cores (the 1x1 wgrad kernel).
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 
@@ -77,32 +77,21 @@ __global__ void __launch_bounds__(128) small_fwd_kernel(const __nv_bfloat16* __r
     }
 }
 
-// partial[block][co][k] = sum over the block's pixels of dz[p][co] * x[p shifted by tap][c]
+// xcol[p][0..9*CIN) = the 3x3 neighbourhood of pixel p (zero outside the image), [9*CIN..64) = 0:
+// the first layer's input unfolded to 64 "channels", so that its weight gradient is a plain
+// [c_out x 64] = dz^T * xcol contraction for the tensor cores.
 template <int CIN>
-__global__ void __launch_bounds__(128) small_wgrad_kernel(const __nv_bfloat16* __restrict__ dz, const __nv_bfloat16* __restrict__ x,
-                                                          float* __restrict__ partial, int n, int h, int wd, int cout,
-                                                          int64_t pixels_per_block) {
+__global__ void __launch_bounds__(256) unfold3x3_kernel(const __nv_bfloat16* __restrict__ x, __nv_bfloat16* __restrict__ xcol,
+                                                        int n, int h, int wd) {
     constexpr int K = 9 * CIN;
-    __shared__ float red[4][64][K + 1];
-    const int co0 = blockIdx.y * 64;
-    const int cg = threadIdx.x % 16;            // 4 output channels: co0 + 4*cg ..
-    const int pl = threadIdx.x / 16;            // pixel lane 0..7
     const int64_t pixels = (int64_t)n * h * wd;
-    const int64_t p_begin = (int64_t)blockIdx.x * pixels_per_block;
-    const int64_t p_end = min(pixels, p_begin + pixels_per_block);
-    float acc[4][K];
-#pragma unroll
-    for (int a = 0; a < 4; ++a)
-#pragma unroll
-        for (int k = 0; k < K; ++k) acc[a][k] = 0.f;
-    for (int64_t p = p_begin + pl; p < p_end; p += 8) {
+    for (int64_t p = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; p < pixels; p += (int64_t)gridDim.x * blockDim.x) {
         const int ow = (int)(p % wd);
         const int oh = (int)((p / wd) % h);
         const int64_t img = p / ((int64_t)wd * h);
-        const uint2 graw = *reinterpret_cast<const uint2*>(dz + p * cout + co0 + 4 * cg);
-        const float2 g01 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&graw.x));
-        const float2 g23 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&graw.y));
-        const float g[4] = {g01.x, g01.y, g23.x, g23.y};
+        __align__(16) __nv_bfloat16 v[64];
+#pragma unroll
+        for (int i = K; i < 64; ++i) v[i] = __float2bfloat16_rn(0.f);
 #pragma unroll
         for (int r = 0; r < 3; ++r) {
 #pragma unroll
@@ -111,41 +100,20 @@ __global__ void __launch_bounds__(128) small_wgrad_kernel(const __nv_bfloat16* _
                 const bool in = ih >= 0 && ih < h && iw >= 0 && iw < wd;
                 const __nv_bfloat16* src = x + ((img * h + ih) * wd + iw) * CIN;
 #pragma unroll
-                for (int c = 0; c < CIN; ++c) {
-                    const float xv = in ? __bfloat162float(src[c]) : 0.f;
-#pragma unroll
-                    for (int a = 0; a < 4; ++a) acc[a][(r * 3 + s) * CIN + c] = fmaf(g[a], xv, acc[a][(r * 3 + s) * CIN + c]);
-                }
+                for (int c = 0; c < CIN; ++c) v[(r * 3 + s) * CIN + c] = in ? src[c] : __float2bfloat16_rn(0.f);
             }
         }
-    }
-    // the two pixel lanes of a warp first, then the four warps, always in the same order
+        uint4* dst = reinterpret_cast<uint4*>(xcol + p * 64);
 #pragma unroll
-    for (int a = 0; a < 4; ++a)
-#pragma unroll
-        for (int k = 0; k < K; ++k) {
-            const float other = __shfl_xor_sync(0xffffffffu, acc[a][k], 16);
-            if ((threadIdx.x & 16) == 0) red[threadIdx.x / 32][4 * cg + a][k] = acc[a][k] + other;
-        }
-    __syncthreads();
-    for (int i = threadIdx.x; i < 64 * K; i += blockDim.x) {
-        const int k = i % K, co = i / K;
-        float s = 0.f;
-#pragma unroll
-        for (int l = 0; l < 4; ++l) s += red[l][co][k];
-        partial[((size_t)blockIdx.x * cout + co0 + co) * K + k] = s;
+        for (int j = 0; j < 8; ++j) dst[j] = reinterpret_cast<const uint4*>(v)[j];
     }
 }
 
-__global__ void small_slice_sum_kernel(const float* __restrict__ partial, float* __restrict__ out, int64_t elems, int slices) {
-    int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (e >= elems) return;
-    float s = 0.f;
-    for (int z = 0; z < slices; ++z) s += partial[(size_t)z * elems + e];
-    out[e] = s;
+// dw[co][0..K) = dwp[co][0..K) out of the padded [c_out][64] result
+__global__ void take_columns_kernel(const float* __restrict__ dwp, float* __restrict__ dw, int cout, int k) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < cout * k) dw[i] = dwp[(i / k) * 64 + i % k];
 }
-
-constexpr int kWgradBlocks = 148 * 4;
 
 }  // namespace
 
@@ -153,7 +121,17 @@ bool small_conv_supported(int dtype, const ConvGeom& g) {
     return dtype == CKPT_DTYPE_BF16 && g.cin == 3 && g.k == 3 && g.stride == 1 && g.pad == 1 && g.cout % 64 == 0;
 }
 
-int64_t small_conv_scratch_bytes(const ConvGeom& g) { return (int64_t)kWgradBlocks * g.cout * 9 * g.cin * 4; }
+static ConvGeom unfolded_geom(const ConvGeom& g) {
+    ConvGeom u = g;
+    u.cin = 64; u.k = 1; u.pad = 0;
+    return u;
+}
+static int64_t xcol_bytes(const ConvGeom& g) { return align_up((int64_t)g.n * g.h * g.w * 128, 256); }
+static int64_t dwp_bytes(const ConvGeom& g) { return align_up((int64_t)g.cout * 64 * 4, 256); }
+
+int64_t small_conv_scratch_bytes(const ConvGeom& g) {
+    return xcol_bytes(g) + dwp_bytes(g) + tc_conv_scratch_bytes(unfolded_geom(g));
+}
 
 int small_conv_fwd(const ConvGeom& g, const void* x, const void* w, void* z, void* stream) {
     const int64_t pixels = (int64_t)g.n * g.h * g.w;
@@ -164,18 +142,22 @@ int small_conv_fwd(const ConvGeom& g, const void* x, const void* w, void* z, voi
     return CKPT_OK;
 }
 
-int small_conv_wgrad(const ConvGeom& g, const void* dz, const void* x, float* dw, void* scratch, int64_t scratch_bytes, void* stream) {
+int small_conv_wgrad(const ConvGeom& g, const void* dz, const void* x, float* dw, void* scratch, int64_t scratch_bytes,
+                     int* device_status, void* stream) {
     if (!scratch || scratch_bytes < small_conv_scratch_bytes(g)) { set_error("first-layer wgrad scratch too small"); return CKPT_E_WORKSPACE; }
+    cudaStream_t st = (cudaStream_t)stream;
+    char* base = (char*)scratch;
+    __nv_bfloat16* xcol = (__nv_bfloat16*)base;
+    float* dwp = (float*)(base + xcol_bytes(g));
+    void* tc_scratch = base + xcol_bytes(g) + dwp_bytes(g);
     const int64_t pixels = (int64_t)g.n * g.h * g.w;
-    const int64_t per_block = ((pixels + kWgradBlocks - 1) / kWgradBlocks + 7) / 8 * 8;
-    const int blocks = (int)((pixels + per_block - 1) / per_block);
-    dim3 grid(blocks, g.cout / 64);
-    small_wgrad_kernel<3><<<grid, 128, 0, (cudaStream_t)stream>>>((const __nv_bfloat16*)dz, (const __nv_bfloat16*)x, (float*)scratch,
-                                                                  g.n, g.h, g.w, g.cout, per_block);
-    CKPT_LAUNCH_CHECK("first-layer conv wgrad");
-    const int64_t elems = (int64_t)g.cout * 27;
-    small_slice_sum_kernel<<<(unsigned)((elems + 255) / 256), 256, 0, (cudaStream_t)stream>>>((const float*)scratch, dw, elems, blocks);
-    CKPT_LAUNCH_CHECK("first-layer wgrad block sum");
+    unfold3x3_kernel<3><<<(unsigned)std::min<int64_t>((pixels + 255) / 256, 148 * 16), 256, 0, st>>>((const __nv_bfloat16*)x, xcol, g.n, g.h, g.w);
+    CKPT_LAUNCH_CHECK("first-layer unfold");
+    const ConvGeom u = unfolded_geom(g);
+    int rc = tc_conv_wgrad(u, dz, xcol, dwp, tc_scratch, scratch_bytes - xcol_bytes(g) - dwp_bytes(g), device_status, stream);
+    if (rc) return rc;
+    take_columns_kernel<<<(g.cout * 27 + 255) / 256, 256, 0, st>>>(dwp, dw, g.cout, 27);
+    CKPT_LAUNCH_CHECK("first-layer wgrad column pick");
     return CKPT_OK;
 }
 

@@ -70,7 +70,7 @@ bool small_conv_supported(int dtype, const ConvGeom& g);
 int64_t small_conv_scratch_bytes(const ConvGeom& g);
 int small_conv_fwd(const ConvGeom& g, const void* x, const void* w, void* z, void* stream);
 int small_conv_wgrad(const ConvGeom& g, const void* dz, const void* x, float* dw, void* scratch,
-                     int64_t scratch_bytes, void* stream);
+                     int64_t scratch_bytes, int* device_status, void* stream);
 
 // Tensor-core (tcgen05) implicit-GEMM kernels; *_supported tells whether the shape has one.
 bool tc_conv_supported(int dtype, const ConvGeom& g);

@@ -198,7 +198,6 @@ static void wgrad_split(const ConvGeom& g, int* slices, int* k_per_slice) {
 }
 
 int64_t simt_wgrad_scratch_bytes(const ConvGeom& g) {
-    if (small_conv_supported(CKPT_DTYPE_BF16, g)) return small_conv_scratch_bytes(g);   // upper bound for both dtypes
     int slices, per;
     wgrad_split(g, &slices, &per);
     if (slices <= 1) return 0;
@@ -233,7 +232,6 @@ int simt_conv_dgrad(int dtype, const ConvGeom& g, const void* dz, const void* w,
                                     : launch_dgrad<float>(g, dz, w, dx, (cudaStream_t)stream);
 }
 int simt_conv_wgrad(int dtype, const ConvGeom& g, const void* dz, const void* x, float* dw, void* scratch, int64_t scratch_bytes, void* stream) {
-    if (small_conv_supported(dtype, g)) return small_conv_wgrad(g, dz, x, dw, scratch, scratch_bytes, stream);
     return dtype == CKPT_DTYPE_BF16 ? launch_wgrad<__nv_bfloat16>(g, dz, x, dw, scratch, scratch_bytes, (cudaStream_t)stream)
                                     : launch_wgrad<float>(g, dz, x, dw, scratch, scratch_bytes, (cudaStream_t)stream);
 }

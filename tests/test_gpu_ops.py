@@ -119,6 +119,32 @@ def test_conv_tensor_core_kernels(case):
     assert max_rel_err(to_host(z2), to_host(z)) <= TIGHT[dtype]
 
 
+@pytest.mark.parametrize("n,h,w,cout", [(3, 21, 18, 64), (2, 40, 40, 128), (5, 32, 32, 64)])
+def test_first_layer_kernels(n, h, w, cout):
+    """3 input channels, bf16, automatic kernel choice: CUDA-core forward, unfolded tensor-core wgrad."""
+    import torch
+    dtype = ck.DTYPE_BF16
+    rng = np.random.default_rng(n * h + cout)
+    x = rounded(rng.standard_normal((n, h, w, 3)), dtype)
+    wt = rounded(rng.standard_normal((cout, 3, 3, 3)) / np.sqrt(27), dtype)
+    z_ref = no.conv2d_fwd(x.astype(np.float64), wt.astype(np.float64), 1, 1)
+    dz = rounded(rng.standard_normal(z_ref.shape), dtype)
+    _, dw_ref = no.conv2d_bwd(x.astype(np.float64), wt.astype(np.float64), dz.astype(np.float64), 1, 1)
+    shape = ck.ConvShape(n, h, w, 3, cout, 3, 1, 1)
+    xd, wd, dzd = to_dev(x, dtype), to_dev(wt, dtype), to_dev(dz, dtype)
+    scratch = torch.empty(max(ck.conv2d_scratch_bytes(shape, dtype), 256), dtype=torch.uint8, device="cuda")
+    z = torch.full(z_ref.shape, float("nan"), device="cuda").to(xd.dtype)
+    dw = torch.full(wt.shape, float("nan"), device="cuda", dtype=torch.float32)
+    dw2 = torch.empty_like(dw)
+    ck.conv2d_forward(shape, dtype, 0, xd, wd, z, scratch)
+    ck.conv2d_wgrad(shape, dtype, 0, dzd, xd, dw, scratch)
+    ck.conv2d_wgrad(shape, dtype, 0, dzd, xd, dw2, scratch)
+    torch.cuda.synchronize()
+    assert max_rel_err(to_host(z), z_ref) <= TIGHT[dtype]
+    assert max_rel_err(to_host(dw), dw_ref) <= 2e-5
+    assert torch.equal(dw, dw2)
+
+
 @pytest.mark.parametrize("dtype", [ck.DTYPE_F32, ck.DTYPE_BF16])
 @pytest.mark.parametrize("rows,c,relu", [(37, 3, 1), (4096, 16, 1), (5000, 64, 1), (777, 40, 0), (64, 1000, 0), (3001, 24, 1)])
 def test_batchnorm_relu(rows, c, relu, dtype):
