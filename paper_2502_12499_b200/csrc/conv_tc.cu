@@ -594,6 +594,135 @@ tc_conv_wgrad_kernel(const __grid_constant__ CUtensorMap map_dz, const __grid_co
     }
 }
 
+// ------------------------------------------------------------------------------------------------
+// wgrad for 64 input channels, 3x3, padding 1.  The generic kernel needs one TMA box per (tap,
+// channel block) and pads c_out = 64 to a 128-row tile; here the roles are swapped and the taps
+// share their loads:
+//   D[(tap pair, c_in) = 128 rows][c_out tile = 64 columns] += X_pair^T * dZ   over the pixels of a tile
+// Per pixel tile (8 wide x th high, one image) the CTA loads the dz tile once and three copies of
+// the input patch (one per horizontal tap offset, with a one-row halo above and below); a vertical
+// offset is a whole number of 1024-byte swizzle atoms, so each tap is an aligned descriptor into a
+// copy.  An MN-major operand is a pair of 64-element blocks `LBO` bytes apart, so two taps form one
+// 128-row A operand: (r,0)+(r,1) are one copy apart, (0,2)+(1,2) one atom apart, and (2,2) is
+// paired with rows that are never read back.  Five accumulators of 64 columns live in TMEM.
+// ------------------------------------------------------------------------------------------------
+struct W64Params {
+    int H, W, N, c_out;
+    int th, tiles_w, tiles_h, m_tiles;
+    int slices;                  // persistent CTAs per output-channel tile
+    int stages;
+    uint32_t dz_bytes, box_stride, stage_bytes;
+};
+
+__global__ void __launch_bounds__(kThreads, 1)
+tc_wgrad_c64_kernel(const __grid_constant__ CUtensorMap map_dz, const __grid_constant__ CUtensorMap map_x,
+                    float* __restrict__ partial, W64Params p, int* status) {
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    const uint32_t bars = base + (uint32_t)p.stages * p.stage_bytes;
+    __shared__ uint32_t tmem_base_slot;
+    __shared__ int failed_flag;
+    volatile int* failed = &failed_flag;
+    auto full_bar = [&](int s) { return bars + 8u * s; };
+    auto empty_bar = [&](int s) { return bars + 8u * (kMaxStages + s); };
+    const uint32_t accum_bar = bars + 8u * (2 * kMaxStages);
+
+    const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
+    const int slice = blockIdx.x, co_tile = blockIdx.y;
+    const int my_tiles = slice < p.m_tiles ? (p.m_tiles - slice + p.slices - 1) / p.slices : 0;
+    const uint32_t patch_bytes = (uint32_t)(8 * (p.th + 2)) * 128;
+
+    if (threadIdx.x == 0) {
+        failed_flag = 0;
+        for (int s = 0; s < p.stages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+        mbar_init(accum_bar, 1);
+        fence_barrier_init();
+        tma_prefetch_desc(&map_dz);
+        tma_prefetch_desc(&map_x);
+    }
+    if (warp == 1) tmem_alloc(smem_u32(&tmem_base_slot), 512);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = tmem_base_slot;
+
+    if (warp == 0) {
+        int issued = 0;
+        for (int j = 0; j < my_tiles; ++j) {
+            const int s = j % p.stages;
+            const uint32_t phase = (uint32_t)(j / p.stages) & 1u;
+            if (!mbar_wait(empty_bar(s), phase ^ 1u, failed, status, 401)) break;
+            int t = slice + j * p.slices;
+            const int w0 = (t % p.tiles_w) * 8; t /= p.tiles_w;
+            const int h0 = (t % p.tiles_h) * p.th;
+            const int img = t / p.tiles_h;
+            if (lane == 0) mbar_expect_tx(full_bar(s), p.dz_bytes + 3 * patch_bytes);
+            __syncwarp();
+            const uint32_t dst = base + (uint32_t)s * p.stage_bytes;
+            if (lane == 0) tma_load_4d(dst, &map_dz, full_bar(s), co_tile * 64, w0, h0, img);
+            else if (lane < 4) tma_load_4d(dst + p.dz_bytes + (lane - 1) * p.box_stride, &map_x, full_bar(s), 0, w0 + lane - 2, h0 - 1, img);
+            issued = j + 1;
+        }
+        if (*failed && lane == 0)
+            for (int j = max(0, issued - p.stages); j < issued; ++j) mbar_drain(full_bar(j % p.stages), (uint32_t)(j / p.stages) & 1u);
+    } else if (warp == 1 && lane == 0) {
+        const uint32_t idesc = instr_desc(128, 64, 1, 1);
+        const int ksteps = p.th / 2;                 // 16 pixels (two 8-pixel rows) per MMA
+        bool ok = true;
+        for (int j = 0; j < my_tiles && ok; ++j) {
+            const int s = j % p.stages;
+            const uint32_t phase = (uint32_t)(j / p.stages) & 1u;
+            if (!mbar_wait(full_bar(s), phase, failed, status, 402)) { ok = false; break; }
+            tc_fence_after();
+            const uint32_t dz_addr = base + (uint32_t)s * p.stage_bytes;
+            const uint32_t x_addr = dz_addr + p.dz_bytes;
+#pragma unroll 1
+            for (int pair = 0; pair < 5; ++pair) {
+                // first tap of the pair and the distance to the second one
+                const uint32_t a0 = pair < 3 ? x_addr + (uint32_t)pair * 1024                       // (r = pair, s = 0) + (r, 1)
+                                  : pair == 3 ? x_addr + 2 * p.box_stride                           // (0, 2) + (1, 2)
+                                              : x_addr + 2 * p.box_stride + 2 * 1024;               // (2, 2) + unused rows
+                const uint32_t lbo = pair < 3 ? p.box_stride : 1024u;
+                for (int kk = 0; kk < ksteps; ++kk)
+                    umma_bf16(tmem_base + (uint32_t)pair * 64, smem_desc(a0 + kk * 2048, lbo, 1024), smem_desc(dz_addr + kk * 2048, 8192, 1024),
+                              idesc, (j > 0 || kk > 0) ? 1u : 0u);
+            }
+            umma_commit(empty_bar(s));
+        }
+        if (ok) umma_commit(accum_bar);
+    } else if (warp >= 2) {
+        const int quarter = warp % 4;
+        const int row = quarter * 32 + lane;         // (tap of the pair) * 64 + c_in
+        const int half = row / 64, ci = row % 64;
+        if (my_tiles > 0 && mbar_wait(accum_bar, 0, failed, status, 403)) {
+            tc_fence_after();
+            for (int pair = 0; pair < 5; ++pair) {
+                const int tap = pair < 3 ? pair * 3 + half : (pair == 3 ? 2 + 3 * half : 8);
+                const bool valid = !(pair == 4 && half == 1);
+                float* dst = partial + (((size_t)slice * p.c_out + (size_t)co_tile * 64) * 9 + tap) * 64 + ci;
+#pragma unroll
+                for (int c0 = 0; c0 < 64; c0 += 32) {
+                    uint32_t v[32];
+                    tmem_ld32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(pair * 64 + c0), v);
+                    if (valid) {
+#pragma unroll
+                        for (int e = 0; e < 32; ++e) dst[(size_t)(c0 + e) * 576] = __uint_as_float(v[e]);
+                    }
+                }
+            }
+        } else if (my_tiles == 0) {
+            for (int i = threadIdx.x - 64; i < 64 * 576; i += 128) partial[((size_t)slice * p.c_out + (size_t)co_tile * 64) * 576 + i] = 0.f;
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        __syncwarp();
+        tc_fence_after();
+        tmem_dealloc(tmem_base, 512);
+    }
+}
+
 // wt[ci][tap'][co] = w[co][taps-1-tap'][ci]: the matrix of the transposed convolution (stride 1).
 __global__ void transpose_flip_kernel(const __nv_bfloat16* __restrict__ w, __nv_bfloat16* __restrict__ wt, int c_out, int taps, int c_in) {
     const int64_t total = (int64_t)c_out * taps * c_in;
@@ -603,6 +732,18 @@ __global__ void transpose_flip_kernel(const __nv_bfloat16* __restrict__ w, __nv_
         const int tap = (int)(t % taps), ci = (int)(t / taps);
         wt[i] = w[((size_t)co * taps + (taps - 1 - tap)) * c_in + ci];
     }
+}
+
+// k = 1: plain [c_out][c_in] -> [c_in][c_out] transpose through a 64x64 shared tile (both sides coalesced)
+__global__ void __launch_bounds__(256) transpose_tile_kernel(const __nv_bfloat16* __restrict__ w, __nv_bfloat16* __restrict__ wt, int c_out, int c_in) {
+    __shared__ __nv_bfloat16 tile[64][66];
+    const int ci0 = blockIdx.x * 64, co0 = blockIdx.y * 64;
+    const int tx = threadIdx.x % 64, ty = threadIdx.x / 64;
+    for (int r = ty; r < 64; r += 4)
+        if (co0 + r < c_out && ci0 + tx < c_in) tile[r][tx] = w[(size_t)(co0 + r) * c_in + ci0 + tx];
+    __syncthreads();
+    for (int r = ty; r < 64; r += 4)
+        if (ci0 + r < c_in && co0 + tx < c_out) wt[(size_t)(ci0 + r) * c_out + co0 + tx] = tile[tx][r];
 }
 
 __global__ void slice_sum_tc_kernel(const float* __restrict__ partial, float* __restrict__ out, int64_t elems, int slices) {
@@ -717,6 +858,10 @@ int launch_fwd_like(const void* x, const void* w_mat, void* out, const float* bi
     choose_tile(128, W, H, N, &p.tw, &p.th, &p.tn);
     p.tiles_w = (W + p.tw - 1) / p.tw; p.tiles_h = (H + p.th - 1) / p.th; p.tiles_n = (N + p.tn - 1) / p.tn;
     p.bn = pick_bn(c_out);
+    {   // few pixel tiles (fully connected layers): narrower channel tiles give every SM a share of the matrix
+        const int64_t m_tiles = (int64_t)p.tiles_w * p.tiles_h * p.tiles_n;
+        while (p.bn > 64 && m_tiles * ((c_out + p.bn - 1) / p.bn) < 148) p.bn /= 2;
+    }
     p.n_tiles = (c_out + p.bn - 1) / p.bn;
     const uint32_t stage_bytes = 128 * 128 + p.bn * 128;
     p.stages = std::min<int>(kMaxStages, kSmemBudget / stage_bytes);
@@ -772,6 +917,27 @@ void wgrad_plan(const ConvGeom& g, WgradParams* p, int* slices, int* groups, int
 
 }  // namespace
 
+namespace {
+bool wgrad_c64_applies(const ConvGeom& g) { return g.cin == 64 && g.k == 3 && g.pad == 1 && g.cout % 64 == 0; }
+void wgrad_c64_plan(const ConvGeom& g, W64Params* p) {
+    p->H = g.h; p->W = g.w; p->N = g.n; p->c_out = g.cout;
+    const int nt = (g.h + 15) / 16;
+    p->th = ((g.h + nt - 1) / nt + 1) / 2 * 2;                   // even: an MMA spans two 8-pixel rows
+    p->tiles_h = (g.h + p->th - 1) / p->th;
+    p->tiles_w = (g.w + 7) / 8;
+    p->m_tiles = p->tiles_w * p->tiles_h * g.n;
+    int sms = 148, dev = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    p->slices = std::max(1, std::min(sms / (g.cout / 64), p->m_tiles));
+    p->dz_bytes = (uint32_t)(8 * p->th) * 128;
+    // the unused partner of tap (2,2) starts 3 rows into a copy: keep its reads inside the copy's slot
+    p->box_stride = (uint32_t)align_up((int64_t)(8 * (p->th + 3)) * 128, 1024);
+    p->stage_bytes = p->dz_bytes + 3 * p->box_stride;
+    p->stages = std::max(2, std::min<int>(4, (int)((210 * 1024) / p->stage_bytes)));
+}
+}  // namespace
+
 bool tc_conv_supported(int dtype, const ConvGeom& g) {
     if (dtype != CKPT_DTYPE_BF16) return false;
     if (g.stride != 1) return false;
@@ -785,6 +951,11 @@ bool tc_conv_supported(int dtype, const ConvGeom& g) {
 }
 
 int64_t tc_conv_scratch_bytes(const ConvGeom& g) {
+    if (wgrad_c64_applies(g)) {
+        W64Params q;
+        wgrad_c64_plan(g, &q);
+        return (int64_t)q.slices * g.cout * 576 * 4;      // also covers the transposed matrix of the dgrad
+    }
     WgradParams p;
     int slices, groups, co_tiles;
     wgrad_plan(g, &p, &slices, &groups, &co_tiles);
@@ -807,8 +978,13 @@ int tc_conv_dgrad(const ConvGeom& g, const void* dz, const void* w, void* dx, vo
     const int64_t elems = (int64_t)g.cout * taps * g.cin;
     if (!scratch || scratch_bytes < elems * 2) { set_error("dgrad scratch too small"); return CKPT_E_WORKSPACE; }
     cudaStream_t st = (cudaStream_t)stream;
-    const unsigned grid = (unsigned)std::min<int64_t>((elems + 255) / 256, 148 * 8);
-    transpose_flip_kernel<<<grid, 256, 0, st>>>((const __nv_bfloat16*)w, (__nv_bfloat16*)scratch, g.cout, taps, g.cin);
+    if (taps == 1) {
+        dim3 tgrid((g.cin + 63) / 64, (g.cout + 63) / 64);
+        transpose_tile_kernel<<<tgrid, 256, 0, st>>>((const __nv_bfloat16*)w, (__nv_bfloat16*)scratch, g.cout, g.cin);
+    } else {
+        const unsigned grid = (unsigned)std::min<int64_t>((elems + 255) / 256, 148 * 8);
+        transpose_flip_kernel<<<grid, 256, 0, st>>>((const __nv_bfloat16*)w, (__nv_bfloat16*)scratch, g.cout, taps, g.cin);
+    }
     CKPT_LAUNCH_CHECK("dgrad matrix transpose");
     return launch_fwd_like(dz, scratch, dx, nullptr, 0, g.n, g.h, g.w, g.cout, g.cin, g.k, g.k - 1 - g.pad, device_status, st,
                            "conv dgrad (tensor cores)");
@@ -817,6 +993,31 @@ int tc_conv_dgrad(const ConvGeom& g, const void* dz, const void* w, void* dx, vo
 int tc_conv_wgrad(const ConvGeom& g, const void* dz, const void* x, float* dw, void* scratch, int64_t scratch_bytes,
                   int* device_status, void* stream) {
     if (!device_status) { set_error("no status word"); return CKPT_E_NULL; }
+    if (wgrad_c64_applies(g)) {
+        W64Params p;
+        wgrad_c64_plan(g, &p);
+        const int64_t elems = (int64_t)g.cout * 576;
+        if (!scratch || scratch_bytes < (int64_t)p.slices * elems * 4) { set_error("wgrad scratch too small"); return CKPT_E_WORKSPACE; }
+        CUtensorMap mdz, mx;
+        int rc = make_act_map(&mdz, dz, g.n, g.h, g.w, g.cout, 8, p.th, 1);
+        if (rc) return rc;
+        rc = make_act_map(&mx, x, g.n, g.h, g.w, 64, 8, p.th + 2, 1);
+        if (rc) return rc;
+        cudaStream_t st = (cudaStream_t)stream;
+        static bool attr_set = false;
+        if (!attr_set) {
+            cudaError_t e = cudaFuncSetAttribute(tc_wgrad_c64_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 222 * 1024);
+            if (e != cudaSuccess) return cuda_fail(e, "raising the shared-memory limit");
+            attr_set = true;
+        }
+        const size_t smem = (size_t)p.stages * p.stage_bytes + 1024 + 256;
+        dim3 grid(p.slices, g.cout / 64);
+        tc_wgrad_c64_kernel<<<grid, kThreads, smem, st>>>(mdz, mx, (float*)scratch, p, device_status);
+        CKPT_LAUNCH_CHECK("conv wgrad, 64 input channels (tensor cores)");
+        slice_sum_tc_kernel<<<(unsigned)((elems + 255) / 256), 256, 0, st>>>((const float*)scratch, dw, elems, p.slices);
+        CKPT_LAUNCH_CHECK("wgrad slice sum");
+        return CKPT_OK;
+    }
     WgradParams p;
     int slices, groups, co_tiles;
     wgrad_plan(g, &p, &slices, &groups, &co_tiles);
