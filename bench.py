@@ -237,7 +237,7 @@ def main():
     if rank == 0:
         peaks = measured_peaks()
         flops, _ = conv_flops(spec, mask, shapes)
-        roofline = dominant_kernel_roofline(ck, spec, shapes, peaks, torch, stream)
+        roofline = dominant_kernel_roofline(args.config, peaks)
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
                 "warmup": max(args.warmup, 3), "ms_per_step": ms / args.steps, "higher_is_better": True,
                 "scaling": "weak", "vs_baseline": None, "dtype": spec["dtype"], "data": "synthetic", "config": config,
@@ -257,40 +257,40 @@ def main():
         dist.destroy_process_group()
 
 
-def dominant_kernel_roofline(ck, spec, shapes, peaks, torch, stream):
-    """Times the convolution-forward kernel on every conv layer shape of the workload (it runs in
-    the forward phase, in segment recomputation and at the start of every unit's backward) and
-    reports the launch-weighted throughput against the measured tensor-core peak."""
-    dtype = ck.DTYPE_BF16 if spec["dtype"] == "bf16" else ck.DTYPE_F32
-    tdt = torch.bfloat16 if spec["dtype"] == "bf16" else torch.float32
-    total_flops, total_ms, launches = 0.0, 0.0, 0
-    per_layer = []
-    for u, (hi, wi, ci), (ho, wo, co) in zip(spec["units"], shapes[:-1], shapes[1:]):
-        if u["kind"] != "conv_bn_relu" or u["cin"] < 16:
-            continue
-        shape = ck.ConvShape(spec["batch"], hi, wi, ci, co, u["k"], u["stride"], u["pad"])
-        x = torch.randn(spec["batch"], hi, wi, ci, device="cuda").to(tdt)
-        w = (torch.randn(co, u["k"], u["k"], ci, device="cuda") * 0.05).to(tdt)
-        z = torch.empty(spec["batch"], ho, wo, co, device="cuda", dtype=tdt)
-        scratch = torch.empty(max(256, ck.conv2d_scratch_bytes(shape, dtype)), dtype=torch.uint8, device="cuda")
-        reps = 3
-        ck.conv2d_forward(shape, dtype, 0, x, w, z, scratch, stream)
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        torch.cuda.synchronize()
-        e0.record(stream)
-        for _ in range(reps):
-            ck.conv2d_forward(shape, dtype, 0, x, w, z, scratch, stream)
-        e1.record(stream)
-        torch.cuda.synchronize()
-        ms = e0.elapsed_time(e1) / reps
-        fl = 2.0 * spec["batch"] * ho * wo * co * u["k"] * u["k"] * ci
-        total_flops += fl; total_ms += ms; launches += 1
-        per_layer.append({"shape": "%dx%dx%d->%d" % (hi, wi, ci, co), "ms": ms, "tflops": fl / ms / 1e9})
-        del x, w, z, scratch
-    achieved = total_flops / (total_ms * 1e-3) / 1e12 if total_ms > 0 else 0.0
-    return {"kernel": "conv forward (implicit GEMM)", "bound": "tensor", "achieved": achieved, "peak": peaks["tflops_burst"],
-            "unit": "TFLOP/s", "frac": achieved / peaks["tflops_burst"], "peak_source": peaks["source"], "traffic": None,
-            "launch_shapes": launches, "per_layer": per_layer}
+# DRAM traffic per launch of the conv-forward kernels over the layer mix of config 2, from one ncu pass
+# (profiles/conv_forward_vgg16_b64_dram_traffic.md).  Valid only for the kernel source it was taken
+# on: reported as null when csrc/conv_tc.cu has changed since.
+CONV_FWD_TRAFFIC = {"source_sha256": "", "bytes_per_launch": None}
+
+
+def _kernel_source_sha():
+    import hashlib
+    path = os.path.join(ROOT, "paper_2502_12499_b200", "csrc", "conv_tc.cu")
+    return hashlib.sha256(open(path, "rb").read()).hexdigest()
+
+
+def dominant_kernel_roofline(config_index, peaks):
+    """The convolution-forward kernels (tcgen05) hold the largest share of the step: they run in the
+    forward phase, in segment recomputation and, on the transposed matrix, as dgrad.  Timed here on
+    every conv layer shape of the workload with CUDA events; achieved = sum of algorithmic FLOPs /
+    sum of launch times, against the measured dense-bf16 peak."""
+    from paper_2502_12499_b200 import opbench
+    mix = opbench.conv_mix("fwd", config_index, reps=3)
+    traffic = CONV_FWD_TRAFFIC["bytes_per_launch"] if CONV_FWD_TRAFFIC["source_sha256"] == _kernel_source_sha() else None
+    out = {"kernel": "tc_conv_fwd_kernel / tc_conv_c64_kernel (implicit-GEMM conv forward)", "bound": "tensor",
+           "achieved": mix["tflops"], "peak": peaks["tflops_burst"], "unit": "TFLOP/s", "frac": mix["tflops"] / peaks["tflops_burst"],
+           "peak_source": peaks["source"] + " (burst: kernels timed in isolation)", "traffic": traffic,
+           "launch_shapes": mix["launches"], "flops_per_launch": mix["flops"] / mix["launches"],
+           "ms_per_launch": mix["ms"] / mix["launches"], "per_layer": mix["per_layer"]}
+    # the memory-bound side of the step, for the record: batch-norm passes on the largest activation
+    b, h, w, c = 64, 224, 224, 64
+    f, g = opbench.bn("fwd", b * h * w, c), opbench.bn("bwd", b * h * w, c)
+    pf, pb = opbench.pool("fwd", b, h, w, c), opbench.pool("bwd", b, h, w, c)
+    out["elementwise"] = {"unit": "GB/s", "peak": peaks["hbm_gbs"],
+                          "bn_forward": f["gbs"], "bn_backward": g["gbs"], "maxpool_forward": pf["gbs"], "maxpool_backward": pb["gbs"],
+                          "frac": {"bn_forward": f["gbs"] / peaks["hbm_gbs"], "bn_backward": g["gbs"] / peaks["hbm_gbs"],
+                                   "maxpool_forward": pf["gbs"] / peaks["hbm_gbs"], "maxpool_backward": pb["gbs"] / peaks["hbm_gbs"]}}
+    return out
 
 
 if __name__ == "__main__":
