@@ -1,0 +1,126 @@
+"""Full-size checks, in the launch configuration bench.py times.
+
+* the tensor-core convolution kernels at the VGG-16 / batch-64 layer shapes, on sampled outputs that
+  the oracle computes one by one (a cropped neighbourhood for forward/dgrad, one (c_out, c_in)
+  channel pair over all pixels for wgrad);
+* the whole checkpointed step of configurations 2 and 5 through properties that hold at any size:
+  arena high-water == highest offset == planner's prediction (arena of exactly that size),
+  gradients bit-identical between the checkpointed and the store-all schedule, finite loss."""
+import time
+
+import numpy as np
+import pytest
+
+from oracle import numeric_oracle as no
+from paper_2502_12499_b200 import binding as ck
+from paper_2502_12499_b200 import workloads as wl
+from tests.gpu_util import StepRunner
+
+pytestmark = pytest.mark.gpu
+
+LAYERS = [
+    # n, h, w, cin, cout   (3x3, stride 1, padding 1)
+    (64, 224, 224, 64, 64),
+    (64, 112, 112, 64, 128),
+    (64, 112, 112, 128, 128),
+    (64, 56, 56, 256, 256),
+    (64, 28, 28, 512, 512),
+    (64, 14, 14, 512, 512),
+    (32, 56, 56, 64, 64),        # the unit of the 1000-layer chain
+]
+
+
+def bf16_host(t):
+    """Exact float64 copy of a bf16 device tensor."""
+    return t.float().cpu().numpy().astype(np.float64)
+
+
+@pytest.mark.parametrize("layer", LAYERS, ids=lambda l: "x".join(map(str, l)))
+def test_conv_kernels_full_size_sampled(layer):
+    import torch
+    n, h, w, cin, cout = layer
+    dt = ck.DTYPE_BF16
+    gen = torch.Generator(device="cuda").manual_seed(n * h + cin)
+    x = torch.randn(n, h, w, cin, device="cuda", generator=gen).bfloat16()
+    wt = (torch.randn(cout, 3, 3, cin, device="cuda", generator=gen) / (3.0 * cin ** 0.5)).bfloat16()
+    dz = torch.randn(n, h, w, cout, device="cuda", generator=gen).bfloat16()
+    shape = ck.ConvShape(n, h, w, cin, cout, 3, 1, 1)
+    scratch = torch.empty(max(256, ck.conv2d_scratch_bytes(shape, dt)), dtype=torch.uint8, device="cuda")
+    z = torch.empty(n, h, w, cout, device="cuda", dtype=torch.bfloat16)
+    dx = torch.empty_like(x)
+    dw = torch.empty(cout, 3, 3, cin, device="cuda")
+    ck.conv2d_forward(shape, dt, 0, x, wt, z, scratch)
+    ck.conv2d_dgrad(shape, dt, 0, dz, wt, dx, scratch)
+    ck.conv2d_wgrad(shape, dt, 0, dz, x, dw, scratch)
+    torch.cuda.synchronize()
+    w64 = bf16_host(wt)
+    rng = np.random.default_rng(7)
+    # corners, edges (tile and image borders) and random interior pixels
+    picks = [(0, 0, 0), (n - 1, h - 1, w - 1), (n // 2, 0, w - 1), (n - 1, h - 1, 0), (1, h // 2, w // 2 + 1)]
+    picks += [(int(rng.integers(n)), int(rng.integers(h)), int(rng.integers(w))) for _ in range(11)]
+    scale_z = float(z.float().abs().max())
+    scale_dx = float(dx.float().abs().max())
+    for (b, i, j) in picks:
+        lo_i, hi_i, lo_j, hi_j = max(i - 2, 0), min(i + 3, h), max(j - 2, 0), min(j + 3, w)
+        xc = bf16_host(x[b:b + 1, lo_i:hi_i, lo_j:hi_j, :])
+        dzc = bf16_host(dz[b:b + 1, lo_i:hi_i, lo_j:hi_j, :])
+        z_ref = no.conv2d_fwd(xc, w64, 1, 1)[0, i - lo_i, j - lo_j, :]
+        dx_ref = no.conv2d_bwd(xc, w64, dzc, 1, 1)[0][0, i - lo_i, j - lo_j, :]
+        assert np.abs(bf16_host(z[b, i, j, :]) - z_ref).max() <= 6e-3 * scale_z
+        assert np.abs(bf16_host(dx[b, i, j, :]) - dx_ref).max() <= 6e-3 * scale_dx
+    scale_dw = float(dw.abs().max())
+    for _ in range(3):
+        co, ci = int(rng.integers(cout)), int(rng.integers(cin))
+        xs = bf16_host(x[..., ci:ci + 1])
+        dzs = bf16_host(dz[..., co:co + 1])
+        dw_ref = no.conv2d_bwd(xs, np.zeros((1, 3, 3, 1)), dzs, 1, 1)[1][0, :, :, 0]
+        assert np.abs(dw[co, :, :, ci].cpu().numpy().astype(np.float64) - dw_ref).max() <= 2e-5 * max(scale_dw, np.abs(dw_ref).max())
+
+
+def step_properties(spec, seed=0):
+    import torch
+    params = wl.make_params(spec, seed=seed)
+    x, labels = wl.make_batch(spec, seed=seed + 1)
+    runner = StepRunner(spec, params)
+    del params
+    d = runner.d
+    mask, peak = ck.plan(ck.ALGO_DYNAMIC_N, d)
+    if spec["loss"] != "softmax_ce":
+        labels = None
+    rep, g = runner.run(ck.POLICY_DYNAMIC, mask, x, labels)
+    assert rep["peak_bytes"] == rep["extent_bytes"] == rep["predicted_bytes"] == peak
+    assert rep["device_status"] == 0 and np.isfinite(rep["loss"])
+    assert rep["recomputed_units"] == runner.n + 1 - int(mask.sum())
+    rep0, g0 = runner.run(ck.POLICY_STORE_ALL, None, x, labels)
+    assert rep0["peak_bytes"] == int(d.sum())
+    assert rep0["loss"] == rep["loss"]
+    for a, b in zip(g, g0):
+        assert np.all(np.isfinite(a))
+        assert np.array_equal(a, b)                     # checkpointed == store-all, bit for bit
+    mask3, peak3 = ck.plan(ck.ALGO_STATIC_N3, d)
+    rep3, g3 = runner.run(ck.POLICY_STATIC, mask3, x, labels)
+    assert rep3["peak_bytes"] == rep3["extent_bytes"] == peak3
+    for a, b in zip(g3, g0):
+        assert np.array_equal(a, b)
+    torch.cuda.empty_cache()
+    return rep, rep0, peak
+
+
+def test_config2_vgg16_full_size_step():
+    rep, rep0, peak = step_properties(wl.config(2))
+    assert peak < 0.65 * rep0["peak_bytes"]             # 1.17 GiB against 1.82 GiB
+    assert abs(rep["loss"] - np.log(1000.0)) < 2.0      # random labels, random weights
+
+
+def test_config5_plain1000_full_size_step():
+    spec = wl.config(5)
+    chain = ck.Chain(spec)
+    d = chain.sizes()
+    t0 = time.perf_counter(); m6, p6 = ck.plan(ck.ALGO_DYNAMIC_N, d); t6 = time.perf_counter() - t0
+    t0 = time.perf_counter(); m5, p5 = ck.plan(ck.ALGO_DYNAMIC_N2, d); t5 = time.perf_counter() - t0
+    t0 = time.perf_counter(); m3, p3 = ck.plan(ck.ALGO_STATIC_N3, d); t3 = time.perf_counter() - t0
+    assert p6 == p5 == 47 * int(d[1]) and np.array_equal(m6, m5)
+    assert p3 == 64 * int(d[1])
+    assert t6 < t3                                      # the O(n) planner beats the O(n^3) one at n = 1000
+    rep, rep0, peak = step_properties(spec)
+    assert rep0["peak_bytes"] > 20 * peak               # 12 GiB stored against 0.56 GiB checkpointed
