@@ -77,7 +77,7 @@ def test_conv_kernels_full_size_sampled(layer):
         assert np.abs(dw[co, :, :, ci].cpu().numpy().astype(np.float64) - dw_ref).max() <= 2e-5 * max(scale_dw, np.abs(dw_ref).max())
 
 
-def step_properties(spec, seed=0):
+def step_properties(spec, seed=0, finite_last_units=None):
     import torch
     params = wl.make_params(spec, seed=seed)
     x, labels = wl.make_batch(spec, seed=seed + 1)
@@ -94,14 +94,15 @@ def step_properties(spec, seed=0):
     rep0, g0 = runner.run(ck.POLICY_STORE_ALL, None, x, labels)
     assert rep0["peak_bytes"] == int(d.sum())
     assert rep0["loss"] == rep["loss"]
-    for a, b in zip(g, g0):
-        assert np.all(np.isfinite(a))
-        assert np.array_equal(a, b)                     # checkpointed == store-all, bit for bit
+    for (ui, name, _), a, b in zip(runner.flat, g, g0):
+        if finite_last_units is None or ui >= runner.n - finite_last_units:
+            assert np.all(np.isfinite(a)), (ui, name)
+        assert np.array_equal(a, b, equal_nan=True)     # checkpointed == store-all, bit for bit
     mask3, peak3 = ck.plan(ck.ALGO_STATIC_N3, d)
     rep3, g3 = runner.run(ck.POLICY_STATIC, mask3, x, labels)
     assert rep3["peak_bytes"] == rep3["extent_bytes"] == peak3
     for a, b in zip(g3, g0):
-        assert np.array_equal(a, b)
+        assert np.array_equal(a, b, equal_nan=True)
     torch.cuda.empty_cache()
     return rep, rep0, peak
 
@@ -122,5 +123,9 @@ def test_config5_plain1000_full_size_step():
     assert p6 == p5 == 47 * int(d[1]) and np.array_equal(m6, m5)
     assert p3 == 64 * int(d[1])
     assert t6 < t3                                      # the O(n) planner beats the O(n^3) one at n = 1000
-    rep, rep0, peak = step_properties(spec)
+    # A BN+ReLU chain at random initialisation multiplies the gradient norm by about 1.18 per unit on
+    # the way back (measured on the float64 oracle), i.e. by 1e70 over 1000 units: the gradients of
+    # the early units lie outside the float32/bfloat16 range in any implementation.  They overflow
+    # identically under every schedule; finiteness is required of the last 300 units only.
+    rep, rep0, peak = step_properties(spec, finite_last_units=300)
     assert rep0["peak_bytes"] > 20 * peak               # 12 GiB stored against 0.56 GiB checkpointed
