@@ -273,6 +273,7 @@ static int run_step(StepCtx& c, double* loss_out) {
     // ---------------- backward phase
     bool have_r = false;            // Algorithm 4: a per-segment gradient buffer is live in the arena
     bool g_in_r = false;            // the current gradient lives in that buffer
+    bool bypass_r_once = false;     // first hop of a segment with an odd number of hops goes carry -> carry
     std::vector<int64_t> live_segment;
     for (int64_t i = n; i >= 1; --i) {
         if (!store_all && c.is_ckpt[i]) {
@@ -303,14 +304,19 @@ static int run_step(StepCtx& c, double* loss_out) {
                 for (int64_t k = h; k < i; ++k) r = std::max(r, d[k]);
                 if ((rc = A.alloc_stack(kGradId, r, &off))) return rc;
                 have_r = true;
+                // The gradient alternates between the segment's buffer and a carry buffer, one hop per
+                // unit.  It has to sit in a carry buffer when the segment ends (its buffer is released
+                // then), so a segment with an odd number of hops starts with one carry -> carry hop.
+                bypass_r_once = h > 0 && ((i - h) % 2 == 1);
             }
         }
         // where the outgoing gradient goes: the segment's buffer (Algorithm 4) or the other carry buffer
         void* g_next;
         bool next_in_r = false;
-        if (c.policy == CKPT_POLICY_DYNAMIC && !g_in_r) { g_next = ptr(kGradId); next_in_r = true; }
-        else if (c.policy == CKPT_POLICY_DYNAMIC) g_next = gbuf[0];
+        if (c.policy == CKPT_POLICY_DYNAMIC && !g_in_r && !bypass_r_once) { g_next = ptr(kGradId); next_in_r = true; }
+        else if (c.policy == CKPT_POLICY_DYNAMIC && g_in_r) g_next = gbuf[0];
         else g_next = (g_cur == gbuf[0]) ? gbuf[1] : gbuf[0];
+        bypass_r_once = false;
         const bool need_dx = i > 1;   // the gradient w.r.t. the input batch is never used
         if ((rc = unit_backward(c, i, ptr(i - 1), ptr(i), g_cur, need_dx ? g_next : nullptr))) return rc;
         if (need_dx) { g_cur = g_next; g_in_r = next_in_r; }
