@@ -19,6 +19,8 @@ struct Unit {
     int param_first = 0, n_params = 0;
     int64_t stats_off = 0;       // float offset of this unit's saved batch statistics
     ConvGeom geom;               // conv / fc as a convolution
+    // bottleneck block: its four convolutions (1x1, 3x3 with the stride, 1x1, projection 1x1 with the stride)
+    ConvGeom g1, g2, g3, gp;
 };
 
 struct ParamInfo { int64_t unit, elems; int32_t dtype; };
@@ -34,7 +36,7 @@ struct ckpt_chain {
     int dtype = 0, loss = 0, impl = 0;
     // workspace layout (byte offsets)
     int64_t max_d = 0, off_g0 = 0, off_g1 = 0, off_z = 0, off_scr = 0, scr_bytes = 0, off_stats = 0,
-            off_misc = 0, ws_bytes = 0;
+            off_misc = 0, off_blk = 0, blk_bytes = 0, ws_bytes = 0;
 };
 
 namespace ckpt {
@@ -114,6 +116,98 @@ static int activated(StepCtx& c, int64_t j, const void* raw, const void** out) {
     return bn_apply(c.ch->dtype, rows_of(c.ch, j), c.ch->shapes[j].c, raw, stats_of(c, j), 1, xbuf, c.stream);
 }
 
+// ---------------------------------------------------------------------------------------------
+// Bottleneck block (ResNet v1.5): z1 = conv1x1(x), a = relu(bn1(z1)), z2 = conv3x3_stride(a),
+// b = relu(bn2(z2)), z3 = conv1x1(b), shortcut = x or bn_p(conv1x1_stride(x)), y = relu(bn3(z3) + shortcut).
+// Only y is chain data; every interior tensor lives in the block region of the workspace and is
+// re-derived from x at the start of the block's backward.
+// ---------------------------------------------------------------------------------------------
+struct BlockBuffers {
+    char *z1, *a, *da, *z2, *b, *db, *z3, *zp, *t0, *t1, *dxs;
+    float *s1, *s2, *s3, *sp;       // statistics blocks of the four normalisations
+};
+static BlockBuffers block_buffers(StepCtx& c, const Unit& u) {
+    const int64_t es = dtype_size(c.ch->dtype);
+    const int64_t in_px = c.ch->batch * u.in.h * u.in.w, out_px = c.ch->batch * u.out.h * u.out.w;
+    const int64_t m_in = align_up(in_px * u.desc.mid * es, 256), m_out = align_up(out_px * u.desc.mid * es, 256);
+    const int64_t c_out = align_up(out_px * u.out.c * es, 256);
+    BlockBuffers B;
+    char* p = c.ws + c.ch->off_blk;
+    B.z1 = p; p += m_in; B.a = p; p += m_in; B.da = p; p += m_in;
+    B.z2 = p; p += m_out; B.b = p; p += m_out; B.db = p; p += m_out;
+    B.z3 = p; p += c_out; B.zp = p; p += c_out; B.t0 = p; p += c_out; B.t1 = p; p += c_out;
+    B.dxs = p;
+    float* st = (float*)(c.ws + c.ch->off_stats) + u.stats_off;
+    B.s1 = st; B.s2 = st + 4 * u.desc.mid; B.s3 = st + 8 * u.desc.mid; B.sp = B.s3 + 4 * u.out.c;
+    return B;
+}
+
+// z1, a, z2, b, z3 (and zp) with their statistics; the residual join is left to the caller.
+static int block_interiors(StepCtx& c, const Unit& u, const void* x, const BlockBuffers& B) {
+    const int dt = c.ch->dtype;
+    void* const* p = c.params + u.param_first;
+    char* scr = c.ws + c.ch->off_scr;
+    const int64_t in_px = c.ch->batch * u.in.h * u.in.w, out_px = c.ch->batch * u.out.h * u.out.w;
+    const int mid = u.desc.mid, co = u.out.c;
+    int rc;
+    if ((rc = conv_forward_any(c, u.g1, x, p[0], B.z1, nullptr, 0))) return rc;
+    if ((rc = bn_statistics(dt, in_px, mid, B.z1, (const float*)p[1], (const float*)p[2], B.s1, scr, c.stream))) return rc;
+    if ((rc = bn_apply(dt, in_px, mid, B.z1, B.s1, 1, B.a, c.stream))) return rc;
+    if ((rc = conv_forward_any(c, u.g2, B.a, p[3], B.z2, nullptr, 0))) return rc;
+    if ((rc = bn_statistics(dt, out_px, mid, B.z2, (const float*)p[4], (const float*)p[5], B.s2, scr, c.stream))) return rc;
+    if ((rc = bn_apply(dt, out_px, mid, B.z2, B.s2, 1, B.b, c.stream))) return rc;
+    if ((rc = conv_forward_any(c, u.g3, B.b, p[6], B.z3, nullptr, 0))) return rc;
+    if ((rc = bn_statistics(dt, out_px, co, B.z3, (const float*)p[7], (const float*)p[8], B.s3, scr, c.stream))) return rc;
+    if (u.desc.flags & 2) {
+        if ((rc = conv_forward_any(c, u.gp, x, p[9], B.zp, nullptr, 0))) return rc;
+        if ((rc = bn_statistics(dt, out_px, co, B.zp, (const float*)p[10], (const float*)p[11], B.sp, scr, c.stream))) return rc;
+    }
+    return CKPT_OK;
+}
+
+static int block_forward(StepCtx& c, const Unit& u, const void* x, void* y) {
+    const BlockBuffers B = block_buffers(c, u);
+    int rc = block_interiors(c, u, x, B);
+    if (rc) return rc;
+    const bool project = (u.desc.flags & 2) != 0;
+    return bn_add_relu(c.ch->dtype, c.ch->batch * u.out.h * u.out.w, u.out.c, B.z3, B.s3, project ? (const void*)B.zp : x,
+                       project ? B.sp : nullptr, y, c.stream);
+}
+
+// g_in = dL/dy (overwritten), g_out = dL/dx or null.
+static int block_backward(StepCtx& c, const Unit& u, const void* x, const void* y, void* g_in, void* g_out) {
+    const int dt = c.ch->dtype;
+    const BlockBuffers B = block_buffers(c, u);
+    void* const* p = c.params + u.param_first;
+    void* const* g = c.grads + u.param_first;
+    char* scr = c.ws + c.ch->off_scr;
+    const int64_t in_px = c.ch->batch * u.in.h * u.in.w, out_px = c.ch->batch * u.out.h * u.out.w;
+    const int mid = u.desc.mid, co = u.out.c;
+    const bool project = (u.desc.flags & 2) != 0;
+    int rc;
+    if ((rc = block_interiors(c, u, x, B))) return rc;
+    // through the final ReLU: g_in <- dL/d(bn3 + shortcut)
+    if ((rc = relu_mask_inplace(dt, out_px * co, g_in, y, c.stream))) return rc;
+    const void* dx_shortcut = g_in;                       // identity shortcut: the same gradient flows to x
+    if (project) {
+        if ((rc = bn_relu_backward(dt, out_px, co, g_in, B.zp, (const float*)p[10], B.sp, 0, B.t0, (float*)g[10], (float*)g[11], scr, c.stream))) return rc;
+        if ((rc = conv_wgrad_any(c, u.gp, B.t0, x, (float*)g[9]))) return rc;
+        if (g_out) { if ((rc = conv_dgrad_any(c, u.gp, B.t0, p[9], B.dxs))) return rc; }
+        dx_shortcut = B.dxs;
+    }
+    if ((rc = bn_relu_backward(dt, out_px, co, g_in, B.z3, (const float*)p[7], B.s3, 0, B.t1, (float*)g[7], (float*)g[8], scr, c.stream))) return rc;
+    if ((rc = conv_wgrad_any(c, u.g3, B.t1, B.b, (float*)g[6]))) return rc;
+    if ((rc = conv_dgrad_any(c, u.g3, B.t1, p[6], B.db))) return rc;
+    if ((rc = bn_relu_backward(dt, out_px, mid, B.db, B.z2, (const float*)p[4], B.s2, 1, B.db, (float*)g[4], (float*)g[5], scr, c.stream))) return rc;
+    if ((rc = conv_wgrad_any(c, u.g2, B.db, B.a, (float*)g[3]))) return rc;
+    if ((rc = conv_dgrad_any(c, u.g2, B.db, p[3], B.da))) return rc;
+    if ((rc = bn_relu_backward(dt, in_px, mid, B.da, B.z1, (const float*)p[1], B.s1, 1, B.da, (float*)g[1], (float*)g[2], scr, c.stream))) return rc;
+    if ((rc = conv_wgrad_any(c, u.g1, B.da, x, (float*)g[0]))) return rc;
+    if (!g_out) return CKPT_OK;
+    if ((rc = conv_dgrad_any(c, u.g1, B.da, p[0], g_out))) return rc;
+    return add_tensors(dt, in_px * u.in.c, g_out, dx_shortcut, g_out, c.stream);
+}
+
 // d_i = f_i(d_{i-1}, w_i)  (Eq. (1)); i is 1-based.
 static int unit_forward(StepCtx& c, int64_t i, const void* x_raw, void* y) {
     if (c.dry) return CKPT_OK;
@@ -144,6 +238,9 @@ static int unit_forward(StepCtx& c, int64_t i, const void* x_raw, void* y) {
         case CKPT_UNIT_FC:
             if ((rc = activated(c, i - 1, x_raw, &x))) return rc;
             return conv_forward_any(c, u.geom, x, p[0], y, (const float*)p[1], u.desc.flags & 1);
+        case CKPT_UNIT_BOTTLENECK:
+            if ((rc = activated(c, i - 1, x_raw, &x))) return rc;
+            return block_forward(c, u, x, y);
     }
     set_error("unit kind %d has no forward kernel", u.desc.kind);
     return CKPT_E_UNSUPPORTED;
@@ -200,6 +297,10 @@ static int unit_backward(StepCtx& c, int64_t i, const void* x_raw, const void* y
             if (g_out && (rc = conv_dgrad_any(c, u.geom, g_in, p[0], g_out))) return rc;
             break;
         }
+        case CKPT_UNIT_BOTTLENECK:
+            if ((rc = activated(c, i - 1, x_raw, &x))) return rc;
+            if ((rc = block_backward(c, u, x, y, g_in, g_out))) return rc;
+            break;
         default:
             set_error("unit kind %d has no backward kernel", u.desc.kind);
             return CKPT_E_UNSUPPORTED;
@@ -452,6 +553,39 @@ int ckpt_chain_create(const ckpt_unit_desc* units, int64_t n, int64_t batch, int
                 if (tc_conv_supported(dtype, u.geom)) scr = std::max(scr, tc_conv_scratch_bytes(u.geom));
                 break;
             }
+            case CKPT_UNIT_BOTTLENECK: {
+                const int mid = u.desc.mid, st = u.desc.stride, co = u.desc.c_out;
+                const bool project = (u.desc.flags & 2) != 0;
+                if (u.desc.c_in != cur.c || mid < 1 || co < 1 || st < 1 || st > 2 || (!project && (co != cur.c || st != 1))) {
+                    set_error("unit %lld: inconsistent bottleneck block", (long long)i); rc = CKPT_E_BAD_ARG; break;
+                }
+                const int ho = out_size(cur.h, 3, st, 1), wo = out_size(cur.w, 3, st, 1);
+                u.out = {ho, wo, co};
+                u.g1 = {(int)batch, cur.h, cur.w, cur.c, cur.h, cur.w, mid, 1, 1, 0};
+                u.g2 = {(int)batch, cur.h, cur.w, mid, ho, wo, mid, 3, st, 1};
+                u.g3 = {(int)batch, ho, wo, mid, ho, wo, co, 1, 1, 0};
+                u.gp = {(int)batch, cur.h, cur.w, cur.c, out_size(cur.h, 1, st, 0), out_size(cur.w, 1, st, 0), co, 1, st, 0};
+                if (project && (u.gp.ho != ho || u.gp.wo != wo)) { set_error("unit %lld: shortcut shape mismatch", (long long)i); rc = CKPT_E_BAD_ARG; break; }
+                const ConvGeom* gs[4] = {&u.g1, &u.g2, &u.g3, &u.gp};
+                for (int q = 0; q < (project ? 4 : 3); ++q) {
+                    const ConvGeom& g = *gs[q];
+                    ch->params.push_back({i, (int64_t)g.cout * g.k * g.k * g.cin, dtype});
+                    ch->params.push_back({i, g.cout, CKPT_DTYPE_F32});
+                    ch->params.push_back({i, g.cout, CKPT_DTYPE_F32});
+                    const int64_t rows = batch * g.ho * g.wo;
+                    scr = std::max(scr, bn_scratch_bytes(rows, g.cout));
+                    scr = std::max(scr, simt_wgrad_scratch_bytes(g));
+                    if (tc_conv_supported(dtype, g)) scr = std::max(scr, tc_conv_scratch_bytes(g));
+                }
+                u.stats_off = stats_floats;
+                stats_floats += 4 * (int64_t)(2 * mid + 2 * co);
+                // interiors and gradient temporaries of one block (see block_buffers)
+                const int64_t in_px = batch * cur.h * cur.w, out_px = batch * ho * wo;
+                const int64_t blk = 3 * align_up(in_px * mid * es, 256) + 3 * align_up(out_px * mid * es, 256) +
+                                    4 * align_up(out_px * co * es, 256) + align_up(in_px * cur.c * es, 256);
+                ch->blk_bytes = std::max(ch->blk_bytes, blk);
+                break;
+            }
             default:
                 set_error("unit %lld: kind %d is not implemented", (long long)i, u.desc.kind);
                 rc = CKPT_E_UNSUPPORTED;
@@ -472,6 +606,7 @@ int ckpt_chain_create(const ckpt_unit_desc* units, int64_t n, int64_t batch, int
     ch->off_scr = o; ch->scr_bytes = align_up(scr, 256); o += ch->scr_bytes;
     ch->off_stats = o; o += align_up(std::max<int64_t>(stats_floats, 1) * 4, 256);
     ch->off_misc = o; o += align_up(128 + 256 + batch * 4, 256);
+    ch->off_blk = o; o += ch->blk_bytes;
     ch->ws_bytes = o;
     *out = ch;
     return CKPT_OK;

@@ -94,6 +94,12 @@ int bn_statistics(int dtype, int64_t rows, int c, const void* z, const float* ga
                   void* scratch, void* stream);
 int bn_apply(int dtype, int64_t rows, int c, const void* z, const float* stats, int relu, void* y, void* stream);
 
+// y = max(z*scale + shift + shortcut, 0); the shortcut is activated data, or pre-normalisation data with
+// its own statistics block (stats_shortcut != null).
+int bn_add_relu(int dtype, int64_t rows, int c, const void* z, const float* stats, const void* shortcut,
+                const float* stats_shortcut, void* y, void* stream);
+int add_tensors(int dtype, int64_t elems, const void* a, const void* b, void* out, void* stream);
+
 // act (may be null): statistics block of the producing conv unit; when given, the pooling kernels
 // read x through its pending normalisation + ReLU.  Only the 2x2/stride-2 kernels can do that.
 bool maxpool_fuses_activation(int dtype, int h, int w, int c, int k, int stride, int pad);

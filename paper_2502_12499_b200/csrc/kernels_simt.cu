@@ -698,6 +698,48 @@ int bn_relu_forward(int dtype, int64_t rows, int c, const void* z, const float* 
     return bn_apply(dtype, rows, c, z, stats, relu, y, stream);
 }
 
+// Residual join of a bottleneck block: y = max(z*scale + shift + shortcut, 0), where the shortcut is
+// either an already activated tensor (stats_sc == nullptr) or a second pre-normalisation tensor with
+// its own scale/shift (projection branch).
+template <typename T>
+__global__ void __launch_bounds__(256) bn_add_relu_kernel(const T* __restrict__ z, const float* __restrict__ stats,
+                                                          const T* __restrict__ sc, const float* __restrict__ stats_sc,
+                                                          int64_t elems, int c, T* __restrict__ y) {
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < elems; i += (int64_t)gridDim.x * blockDim.x) {
+        const int ch = (int)(i % c);
+        float v = fmaf(ld(z + i), stats[2 * c + ch], stats[3 * c + ch]);
+        float s = ld(sc + i);
+        if (stats_sc) s = fmaf(s, stats_sc[2 * c + ch], stats_sc[3 * c + ch]);
+        y[i] = cvt<T>(fmaxf(v + s, 0.f));
+    }
+}
+int bn_add_relu(int dtype, int64_t rows, int c, const void* z, const float* stats, const void* shortcut,
+                const float* stats_shortcut, void* y, void* stream) {
+    const int64_t elems = rows * c;
+    if (dtype == CKPT_DTYPE_BF16)
+        bn_add_relu_kernel<__nv_bfloat16><<<elementwise_grid(elems), 256, 0, (cudaStream_t)stream>>>(
+            (const __nv_bfloat16*)z, stats, (const __nv_bfloat16*)shortcut, stats_shortcut, elems, c, (__nv_bfloat16*)y);
+    else
+        bn_add_relu_kernel<float><<<elementwise_grid(elems), 256, 0, (cudaStream_t)stream>>>(
+            (const float*)z, stats, (const float*)shortcut, stats_shortcut, elems, c, (float*)y);
+    CKPT_LAUNCH_CHECK("residual join");
+    return CKPT_OK;
+}
+
+template <typename T>
+__global__ void __launch_bounds__(256) add_kernel(const T* __restrict__ a, const T* __restrict__ b, T* __restrict__ out, int64_t elems) {
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < elems; i += (int64_t)gridDim.x * blockDim.x)
+        out[i] = cvt<T>(ld(a + i) + ld(b + i));
+}
+int add_tensors(int dtype, int64_t elems, const void* a, const void* b, void* out, void* stream) {
+    if (dtype == CKPT_DTYPE_BF16)
+        add_kernel<__nv_bfloat16><<<elementwise_grid(elems), 256, 0, (cudaStream_t)stream>>>((const __nv_bfloat16*)a, (const __nv_bfloat16*)b, (__nv_bfloat16*)out, elems);
+    else
+        add_kernel<float><<<elementwise_grid(elems), 256, 0, (cudaStream_t)stream>>>((const float*)a, (const float*)b, (float*)out, elems);
+    CKPT_LAUNCH_CHECK("gradient join");
+    return CKPT_OK;
+}
+
 int bn_relu_backward(int dtype, int64_t rows, int c, const void* dy, const void* z, const float* gamma, const float* stats,
                      int relu, void* dz, float* dgamma, float* dbeta, void* scratch, void* stream) {
     (void)gamma;   // scale = gamma * inv_std is part of the saved statistics

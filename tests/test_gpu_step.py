@@ -192,6 +192,54 @@ def test_ragged_chain_fp32():
     compare_with_oracle(runner, g0, ref, TOL["f32"])
 
 
+def mini_resnet(dtype, batch=4):
+    """Stem (7x7 stride 2), 3x3 stride-2 max-pool, bottleneck blocks with and without projection and
+    stride, global average pool, classifier: every unit kind of the ResNet configurations."""
+    units = [wl.conv_unit(3, 8, k=7, stride=2, pad=3), {"kind": "maxpool", "k": 3, "stride": 2, "pad": 1},
+             {"kind": "bottleneck", "cin": 8, "mid": 4, "cout": 16, "stride": 1, "project": True},
+             {"kind": "bottleneck", "cin": 16, "mid": 4, "cout": 16, "stride": 1, "project": False},
+             {"kind": "bottleneck", "cin": 16, "mid": 8, "cout": 32, "stride": 2, "project": True},
+             {"kind": "bottleneck", "cin": 32, "mid": 8, "cout": 32, "stride": 1, "project": False},
+             {"kind": "avgpool"}, {"kind": "fc", "cin": 32, "cout": 10, "relu": False}]
+    return dict(units=units, input_hwc=(40, 36, 3), batch=batch, dtype=dtype, loss="softmax_ce", name="mini_resnet_" + dtype)
+
+
+def test_mini_resnet_fp32_against_exact_oracle():
+    spec = mini_resnet("f32")
+    params = wl.make_params(spec, seed=21, bn_affine="random")
+    x, labels = wl.make_batch(spec, seed=22)
+    runner = StepRunner(spec, params)
+    n = runner.n
+    masks = [ck.plan(ck.ALGO_DYNAMIC_N, runner.d)[0], ck.mask_from_set(n, [0, n]), ck.mask_from_set(n, [0, 3, 5, n])]
+    rep0, g0 = all_policies_agree(runner, x, labels, masks, masks + [ck.plan(ck.ALGO_STATIC_N3, runner.d)[0]])
+    ref = oracle_step(spec, params, x, labels)
+    assert abs(rep0["loss"] - ref["loss"]) <= 1e-5 * abs(ref["loss"])
+    compare_with_oracle(runner, g0, ref, TOL["f32"])
+
+
+def test_bottleneck_bf16_on_tensor_cores():
+    """One block wide enough for the tcgen05 kernels (1x1 and 3x3, 64/256 channels), bf16, against the
+    oracle with the same storage rounding."""
+    units = [{"kind": "bottleneck", "cin": 64, "mid": 64, "cout": 256, "stride": 1, "project": True},
+             {"kind": "bottleneck", "cin": 256, "mid": 64, "cout": 256, "stride": 1, "project": False},
+             {"kind": "avgpool"}, {"kind": "fc", "cin": 256, "cout": 10, "relu": False}]
+    spec = dict(units=units, input_hwc=(12, 12, 64), batch=8, dtype="bf16", loss="softmax_ce", name="blocks_bf16")
+    params = wl.make_params(spec, seed=31, bn_affine="random")
+    x, labels = wl.make_batch(spec, seed=32)
+    runner = StepRunner(spec, params)
+    n = runner.n
+    masks = [ck.mask_from_set(n, [0, n]), ck.plan(ck.ALGO_DYNAMIC_N, runner.d)[0]]
+    rep0, g0 = all_policies_agree(runner, x, labels, masks, masks)
+    exact = oracle_step(spec, params, x, labels)
+    stored = oracle_step(spec, params, x, labels, storage="bf16")
+    assert abs(rep0["loss"] - exact["loss"]) <= 2e-2 * abs(exact["loss"])
+    for (ui, name, _), g in zip(runner.flat, g0):
+        assert np.all(np.isfinite(g))
+        mine = rel_l2(g, exact["grads"][ui][name])
+        theirs = rel_l2(stored["grads"][ui][name], exact["grads"][ui][name])
+        assert mine <= 1.5 * theirs + 0.02, (ui, name, mine, theirs)
+
+
 def test_arena_too_small_is_rejected_before_any_launch():
     spec = wl.config(1)
     runner = StepRunner(spec, wl.make_params(spec, seed=0))

@@ -156,12 +156,12 @@ def test_config_plans(index):
 
 
 def test_chain_sizes_match_oracle_shapes():
-    for index in (1, 2, 5):
+    for index in (1, 2, 3, 4, 5):
         spec = wl.config(index)
         chain = ck.Chain(spec)
         assert list(chain.sizes()) == oracle_sizes(spec)
         assert [tuple(s) for s in chain.shapes()] == no.output_shapes(spec)
-        flat = ck.flatten_params(spec, wl.make_params(spec) if index != 5 else
+        flat = ck.flatten_params(spec, wl.make_params(spec) if index in (1, 2) else
                                  [{k: np.zeros(s, np.float32) for k, s in wl.param_shapes(u).items()} for u in spec["units"]])
         assert chain.num_params() == len(flat)
         for p, (ui, name, arr) in enumerate(flat):
