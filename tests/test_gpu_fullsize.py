@@ -3,7 +3,7 @@
 * the tensor-core convolution kernels at the VGG-16 / batch-64 layer shapes, on sampled outputs that
   the oracle computes one by one (a cropped neighbourhood for forward/dgrad, one (c_out, c_in)
   channel pair over all pixels for wgrad);
-* the whole checkpointed step of configurations 2 and 5 through properties that hold at any size:
+* the whole checkpointed step of configurations 2, 3, 4 and 5 through properties that hold at any size:
   arena high-water == highest offset == planner's prediction (arena of exactly that size),
   gradients bit-identical between the checkpointed and the store-all schedule, finite loss."""
 import time
@@ -111,6 +111,17 @@ def test_config2_vgg16_full_size_step():
     rep, rep0, peak = step_properties(wl.config(2))
     assert peak < 0.65 * rep0["peak_bytes"]             # 1.17 GiB against 1.82 GiB
     assert abs(rep["loss"] - np.log(1000.0)) < 2.0      # random labels, random weights
+
+
+def test_config3_resnet50_full_size_step():
+    rep, rep0, peak = step_properties(wl.config(3))
+    assert peak == int(771.75 * 2 ** 20)                # planner value of the ResNet-50 chain at batch 128
+
+
+def test_config4_resnet152_full_size_step():
+    rep, rep0, peak = step_properties(wl.config(4))
+    assert peak == int(1837.5 * 2 ** 20)
+    assert rep0["peak_bytes"] > 3.7 * peak              # the O(n) plan stores 3.8x less than keeping everything
 
 
 def test_config5_plain1000_full_size_step():
