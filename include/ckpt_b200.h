@@ -70,6 +70,9 @@ CKPT_API const char* ckpt_last_error(void);
 #define CKPT_ALGO_STATIC_N3 0
 #define CKPT_ALGO_DYNAMIC_N2 1
 #define CKPT_ALGO_DYNAMIC_N 2
+/* Comparison plan of Sections 2.1 and 5.3 (not optimal): a checkpoint every ceil(sqrt(n)) units plus
+ * d_n; peak_bytes is its value under Eq. (memory). */
+#define CKPT_ALGO_SQRT_N 3
 
 /* d: host, n+1 sizes (>= 1).  is_ckpt: host, n+1 bytes, written (0/1).  peak_bytes: host, written:
  * the objective value of the returned set under the algorithm's own memory model. */
@@ -111,6 +114,13 @@ CKPT_API int ckpt_eval(int model, int64_t n, const int64_t* d, const uint8_t* is
 CKPT_API int ckpt_arena_dry_run(int policy, int64_t n, const int64_t* d, const uint8_t* is_ckpt,
                        int64_t* events, int64_t max_events, int64_t* n_events,
                        int64_t* high_water_bytes, int64_t* extent_bytes);
+
+/* Memory at the end of every "training phase index" of Section 5.1.1: trace[0] = before the step
+ * (d_0 only), trace[1..n] = end of the forward stage of unit i, trace[n+1..2n] = end of the backward
+ * stage of unit n, n-1, .., 1, trace[2n+1] = after the step (everything but d_0 released; under
+ * policies that keep tensors to the end, their release is counted here).  Bytes of the arena's
+ * objects only (no weights, no workspace).  trace: host, 2n+2 entries written. */
+CKPT_API int ckpt_arena_stage_trace(int policy, int64_t n, const int64_t* d, const uint8_t* is_ckpt, int64_t* trace);
 
 /* ---------------------------------------------------------------- layer-chain description
  *

@@ -21,6 +21,7 @@ Functions and the passage each one restates:
                          allocation event list.  Reading taken where the listing and Eq. (memory)
                          disagree: the previous gradient buffer is released *before* the segment is
                          recomputed, so that the event high-water equals Eq. (memory) exactly.
+* ``stage_trace``      - bytes at the end of every training phase index of Section 5.1.1.
 * ``brute_force_static`` / ``brute_force_dynamic`` - the optimum by enumerating every feasible set
                          (2^(n-1) of the 2^n masks over d_1..d_n contain n), plus the canonical
                          optimal set under the tie rule stated below.
@@ -180,6 +181,42 @@ def simulate_alg4(d, C):
             have_r = True
         L.free("d%d" % i)                               # released as soon as step i is done
     return L.high_water, L.events
+
+
+def stage_trace(d, C, schedule):
+    """Live bytes at the end of every training phase index 0..2n+1 (Section 5.1.1) under
+    Algorithm 2 (``schedule="alg2"``) or Algorithm 4 (``"alg4"``, with the buffer release moved
+    before the recompute): index 0 = before the step (d_0 only), 1..n = end of the forward stage
+    of unit i, n+1..2n = end of the backward stage of unit n..1, 2n+1 = after the step (d_0 only).
+    Written from the two listings directly, independently of the event simulators above."""
+    n = _check_sizes(d)
+    cs = _check_set(n, C)
+    is_c = [i in set(cs) for i in range(n + 1)]
+    live = {0: d[0]}
+    trace = [d[0]]
+    for i in range(1, n + 1):                               # forward phase (identical in both)
+        live[i] = d[i]
+        if not is_c[i - 1]:
+            del live[i - 1]
+        trace.append(sum(live.values()))
+    r = 0
+    for i in range(n, 0, -1):
+        if is_c[i]:
+            h = max(c for c in cs if c < i)
+            if schedule == "alg2":
+                for k in [k for k in live if k > i and not is_c[k]]:
+                    del live[k]                             # free the segment after d_i
+            else:
+                r = 0                                       # release the previous gradient buffer
+            for k in range(h + 1, i):
+                live[k] = d[k]                              # allocate + recompute the segment
+            if schedule == "alg4":
+                r = max(d[k] for k in range(h, i))
+        if schedule == "alg4":
+            del live[i]                                     # d_i released as soon as step i is done
+        trace.append(sum(live.values()) + r)
+    trace.append(d[0])
+    return trace
 
 
 # --------------------------------------------------------------------------------------------

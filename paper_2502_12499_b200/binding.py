@@ -13,7 +13,7 @@ import numpy as np
 HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(HERE, "libckpt_b200.so")
 
-ALGO_STATIC_N3, ALGO_DYNAMIC_N2, ALGO_DYNAMIC_N = 0, 1, 2
+ALGO_STATIC_N3, ALGO_DYNAMIC_N2, ALGO_DYNAMIC_N, ALGO_SQRT_N = 0, 1, 2, 3
 MODEL_STATIC, MODEL_DYNAMIC, MODEL_STORE_ALL = 0, 1, 2
 POLICY_STORE_ALL, POLICY_STATIC, POLICY_DYNAMIC = 0, 1, 2
 DTYPE_F32, DTYPE_BF16 = 0, 1
@@ -137,6 +137,19 @@ def arena_dry_run(policy, d, is_ckpt):
     _check(lib().ckpt_arena_dry_run(C.c_int(policy), C.c_int64(n), _ptr(d, C.c_int64), mask_p, _ptr(ev, C.c_int64),
                                     C.c_int64(cap), C.byref(n_ev), C.byref(hw), C.byref(ext)))
     return dict(events=ev[: n_ev.value].copy(), high_water=hw.value, extent=ext.value)
+
+
+def arena_stage_trace(policy, d, is_ckpt):
+    """ckpt_arena_stage_trace: int64[2n+2], arena bytes at the end of every training phase index."""
+    d = _i64(d)
+    n = len(d) - 1
+    mask_p = None
+    if is_ckpt is not None:
+        mask = np.ascontiguousarray(is_ckpt, dtype=np.uint8)
+        mask_p = _ptr(mask, C.c_uint8)
+    trace = np.zeros(2 * n + 2, dtype=np.int64)
+    _check(lib().ckpt_arena_stage_trace(C.c_int(policy), C.c_int64(n), _ptr(d, C.c_int64), mask_p, _ptr(trace, C.c_int64)))
+    return trace
 
 
 def mask_from_set(n, checkpoints):

@@ -71,6 +71,7 @@ struct StepCtx {
     cudaStream_t stream;
     Arena* arena;
     int64_t recomputed = 0;
+    int64_t* stage_trace = nullptr;     // optional: live arena bytes at the end of each of the 2n+2 stages
     int* status() const { return (int*)(ws + ch->off_misc + 64); }
 };
 
@@ -326,6 +327,7 @@ static int run_step(StepCtx& c, double* loss_out) {
 
     // ---------------- forward phase
     if ((rc = A.alloc_stack(0, d[0], &off))) return rc;
+    if (c.stage_trace) c.stage_trace[0] = A.live_bytes();
     if (!c.dry) {
         const int64_t payload = ch->batch * ch->shapes[0].h * ch->shapes[0].w * ch->shapes[0].c * dtype_size(ch->dtype);
         cudaError_t e = cudaMemcpyAsync(c.arena_base + off, c.batch, payload, cudaMemcpyDefault, c.stream);
@@ -348,6 +350,7 @@ static int run_step(StepCtx& c, double* loss_out) {
         }
         if ((rc = unit_forward(c, i, ptr(i - 1), ptr(i)))) return rc;
         if (!ck(i - 1)) if ((rc = A.release(i - 1))) return rc;
+        if (c.stage_trace) c.stage_trace[i] = A.live_bytes();
     }
 
     // ---------------- loss and dL/dd_n
@@ -422,7 +425,9 @@ static int run_step(StepCtx& c, double* loss_out) {
         if ((rc = unit_backward(c, i, ptr(i - 1), ptr(i), g_cur, need_dx ? g_next : nullptr))) return rc;
         if (need_dx) { g_cur = g_next; g_in_r = next_in_r; }
         if (c.policy == CKPT_POLICY_DYNAMIC) if ((rc = A.release(i))) return rc;
+        if (c.stage_trace) c.stage_trace[2 * n + 1 - i] = A.live_bytes();
     }
+    if (c.stage_trace) c.stage_trace[2 * n + 1] = d[0];
 
     if (!c.dry) {
         int status = 0;
@@ -487,6 +492,23 @@ int ckpt_arena_dry_run(int policy, int64_t n, const int64_t* d, const uint8_t* i
     if (high_water_bytes) *high_water_bytes = arena.high_water();
     if (extent_bytes) *extent_bytes = arena.extent();
     return CKPT_OK;
+}
+
+int ckpt_arena_stage_trace(int policy, int64_t n, const int64_t* d, const uint8_t* is_ckpt, int64_t* trace) {
+    if (policy < 0 || policy > 2) { set_error("unknown policy %d", policy); return CKPT_E_BAD_ARG; }
+    if (!trace) { set_error("trace is null"); return CKPT_E_NULL; }
+    int64_t predicted = 0;
+    int rc = eval_model(policy_model(policy), n, d, is_ckpt, &predicted);
+    if (rc) return rc;
+    ckpt_chain fake;
+    fake.units.resize(n);
+    fake.d.assign(d, d + n + 1);
+    fake.shapes.resize(n + 1);
+    Arena arena(predicted);
+    StepCtx c{};
+    c.ch = &fake; c.is_ckpt = is_ckpt; c.policy = policy; c.dry = true; c.arena = &arena; c.stage_trace = trace;
+    double loss = 0;
+    return run_step(c, &loss);
 }
 
 int ckpt_chain_create(const ckpt_unit_desc* units, int64_t n, int64_t batch, int32_t in_h, int32_t in_w,

@@ -23,6 +23,7 @@ int validate_sizes(int64_t n, const int64_t* d);
 int plan_static_n3(int64_t n, const int64_t* d, uint8_t* is_ckpt, int64_t* peak, int64_t* work);
 int plan_dynamic_n2(int64_t n, const int64_t* d, uint8_t* is_ckpt, int64_t* peak, int64_t* work);
 int plan_dynamic_n(int64_t n, const int64_t* d, uint8_t* is_ckpt, int64_t* peak, int64_t* work);
+int plan_sqrt_n(int64_t n, const int64_t* d, uint8_t* is_ckpt, int64_t* peak);
 int eval_model(int model, int64_t n, const int64_t* d, const uint8_t* is_ckpt, int64_t* peak);
 
 // ------------------------------------------------------------------ arena bookkeeping (arena.cpp)
@@ -40,6 +41,7 @@ public:
     bool is_live(int64_t id) const;
     int64_t offset_of(int64_t id) const;
     int64_t high_water() const { return high_water_; }
+    int64_t live_bytes() const { return live_bytes_; }
     int64_t extent() const { return extent_; }
     std::vector<ArenaEvent> events;
 private:

@@ -250,6 +250,19 @@ int plan_dynamic_n(int64_t n, const int64_t* d, uint8_t* is_ckpt, int64_t* peak,
     return CKPT_OK;
 }
 
+// ------------------------------------------------------------------------------------------------
+// The uniform heuristic the paper compares against (Section 2.1 / 5.3): a checkpoint every
+// ceil(sqrt(n)) units plus d_n; its peak is reported under Eq. (memory).
+// ------------------------------------------------------------------------------------------------
+int plan_sqrt_n(int64_t n, const int64_t* d, uint8_t* is_ckpt, int64_t* peak) {
+    int64_t step = 1;
+    while (step * step < n) ++step;
+    for (int64_t i = 0; i <= n; ++i) is_ckpt[i] = (i % step == 0) ? 1 : 0;
+    is_ckpt[0] = 1;
+    is_ckpt[n] = 1;
+    return eval_model(CKPT_MODEL_DYNAMIC, n, d, is_ckpt, peak);
+}
+
 }  // namespace ckpt
 
 // ------------------------------------------------------------------------------------------------
@@ -269,6 +282,7 @@ int ckpt_plan_counted(int algo, int64_t n, const int64_t* d, uint8_t* is_ckpt, i
         case CKPT_ALGO_STATIC_N3: return ckpt::plan_static_n3(n, d, is_ckpt, peak_bytes, work);
         case CKPT_ALGO_DYNAMIC_N2: return ckpt::plan_dynamic_n2(n, d, is_ckpt, peak_bytes, work);
         case CKPT_ALGO_DYNAMIC_N: return ckpt::plan_dynamic_n(n, d, is_ckpt, peak_bytes, work);
+        case CKPT_ALGO_SQRT_N: return ckpt::plan_sqrt_n(n, d, is_ckpt, peak_bytes);
     }
     ckpt::set_error("unknown algorithm %d", algo);
     return CKPT_E_BAD_ARG;

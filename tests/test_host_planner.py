@@ -228,3 +228,20 @@ def test_arena_schedule_on_optimal_plans_of_configs():
         m, peak = ck.plan(ck.ALGO_STATIC_N3, d)
         r = ck.arena_dry_run(ck.POLICY_STATIC, d, m)
         assert r["high_water"] == r["extent"] == peak
+
+
+def test_stage_trace_and_sqrt_plan_match_oracle(vgg19_golden):
+    rng = random.Random(400)
+    for _ in range(150):
+        n = rng.randint(1, 14)
+        d = [256 * rng.randint(1, 40) for _ in range(n + 1)]
+        C = [0] + [i for i in range(1, n) if rng.random() < 0.45] + [n]
+        mask = ck.mask_from_set(n, C)
+        assert list(ck.arena_stage_trace(ck.POLICY_DYNAMIC, d, mask)) == po.stage_trace(d, C, "alg4")
+        assert list(ck.arena_stage_trace(ck.POLICY_STATIC, d, mask)) == po.stage_trace(d, C, "alg2")
+        m, peak = ck.plan(ck.ALGO_SQRT_N, d)
+        assert as_set(m) == po.sqrt_n_plan(n) and peak == po.eval_dynamic(d, po.sqrt_n_plan(n))
+    d = [v * 128 * 4 for v in vgg19_golden["sizes_per_image"]]
+    m, peak = ck.plan(ck.ALGO_SQRT_N, d)
+    assert as_set(m)[1:] == vgg19_golden["sqrtn_set"]
+    assert peak - ck.plan(ck.ALGO_DYNAMIC_N, d)[1] == 1960 * 2 ** 20      # Table 2: 8404 - 6444 MiB

@@ -216,3 +216,27 @@ def test_vgg19_fig2_segment_start_jump(vgg19_golden):
     # stage 37 of the print (input excluded: it sits in the constant base) is the level before that
     base = vgg19_golden["fig2_stage0_gib"][0] * GIB
     assert abs(events[free_old - 1][3] - d[0] + base - vgg19_golden["fig2_stage37_gib"][0] * GIB) < 1
+
+
+def test_stage_trace_consistent_with_events_and_print(vgg19_golden):
+    rng = random.Random(8)
+    for _ in range(100):
+        n = rng.randint(1, 12)
+        d = rand_chain(rng, n)
+        C = [0] + [i for i in range(1, n) if rng.random() < 0.4] + [n]
+        t4 = po.stage_trace(d, C, "alg4")
+        t2 = po.stage_trace(d, C, "alg2")
+        assert len(t4) == len(t2) == 2 * n + 2 and t4[0] == t4[-1] == d[0]
+        assert max(t2) <= po.eval_static(d, C) and max(t4) <= po.eval_dynamic(d, C)
+        assert t4[n] == t2[n] == sum(d[c] for c in C)           # end of the forward phase: checkpoints only
+        assert t2[2 * n] == po.simulate_alg2(d, C)[1][-1][3]    # last event of the event list
+    # Fig. 2 (VGG-19, b = 128, C = {3,11,24}): forward stages 3 and 11 (ends of stages whose output is a
+    # checkpoint) and the whole run of backward stages 26..37, relative to the printed constant base.
+    # The printed series excludes the input (it sits in the base) and carries one d_24 (0.49 MiB) of
+    # the loss gradient through the backward phase.
+    d = [v * 128 * 4 for v in vgg19_golden["sizes_per_image"]]
+    t = po.stage_trace(d, [0] + vgg19_golden["fig2_set"], "alg4")
+    GIB = 1024 * MIB
+    base = vgg19_golden["fig2_stage0_gib"][0] * GIB
+    assert abs((t[37] - d[0]) - (vgg19_golden["fig2_stage37_gib"][0] * GIB - base)) < 1
+    assert abs((t[45] - d[0] + d[24]) - (vgg19_golden["fig2_stage45_gib"][0] * GIB - base)) < 1 * MIB
