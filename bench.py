@@ -277,7 +277,7 @@ def dominant_kernel_roofline(config_index, peaks):
     from paper_2502_12499_b200 import opbench
     mix = opbench.conv_mix("fwd", config_index, reps=3)
     traffic = CONV_FWD_TRAFFIC["bytes_per_launch"] if CONV_FWD_TRAFFIC["source_sha256"] == _kernel_source_sha() else None
-    out = {"kernel": "tc_conv_fwd_kernel / tc_conv_c64_kernel (implicit-GEMM conv forward)", "bound": "tensor",
+    out = {"kernel": "tc_conv_fwd_kernel / tc_conv_halo_kernel / tc_conv_c64_kernel (implicit-GEMM conv forward)", "bound": "tensor",
            "achieved": mix["tflops"], "peak": peaks["tflops_burst"], "unit": "TFLOP/s", "frac": mix["tflops"] / peaks["tflops_burst"],
            "peak_source": peaks["source"] + " (burst: kernels timed in isolation)", "traffic": traffic,
            "launch_shapes": mix["launches"], "flops_per_launch": mix["flops"] / mix["launches"],

@@ -457,6 +457,180 @@ tc_conv_c64_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_const
 }
 
 // ------------------------------------------------------------------------------------------------
+// Forward / dgrad, 3x3, padding 1, any multiple of 64 reduction channels: the halo-patch scheme of
+// the 64-channel kernel with the filter streamed instead of resident.  Per pixel tile (8 wide x th
+// high) and per 64-channel block the CTA fetches the three column-shifted halo patches once and
+// uses them for all nine taps (operand traffic for A drops from 9 to 3.4 tile loads); the filter
+// tile of each (tap, block) flows through its own ring.  Persistent CTAs, double-buffered TMEM
+// accumulator (2 x bn columns), epilogue of one tile under the MMAs of the next.
+// ------------------------------------------------------------------------------------------------
+struct HaloParams {
+    int H, W, N, c_red, c_out;
+    int th, tiles_w, tiles_h;
+    int bn, n_tiles, m_tiles, ctas_per_n;
+    int b_slots;                 // filter ring depth
+    uint32_t box_stride;         // bytes between the three shifted copies of a patch
+};
+
+__global__ void __launch_bounds__(kThreads, 1)
+tc_conv_halo_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w,
+                    __nv_bfloat16* __restrict__ out, HaloParams p, int* status) {
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    const uint32_t a_slot_bytes = 3 * p.box_stride, b_slot_bytes = (uint32_t)p.bn * 128;
+    const uint32_t b_base = base + 2 * a_slot_bytes;
+    const uint32_t bars = b_base + (uint32_t)p.b_slots * b_slot_bytes;
+    __shared__ uint32_t tmem_base_slot;
+    __shared__ int failed_flag;
+    volatile int* failed = &failed_flag;
+    // barrier map: a_full[2], a_empty[2], acc_full[2], acc_empty[2], then b_full[8], b_empty[8]
+    const uint32_t a_full0 = bars, a_empty0 = bars + 16, acc_full0 = bars + 32, acc_empty0 = bars + 48;
+    const uint32_t b_full0 = bars + 64, b_empty0 = bars + 64 + 8 * kMaxStages;
+
+    const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
+    const int n_tile = blockIdx.x % p.n_tiles;
+    const int first = blockIdx.x / p.n_tiles;
+    const int my_tiles = first < p.m_tiles ? (p.m_tiles - first + p.ctas_per_n - 1) / p.ctas_per_n : 0;
+    const int blocks = p.c_red / 64;
+    const uint32_t patch_bytes = (uint32_t)(8 * (p.th + 2)) * 128;
+    const uint32_t tmem_cols = 2 * p.bn <= 128 ? 128 : (2 * p.bn <= 256 ? 256 : 512);
+
+    if (threadIdx.x == 0) {
+        failed_flag = 0;
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(a_full0 + 8 * b, 1); mbar_init(a_empty0 + 8 * b, 1);
+            mbar_init(acc_full0 + 8 * b, 1); mbar_init(acc_empty0 + 8 * b, 128);
+        }
+        for (int s = 0; s < p.b_slots; ++s) { mbar_init(b_full0 + 8 * s, 1); mbar_init(b_empty0 + 8 * s, 1); }
+        fence_barrier_init();
+        tma_prefetch_desc(&map_x);
+        tma_prefetch_desc(&map_w);
+    }
+    if (warp == 1) tmem_alloc(smem_u32(&tmem_base_slot), tmem_cols);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = tmem_base_slot;
+
+    auto tile_origin = [&](int j, int& w0, int& h0, int& img) {
+        int t = first + j * p.ctas_per_n;
+        w0 = (t % p.tiles_w) * 8; t /= p.tiles_w;
+        h0 = (t % p.tiles_h) * p.th;
+        img = t / p.tiles_h;
+    };
+
+    if (warp == 0) {
+        // ---------------- producer.  Work items are (tile, channel block) pairs q = 0, 1, ...; pair q
+        // needs its three patches (A ring, 2 slots) and nine filter tiles (B ring).  The patches of pair
+        // q+1 are issued after the third filter tile of pair q: by then the MMAs have left pair q-1 (its
+        // A slot is free) and six taps of MMA time remain to hide the patch load.
+        // Lanes 0-2 issue the patches, lane 3 the filter tiles; every lane walks both rings.
+        const int total_pairs = my_tiles * blocks;
+        int a_count = 0, b_count = 0;          // patches / filter tiles issued so far
+        bool ok = true;
+        auto issue_patches = [&](int q) -> bool {
+            int w0, h0, img;
+            tile_origin(q / blocks, w0, h0, img);
+            const int as = q & 1;
+            if (!mbar_wait(a_empty0 + 8 * as, ((uint32_t)(q >> 1) & 1u) ^ 1u, failed, status, 501)) return false;
+            if (lane == 0) mbar_expect_tx(a_full0 + 8 * as, 3 * patch_bytes);
+            __syncwarp();
+            if (lane < 3)
+                tma_load_4d(base + as * a_slot_bytes + lane * p.box_stride, &map_x, a_full0 + 8 * as, (q % blocks) * 64, w0 + lane - 1, h0 - 1, img);
+            a_count = q + 1;
+            return true;
+        };
+        if (total_pairs > 0) ok = issue_patches(0);
+        for (int q = 0; q < total_pairs && ok; ++q) {
+            const int cb = q % blocks;
+            for (int tap = 0; tap < 9; ++tap) {
+                if (tap == 3 && q + 1 < total_pairs && !issue_patches(q + 1)) { ok = false; break; }
+                const int bs = b_count % p.b_slots;
+                if (!mbar_wait(b_empty0 + 8 * bs, ((uint32_t)(b_count / p.b_slots) & 1u) ^ 1u, failed, status, 502)) { ok = false; break; }
+                if (lane == 3) {
+                    mbar_expect_tx(b_full0 + 8 * bs, b_slot_bytes);
+                    tma_load_2d(b_base + bs * b_slot_bytes, &map_w, b_full0 + 8 * bs, tap * p.c_red + cb * 64, n_tile * p.bn);
+                }
+                ++b_count;
+            }
+        }
+        if (*failed) {
+            if (lane == 0) for (int q = max(0, a_count - 2); q < a_count; ++q) mbar_drain(a_full0 + 8 * (q & 1), (uint32_t)(q >> 1) & 1u);
+            if (lane == 3) for (int q = max(0, b_count - p.b_slots); q < b_count; ++q) mbar_drain(b_full0 + 8 * (q % p.b_slots), (uint32_t)(q / p.b_slots) & 1u);
+        }
+    } else if (warp == 1 && lane == 0) {
+        // ---------------- MMA issuer
+        const uint32_t idesc = instr_desc(128, p.bn, 0, 0);
+        int a_count = 0, b_count = 0;
+        bool ok = true;
+        for (int j = 0; j < my_tiles && ok; ++j) {
+            const int buf = j & 1;
+            if (!mbar_wait(acc_empty0 + 8 * buf, ((uint32_t)(j >> 1) & 1u) ^ 1u, failed, status, 503)) { ok = false; break; }
+            const uint32_t acc = tmem_base + (uint32_t)(buf * p.bn);
+            for (int cb = 0; cb < blocks && ok; ++cb) {
+                const int as = a_count & 1;
+                if (!mbar_wait(a_full0 + 8 * as, (uint32_t)(a_count >> 1) & 1u, failed, status, 504)) { ok = false; break; }
+                tc_fence_after();
+                for (int tap = 0; tap < 9; ++tap) {
+                    const int bs = b_count % p.b_slots;
+                    if (!mbar_wait(b_full0 + 8 * bs, (uint32_t)(b_count / p.b_slots) & 1u, failed, status, 505)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint32_t a_addr = base + as * a_slot_bytes + (tap % 3) * p.box_stride + (tap / 3) * 1024;
+                    const uint32_t b_addr = b_base + bs * b_slot_bytes;
+#pragma unroll
+                    for (int kk = 0; kk < 4; ++kk)
+                        umma_bf16(acc, smem_desc(a_addr + kk * 32, 0, 1024), smem_desc(b_addr + kk * 32, 0, 1024), idesc,
+                                  (cb > 0 || tap > 0 || kk > 0) ? 1u : 0u);
+                    umma_commit(b_empty0 + 8 * bs);
+                    ++b_count;
+                }
+                if (ok) umma_commit(a_empty0 + 8 * as);
+                ++a_count;
+            }
+            if (ok) umma_commit(acc_full0 + 8 * buf);
+        }
+    } else if (warp >= 2) {
+        // ---------------- epilogue
+        const int quarter = warp % 4;
+        const int row = quarter * 32 + lane;
+        const int wl = row % 8, hl = row / 8;
+        for (int j = 0; j < my_tiles; ++j) {
+            const int buf = j & 1;
+            if (!mbar_wait(acc_full0 + 8 * buf, (uint32_t)(j >> 1) & 1u, failed, status, 506)) break;
+            tc_fence_after();
+            int w0, h0, img;
+            tile_origin(j, w0, h0, img);
+            const bool valid = hl < p.th && (h0 + hl) < p.H && (w0 + wl) < p.W;
+            __nv_bfloat16* dst = out + ((((size_t)img * p.H + (h0 + hl)) * p.W + (w0 + wl)) * p.c_out + (size_t)n_tile * p.bn);
+            for (int c0 = 0; c0 < p.bn; c0 += 32) {
+                uint32_t v[32];
+                tmem_ld32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * p.bn + c0), v);
+                if (valid) {
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        uint4 pk;
+                        __nv_bfloat162* h = reinterpret_cast<__nv_bfloat162*>(&pk);
+#pragma unroll
+                        for (int e = 0; e < 4; ++e)
+                            h[e] = __floats2bfloat162_rn(__uint_as_float(v[8 * q + 2 * e]), __uint_as_float(v[8 * q + 2 * e + 1]));
+                        *reinterpret_cast<uint4*>(dst + c0 + 8 * q) = pk;
+                    }
+                }
+            }
+            tc_fence_before();
+            mbar_arrive(acc_empty0 + 8 * buf);
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        __syncwarp();
+        tc_fence_after();
+        tmem_dealloc(tmem_base, tmem_cols);
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
 // wgrad kernel: D[c_out tile of 128][up to 4 blocks of 64 (tap, c_in) columns], K = pixels
 // ------------------------------------------------------------------------------------------------
 struct WgradParams {
@@ -849,10 +1023,55 @@ int launch_c64(const void* x, const void* w_mat, void* out, int N, int H, int W,
     return CKPT_OK;
 }
 
+// Halo-patch kernel: worth it where the 8-wide tiles lose no pixels (W a multiple of 8, at least 112 of
+// the 128 accumulator rows used) and the reduction spans more than one channel block.
+bool halo_applies(int H, int W, int c_red, int c_out, int k, int pad) {
+    if (k != 3 || pad != 1 || c_red % 64 || c_red < 128 || c_out % 64 || W % 8) return false;
+    const int nt = (H + 15) / 16, th = (H + nt - 1) / nt;
+    return 8 * th >= 112 && H % th == 0;
+}
+
+int launch_halo(const void* x, const void* w_mat, void* out, int N, int H, int W, int c_red, int c_out, int* status,
+                cudaStream_t st, const char* what) {
+    HaloParams p;
+    p.H = H; p.W = W; p.N = N; p.c_red = c_red; p.c_out = c_out;
+    const int nt = (H + 15) / 16;
+    p.th = (H + nt - 1) / nt;
+    p.tiles_h = (H + p.th - 1) / p.th;
+    p.tiles_w = (W + 7) / 8;
+    p.bn = pick_bn(c_out);
+    p.n_tiles = c_out / p.bn;
+    p.m_tiles = p.tiles_w * p.tiles_h * N;
+    int sms = 148, dev = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    p.ctas_per_n = std::max(1, std::min(sms / p.n_tiles, p.m_tiles));
+    p.box_stride = (uint32_t)align_up((int64_t)std::max(8 * (p.th + 2), 16 + 128) * 128, 1024);
+    const uint32_t a_bytes = 2 * 3 * p.box_stride, b_slot = (uint32_t)p.bn * 128;
+    p.b_slots = std::min<int>(kMaxStages, (int)((208 * 1024 - a_bytes) / b_slot));
+    CUtensorMap mx, mw;
+    int rc = make_act_map(&mx, x, N, H, W, c_red, 8, p.th + 2, 1);
+    if (rc) return rc;
+    rc = make_mat_map(&mw, w_mat, c_out, (int64_t)9 * c_red, p.bn);
+    if (rc) return rc;
+    const size_t smem = (size_t)a_bytes + (size_t)p.b_slots * b_slot + 1024 + 256;
+    static bool attr_set = false;
+    if (!attr_set) {
+        cudaError_t e = cudaFuncSetAttribute(tc_conv_halo_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 224 * 1024);
+        if (e != cudaSuccess) return cuda_fail(e, "raising the shared-memory limit");
+        attr_set = true;
+    }
+    tc_conv_halo_kernel<<<p.ctas_per_n * p.n_tiles, kThreads, smem, st>>>(mx, mw, (__nv_bfloat16*)out, p, status);
+    CKPT_LAUNCH_CHECK(what);
+    return CKPT_OK;
+}
+
 int launch_fwd_like(const void* x, const void* w_mat, void* out, const float* bias, int relu, int N, int H, int W, int c_red,
                     int c_out, int k, int pad, int* status, cudaStream_t st, const char* what) {
     if (c_red == 64 && k == 3 && pad == 1 && c_out % 64 == 0 && !bias && !relu)
         return launch_c64(x, w_mat, out, N, H, W, c_out, status, st, what);
+    if (!bias && !relu && halo_applies(H, W, c_red, c_out, k, pad))
+        return launch_halo(x, w_mat, out, N, H, W, c_red, c_out, status, st, what);
     FwdParams p;
     p.H = H; p.W = W; p.N = N; p.c_red = c_red; p.c_out = c_out; p.k = k; p.pad = pad;
     choose_tile(128, W, H, N, &p.tw, &p.th, &p.tn);

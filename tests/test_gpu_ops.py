@@ -44,6 +44,10 @@ TC_CASES = [
     (64, 1, 1, 512, 192, 1, 0),      # fully connected shape
     (48, 1, 1, 256, 1000, 1, 0),     # classifier: output channels not a multiple of 64
     (2, 56, 56, 64, 64, 3, 1),
+    (2, 16, 16, 128, 128, 3, 1),     # halo-patch kernel, one tile per CTA
+    (2, 28, 24, 128, 256, 3, 1),     # halo-patch kernel, 14-row tiles, 256-wide output tile
+    (2, 32, 16, 192, 64, 3, 1),      # halo-patch kernel, three channel blocks, 64-wide output tile
+    (2, 112, 112, 128, 128, 3, 1),   # halo-patch kernel, several tiles per persistent CTA
 ]
 
 
