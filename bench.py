@@ -88,8 +88,14 @@ def conv_flops(spec, plan_mask, shapes):
     fwd = []
     h, w, c = spec["input_hwc"]
     for u, (ho, wo, co) in zip(spec["units"], shapes[1:]):
-        if u["kind"] == "conv_bn_relu":
+        if u["kind"] in ("conv_bn_relu", "conv"):
             fwd.append(2.0 * spec["batch"] * ho * wo * co * u["k"] * u["k"] * u["cin"])
+        elif u["kind"] == "bottleneck":
+            st, mid = u["stride"], u["mid"]
+            macs = ho * st * wo * st * u["cin"] * mid + ho * wo * 9 * mid * mid + ho * wo * mid * co
+            if u["project"]:
+                macs += ho * wo * u["cin"] * co
+            fwd.append(2.0 * spec["batch"] * macs)
         elif u["kind"] == "fc":
             fwd.append(2.0 * spec["batch"] * u["cin"] * u["cout"])
         else:
@@ -142,6 +148,8 @@ def main():
     ap.add_argument("--steps-cpu", type=int, default=1)
     ap.add_argument("--warmup-cpu", type=int, default=0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--split-units", action="store_true",
+                    help="finer granularity: conv, batch norm and ReLU as chain units of their own")
     args = ap.parse_args()
 
     rank = int(os.environ.get("RANK", "0"))
@@ -150,6 +158,8 @@ def main():
     spec = wl.config(args.config)
     if args.batch:
         spec = dict(spec, batch=args.batch)
+    if args.split_units:
+        spec, _ = wl.split_units(spec)
     config = {"workload": "%s: %d units, batch %d of %dx%dx%d %s, plan = Algorithm 6, schedule = Algorithm 4"
                           % (spec["name"], len(spec["units"]), spec["batch"], *spec["input_hwc"], spec["dtype"]),
               "l2": "inputs larger than L2 (every step streams > 1 GB of activations)",

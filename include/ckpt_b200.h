@@ -137,6 +137,10 @@ CKPT_API int ckpt_arena_stage_trace(int policy, int64_t n, const int64_t* d, con
  *       (mid -> mid), 1x1 (mid -> c_out), each with batch norm; projection shortcut when
  *       (flags & 2); ReLU after the residual add.  parameters: w1,g1,b1,w2,g2,b2,w3,g3,b3
  *       [,wp,gp,bp].
+ *   CKPT_UNIT_CONV, CKPT_UNIT_BN, CKPT_UNIT_RELU - the three steps of a CONV_BN_RELU unit as chain
+ *       units of their own (the finer layer granularity of Section 5.4: every step's output is a
+ *       d_i the planner may keep or drop).  CONV: parameters w; BN: c_in = c_out = channels,
+ *       parameters gamma, beta; RELU: no parameters.
  * Parameter tensors are numbered consecutively over the chain in the order listed above.
  * Gradients are always float32 with the parameter's shape.
  */
@@ -145,6 +149,9 @@ CKPT_API int ckpt_arena_stage_trace(int policy, int64_t n, const int64_t* d, con
 #define CKPT_UNIT_FC 2
 #define CKPT_UNIT_AVGPOOL 3
 #define CKPT_UNIT_BOTTLENECK 4
+#define CKPT_UNIT_CONV 5
+#define CKPT_UNIT_BN 6
+#define CKPT_UNIT_RELU 7
 
 #define CKPT_DTYPE_F32 0   /* float32 storage and arithmetic (no tensor cores)                    */
 #define CKPT_DTYPE_BF16 1  /* bfloat16 storage, float32 accumulation                              */

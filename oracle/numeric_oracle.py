@@ -178,6 +178,14 @@ def unit_forward(unit, p, x, storage="exact"):
         y, c = _cbr_fwd(x, p["w"], p["gamma"], p["beta"], unit["stride"], unit["pad"], True, storage)
         y = _store(y, storage)
         return y, (c, y)
+    if kind == "conv":                                   # finer granularity (Section 5.4): the three
+        return _store(conv2d_fwd(x, p["w"], unit["stride"], unit["pad"]), storage), x
+    if kind == "bn":                                     # steps of a conv unit as chain units of their own
+        y, c = bn_fwd(x, p["gamma"], p["beta"])
+        return _store(y, storage), c
+    if kind == "relu":
+        y = np.maximum(x, 0.0)
+        return y, y
     if kind == "maxpool":
         y, arg = maxpool_fwd(x, unit["k"], unit["stride"], unit["pad"])
         return y, (arg, x.shape)
@@ -212,6 +220,14 @@ def unit_backward(unit, p, dy, cache, storage="exact"):
         c, y = cache
         dx, dw, dg, db = _cbr_bwd(dy, y, c, p["w"], p["gamma"], unit["stride"], unit["pad"], True, storage)
         return _store(dx, storage), {"w": dw, "gamma": dg, "beta": db}
+    if kind == "conv":
+        dx, dw = conv2d_bwd(cache, p["w"], dy, unit["stride"], unit["pad"])
+        return _store(dx, storage), {"w": dw}
+    if kind == "bn":
+        dx, dgamma, dbeta = bn_bwd(dy, cache, p["gamma"])
+        return _store(dx, storage), {"gamma": dgamma, "beta": dbeta}
+    if kind == "relu":
+        return dy * (cache > 0), {}
     if kind == "maxpool":
         arg, xs = cache
         return maxpool_bwd(dy, arg, xs, unit["k"], unit["stride"], unit["pad"]), {}
@@ -287,7 +303,7 @@ def output_shapes(chain):
     out = [(h, w, c)]
     for u in chain["units"]:
         k = u["kind"]
-        if k == "conv_bn_relu":
+        if k in ("conv_bn_relu", "conv"):
             h, w, c = conv_out_size(h, u["k"], u["stride"], u["pad"]), conv_out_size(w, u["k"], u["stride"], u["pad"]), u["cout"]
         elif k == "maxpool":
             h, w = conv_out_size(h, u["k"], u["stride"], u["pad"]), conv_out_size(w, u["k"], u["stride"], u["pad"])

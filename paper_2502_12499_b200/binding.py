@@ -18,7 +18,7 @@ MODEL_STATIC, MODEL_DYNAMIC, MODEL_STORE_ALL = 0, 1, 2
 POLICY_STORE_ALL, POLICY_STATIC, POLICY_DYNAMIC = 0, 1, 2
 DTYPE_F32, DTYPE_BF16 = 0, 1
 LOSS_SUM, LOSS_SOFTMAX_CE = 0, 1
-UNIT_KINDS = {"conv_bn_relu": 0, "maxpool": 1, "fc": 2, "avgpool": 3, "bottleneck": 4}
+UNIT_KINDS = {"conv_bn_relu": 0, "maxpool": 1, "fc": 2, "avgpool": 3, "bottleneck": 4, "conv": 5, "bn": 6, "relu": 7}
 ERROR_NAMES = {-1: "E_NULL", -2: "E_BAD_N", -3: "E_BAD_SIZE", -4: "E_OVERFLOW", -5: "E_BAD_PLAN",
                -6: "E_BAD_ARG", -7: "E_ARENA_OOM", -8: "E_WORKSPACE", -9: "E_CUDA",
                -10: "E_DEVICE_TIMEOUT", -11: "E_UNSUPPORTED", -12: "E_NO_DEVICE"}

@@ -224,6 +224,17 @@ static int unit_forward(StepCtx& c, int64_t i, const void* x_raw, void* y) {
             if ((rc = conv_forward_any(c, u.geom, x, p[0], y, nullptr, 0))) return rc;
             return bn_statistics(dt, rows_of(c.ch, i), u.out.c, y, (const float*)p[1], (const float*)p[2], stats_of(c, i),
                                  ws + c.ch->off_scr, c.stream);
+        case CKPT_UNIT_CONV:
+            if ((rc = activated(c, i - 1, x_raw, &x))) return rc;
+            return conv_forward_any(c, u.geom, x, p[0], y, nullptr, 0);
+        case CKPT_UNIT_BN:
+            if ((rc = activated(c, i - 1, x_raw, &x))) return rc;
+            if ((rc = bn_statistics(dt, rows_of(c.ch, i), u.out.c, x, (const float*)p[0], (const float*)p[1], stats_of(c, i),
+                                    ws + c.ch->off_scr, c.stream))) return rc;
+            return bn_apply(dt, rows_of(c.ch, i), u.out.c, x, stats_of(c, i), 0, y, c.stream);
+        case CKPT_UNIT_RELU:
+            if ((rc = activated(c, i - 1, x_raw, &x))) return rc;
+            return relu_forward(dt, rows_of(c.ch, i) * u.out.c, x, y, c.stream);
         case CKPT_UNIT_MAXPOOL: {
             const float* act = nullptr;
             if (pending_act(c.ch, i - 1)) {
@@ -272,6 +283,20 @@ static int unit_backward(StepCtx& c, int64_t i, const void* x_raw, const void* y
             if ((rc = activated(c, i - 1, x_raw, &x))) return rc;
             if ((rc = conv_wgrad_any(c, u.geom, g_in, x, (float*)g[0]))) return rc;
             if (g_out && (rc = conv_dgrad_any(c, u.geom, g_in, p[0], g_out))) return rc;
+            break;
+        case CKPT_UNIT_CONV:
+            if ((rc = activated(c, i - 1, x_raw, &x))) return rc;
+            if ((rc = conv_wgrad_any(c, u.geom, g_in, x, (float*)g[0]))) return rc;
+            if (g_out && (rc = conv_dgrad_any(c, u.geom, g_in, p[0], g_out))) return rc;
+            break;
+        case CKPT_UNIT_BN:
+            // the statistics saved by this unit's (re)computed forward are those of its input
+            if ((rc = activated(c, i - 1, x_raw, &x))) return rc;
+            if ((rc = bn_relu_backward(dt, rows_of(c.ch, i), u.out.c, g_in, x, (const float*)p[0], stats_of(c, i), 0,
+                                       g_out ? g_out : g_in, (float*)g[0], (float*)g[1], c.ws + c.ch->off_scr, c.stream))) return rc;
+            break;
+        case CKPT_UNIT_RELU:
+            if (g_out && (rc = relu_backward(dt, rows_of(c.ch, i) * u.out.c, g_in, y, g_out, c.stream))) return rc;
             break;
         case CKPT_UNIT_MAXPOOL: {
             if (!g_out) break;
@@ -551,6 +576,33 @@ int ckpt_chain_create(const ckpt_unit_desc* units, int64_t n, int64_t batch, int
                 if (small_conv_supported(dtype, u.geom)) scr = std::max(scr, small_conv_scratch_bytes(u.geom));
                 break;
             }
+            case CKPT_UNIT_CONV: {
+                rc = check_conv(u.desc, cur, i);
+                if (rc) break;
+                u.out = {out_size(cur.h, u.desc.k, u.desc.stride, u.desc.pad),
+                         out_size(cur.w, u.desc.k, u.desc.stride, u.desc.pad), u.desc.c_out};
+                u.geom = {(int)batch, cur.h, cur.w, cur.c, u.out.h, u.out.w, u.out.c, u.desc.k, u.desc.stride, u.desc.pad};
+                ch->params.push_back({i, (int64_t)u.desc.c_out * u.desc.k * u.desc.k * u.desc.c_in, dtype});
+                scr = std::max(scr, simt_wgrad_scratch_bytes(u.geom));
+                if (tc_conv_supported(dtype, u.geom)) scr = std::max(scr, tc_conv_scratch_bytes(u.geom));
+                if (small_conv_supported(dtype, u.geom)) scr = std::max(scr, small_conv_scratch_bytes(u.geom));
+                break;
+            }
+            case CKPT_UNIT_BN:
+                if (u.desc.c_in != cur.c || u.desc.c_out != cur.c) {
+                    set_error("unit %lld: batch norm over %d channels on %d incoming channels", (long long)i, u.desc.c_out, cur.c);
+                    rc = CKPT_E_BAD_ARG; break;
+                }
+                u.out = cur;
+                ch->params.push_back({i, cur.c, CKPT_DTYPE_F32});
+                ch->params.push_back({i, cur.c, CKPT_DTYPE_F32});
+                u.stats_off = stats_floats;
+                stats_floats += 4 * (int64_t)cur.c;
+                scr = std::max(scr, bn_scratch_bytes(batch * cur.h * cur.w, cur.c));
+                break;
+            case CKPT_UNIT_RELU:
+                u.out = cur;
+                break;
             case CKPT_UNIT_MAXPOOL:
                 if (u.desc.k < 1 || u.desc.stride < 1 || u.desc.pad < 0 || 2 * u.desc.pad > u.desc.k ||
                     cur.h + 2 * u.desc.pad < u.desc.k || cur.w + 2 * u.desc.pad < u.desc.k) {

@@ -114,6 +114,8 @@ int avgpool_backward(int dtype, int n, int h, int w, int c, const void* dy, void
 
 // g <- g * (y > 0), elementwise over `elems`.
 int relu_mask_inplace(int dtype, int64_t elems, void* g, const void* y, void* stream);
+int relu_forward(int dtype, int64_t elems, const void* x, void* y, void* stream);
+int relu_backward(int dtype, int64_t elems, const void* dy, const void* y, void* dx, void* stream);
 // out[c] (f32) = sum over rows of g[row][c], rows summed in index order.
 int column_sums(int dtype, int64_t rows, int c, const void* g, float* out, void* stream);
 int softmax_ce(int dtype, int batch, int classes, const void* logits, const int32_t* labels,

@@ -980,6 +980,53 @@ int relu_mask_inplace(int dtype, int64_t elems, void* g, const void* y, void* st
     return CKPT_OK;
 }
 
+// ReLU as a chain unit of its own: 16-byte accesses, scalar tail.  y may alias x, dx may alias dy.
+template <typename T>
+__global__ void __launch_bounds__(256) relu_fwd_kernel(const T* __restrict__ x, T* __restrict__ y, int64_t elems) {
+    constexpr int V = 16 / sizeof(T);
+    const int64_t vecs = elems / V;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < vecs; i += (int64_t)gridDim.x * blockDim.x) {
+        uint4 raw = __ldg(reinterpret_cast<const uint4*>(x) + i);
+        T* e = reinterpret_cast<T*>(&raw);
+#pragma unroll
+        for (int k = 0; k < V; ++k) e[k] = cvt<T>(fmaxf(ld(e + k), 0.f));
+        reinterpret_cast<uint4*>(y)[i] = raw;
+    }
+    if (blockIdx.x == 0)
+        for (int64_t i = vecs * V + threadIdx.x; i < elems; i += blockDim.x) y[i] = cvt<T>(fmaxf(ld(x + i), 0.f));
+}
+template <typename T>
+__global__ void __launch_bounds__(256) relu_bwd_kernel(const T* __restrict__ dy, const T* __restrict__ y, T* __restrict__ dx,
+                                                       int64_t elems) {
+    constexpr int V = 16 / sizeof(T);
+    const int64_t vecs = elems / V;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < vecs; i += (int64_t)gridDim.x * blockDim.x) {
+        uint4 g = __ldg(reinterpret_cast<const uint4*>(dy) + i);
+        uint4 o = __ldg(reinterpret_cast<const uint4*>(y) + i);
+        T* ge = reinterpret_cast<T*>(&g);
+        const T* oe = reinterpret_cast<const T*>(&o);
+#pragma unroll
+        for (int k = 0; k < V; ++k) if (!(ld(oe + k) > 0.f)) ge[k] = cvt<T>(0.f);
+        reinterpret_cast<uint4*>(dx)[i] = g;
+    }
+    if (blockIdx.x == 0)
+        for (int64_t i = vecs * V + threadIdx.x; i < elems; i += blockDim.x) dx[i] = ld(y + i) > 0.f ? dy[i] : cvt<T>(0.f);
+}
+int relu_forward(int dtype, int64_t elems, const void* x, void* y, void* stream) {
+    const int64_t vecs = elems / (dtype == CKPT_DTYPE_BF16 ? 8 : 4);
+    if (dtype == CKPT_DTYPE_BF16) relu_fwd_kernel<__nv_bfloat16><<<elementwise_grid(vecs), 256, 0, (cudaStream_t)stream>>>((const __nv_bfloat16*)x, (__nv_bfloat16*)y, elems);
+    else relu_fwd_kernel<float><<<elementwise_grid(vecs), 256, 0, (cudaStream_t)stream>>>((const float*)x, (float*)y, elems);
+    CKPT_LAUNCH_CHECK("ReLU forward");
+    return CKPT_OK;
+}
+int relu_backward(int dtype, int64_t elems, const void* dy, const void* y, void* dx, void* stream) {
+    const int64_t vecs = elems / (dtype == CKPT_DTYPE_BF16 ? 8 : 4);
+    if (dtype == CKPT_DTYPE_BF16) relu_bwd_kernel<__nv_bfloat16><<<elementwise_grid(vecs), 256, 0, (cudaStream_t)stream>>>((const __nv_bfloat16*)dy, (const __nv_bfloat16*)y, (__nv_bfloat16*)dx, elems);
+    else relu_bwd_kernel<float><<<elementwise_grid(vecs), 256, 0, (cudaStream_t)stream>>>((const float*)dy, (const float*)y, (float*)dx, elems);
+    CKPT_LAUNCH_CHECK("ReLU backward");
+    return CKPT_OK;
+}
+
 template <typename T>
 __global__ void column_sum_kernel(const T* __restrict__ g, float* __restrict__ out, int64_t rows, int c) {
     int ch = blockIdx.x * blockDim.x + threadIdx.x;

@@ -9,6 +9,8 @@ loss="sum"|"softmax_ce", name=...)``.  Unit dicts:
 
 * ``{"kind": "conv_bn_relu", "cin", "cout", "k", "stride", "pad"}`` - convolution without bias,
   training-mode batch normalisation, ReLU; parameters ``w [cout,k,k,cin]``, ``gamma``, ``beta``.
+* ``{"kind": "conv", ...}``, ``{"kind": "bn", "cin", "cout"}``, ``{"kind": "relu"}`` - the three steps of a
+  conv_bn_relu unit as chain units of their own (finer granularity).
 * ``{"kind": "maxpool", "k", "stride", "pad"}``
 * ``{"kind": "avgpool"}`` - global average over H and W.
 * ``{"kind": "fc", "cin", "cout", "relu"}`` - fully connected with bias on the NHWC-flattened input;
@@ -28,6 +30,9 @@ PARAM_NAMES = {
     "maxpool": [],
     "avgpool": [],
     "fc": ["w", "b"],
+    "conv": ["w"],
+    "bn": ["gamma", "beta"],
+    "relu": [],
     "bottleneck": ["w1", "g1", "b1", "w2", "g2", "b2", "w3", "g3", "b3", "wp", "gp", "bp"],
 }
 
@@ -99,6 +104,31 @@ def resnet_chain(blocks, batch, hw=(224, 224), dtype="bf16", base=64, classes=10
                 loss="softmax_ce", name=name)
 
 
+def split_units(chain):
+    """Finer granularity (Section 5.4): every conv+BN+ReLU unit becomes three chain units - convolution,
+    batch normalisation, ReLU - each with an output of its own that the planner may keep or drop.
+    Returns the new chain and, per new unit, (index of the original unit, names of the parameters it takes)."""
+    units, origin = [], []
+    for ui, u in enumerate(chain["units"]):
+        if u["kind"] == "conv_bn_relu":
+            units.append({"kind": "conv", "cin": u["cin"], "cout": u["cout"], "k": u["k"], "stride": u["stride"], "pad": u["pad"]})
+            units.append({"kind": "bn", "cin": u["cout"], "cout": u["cout"]})
+            units.append({"kind": "relu"})
+            origin += [(ui, ["w"]), (ui, ["gamma", "beta"]), (ui, [])]
+        else:
+            units.append(dict(u))
+            origin.append((ui, PARAM_NAMES[u["kind"]]))
+    fine = dict(chain)
+    fine["units"] = units
+    fine["name"] = chain.get("name", "chain") + "_fine"
+    return fine, origin
+
+
+def split_params(origin, params):
+    """Parameters of the original chain re-filed under the units of the split chain."""
+    return [{name: params[ui][name] for name in names if name in params[ui]} for ui, names in origin]
+
+
 def config(index):
     """The five benchmark configurations (index 1..5)."""
     if index == 1:
@@ -125,6 +155,10 @@ def param_shapes(unit):
     if k == "conv_bn_relu":
         return {"w": (unit["cout"], unit["k"], unit["k"], unit["cin"]),
                 "gamma": (unit["cout"],), "beta": (unit["cout"],)}
+    if k == "conv":
+        return {"w": (unit["cout"], unit["k"], unit["k"], unit["cin"])}
+    if k == "bn":
+        return {"gamma": (unit["cout"],), "beta": (unit["cout"],)}
     if k == "fc":
         return {"w": (unit["cout"], unit["cin"]), "b": (unit["cout"],)}
     if k == "bottleneck":

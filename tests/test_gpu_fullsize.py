@@ -113,6 +113,15 @@ def test_config2_vgg16_full_size_step():
     assert abs(rep["loss"] - np.log(1000.0)) < 2.0      # random labels, random weights
 
 
+def test_config2_vgg16_split_units_full_size_step():
+    """Finer granularity (Section 5.4): the 47-unit split of the VGG-16 chain at full size."""
+    fine, _ = wl.split_units(wl.config(2))
+    rep, rep0, peak = step_properties(fine)
+    assert rep0["peak_bytes"] == int(sum(ck.Chain(fine).sizes()))
+    assert peak < 0.5 * rep0["peak_bytes"]
+    assert abs(rep["loss"] - np.log(1000.0)) < 2.0
+
+
 def test_config3_resnet50_full_size_step():
     rep, rep0, peak = step_properties(wl.config(3))
     assert peak == int(771.75 * 2 ** 20)                # planner value of the ResNet-50 chain at batch 128

@@ -240,6 +240,51 @@ def test_bottleneck_bf16_on_tensor_cores():
         assert mine <= 1.5 * theirs + 0.02, (ui, name, mine, theirs)
 
 
+def test_split_mini_vgg_fp32_against_exact_oracle():
+    """Finer granularity (Section 5.4): conv, bn and relu as chain units of their own (39 + 8 units).
+    Same function as the fused chain, so the oracle of the *split* chain and of the fused chain both
+    apply; the arena follows the planner's prediction on the longer chain."""
+    coarse = mini_vgg("f32")
+    spec, origin = wl.split_units(coarse)
+    cparams = wl.make_params(coarse, seed=3, bn_affine="random")
+    params = wl.split_params(origin, cparams)
+    x, labels = wl.make_batch(coarse, seed=4)
+    runner = StepRunner(spec, params)
+    n = runner.n
+    assert n == len(coarse["units"]) + 2 * 13
+    d = [int(v) for v in runner.d]
+    m6, _ = ck.plan(ck.ALGO_DYNAMIC_N, d)
+    m3, _ = ck.plan(ck.ALGO_STATIC_N3, d)
+    rng = random.Random(2)
+    extra = [ck.mask_from_set(n, [0] + [i for i in range(1, n) if rng.random() < 0.35] + [n]) for _ in range(4)]
+    extra.append(ck.mask_from_set(n, [0, n]))
+    rep0, g0 = all_policies_agree(runner, x, labels, [m6] + extra, [m3] + extra)
+    ref = oracle_step(spec, params, x, labels)
+    assert abs(rep0["loss"] - ref["loss"]) <= 1e-5 * abs(ref["loss"])
+    compare_with_oracle(runner, g0, ref, TOL["f32"])
+    # and against the fused chain's oracle gradients, re-filed
+    fused = oracle_step(coarse, cparams, x, labels)
+    for (fi, name, _), g in zip(runner.flat, g0):
+        want = fused["grads"][origin[fi][0]][name]
+        assert max_rel_err(g.reshape(want.shape), want) <= TOL["f32"]
+
+
+def test_split_shallow_bf16_chain():
+    """bfloat16 split chain on the tensor-core kernels, element-wise against the storage-rounded oracle."""
+    coarse = [c for c in shallow_chains() if c["name"] == "conv64+conv64+fc"][0]
+    spec, origin = wl.split_units(coarse)
+    params = wl.split_params(origin, wl.make_params(coarse, seed=11, bn_affine="random"))
+    x, labels = wl.make_batch(coarse, seed=12)
+    runner = StepRunner(spec, params)
+    n = runner.n
+    m6, _ = ck.plan(ck.ALGO_DYNAMIC_N, runner.d)
+    rep0, g0 = all_policies_agree(runner, x, labels, [m6, ck.mask_from_set(n, [0, n]), ck.mask_from_set(n, [0, 2, 5, n])],
+                                  [ck.mask_from_set(n, [0, 3, n])])
+    ref = oracle_step(spec, params, x, labels, storage="bf16")
+    assert abs(rep0["loss"] - ref["loss"]) <= 1e-2 * abs(ref["loss"])
+    compare_with_oracle(runner, g0, ref, TOL["bf16"])
+
+
 def test_arena_too_small_is_rejected_before_any_launch():
     spec = wl.config(1)
     runner = StepRunner(spec, wl.make_params(spec, seed=0))

@@ -245,3 +245,36 @@ def test_stage_trace_and_sqrt_plan_match_oracle(vgg19_golden):
     m, peak = ck.plan(ck.ALGO_SQRT_N, d)
     assert as_set(m)[1:] == vgg19_golden["sqrtn_set"]
     assert peak - ck.plan(ck.ALGO_DYNAMIC_N, d)[1] == 1960 * 2 ** 20      # Table 2: 8404 - 6444 MiB
+
+
+def test_split_units_chain_and_plan():
+    """Finer granularity (Section 5.4): the split VGG-16 chain has 47 units; conv, bn and relu outputs
+    have the size of the fused unit's output; the O(n) planner still matches the O(n^2) recursion, and
+    its optimum is below that of the same chain with every tensor stored."""
+    coarse = wl.config(2)
+    fine, origin = wl.split_units(coarse)
+    assert len(fine["units"]) == 21 + 2 * 13 == len(origin)
+    chain = ck.Chain(fine)
+    d = [int(v) for v in chain.sizes()]
+    assert d == oracle_sizes(fine)
+    dc = oracle_sizes(coarse)
+    k = 1
+    for ui, u in enumerate(coarse["units"]):
+        if u["kind"] == "conv_bn_relu":
+            assert d[k] == d[k + 1] == d[k + 2] == dc[ui + 1]
+            k += 3
+        else:
+            assert d[k] == dc[ui + 1]
+            k += 1
+    vd, Cd, _ = po.dp_dynamic_reference(d)
+    m, peak = ck.plan(ck.ALGO_DYNAMIC_N, d)
+    assert (peak, as_set(m)) == (vd, Cd)
+    assert peak < sum(d) / 2
+    r = ck.arena_dry_run(ck.POLICY_DYNAMIC, d, m)
+    assert r["high_water"] == r["extent"] == peak
+    # the parameters of the fused chain re-file one to one
+    shapes = [{k2: np.zeros(s, np.float32) for k2, s in wl.param_shapes(u).items()} for u in coarse["units"]]
+    flat_c = ck.flatten_params(coarse, shapes)
+    flat_f = ck.flatten_params(fine, wl.split_params(origin, shapes))
+    assert [(origin[fi][0], name) for fi, name, _ in flat_f] == [(ui, name) for ui, name, _ in flat_c]
+    assert chain.num_params() == len(flat_f)

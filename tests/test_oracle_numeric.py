@@ -196,3 +196,33 @@ def test_bf16_storage_mode_rounds_stored_tensors_only():
         for k in ge:
             assert np.abs(ge[k] - gs[k]).max() <= 3e-2 * np.abs(ge[k]).max()
     assert abs(exact["loss"] - stored["loss"]) <= 5e-3 * abs(exact["loss"])
+
+
+def test_split_chain_equals_fused_chain():
+    """Finer granularity (Section 5.4): conv, bn and relu as chain units of their own compute the same
+    function as the fused unit, so every gradient agrees to rounding; and the central-difference check
+    runs on the split chain too (it exercises the three new unit kinds by themselves)."""
+    for chain in tiny_chains():
+        if not any(u["kind"] == "conv_bn_relu" for u in chain["units"]):
+            continue
+        fine, origin = wl.split_units(chain)
+        params = [{k: v.astype(np.float64) for k, v in p.items()} for p in wl.make_params(chain, seed=3, bn_affine="random")]
+        fparams = wl.split_params(origin, params)
+        x, labels = wl.make_batch(chain, seed=4)
+        a = no.chain_forward_backward(chain, params, x.astype(np.float64), labels)
+        b = no.chain_forward_backward(fine, fparams, x.astype(np.float64), labels)
+        assert len(fine["units"]) > len(chain["units"])
+        assert abs(a["loss"] - b["loss"]) <= 1e-12 * max(1.0, abs(a["loss"]))
+        np.testing.assert_allclose(a["input_grad"], b["input_grad"], rtol=0, atol=1e-12)
+        for fi, (ui, names) in enumerate(origin):
+            for name in names:
+                if name in params[ui]:
+                    np.testing.assert_allclose(b["grads"][fi][name], a["grads"][ui][name], rtol=0, atol=1e-11)
+        shapes = no.output_shapes(fine)
+        assert [t.shape[1:] for t in b["d"]] == shapes
+        # a relu unit's output is its input clipped; a bn unit's output has per-channel mean beta
+        for fi, u in enumerate(fine["units"]):
+            if u["kind"] == "relu":
+                assert np.array_equal(b["d"][fi + 1], np.maximum(b["d"][fi], 0))
+            if u["kind"] == "bn":
+                np.testing.assert_allclose(b["d"][fi + 1].mean(axis=(0, 1, 2)), fparams[fi]["beta"], atol=1e-12)
