@@ -53,6 +53,7 @@ int ckpt_conv2d_forward(const ckpt_conv_shape* s, int dtype, int impl, const voi
     if (rc) return rc;
     if (!x || !w || !z) { set_error("null tensor"); return CKPT_E_NULL; }
     ConvGeom g = make_geom(*s);
+    if (impl != 1 && tc_first_conv_supported(dtype, g)) return tc_first_conv_fwd(g, x, w, z, op_status_word(), stream);
     if (want_tc(impl, dtype, g, &rc)) return tc_conv_fwd(g, x, w, z, nullptr, 0, scratch, scratch_bytes, op_status_word(), stream);
     if (rc) return rc;
     return simt_conv_fwd(dtype, g, x, w, z, nullptr, 0, stream);

@@ -81,6 +81,8 @@ static int conv_forward_any(StepCtx& c, const ConvGeom& g, const void* x, const 
                             const float* bias, int relu) {
     if (use_tc(c.ch, g))
         return tc_conv_fwd(g, x, w, z, bias, relu, c.ws + c.ch->off_scr, c.ch->scr_bytes, c.status(), c.stream);
+    if (c.ch->impl == 0 && !bias && !relu && tc_first_conv_supported(c.ch->dtype, g))
+        return tc_first_conv_fwd(g, x, w, z, c.status(), c.stream);
     return simt_conv_fwd(c.ch->dtype, g, x, w, z, bias, relu, c.stream);
 }
 static int conv_dgrad_any(StepCtx& c, const ConvGeom& g, const void* dz, const void* w, void* dx) {

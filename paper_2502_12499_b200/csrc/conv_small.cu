@@ -1,8 +1,8 @@
-// First-layer convolution: 3x3, stride 1, padding 1, at most 4 input channels (an RGB image),
-// bf16 storage.  With K = 9*c_in <= 36 the contraction is far too shallow for the tensor cores and
-// the layer is bound by writing its 64-channel output, so it runs on the CUDA cores:
-//   forward: one thread per output pixel, 64 output channels in registers, the filter in shared
-//            memory (read as broadcast float4), the pixel's 128-byte output row written as 8 x 16 B;
+// First-layer convolution: 3x3, stride 1, padding 1, 3 input channels (an RGB image), bf16 storage.
+//   forward: CUDA-core version (the tensor-core version that gathers its operand tiles with plain
+//            loads lives with the other tcgen05 kernels): one thread per output pixel, 64 output
+//            channels in registers, the filter in shared memory (read as broadcast float4), the
+//            pixel's 128-byte output row written as 8 x 16 B;
 //   wgrad  : the input is unfolded to [pixel][9*c_in padded to 64] and the gradient becomes a
 //            [c_out x 64] contraction over pixels on the tensor cores (the 1x1 wgrad kernel).
 #include <cuda_bf16.h>

@@ -897,6 +897,161 @@ tc_wgrad_c64_kernel(const __grid_constant__ CUtensorMap map_dz, const __grid_con
     }
 }
 
+// ------------------------------------------------------------------------------------------------
+// First layer: 3 input channels, 3x3, padding 1, 64 output channels per CTA column.  K = 27 is padded
+// to 32 (two MMAs of K = 16).  Six bytes per pixel cannot be fetched by TMA, so four warps gather
+// the 27 values of their pixel with plain loads and write the operand tile in the layout the other
+// kernels get from TMA (128-byte rows, 16-byte chunk c of row r at position c ^ (r % 8); only the
+// first 64 bytes of a row are ever read).  The filter tile is built once per CTA.  Persistent CTAs,
+// two operand tiles and two 64-column accumulators so that gather, MMA and epilogue of consecutive
+// tiles overlap.  Warps 0-3 gather, warp 4 owns tensor memory and issues the MMAs, warps 5-8 store.
+// ------------------------------------------------------------------------------------------------
+struct FirstParams {
+    int H, W, c_out;
+    long long pixels;
+    int m_tiles;
+};
+constexpr int kFirstThreads = 288;
+
+__global__ void __launch_bounds__(kFirstThreads, 2)
+tc_conv_first_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __restrict__ w, __nv_bfloat16* __restrict__ out,
+                     FirstParams p, int* status) {
+    __shared__ __align__(1024) uint8_t a_tiles[2][128 * 128];
+    __shared__ __align__(1024) uint8_t b_tile[64 * 128];
+    __shared__ __align__(8) uint64_t bar_mem[8];
+    __shared__ uint32_t tmem_base_slot;
+    __shared__ int failed_flag;
+    volatile int* failed = &failed_flag;
+    const uint32_t bars = smem_u32(bar_mem);
+    const uint32_t a_full0 = bars, a_empty0 = bars + 16, acc_full0 = bars + 32, acc_empty0 = bars + 48;
+
+    const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
+    const int co0 = blockIdx.y * 64;
+    const int my_tiles = (int)blockIdx.x < p.m_tiles ? (p.m_tiles - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x : 0;
+
+    if (threadIdx.x == 0) {
+        failed_flag = 0;
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(a_full0 + 8 * b, 128); mbar_init(a_empty0 + 8 * b, 1);
+            mbar_init(acc_full0 + 8 * b, 1); mbar_init(acc_empty0 + 8 * b, 128);
+        }
+        fence_barrier_init();
+    }
+    // filter tile: row = output channel, K = (tap, channel) in the first 27 of 64 columns
+    for (int i = threadIdx.x; i < 64 * 8; i += blockDim.x) {
+        const int co = i / 8, chunk = i % 8;
+        __align__(16) uint16_t v[8];
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+            const int k = chunk * 8 + e;
+            v[e] = k < 27 ? __ldg(reinterpret_cast<const uint16_t*>(w) + (size_t)(co0 + co) * 27 + k) : (uint16_t)0;
+        }
+        *reinterpret_cast<uint4*>(b_tile + co * 128 + ((chunk ^ (co & 7)) * 16)) = *reinterpret_cast<const uint4*>(v);
+    }
+    fence_proxy_async();
+    if ((smem_u32(a_tiles[0]) | smem_u32(b_tile)) & 1023u) {       // the swizzle pattern assumes 1024-byte aligned tiles
+        if (threadIdx.x == 0) atomicCAS(status, 0, 600);
+        return;
+    }
+    if (warp == 4) tmem_alloc(smem_u32(&tmem_base_slot), 128);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = tmem_base_slot;
+
+    if (warp < 4) {
+        // ---------------- gather: thread t builds row t of the operand tile
+        const int t = threadIdx.x;
+        const uint16_t* x16 = reinterpret_cast<const uint16_t*>(x);
+        for (int j = 0; j < my_tiles; ++j) {
+            const int buf = j & 1;
+            const long long pix = ((long long)blockIdx.x + (long long)j * gridDim.x) * 128 + t;
+            __align__(16) uint16_t v[32];
+#pragma unroll
+            for (int e = 0; e < 32; ++e) v[e] = 0;
+            if (pix < p.pixels) {
+                const int ow = (int)(pix % p.W);
+                const int oh = (int)((pix / p.W) % p.H);
+                const long long img = pix / ((long long)p.W * p.H);
+#pragma unroll
+                for (int r = 0; r < 3; ++r) {
+                    const int ih = oh + r - 1;
+                    if (ih < 0 || ih >= p.H) continue;
+                    const uint16_t* row = x16 + ((img * p.H + ih) * p.W + ow) * 3;
+#pragma unroll
+                    for (int s2 = 0; s2 < 3; ++s2) {
+                        const int iw = ow + s2 - 1;
+                        if (iw < 0 || iw >= p.W) continue;
+#pragma unroll
+                        for (int c = 0; c < 3; ++c) v[(r * 3 + s2) * 3 + c] = __ldg(row + (s2 - 1) * 3 + c);
+                    }
+                }
+            }
+            if (!mbar_wait(a_empty0 + 8 * buf, ((uint32_t)(j >> 1) & 1u) ^ 1u, failed, status, 601)) break;
+            uint8_t* dst = a_tiles[buf] + t * 128;
+#pragma unroll
+            for (int chunk = 0; chunk < 4; ++chunk)
+                *reinterpret_cast<uint4*>(dst + ((chunk ^ (t & 7)) * 16)) = reinterpret_cast<const uint4*>(v)[chunk];
+            fence_proxy_async();
+            mbar_arrive(a_full0 + 8 * buf);
+        }
+    } else if (warp == 4) {
+        if (lane == 0) {
+            const uint32_t idesc = instr_desc(128, 64, 0, 0);
+            const uint32_t b_addr = smem_u32(b_tile);
+            for (int j = 0; j < my_tiles; ++j) {
+                const int buf = j & 1;
+                if (!mbar_wait(acc_empty0 + 8 * buf, ((uint32_t)(j >> 1) & 1u) ^ 1u, failed, status, 602)) break;
+                if (!mbar_wait(a_full0 + 8 * buf, (uint32_t)(j >> 1) & 1u, failed, status, 603)) break;
+                tc_fence_after();
+                const uint32_t a_addr = smem_u32(a_tiles[buf]);
+#pragma unroll
+                for (int kk = 0; kk < 2; ++kk)
+                    umma_bf16(tmem_base + (uint32_t)(buf * 64), smem_desc(a_addr + kk * 32, 0, 1024), smem_desc(b_addr + kk * 32, 0, 1024),
+                              idesc, kk > 0 ? 1u : 0u);
+                umma_commit(a_empty0 + 8 * buf);
+                umma_commit(acc_full0 + 8 * buf);
+            }
+        }
+    } else {
+        // ---------------- epilogue: thread = accumulator lane = pixel of the tile
+        const int quarter = warp % 4;
+        const int row = quarter * 32 + lane;
+        for (int j = 0; j < my_tiles; ++j) {
+            const int buf = j & 1;
+            if (!mbar_wait(acc_full0 + 8 * buf, (uint32_t)(j >> 1) & 1u, failed, status, 604)) break;
+            tc_fence_after();
+            const long long pix = ((long long)blockIdx.x + (long long)j * gridDim.x) * 128 + row;
+            __nv_bfloat16* dst = out + pix * p.c_out + co0;
+#pragma unroll
+            for (int c0 = 0; c0 < 64; c0 += 32) {
+                uint32_t v[32];
+                tmem_ld32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * 64 + c0), v);
+                if (pix < p.pixels) {
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        uint4 pk;
+                        __nv_bfloat162* h = reinterpret_cast<__nv_bfloat162*>(&pk);
+#pragma unroll
+                        for (int e = 0; e < 4; ++e)
+                            h[e] = __floats2bfloat162_rn(__uint_as_float(v[8 * q + 2 * e]), __uint_as_float(v[8 * q + 2 * e + 1]));
+                        *reinterpret_cast<uint4*>(dst + c0 + 8 * q) = pk;
+                    }
+                }
+            }
+            tc_fence_before();
+            mbar_arrive(acc_empty0 + 8 * buf);
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 4) {
+        __syncwarp();
+        tc_fence_after();
+        tmem_dealloc(tmem_base, 128);
+    }
+}
+
 // wt[ci][tap'][co] = w[co][taps-1-tap'][ci]: the matrix of the transposed convolution (stride 1).
 __global__ void transpose_flip_kernel(const __nv_bfloat16* __restrict__ w, __nv_bfloat16* __restrict__ wt, int c_out, int taps, int c_in) {
     const int64_t total = (int64_t)c_out * taps * c_in;
@@ -1181,6 +1336,27 @@ int64_t tc_conv_scratch_bytes(const ConvGeom& g) {
     const int64_t elems = (int64_t)g.cout * g.k * g.k * g.cin;
     const int64_t partial = slices > 1 ? (int64_t)slices * elems * 4 : 0;
     return std::max<int64_t>(partial, elems * 2);
+}
+
+bool tc_first_conv_supported(int dtype, const ConvGeom& g) {
+    return dtype == CKPT_DTYPE_BF16 && g.cin == 3 && g.k == 3 && g.stride == 1 && g.pad == 1 && g.cout % 64 == 0;
+}
+
+int tc_first_conv_fwd(const ConvGeom& g, const void* x, const void* w, void* z, int* device_status, void* stream) {
+    if (!tc_first_conv_supported(CKPT_DTYPE_BF16, g)) { set_error("first-layer kernel: unsupported shape"); return CKPT_E_UNSUPPORTED; }
+    if (!device_status) { set_error("device status word missing"); return CKPT_E_NULL; }
+    FirstParams p;
+    p.H = g.h; p.W = g.w; p.c_out = g.cout;
+    p.pixels = (long long)g.n * g.h * g.w;
+    p.m_tiles = (int)((p.pixels + 127) / 128);
+    int sms = 148, dev = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    dim3 grid((unsigned)std::min(p.m_tiles, 2 * sms), (unsigned)(g.cout / 64));
+    tc_conv_first_kernel<<<grid, kFirstThreads, 0, (cudaStream_t)stream>>>((const __nv_bfloat16*)x, (const __nv_bfloat16*)w,
+                                                                          (__nv_bfloat16*)z, p, device_status);
+    CKPT_LAUNCH_CHECK("first-layer conv forward (tensor cores)");
+    return CKPT_OK;
 }
 
 int tc_conv_fwd(const ConvGeom& g, const void* x, const void* w, void* z, const float* bias, int relu, void*, int64_t,

@@ -20,6 +20,7 @@ pytestmark = pytest.mark.gpu
 
 LAYERS = [
     # n, h, w, cin, cout   (3x3, stride 1, padding 1)
+    (64, 224, 224, 3, 64),       # first layer: operand tiles gathered by threads
     (64, 224, 224, 64, 64),
     (64, 112, 112, 64, 128),
     (64, 112, 112, 128, 128),

@@ -123,9 +123,10 @@ def test_conv_tensor_core_kernels(case):
     assert max_rel_err(to_host(z2), to_host(z)) <= TIGHT[dtype]
 
 
-@pytest.mark.parametrize("n,h,w,cout", [(3, 21, 18, 64), (2, 40, 40, 128), (5, 32, 32, 64)])
+@pytest.mark.parametrize("n,h,w,cout", [(3, 21, 18, 64), (2, 40, 40, 128), (5, 32, 32, 64), (1, 5, 3, 64), (7, 96, 80, 64)])
 def test_first_layer_kernels(n, h, w, cout):
-    """3 input channels, bf16, automatic kernel choice: CUDA-core forward, unfolded tensor-core wgrad."""
+    """3 input channels, bf16, automatic kernel choice: tensor-core forward on thread-gathered operand tiles
+    (checked against the CUDA-core kernel too), unfolded tensor-core wgrad."""
     import torch
     dtype = ck.DTYPE_BF16
     rng = np.random.default_rng(n * h + cout)
@@ -147,6 +148,11 @@ def test_first_layer_kernels(n, h, w, cout):
     assert max_rel_err(to_host(z), z_ref) <= TIGHT[dtype]
     assert max_rel_err(to_host(dw), dw_ref) <= 2e-5
     assert torch.equal(dw, dw2)
+    z1 = torch.full(z_ref.shape, float("nan"), device="cuda").to(xd.dtype)
+    ck.conv2d_forward(shape, dtype, 1, xd, wd, z1, scratch)
+    torch.cuda.synchronize()
+    assert max_rel_err(to_host(z1), z_ref) <= TIGHT[dtype]
+    assert not torch.isnan(z.float()).any()
 
 
 @pytest.mark.parametrize("dtype", [ck.DTYPE_F32, ck.DTYPE_BF16])
