@@ -912,8 +912,12 @@ struct FirstParams {
     int m_tiles;
 };
 constexpr int kFirstThreads = 288;
+#ifndef FIRST_CTAS
+#define FIRST_CTAS 3
+#endif
+constexpr int kFirstCtasPerSm = FIRST_CTAS;      // each holds 128 of the 512 tensor-memory columns
 
-__global__ void __launch_bounds__(kFirstThreads, 2)
+__global__ void __launch_bounds__(kFirstThreads, kFirstCtasPerSm)
 tc_conv_first_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __restrict__ w, __nv_bfloat16* __restrict__ out,
                      FirstParams p, int* status) {
     __shared__ __align__(1024) uint8_t a_tiles[2][128 * 128];
@@ -963,13 +967,11 @@ tc_conv_first_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* _
         // ---------------- gather: thread t builds row t of the operand tile
         const int t = threadIdx.x;
         const uint16_t* x16 = reinterpret_cast<const uint16_t*>(x);
-        for (int j = 0; j < my_tiles; ++j) {
-            const int buf = j & 1;
+        auto gather = [&](int j, uint16_t (&v)[32]) {
             const long long pix = ((long long)blockIdx.x + (long long)j * gridDim.x) * 128 + t;
-            __align__(16) uint16_t v[32];
 #pragma unroll
             for (int e = 0; e < 32; ++e) v[e] = 0;
-            if (pix < p.pixels) {
+            if (j < my_tiles && pix < p.pixels) {
                 const int ow = (int)(pix % p.W);
                 const int oh = (int)((pix / p.W) % p.H);
                 const long long img = pix / ((long long)p.W * p.H);
@@ -987,13 +989,22 @@ tc_conv_first_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* _
                     }
                 }
             }
+        };
+        // the loads of tile j+1 are in flight while tile j is written to shared memory
+        __align__(16) uint16_t cur[32], nxt[32];
+        gather(0, cur);
+        for (int j = 0; j < my_tiles; ++j) {
+            const int buf = j & 1;
+            gather(j + 1, nxt);
             if (!mbar_wait(a_empty0 + 8 * buf, ((uint32_t)(j >> 1) & 1u) ^ 1u, failed, status, 601)) break;
             uint8_t* dst = a_tiles[buf] + t * 128;
 #pragma unroll
             for (int chunk = 0; chunk < 4; ++chunk)
-                *reinterpret_cast<uint4*>(dst + ((chunk ^ (t & 7)) * 16)) = reinterpret_cast<const uint4*>(v)[chunk];
+                *reinterpret_cast<uint4*>(dst + ((chunk ^ (t & 7)) * 16)) = reinterpret_cast<const uint4*>(cur)[chunk];
             fence_proxy_async();
             mbar_arrive(a_full0 + 8 * buf);
+#pragma unroll
+            for (int e = 0; e < 32; ++e) cur[e] = nxt[e];
         }
     } else if (warp == 4) {
         if (lane == 0) {
@@ -1352,7 +1363,7 @@ int tc_first_conv_fwd(const ConvGeom& g, const void* x, const void* w, void* z, 
     int sms = 148, dev = 0;
     cudaGetDevice(&dev);
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    dim3 grid((unsigned)std::min(p.m_tiles, 2 * sms), (unsigned)(g.cout / 64));
+    dim3 grid((unsigned)std::min(p.m_tiles, kFirstCtasPerSm * sms), (unsigned)(g.cout / 64));
     tc_conv_first_kernel<<<grid, kFirstThreads, 0, (cudaStream_t)stream>>>((const __nv_bfloat16*)x, (const __nv_bfloat16*)w,
                                                                           (__nv_bfloat16*)z, p, device_status);
     CKPT_LAUNCH_CHECK("first-layer conv forward (tensor cores)");
