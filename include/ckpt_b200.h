@@ -254,6 +254,17 @@ CKPT_API int ckpt_conv2d_dgrad(const ckpt_conv_shape* s, int dtype, int impl, co
 CKPT_API int ckpt_conv2d_wgrad(const ckpt_conv_shape* s, int dtype, int impl, const void* dz, const void* x,
                       float* dw, void* scratch, int64_t scratch_bytes, void* stream);
 
+/* Convolution forward followed by the batch statistics of its output, as the conv+BN+ReLU unit of the
+ * chain runs them (the forward step d_i = f_i(d_{i-1}, w_i) of Eq. (1) up to the point where d_i is
+ * stored): z = conv(x, w) and stats[0..4c) as for ckpt_bn_relu_forward, computed over the stored
+ * (rounded) z.  Where the tensor-core kernel for the shape is a persistent one, the per-channel sums
+ * are gathered in its epilogue and z is not read again; otherwise two kernels run.
+ * scratch: max(ckpt_conv2d_scratch_bytes, ckpt_bn_scratch_bytes(n*h_out*w_out, c_out)) bytes.
+ * fused (host, optional): set to 1 when the sums came from the convolution's epilogue, else 0. */
+CKPT_API int ckpt_conv2d_bn_statistics(const ckpt_conv_shape* s, int dtype, const void* x, const void* w, void* z,
+                              const float* gamma, const float* beta, float* stats, void* scratch,
+                              int64_t scratch_bytes, int32_t* fused, void* stream);
+
 /* Batch normalisation (training mode) + ReLU over rows x channels (rows = N*H*W).
  * forward : stats[0..c) = mean, [c..2c) = 1/sqrt(var+eps), [2c..3c) = scale, [3c..4c) = shift
  *           (y = max(z*scale + shift, 0) when relu != 0, else z*scale+shift).

@@ -291,6 +291,15 @@ def conv2d_forward(shape, dtype, impl, x, w, z, scratch=None, stream=None):
     _check(lib().ckpt_conv2d_forward(C.byref(shape), C.c_int(dtype), C.c_int(impl), _dev(x), _dev(w), _dev(z), sp, sb, _stream(stream)))
 
 
+def conv2d_bn_statistics(shape, dtype, x, w, z, gamma, beta, stats, scratch, stream=None):
+    """ckpt_conv2d_bn_statistics; returns True when the sums were gathered in the convolution's epilogue."""
+    sp, sb = _scratch_args(scratch)
+    fused = C.c_int32(0)
+    _check(lib().ckpt_conv2d_bn_statistics(C.byref(shape), C.c_int(dtype), _dev(x), _dev(w), _dev(z), _dev(gamma), _dev(beta),
+                                           _dev(stats), sp, sb, C.byref(fused), _stream(stream)))
+    return bool(fused.value)
+
+
 def conv2d_dgrad(shape, dtype, impl, dz, w, dx, scratch=None, stream=None):
     sp, sb = _scratch_args(scratch)
     _check(lib().ckpt_conv2d_dgrad(C.byref(shape), C.c_int(dtype), C.c_int(impl), _dev(dz), _dev(w), _dev(dx), sp, sb, _stream(stream)))

@@ -59,6 +59,31 @@ int ckpt_conv2d_forward(const ckpt_conv_shape* s, int dtype, int impl, const voi
     return simt_conv_fwd(dtype, g, x, w, z, nullptr, 0, stream);
 }
 
+int ckpt_conv2d_bn_statistics(const ckpt_conv_shape* s, int dtype, const void* x, const void* w, void* z, const float* gamma,
+                              const float* beta, float* stats, void* scratch, int64_t scratch_bytes, int32_t* fused,
+                              void* stream) {
+    int rc = check_shape(s, dtype);
+    if (rc) return rc;
+    if (!x || !w || !z || !gamma || !beta || !stats || !scratch) { set_error("null tensor"); return CKPT_E_NULL; }
+    ConvGeom g = make_geom(*s);
+    const int64_t rows = (int64_t)g.n * g.ho * g.wo;
+    if (scratch_bytes < bn_scratch_bytes(rows, g.cout)) { set_error("scratch too small for the statistics"); return CKPT_E_WORKSPACE; }
+    if (fused) *fused = 0;
+    if (tc_conv_supported(dtype, g)) {
+        int blocks = 0;
+        if ((rc = tc_conv_fwd_stats(g, x, w, z, (float*)scratch, &blocks, op_status_word(), stream))) return rc;
+        if (blocks > 0) {
+            if (fused) *fused = 1;
+            return bn_statistics_from_partials((const float*)scratch, blocks, rows, g.cout, gamma, beta, stats, stream);
+        }
+    } else if (tc_first_conv_supported(dtype, g)) {
+        if ((rc = tc_first_conv_fwd(g, x, w, z, op_status_word(), stream))) return rc;
+    } else if ((rc = simt_conv_fwd(dtype, g, x, w, z, nullptr, 0, stream))) {
+        return rc;
+    }
+    return bn_statistics(dtype, rows, g.cout, z, gamma, beta, stats, scratch, stream);
+}
+
 int ckpt_conv2d_dgrad(const ckpt_conv_shape* s, int dtype, int impl, const void* dz, const void* w, void* dx,
                       void* scratch, int64_t scratch_bytes, void* stream) {
     int rc = check_shape(s, dtype);

@@ -223,7 +223,15 @@ static int unit_forward(StepCtx& c, int64_t i, const void* x_raw, void* y) {
     switch (u.desc.kind) {
         case CKPT_UNIT_CONV_BN_RELU:
             if ((rc = activated(c, i - 1, x_raw, &x))) return rc;
-            if ((rc = conv_forward_any(c, u.geom, x, p[0], y, nullptr, 0))) return rc;
+            if (use_tc(c.ch, u.geom)) {
+                // the persistent tensor-core kernels gather the statistics of their output in the epilogue
+                int blocks = 0;
+                float* partial = (float*)(ws + c.ch->off_scr);
+                if ((rc = tc_conv_fwd_stats(u.geom, x, p[0], y, partial, &blocks, c.status(), c.stream))) return rc;
+                if (blocks > 0)
+                    return bn_statistics_from_partials(partial, blocks, rows_of(c.ch, i), u.out.c, (const float*)p[1],
+                                                       (const float*)p[2], stats_of(c, i), c.stream);
+            } else if ((rc = conv_forward_any(c, u.geom, x, p[0], y, nullptr, 0))) return rc;
             return bn_statistics(dt, rows_of(c.ch, i), u.out.c, y, (const float*)p[1], (const float*)p[2], stats_of(c, i),
                                  ws + c.ch->off_scr, c.stream);
         case CKPT_UNIT_CONV:

@@ -323,9 +323,53 @@ __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
 
+// Column sums of a 32 x 32 block held one row per lane (v[c] = element of column c in this lane's row):
+// a butterfly of 31 exchanges in a fixed order; afterwards lane l holds the sum of column l.
+__device__ __forceinline__ float warp_column_sum(float (&v)[32], int lane) {
+#pragma unroll
+    for (int o = 16; o >= 1; o >>= 1) {
+        const bool upper = (lane & o) != 0;
+#pragma unroll
+        for (int i = 0; i < o; ++i) {
+            const float send = upper ? v[i] : v[i + o];
+            const float keep = upper ? v[i + o] : v[i];
+            v[i] = keep + __shfl_xor_sync(0xffffffffu, send, o);
+        }
+    }
+    return v[0];
+}
+
+// Epilogue of one 32-column chunk: rounds the accumulators to bf16, stores the valid rows and, when the
+// batch-norm statistics are gathered here, adds the chunk's per-column sum and sum of squares (of
+// the rounded values, i.e. of what is stored) into the lane's running totals.
+__device__ __forceinline__ void store_chunk(const uint32_t (&v)[32], bool valid, __nv_bfloat16* dst, bool stats, int lane,
+                                            float& sum, float& sumsq) {
+    float r[32];
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+        uint4 pk;
+        __nv_bfloat162* h = reinterpret_cast<__nv_bfloat162*>(&pk);
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            h[e] = __floats2bfloat162_rn(__uint_as_float(v[8 * q + 2 * e]), __uint_as_float(v[8 * q + 2 * e + 1]));
+            const float2 f = __bfloat1622float2(h[e]);
+            r[8 * q + 2 * e] = valid ? f.x : 0.f;
+            r[8 * q + 2 * e + 1] = valid ? f.y : 0.f;
+        }
+        if (valid) *reinterpret_cast<uint4*>(dst + 8 * q) = pk;
+    }
+    if (stats) {
+        float sq[32];
+#pragma unroll
+        for (int e = 0; e < 32; ++e) sq[e] = r[e] * r[e];
+        sum += warp_column_sum(r, lane);
+        sumsq += warp_column_sum(sq, lane);
+    }
+}
+
 __global__ void __launch_bounds__(kThreads, 1)
 tc_conv_c64_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w,
-                   __nv_bfloat16* __restrict__ out, C64Params p, int* status) {
+                   __nv_bfloat16* __restrict__ out, float* __restrict__ stat_partial, C64Params p, int* status) {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     constexpr uint32_t w_bytes = 9 * 64 * 128;                       // resident filter
@@ -419,6 +463,8 @@ tc_conv_c64_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_const
         const int quarter = warp % 4;
         const int row = quarter * 32 + lane;
         const int wl = row % 8, hl = row / 8;
+        const bool stats = stat_partial != nullptr;
+        float s_acc[2] = {0.f, 0.f}, q_acc[2] = {0.f, 0.f};
         for (int j = 0; j < my_tiles; ++j) {
             const int b = j & 1;
             if (!mbar_wait(acc_full0 + 8 * b, (uint32_t)(j >> 1) & 1u, failed, status, 305)) break;
@@ -428,23 +474,23 @@ tc_conv_c64_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_const
             const bool valid = hl < p.th && (h0 + hl) < p.H && (w0 + wl) < p.W;
             __nv_bfloat16* dst = out + ((((size_t)img * p.H + (h0 + hl)) * p.W + (w0 + wl)) * p.c_out + (size_t)n_tile * 64);
 #pragma unroll
-            for (int c0 = 0; c0 < 64; c0 += 32) {
+            for (int ci = 0; ci < 2; ++ci) {
                 uint32_t v[32];
-                tmem_ld32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(b * 64 + c0), v);
-                if (valid) {
-#pragma unroll
-                    for (int q = 0; q < 4; ++q) {
-                        uint4 pk;
-                        __nv_bfloat162* h = reinterpret_cast<__nv_bfloat162*>(&pk);
-#pragma unroll
-                        for (int e = 0; e < 4; ++e)
-                            h[e] = __floats2bfloat162_rn(__uint_as_float(v[8 * q + 2 * e]), __uint_as_float(v[8 * q + 2 * e + 1]));
-                        *reinterpret_cast<uint4*>(dst + c0 + 8 * q) = pk;
-                    }
-                }
+                tmem_ld32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(b * 64 + ci * 32), v);
+                store_chunk(v, valid, dst + ci * 32, stats, lane, s_acc[ci], q_acc[ci]);
             }
             tc_fence_before();
             mbar_arrive(acc_empty0 + 8 * b);
+        }
+        if (stats) {
+            // one block of partial sums per epilogue warp: [block][sum | sum of squares][channel]
+            const size_t blk = (size_t)first * 4 + quarter;
+#pragma unroll
+            for (int ci = 0; ci < 2; ++ci) {
+                const int ch = n_tile * 64 + ci * 32 + lane;
+                stat_partial[(blk * 2) * p.c_out + ch] = s_acc[ci];
+                stat_partial[(blk * 2 + 1) * p.c_out + ch] = q_acc[ci];
+            }
         }
     }
     tc_fence_before();
@@ -474,7 +520,7 @@ struct HaloParams {
 
 __global__ void __launch_bounds__(kThreads, 1)
 tc_conv_halo_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w,
-                    __nv_bfloat16* __restrict__ out, HaloParams p, int* status) {
+                    __nv_bfloat16* __restrict__ out, float* __restrict__ stat_partial, HaloParams p, int* status) {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const uint32_t a_slot_bytes = 3 * p.box_stride, b_slot_bytes = (uint32_t)p.bn * 128;
@@ -594,6 +640,10 @@ tc_conv_halo_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_cons
         const int quarter = warp % 4;
         const int row = quarter * 32 + lane;
         const int wl = row % 8, hl = row / 8;
+        const bool stats = stat_partial != nullptr;
+        float s_acc[8], q_acc[8];
+#pragma unroll
+        for (int ci = 0; ci < 8; ++ci) { s_acc[ci] = 0.f; q_acc[ci] = 0.f; }
         for (int j = 0; j < my_tiles; ++j) {
             const int buf = j & 1;
             if (!mbar_wait(acc_full0 + 8 * buf, (uint32_t)(j >> 1) & 1u, failed, status, 506)) break;
@@ -602,23 +652,27 @@ tc_conv_halo_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_cons
             tile_origin(j, w0, h0, img);
             const bool valid = hl < p.th && (h0 + hl) < p.H && (w0 + wl) < p.W;
             __nv_bfloat16* dst = out + ((((size_t)img * p.H + (h0 + hl)) * p.W + (w0 + wl)) * p.c_out + (size_t)n_tile * p.bn);
-            for (int c0 = 0; c0 < p.bn; c0 += 32) {
-                uint32_t v[32];
-                tmem_ld32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * p.bn + c0), v);
-                if (valid) {
 #pragma unroll
-                    for (int q = 0; q < 4; ++q) {
-                        uint4 pk;
-                        __nv_bfloat162* h = reinterpret_cast<__nv_bfloat162*>(&pk);
-#pragma unroll
-                        for (int e = 0; e < 4; ++e)
-                            h[e] = __floats2bfloat162_rn(__uint_as_float(v[8 * q + 2 * e]), __uint_as_float(v[8 * q + 2 * e + 1]));
-                        *reinterpret_cast<uint4*>(dst + c0 + 8 * q) = pk;
-                    }
+            for (int ci = 0; ci < 8; ++ci) {
+                if (ci * 32 < p.bn) {
+                    uint32_t v[32];
+                    tmem_ld32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * p.bn + ci * 32), v);
+                    store_chunk(v, valid, dst + ci * 32, stats, lane, s_acc[ci], q_acc[ci]);
                 }
             }
             tc_fence_before();
             mbar_arrive(acc_empty0 + 8 * buf);
+        }
+        if (stats) {
+            const size_t blk = (size_t)first * 4 + quarter;
+#pragma unroll
+            for (int ci = 0; ci < 8; ++ci) {
+                if (ci * 32 < p.bn) {
+                    const int ch = n_tile * p.bn + ci * 32 + lane;
+                    stat_partial[(blk * 2) * p.c_out + ch] = s_acc[ci];
+                    stat_partial[(blk * 2 + 1) * p.c_out + ch] = q_acc[ci];
+                }
+            }
         }
     }
     tc_fence_before();
@@ -1156,8 +1210,8 @@ void choose_tile(int pixels, int W, int H, int N, int* tw, int* th, int* tn) {
 
 int pick_bn(int c_out) { return c_out % 256 == 0 ? 256 : (c_out % 128 == 0 ? 128 : 64); }
 
-int launch_c64(const void* x, const void* w_mat, void* out, int N, int H, int W, int c_out, int* status, cudaStream_t st,
-               const char* what) {
+int launch_c64(const void* x, const void* w_mat, void* out, float* stat_partial, int* stat_blocks, int N, int H, int W, int c_out,
+               int* status, cudaStream_t st, const char* what) {
     C64Params p;
     p.H = H; p.W = W; p.N = N; p.c_out = c_out;
     const int nt = (H + 15) / 16;
@@ -1184,8 +1238,9 @@ int launch_c64(const void* x, const void* w_mat, void* out, int N, int H, int W,
         if (e != cudaSuccess) return cuda_fail(e, "raising the shared-memory limit");
         attr_set = true;
     }
-    tc_conv_c64_kernel<<<p.ctas_per_n * p.n_tiles, kThreads, smem, st>>>(mx, mw, (__nv_bfloat16*)out, p, status);
+    tc_conv_c64_kernel<<<p.ctas_per_n * p.n_tiles, kThreads, smem, st>>>(mx, mw, (__nv_bfloat16*)out, stat_partial, p, status);
     CKPT_LAUNCH_CHECK(what);
+    if (stat_blocks) *stat_blocks = 4 * p.ctas_per_n;
     return CKPT_OK;
 }
 
@@ -1197,8 +1252,8 @@ bool halo_applies(int H, int W, int c_red, int c_out, int k, int pad) {
     return 8 * th >= 112 && H % th == 0;
 }
 
-int launch_halo(const void* x, const void* w_mat, void* out, int N, int H, int W, int c_red, int c_out, int* status,
-                cudaStream_t st, const char* what) {
+int launch_halo(const void* x, const void* w_mat, void* out, float* stat_partial, int* stat_blocks, int N, int H, int W, int c_red,
+                int c_out, int* status, cudaStream_t st, const char* what) {
     HaloParams p;
     p.H = H; p.W = W; p.N = N; p.c_red = c_red; p.c_out = c_out;
     const int nt = (H + 15) / 16;
@@ -1227,17 +1282,27 @@ int launch_halo(const void* x, const void* w_mat, void* out, int N, int H, int W
         if (e != cudaSuccess) return cuda_fail(e, "raising the shared-memory limit");
         attr_set = true;
     }
-    tc_conv_halo_kernel<<<p.ctas_per_n * p.n_tiles, kThreads, smem, st>>>(mx, mw, (__nv_bfloat16*)out, p, status);
+    tc_conv_halo_kernel<<<p.ctas_per_n * p.n_tiles, kThreads, smem, st>>>(mx, mw, (__nv_bfloat16*)out, stat_partial, p, status);
     CKPT_LAUNCH_CHECK(what);
+    if (stat_blocks) *stat_blocks = 4 * p.ctas_per_n;
     return CKPT_OK;
 }
 
+// The persistent kernels can gather the per-channel sums of their output on the way out.
+bool persistent_applies(int H, int W, int c_red, int c_out, int k, int pad) {
+    return (c_red == 64 && k == 3 && pad == 1 && c_out % 64 == 0) || halo_applies(H, W, c_red, c_out, k, pad);
+}
+
+// stat_partial / stat_blocks: null, or where the kernel leaves the batch-norm partial sums of its output
+// ([block][sum | sum of squares][c_out] floats) and how many blocks it wrote (0 = this kernel does not gather them).
 int launch_fwd_like(const void* x, const void* w_mat, void* out, const float* bias, int relu, int N, int H, int W, int c_red,
-                    int c_out, int k, int pad, int* status, cudaStream_t st, const char* what) {
+                    int c_out, int k, int pad, int* status, cudaStream_t st, const char* what, float* stat_partial = nullptr,
+                    int* stat_blocks = nullptr) {
+    if (stat_blocks) *stat_blocks = 0;
     if (c_red == 64 && k == 3 && pad == 1 && c_out % 64 == 0 && !bias && !relu)
-        return launch_c64(x, w_mat, out, N, H, W, c_out, status, st, what);
+        return launch_c64(x, w_mat, out, stat_partial, stat_blocks, N, H, W, c_out, status, st, what);
     if (!bias && !relu && halo_applies(H, W, c_red, c_out, k, pad))
-        return launch_halo(x, w_mat, out, N, H, W, c_red, c_out, status, st, what);
+        return launch_halo(x, w_mat, out, stat_partial, stat_blocks, N, H, W, c_red, c_out, status, st, what);
     FwdParams p;
     p.H = H; p.W = W; p.N = N; p.c_red = c_red; p.c_out = c_out; p.k = k; p.pad = pad;
     choose_tile(128, W, H, N, &p.tw, &p.th, &p.tn);
@@ -1368,6 +1433,16 @@ int tc_first_conv_fwd(const ConvGeom& g, const void* x, const void* w, void* z, 
                                                                           (__nv_bfloat16*)z, p, device_status);
     CKPT_LAUNCH_CHECK("first-layer conv forward (tensor cores)");
     return CKPT_OK;
+}
+
+// Forward convolution that also leaves the batch-norm partial sums of its output in `partial`
+// (*blocks of them; 0 when the kernel chosen for this shape does not gather them).
+int tc_conv_fwd_stats(const ConvGeom& g, const void* x, const void* w, void* z, float* partial, int* blocks, int* device_status,
+                      void* stream) {
+    if (!tc_conv_supported(CKPT_DTYPE_BF16, g)) { set_error("tensor-core conv: unsupported shape"); return CKPT_E_UNSUPPORTED; }
+    if (!device_status || !blocks) { set_error("device status word missing"); return CKPT_E_NULL; }
+    return launch_fwd_like(x, w, z, nullptr, 0, g.n, g.h, g.w, g.cin, g.cout, g.k, g.pad, device_status, (cudaStream_t)stream,
+                           "conv forward (tensor cores)", partial, blocks);
 }
 
 int tc_conv_fwd(const ConvGeom& g, const void* x, const void* w, void* z, const float* bias, int relu, void*, int64_t,

@@ -83,6 +83,10 @@ bool tc_conv_supported(int dtype, const ConvGeom& g);
 int64_t tc_conv_scratch_bytes(const ConvGeom& g);
 int tc_conv_fwd(const ConvGeom& g, const void* x, const void* w, void* z, const float* bias, int relu,
                 void* scratch, int64_t scratch_bytes, int* device_status, void* stream);
+// Forward that also writes the batch-norm partial sums of its output ([blocks][sum | sum of squares][c_out]
+// floats, at most 4 per SM); *blocks == 0 when the kernel for this shape does not gather them.
+int tc_conv_fwd_stats(const ConvGeom& g, const void* x, const void* w, void* z, float* partial, int* blocks,
+                      int* device_status, void* stream);
 int tc_conv_dgrad(const ConvGeom& g, const void* dz, const void* w, void* dx, void* scratch,
                   int64_t scratch_bytes, int* device_status, void* stream);
 int tc_conv_wgrad(const ConvGeom& g, const void* dz, const void* x, float* dw, void* scratch,
@@ -98,6 +102,8 @@ int bn_relu_backward(int dtype, int64_t rows, int c, const void* dy, const void*
 // stats = the 4*c floats written by bn_statistics (mean, 1/std, scale, shift).
 int bn_statistics(int dtype, int64_t rows, int c, const void* z, const float* gamma, const float* beta, float* stats,
                   void* scratch, void* stream);
+int bn_statistics_from_partials(const float* partial, int blocks, int64_t rows, int c, const float* gamma, const float* beta,
+                                float* stats, void* stream);
 int bn_apply(int dtype, int64_t rows, int c, const void* z, const float* stats, int relu, void* y, void* stream);
 
 // y = max(z*scale + shift + shortcut, 0); the shortcut is activated data, or pre-normalisation data with

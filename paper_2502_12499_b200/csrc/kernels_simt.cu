@@ -672,6 +672,15 @@ static int bn_backward_t(int64_t rows, int c, const void* dy, const void* z, con
     return CKPT_OK;
 }
 
+// Statistics from partial sums that another kernel (a convolution epilogue) has already written:
+// partial = [blocks][sum | sum of squares][c] floats.
+int bn_statistics_from_partials(const float* partial, int blocks, int64_t rows, int c, const float* gamma, const float* beta,
+                                float* stats, void* stream) {
+    bn_finalize_fwd_kernel<<<c, 32, 0, (cudaStream_t)stream>>>(partial, blocks, c, 1.0 / (double)rows, gamma, beta, stats);
+    CKPT_LAUNCH_CHECK("batch-norm finalize");
+    return CKPT_OK;
+}
+
 int bn_statistics(int dtype, int64_t rows, int c, const void* z, const float* gamma, const float* beta, float* stats,
                   void* scratch, void* stream) {
     cudaStream_t st = (cudaStream_t)stream;

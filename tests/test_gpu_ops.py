@@ -155,6 +155,65 @@ def test_first_layer_kernels(n, h, w, cout):
     assert not torch.isnan(z.float()).any()
 
 
+@pytest.mark.parametrize("case,expect_fused", [
+    ((8, 56, 56, 64, 64, 3, 1), True),        # 64-channel persistent kernel, two tiles for some CTAs
+    ((3, 13, 19, 64, 128, 3, 1), True),       # ragged tiles: rows outside the image must not count
+    ((2, 112, 112, 128, 128, 3, 1), True),    # halo-patch kernel, 128-wide output tile
+    ((4, 56, 56, 128, 256, 3, 1), True),      # halo-patch kernel, 256-wide output tile
+    ((2, 14, 14, 192, 64, 3, 1), False),      # generic tensor-core kernel + separate statistics kernel
+    ((3, 21, 18, 3, 64, 3, 1), False),        # first-layer kernel + separate statistics kernel
+    ((2, 9, 9, 16, 24, 3, 1), False),         # CUDA-core kernel + separate statistics kernel
+])
+def test_conv_bn_statistics(case, expect_fused):
+    """Convolution + batch statistics of its stored output (gathered in the epilogue of the persistent
+    tensor-core kernels) against the oracle's convolution, bf16 rounding and batch norm."""
+    import torch
+    dtype = ck.DTYPE_BF16
+    n, h, w, cin, cout, k, pad = case
+    rng = np.random.default_rng(sum(case))
+    x = rounded(rng.standard_normal((n, h, w, cin)) + 0.3, dtype)
+    wt = rounded(rng.standard_normal((cout, k, k, cin)) / np.sqrt(k * k * cin), dtype)
+    gamma = rng.uniform(0.5, 1.5, cout).astype(np.float32)
+    beta = (rng.standard_normal(cout) * 0.3).astype(np.float32)
+    z_ref = no.round_bf16(no.conv2d_fwd(x.astype(np.float64), wt.astype(np.float64), 1, pad))
+    y_ref, (xhat, inv_std) = no.bn_fwd(z_ref, gamma.astype(np.float64), beta.astype(np.float64))
+    mean_ref = z_ref.mean(axis=(0, 1, 2))
+    shape = ck.ConvShape(n, h, w, cin, cout, k, 1, pad)
+    rows = n * h * w
+    xd, wd = to_dev(x, dtype), to_dev(wt, dtype)
+    gd, bd = torch.from_numpy(gamma).cuda(), torch.from_numpy(beta).cuda()
+    scratch = torch.empty(max(ck.conv2d_scratch_bytes(shape, dtype), ck.bn_scratch_bytes(rows, cout)), dtype=torch.uint8, device="cuda")
+    outs = []
+    for rep in range(2):
+        z = torch.full(z_ref.shape, float("nan"), device="cuda").to(xd.dtype)
+        stats = torch.full((4 * cout,), float("nan"), device="cuda")
+        scratch.fill_(0xFF)
+        fused = ck.conv2d_bn_statistics(shape, dtype, xd, wd, z, gd, bd, stats, scratch)
+        torch.cuda.synchronize()
+        assert fused == expect_fused
+        outs.append((z, stats))
+    assert torch.equal(outs[0][0], outs[1][0]) and torch.equal(outs[0][1], outs[1][1])
+    z, stats = outs[0]
+    st = to_host(stats).astype(np.float64)
+    mean, inv, scale, shift = st[:cout], st[cout:2 * cout], st[2 * cout:3 * cout], st[3 * cout:]
+    assert max_rel_err(to_host(z), z_ref) <= TIGHT[dtype]
+    std_ref = 1.0 / inv_std
+    assert np.abs(mean - mean_ref).max() <= 2e-3 * std_ref.max()
+    assert max_rel_err(inv, inv_std) <= 5e-4
+    assert max_rel_err(scale, gamma * inv_std) <= 5e-4
+    assert np.abs(shift - (beta - mean_ref * gamma * inv_std)).max() <= 3e-3
+    # the normalised tensor that a consumer of (z, stats) would see
+    y = to_host(z).astype(np.float64) * scale + shift
+    assert max_rel_err(y, y_ref) <= 1e-2
+    # the stand-alone statistics kernel on the same stored tensor agrees to accumulation order
+    stats2 = torch.empty_like(stats)
+    y2 = torch.empty_like(z)
+    ck.bn_relu_forward(dtype, rows, cout, z, gd, bd, 0, y2, stats2, scratch)
+    torch.cuda.synchronize()
+    assert max_rel_err(to_host(stats2[cout:2 * cout]), inv) <= 1e-5
+    assert np.abs(to_host(stats2[:cout]) - mean).max() <= 1e-5 * max(1.0, np.abs(mean).max())
+
+
 @pytest.mark.parametrize("dtype", [ck.DTYPE_F32, ck.DTYPE_BF16])
 @pytest.mark.parametrize("rows,c,relu", [(37, 3, 1), (4096, 16, 1), (5000, 64, 1), (777, 40, 0), (64, 1000, 0), (3001, 24, 1)])
 def test_batchnorm_relu(rows, c, relu, dtype):
