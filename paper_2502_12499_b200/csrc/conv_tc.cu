@@ -952,6 +952,142 @@ tc_wgrad_c64_kernel(const __grid_constant__ CUtensorMap map_dz, const __grid_con
 }
 
 // ------------------------------------------------------------------------------------------------
+// wgrad, 3x3, padding 1, an even number of 64-channel input blocks: the vertical taps share their loads.
+// A "column" is (input-channel block, horizontal tap offset dx).  Per pixel tile (8 wide x th high,
+// one image) the CTA loads the dz tile (128 output channels) once and, for each of its two columns,
+// ONE input patch with a one-row halo above and below, shifted by dx; the three vertical taps of a
+// column are the three 64-element blocks of one MN-major B operand, 1024 bytes (one 8-pixel patch
+// row) apart, so a single MMA of N = 192 covers them:
+//   D[c_out 128][(dy, c_in) 192] += dZ^T[c_out][pixels] * Xpatch[pixels + dy rows][c_in]
+// Per 16 pixels the tensor core reads 4 KB of A and 6 KB of B for 96 clocks of work (107 B/clk of the
+// 128 B/clk shared-memory port) and the stage's 60-68 KB arrive over 1300-1500 clocks (45 B/clk),
+// against 94 B/clk for one box per tap.  Two accumulators of 192 columns live in tensor memory.
+// ------------------------------------------------------------------------------------------------
+struct WRowsParams {
+    int H, W, N, c_out, c_in;
+    int th, tiles_w, tiles_h, m_tiles;
+    int slices;                  // persistent CTAs along the pixel range
+    int stages;
+    uint32_t dz_box, patch_bytes, stage_bytes;
+};
+
+__global__ void __launch_bounds__(kThreads, 1)
+tc_wgrad_rows_kernel(const __grid_constant__ CUtensorMap map_dz, const __grid_constant__ CUtensorMap map_x,
+                     float* __restrict__ partial, WRowsParams p, int* status) {
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    const uint32_t bars = base + (uint32_t)p.stages * p.stage_bytes;
+    __shared__ uint32_t tmem_base_slot;
+    __shared__ int failed_flag;
+    volatile int* failed = &failed_flag;
+    auto full_bar = [&](int s) { return bars + 8u * s; };
+    auto empty_bar = [&](int s) { return bars + 8u * (kMaxStages + s); };
+    const uint32_t accum_bar = bars + 8u * (2 * kMaxStages);
+
+    const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
+    const int slice = blockIdx.x, pair = blockIdx.y, co_tile = blockIdx.z;
+    const int my_tiles = slice < p.m_tiles ? (p.m_tiles - slice + p.slices - 1) / p.slices : 0;
+    const int cin_blocks = p.c_in / 64;
+
+    if (threadIdx.x == 0) {
+        failed_flag = 0;
+        for (int s = 0; s < p.stages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+        mbar_init(accum_bar, 1);
+        fence_barrier_init();
+        tma_prefetch_desc(&map_dz);
+        tma_prefetch_desc(&map_x);
+    }
+    if (warp == 1) tmem_alloc(smem_u32(&tmem_base_slot), 512);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = tmem_base_slot;
+
+    if (warp == 0) {
+        // four copies per stage, one lane each; every lane watches the barrier itself
+        int issued = 0;
+        for (int j = 0; j < my_tiles; ++j) {
+            const int s = j % p.stages;
+            if (!mbar_wait(empty_bar(s), (((uint32_t)(j / p.stages)) & 1u) ^ 1u, failed, status, 701)) break;
+            int t = slice + j * p.slices;
+            const int w0 = (t % p.tiles_w) * 8; t /= p.tiles_w;
+            const int h0 = (t % p.tiles_h) * p.th;
+            const int img = t / p.tiles_h;
+            if (lane == 0) mbar_expect_tx(full_bar(s), 2 * p.dz_box + 2 * p.patch_bytes);
+            __syncwarp();
+            const uint32_t dst = base + (uint32_t)s * p.stage_bytes;
+            if (lane < 2) {
+                tma_load_4d(dst + lane * p.dz_box, &map_dz, full_bar(s), co_tile * 128 + 64 * lane, w0, h0, img);
+            } else if (lane < 4) {
+                const int col = 2 * pair + (lane - 2), cib = col / 3, dx = col % 3;
+                tma_load_4d(dst + 2 * p.dz_box + (lane - 2) * p.patch_bytes, &map_x, full_bar(s), cib * 64, w0 + dx - 1, h0 - 1, img);
+            }
+            issued = j + 1;
+        }
+        if (*failed && lane == 0)
+            for (int j = max(0, issued - p.stages); j < issued; ++j) mbar_drain(full_bar(j % p.stages), (uint32_t)(j / p.stages) & 1u);
+    } else if (warp == 1 && lane == 0) {
+        const uint32_t idesc = instr_desc(128, 192, 1, 1);
+        const int ksteps = p.th / 2;                 // 16 pixels (two 8-pixel rows) per MMA
+        bool ok = true;
+        for (int j = 0; j < my_tiles && ok; ++j) {
+            const int s = j % p.stages;
+            if (!mbar_wait(full_bar(s), (uint32_t)(j / p.stages) & 1u, failed, status, 702)) { ok = false; break; }
+            tc_fence_after();
+            const uint32_t dz_addr = base + (uint32_t)s * p.stage_bytes;
+#pragma unroll 1
+            for (int c = 0; c < 2; ++c) {
+                const uint32_t x_addr = dz_addr + 2 * p.dz_box + (uint32_t)c * p.patch_bytes;
+                for (int kk = 0; kk < ksteps; ++kk)
+                    umma_bf16(tmem_base + (uint32_t)c * 192, smem_desc(dz_addr + kk * 2048, p.dz_box, 1024),
+                              smem_desc(x_addr + kk * 2048, 1024, 1024), idesc, (j > 0 || kk > 0) ? 1u : 0u);
+            }
+            umma_commit(empty_bar(s));
+        }
+        if (ok) umma_commit(accum_bar);
+    } else if (warp >= 2) {
+        const int quarter = warp % 4;
+        const int co = co_tile * 128 + quarter * 32 + lane;
+        const bool valid = co < p.c_out;
+        const size_t row_elems = (size_t)9 * p.c_in;
+        float* dst_row = partial + ((size_t)slice * p.c_out + (valid ? co : 0)) * row_elems;
+        if (my_tiles > 0 && mbar_wait(accum_bar, 0, failed, status, 703)) {
+            tc_fence_after();
+            for (int c = 0; c < 2; ++c) {
+                const int col = 2 * pair + c, cib = col / 3, dx = col % 3;
+                for (int dy = 0; dy < 3; ++dy) {
+                    float* dst = dst_row + (size_t)((dy * 3 + dx) * cin_blocks + cib) * 64;   // column (tap, c_in)
+#pragma unroll
+                    for (int c0 = 0; c0 < 64; c0 += 32) {
+                        uint32_t v[32];
+                        tmem_ld32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(c * 192 + dy * 64 + c0), v);
+                        if (valid) {
+#pragma unroll
+                            for (int e = 0; e < 8; ++e)
+                                *reinterpret_cast<float4*>(dst + c0 + 4 * e) =
+                                    make_float4(__uint_as_float(v[4 * e]), __uint_as_float(v[4 * e + 1]), __uint_as_float(v[4 * e + 2]), __uint_as_float(v[4 * e + 3]));
+                        }
+                    }
+                }
+            }
+        } else if (my_tiles == 0 && valid) {
+            for (int c = 0; c < 2; ++c) {
+                const int col = 2 * pair + c, cib = col / 3, dx = col % 3;
+                for (int dy = 0; dy < 3; ++dy)
+                    for (int e = 0; e < 64; ++e) dst_row[(size_t)((dy * 3 + dx) * cin_blocks + cib) * 64 + e] = 0.f;
+            }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        __syncwarp();
+        tc_fence_after();
+        tmem_dealloc(tmem_base, 512);
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
 // First layer: 3 input channels, 3x3, padding 1, 64 output channels per CTA column.  K = 27 is padded
 // to 32 (two MMAs of K = 16).  Six bytes per pixel cannot be fetched by TMA, so four warps gather
 // the 27 values of their pixel with plain loads and write the operand tile in the layout the other
@@ -1388,6 +1524,34 @@ void wgrad_c64_plan(const ConvGeom& g, W64Params* p) {
 }
 }  // namespace
 
+namespace {
+#ifndef WROWS_MIN_W
+#define WROWS_MIN_W 14
+#endif
+bool wgrad_rows_applies(const ConvGeom& g) {
+    return g.k == 3 && g.pad == 1 && g.stride == 1 && g.cin % 128 == 0 && g.cout % 64 == 0 && g.w >= WROWS_MIN_W && g.h >= 8;
+}
+void wgrad_rows_plan(const ConvGeom& g, WRowsParams* p, int* pairs, int* co_tiles) {
+    p->H = g.h; p->W = g.w; p->N = g.n; p->c_out = g.cout; p->c_in = g.cin;
+    const int nt = (g.h + 15) / 16;
+    p->th = ((g.h + nt - 1) / nt + 1) / 2 * 2;                   // even: an MMA spans two 8-pixel rows
+    p->tiles_h = (g.h + p->th - 1) / p->th;
+    p->tiles_w = (g.w + 7) / 8;
+    p->m_tiles = p->tiles_w * p->tiles_h * g.n;
+    *pairs = 3 * (g.cin / 64) / 2;
+    *co_tiles = (g.cout + 127) / 128;
+    int sms = 148, dev = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    const int base_ctas = *pairs * *co_tiles;
+    p->slices = std::max(1, std::min(sms / base_ctas, p->m_tiles));
+    p->dz_box = (uint32_t)(8 * p->th) * 128;
+    p->patch_bytes = (uint32_t)(8 * (p->th + 2)) * 128;
+    p->stage_bytes = 2 * p->dz_box + 2 * p->patch_bytes;
+    p->stages = std::max(2, std::min<int>(kMaxStages, (int)((208 * 1024) / p->stage_bytes)));
+}
+}  // namespace
+
 bool tc_conv_supported(int dtype, const ConvGeom& g) {
     if (dtype != CKPT_DTYPE_BF16) return false;
     if (g.stride != 1) return false;
@@ -1410,7 +1574,13 @@ int64_t tc_conv_scratch_bytes(const ConvGeom& g) {
     int slices, groups, co_tiles;
     wgrad_plan(g, &p, &slices, &groups, &co_tiles);
     const int64_t elems = (int64_t)g.cout * g.k * g.k * g.cin;
-    const int64_t partial = slices > 1 ? (int64_t)slices * elems * 4 : 0;
+    int64_t partial = slices > 1 ? (int64_t)slices * elems * 4 : 0;
+    if (wgrad_rows_applies(g)) {
+        WRowsParams q;
+        int pairs, tiles;
+        wgrad_rows_plan(g, &q, &pairs, &tiles);
+        partial = std::max<int64_t>(partial, (int64_t)q.slices * elems * 4);
+    }
     return std::max<int64_t>(partial, elems * 2);
 }
 
@@ -1495,6 +1665,32 @@ int tc_conv_wgrad(const ConvGeom& g, const void* dz, const void* x, float* dw, v
         dim3 grid(p.slices, g.cout / 64);
         tc_wgrad_c64_kernel<<<grid, kThreads, smem, st>>>(mdz, mx, (float*)scratch, p, device_status);
         CKPT_LAUNCH_CHECK("conv wgrad, 64 input channels (tensor cores)");
+        slice_sum_tc_kernel<<<(unsigned)((elems + 255) / 256), 256, 0, st>>>((const float*)scratch, dw, elems, p.slices);
+        CKPT_LAUNCH_CHECK("wgrad slice sum");
+        return CKPT_OK;
+    }
+    if (wgrad_rows_applies(g)) {
+        WRowsParams p;
+        int pairs, co_tiles;
+        wgrad_rows_plan(g, &p, &pairs, &co_tiles);
+        const int64_t elems = (int64_t)g.cout * 9 * g.cin;
+        if (!scratch || scratch_bytes < (int64_t)p.slices * elems * 4) { set_error("wgrad scratch too small"); return CKPT_E_WORKSPACE; }
+        CUtensorMap mdz, mx;
+        int rc = make_act_map(&mdz, dz, g.n, g.h, g.w, g.cout, 8, p.th, 1);
+        if (rc) return rc;
+        rc = make_act_map(&mx, x, g.n, g.h, g.w, g.cin, 8, p.th + 2, 1);
+        if (rc) return rc;
+        cudaStream_t st = (cudaStream_t)stream;
+        static bool attr_set = false;
+        if (!attr_set) {
+            cudaError_t e = cudaFuncSetAttribute(tc_wgrad_rows_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 222 * 1024);
+            if (e != cudaSuccess) return cuda_fail(e, "raising the shared-memory limit");
+            attr_set = true;
+        }
+        const size_t smem = (size_t)p.stages * p.stage_bytes + 1024 + 256;
+        dim3 grid(p.slices, pairs, co_tiles);
+        tc_wgrad_rows_kernel<<<grid, kThreads, smem, st>>>(mdz, mx, (float*)scratch, p, device_status);
+        CKPT_LAUNCH_CHECK("conv wgrad, shared vertical taps (tensor cores)");
         slice_sum_tc_kernel<<<(unsigned)((elems + 255) / 256), 256, 0, st>>>((const float*)scratch, dw, elems, p.slices);
         CKPT_LAUNCH_CHECK("wgrad slice sum");
         return CKPT_OK;
