@@ -7,7 +7,8 @@
 //             A = one TMA box of the NHWC input per (tap, block): 128 pixels x 64 channels; the
 //             hardware zero-fills coordinates outside the image, which is the padding.
 //             B = one TMA box of the [c_out][k*k*c_in] matrix.  Both operands K-major.
-//   dgrad   : the same kernel on dz with the matrix transposed and the taps reversed (stride 1).
+//   dgrad   : the same kernels on dz with the matrix transposed and the taps reversed (stride 1); a 1x1 filter
+//             is read in place as an MN-major B operand (reduction channel = row), without a transposed copy.
 //   wgrad   : D[c_out][(tap, c_in)] = sum over pixels of dz[pixel][c_out] * x[pixel shifted][c_in]
 //             Both operands are pixel-major in memory, i.e. MN-major for the tensor core; the
 //             pixel range is split over CTAs and the partial results are added in a fixed order.
@@ -173,6 +174,7 @@ struct FwdParams {
     int stages;
 };
 
+template <bool B_MN>
 __global__ void __launch_bounds__(kThreads, 1)
 tc_conv_fwd_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w,
                    __nv_bfloat16* __restrict__ out, const float* __restrict__ bias, int relu, FwdParams p, int* status) {
@@ -213,8 +215,10 @@ tc_conv_fwd_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_const
     tc_fence_after();
     const uint32_t tmem_base = tmem_base_slot;
 
-    if (warp == 0 && lane == 0) {
-        // ---------------- TMA producer (two copies per stage: measured fastest from a single thread)
+    if (warp == 0 && (lane == 0 || B_MN)) {
+        // ---------------- TMA producer.  Filter as a [c_out][k*k*c_red] matrix: two copies per stage, measured
+        // fastest from a single thread.  Filter read in place for a 1x1 dgrad (B_MN): the tile is bn/64 boxes of
+        // 64 reduction channels x 64 output channels, one lane per copy, every lane watching the barrier.
         int issued = 0;
         for (int it = 0; it < iters; ++it) {
             const int s = it % p.stages;
@@ -222,20 +226,29 @@ tc_conv_fwd_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_const
             if (!mbar_wait(empty_bar(s), phase ^ 1u, failed, status, 101)) break;
             const int tap = it / blocks, blk = it % blocks;
             const int r = tap / p.k, q = tap % p.k;
-            mbar_expect_tx(full_bar(s), stage_bytes);
             const uint32_t a_dst = base + (uint32_t)s * stage_bytes;
-            tma_load_4d(a_dst, &map_x, full_bar(s), blk * 64, w0 + q - p.pad, h0 + r - p.pad, n0);
-            tma_load_2d(a_dst + a_bytes, &map_w, full_bar(s), tap * p.c_red + blk * 64, n_tile * p.bn);
+            if (lane == 0) {
+                mbar_expect_tx(full_bar(s), stage_bytes);
+                tma_load_4d(a_dst, &map_x, full_bar(s), blk * 64, w0 + q - p.pad, h0 + r - p.pad, n0);
+                if (!B_MN) tma_load_2d(a_dst + a_bytes, &map_w, full_bar(s), tap * p.c_red + blk * 64, n_tile * p.bn);
+            }
+            if (B_MN) {
+                __syncwarp();
+                if (lane >= 1 && lane <= p.bn / 64)
+                    tma_load_2d(a_dst + a_bytes + (lane - 1) * 8192, &map_w, full_bar(s),
+                                (p.k * p.k - 1 - tap) * p.c_out + n_tile * p.bn + (lane - 1) * 64, blk * 64);
+            }
             issued = it + 1;
         }
-        if (*failed) {
+        if (*failed && lane == 0) {
             // copies that were issued but never consumed must land before the CTA may exit
             for (int it = max(0, issued - p.stages); it < issued; ++it)
                 mbar_drain(full_bar(it % p.stages), (uint32_t)(it / p.stages) & 1u);
         }
     } else if (warp == 1 && lane == 0) {
         // ---------------- MMA issuer
-        const uint32_t idesc = instr_desc(128, p.bn, 0, 0);
+        const uint32_t idesc = instr_desc(128, p.bn, 0, B_MN ? 1 : 0);
+        constexpr uint32_t b_step = B_MN ? 2048u : 32u, b_lbo = B_MN ? 8192u : 0u;
         bool ok = true;
         for (int it = 0; it < iters && ok; ++it) {
             const int s = it % p.stages;
@@ -245,8 +258,8 @@ tc_conv_fwd_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_const
             const uint32_t a_addr = base + (uint32_t)s * stage_bytes;
             const uint32_t b_addr = a_addr + a_bytes;
 #pragma unroll
-            for (int kk = 0; kk < 4; ++kk) {        // 4 x (K = 16 bf16 = 32 bytes) per 64-channel block
-                umma_bf16(tmem_base, smem_desc(a_addr + kk * 32, 0, 1024), smem_desc(b_addr + kk * 32, 0, 1024), idesc,
+            for (int kk = 0; kk < 4; ++kk) {        // 4 x (K = 16 bf16): 32 bytes along a row, or 16 rows when B_MN
+                umma_bf16(tmem_base, smem_desc(a_addr + kk * 32, 0, 1024), smem_desc(b_addr + kk * b_step, b_lbo, 1024), idesc,
                           (it > 0 || kk > 0) ? 1u : 0u);
             }
             umma_commit(empty_bar(s));              // frees the stage when these MMAs have read it
@@ -1264,18 +1277,6 @@ __global__ void transpose_flip_kernel(const __nv_bfloat16* __restrict__ w, __nv_
     }
 }
 
-// k = 1: plain [c_out][c_in] -> [c_in][c_out] transpose through a 64x64 shared tile (both sides coalesced)
-__global__ void __launch_bounds__(256) transpose_tile_kernel(const __nv_bfloat16* __restrict__ w, __nv_bfloat16* __restrict__ wt, int c_out, int c_in) {
-    __shared__ __nv_bfloat16 tile[64][66];
-    const int ci0 = blockIdx.x * 64, co0 = blockIdx.y * 64;
-    const int tx = threadIdx.x % 64, ty = threadIdx.x / 64;
-    for (int r = ty; r < 64; r += 4)
-        if (co0 + r < c_out && ci0 + tx < c_in) tile[r][tx] = w[(size_t)(co0 + r) * c_in + ci0 + tx];
-    __syncthreads();
-    for (int r = ty; r < 64; r += 4)
-        if (ci0 + r < c_in && co0 + tx < c_out) wt[(size_t)(ci0 + r) * c_out + co0 + tx] = tile[tx][r];
-}
-
 __global__ void slice_sum_tc_kernel(const float* __restrict__ partial, float* __restrict__ out, int64_t elems, int slices) {
     int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (e >= elems) return;
@@ -1346,8 +1347,8 @@ void choose_tile(int pixels, int W, int H, int N, int* tw, int* th, int* tn) {
 
 int pick_bn(int c_out) { return c_out % 256 == 0 ? 256 : (c_out % 128 == 0 ? 128 : 64); }
 
-int launch_c64(const void* x, const void* w_mat, void* out, float* stat_partial, int* stat_blocks, int N, int H, int W, int c_out,
-               int* status, cudaStream_t st, const char* what) {
+int launch_c64(const void* x, const void* w_mat, void* out, float* stat_partial, int* stat_blocks, int N, int H, int W,
+               int c_out, int* status, cudaStream_t st, const char* what) {
     C64Params p;
     p.H = H; p.W = W; p.N = N; p.c_out = c_out;
     const int nt = (H + 15) / 16;
@@ -1388,8 +1389,8 @@ bool halo_applies(int H, int W, int c_red, int c_out, int k, int pad) {
     return 8 * th >= 112 && H % th == 0;
 }
 
-int launch_halo(const void* x, const void* w_mat, void* out, float* stat_partial, int* stat_blocks, int N, int H, int W, int c_red,
-                int c_out, int* status, cudaStream_t st, const char* what) {
+int launch_halo(const void* x, const void* w_mat, void* out, float* stat_partial, int* stat_blocks, int N, int H, int W,
+                int c_red, int c_out, int* status, cudaStream_t st, const char* what) {
     HaloParams p;
     p.H = H; p.W = W; p.N = N; p.c_red = c_red; p.c_out = c_out;
     const int nt = (H + 15) / 16;
@@ -1424,16 +1425,12 @@ int launch_halo(const void* x, const void* w_mat, void* out, float* stat_partial
     return CKPT_OK;
 }
 
-// The persistent kernels can gather the per-channel sums of their output on the way out.
-bool persistent_applies(int H, int W, int c_red, int c_out, int k, int pad) {
-    return (c_red == 64 && k == 3 && pad == 1 && c_out % 64 == 0) || halo_applies(H, W, c_red, c_out, k, pad);
-}
-
 // stat_partial / stat_blocks: null, or where the kernel leaves the batch-norm partial sums of its output
 // ([block][sum | sum of squares][c_out] floats) and how many blocks it wrote (0 = this kernel does not gather them).
 int launch_fwd_like(const void* x, const void* w_mat, void* out, const float* bias, int relu, int N, int H, int W, int c_red,
                     int c_out, int k, int pad, int* status, cudaStream_t st, const char* what, float* stat_partial = nullptr,
-                    int* stat_blocks = nullptr) {
+                    int* stat_blocks = nullptr, bool b_mn = false) {
+    // b_mn (1x1 only): w_mat is the forward filter [c_red][c_out] read in place (c_out a multiple of 64)
     if (stat_blocks) *stat_blocks = 0;
     if (c_red == 64 && k == 3 && pad == 1 && c_out % 64 == 0 && !bias && !relu)
         return launch_c64(x, w_mat, out, stat_partial, stat_blocks, N, H, W, c_out, status, st, what);
@@ -1446,7 +1443,8 @@ int launch_fwd_like(const void* x, const void* w_mat, void* out, const float* bi
     p.bn = pick_bn(c_out);
     {   // few pixel tiles (fully connected layers): narrower channel tiles give every SM a share of the matrix
         const int64_t m_tiles = (int64_t)p.tiles_w * p.tiles_h * p.tiles_n;
-        while (p.bn > 64 && m_tiles * ((c_out + p.bn - 1) / p.bn) < 148) p.bn /= 2;
+        const int floor_bn = b_mn ? 64 : 32;
+        while (p.bn > floor_bn && m_tiles * ((c_out + p.bn - 1) / p.bn) < 148) p.bn /= 2;
     }
     p.n_tiles = (c_out + p.bn - 1) / p.bn;
     const uint32_t stage_bytes = 128 * 128 + p.bn * 128;
@@ -1454,17 +1452,19 @@ int launch_fwd_like(const void* x, const void* w_mat, void* out, const float* bi
     CUtensorMap mx, mw;
     int rc = make_act_map(&mx, x, N, H, W, c_red, p.tw, p.th, p.tn);
     if (rc) return rc;
-    rc = make_mat_map(&mw, w_mat, c_out, (int64_t)k * k * c_red, p.bn);
+    rc = b_mn ? make_mat_map(&mw, w_mat, c_red, (int64_t)k * k * c_out, 64) : make_mat_map(&mw, w_mat, c_out, (int64_t)k * k * c_red, p.bn);
     if (rc) return rc;
     const size_t smem = (size_t)p.stages * stage_bytes + 1024 + 256;
     static bool attr_set = false;
     if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(tc_conv_fwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget + 2048);
+        cudaError_t e = cudaFuncSetAttribute(tc_conv_fwd_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget + 2048);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_conv_fwd_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget + 2048);
         if (e != cudaSuccess) return cuda_fail(e, "raising the shared-memory limit");
         attr_set = true;
     }
     const int64_t ctas = (int64_t)p.tiles_w * p.tiles_h * p.tiles_n * p.n_tiles;
-    tc_conv_fwd_kernel<<<(unsigned)ctas, kThreads, smem, st>>>(mx, mw, (__nv_bfloat16*)out, bias, relu, p, status);
+    if (b_mn) tc_conv_fwd_kernel<true><<<(unsigned)ctas, kThreads, smem, st>>>(mx, mw, (__nv_bfloat16*)out, bias, relu, p, status);
+    else tc_conv_fwd_kernel<false><<<(unsigned)ctas, kThreads, smem, st>>>(mx, mw, (__nv_bfloat16*)out, bias, relu, p, status);
     CKPT_LAUNCH_CHECK(what);
     return CKPT_OK;
 }
@@ -1568,7 +1568,7 @@ int64_t tc_conv_scratch_bytes(const ConvGeom& g) {
     if (wgrad_c64_applies(g)) {
         W64Params q;
         wgrad_c64_plan(g, &q);
-        return (int64_t)q.slices * g.cout * 576 * 4;      // also covers the transposed matrix of the dgrad
+        return (int64_t)q.slices * g.cout * 576 * 4;
     }
     WgradParams p;
     int slices, groups, co_tiles;
@@ -1626,16 +1626,18 @@ int tc_conv_dgrad(const ConvGeom& g, const void* dz, const void* w, void* dx, vo
                   int* device_status, void* stream) {
     if (!device_status) { set_error("no status word"); return CKPT_E_NULL; }
     const int taps = g.k * g.k;
-    const int64_t elems = (int64_t)g.cout * taps * g.cin;
-    if (!scratch || scratch_bytes < elems * 2) { set_error("dgrad scratch too small"); return CKPT_E_WORKSPACE; }
     cudaStream_t st = (cudaStream_t)stream;
     if (taps == 1) {
-        dim3 tgrid((g.cin + 63) / 64, (g.cout + 63) / 64);
-        transpose_tile_kernel<<<tgrid, 256, 0, st>>>((const __nv_bfloat16*)w, (__nv_bfloat16*)scratch, g.cout, g.cin);
-    } else {
-        const unsigned grid = (unsigned)std::min<int64_t>((elems + 255) / 256, 148 * 8);
-        transpose_flip_kernel<<<grid, 256, 0, st>>>((const __nv_bfloat16*)w, (__nv_bfloat16*)scratch, g.cout, taps, g.cin);
+        // [c_out][c_in] is already the dgrad's B operand with the reduction (c_out) as rows: the tensor core reads
+        // it MN-major in place.  (For 3x3 the in-place read needs four 8 KB copies per stage instead of one
+        // and measured 10-30 % slower than a transposed copy, which costs under 10 us per layer.)
+        return launch_fwd_like(dz, w, dx, nullptr, 0, g.n, g.h, g.w, g.cout, g.cin, g.k, g.k - 1 - g.pad, device_status, st,
+                               "conv dgrad (tensor cores)", nullptr, nullptr, true);
     }
+    const int64_t elems = (int64_t)g.cout * taps * g.cin;
+    if (!scratch || scratch_bytes < elems * 2) { set_error("dgrad scratch too small"); return CKPT_E_WORKSPACE; }
+    const unsigned grid = (unsigned)std::min<int64_t>((elems + 255) / 256, 148 * 8);
+    transpose_flip_kernel<<<grid, 256, 0, st>>>((const __nv_bfloat16*)w, (__nv_bfloat16*)scratch, g.cout, taps, g.cin);
     CKPT_LAUNCH_CHECK("dgrad matrix transpose");
     return launch_fwd_like(dz, scratch, dx, nullptr, 0, g.n, g.h, g.w, g.cout, g.cin, g.k, g.k - 1 - g.pad, device_status, st,
                            "conv dgrad (tensor cores)");
