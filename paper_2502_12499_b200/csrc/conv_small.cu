@@ -3,8 +3,11 @@
 //            loads lives with the other tcgen05 kernels): one thread per output pixel, 64 output
 //            channels in registers, the filter in shared memory (read as broadcast float4), the
 //            pixel's 128-byte output row written as 8 x 16 B;
-//   wgrad  : the input is unfolded to [pixel][9*c_in padded to 64] and the gradient becomes a
-//            [c_out x 64] contraction over pixels on the tensor cores (the 1x1 wgrad kernel).
+//   wgrad  : the input is unfolded to [pixel][9*c_in padded to 32]; two horizontally adjacent pixels form
+//            one 64-"channel" row, and dz is read with the same pairing as 2*c_out channels, so the
+//            gradient becomes a [2*c_out x 64] contraction over pixel pairs on the tensor cores (the
+//            1x1 wgrad kernel, full 128-row tiles for c_out = 64) whose two diagonal blocks are added.
+//            Odd image widths fall back to one pixel per 64-wide row.
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 
@@ -77,10 +80,10 @@ __global__ void __launch_bounds__(128) small_fwd_kernel(const __nv_bfloat16* __r
     }
 }
 
-// xcol[p][0..9*CIN) = the 3x3 neighbourhood of pixel p (zero outside the image), [9*CIN..64) = 0:
-// the first layer's input unfolded to 64 "channels", so that its weight gradient is a plain
-// [c_out x 64] = dz^T * xcol contraction for the tensor cores.
-template <int CIN>
+// xcol[p][0..9*CIN) = the 3x3 neighbourhood of pixel p (zero outside the image), [9*CIN..WIDTH) = 0:
+// the first layer's input unfolded to WIDTH "channels" per pixel (64, or 32 when pixels are paired), so
+// that its weight gradient is a plain dz^T * xcol contraction for the tensor cores.
+template <int CIN, int WIDTH>
 __global__ void __launch_bounds__(256) unfold3x3_kernel(const __nv_bfloat16* __restrict__ x, __nv_bfloat16* __restrict__ xcol,
                                                         int n, int h, int wd) {
     constexpr int K = 9 * CIN;
@@ -89,9 +92,9 @@ __global__ void __launch_bounds__(256) unfold3x3_kernel(const __nv_bfloat16* __r
         const int ow = (int)(p % wd);
         const int oh = (int)((p / wd) % h);
         const int64_t img = p / ((int64_t)wd * h);
-        __align__(16) __nv_bfloat16 v[64];
+        __align__(16) __nv_bfloat16 v[WIDTH];
 #pragma unroll
-        for (int i = K; i < 64; ++i) v[i] = __float2bfloat16_rn(0.f);
+        for (int i = K; i < WIDTH; ++i) v[i] = __float2bfloat16_rn(0.f);
 #pragma unroll
         for (int r = 0; r < 3; ++r) {
 #pragma unroll
@@ -103,9 +106,9 @@ __global__ void __launch_bounds__(256) unfold3x3_kernel(const __nv_bfloat16* __r
                 for (int c = 0; c < CIN; ++c) v[(r * 3 + s) * CIN + c] = in ? src[c] : __float2bfloat16_rn(0.f);
             }
         }
-        uint4* dst = reinterpret_cast<uint4*>(xcol + p * 64);
+        uint4* dst = reinterpret_cast<uint4*>(xcol + p * WIDTH);
 #pragma unroll
-        for (int j = 0; j < 8; ++j) dst[j] = reinterpret_cast<const uint4*>(v)[j];
+        for (int j = 0; j < WIDTH / 8; ++j) dst[j] = reinterpret_cast<const uint4*>(v)[j];
     }
 }
 
@@ -114,6 +117,14 @@ __global__ void take_columns_kernel(const float* __restrict__ dwp, float* __rest
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i < cout * k) dw[i] = dwp[(i / k) * 64 + i % k];
 }
+// Paired pixels: dwp is [(parity, co)][(parity, k)]; the gradient is the sum of its two diagonal blocks.
+__global__ void take_paired_columns_kernel(const float* __restrict__ dwp, float* __restrict__ dw, int cout, int k) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < cout * k) {
+        const int co = i / k, kk = i % k;
+        dw[i] = dwp[(size_t)co * 64 + kk] + dwp[(size_t)(cout + co) * 64 + 32 + kk];
+    }
+}
 
 }  // namespace
 
@@ -121,13 +132,15 @@ bool small_conv_supported(int dtype, const ConvGeom& g) {
     return dtype == CKPT_DTYPE_BF16 && g.cin == 3 && g.k == 3 && g.stride == 1 && g.pad == 1 && g.cout % 64 == 0;
 }
 
+static bool paired(const ConvGeom& g) { return g.w % 2 == 0; }
 static ConvGeom unfolded_geom(const ConvGeom& g) {
     ConvGeom u = g;
     u.cin = 64; u.k = 1; u.pad = 0;
+    if (paired(g)) { u.w = g.w / 2; u.wo = g.wo / 2; u.cout = 2 * g.cout; }
     return u;
 }
-static int64_t xcol_bytes(const ConvGeom& g) { return align_up((int64_t)g.n * g.h * g.w * 128, 256); }
-static int64_t dwp_bytes(const ConvGeom& g) { return align_up((int64_t)g.cout * 64 * 4, 256); }
+static int64_t xcol_bytes(const ConvGeom& g) { return align_up((int64_t)g.n * g.h * g.w * (paired(g) ? 64 : 128), 256); }
+static int64_t dwp_bytes(const ConvGeom& g) { return align_up((int64_t)(paired(g) ? 2 : 1) * g.cout * 64 * 4, 256); }
 
 int64_t small_conv_scratch_bytes(const ConvGeom& g) {
     return xcol_bytes(g) + dwp_bytes(g) + tc_conv_scratch_bytes(unfolded_geom(g));
@@ -151,12 +164,15 @@ int small_conv_wgrad(const ConvGeom& g, const void* dz, const void* x, float* dw
     float* dwp = (float*)(base + xcol_bytes(g));
     void* tc_scratch = base + xcol_bytes(g) + dwp_bytes(g);
     const int64_t pixels = (int64_t)g.n * g.h * g.w;
-    unfold3x3_kernel<3><<<(unsigned)std::min<int64_t>((pixels + 255) / 256, 148 * 16), 256, 0, st>>>((const __nv_bfloat16*)x, xcol, g.n, g.h, g.w);
+    const unsigned ugrid = (unsigned)std::min<int64_t>((pixels + 255) / 256, 148 * 16);
+    if (paired(g)) unfold3x3_kernel<3, 32><<<ugrid, 256, 0, st>>>((const __nv_bfloat16*)x, xcol, g.n, g.h, g.w);
+    else unfold3x3_kernel<3, 64><<<ugrid, 256, 0, st>>>((const __nv_bfloat16*)x, xcol, g.n, g.h, g.w);
     CKPT_LAUNCH_CHECK("first-layer unfold");
     const ConvGeom u = unfolded_geom(g);
     int rc = tc_conv_wgrad(u, dz, xcol, dwp, tc_scratch, scratch_bytes - xcol_bytes(g) - dwp_bytes(g), device_status, stream);
     if (rc) return rc;
-    take_columns_kernel<<<(g.cout * 27 + 255) / 256, 256, 0, st>>>(dwp, dw, g.cout, 27);
+    if (paired(g)) take_paired_columns_kernel<<<(g.cout * 27 + 255) / 256, 256, 0, st>>>(dwp, dw, g.cout, 27);
+    else take_columns_kernel<<<(g.cout * 27 + 255) / 256, 256, 0, st>>>(dwp, dw, g.cout, 27);
     CKPT_LAUNCH_CHECK("first-layer wgrad column pick");
     return CKPT_OK;
 }
