@@ -279,6 +279,45 @@ __device__ __forceinline__ void store_vec(T* p, const float (&v)[VEC]) {
     }
 }
 
+// A vector as loaded: kept packed in registers until it is used, so that many loads can be in flight
+// per thread without the register cost of their unpacked form.
+template <typename T, int VEC> struct RawVec { T e[VEC]; };
+template <> struct RawVec<__nv_bfloat16, 8> { uint4 q; };
+template <> struct RawVec<float, 4> { float4 q; };
+template <typename T, int VEC>
+__device__ __forceinline__ RawVec<T, VEC> load_raw(const T* p) {
+    RawVec<T, VEC> r;
+    if constexpr (VEC == 1) r.e[0] = *p;
+    else if constexpr (sizeof(T) == 4) r.q = *reinterpret_cast<const float4*>(p);
+    else r.q = *reinterpret_cast<const uint4*>(p);
+    return r;
+}
+template <typename T, int VEC>
+__device__ __forceinline__ void unpack(const RawVec<T, VEC>& r, float (&v)[VEC]) {
+    if constexpr (VEC == 1) {
+        v[0] = (float)r.e[0];
+    } else if constexpr (sizeof(T) == 4) {
+        v[0] = r.q.x; v[1] = r.q.y; v[2] = r.q.z; v[3] = r.q.w;
+    } else {
+        const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&r.q);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) { float2 f = __bfloat1622float2(h[i]); v[2 * i] = f.x; v[2 * i + 1] = f.y; }
+    }
+}
+
+// Launch shape of the streaming element-wise kernels: a block works through `per_block` consecutive
+// chunks of THREADS*U vectors.  Few chunks per block on large tensors (many short-lived blocks keep
+// the memory system busier than a grid that marches in lock step), one per block on small ones.
+struct StreamGrid { unsigned blocks; int per_block; };
+static StreamGrid stream_grid(int64_t vecs, int threads, int unroll) {
+    const int64_t chunk = (int64_t)threads * unroll;
+    const int64_t chunks = std::max<int64_t>(1, (vecs + chunk - 1) / chunk);
+    StreamGrid g;
+    g.per_block = (int)std::max<int64_t>(1, std::min<int64_t>(4, chunks / (148 * 8)));
+    g.blocks = (unsigned)((chunks + g.per_block - 1) / g.per_block);
+    return g;
+}
+
 struct BnLayout {
     int lanes;          // threads across the channel dimension (c / VEC)
     int rows_per_iter;  // rows covered by one sweep of a block
@@ -433,39 +472,45 @@ __global__ void __launch_bounds__(32) bn_finalize_bwd_kernel(const float* __rest
     coef[c + ch] = (float)(inv * k2);
 }
 
-// y = max(z*scale + shift, 0).  When the grid's thread count is a multiple of the number of channel
-// groups, every thread stays on one channel group: its coefficients live in registers and four
-// independent 16-byte loads are in flight per thread.
+// y = max(z*scale + shift, 0).  A block walks consecutive chunks of 256*U vectors; when the block size
+// is a multiple of the number of channel groups every thread stays on one channel group, keeps its
+// coefficients in registers and has U packed 16-byte loads in flight.
+constexpr int BN_APPLY_U = 8;
 template <typename T, int VEC>
-__global__ void __launch_bounds__(256) bn_apply_kernel(const T* __restrict__ z, const float* __restrict__ stats, int relu,
-                                                       int64_t vecs, int lanes, int c, T* __restrict__ y) {
-    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
-    const int64_t first = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (stride % lanes == 0) {
-        const int ch = (int)(first % lanes) * VEC;
+__global__ void __launch_bounds__(256, 4) bn_apply_kernel(const T* __restrict__ z, const float* __restrict__ stats, int relu,
+                                                          int64_t vecs, int lanes, int c, int per_block, T* __restrict__ y) {
+    constexpr int U = BN_APPLY_U;
+    const int64_t chunk = 256 * U;
+    const int64_t begin = (int64_t)blockIdx.x * per_block * chunk;
+    if (256 % lanes == 0) {
+        const int ch = (int)(threadIdx.x % lanes) * VEC;
         float sc[VEC], sh[VEC];
 #pragma unroll
         for (int k = 0; k < VEC; ++k) { sc[k] = stats[2 * c + ch + k]; sh[k] = stats[3 * c + ch + k]; }
-        for (int64_t i = first; i < vecs; i += 4 * stride) {
-            float v[4][VEC];
+        for (int it = 0; it < per_block; ++it) {
+            const int64_t i0 = begin + it * chunk + threadIdx.x;
+            if (i0 >= vecs) break;
+            RawVec<T, VEC> r[U];
 #pragma unroll
-            for (int u = 0; u < 4; ++u)
-                if (i + u * stride < vecs) load_vec<T, VEC>(z + (i + u * stride) * VEC, v[u]);
+            for (int u = 0; u < U; ++u)
+                if (i0 + u * 256 < vecs) r[u] = load_raw<T, VEC>(z + (i0 + u * 256) * VEC);
 #pragma unroll
-            for (int u = 0; u < 4; ++u) {
-                if (i + u * stride >= vecs) break;
-                float o[VEC];
+            for (int u = 0; u < U; ++u) {
+                if (i0 + u * 256 >= vecs) break;
+                float v[VEC], o[VEC];
+                unpack<T, VEC>(r[u], v);
 #pragma unroll
                 for (int k = 0; k < VEC; ++k) {
-                    float t = fmaf(v[u][k], sc[k], sh[k]);
+                    float t = fmaf(v[k], sc[k], sh[k]);
                     o[k] = relu ? fmaxf(t, 0.f) : t;
                 }
-                store_vec<T, VEC>(y + (i + u * stride) * VEC, o);
+                store_vec<T, VEC>(y + (i0 + u * 256) * VEC, o);
             }
         }
         return;
     }
-    for (int64_t i = first; i < vecs; i += stride) {
+    const int64_t end = min(vecs, begin + per_block * chunk);
+    for (int64_t i = begin + threadIdx.x; i < end; i += 256) {
         const int ch = (int)(i % lanes) * VEC;
         float v[VEC], o[VEC];
         load_vec<T, VEC>(z + i * VEC, v);
@@ -491,13 +536,15 @@ __device__ __forceinline__ void bn_bwd_point(const float (&v)[VEC], const float 
     }
 }
 
+constexpr int BN_BWD_U = 4;
 template <typename T, int VEC>
 __global__ void __launch_bounds__(256, 3) bn_bwd_apply_kernel(const T* __restrict__ dy, const T* __restrict__ z,
                                                               const float* __restrict__ stats, const float* __restrict__ coef,
-                                                              int relu, int64_t vecs, int lanes, int c, T* __restrict__ dz) {
-    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
-    const int64_t first = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    const bool fixed = stride % lanes == 0;
+                                                              int relu, int64_t vecs, int lanes, int c, int per_block,
+                                                              T* __restrict__ dz) {
+    constexpr int U = BN_BWD_U;
+    const int64_t chunk = 256 * U;
+    const int64_t begin = (int64_t)blockIdx.x * per_block * chunk;
     float sc[VEC], sh[VEC], ca[VEC], cb[VEC];
     auto load_coef = [&](int ch) {
 #pragma unroll
@@ -506,24 +553,29 @@ __global__ void __launch_bounds__(256, 3) bn_bwd_apply_kernel(const T* __restric
             ca[k] = coef[ch + k]; cb[k] = coef[c + ch + k];
         }
     };
-    if (fixed) {
-        load_coef((int)(first % lanes) * VEC);
-        for (int64_t i = first; i < vecs; i += 2 * stride) {
-            float v[2][VEC], g[2][VEC];
+    if (256 % lanes == 0) {
+        load_coef((int)(threadIdx.x % lanes) * VEC);
+        for (int it = 0; it < per_block; ++it) {
+            const int64_t i0 = begin + it * chunk + threadIdx.x;
+            if (i0 >= vecs) break;
+            RawVec<T, VEC> rv[U], rg[U];
 #pragma unroll
-            for (int u = 0; u < 2; ++u)
-                if (i + u * stride < vecs) { load_vec<T, VEC>(z + (i + u * stride) * VEC, v[u]); load_vec<T, VEC>(dy + (i + u * stride) * VEC, g[u]); }
+            for (int u = 0; u < U; ++u)
+                if (i0 + u * 256 < vecs) { rv[u] = load_raw<T, VEC>(z + (i0 + u * 256) * VEC); rg[u] = load_raw<T, VEC>(dy + (i0 + u * 256) * VEC); }
 #pragma unroll
-            for (int u = 0; u < 2; ++u) {
-                if (i + u * stride >= vecs) break;
-                float o[VEC];
-                bn_bwd_point<T, VEC>(v[u], g[u], sc, sh, ca, cb, relu, o);
-                store_vec<T, VEC>(dz + (i + u * stride) * VEC, o);
+            for (int u = 0; u < U; ++u) {
+                if (i0 + u * 256 >= vecs) break;
+                float v[VEC], g[VEC], o[VEC];
+                unpack<T, VEC>(rv[u], v);
+                unpack<T, VEC>(rg[u], g);
+                bn_bwd_point<T, VEC>(v, g, sc, sh, ca, cb, relu, o);
+                store_vec<T, VEC>(dz + (i0 + u * 256) * VEC, o);
             }
         }
         return;
     }
-    for (int64_t i = first; i < vecs; i += stride) {
+    const int64_t end = min(vecs, begin + per_block * chunk);
+    for (int64_t i = begin + threadIdx.x; i < end; i += 256) {
         load_coef((int)(i % lanes) * VEC);
         float v[VEC], g[VEC], o[VEC];
         load_vec<T, VEC>(z + i * VEC, v);
@@ -544,7 +596,7 @@ __global__ void __launch_bounds__(BNF_THREADS, 2) bn_partial_stream_kernel(const
                                                                            int64_t vecs, int lanes, int c,
                                                                            float* __restrict__ partial) {
     __shared__ float red[BNF_THREADS][2 * VEC + 1];
-    constexpr int U = WHAT == 0 ? 4 : 2;
+    constexpr int U = WHAT == 0 ? 8 : 4;
     const int64_t stride = (int64_t)gridDim.x * BNF_THREADS;
     const int64_t first = (int64_t)blockIdx.x * BNF_THREADS + threadIdx.x;
     const int ch = (int)(first % lanes) * VEC;
@@ -556,28 +608,31 @@ __global__ void __launch_bounds__(BNF_THREADS, 2) bn_partial_stream_kernel(const
         for (int k = 0; k < VEC; ++k) { sc[k] = stats[2 * c + ch + k]; sh[k] = stats[3 * c + ch + k]; }
     }
     for (int64_t i = first; i < vecs; i += U * stride) {
-        float v[U][VEC], g[WHAT == 1 ? U : 1][VEC];
+        RawVec<T, VEC> rv[U], rg[WHAT == 1 ? U : 1];
 #pragma unroll
         for (int u = 0; u < U; ++u) {
             if (i + u * stride < vecs) {
-                load_vec<T, VEC>(z + (i + u * stride) * VEC, v[u]);
-                if (WHAT == 1) load_vec<T, VEC>(dy + (i + u * stride) * VEC, g[WHAT == 1 ? u : 0]);
+                rv[u] = load_raw<T, VEC>(z + (i + u * stride) * VEC);
+                if (WHAT == 1) rg[WHAT == 1 ? u : 0] = load_raw<T, VEC>(dy + (i + u * stride) * VEC);
             }
         }
 #pragma unroll
         for (int u = 0; u < U; ++u) {
             if (i + u * stride >= vecs) break;
+            float v[VEC], g[VEC];
+            unpack<T, VEC>(rv[u], v);
+            if (WHAT == 1) unpack<T, VEC>(rg[WHAT == 1 ? u : 0], g);
 #pragma unroll
             for (int k = 0; k < VEC; ++k) {
                 if (WHAT == 0) {
-                    s0[k] += v[u][k];
-                    s1[k] = fmaf(v[u][k], v[u][k], s1[k]);
+                    s0[k] += v[k];
+                    s1[k] = fmaf(v[k], v[k], s1[k]);
                 } else {
-                    float yv = fmaf(v[u][k], sc[k], sh[k]);
+                    float yv = fmaf(v[k], sc[k], sh[k]);
                     bool pass = !relu || (float)cvt<T>(fmaxf(yv, 0.f)) > 0.f;
-                    float gi = pass ? g[WHAT == 1 ? u : 0][k] : 0.f;
+                    float gi = pass ? g[k] : 0.f;
                     s0[k] += gi;
-                    s1[k] = fmaf(gi, v[u][k], s1[k]);
+                    s1[k] = fmaf(gi, v[k], s1[k]);
                 }
             }
         }
@@ -641,7 +696,8 @@ static int bn_stats_t(int64_t rows, int c, const void* z, const float* gamma, co
 template <typename T, int VEC>
 static int bn_apply_t(int64_t rows, int c, const void* z, const float* stats, int relu, void* y, cudaStream_t st) {
     int64_t vecs = rows * c / VEC;
-    bn_apply_kernel<T, VEC><<<elementwise_grid(vecs), 256, 0, st>>>((const T*)z, stats, relu, vecs, c / VEC, c, (T*)y);
+    const StreamGrid sg = stream_grid(vecs, 256, BN_APPLY_U);
+    bn_apply_kernel<T, VEC><<<sg.blocks, 256, 0, st>>>((const T*)z, stats, relu, vecs, c / VEC, c, sg.per_block, (T*)y);
     CKPT_LAUNCH_CHECK("batch-norm apply");
     return CKPT_OK;
 }
@@ -666,8 +722,9 @@ static int bn_backward_t(int64_t rows, int c, const void* dy, const void* z, con
     bn_finalize_bwd_kernel<<<c, 32, 0, st>>>(partial, blocks, c, 1.0 / (double)rows, stats, dgamma, dbeta, coef);
     CKPT_LAUNCH_CHECK("batch-norm backward finalize");
     int64_t vecs = rows * c / VEC;
-    bn_bwd_apply_kernel<T, VEC><<<elementwise_grid(vecs), 256, 0, st>>>((const T*)dy, (const T*)z, stats, coef, relu, vecs,
-                                                                         L.lanes, c, (T*)dz);
+    const StreamGrid sg = stream_grid(vecs, 256, BN_BWD_U);
+    bn_bwd_apply_kernel<T, VEC><<<sg.blocks, 256, 0, st>>>((const T*)dy, (const T*)z, stats, coef, relu, vecs, L.lanes, c,
+                                                           sg.per_block, (T*)dz);
     CKPT_LAUNCH_CHECK("batch-norm backward apply");
     return CKPT_OK;
 }
