@@ -247,7 +247,7 @@ def main():
     if rank == 0:
         peaks = measured_peaks()
         flops, _ = conv_flops(spec, mask, shapes)
-        roofline = dominant_kernel_roofline(args.config, peaks)
+        roofline = dominant_kernel_roofline(args.config, peaks, spec["batch"], shapes[1])
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
                 "warmup": max(args.warmup, 3), "ms_per_step": ms / args.steps, "higher_is_better": True,
                 "scaling": "weak", "vs_baseline": None, "dtype": spec["dtype"], "data": "synthetic", "config": config,
@@ -279,7 +279,7 @@ def _kernel_source_sha():
     return hashlib.sha256(open(path, "rb").read()).hexdigest()
 
 
-def dominant_kernel_roofline(config_index, peaks):
+def dominant_kernel_roofline(config_index, peaks, batch, first_shape):
     """The convolution-forward kernels (tcgen05) hold the largest share of the step: they run in the
     forward phase, in segment recomputation and, on the transposed matrix, as dgrad.  Timed here on
     every conv layer shape of the workload with CUDA events; achieved = sum of algorithmic FLOPs /
@@ -292,8 +292,9 @@ def dominant_kernel_roofline(config_index, peaks):
            "peak_source": peaks["source"] + " (burst: kernels timed in isolation)", "traffic": traffic,
            "launch_shapes": mix["launches"], "flops_per_launch": mix["flops"] / mix["launches"],
            "ms_per_launch": mix["ms"] / mix["launches"], "per_layer": mix["per_layer"]}
-    # the memory-bound side of the step, for the record: batch-norm passes on the largest activation
-    b, h, w, c = 64, 224, 224, 64
+    # the memory-bound side of the step, for the record: batch-norm and 2x2 pooling passes on the largest
+    # activation of the chain (the output of its first unit)
+    b, (h, w, c) = batch, first_shape
     f, g = opbench.bn("fwd", b * h * w, c), opbench.bn("bwd", b * h * w, c)
     pf, pb = opbench.pool("fwd", b, h, w, c), opbench.pool("bwd", b, h, w, c)
     out["elementwise"] = {"unit": "GB/s", "peak": peaks["hbm_gbs"],

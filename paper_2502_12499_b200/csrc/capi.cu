@@ -77,7 +77,12 @@ int ckpt_conv2d_bn_statistics(const ckpt_conv_shape* s, int dtype, const void* x
             return bn_statistics_from_partials((const float*)scratch, blocks, rows, g.cout, gamma, beta, stats, stream);
         }
     } else if (tc_first_conv_supported(dtype, g)) {
-        if ((rc = tc_first_conv_fwd(g, x, w, z, op_status_word(), stream))) return rc;
+        int blocks = 0;
+        if ((rc = tc_first_conv_fwd(g, x, w, z, op_status_word(), stream, (float*)scratch, &blocks))) return rc;
+        if (blocks > 0) {
+            if (fused) *fused = 1;
+            return bn_statistics_from_partials((const float*)scratch, blocks, rows, g.cout, gamma, beta, stats, stream);
+        }
     } else if ((rc = simt_conv_fwd(dtype, g, x, w, z, nullptr, 0, stream))) {
         return rc;
     }

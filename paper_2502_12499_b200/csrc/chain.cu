@@ -223,11 +223,13 @@ static int unit_forward(StepCtx& c, int64_t i, const void* x_raw, void* y) {
     switch (u.desc.kind) {
         case CKPT_UNIT_CONV_BN_RELU:
             if ((rc = activated(c, i - 1, x_raw, &x))) return rc;
-            if (use_tc(c.ch, u.geom)) {
+            if (use_tc(c.ch, u.geom) || (c.ch->impl == 0 && tc_first_conv_supported(dt, u.geom))) {
                 // the persistent tensor-core kernels gather the statistics of their output in the epilogue
                 int blocks = 0;
                 float* partial = (float*)(ws + c.ch->off_scr);
-                if ((rc = tc_conv_fwd_stats(u.geom, x, p[0], y, partial, &blocks, c.status(), c.stream))) return rc;
+                if (use_tc(c.ch, u.geom)) rc = tc_conv_fwd_stats(u.geom, x, p[0], y, partial, &blocks, c.status(), c.stream);
+                else rc = tc_first_conv_fwd(u.geom, x, p[0], y, c.status(), c.stream, partial, &blocks);
+                if (rc) return rc;
                 if (blocks > 0)
                     return bn_statistics_from_partials(partial, blocks, rows_of(c.ch, i), u.out.c, (const float*)p[1],
                                                        (const float*)p[2], stats_of(c, i), c.stream);

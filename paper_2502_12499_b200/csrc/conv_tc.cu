@@ -100,6 +100,17 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
 __device__ __forceinline__ void tma_prefetch_desc(const CUtensorMap* map) {
     asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
 }
+// Tile store from shared memory (async proxy): rows outside the tensor are clipped by the hardware.
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, uint32_t src, int c0, int c1) {
+    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
+                 ::"l"(map), "r"(src), "r"(c0), "r"(c1) : "memory");
+}
+__device__ __forceinline__ void tma_store_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+// Waits until at most N of this thread's store groups still read their shared-memory source.
+template <int N> __device__ __forceinline__ void tma_store_wait_read() {
+    asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory");
+}
+__device__ __forceinline__ void tma_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 
 __device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t cols) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(cols) : "memory");
@@ -1120,11 +1131,17 @@ constexpr int kFirstThreads = 288;
 #endif
 constexpr int kFirstCtasPerSm = FIRST_CTAS;      // each holds 128 of the 512 tensor-memory columns
 
+constexpr uint32_t kFirstSmem = 2 * 16384 + 8192 + 2 * 16384 + 1024;   // operand tiles, filter tile, output tiles, alignment
+
 __global__ void __launch_bounds__(kFirstThreads, kFirstCtasPerSm)
-tc_conv_first_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __restrict__ w, __nv_bfloat16* __restrict__ out,
-                     FirstParams p, int* status) {
-    __shared__ __align__(1024) uint8_t a_tiles[2][128 * 128];
-    __shared__ __align__(1024) uint8_t b_tile[64 * 128];
+tc_conv_first_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __restrict__ w,
+                     const __grid_constant__ CUtensorMap map_out, float* __restrict__ stat_partial, FirstParams p, int* status) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* const smem_al = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
+    uint8_t (*a_tiles)[128 * 128] = reinterpret_cast<uint8_t (*)[128 * 128]>(smem_al);
+    uint8_t* const b_tile = smem_al + 2 * 16384;
+    uint8_t (*o_tiles)[128 * 128] = reinterpret_cast<uint8_t (*)[128 * 128]>(smem_al + 2 * 16384 + 8192);
+    __shared__ float stat_red[4][2][64];
     __shared__ __align__(8) uint64_t bar_mem[8];
     __shared__ uint32_t tmem_base_slot;
     __shared__ int failed_flag;
@@ -1143,6 +1160,7 @@ tc_conv_first_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* _
             mbar_init(acc_full0 + 8 * b, 1); mbar_init(acc_empty0 + 8 * b, 128);
         }
         fence_barrier_init();
+        tma_prefetch_desc(&map_out);
     }
     // filter tile: row = output channel, K = (tap, channel) in the first 27 of 64 columns
     for (int i = threadIdx.x; i < 64 * 8; i += blockDim.x) {
@@ -1228,33 +1246,73 @@ tc_conv_first_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* _
             }
         }
     } else {
-        // ---------------- epilogue: thread = accumulator lane = pixel of the tile
+        // ---------------- epilogue: thread = accumulator lane = pixel of the tile.  The rounded rows go to a
+        // swizzled tile in shared memory and leave as one tile store per warp (full 128-byte lines), the
+        // batch-norm sums of the stored values are taken on the way.
         const int quarter = warp % 4;
         const int row = quarter * 32 + lane;
+        const bool stats = stat_partial != nullptr;
+        float s_acc[2] = {0.f, 0.f}, q_acc[2] = {0.f, 0.f};
         for (int j = 0; j < my_tiles; ++j) {
             const int buf = j & 1;
             if (!mbar_wait(acc_full0 + 8 * buf, (uint32_t)(j >> 1) & 1u, failed, status, 604)) break;
             tc_fence_after();
-            const long long pix = ((long long)blockIdx.x + (long long)j * gridDim.x) * 128 + row;
-            __nv_bfloat16* dst = out + pix * p.c_out + co0;
+            if (lane == 0) tma_store_wait_read<1>();          // the store that last read this output tile has left it
+            __syncwarp();
+            const long long pix0 = ((long long)blockIdx.x + (long long)j * gridDim.x) * 128;
+            const bool valid = pix0 + row < p.pixels;
+            uint8_t* const orow = o_tiles[buf] + row * 128;
 #pragma unroll
             for (int c0 = 0; c0 < 64; c0 += 32) {
                 uint32_t v[32];
                 tmem_ld32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * 64 + c0), v);
-                if (pix < p.pixels) {
+                float r[32];
 #pragma unroll
-                    for (int q = 0; q < 4; ++q) {
-                        uint4 pk;
-                        __nv_bfloat162* h = reinterpret_cast<__nv_bfloat162*>(&pk);
+                for (int q = 0; q < 4; ++q) {
+                    uint4 pk;
+                    __nv_bfloat162* h = reinterpret_cast<__nv_bfloat162*>(&pk);
 #pragma unroll
-                        for (int e = 0; e < 4; ++e)
-                            h[e] = __floats2bfloat162_rn(__uint_as_float(v[8 * q + 2 * e]), __uint_as_float(v[8 * q + 2 * e + 1]));
-                        *reinterpret_cast<uint4*>(dst + c0 + 8 * q) = pk;
+                    for (int e = 0; e < 4; ++e) {
+                        h[e] = __floats2bfloat162_rn(__uint_as_float(v[8 * q + 2 * e]), __uint_as_float(v[8 * q + 2 * e + 1]));
+                        const float2 f = __bfloat1622float2(h[e]);
+                        r[8 * q + 2 * e] = valid ? f.x : 0.f;
+                        r[8 * q + 2 * e + 1] = valid ? f.y : 0.f;
                     }
+                    *reinterpret_cast<uint4*>(orow + (((c0 / 8 + q) ^ (row & 7)) * 16)) = pk;
+                }
+                if (stats) {
+                    float sq[32];
+#pragma unroll
+                    for (int e = 0; e < 32; ++e) sq[e] = r[e] * r[e];
+                    s_acc[c0 / 32] += warp_column_sum(r, lane);
+                    q_acc[c0 / 32] += warp_column_sum(sq, lane);
                 }
             }
             tc_fence_before();
             mbar_arrive(acc_empty0 + 8 * buf);
+            fence_proxy_async();
+            __syncwarp();
+            if (lane == 0 && pix0 + quarter * 32 < p.pixels) {
+                tma_store_2d(&map_out, smem_u32(o_tiles[buf]) + (uint32_t)(quarter * 4096), co0, (int)(pix0 + quarter * 32));
+                tma_store_commit();
+            }
+        }
+        if (lane == 0) tma_store_wait_all();
+        if (stats) {
+            // the four quarters of the CTA are added in a fixed order: one partial row per CTA
+#pragma unroll
+            for (int h = 0; h < 2; ++h) { stat_red[quarter][0][h * 32 + lane] = s_acc[h]; stat_red[quarter][1][h * 32 + lane] = q_acc[h]; }
+            asm volatile("bar.sync 1, 128;" ::: "memory");
+            if (quarter == 0) {
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    const int col = h * 32 + lane;
+#pragma unroll
+                    for (int k = 0; k < 2; ++k)
+                        stat_partial[((size_t)blockIdx.x * 2 + k) * p.c_out + co0 + col] =
+                            (stat_red[0][k][col] + stat_red[1][k][col]) + (stat_red[2][k][col] + stat_red[3][k][col]);
+                }
+            }
         }
     }
     tc_fence_before();
@@ -1588,7 +1646,10 @@ bool tc_first_conv_supported(int dtype, const ConvGeom& g) {
     return dtype == CKPT_DTYPE_BF16 && g.cin == 3 && g.k == 3 && g.stride == 1 && g.pad == 1 && g.cout % 64 == 0;
 }
 
-int tc_first_conv_fwd(const ConvGeom& g, const void* x, const void* w, void* z, int* device_status, void* stream) {
+// partial / blocks: null, or where the kernel leaves the batch-norm partial sums of its output
+// ([*blocks][sum | sum of squares][c_out] floats, one row pair per CTA).
+int tc_first_conv_fwd(const ConvGeom& g, const void* x, const void* w, void* z, int* device_status, void* stream,
+                      float* partial, int* blocks) {
     if (!tc_first_conv_supported(CKPT_DTYPE_BF16, g)) { set_error("first-layer kernel: unsupported shape"); return CKPT_E_UNSUPPORTED; }
     if (!device_status) { set_error("device status word missing"); return CKPT_E_NULL; }
     FirstParams p;
@@ -1598,9 +1659,19 @@ int tc_first_conv_fwd(const ConvGeom& g, const void* x, const void* w, void* z, 
     int sms = 148, dev = 0;
     cudaGetDevice(&dev);
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    CUtensorMap map_out;
+    int rc = make_mat_map(&map_out, z, p.pixels, g.cout, 32);
+    if (rc) return rc;
+    static bool attr_set = false;
+    if (!attr_set) {
+        cudaError_t e = cudaFuncSetAttribute(tc_conv_first_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kFirstSmem);
+        if (e != cudaSuccess) return cuda_fail(e, "shared-memory opt-in of the first-layer kernel");
+        attr_set = true;
+    }
     dim3 grid((unsigned)std::min(p.m_tiles, kFirstCtasPerSm * sms), (unsigned)(g.cout / 64));
-    tc_conv_first_kernel<<<grid, kFirstThreads, 0, (cudaStream_t)stream>>>((const __nv_bfloat16*)x, (const __nv_bfloat16*)w,
-                                                                          (__nv_bfloat16*)z, p, device_status);
+    if (blocks) *blocks = partial ? (int)grid.x : 0;
+    tc_conv_first_kernel<<<grid, kFirstThreads, kFirstSmem, (cudaStream_t)stream>>>((const __nv_bfloat16*)x, (const __nv_bfloat16*)w,
+                                                                                   map_out, partial, p, device_status);
     CKPT_LAUNCH_CHECK("first-layer conv forward (tensor cores)");
     return CKPT_OK;
 }

@@ -76,7 +76,8 @@ int small_conv_wgrad(const ConvGeom& g, const void* dz, const void* x, float* dw
 
 // First layer on the tensor cores (operand tiles gathered by threads, K = 27 padded to 32).
 bool tc_first_conv_supported(int dtype, const ConvGeom& g);
-int tc_first_conv_fwd(const ConvGeom& g, const void* x, const void* w, void* z, int* device_status, void* stream);
+int tc_first_conv_fwd(const ConvGeom& g, const void* x, const void* w, void* z, int* device_status, void* stream,
+                      float* partial = nullptr, int* blocks = nullptr);
 
 // Tensor-core (tcgen05) implicit-GEMM kernels; *_supported tells whether the shape has one.
 bool tc_conv_supported(int dtype, const ConvGeom& g);

@@ -88,15 +88,27 @@ def pool(what, n, h, w, c, reps=5):
 
 
 def conv_layers(spec):
-    """(n, h, w, c_in, c_out, k, pad) of every stride-1 conv unit of a chain description."""
+    """(n, h, w, c_in, c_out, k, pad) of every stride-1 convolution of a chain description: the conv units and
+    the convolutions inside bottleneck blocks (input size of each convolution)."""
     out = []
     h, w, c = spec["input_hwc"]
+    b = spec["batch"]
     for u in spec["units"]:
-        if u["kind"] == "conv_bn_relu":
+        if u["kind"] in ("conv_bn_relu", "conv"):
             if u["stride"] == 1:
-                out.append((spec["batch"], h, w, u["cin"], u["cout"], u["k"], u["pad"]))
+                out.append((b, h, w, u["cin"], u["cout"], u["k"], u["pad"]))
             h = (h + 2 * u["pad"] - u["k"]) // u["stride"] + 1
             w = (w + 2 * u["pad"] - u["k"]) // u["stride"] + 1
+            c = u["cout"]
+        elif u["kind"] == "bottleneck":
+            st, mid = u["stride"], u["mid"]
+            out.append((b, h, w, u["cin"], mid, 1, 0))
+            if st == 1:
+                out.append((b, h, w, mid, mid, 3, 1))
+            h, w = (h + 2 - 3) // st + 1, (w + 2 - 3) // st + 1
+            out.append((b, h, w, mid, u["cout"], 1, 0))
+            if u["project"] and st == 1:
+                out.append((b, h, w, u["cin"], u["cout"], 1, 0))
             c = u["cout"]
         elif u["kind"] == "maxpool":
             h = (h + 2 * u["pad"] - u["k"]) // u["stride"] + 1

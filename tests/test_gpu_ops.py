@@ -161,7 +161,8 @@ def test_first_layer_kernels(n, h, w, cout):
     ((2, 112, 112, 128, 128, 3, 1), True),    # halo-patch kernel, 128-wide output tile
     ((4, 56, 56, 128, 256, 3, 1), True),      # halo-patch kernel, 256-wide output tile
     ((2, 14, 14, 192, 64, 3, 1), False),      # generic tensor-core kernel + separate statistics kernel
-    ((3, 21, 18, 3, 64, 3, 1), False),        # first-layer kernel + separate statistics kernel
+    ((3, 21, 18, 3, 64, 3, 1), True),         # first-layer kernel, ragged last tile
+    ((9, 96, 80, 3, 128, 3, 1), True),        # first-layer kernel, several tiles per CTA, two channel blocks
     ((2, 9, 9, 16, 24, 3, 1), False),         # CUDA-core kernel + separate statistics kernel
 ])
 def test_conv_bn_statistics(case, expect_fused):
