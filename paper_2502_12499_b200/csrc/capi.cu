@@ -43,6 +43,7 @@ int ckpt_conv2d_scratch_bytes(const ckpt_conv_shape* s, int dtype, int64_t* byte
     int64_t b = simt_wgrad_scratch_bytes(g);
     if (tc_conv_supported(dtype, g)) b = b > tc_conv_scratch_bytes(g) ? b : tc_conv_scratch_bytes(g);
     if (small_conv_supported(dtype, g)) b = b > small_conv_scratch_bytes(g) ? b : small_conv_scratch_bytes(g);
+    if (stem_conv_supported(dtype, g)) b = b > stem_conv_scratch_bytes(g) ? b : stem_conv_scratch_bytes(g);
     *bytes = b;
     return CKPT_OK;
 }
@@ -54,6 +55,7 @@ int ckpt_conv2d_forward(const ckpt_conv_shape* s, int dtype, int impl, const voi
     if (!x || !w || !z) { set_error("null tensor"); return CKPT_E_NULL; }
     ConvGeom g = make_geom(*s);
     if (impl != 1 && tc_first_conv_supported(dtype, g)) return tc_first_conv_fwd(g, x, w, z, op_status_word(), stream);
+    if (impl != 1 && stem_conv_supported(dtype, g)) return stem_conv_fwd(g, x, w, z, scratch, scratch_bytes, op_status_word(), stream);
     if (want_tc(impl, dtype, g, &rc)) return tc_conv_fwd(g, x, w, z, nullptr, 0, scratch, scratch_bytes, op_status_word(), stream);
     if (rc) return rc;
     return simt_conv_fwd(dtype, g, x, w, z, nullptr, 0, stream);
@@ -76,6 +78,8 @@ int ckpt_conv2d_bn_statistics(const ckpt_conv_shape* s, int dtype, const void* x
             if (fused) *fused = 1;
             return bn_statistics_from_partials((const float*)scratch, blocks, rows, g.cout, gamma, beta, stats, stream);
         }
+    } else if (stem_conv_supported(dtype, g) && scratch_bytes >= stem_conv_scratch_bytes(g)) {
+        if ((rc = stem_conv_fwd(g, x, w, z, scratch, scratch_bytes, op_status_word(), stream))) return rc;
     } else if (tc_first_conv_supported(dtype, g)) {
         int blocks = 0;
         if ((rc = tc_first_conv_fwd(g, x, w, z, op_status_word(), stream, (float*)scratch, &blocks))) return rc;
@@ -108,6 +112,8 @@ int ckpt_conv2d_wgrad(const ckpt_conv_shape* s, int dtype, int impl, const void*
     ConvGeom g = make_geom(*s);
     if (impl != 1 && small_conv_supported(dtype, g))
         return small_conv_wgrad(g, dz, x, dw, scratch, scratch_bytes, op_status_word(), stream);
+    if (impl != 1 && stem_conv_supported(dtype, g))
+        return stem_conv_wgrad(g, dz, x, dw, scratch, scratch_bytes, op_status_word(), stream);
     if (want_tc(impl, dtype, g, &rc)) return tc_conv_wgrad(g, dz, x, dw, scratch, scratch_bytes, op_status_word(), stream);
     if (rc) return rc;
     return simt_conv_wgrad(dtype, g, dz, x, dw, scratch, scratch_bytes, stream);

@@ -83,6 +83,8 @@ static int conv_forward_any(StepCtx& c, const ConvGeom& g, const void* x, const 
         return tc_conv_fwd(g, x, w, z, bias, relu, c.ws + c.ch->off_scr, c.ch->scr_bytes, c.status(), c.stream);
     if (c.ch->impl == 0 && !bias && !relu && tc_first_conv_supported(c.ch->dtype, g))
         return tc_first_conv_fwd(g, x, w, z, c.status(), c.stream);
+    if (c.ch->impl == 0 && !bias && !relu && stem_conv_supported(c.ch->dtype, g))
+        return stem_conv_fwd(g, x, w, z, c.ws + c.ch->off_scr, c.ch->scr_bytes, c.status(), c.stream);
     return simt_conv_fwd(c.ch->dtype, g, x, w, z, bias, relu, c.stream);
 }
 static int conv_dgrad_any(StepCtx& c, const ConvGeom& g, const void* dz, const void* w, void* dx) {
@@ -93,6 +95,8 @@ static int conv_dgrad_any(StepCtx& c, const ConvGeom& g, const void* dz, const v
 static int conv_wgrad_any(StepCtx& c, const ConvGeom& g, const void* dz, const void* x, float* dw) {
     if (c.ch->impl == 0 && small_conv_supported(c.ch->dtype, g))
         return small_conv_wgrad(g, dz, x, dw, c.ws + c.ch->off_scr, c.ch->scr_bytes, c.status(), c.stream);
+    if (c.ch->impl == 0 && stem_conv_supported(c.ch->dtype, g))
+        return stem_conv_wgrad(g, dz, x, dw, c.ws + c.ch->off_scr, c.ch->scr_bytes, c.status(), c.stream);
     if (use_tc(c.ch, g))
         return tc_conv_wgrad(g, dz, x, dw, c.ws + c.ch->off_scr, c.ch->scr_bytes, c.status(), c.stream);
     return simt_conv_wgrad(c.ch->dtype, g, dz, x, dw, c.ws + c.ch->off_scr, c.ch->scr_bytes, c.stream);
@@ -586,6 +590,7 @@ int ckpt_chain_create(const ckpt_unit_desc* units, int64_t n, int64_t batch, int
                 scr = std::max(scr, simt_wgrad_scratch_bytes(u.geom));
                 if (tc_conv_supported(dtype, u.geom)) scr = std::max(scr, tc_conv_scratch_bytes(u.geom));
                 if (small_conv_supported(dtype, u.geom)) scr = std::max(scr, small_conv_scratch_bytes(u.geom));
+                if (stem_conv_supported(dtype, u.geom)) scr = std::max(scr, stem_conv_scratch_bytes(u.geom));
                 break;
             }
             case CKPT_UNIT_CONV: {
@@ -598,6 +603,7 @@ int ckpt_chain_create(const ckpt_unit_desc* units, int64_t n, int64_t batch, int
                 scr = std::max(scr, simt_wgrad_scratch_bytes(u.geom));
                 if (tc_conv_supported(dtype, u.geom)) scr = std::max(scr, tc_conv_scratch_bytes(u.geom));
                 if (small_conv_supported(dtype, u.geom)) scr = std::max(scr, small_conv_scratch_bytes(u.geom));
+                if (stem_conv_supported(dtype, u.geom)) scr = std::max(scr, stem_conv_scratch_bytes(u.geom));
                 break;
             }
             case CKPT_UNIT_BN:

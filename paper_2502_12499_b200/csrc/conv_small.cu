@@ -1,4 +1,4 @@
-// First-layer convolution: 3x3, stride 1, padding 1, 3 input channels (an RGB image), bf16 storage.
+// First-layer convolutions on 3 input channels (an RGB image), bf16 storage.  3x3, stride 1, padding 1:
 //   forward: CUDA-core version (the tensor-core version that gathers its operand tiles with plain
 //            loads lives with the other tcgen05 kernels): one thread per output pixel, 64 output
 //            channels in registers, the filter in shared memory (read as broadcast float4), the
@@ -126,6 +126,52 @@ __global__ void take_paired_columns_kernel(const float* __restrict__ dwp, float*
     }
 }
 
+// Stem of the residual networks: KS x KS filter, stride and padding as template constants, CIN input
+// channels.  xcol[output pixel][(r, s, c) padded to WIDTH] so that forward and weight gradient become
+// plain contractions over WIDTH "channels" (a 1x1 convolution) for the tensor cores.
+template <int CIN, int KS, int STRIDE, int PAD, int WIDTH>
+__global__ void __launch_bounds__(128) unfold_stem_kernel(const __nv_bfloat16* __restrict__ x, __nv_bfloat16* __restrict__ xcol,
+                                                          int n, int h, int wd, int ho, int wo) {
+    constexpr int K = KS * KS * CIN;
+    const int64_t pixels = (int64_t)n * ho * wo;
+    const uint16_t* x16 = reinterpret_cast<const uint16_t*>(x);
+    for (int64_t p = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; p < pixels; p += (int64_t)gridDim.x * blockDim.x) {
+        const int ow = (int)(p % wo);
+        const int oh = (int)((p / wo) % ho);
+        const int64_t img = p / ((int64_t)wo * ho);
+        const int ih0 = oh * STRIDE - PAD, iw0 = ow * STRIDE - PAD;
+        const uint16_t* origin = x16 + ((img * h + ih0) * wd + iw0) * CIN;     // may point outside: only dereferenced in bounds
+        uint4* dst = reinterpret_cast<uint4*>(xcol + p * WIDTH);
+#pragma unroll
+        for (int j = 0; j < WIDTH / 8; ++j) {
+            __align__(16) uint16_t v[8];
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+                const int idx = j * 8 + e;
+                if (idx < K) {
+                    const int c = idx % CIN, tap = idx / CIN, r = tap / KS, q = tap % KS;
+                    const bool in = ih0 + r >= 0 && ih0 + r < h && iw0 + q >= 0 && iw0 + q < wd;
+                    v[e] = in ? __ldg(origin + ((int64_t)r * wd + q) * CIN + c) : (uint16_t)0;
+                } else {
+                    v[e] = 0;
+                }
+            }
+            dst[j] = *reinterpret_cast<const uint4*>(v);
+        }
+    }
+}
+
+// wp[co][0..width) = w[co][0..k) followed by zeros
+__global__ void pad_rows_kernel(const __nv_bfloat16* __restrict__ w, __nv_bfloat16* __restrict__ wp, int cout, int k, int width) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < cout * width) wp[i] = (i % width) < k ? w[(size_t)(i / width) * k + i % width] : __float2bfloat16_rn(0.f);
+}
+// dw[co][0..k) = dwp[co][0..k) out of rows of `width` floats
+__global__ void take_row_heads_kernel(const float* __restrict__ dwp, float* __restrict__ dw, int cout, int k, int width) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < cout * k) dw[i] = dwp[(size_t)(i / k) * width + i % k];
+}
+
 }  // namespace
 
 bool small_conv_supported(int dtype, const ConvGeom& g) {
@@ -174,6 +220,68 @@ int small_conv_wgrad(const ConvGeom& g, const void* dz, const void* x, float* dw
     if (paired(g)) take_paired_columns_kernel<<<(g.cout * 27 + 255) / 256, 256, 0, st>>>(dwp, dw, g.cout, 27);
     else take_columns_kernel<<<(g.cout * 27 + 255) / 256, 256, 0, st>>>(dwp, dw, g.cout, 27);
     CKPT_LAUNCH_CHECK("first-layer wgrad column pick");
+    return CKPT_OK;
+}
+
+// ------------------------------------------------------------------------------------------------
+// 7x7 stride-2 padding-3 stem on 3 input channels: unfold, then the tensor-core 1x1 kernels.
+// ------------------------------------------------------------------------------------------------
+constexpr int kStemWidth = 192;      // 7*7*3 = 147 padded to whole 64-channel blocks
+
+bool stem_conv_supported(int dtype, const ConvGeom& g) {
+    return dtype == CKPT_DTYPE_BF16 && g.cin == 3 && g.k == 7 && g.stride == 2 && g.pad == 3 && g.cout % 64 == 0;
+}
+static ConvGeom stem_unfolded_geom(const ConvGeom& g) {
+    ConvGeom u = g;
+    u.h = g.ho; u.w = g.wo; u.cin = kStemWidth; u.k = 1; u.stride = 1; u.pad = 0;
+    return u;
+}
+static int64_t stem_xcol_bytes(const ConvGeom& g) { return align_up((int64_t)g.n * g.ho * g.wo * kStemWidth * 2, 256); }
+static int64_t stem_mat_bytes(const ConvGeom& g) { return align_up((int64_t)g.cout * kStemWidth * 4, 256); }
+
+int64_t stem_conv_scratch_bytes(const ConvGeom& g) {
+    return stem_xcol_bytes(g) + stem_mat_bytes(g) + tc_conv_scratch_bytes(stem_unfolded_geom(g));
+}
+
+static int stem_unfold(const ConvGeom& g, const void* x, __nv_bfloat16* xcol, cudaStream_t st) {
+    const int64_t pixels = (int64_t)g.n * g.ho * g.wo;
+    const unsigned grid = (unsigned)std::min<int64_t>((pixels + 127) / 128, 148 * 32);
+    unfold_stem_kernel<3, 7, 2, 3, kStemWidth><<<grid, 128, 0, st>>>((const __nv_bfloat16*)x, xcol, g.n, g.h, g.w, g.ho, g.wo);
+    CKPT_LAUNCH_CHECK("stem unfold");
+    return CKPT_OK;
+}
+
+int stem_conv_fwd(const ConvGeom& g, const void* x, const void* w, void* z, void* scratch, int64_t scratch_bytes,
+                  int* device_status, void* stream) {
+    if (!scratch || scratch_bytes < stem_conv_scratch_bytes(g)) { set_error("stem conv scratch too small"); return CKPT_E_WORKSPACE; }
+    cudaStream_t st = (cudaStream_t)stream;
+    char* base = (char*)scratch;
+    __nv_bfloat16* xcol = (__nv_bfloat16*)base;
+    __nv_bfloat16* wp = (__nv_bfloat16*)(base + stem_xcol_bytes(g));
+    int rc = stem_unfold(g, x, xcol, st);
+    if (rc) return rc;
+    const int k = g.k * g.k * g.cin;
+    pad_rows_kernel<<<(g.cout * kStemWidth + 255) / 256, 256, 0, st>>>((const __nv_bfloat16*)w, wp, g.cout, k, kStemWidth);
+    CKPT_LAUNCH_CHECK("stem filter padding");
+    return tc_conv_fwd(stem_unfolded_geom(g), xcol, wp, z, nullptr, 0, nullptr, 0, device_status, stream);
+}
+
+int stem_conv_wgrad(const ConvGeom& g, const void* dz, const void* x, float* dw, void* scratch, int64_t scratch_bytes,
+                    int* device_status, void* stream) {
+    if (!scratch || scratch_bytes < stem_conv_scratch_bytes(g)) { set_error("stem conv scratch too small"); return CKPT_E_WORKSPACE; }
+    cudaStream_t st = (cudaStream_t)stream;
+    char* base = (char*)scratch;
+    __nv_bfloat16* xcol = (__nv_bfloat16*)base;
+    float* dwp = (float*)(base + stem_xcol_bytes(g));
+    void* tc_scratch = base + stem_xcol_bytes(g) + stem_mat_bytes(g);
+    int rc = stem_unfold(g, x, xcol, st);
+    if (rc) return rc;
+    rc = tc_conv_wgrad(stem_unfolded_geom(g), dz, xcol, dwp, tc_scratch, scratch_bytes - stem_xcol_bytes(g) - stem_mat_bytes(g),
+                       device_status, stream);
+    if (rc) return rc;
+    const int k = g.k * g.k * g.cin;
+    take_row_heads_kernel<<<(g.cout * k + 255) / 256, 256, 0, st>>>(dwp, dw, g.cout, k, kStemWidth);
+    CKPT_LAUNCH_CHECK("stem wgrad column pick");
     return CKPT_OK;
 }
 

@@ -176,9 +176,15 @@ __host__ __device__ inline uint32_t instr_desc(int M, int N, int a_mn_major, int
 // Forward / dgrad kernel
 // ------------------------------------------------------------------------------------------------
 struct FwdParams {
-    int H, W, N;                 // spatial size (same for input and output: stride 1) and batch
+    int H, W, N;                 // pixel grid walked by the tiles: the output of a forward convolution, or one
+                                 // parity class of the input gradient of a strided one
     int c_red, c_out;            // reduction channels (multiple of 64) and output channels
-    int k, pad;                  // filter size and padding
+    int taps;                    // terms of the sum over filter positions
+    int tap_dh[9], tap_dw[9];    // A box origin of a term = tile origin * in_stride + (tap_dw, tap_dh)
+    int tap_col[9];              // 64-channel column group of the term in the filter matrix, in units of c_red
+    int in_stride;
+    int out_H, out_W;            // the tensor written: pixel (h, w) of the grid lands at
+    int out_stride, out_oh, out_ow;   //   (h * out_stride + out_oh, w * out_stride + out_ow)
     int tw, th, tn;              // pixel tile, tw*th*tn = 128
     int tiles_w, tiles_h, tiles_n;
     int bn, n_tiles;             // output-channel tile and their count
@@ -205,7 +211,7 @@ tc_conv_fwd_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_const
     const int tile_n = mt / p.tiles_h;
     const int w0 = tile_w * p.tw, h0 = tile_h * p.th, n0 = tile_n * p.tn;
     const int blocks = (p.c_red + 63) / 64;      // a ragged last block is zero-filled by the TMA unit
-    const int iters = p.k * p.k * blocks;
+    const int iters = p.taps * blocks;
     const uint32_t tmem_cols = p.bn < 32 ? 32 : p.bn;
 
     auto full_bar = [&](int s) { return bars + 8u * s; };
@@ -236,18 +242,17 @@ tc_conv_fwd_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_const
             const uint32_t phase = (uint32_t)(it / p.stages) & 1u;
             if (!mbar_wait(empty_bar(s), phase ^ 1u, failed, status, 101)) break;
             const int tap = it / blocks, blk = it % blocks;
-            const int r = tap / p.k, q = tap % p.k;
             const uint32_t a_dst = base + (uint32_t)s * stage_bytes;
             if (lane == 0) {
                 mbar_expect_tx(full_bar(s), stage_bytes);
-                tma_load_4d(a_dst, &map_x, full_bar(s), blk * 64, w0 + q - p.pad, h0 + r - p.pad, n0);
-                if (!B_MN) tma_load_2d(a_dst + a_bytes, &map_w, full_bar(s), tap * p.c_red + blk * 64, n_tile * p.bn);
+                tma_load_4d(a_dst, &map_x, full_bar(s), blk * 64, w0 * p.in_stride + p.tap_dw[tap], h0 * p.in_stride + p.tap_dh[tap], n0);
+                if (!B_MN) tma_load_2d(a_dst + a_bytes, &map_w, full_bar(s), p.tap_col[tap] * p.c_red + blk * 64, n_tile * p.bn);
             }
             if (B_MN) {
                 __syncwarp();
                 if (lane >= 1 && lane <= p.bn / 64)
                     tma_load_2d(a_dst + a_bytes + (lane - 1) * 8192, &map_w, full_bar(s),
-                                (p.k * p.k - 1 - tap) * p.c_out + n_tile * p.bn + (lane - 1) * 64, blk * 64);
+                                p.tap_col[tap] * p.c_out + n_tile * p.bn + (lane - 1) * 64, blk * 64);
             }
             issued = it + 1;
         }
@@ -281,8 +286,9 @@ tc_conv_fwd_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_const
         const int quarter = warp % 4;               // a warp may only touch its own 32 TMEM lanes
         const int row = quarter * 32 + lane;
         const int wl = row % p.tw, hl = (row / p.tw) % p.th, nl = row / (p.tw * p.th);
-        const bool valid = (w0 + wl < p.W) && (h0 + hl < p.H) && (n0 + nl < p.N);
-        __nv_bfloat16* dst = out + ((((size_t)(n0 + nl) * p.H + (h0 + hl)) * p.W + (w0 + wl)) * p.c_out + (size_t)n_tile * p.bn);
+        const int oh = (h0 + hl) * p.out_stride + p.out_oh, ow = (w0 + wl) * p.out_stride + p.out_ow;
+        const bool valid = (w0 + wl < p.W) && (h0 + hl < p.H) && (n0 + nl < p.N) && oh < p.out_H && ow < p.out_W;
+        __nv_bfloat16* dst = out + ((((size_t)(n0 + nl) * p.out_H + oh) * p.out_W + ow) * p.c_out + (size_t)n_tile * p.bn);
         if (mbar_wait(accum_bar, 0, failed, status, 103)) {
             tc_fence_after();
             for (int c0 = 0; c0 < p.bn; c0 += 32) {
@@ -712,9 +718,9 @@ tc_conv_halo_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_cons
 // wgrad kernel: D[c_out tile of 128][up to 4 blocks of 64 (tap, c_in) columns], K = pixels
 // ------------------------------------------------------------------------------------------------
 struct WgradParams {
-    int H, W, N;
+    int H, W, N;                 // the dz pixel grid
     int c_out, c_in;
-    int k, pad;
+    int k, pad, stride;          // input pixel of a term = dz pixel * stride + filter position - pad
     int tw, th, tn;              // pixel tile, tw*th*tn = 64
     int tiles_w, tiles_h, tiles_n;
     int nb;                      // column blocks per CTA (1..4)
@@ -785,7 +791,7 @@ tc_conv_wgrad_kernel(const __grid_constant__ CUtensorMap map_dz, const __grid_co
             } else if (lane < 2 + nb_here) {
                 const int j = lane - 2;
                 const int b = blk_begin + j, tap = b / cin_blocks, cib = b % cin_blocks;
-                tma_load_4d(dst + (2 + j) * box_bytes, &map_x, full_bar(s), cib * 64, w0 + tap % p.k - p.pad, h0 + tap / p.k - p.pad, n0);
+                tma_load_4d(dst + (2 + j) * box_bytes, &map_x, full_bar(s), cib * 64, w0 * p.stride + tap % p.k - p.pad, h0 * p.stride + tap / p.k - p.pad, n0);
             }
             issued = it + 1;
         }
@@ -1361,14 +1367,17 @@ EncodeTiledFn encode_fn() {
     return fn;
 }
 
-// NHWC bf16 tensor as (C, W, H, N); box = 64 channels x tw x th x tn pixels, 128-byte swizzle.
-int make_act_map(CUtensorMap* map, const void* ptr, int N, int H, int W, int C, int tw, int th, int tn) {
+// NHWC bf16 tensor as (C, W, H, N); box = 64 channels x tw x th x tn pixels, 128-byte swizzle.  With
+// stride s the box takes every s-th pixel along W and H (the bounding box is s times larger, at most
+// 256 elements per dimension).
+int make_act_map(CUtensorMap* map, const void* ptr, int N, int H, int W, int C, int tw, int th, int tn, int stride = 1) {
     EncodeTiledFn fn = encode_fn();
     if (!fn) { set_error("cuTensorMapEncodeTiled is not available from this driver"); return CKPT_E_CUDA; }
     cuuint64_t dims[4] = {(cuuint64_t)C, (cuuint64_t)W, (cuuint64_t)H, (cuuint64_t)N};
     cuuint64_t strides[3] = {(cuuint64_t)C * 2, (cuuint64_t)W * C * 2, (cuuint64_t)H * W * C * 2};
-    cuuint32_t box[4] = {64, (cuuint32_t)tw, (cuuint32_t)th, (cuuint32_t)tn};
-    cuuint32_t es[4] = {1, 1, 1, 1};
+    if (tw * stride > 256 || th * stride > 256) { set_error("tensor map: strided box exceeds 256 elements"); return CKPT_E_UNSUPPORTED; }
+    cuuint32_t box[4] = {64, (cuuint32_t)(tw * stride), (cuuint32_t)(th * stride), (cuuint32_t)tn};
+    cuuint32_t es[4] = {1, (cuuint32_t)stride, (cuuint32_t)stride, 1};
     CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(ptr), dims, strides, box, es,
                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
@@ -1483,21 +1492,15 @@ int launch_halo(const void* x, const void* w_mat, void* out, float* stat_partial
     return CKPT_OK;
 }
 
-// stat_partial / stat_blocks: null, or where the kernel leaves the batch-norm partial sums of its output
-// ([block][sum | sum of squares][c_out] floats) and how many blocks it wrote (0 = this kernel does not gather them).
-int launch_fwd_like(const void* x, const void* w_mat, void* out, const float* bias, int relu, int N, int H, int W, int c_red,
-                    int c_out, int k, int pad, int* status, cudaStream_t st, const char* what, float* stat_partial = nullptr,
-                    int* stat_blocks = nullptr, bool b_mn = false) {
-    // b_mn (1x1 only): w_mat is the forward filter [c_red][c_out] read in place (c_out a multiple of 64)
-    if (stat_blocks) *stat_blocks = 0;
-    if (c_red == 64 && k == 3 && pad == 1 && c_out % 64 == 0 && !bias && !relu)
-        return launch_c64(x, w_mat, out, stat_partial, stat_blocks, N, H, W, c_out, status, st, what);
-    if (!bias && !relu && halo_applies(H, W, c_red, c_out, k, pad))
-        return launch_halo(x, w_mat, out, stat_partial, stat_blocks, N, H, W, c_red, c_out, status, st, what);
-    FwdParams p;
-    p.H = H; p.W = W; p.N = N; p.c_red = c_red; p.c_out = c_out; p.k = k; p.pad = pad;
-    choose_tile(128, W, H, N, &p.tw, &p.th, &p.tn);
-    p.tiles_w = (W + p.tw - 1) / p.tw; p.tiles_h = (H + p.th - 1) / p.th; p.tiles_n = (N + p.tn - 1) / p.tn;
+// The generic kernel on a prepared term table (p.taps, p.tap_*, p.in_stride, p.out_*).  The operand tensor is
+// [a_n][a_h][a_w][c_red]; the tiles walk an n x gh x gw pixel grid.  `taps_total` = 64-channel column groups of
+// the filter matrix per reduction block (k*k).
+int launch_generic(FwdParams p, const void* a, int a_n, int a_h, int a_w, const void* w_mat, int taps_total, void* out,
+                   const float* bias, int relu, int n, int gh, int gw, int c_red, int c_out, int* status, cudaStream_t st,
+                   const char* what, bool b_mn) {
+    p.H = gh; p.W = gw; p.N = n; p.c_red = c_red; p.c_out = c_out;
+    choose_tile(128, gw, gh, n, &p.tw, &p.th, &p.tn);
+    p.tiles_w = (gw + p.tw - 1) / p.tw; p.tiles_h = (gh + p.th - 1) / p.th; p.tiles_n = (n + p.tn - 1) / p.tn;
     p.bn = pick_bn(c_out);
     {   // few pixel tiles (fully connected layers): narrower channel tiles give every SM a share of the matrix
         const int64_t m_tiles = (int64_t)p.tiles_w * p.tiles_h * p.tiles_n;
@@ -1508,9 +1511,9 @@ int launch_fwd_like(const void* x, const void* w_mat, void* out, const float* bi
     const uint32_t stage_bytes = 128 * 128 + p.bn * 128;
     p.stages = std::min<int>(kMaxStages, kSmemBudget / stage_bytes);
     CUtensorMap mx, mw;
-    int rc = make_act_map(&mx, x, N, H, W, c_red, p.tw, p.th, p.tn);
+    int rc = make_act_map(&mx, a, a_n, a_h, a_w, c_red, p.tw, p.th, p.tn, p.in_stride);
     if (rc) return rc;
-    rc = b_mn ? make_mat_map(&mw, w_mat, c_red, (int64_t)k * k * c_out, 64) : make_mat_map(&mw, w_mat, c_out, (int64_t)k * k * c_red, p.bn);
+    rc = b_mn ? make_mat_map(&mw, w_mat, c_red, (int64_t)taps_total * c_out, 64) : make_mat_map(&mw, w_mat, c_out, (int64_t)taps_total * c_red, p.bn);
     if (rc) return rc;
     const size_t smem = (size_t)p.stages * stage_bytes + 1024 + 256;
     static bool attr_set = false;
@@ -1527,10 +1530,32 @@ int launch_fwd_like(const void* x, const void* w_mat, void* out, const float* bi
     return CKPT_OK;
 }
 
+// stat_partial / stat_blocks: null, or where the kernel leaves the batch-norm partial sums of its output
+// ([block][sum | sum of squares][c_out] floats) and how many blocks it wrote (0 = this kernel does not gather them).
+int launch_fwd_like(const void* x, const void* w_mat, void* out, const float* bias, int relu, int N, int H, int W, int c_red,
+                    int c_out, int k, int pad, int* status, cudaStream_t st, const char* what, float* stat_partial = nullptr,
+                    int* stat_blocks = nullptr, bool b_mn = false) {
+    // b_mn (1x1 only): w_mat is the forward filter [c_red][c_out] read in place (c_out a multiple of 64)
+    if (stat_blocks) *stat_blocks = 0;
+    if (c_red == 64 && k == 3 && pad == 1 && c_out % 64 == 0 && !bias && !relu)
+        return launch_c64(x, w_mat, out, stat_partial, stat_blocks, N, H, W, c_out, status, st, what);
+    if (!bias && !relu && halo_applies(H, W, c_red, c_out, k, pad))
+        return launch_halo(x, w_mat, out, stat_partial, stat_blocks, N, H, W, c_red, c_out, status, st, what);
+    FwdParams p;
+    p.taps = k * k;
+    for (int t = 0; t < k * k; ++t) {
+        p.tap_dh[t] = t / k - pad; p.tap_dw[t] = t % k - pad;
+        p.tap_col[t] = b_mn ? k * k - 1 - t : t;
+    }
+    p.in_stride = 1;
+    p.out_H = H; p.out_W = W; p.out_stride = 1; p.out_oh = 0; p.out_ow = 0;
+    return launch_generic(p, x, N, H, W, w_mat, k * k, out, bias, relu, N, H, W, c_red, c_out, status, st, what, b_mn);
+}
+
 void wgrad_plan(const ConvGeom& g, WgradParams* p, int* slices, int* groups, int* co_tiles) {
-    p->H = g.h; p->W = g.w; p->N = g.n; p->c_out = g.cout; p->c_in = g.cin; p->k = g.k; p->pad = g.pad;
-    choose_tile(64, g.w, g.h, g.n, &p->tw, &p->th, &p->tn);
-    p->tiles_w = (g.w + p->tw - 1) / p->tw; p->tiles_h = (g.h + p->th - 1) / p->th; p->tiles_n = (g.n + p->tn - 1) / p->tn;
+    p->H = g.ho; p->W = g.wo; p->N = g.n; p->c_out = g.cout; p->c_in = g.cin; p->k = g.k; p->pad = g.pad; p->stride = g.stride;
+    choose_tile(64, g.wo, g.ho, g.n, &p->tw, &p->th, &p->tn);
+    p->tiles_w = (g.wo + p->tw - 1) / p->tw; p->tiles_h = (g.ho + p->th - 1) / p->th; p->tiles_n = (g.n + p->tn - 1) / p->tn;
     p->total_tiles = p->tiles_w * p->tiles_h * p->tiles_n;
     p->total_blocks = g.k * g.k * g.cin / 64;
     // column blocks per CTA: 4 when that divides evenly or the remainder is small, else 3
@@ -1562,7 +1587,7 @@ void wgrad_plan(const ConvGeom& g, WgradParams* p, int* slices, int* groups, int
 }  // namespace
 
 namespace {
-bool wgrad_c64_applies(const ConvGeom& g) { return g.cin == 64 && g.k == 3 && g.pad == 1 && g.cout % 64 == 0; }
+bool wgrad_c64_applies(const ConvGeom& g) { return g.cin == 64 && g.k == 3 && g.pad == 1 && g.stride == 1 && g.cout % 64 == 0; }
 void wgrad_c64_plan(const ConvGeom& g, W64Params* p) {
     p->H = g.h; p->W = g.w; p->N = g.n; p->c_out = g.cout;
     const int nt = (g.h + 15) / 16;
@@ -1612,11 +1637,12 @@ void wgrad_rows_plan(const ConvGeom& g, WRowsParams* p, int* pairs, int* co_tile
 
 bool tc_conv_supported(int dtype, const ConvGeom& g) {
     if (dtype != CKPT_DTYPE_BF16) return false;
-    if (g.stride != 1) return false;
+    if (g.stride != 1 && g.stride != 2) return false;
     if (!((g.k == 3 && g.pad == 1) || (g.k == 1 && g.pad == 0))) return false;
-    // the reduction runs over whole 64-channel blocks per tap; only a 1x1 filter may end in a ragged
-    // block (zero-filled), and stores are 8 channels wide
+    // the reduction runs over whole 64-channel blocks per tap; only a stride-1 1x1 filter may end in a
+    // ragged block (zero-filled), and stores are 8 channels wide
     if (g.cin % 64) return false;
+    if (g.stride == 2) return g.cout % 64 == 0;
     if (g.cout % 64 && !(g.k == 1 && g.cout % 8 == 0)) return false;
     if (g.ho != g.h || g.wo != g.w) return false;
     return true;
@@ -1676,12 +1702,24 @@ int tc_first_conv_fwd(const ConvGeom& g, const void* x, const void* w, void* z, 
     return CKPT_OK;
 }
 
+// Strided forward: the operand boxes take every stride-th input pixel, the tiles walk the output grid.
+static int launch_strided_fwd(const ConvGeom& g, const void* x, const void* w, void* z, int* status, cudaStream_t st) {
+    FwdParams p;
+    p.taps = g.k * g.k;
+    for (int t = 0; t < p.taps; ++t) { p.tap_dh[t] = t / g.k - g.pad; p.tap_dw[t] = t % g.k - g.pad; p.tap_col[t] = t; }
+    p.in_stride = g.stride;
+    p.out_H = g.ho; p.out_W = g.wo; p.out_stride = 1; p.out_oh = 0; p.out_ow = 0;
+    return launch_generic(p, x, g.n, g.h, g.w, w, p.taps, z, nullptr, 0, g.n, g.ho, g.wo, g.cin, g.cout, status, st,
+                          "strided conv forward (tensor cores)", false);
+}
+
 // Forward convolution that also leaves the batch-norm partial sums of its output in `partial`
 // (*blocks of them; 0 when the kernel chosen for this shape does not gather them).
 int tc_conv_fwd_stats(const ConvGeom& g, const void* x, const void* w, void* z, float* partial, int* blocks, int* device_status,
                       void* stream) {
     if (!tc_conv_supported(CKPT_DTYPE_BF16, g)) { set_error("tensor-core conv: unsupported shape"); return CKPT_E_UNSUPPORTED; }
     if (!device_status || !blocks) { set_error("device status word missing"); return CKPT_E_NULL; }
+    if (g.stride != 1) { *blocks = 0; return launch_strided_fwd(g, x, w, z, device_status, (cudaStream_t)stream); }
     return launch_fwd_like(x, w, z, nullptr, 0, g.n, g.h, g.w, g.cin, g.cout, g.k, g.pad, device_status, (cudaStream_t)stream,
                            "conv forward (tensor cores)", partial, blocks);
 }
@@ -1689,6 +1727,10 @@ int tc_conv_fwd_stats(const ConvGeom& g, const void* x, const void* w, void* z, 
 int tc_conv_fwd(const ConvGeom& g, const void* x, const void* w, void* z, const float* bias, int relu, void*, int64_t,
                 int* device_status, void* stream) {
     if (!device_status) { set_error("no status word"); return CKPT_E_NULL; }
+    if (g.stride != 1) {
+        if (bias || relu) { set_error("strided tensor-core conv has no bias/ReLU epilogue"); return CKPT_E_UNSUPPORTED; }
+        return launch_strided_fwd(g, x, w, z, device_status, (cudaStream_t)stream);
+    }
     return launch_fwd_like(x, w, z, bias, relu, g.n, g.h, g.w, g.cin, g.cout, g.k, g.pad, device_status, (cudaStream_t)stream,
                            "conv forward (tensor cores)");
 }
@@ -1698,6 +1740,52 @@ int tc_conv_dgrad(const ConvGeom& g, const void* dz, const void* w, void* dx, vo
     if (!device_status) { set_error("no status word"); return CKPT_E_NULL; }
     const int taps = g.k * g.k;
     cudaStream_t st = (cudaStream_t)stream;
+    if (g.stride != 1) {
+        // Input pixels fall into stride x stride parity classes; class (ph, pw) = pixels (stride*a + ph, stride*b + pw)
+        // receives the filter positions r with (ph + pad - r) divisible by the stride, from output row
+        // a + (ph + pad - r)/stride (likewise along the width): one stride-1 sum over dz per class.
+        const int sd = g.stride;
+        const void* w_mat = w;
+        if (taps > 1) {
+            const int64_t elems = (int64_t)g.cout * taps * g.cin;
+            if (!scratch || scratch_bytes < elems * 2) { set_error("dgrad scratch too small"); return CKPT_E_WORKSPACE; }
+            const unsigned grid = (unsigned)std::min<int64_t>((elems + 255) / 256, 148 * 8);
+            transpose_flip_kernel<<<grid, 256, 0, st>>>((const __nv_bfloat16*)w, (__nv_bfloat16*)scratch, g.cout, taps, g.cin);
+            CKPT_LAUNCH_CHECK("dgrad matrix transpose");
+            w_mat = scratch;
+        }
+        // a filter narrower than the stride leaves whole classes without a term: their gradient is zero
+        if (g.k < sd) {
+            cudaError_t e = cudaMemsetAsync(dx, 0, (size_t)g.n * g.h * g.w * g.cin * 2, st);
+            if (e != cudaSuccess) return cuda_fail(e, "clearing the input gradient");
+        }
+        for (int ph = 0; ph < sd; ++ph) {
+            for (int pw = 0; pw < sd; ++pw) {
+                FwdParams p;
+                p.taps = 0;
+                for (int r = 0; r < g.k; ++r) {
+                    if ((ph + g.pad - r) % sd != 0) continue;
+                    for (int q = 0; q < g.k; ++q) {
+                        if ((pw + g.pad - q) % sd != 0) continue;
+                        p.tap_dh[p.taps] = (ph + g.pad - r) / sd;
+                        p.tap_dw[p.taps] = (pw + g.pad - q) / sd;
+                        // transposed copy: position (r, q) sits at taps-1-(r*k+q); a 1x1 filter is read in place
+                        p.tap_col[p.taps] = taps > 1 ? taps - 1 - (r * g.k + q) : 0;
+                        ++p.taps;
+                    }
+                }
+                const int gh = (g.h - ph + sd - 1) / sd, gw = (g.w - pw + sd - 1) / sd;
+                if (gh <= 0 || gw <= 0) continue;
+                if (p.taps == 0) continue;          // cleared above
+                p.in_stride = 1;
+                p.out_H = g.h; p.out_W = g.w; p.out_stride = sd; p.out_oh = ph; p.out_ow = pw;
+                int rc = launch_generic(p, dz, g.n, g.ho, g.wo, w_mat, taps, dx, nullptr, 0, g.n, gh, gw, g.cout, g.cin,
+                                        device_status, st, "strided conv dgrad (tensor cores)", taps == 1);
+                if (rc) return rc;
+            }
+        }
+        return CKPT_OK;
+    }
     if (taps == 1) {
         // [c_out][c_in] is already the dgrad's B operand with the reduction (c_out) as rows: the tensor core reads
         // it MN-major in place.  (For 3x3 the in-place read needs four 8 KB copies per stage instead of one
@@ -1774,9 +1862,9 @@ int tc_conv_wgrad(const ConvGeom& g, const void* dz, const void* x, float* dw, v
     const int64_t elems = (int64_t)g.cout * g.k * g.k * g.cin;
     if (slices > 1 && (!scratch || scratch_bytes < (int64_t)slices * elems * 4)) { set_error("wgrad scratch too small"); return CKPT_E_WORKSPACE; }
     CUtensorMap mdz, mx;
-    int rc = make_act_map(&mdz, dz, g.n, g.h, g.w, g.cout, p.tw, p.th, p.tn);
+    int rc = make_act_map(&mdz, dz, g.n, g.ho, g.wo, g.cout, p.tw, p.th, p.tn);
     if (rc) return rc;
-    rc = make_act_map(&mx, x, g.n, g.h, g.w, g.cin, p.tw, p.th, p.tn);
+    rc = make_act_map(&mx, x, g.n, g.h, g.w, g.cin, p.tw, p.th, p.tn, g.stride);
     if (rc) return rc;
     cudaStream_t st = (cudaStream_t)stream;
     static bool attr_set = false;

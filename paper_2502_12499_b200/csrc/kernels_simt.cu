@@ -955,6 +955,84 @@ bool maxpool_fuses_activation(int dtype, int h, int w, int c, int k, int stride,
     return k == 2 && stride == 2 && pad == 0 && h % 2 == 0 && w % 2 == 0 && c % vec == 0;
 }
 
+// Vector forms of the two general pooling kernels: one thread handles VEC consecutive channels of a
+// pixel with 16-byte accesses; same window order and tie rule as the scalar kernels.
+template <typename T, int VEC>
+__global__ void __launch_bounds__(256) maxpool_fwd_vec_kernel(const T* __restrict__ x, T* __restrict__ y, int64_t items, int h, int w,
+                                                              int c, int ho, int wo, int k, int stride, int pad) {
+    const int lanes = c / VEC;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < items; i += (int64_t)gridDim.x * blockDim.x) {
+        const int ch = (int)(i % lanes) * VEC;
+        int64_t t = i / lanes;
+        const int ow = (int)(t % wo); t /= wo;
+        const int oh = (int)(t % ho);
+        const int64_t img = t / ho;
+        float best[VEC];
+#pragma unroll
+        for (int e = 0; e < VEC; ++e) best[e] = -INFINITY;
+        for (int r = 0; r < k; ++r) {
+            const int ih = oh * stride - pad + r;
+            if (ih < 0 || ih >= h) continue;
+            for (int q = 0; q < k; ++q) {
+                const int iw = ow * stride - pad + q;
+                if (iw < 0 || iw >= w) continue;
+                float v[VEC];
+                load_vec<T, VEC>(x + ((img * h + ih) * w + iw) * c + ch, v);
+#pragma unroll
+                for (int e = 0; e < VEC; ++e) best[e] = fmaxf(best[e], v[e]);
+            }
+        }
+        store_vec<T, VEC>(y + i * VEC, best);
+    }
+}
+
+template <typename T, int VEC>
+__global__ void __launch_bounds__(256) maxpool_bwd_vec_kernel(const T* __restrict__ x, const T* __restrict__ dy, T* __restrict__ dx,
+                                                              int64_t items, int h, int w, int c, int ho, int wo, int k, int stride,
+                                                              int pad) {
+    const int lanes = c / VEC;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < items; i += (int64_t)gridDim.x * blockDim.x) {
+        const int ch = (int)(i % lanes) * VEC;
+        int64_t t = i / lanes;
+        const int iw = (int)(t % w); t /= w;
+        const int ih = (int)(t % h);
+        const int64_t img = t / h;
+        float mine[VEC], acc[VEC];
+        load_vec<T, VEC>(x + i * VEC, mine);
+#pragma unroll
+        for (int e = 0; e < VEC; ++e) acc[e] = 0.f;
+        const int oh_lo = max(0, (ih + pad - k + stride) / stride), oh_hi = min(ho - 1, (ih + pad) / stride);
+        const int ow_lo = max(0, (iw + pad - k + stride) / stride), ow_hi = min(wo - 1, (iw + pad) / stride);
+        for (int oh = oh_lo; oh <= oh_hi; ++oh) {
+            for (int ow = ow_lo; ow <= ow_hi; ++ow) {
+                // in which channels am I the first maximum of window (oh, ow)?
+                bool first[VEC];
+#pragma unroll
+                for (int e = 0; e < VEC; ++e) first[e] = true;
+                for (int r = 0; r < k; ++r) {
+                    const int yy = oh * stride - pad + r;
+                    if (yy < 0 || yy >= h) continue;
+                    for (int q = 0; q < k; ++q) {
+                        const int xx = ow * stride - pad + q;
+                        if (xx < 0 || xx >= w || (yy == ih && xx == iw)) continue;
+                        float v[VEC];
+                        load_vec<T, VEC>(x + ((img * h + yy) * w + xx) * c + ch, v);
+                        const bool before = (yy < ih) || (yy == ih && xx < iw);
+#pragma unroll
+                        for (int e = 0; e < VEC; ++e)
+                            if (v[e] > mine[e] || (before && v[e] == mine[e])) first[e] = false;
+                    }
+                }
+                float g[VEC];
+                load_vec<T, VEC>(dy + ((img * ho + oh) * wo + ow) * c + ch, g);
+#pragma unroll
+                for (int e = 0; e < VEC; ++e) acc[e] += first[e] ? g[e] : 0.f;
+            }
+        }
+        store_vec<T, VEC>(dx + i * VEC, acc);
+    }
+}
+
 int maxpool_forward(int dtype, int n, int h, int w, int c, int k, int stride, int pad, const void* x, void* y, const float* act, void* stream) {
     int ho = (h + 2 * pad - k) / stride + 1, wo = (w + 2 * pad - k) / stride + 1;
     if (maxpool_fuses_activation(dtype, h, w, c, k, stride, pad)) {
@@ -968,6 +1046,15 @@ int maxpool_forward(int dtype, int n, int h, int w, int c, int k, int stride, in
         return CKPT_OK;
     }
     if (act) { set_error("the general pooling kernel takes an activated input"); return CKPT_E_BAD_ARG; }
+    if (c % bn_vec(dtype, c) == 0 && bn_vec(dtype, c) > 1) {
+        const int64_t items = (int64_t)n * ho * wo * (c / bn_vec(dtype, c));
+        if (dtype == CKPT_DTYPE_BF16)
+            maxpool_fwd_vec_kernel<__nv_bfloat16, 8><<<elementwise_grid(items), 256, 0, (cudaStream_t)stream>>>((const __nv_bfloat16*)x, (__nv_bfloat16*)y, items, h, w, c, ho, wo, k, stride, pad);
+        else
+            maxpool_fwd_vec_kernel<float, 4><<<elementwise_grid(items), 256, 0, (cudaStream_t)stream>>>((const float*)x, (float*)y, items, h, w, c, ho, wo, k, stride, pad);
+        CKPT_LAUNCH_CHECK("max-pool forward");
+        return CKPT_OK;
+    }
     unsigned grid = elementwise_grid((int64_t)n * ho * wo * c);
     if (dtype == CKPT_DTYPE_BF16)
         maxpool_fwd_kernel<__nv_bfloat16><<<grid, 256, 0, (cudaStream_t)stream>>>((const __nv_bfloat16*)x, (__nv_bfloat16*)y, n, h, w, c, ho, wo, k, stride, pad);
@@ -990,6 +1077,15 @@ int maxpool_backward(int dtype, int n, int h, int w, int c, int k, int stride, i
         return CKPT_OK;
     }
     if (act) { set_error("the general pooling kernel takes an activated input"); return CKPT_E_BAD_ARG; }
+    if (c % bn_vec(dtype, c) == 0 && bn_vec(dtype, c) > 1) {
+        const int64_t items = (int64_t)n * h * w * (c / bn_vec(dtype, c));
+        if (dtype == CKPT_DTYPE_BF16)
+            maxpool_bwd_vec_kernel<__nv_bfloat16, 8><<<elementwise_grid(items), 256, 0, (cudaStream_t)stream>>>((const __nv_bfloat16*)x, (const __nv_bfloat16*)dy, (__nv_bfloat16*)dx, items, h, w, c, ho, wo, k, stride, pad);
+        else
+            maxpool_bwd_vec_kernel<float, 4><<<elementwise_grid(items), 256, 0, (cudaStream_t)stream>>>((const float*)x, (const float*)dy, (float*)dx, items, h, w, c, ho, wo, k, stride, pad);
+        CKPT_LAUNCH_CHECK("max-pool backward");
+        return CKPT_OK;
+    }
     unsigned grid = elementwise_grid((int64_t)n * h * w * c);
     if (dtype == CKPT_DTYPE_BF16)
         maxpool_bwd_kernel<__nv_bfloat16><<<grid, 256, 0, (cudaStream_t)stream>>>((const __nv_bfloat16*)x, (const __nv_bfloat16*)dy, (__nv_bfloat16*)dx, n, h, w, c, ho, wo, k, stride, pad);

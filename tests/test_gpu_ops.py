@@ -48,6 +48,11 @@ TC_CASES = [
     (2, 28, 24, 128, 256, 3, 1),     # halo-patch kernel, 14-row tiles, 256-wide output tile
     (2, 32, 16, 192, 64, 3, 1),      # halo-patch kernel, three channel blocks, 64-wide output tile
     (2, 112, 112, 128, 128, 3, 1),   # halo-patch kernel, several tiles per persistent CTA
+    # stride 2 (8th field): strided operand boxes forward and in wgrad, one stride-1 sum per parity class in dgrad
+    (2, 28, 28, 128, 128, 3, 1, 2),  # first 3x3 of a residual stage
+    (3, 15, 13, 64, 192, 3, 1, 2),   # odd sizes: ragged parity classes
+    (2, 56, 56, 256, 128, 1, 0, 2),  # projection shortcut: three of four input classes get a zero gradient
+    (3, 9, 11, 64, 64, 1, 0, 2),
 ]
 
 
@@ -90,14 +95,15 @@ def test_conv_tensor_core_kernels(case):
     """tcgen05 forward / dgrad / wgrad against the float64 oracle, and bit-reproducible."""
     import torch
     dtype = ck.DTYPE_BF16
-    n, h, w, cin, cout, k, pad = case
+    n, h, w, cin, cout, k, pad = case[:7]
+    stride = case[7] if len(case) > 7 else 1
     rng = np.random.default_rng(hash(case) % 2 ** 31)
     x = rounded(rng.standard_normal((n, h, w, cin)), dtype)
     wt = rounded(rng.standard_normal((cout, k, k, cin)) / np.sqrt(k * k * cin), dtype)
-    z_ref = no.conv2d_fwd(x.astype(np.float64), wt.astype(np.float64), 1, pad)
+    z_ref = no.conv2d_fwd(x.astype(np.float64), wt.astype(np.float64), stride, pad)
     dz = rounded(rng.standard_normal(z_ref.shape), dtype)
-    dx_ref, dw_ref = no.conv2d_bwd(x.astype(np.float64), wt.astype(np.float64), dz.astype(np.float64), 1, pad)
-    shape = ck.ConvShape(n, h, w, cin, cout, k, 1, pad)
+    dx_ref, dw_ref = no.conv2d_bwd(x.astype(np.float64), wt.astype(np.float64), dz.astype(np.float64), stride, pad)
+    shape = ck.ConvShape(n, h, w, cin, cout, k, stride, pad)
     xd, wd, dzd = to_dev(x, dtype), to_dev(wt, dtype), to_dev(dz, dtype)
     scratch = torch.empty(max(ck.conv2d_scratch_bytes(shape, dtype), 256), dtype=torch.uint8, device="cuda")
     results = []
@@ -153,6 +159,41 @@ def test_first_layer_kernels(n, h, w, cout):
     torch.cuda.synchronize()
     assert max_rel_err(to_host(z1), z_ref) <= TIGHT[dtype]
     assert not torch.isnan(z.float()).any()
+
+
+@pytest.mark.parametrize("n,h,w,cout", [(2, 23, 19, 64), (3, 64, 64, 64), (1, 224, 224, 64), (2, 30, 37, 128)])
+def test_stem_kernels(n, h, w, cout):
+    """7x7 stride-2 padding-3 convolution on 3 input channels, bf16, automatic kernel choice: unfolded input and
+    the tensor-core 1x1 kernels for forward and wgrad, against the oracle and the CUDA-core kernels."""
+    import torch
+    dtype = ck.DTYPE_BF16
+    rng = np.random.default_rng(n * h + w + cout)
+    x = rounded(rng.standard_normal((n, h, w, 3)), dtype)
+    wt = rounded(rng.standard_normal((cout, 7, 7, 3)) / np.sqrt(147), dtype)
+    z_ref = no.conv2d_fwd(x.astype(np.float64), wt.astype(np.float64), 2, 3)
+    dz = rounded(rng.standard_normal(z_ref.shape), dtype)
+    _, dw_ref = no.conv2d_bwd(x.astype(np.float64), wt.astype(np.float64), dz.astype(np.float64), 2, 3)
+    shape = ck.ConvShape(n, h, w, 3, cout, 7, 2, 3)
+    xd, wd, dzd = to_dev(x, dtype), to_dev(wt, dtype), to_dev(dz, dtype)
+    scratch = torch.empty(max(ck.conv2d_scratch_bytes(shape, dtype), 256), dtype=torch.uint8, device="cuda")
+    outs = []
+    for rep in range(2):
+        z = torch.full(z_ref.shape, float("nan"), device="cuda").to(xd.dtype)
+        dw = torch.full(wt.shape, float("nan"), device="cuda", dtype=torch.float32)
+        scratch.fill_(0xFF)
+        ck.conv2d_forward(shape, dtype, 0, xd, wd, z, scratch)
+        scratch.fill_(0xFF)
+        ck.conv2d_wgrad(shape, dtype, 0, dzd, xd, dw, scratch)
+        torch.cuda.synchronize()
+        outs.append((z, dw))
+    z, dw = outs[0]
+    assert max_rel_err(to_host(z), z_ref) <= TIGHT[dtype]
+    assert max_rel_err(to_host(dw), dw_ref) <= 2e-5
+    assert torch.equal(outs[0][0], outs[1][0]) and torch.equal(outs[0][1], outs[1][1])
+    z1 = torch.empty_like(z)
+    ck.conv2d_forward(shape, dtype, 1, xd, wd, z1, scratch)
+    torch.cuda.synchronize()
+    assert max_rel_err(to_host(z1), z_ref) <= TIGHT[dtype]
 
 
 @pytest.mark.parametrize("case,expect_fused", [
@@ -254,7 +295,8 @@ def test_batchnorm_relu(rows, c, relu, dtype):
 
 
 @pytest.mark.parametrize("dtype", [ck.DTYPE_F32, ck.DTYPE_BF16])
-@pytest.mark.parametrize("n,h,w,c,k,stride,pad", [(2, 8, 6, 5, 2, 2, 0), (3, 13, 11, 8, 3, 2, 1), (2, 32, 32, 16, 2, 2, 0)])
+@pytest.mark.parametrize("n,h,w,c,k,stride,pad", [(2, 8, 6, 5, 2, 2, 0), (3, 13, 11, 8, 3, 2, 1), (2, 32, 32, 16, 2, 2, 0),
+                                                 (2, 20, 18, 64, 3, 2, 1), (2, 9, 9, 6, 3, 2, 1)])
 def test_maxpool(n, h, w, c, k, stride, pad, dtype):
     import torch
     rng = np.random.default_rng(h * w)
