@@ -130,34 +130,29 @@ __global__ void take_paired_columns_kernel(const float* __restrict__ dwp, float*
 // channels.  xcol[output pixel][(r, s, c) padded to WIDTH] so that forward and weight gradient become
 // plain contractions over WIDTH "channels" (a 1x1 convolution) for the tensor cores.
 template <int CIN, int KS, int STRIDE, int PAD, int WIDTH>
-__global__ void __launch_bounds__(128) unfold_stem_kernel(const __nv_bfloat16* __restrict__ x, __nv_bfloat16* __restrict__ xcol,
+__global__ void __launch_bounds__(256) unfold_stem_kernel(const __nv_bfloat16* __restrict__ x, __nv_bfloat16* __restrict__ xcol,
                                                           int n, int h, int wd, int ho, int wo) {
-    constexpr int K = KS * KS * CIN;
-    const int64_t pixels = (int64_t)n * ho * wo;
+    // one thread per 16-byte piece of a row: consecutive threads write consecutive pieces (full lines)
+    constexpr int K = KS * KS * CIN, PIECES = WIDTH / 8;
+    const int64_t items = (int64_t)n * ho * wo * PIECES;
     const uint16_t* x16 = reinterpret_cast<const uint16_t*>(x);
-    for (int64_t p = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; p < pixels; p += (int64_t)gridDim.x * blockDim.x) {
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < items; i += (int64_t)gridDim.x * blockDim.x) {
+        const int j = (int)(i % PIECES);
+        const int64_t p = i / PIECES;
         const int ow = (int)(p % wo);
         const int oh = (int)((p / wo) % ho);
         const int64_t img = p / ((int64_t)wo * ho);
         const int ih0 = oh * STRIDE - PAD, iw0 = ow * STRIDE - PAD;
         const uint16_t* origin = x16 + ((img * h + ih0) * wd + iw0) * CIN;     // may point outside: only dereferenced in bounds
-        uint4* dst = reinterpret_cast<uint4*>(xcol + p * WIDTH);
+        __align__(16) uint16_t v[8];
 #pragma unroll
-        for (int j = 0; j < WIDTH / 8; ++j) {
-            __align__(16) uint16_t v[8];
-#pragma unroll
-            for (int e = 0; e < 8; ++e) {
-                const int idx = j * 8 + e;
-                if (idx < K) {
-                    const int c = idx % CIN, tap = idx / CIN, r = tap / KS, q = tap % KS;
-                    const bool in = ih0 + r >= 0 && ih0 + r < h && iw0 + q >= 0 && iw0 + q < wd;
-                    v[e] = in ? __ldg(origin + ((int64_t)r * wd + q) * CIN + c) : (uint16_t)0;
-                } else {
-                    v[e] = 0;
-                }
-            }
-            dst[j] = *reinterpret_cast<const uint4*>(v);
+        for (int e = 0; e < 8; ++e) {
+            const int idx = j * 8 + e;
+            const int c = idx % CIN, tap = idx / CIN, r = tap / KS, q = tap % KS;
+            const bool in = idx < K && ih0 + r >= 0 && ih0 + r < h && iw0 + q >= 0 && iw0 + q < wd;
+            v[e] = in ? __ldg(origin + ((int64_t)r * wd + q) * CIN + c) : (uint16_t)0;
         }
+        reinterpret_cast<uint4*>(xcol)[i] = *reinterpret_cast<const uint4*>(v);
     }
 }
 
@@ -244,9 +239,9 @@ int64_t stem_conv_scratch_bytes(const ConvGeom& g) {
 }
 
 static int stem_unfold(const ConvGeom& g, const void* x, __nv_bfloat16* xcol, cudaStream_t st) {
-    const int64_t pixels = (int64_t)g.n * g.ho * g.wo;
-    const unsigned grid = (unsigned)std::min<int64_t>((pixels + 127) / 128, 148 * 32);
-    unfold_stem_kernel<3, 7, 2, 3, kStemWidth><<<grid, 128, 0, st>>>((const __nv_bfloat16*)x, xcol, g.n, g.h, g.w, g.ho, g.wo);
+    const int64_t items = (int64_t)g.n * g.ho * g.wo * (kStemWidth / 8);
+    const unsigned grid = (unsigned)std::min<int64_t>((items + 255) / 256, 148 * 64);
+    unfold_stem_kernel<3, 7, 2, 3, kStemWidth><<<grid, 256, 0, st>>>((const __nv_bfloat16*)x, xcol, g.n, g.h, g.w, g.ho, g.wo);
     CKPT_LAUNCH_CHECK("stem unfold");
     return CKPT_OK;
 }

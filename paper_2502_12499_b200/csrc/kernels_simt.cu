@@ -8,6 +8,7 @@
 #include <cuda_runtime.h>
 
 #include <algorithm>
+#include <cstdint>
 #include <cstdio>
 
 #include "internal.h"
@@ -779,15 +780,69 @@ __global__ void __launch_bounds__(256) bn_add_relu_kernel(const T* __restrict__ 
         y[i] = cvt<T>(fmaxf(v + s, 0.f));
     }
 }
+// Vector form: a block walks consecutive chunks of 256*U vectors, every thread stays on one channel group
+// (the block size is a multiple of the number of groups) and keeps its coefficients in registers.
+constexpr int BN_JOIN_U = 4;
+template <typename T, int VEC>
+__global__ void __launch_bounds__(256, 3) bn_add_relu_vec_kernel(const T* __restrict__ z, const float* __restrict__ stats,
+                                                                 const T* __restrict__ sc, const float* __restrict__ stats_sc,
+                                                                 int64_t vecs, int lanes, int c, int per_block, T* __restrict__ y) {
+    constexpr int U = BN_JOIN_U;
+    const int64_t chunk = 256 * U;
+    const int64_t begin = (int64_t)blockIdx.x * per_block * chunk;
+    const int ch = (int)(threadIdx.x % lanes) * VEC;
+    float a[VEC], b[VEC], as[VEC], bs[VEC];
+#pragma unroll
+    for (int k = 0; k < VEC; ++k) {
+        a[k] = stats[2 * c + ch + k]; b[k] = stats[3 * c + ch + k];
+        as[k] = stats_sc ? stats_sc[2 * c + ch + k] : 1.f;
+        bs[k] = stats_sc ? stats_sc[3 * c + ch + k] : 0.f;
+    }
+    for (int it = 0; it < per_block; ++it) {
+        const int64_t i0 = begin + it * chunk + threadIdx.x;
+        if (i0 >= vecs) break;
+        RawVec<T, VEC> rz[U], rs[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u)
+            if (i0 + u * 256 < vecs) { rz[u] = load_raw<T, VEC>(z + (i0 + u * 256) * VEC); rs[u] = load_raw<T, VEC>(sc + (i0 + u * 256) * VEC); }
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            if (i0 + u * 256 >= vecs) break;
+            float v[VEC], sv[VEC], o[VEC];
+            unpack<T, VEC>(rz[u], v);
+            unpack<T, VEC>(rs[u], sv);
+#pragma unroll
+            for (int k = 0; k < VEC; ++k) {
+                const float t = fmaf(v[k], a[k], b[k]);
+                const float s2 = stats_sc ? fmaf(sv[k], as[k], bs[k]) : sv[k];
+                o[k] = fmaxf(t + s2, 0.f);
+            }
+            store_vec<T, VEC>(y + (i0 + u * 256) * VEC, o);
+        }
+    }
+}
+template <typename T, int VEC>
+static bool bn_add_relu_vec(int64_t rows, int c, const void* z, const float* stats, const void* shortcut,
+                            const float* stats_shortcut, void* y, cudaStream_t st) {
+    if (c % VEC || 256 % (c / VEC)) return false;
+    const int64_t vecs = rows * c / VEC;
+    const StreamGrid sg = stream_grid(vecs, 256, BN_JOIN_U);
+    bn_add_relu_vec_kernel<T, VEC><<<sg.blocks, 256, 0, st>>>((const T*)z, stats, (const T*)shortcut, stats_shortcut, vecs, c / VEC, c,
+                                                              sg.per_block, (T*)y);
+    return true;
+}
 int bn_add_relu(int dtype, int64_t rows, int c, const void* z, const float* stats, const void* shortcut,
                 const float* stats_shortcut, void* y, void* stream) {
     const int64_t elems = rows * c;
-    if (dtype == CKPT_DTYPE_BF16)
-        bn_add_relu_kernel<__nv_bfloat16><<<elementwise_grid(elems), 256, 0, (cudaStream_t)stream>>>(
-            (const __nv_bfloat16*)z, stats, (const __nv_bfloat16*)shortcut, stats_shortcut, elems, c, (__nv_bfloat16*)y);
-    else
-        bn_add_relu_kernel<float><<<elementwise_grid(elems), 256, 0, (cudaStream_t)stream>>>(
+    cudaStream_t st = (cudaStream_t)stream;
+    if (dtype == CKPT_DTYPE_BF16) {
+        if (!bn_add_relu_vec<__nv_bfloat16, 8>(rows, c, z, stats, shortcut, stats_shortcut, y, st))
+            bn_add_relu_kernel<__nv_bfloat16><<<elementwise_grid(elems), 256, 0, st>>>(
+                (const __nv_bfloat16*)z, stats, (const __nv_bfloat16*)shortcut, stats_shortcut, elems, c, (__nv_bfloat16*)y);
+    } else if (!bn_add_relu_vec<float, 4>(rows, c, z, stats, shortcut, stats_shortcut, y, st)) {
+        bn_add_relu_kernel<float><<<elementwise_grid(elems), 256, 0, st>>>(
             (const float*)z, stats, (const float*)shortcut, stats_shortcut, elems, c, (float*)y);
+    }
     CKPT_LAUNCH_CHECK("residual join");
     return CKPT_OK;
 }
@@ -797,11 +852,41 @@ __global__ void __launch_bounds__(256) add_kernel(const T* __restrict__ a, const
     for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < elems; i += (int64_t)gridDim.x * blockDim.x)
         out[i] = cvt<T>(ld(a + i) + ld(b + i));
 }
+// 16-byte form of the sum (out may alias an input); four packed loads per operand in flight.
+template <typename T, int VEC>
+__global__ void __launch_bounds__(256) add_vec_kernel(const T* a, const T* b, T* out, int64_t vecs) {
+    constexpr int U = 4;
+    for (int64_t i0 = (int64_t)blockIdx.x * (256 * U) + threadIdx.x; i0 < vecs; i0 += (int64_t)gridDim.x * (256 * U)) {
+        RawVec<T, VEC> ra[U], rb[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u)
+            if (i0 + u * 256 < vecs) { ra[u] = load_raw<T, VEC>(a + (i0 + u * 256) * VEC); rb[u] = load_raw<T, VEC>(b + (i0 + u * 256) * VEC); }
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            if (i0 + u * 256 >= vecs) break;
+            float x[VEC], y[VEC], o[VEC];
+            unpack<T, VEC>(ra[u], x);
+            unpack<T, VEC>(rb[u], y);
+#pragma unroll
+            for (int k = 0; k < VEC; ++k) o[k] = x[k] + y[k];
+            store_vec<T, VEC>(out + (i0 + u * 256) * VEC, o);
+        }
+    }
+}
+static bool aligned16(const void* p) { return ((uintptr_t)p & 15u) == 0; }
 int add_tensors(int dtype, int64_t elems, const void* a, const void* b, void* out, void* stream) {
-    if (dtype == CKPT_DTYPE_BF16)
-        add_kernel<__nv_bfloat16><<<elementwise_grid(elems), 256, 0, (cudaStream_t)stream>>>((const __nv_bfloat16*)a, (const __nv_bfloat16*)b, (__nv_bfloat16*)out, elems);
-    else
-        add_kernel<float><<<elementwise_grid(elems), 256, 0, (cudaStream_t)stream>>>((const float*)a, (const float*)b, (float*)out, elems);
+    cudaStream_t st = (cudaStream_t)stream;
+    const int vec = dtype == CKPT_DTYPE_BF16 ? 8 : 4;
+    if (elems % vec == 0 && aligned16(a) && aligned16(b) && aligned16(out)) {
+        const int64_t vecs = elems / vec;
+        const unsigned grid = (unsigned)std::max<int64_t>(1, std::min<int64_t>((vecs + 1023) / 1024, 148 * 32));
+        if (dtype == CKPT_DTYPE_BF16) add_vec_kernel<__nv_bfloat16, 8><<<grid, 256, 0, st>>>((const __nv_bfloat16*)a, (const __nv_bfloat16*)b, (__nv_bfloat16*)out, vecs);
+        else add_vec_kernel<float, 4><<<grid, 256, 0, st>>>((const float*)a, (const float*)b, (float*)out, vecs);
+    } else if (dtype == CKPT_DTYPE_BF16) {
+        add_kernel<__nv_bfloat16><<<elementwise_grid(elems), 256, 0, st>>>((const __nv_bfloat16*)a, (const __nv_bfloat16*)b, (__nv_bfloat16*)out, elems);
+    } else {
+        add_kernel<float><<<elementwise_grid(elems), 256, 0, st>>>((const float*)a, (const float*)b, (float*)out, elems);
+    }
     CKPT_LAUNCH_CHECK("gradient join");
     return CKPT_OK;
 }
@@ -1135,9 +1220,40 @@ __global__ void relu_mask_kernel(T* __restrict__ g, const T* __restrict__ y, int
     for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < elems; i += (int64_t)gridDim.x * blockDim.x)
         if (!(ld(y + i) > 0.f)) g[i] = cvt<T>(0.f);
 }
+// 16-byte form: g is rewritten whole (the kept elements unchanged), four packed loads per operand in flight.
+template <typename T, int VEC>
+__global__ void __launch_bounds__(256) relu_mask_vec_kernel(T* __restrict__ g, const T* __restrict__ y, int64_t vecs) {
+    constexpr int U = 4;
+    for (int64_t i0 = (int64_t)blockIdx.x * (256 * U) + threadIdx.x; i0 < vecs; i0 += (int64_t)gridDim.x * (256 * U)) {
+        RawVec<T, VEC> rg[U], ry[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u)
+            if (i0 + u * 256 < vecs) { rg[u] = load_raw<T, VEC>(g + (i0 + u * 256) * VEC); ry[u] = load_raw<T, VEC>(y + (i0 + u * 256) * VEC); }
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            if (i0 + u * 256 >= vecs) break;
+            float gv[VEC], yv[VEC], o[VEC];
+            unpack<T, VEC>(rg[u], gv);
+            unpack<T, VEC>(ry[u], yv);
+#pragma unroll
+            for (int k = 0; k < VEC; ++k) o[k] = yv[k] > 0.f ? gv[k] : 0.f;
+            store_vec<T, VEC>(g + (i0 + u * 256) * VEC, o);
+        }
+    }
+}
 int relu_mask_inplace(int dtype, int64_t elems, void* g, const void* y, void* stream) {
-    if (dtype == CKPT_DTYPE_BF16) relu_mask_kernel<__nv_bfloat16><<<elementwise_grid(elems), 256, 0, (cudaStream_t)stream>>>((__nv_bfloat16*)g, (const __nv_bfloat16*)y, elems);
-    else relu_mask_kernel<float><<<elementwise_grid(elems), 256, 0, (cudaStream_t)stream>>>((float*)g, (const float*)y, elems);
+    cudaStream_t st = (cudaStream_t)stream;
+    const int vec = dtype == CKPT_DTYPE_BF16 ? 8 : 4;
+    if (elems % vec == 0 && aligned16(g) && aligned16(y)) {
+        const int64_t vecs = elems / vec;
+        const unsigned grid = (unsigned)std::max<int64_t>(1, std::min<int64_t>((vecs + 1023) / 1024, 148 * 32));
+        if (dtype == CKPT_DTYPE_BF16) relu_mask_vec_kernel<__nv_bfloat16, 8><<<grid, 256, 0, st>>>((__nv_bfloat16*)g, (const __nv_bfloat16*)y, vecs);
+        else relu_mask_vec_kernel<float, 4><<<grid, 256, 0, st>>>((float*)g, (const float*)y, vecs);
+    } else if (dtype == CKPT_DTYPE_BF16) {
+        relu_mask_kernel<__nv_bfloat16><<<elementwise_grid(elems), 256, 0, st>>>((__nv_bfloat16*)g, (const __nv_bfloat16*)y, elems);
+    } else {
+        relu_mask_kernel<float><<<elementwise_grid(elems), 256, 0, st>>>((float*)g, (const float*)y, elems);
+    }
     CKPT_LAUNCH_CHECK("ReLU mask");
     return CKPT_OK;
 }
