@@ -102,6 +102,26 @@ static int conv_wgrad_any(StepCtx& c, const ConvGeom& g, const void* dz, const v
     return simt_conv_wgrad(c.ch->dtype, g, dz, x, dw, c.ws + c.ch->off_scr, c.ch->scr_bytes, c.stream);
 }
 
+// Convolution followed by the batch statistics of its stored output.  The tensor-core kernels gather the
+// partial sums in their epilogue; every other shape takes a separate pass over z.
+static int conv_with_statistics(StepCtx& c, const ConvGeom& g, const void* x, const void* w, void* z, const float* gamma,
+                                const float* beta, float* stats) {
+    const int dt = c.ch->dtype;
+    const int64_t rows = (int64_t)g.n * g.ho * g.wo;
+    char* scr = c.ws + c.ch->off_scr;
+    int rc;
+    if (use_tc(c.ch, g) || (c.ch->impl == 0 && tc_first_conv_supported(dt, g))) {
+        int blocks = 0;
+        if (use_tc(c.ch, g)) rc = tc_conv_fwd_stats(g, x, w, z, (float*)scr, &blocks, c.status(), c.stream);
+        else rc = tc_first_conv_fwd(g, x, w, z, c.status(), c.stream, (float*)scr, &blocks);
+        if (rc) return rc;
+        if (blocks > 0) return bn_statistics_from_partials((const float*)scr, blocks, rows, g.cout, gamma, beta, stats, c.stream);
+    } else if ((rc = conv_forward_any(c, g, x, w, z, nullptr, 0))) {
+        return rc;
+    }
+    return bn_statistics(dt, rows, g.cout, z, gamma, beta, stats, scr, c.stream);
+}
+
 // A conv+BN+ReLU unit stores its convolution output *before* normalisation as d_i; normalisation and
 // ReLU (fixed by the batch statistics saved next to the parameters) are applied by whoever reads
 // d_i.  The unit's backward then has everything it needs - its input, its own pre-normalisation
@@ -153,21 +173,16 @@ static BlockBuffers block_buffers(StepCtx& c, const Unit& u) {
 static int block_interiors(StepCtx& c, const Unit& u, const void* x, const BlockBuffers& B) {
     const int dt = c.ch->dtype;
     void* const* p = c.params + u.param_first;
-    char* scr = c.ws + c.ch->off_scr;
     const int64_t in_px = c.ch->batch * u.in.h * u.in.w, out_px = c.ch->batch * u.out.h * u.out.w;
-    const int mid = u.desc.mid, co = u.out.c;
+    const int mid = u.desc.mid;
     int rc;
-    if ((rc = conv_forward_any(c, u.g1, x, p[0], B.z1, nullptr, 0))) return rc;
-    if ((rc = bn_statistics(dt, in_px, mid, B.z1, (const float*)p[1], (const float*)p[2], B.s1, scr, c.stream))) return rc;
+    if ((rc = conv_with_statistics(c, u.g1, x, p[0], B.z1, (const float*)p[1], (const float*)p[2], B.s1))) return rc;
     if ((rc = bn_apply(dt, in_px, mid, B.z1, B.s1, 1, B.a, c.stream))) return rc;
-    if ((rc = conv_forward_any(c, u.g2, B.a, p[3], B.z2, nullptr, 0))) return rc;
-    if ((rc = bn_statistics(dt, out_px, mid, B.z2, (const float*)p[4], (const float*)p[5], B.s2, scr, c.stream))) return rc;
+    if ((rc = conv_with_statistics(c, u.g2, B.a, p[3], B.z2, (const float*)p[4], (const float*)p[5], B.s2))) return rc;
     if ((rc = bn_apply(dt, out_px, mid, B.z2, B.s2, 1, B.b, c.stream))) return rc;
-    if ((rc = conv_forward_any(c, u.g3, B.b, p[6], B.z3, nullptr, 0))) return rc;
-    if ((rc = bn_statistics(dt, out_px, co, B.z3, (const float*)p[7], (const float*)p[8], B.s3, scr, c.stream))) return rc;
+    if ((rc = conv_with_statistics(c, u.g3, B.b, p[6], B.z3, (const float*)p[7], (const float*)p[8], B.s3))) return rc;
     if (u.desc.flags & 2) {
-        if ((rc = conv_forward_any(c, u.gp, x, p[9], B.zp, nullptr, 0))) return rc;
-        if ((rc = bn_statistics(dt, out_px, co, B.zp, (const float*)p[10], (const float*)p[11], B.sp, scr, c.stream))) return rc;
+        if ((rc = conv_with_statistics(c, u.gp, x, p[9], B.zp, (const float*)p[10], (const float*)p[11], B.sp))) return rc;
     }
     return CKPT_OK;
 }
@@ -227,19 +242,7 @@ static int unit_forward(StepCtx& c, int64_t i, const void* x_raw, void* y) {
     switch (u.desc.kind) {
         case CKPT_UNIT_CONV_BN_RELU:
             if ((rc = activated(c, i - 1, x_raw, &x))) return rc;
-            if (use_tc(c.ch, u.geom) || (c.ch->impl == 0 && tc_first_conv_supported(dt, u.geom))) {
-                // the persistent tensor-core kernels gather the statistics of their output in the epilogue
-                int blocks = 0;
-                float* partial = (float*)(ws + c.ch->off_scr);
-                if (use_tc(c.ch, u.geom)) rc = tc_conv_fwd_stats(u.geom, x, p[0], y, partial, &blocks, c.status(), c.stream);
-                else rc = tc_first_conv_fwd(u.geom, x, p[0], y, c.status(), c.stream, partial, &blocks);
-                if (rc) return rc;
-                if (blocks > 0)
-                    return bn_statistics_from_partials(partial, blocks, rows_of(c.ch, i), u.out.c, (const float*)p[1],
-                                                       (const float*)p[2], stats_of(c, i), c.stream);
-            } else if ((rc = conv_forward_any(c, u.geom, x, p[0], y, nullptr, 0))) return rc;
-            return bn_statistics(dt, rows_of(c.ch, i), u.out.c, y, (const float*)p[1], (const float*)p[2], stats_of(c, i),
-                                 ws + c.ch->off_scr, c.stream);
+            return conv_with_statistics(c, u.geom, x, p[0], y, (const float*)p[1], (const float*)p[2], stats_of(c, i));
         case CKPT_UNIT_CONV:
             if ((rc = activated(c, i - 1, x_raw, &x))) return rc;
             return conv_forward_any(c, u.geom, x, p[0], y, nullptr, 0);

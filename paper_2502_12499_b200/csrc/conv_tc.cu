@@ -172,6 +172,54 @@ __host__ __device__ inline uint32_t instr_desc(int M, int N, int a_mn_major, int
     return d;
 }
 
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+
+// Column sums of a 32 x 32 block held one row per lane (v[c] = element of column c in this lane's row):
+// a butterfly of 31 exchanges in a fixed order; afterwards lane l holds the sum of column l.
+__device__ __forceinline__ float warp_column_sum(float (&v)[32], int lane) {
+#pragma unroll
+    for (int o = 16; o >= 1; o >>= 1) {
+        const bool upper = (lane & o) != 0;
+#pragma unroll
+        for (int i = 0; i < o; ++i) {
+            const float send = upper ? v[i] : v[i + o];
+            const float keep = upper ? v[i + o] : v[i];
+            v[i] = keep + __shfl_xor_sync(0xffffffffu, send, o);
+        }
+    }
+    return v[0];
+}
+
+// Epilogue of one 32-column chunk: rounds the accumulators to bf16, stores the valid rows and, when the
+// batch-norm statistics are gathered here, adds the chunk's per-column sum and sum of squares (of
+// the rounded values, i.e. of what is stored) into the lane's running totals.
+__device__ __forceinline__ void store_chunk(const uint32_t (&v)[32], bool valid, __nv_bfloat16* dst, bool stats, int lane,
+                                            float& sum, float& sumsq) {
+    float r[32];
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+        uint4 pk;
+        __nv_bfloat162* h = reinterpret_cast<__nv_bfloat162*>(&pk);
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            h[e] = __floats2bfloat162_rn(__uint_as_float(v[8 * q + 2 * e]), __uint_as_float(v[8 * q + 2 * e + 1]));
+            const float2 f = __bfloat1622float2(h[e]);
+            r[8 * q + 2 * e] = valid ? f.x : 0.f;
+            r[8 * q + 2 * e + 1] = valid ? f.y : 0.f;
+        }
+        if (valid) *reinterpret_cast<uint4*>(dst + 8 * q) = pk;
+    }
+    if (stats) {
+        float sq[32];
+#pragma unroll
+        for (int e = 0; e < 32; ++e) sq[e] = r[e] * r[e];
+        sum += warp_column_sum(r, lane);
+        sumsq += warp_column_sum(sq, lane);
+    }
+}
+
 // ------------------------------------------------------------------------------------------------
 // Forward / dgrad kernel
 // ------------------------------------------------------------------------------------------------
@@ -194,8 +242,10 @@ struct FwdParams {
 template <bool B_MN>
 __global__ void __launch_bounds__(kThreads, 1)
 tc_conv_fwd_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w,
-                   __nv_bfloat16* __restrict__ out, const float* __restrict__ bias, int relu, FwdParams p, int* status) {
+                   __nv_bfloat16* __restrict__ out, const float* __restrict__ bias, int relu, float* __restrict__ stat_partial,
+                   FwdParams p, int* status) {
     extern __shared__ uint8_t smem_raw[];
+    __shared__ float stat_red[4][2][256];        // per-quarter column sums of the tile (batch-norm statistics)
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const uint32_t a_bytes = 128 * 128, b_bytes = (uint32_t)p.bn * 128, stage_bytes = a_bytes + b_bytes;
     const uint32_t bars = base + (uint32_t)p.stages * stage_bytes;           // full[s], empty[s], accum
@@ -289,7 +339,31 @@ tc_conv_fwd_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_const
         const int oh = (h0 + hl) * p.out_stride + p.out_oh, ow = (w0 + wl) * p.out_stride + p.out_ow;
         const bool valid = (w0 + wl < p.W) && (h0 + hl < p.H) && (n0 + nl < p.N) && oh < p.out_H && ow < p.out_W;
         __nv_bfloat16* dst = out + ((((size_t)(n0 + nl) * p.out_H + oh) * p.out_W + ow) * p.c_out + (size_t)n_tile * p.bn);
-        if (mbar_wait(accum_bar, 0, failed, status, 103)) {
+        if (stat_partial) {
+            // batch-norm sums of the stored tile: one partial row pair per pixel tile, the four quarters added
+            // in a fixed order (the caller guarantees whole 32-column chunks and no bias/ReLU)
+            if (mbar_wait(accum_bar, 0, failed, status, 103)) {
+                tc_fence_after();
+                for (int c0 = 0; c0 < p.bn; c0 += 32) {
+                    uint32_t v[32];
+                    tmem_ld32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)c0, v);
+                    float sum = 0.f, sumsq = 0.f;
+                    store_chunk(v, valid, dst + c0, true, lane, sum, sumsq);
+                    stat_red[quarter][0][c0 + lane] = sum;
+                    stat_red[quarter][1][c0 + lane] = sumsq;
+                }
+            } else {
+                for (int c0 = 0; c0 < p.bn; c0 += 32) { stat_red[quarter][0][c0 + lane] = 0.f; stat_red[quarter][1][c0 + lane] = 0.f; }
+            }
+            asm volatile("bar.sync 1, 128;" ::: "memory");
+            const size_t m_tile = blockIdx.x / p.n_tiles;
+            for (int col = quarter * 32 + lane; col < p.bn; col += 128) {
+#pragma unroll
+                for (int k = 0; k < 2; ++k)
+                    stat_partial[(m_tile * 2 + k) * p.c_out + (size_t)n_tile * p.bn + col] =
+                        (stat_red[0][k][col] + stat_red[1][k][col]) + (stat_red[2][k][col] + stat_red[3][k][col]);
+            }
+        } else if (mbar_wait(accum_bar, 0, failed, status, 103)) {
             tc_fence_after();
             for (int c0 = 0; c0 < p.bn; c0 += 32) {
                 uint32_t v[32];
@@ -348,54 +422,6 @@ struct C64Params {
     int ctas_per_n;              // persistent CTAs that share one output-channel tile
     uint32_t box_stride;         // bytes between the three shifted copies of a patch
 };
-
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-
-// Column sums of a 32 x 32 block held one row per lane (v[c] = element of column c in this lane's row):
-// a butterfly of 31 exchanges in a fixed order; afterwards lane l holds the sum of column l.
-__device__ __forceinline__ float warp_column_sum(float (&v)[32], int lane) {
-#pragma unroll
-    for (int o = 16; o >= 1; o >>= 1) {
-        const bool upper = (lane & o) != 0;
-#pragma unroll
-        for (int i = 0; i < o; ++i) {
-            const float send = upper ? v[i] : v[i + o];
-            const float keep = upper ? v[i + o] : v[i];
-            v[i] = keep + __shfl_xor_sync(0xffffffffu, send, o);
-        }
-    }
-    return v[0];
-}
-
-// Epilogue of one 32-column chunk: rounds the accumulators to bf16, stores the valid rows and, when the
-// batch-norm statistics are gathered here, adds the chunk's per-column sum and sum of squares (of
-// the rounded values, i.e. of what is stored) into the lane's running totals.
-__device__ __forceinline__ void store_chunk(const uint32_t (&v)[32], bool valid, __nv_bfloat16* dst, bool stats, int lane,
-                                            float& sum, float& sumsq) {
-    float r[32];
-#pragma unroll
-    for (int q = 0; q < 4; ++q) {
-        uint4 pk;
-        __nv_bfloat162* h = reinterpret_cast<__nv_bfloat162*>(&pk);
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-            h[e] = __floats2bfloat162_rn(__uint_as_float(v[8 * q + 2 * e]), __uint_as_float(v[8 * q + 2 * e + 1]));
-            const float2 f = __bfloat1622float2(h[e]);
-            r[8 * q + 2 * e] = valid ? f.x : 0.f;
-            r[8 * q + 2 * e + 1] = valid ? f.y : 0.f;
-        }
-        if (valid) *reinterpret_cast<uint4*>(dst + 8 * q) = pk;
-    }
-    if (stats) {
-        float sq[32];
-#pragma unroll
-        for (int e = 0; e < 32; ++e) sq[e] = r[e] * r[e];
-        sum += warp_column_sum(r, lane);
-        sumsq += warp_column_sum(sq, lane);
-    }
-}
 
 __global__ void __launch_bounds__(kThreads, 1)
 tc_conv_c64_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w,
@@ -1495,9 +1521,15 @@ int launch_halo(const void* x, const void* w_mat, void* out, float* stat_partial
 // The generic kernel on a prepared term table (p.taps, p.tap_*, p.in_stride, p.out_*).  The operand tensor is
 // [a_n][a_h][a_w][c_red]; the tiles walk an n x gh x gw pixel grid.  `taps_total` = 64-channel column groups of
 // the filter matrix per reduction block (k*k).
+int64_t generic_stat_rows(int n, int gh, int gw) {
+    int tw, th, tn;
+    choose_tile(128, gw, gh, n, &tw, &th, &tn);
+    return (int64_t)((gw + tw - 1) / tw) * ((gh + th - 1) / th) * ((n + tn - 1) / tn);
+}
+
 int launch_generic(FwdParams p, const void* a, int a_n, int a_h, int a_w, const void* w_mat, int taps_total, void* out,
                    const float* bias, int relu, int n, int gh, int gw, int c_red, int c_out, int* status, cudaStream_t st,
-                   const char* what, bool b_mn) {
+                   const char* what, bool b_mn, float* stat_partial = nullptr, int* stat_blocks = nullptr) {
     p.H = gh; p.W = gw; p.N = n; p.c_red = c_red; p.c_out = c_out;
     choose_tile(128, gw, gh, n, &p.tw, &p.th, &p.tn);
     p.tiles_w = (gw + p.tw - 1) / p.tw; p.tiles_h = (gh + p.th - 1) / p.th; p.tiles_n = (n + p.tn - 1) / p.tn;
@@ -1524,8 +1556,11 @@ int launch_generic(FwdParams p, const void* a, int a_n, int a_h, int a_w, const 
         attr_set = true;
     }
     const int64_t ctas = (int64_t)p.tiles_w * p.tiles_h * p.tiles_n * p.n_tiles;
-    if (b_mn) tc_conv_fwd_kernel<true><<<(unsigned)ctas, kThreads, smem, st>>>(mx, mw, (__nv_bfloat16*)out, bias, relu, p, status);
-    else tc_conv_fwd_kernel<false><<<(unsigned)ctas, kThreads, smem, st>>>(mx, mw, (__nv_bfloat16*)out, bias, relu, p, status);
+    // statistics in the epilogue: whole 32-column chunks, plain stores, output written once per pixel
+    const bool gather = stat_partial && stat_blocks && !bias && !relu && !b_mn && c_out % 64 == 0 && p.bn >= 32 && p.out_stride == 1;
+    if (gather) *stat_blocks = (int)(ctas / p.n_tiles);
+    if (b_mn) tc_conv_fwd_kernel<true><<<(unsigned)ctas, kThreads, smem, st>>>(mx, mw, (__nv_bfloat16*)out, bias, relu, nullptr, p, status);
+    else tc_conv_fwd_kernel<false><<<(unsigned)ctas, kThreads, smem, st>>>(mx, mw, (__nv_bfloat16*)out, bias, relu, gather ? stat_partial : nullptr, p, status);
     CKPT_LAUNCH_CHECK(what);
     return CKPT_OK;
 }
@@ -1549,7 +1584,8 @@ int launch_fwd_like(const void* x, const void* w_mat, void* out, const float* bi
     }
     p.in_stride = 1;
     p.out_H = H; p.out_W = W; p.out_stride = 1; p.out_oh = 0; p.out_ow = 0;
-    return launch_generic(p, x, N, H, W, w_mat, k * k, out, bias, relu, N, H, W, c_red, c_out, status, st, what, b_mn);
+    return launch_generic(p, x, N, H, W, w_mat, k * k, out, bias, relu, N, H, W, c_red, c_out, status, st, what, b_mn, stat_partial,
+                          stat_blocks);
 }
 
 void wgrad_plan(const ConvGeom& g, WgradParams* p, int* slices, int* groups, int* co_tiles) {
@@ -1648,7 +1684,18 @@ bool tc_conv_supported(int dtype, const ConvGeom& g) {
     return true;
 }
 
+// batch-norm partial sums left by the forward kernel: one row pair per pixel tile
+static int64_t tc_conv_stat_bytes(const ConvGeom& g) {
+    return generic_stat_rows(g.n, g.ho, g.wo) * 2 * (int64_t)g.cout * 4;
+}
+
+static int64_t tc_conv_work_bytes(const ConvGeom& g);
 int64_t tc_conv_scratch_bytes(const ConvGeom& g) {
+    return std::max(tc_conv_stat_bytes(g), tc_conv_work_bytes(g));
+}
+
+// partial sums of the split weight gradient, or the transposed filter of the input gradient
+static int64_t tc_conv_work_bytes(const ConvGeom& g) {
     if (wgrad_c64_applies(g)) {
         W64Params q;
         wgrad_c64_plan(g, &q);
@@ -1703,14 +1750,15 @@ int tc_first_conv_fwd(const ConvGeom& g, const void* x, const void* w, void* z, 
 }
 
 // Strided forward: the operand boxes take every stride-th input pixel, the tiles walk the output grid.
-static int launch_strided_fwd(const ConvGeom& g, const void* x, const void* w, void* z, int* status, cudaStream_t st) {
+static int launch_strided_fwd(const ConvGeom& g, const void* x, const void* w, void* z, int* status, cudaStream_t st,
+                              float* stat_partial = nullptr, int* stat_blocks = nullptr) {
     FwdParams p;
     p.taps = g.k * g.k;
     for (int t = 0; t < p.taps; ++t) { p.tap_dh[t] = t / g.k - g.pad; p.tap_dw[t] = t % g.k - g.pad; p.tap_col[t] = t; }
     p.in_stride = g.stride;
     p.out_H = g.ho; p.out_W = g.wo; p.out_stride = 1; p.out_oh = 0; p.out_ow = 0;
     return launch_generic(p, x, g.n, g.h, g.w, w, p.taps, z, nullptr, 0, g.n, g.ho, g.wo, g.cin, g.cout, status, st,
-                          "strided conv forward (tensor cores)", false);
+                          "strided conv forward (tensor cores)", false, stat_partial, stat_blocks);
 }
 
 // Forward convolution that also leaves the batch-norm partial sums of its output in `partial`
@@ -1719,7 +1767,8 @@ int tc_conv_fwd_stats(const ConvGeom& g, const void* x, const void* w, void* z, 
                       void* stream) {
     if (!tc_conv_supported(CKPT_DTYPE_BF16, g)) { set_error("tensor-core conv: unsupported shape"); return CKPT_E_UNSUPPORTED; }
     if (!device_status || !blocks) { set_error("device status word missing"); return CKPT_E_NULL; }
-    if (g.stride != 1) { *blocks = 0; return launch_strided_fwd(g, x, w, z, device_status, (cudaStream_t)stream); }
+    *blocks = 0;
+    if (g.stride != 1) return launch_strided_fwd(g, x, w, z, device_status, (cudaStream_t)stream, partial, blocks);
     return launch_fwd_like(x, w, z, nullptr, 0, g.n, g.h, g.w, g.cin, g.cout, g.k, g.pad, device_status, (cudaStream_t)stream,
                            "conv forward (tensor cores)", partial, blocks);
 }
