@@ -192,6 +192,17 @@ CKPT_API int ckpt_chain_workspace_bytes(const ckpt_chain* chain, int64_t* bytes)
 /* Kernel selection for dense contractions: 0 = automatic (tensor cores where a kernel exists),
  * 1 = plain CUDA-core kernels only. */
 CKPT_API int ckpt_chain_set_impl(ckpt_chain* chain, int impl);
+/* Graph replay of the training step (off by default).  The launch sequence of a step (Algorithms 1, 2
+ * and 4 as executed here) is a function of the chain, the plan, the policy and the pointers passed to
+ * ckpt_train_step.  With enable = 1 the first step with a given set of those arguments runs launch by
+ * launch, the second is recorded as a CUDA graph while it runs, and later ones replay the recording:
+ * one submission per step, which matters for chains whose kernels are shorter than a launch (hundreds
+ * of units on small tensors).  Results are bit-identical to the launch-by-launch step.  Up to four
+ * recordings are kept per chain (least recently used dropped).  The caller keeps every buffer of a
+ * recorded step alive and unchanged in place (contents may change, addresses may not); a batch or
+ * label pointer in pageable host memory disables recording for that call.  enable = 0 drops the
+ * recordings.  The library holds 64 bytes of pinned host memory per chain while enabled. */
+CKPT_API int ckpt_chain_set_graph(ckpt_chain* chain, int enable);
 
 /* ---------------------------------------------------------------- the training step
  *
@@ -221,7 +232,7 @@ typedef struct ckpt_step_report {
     int64_t recomputed_units;/* unit forwards re-run during the backward phase                   */
     double loss;
     int32_t device_status;   /* 0, or the code written by a kernel whose bounded wait gave up    */
-    int32_t reserved;
+    int32_t replayed;        /* 1 when the step ran as a replay of its captured launch sequence  */
 } ckpt_step_report;
 
 CKPT_API int ckpt_train_step(ckpt_chain* chain, const uint8_t* is_ckpt, int policy, const void* batch,

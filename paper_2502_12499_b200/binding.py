@@ -43,7 +43,7 @@ class ConvShape(C.Structure):
 class StepReport(C.Structure):
     _fields_ = [("peak_bytes", C.c_int64), ("extent_bytes", C.c_int64), ("predicted_bytes", C.c_int64),
                 ("workspace_bytes", C.c_int64), ("launches", C.c_int64), ("recomputed_units", C.c_int64),
-                ("loss", C.c_double), ("device_status", C.c_int32), ("reserved", C.c_int32)]
+                ("loss", C.c_double), ("device_status", C.c_int32), ("replayed", C.c_int32)]
 
 
 _lib = None
@@ -216,6 +216,10 @@ class Chain:
 
     def set_impl(self, impl):
         _check(lib().ckpt_chain_set_impl(self._h, C.c_int(impl)))
+
+    def set_graph(self, enable):
+        """ckpt_chain_set_graph: record the launch sequence of a repeated step once and replay it."""
+        _check(lib().ckpt_chain_set_graph(self._h, C.c_int(1 if enable else 0)))
 
 
 def flatten_params(chain_spec, params):

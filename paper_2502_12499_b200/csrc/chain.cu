@@ -5,6 +5,7 @@
 #include <cuda_runtime.h>
 
 #include <algorithm>
+#include <cstdint>
 #include <cstring>
 
 #include "internal.h"
@@ -25,6 +26,15 @@ struct Unit {
 
 struct ParamInfo { int64_t unit, elems; int32_t dtype; };
 
+// One captured step: the launch sequence of run_step for a fixed set of arguments.
+struct StepGraph {
+    uint64_t key = 0;
+    cudaGraph_t graph = nullptr;
+    cudaGraphExec_t exec = nullptr;
+    int64_t peak = 0, extent = 0, launches = 0, recomputed = 0;
+    uint64_t last_use = 0;
+};
+
 }  // namespace ckpt
 
 struct ckpt_chain {
@@ -37,6 +47,14 @@ struct ckpt_chain {
     // workspace layout (byte offsets)
     int64_t max_d = 0, off_g0 = 0, off_g1 = 0, off_z = 0, off_scr = 0, scr_bytes = 0, off_stats = 0,
             off_misc = 0, off_blk = 0, blk_bytes = 0, ws_bytes = 0;
+    // graph replay: steps captured once per distinct argument set (pointers, plan, policy)
+    int use_graph = 0;
+    std::vector<ckpt::StepGraph> graphs;
+    std::vector<uint64_t> seen_keys;     // argument sets that have run once without capture
+    void* host_result = nullptr;         // pinned: loss (8 bytes) and status word of the last step
+    cudaStream_t capture_stream = nullptr;   // recording happens here (the caller's stream may be the default one,
+                                             // which cannot record); replays run on the caller's stream
+    ~ckpt_chain();
 };
 
 namespace ckpt {
@@ -72,6 +90,7 @@ struct StepCtx {
     Arena* arena;
     int64_t recomputed = 0;
     int64_t* stage_trace = nullptr;     // optional: live arena bytes at the end of each of the 2n+2 stages
+    void* host_result = nullptr;        // capture: pinned destination of the loss and the status word (no wait)
     int* status() const { return (int*)(ws + ch->off_misc + 64); }
 };
 
@@ -355,6 +374,16 @@ static int unit_backward(StepCtx& c, int64_t i, const void* x_raw, const void* y
     return CKPT_OK;
 }
 
+// loss (float for softmax cross-entropy, double for the sum loss) at byte 0, device status word at byte 8
+static int decode_result(const ckpt_chain* ch, const void* result, double* loss_out) {
+    int status = 0;
+    memcpy(&status, (const char*)result + 8, sizeof(int));
+    if (ch->loss == CKPT_LOSS_SOFTMAX_CE) { float l; memcpy(&l, result, sizeof(float)); *loss_out = l; }
+    else { double l; memcpy(&l, result, sizeof(double)); *loss_out = l; }
+    if (status != 0) { set_error("a device-side wait gave up (status %d)", status); return CKPT_E_DEVICE_TIMEOUT; }
+    return CKPT_OK;
+}
+
 static int run_step(StepCtx& c, double* loss_out) {
     ckpt_chain* ch = c.ch;
     const int64_t n = (int64_t)ch->units.size();
@@ -474,23 +503,20 @@ static int run_step(StepCtx& c, double* loss_out) {
     if (c.stage_trace) c.stage_trace[2 * n + 1] = d[0];
 
     if (!c.dry) {
-        int status = 0;
-        cudaError_t e;
-        if (ch->loss == CKPT_LOSS_SOFTMAX_CE) {
-            float l = 0;
-            e = cudaMemcpyAsync(&l, c.ws + ch->off_misc, sizeof(float), cudaMemcpyDeviceToHost, c.stream);
-            if (e == cudaSuccess) e = cudaMemcpyAsync(&status, c.status(), sizeof(int), cudaMemcpyDeviceToHost, c.stream);
-            if (e == cudaSuccess) e = cudaStreamSynchronize(c.stream);
-            *loss_out = l;
-        } else {
-            double l = 0;
-            e = cudaMemcpyAsync(&l, c.ws + ch->off_misc, sizeof(double), cudaMemcpyDeviceToHost, c.stream);
-            if (e == cudaSuccess) e = cudaMemcpyAsync(&status, c.status(), sizeof(int), cudaMemcpyDeviceToHost, c.stream);
-            if (e == cudaSuccess) e = cudaStreamSynchronize(c.stream);
-            *loss_out = l;
+        const size_t loss_bytes = ch->loss == CKPT_LOSS_SOFTMAX_CE ? sizeof(float) : sizeof(double);
+        if (c.host_result) {
+            // being captured: the results travel to pinned memory; whoever launches the graph waits and decodes
+            cudaError_t e = cudaMemcpyAsync(c.host_result, c.ws + ch->off_misc, loss_bytes, cudaMemcpyDeviceToHost, c.stream);
+            if (e == cudaSuccess) e = cudaMemcpyAsync((char*)c.host_result + 8, c.status(), sizeof(int), cudaMemcpyDeviceToHost, c.stream);
+            if (e != cudaSuccess) return cuda_fail(e, "queueing the end-of-step copies");
+            return CKPT_OK;
         }
+        char result[16] = {0};
+        cudaError_t e = cudaMemcpyAsync(result, c.ws + ch->off_misc, loss_bytes, cudaMemcpyDeviceToHost, c.stream);
+        if (e == cudaSuccess) e = cudaMemcpyAsync(result + 8, c.status(), sizeof(int), cudaMemcpyDeviceToHost, c.stream);
+        if (e == cudaSuccess) e = cudaStreamSynchronize(c.stream);
         if (e != cudaSuccess) return cuda_fail(e, "end-of-step synchronisation");
-        if (status != 0) { set_error("a device-side wait gave up (status %d)", status); return CKPT_E_DEVICE_TIMEOUT; }
+        return decode_result(ch, result, loss_out);
     }
     return CKPT_OK;
 }
@@ -500,7 +526,102 @@ static int policy_model(int policy) {
          : policy == CKPT_POLICY_STATIC ? CKPT_MODEL_STATIC : CKPT_MODEL_DYNAMIC;
 }
 
+// ---------------------------------------------------------------------------------------------
+// Graph replay.  Every launch of a step depends only on the chain, the plan, the policy and the
+// pointers it is given (tensor maps and arena offsets are functions of those), so a step whose
+// arguments repeat is recorded once as a CUDA graph and replayed: one submission instead of
+// hundreds to tens of thousands of launches.
+// ---------------------------------------------------------------------------------------------
+static const size_t kMaxGraphs = 4;
+
+static uint64_t mix(uint64_t h, uint64_t v) {
+    h ^= v + 0x9E3779B97F4A7C15ull + (h << 6) + (h >> 2);
+    return h * 0xFF51AFD7ED558CCDull;
+}
+static uint64_t step_key(const ckpt_chain* ch, const uint8_t* is_ckpt, int policy, const void* batch, const int32_t* labels,
+                         void* const* params, void* const* grads, const void* arena, const void* ws) {
+    uint64_t h = mix(0x1234567ull, (uint64_t)policy);
+    h = mix(h, (uint64_t)(uintptr_t)batch); h = mix(h, (uint64_t)(uintptr_t)labels);
+    h = mix(h, (uint64_t)(uintptr_t)arena); h = mix(h, (uint64_t)(uintptr_t)ws);
+    h = mix(h, (uint64_t)ch->impl);
+    for (size_t p = 0; p < ch->params.size(); ++p) { h = mix(h, (uint64_t)(uintptr_t)params[p]); h = mix(h, (uint64_t)(uintptr_t)grads[p]); }
+    if (policy != CKPT_POLICY_STORE_ALL)
+        for (size_t i = 0; i <= ch->units.size(); ++i) h = mix(h, (uint64_t)is_ckpt[i] + 3 * i);
+    return h;
+}
+// A copy from pageable host memory cannot be part of a captured sequence.
+static bool graph_eligible(const void* batch, const int32_t* labels) {
+    const void* ptrs[2] = {batch, labels};
+    for (const void* p : ptrs) {
+        if (!p) continue;
+        cudaPointerAttributes a;
+        if (cudaPointerGetAttributes(&a, p) != cudaSuccess) { cudaGetLastError(); return false; }
+        if (a.type == cudaMemoryTypeUnregistered) return false;
+    }
+    return true;
+}
+static StepGraph* find_graph(ckpt_chain* ch, uint64_t key) {
+    static uint64_t clock = 0;
+    for (StepGraph& g : ch->graphs)
+        if (g.key == key) { g.last_use = ++clock; return &g; }
+    return nullptr;
+}
+static void destroy_graph(StepGraph& g) {
+    if (g.exec) cudaGraphExecDestroy(g.exec);
+    if (g.graph) cudaGraphDestroy(g.graph);
+    g.exec = nullptr; g.graph = nullptr;
+}
+static void drop_graphs(ckpt_chain* ch) {
+    for (StepGraph& g : ch->graphs) destroy_graph(g);
+    ch->graphs.clear();
+    ch->seen_keys.clear();
+}
+static int capture_step(ckpt_chain* ch, StepCtx c, uint64_t key, StepGraph** out) {
+    Arena ar(c.arena->capacity());
+    c.arena = &ar;
+    c.host_result = ch->host_result;
+    c.recomputed = 0;
+    cudaError_t e = cudaSuccess;
+    if (!ch->capture_stream) {
+        e = cudaStreamCreateWithFlags(&ch->capture_stream, cudaStreamNonBlocking);
+        if (e != cudaSuccess) { ch->capture_stream = nullptr; return cuda_fail(e, "creating the recording stream"); }
+    }
+    c.stream = ch->capture_stream;
+    e = cudaStreamBeginCapture(c.stream, cudaStreamCaptureModeThreadLocal);
+    if (e != cudaSuccess) return cuda_fail(e, "beginning the capture of a step");
+    const int64_t launches0 = g_launches;
+    double unused = 0;
+    int rc = CKPT_OK;
+    e = cudaMemsetAsync(c.ws + ch->off_misc, 0, 128, c.stream);
+    if (e != cudaSuccess) rc = cuda_fail(e, "clearing the status words");
+    if (!rc) rc = run_step(c, &unused);
+    StepGraph g;
+    e = cudaStreamEndCapture(c.stream, &g.graph);
+    if (rc) { if (g.graph) cudaGraphDestroy(g.graph); return rc; }
+    if (e != cudaSuccess) return cuda_fail(e, "ending the capture of a step");
+    e = cudaGraphInstantiate(&g.exec, g.graph, 0);
+    if (e != cudaSuccess) { cudaGraphDestroy(g.graph); return cuda_fail(e, "instantiating the captured step"); }
+    g.key = key;
+    g.peak = ar.high_water(); g.extent = ar.extent();
+    g.launches = g_launches - launches0; g.recomputed = c.recomputed;
+    if (ch->graphs.size() >= kMaxGraphs) {
+        size_t victim = 0;
+        for (size_t i = 1; i < ch->graphs.size(); ++i) if (ch->graphs[i].last_use < ch->graphs[victim].last_use) victim = i;
+        destroy_graph(ch->graphs[victim]);
+        ch->graphs.erase(ch->graphs.begin() + victim);
+    }
+    ch->graphs.push_back(g);
+    *out = find_graph(ch, key);
+    return CKPT_OK;
+}
+
 }  // namespace ckpt
+
+ckpt_chain::~ckpt_chain() {
+    ckpt::drop_graphs(this);
+    if (host_result) cudaFreeHost(host_result);
+    if (capture_stream) cudaStreamDestroy(capture_stream);
+}
 
 using namespace ckpt;
 
@@ -778,10 +899,36 @@ int ckpt_train_step(ckpt_chain* chain, const uint8_t* is_ckpt, int policy, const
     c.ch = chain; c.is_ckpt = is_ckpt; c.policy = policy; c.dry = false;
     c.arena_base = (char*)arena; c.ws = (char*)workspace; c.params = params; c.grads = grads;
     c.batch = batch; c.labels = labels; c.stream = (cudaStream_t)stream; c.arena = &ar;
+    double loss = 0;
+    if (chain->use_graph && graph_eligible(batch, labels)) {
+        const uint64_t key = step_key(chain, is_ckpt, policy, batch, labels, params, grads, arena, workspace);
+        StepGraph* g = find_graph(chain, key);
+        const bool seen = std::find(chain->seen_keys.begin(), chain->seen_keys.end(), key) != chain->seen_keys.end();
+        if (!g && seen) {
+            // second step with these arguments: record its launch sequence
+            rc = capture_step(chain, c, key, &g);
+            if (rc) return rc;
+        }
+        if (g) {
+            cudaError_t e = cudaGraphLaunch(g->exec, c.stream);
+            if (e == cudaSuccess) e = cudaStreamSynchronize(c.stream);
+            if (e != cudaSuccess) return cuda_fail(e, "replaying the captured step");
+            rc = decode_result(chain, chain->host_result, &loss);
+            report->peak_bytes = g->peak;
+            report->extent_bytes = g->extent;
+            report->launches = g->launches;
+            report->recomputed_units = g->recomputed;
+            report->loss = loss;
+            report->replayed = 1;
+            if (rc == CKPT_E_DEVICE_TIMEOUT) report->device_status = 1;
+            return rc;
+        }
+        chain->seen_keys.push_back(key);       // first step with these arguments runs launch by launch
+        if (chain->seen_keys.size() > 64) chain->seen_keys.erase(chain->seen_keys.begin());
+    }
     cudaError_t e = cudaMemsetAsync(c.ws + chain->off_misc, 0, 128, c.stream);
     if (e != cudaSuccess) return cuda_fail(e, "clearing the status words");
     const int64_t launches0 = g_launches;
-    double loss = 0;
     rc = run_step(c, &loss);
     report->peak_bytes = ar.high_water();
     report->extent_bytes = ar.extent();
@@ -790,6 +937,17 @@ int ckpt_train_step(ckpt_chain* chain, const uint8_t* is_ckpt, int policy, const
     report->loss = loss;
     if (rc == CKPT_E_DEVICE_TIMEOUT) report->device_status = 1;
     return rc;
+}
+
+int ckpt_chain_set_graph(ckpt_chain* chain, int enable) {
+    if (!chain) { set_error("null pointer"); return CKPT_E_NULL; }
+    if (enable && !chain->host_result) {
+        cudaError_t e = cudaHostAlloc(&chain->host_result, 64, cudaHostAllocDefault);
+        if (e != cudaSuccess) { chain->host_result = nullptr; return cuda_fail(e, "pinned result buffer of the captured step"); }
+    }
+    chain->use_graph = enable ? 1 : 0;
+    if (!enable) drop_graphs(chain);
+    return CKPT_OK;
 }
 
 }  // extern "C"

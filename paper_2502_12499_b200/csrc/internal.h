@@ -35,6 +35,7 @@ struct ArenaEvent { int64_t kind, id, offset, size; };
 class Arena {
 public:
     explicit Arena(int64_t capacity) : capacity_(capacity) {}
+    int64_t capacity() const { return capacity_; }
     int alloc_stack(int64_t id, int64_t size, int64_t* offset);
     int alloc_top(int64_t id, int64_t size, int64_t* offset);
     int release(int64_t id);

@@ -295,3 +295,55 @@ def test_arena_too_small_is_rejected_before_any_launch():
     assert e.value.code == -7
     rep, _ = runner.run(ck.POLICY_DYNAMIC, mask, x, None, arena_bytes=peak)
     assert rep["peak_bytes"] == peak
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_graph_replay_is_bit_identical(dtype):
+    """ckpt_chain_set_graph: the first step with a set of arguments runs launch by launch, the second is
+    recorded, later ones replay the recording.  Same buffers, new batch contents each step: gradients,
+    loss and report must equal those of a chain that never records."""
+    import torch
+    spec = mini_vgg(dtype)
+    params = wl.make_params(spec, seed=41, bn_affine="random")
+    plain, graphed = StepRunner(spec, params), StepRunner(spec, params)
+    graphed.chain.set_graph(True)
+    mask = ck.plan(ck.ALGO_DYNAMIC_N, plain.d)[0]
+    peak = ck.eval(ck.MODEL_DYNAMIC, plain.d, mask)
+    tdt = torch.bfloat16 if dtype == "bf16" else torch.float32
+    xb = torch.empty((spec["batch"],) + tuple(spec["input_hwc"]), dtype=tdt, device="cuda")
+    lab = torch.empty(spec["batch"], dtype=torch.int32, device="cuda")
+    arenas = [torch.empty(peak, dtype=torch.uint8, device="cuda") for _ in range(2)]
+    replayed = []
+    for step in range(5):
+        x, labels = wl.make_batch(spec, seed=50 + step)
+        xb.copy_(torch.from_numpy(x).to(tdt))
+        lab.copy_(torch.from_numpy(np.ascontiguousarray(labels, dtype=np.int32)))
+        out = []
+        for runner, arena in ((plain, arenas[0]), (graphed, arenas[1])):
+            arena.fill_(0xFF)
+            for g in runner.grads:
+                g.fill_(float("nan"))
+            rep = ck.train_step(runner.chain, mask, ck.POLICY_DYNAMIC, xb, lab, runner.params, runner.grads, arena, runner.workspace)
+            torch.cuda.synchronize()
+            out.append((rep, [g.detach().cpu().numpy().copy() for g in runner.grads]))
+        (rep_a, g_a), (rep_b, g_b) = out
+        replayed.append(rep_b["replayed"])
+        assert rep_a["replayed"] == 0
+        for key in ("peak_bytes", "extent_bytes", "predicted_bytes", "launches", "recomputed_units", "loss", "device_status"):
+            assert rep_a[key] == rep_b[key], (step, key)
+        for a, b in zip(g_a, g_b):
+            assert np.array_equal(a, b)
+    assert replayed == [0, 1, 1, 1, 1]
+    # another plan is another recording; switching the feature off drops them
+    mask2 = ck.mask_from_set(plain.n, [0, plain.n])
+    arena2 = torch.empty(ck.eval(ck.MODEL_DYNAMIC, plain.d, mask2), dtype=torch.uint8, device="cuda")
+    seq = [ck.train_step(graphed.chain, mask2, ck.POLICY_DYNAMIC, xb, lab, graphed.params, graphed.grads, arena2, graphed.workspace)["replayed"]
+           for _ in range(3)]
+    assert seq == [0, 1, 1]
+    g_two = [g.detach().cpu().numpy().copy() for g in graphed.grads]
+    graphed.chain.set_graph(False)
+    rep = ck.train_step(graphed.chain, mask2, ck.POLICY_DYNAMIC, xb, lab, graphed.params, graphed.grads, arena2, graphed.workspace)
+    torch.cuda.synchronize()
+    assert rep["replayed"] == 0
+    for a, b in zip(g_two, graphed.grads):
+        assert np.array_equal(a, b.detach().cpu().numpy())
