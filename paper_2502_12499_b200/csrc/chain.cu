@@ -298,11 +298,16 @@ static int unit_forward(StepCtx& c, int64_t i, const void* x_raw, void* y) {
 
 // Turns dL/d(activated d_j) into dL/d(d_j) in place when d_j carries a pending normalisation, and
 // writes the gradients of that normalisation's scale and shift.
-static int through_pending_act(StepCtx& c, int64_t j, const void* d_j, void* g) {
+// sum_blocks > 0: the kernel that wrote g has already left that many partial row pairs of the backward sums
+// in the scratch region.
+static int through_pending_act(StepCtx& c, int64_t j, const void* d_j, void* g, int sum_blocks = 0) {
     if (!pending_act(c.ch, j)) return CKPT_OK;
     const Unit& uj = c.ch->units[j - 1];
     void* const* p = c.params + uj.param_first;
     void* const* gr = c.grads + uj.param_first;
+    if (sum_blocks > 0)
+        return bn_relu_backward_from_partials(c.ch->dtype, rows_of(c.ch, j), uj.out.c, g, d_j, stats_of(c, j), 1, g,
+                                              (float*)gr[1], (float*)gr[2], c.ws + c.ch->off_scr, sum_blocks, c.stream);
     return bn_relu_backward(c.ch->dtype, rows_of(c.ch, j), uj.out.c, g, d_j, (const float*)p[1], stats_of(c, j), 1, g,
                             (float*)gr[1], (float*)gr[2], c.ws + c.ch->off_scr, c.stream);
 }
@@ -315,7 +320,7 @@ static int unit_backward(StepCtx& c, int64_t i, const void* x_raw, const void* y
     void* const* p = c.params + u.param_first;
     void* const* g = c.grads + u.param_first;
     const void* x = x_raw;
-    int rc;
+    int rc, sum_blocks = 0;
     switch (u.desc.kind) {
         case CKPT_UNIT_CONV_BN_RELU:
             if ((rc = activated(c, i - 1, x_raw, &x))) return rc;
@@ -344,7 +349,7 @@ static int unit_backward(StepCtx& c, int64_t i, const void* x_raw, const void* y
                 else if ((rc = activated(c, i - 1, x_raw, &x))) return rc;
             }
             if ((rc = maxpool_backward(dt, (int)c.ch->batch, u.in.h, u.in.w, u.in.c, u.desc.k, u.desc.stride, u.desc.pad, x, g_in,
-                                       g_out, act, c.stream))) return rc;
+                                       g_out, act, c.stream, act ? (float*)(c.ws + c.ch->off_scr) : nullptr, &sum_blocks))) return rc;
             break;
         }
         case CKPT_UNIT_AVGPOOL:
@@ -370,7 +375,7 @@ static int unit_backward(StepCtx& c, int64_t i, const void* x_raw, const void* y
             return CKPT_E_UNSUPPORTED;
     }
     // the producer of d_{i-1} may have left its normalisation pending: finish the chain rule through it
-    if (g_out) return through_pending_act(c, i - 1, x_raw, g_out);
+    if (g_out) return through_pending_act(c, i - 1, x_raw, g_out, sum_blocks);
     return CKPT_OK;
 }
 

@@ -126,8 +126,13 @@ int add_tensors(int dtype, int64_t elems, const void* a, const void* b, void* ou
 bool maxpool_fuses_activation(int dtype, int h, int w, int c, int k, int stride, int pad);
 int maxpool_forward(int dtype, int n, int h, int w, int c, int k, int stride, int pad, const void* x,
                     void* y, const float* act, void* stream);
+// bn_partial / bn_blocks (optional, with act): the 2x2 kernel also leaves the producer's batch-norm backward
+// sums there ([*bn_blocks][sum g | sum g*z][c] floats; *bn_blocks = 0 when it did not)
 int maxpool_backward(int dtype, int n, int h, int w, int c, int k, int stride, int pad, const void* x,
-                     const void* dy, void* dx, const float* act, void* stream);
+                     const void* dy, void* dx, const float* act, void* stream, float* bn_partial = nullptr,
+                     int* bn_blocks = nullptr);
+int bn_relu_backward_from_partials(int dtype, int64_t rows, int c, const void* dy, const void* z, const float* stats, int relu,
+                                   void* dz, float* dgamma, float* dbeta, void* scratch, int blocks, void* stream);
 int avgpool_forward(int dtype, int n, int h, int w, int c, const void* x, void* y, void* stream);
 int avgpool_backward(int dtype, int n, int h, int w, int c, const void* dy, void* dx, void* stream);
 

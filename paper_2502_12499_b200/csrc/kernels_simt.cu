@@ -903,6 +903,34 @@ int bn_relu_backward(int dtype, int64_t rows, int c, const void* dy, const void*
                     : bn_backward_t<float, 1>(rows, c, dy, z, stats, relu, dz, dgamma, dbeta, scratch, st);
 }
 
+// Batch-norm backward whose per-channel sums (sum g, sum g*z over `blocks` partial row pairs at the start of
+// `scratch`) were left by the kernel that produced dy: finalize and apply only.
+template <typename T, int VEC>
+static int bn_backward_tail_t(int64_t rows, int c, const void* dy, const void* z, const float* stats, int relu, void* dz,
+                              float* dgamma, float* dbeta, void* scratch, int blocks, cudaStream_t st) {
+    float* partial = (float*)scratch;
+    float* coef = partial + (size_t)BN_MAX_BLOCKS * c * 2;
+    bn_finalize_bwd_kernel<<<c, 32, 0, st>>>(partial, blocks, c, 1.0 / (double)rows, stats, dgamma, dbeta, coef);
+    CKPT_LAUNCH_CHECK("batch-norm backward finalize");
+    const int64_t vecs = rows * c / VEC;
+    const StreamGrid sg = stream_grid(vecs, 256, BN_BWD_U);
+    bn_bwd_apply_kernel<T, VEC><<<sg.blocks, 256, 0, st>>>((const T*)dy, (const T*)z, stats, coef, relu, vecs, c / VEC, c,
+                                                           sg.per_block, (T*)dz);
+    CKPT_LAUNCH_CHECK("batch-norm backward apply");
+    return CKPT_OK;
+}
+int bn_relu_backward_from_partials(int dtype, int64_t rows, int c, const void* dy, const void* z, const float* stats, int relu,
+                                   void* dz, float* dgamma, float* dbeta, void* scratch, int blocks, void* stream) {
+    cudaStream_t st = (cudaStream_t)stream;
+    if (blocks < 1 || blocks > BN_MAX_BLOCKS) { set_error("batch-norm backward: %d partial rows", blocks); return CKPT_E_BAD_ARG; }
+    int vec = bn_vec(dtype, c);
+    if (dtype == CKPT_DTYPE_BF16)
+        return vec == 8 ? bn_backward_tail_t<__nv_bfloat16, 8>(rows, c, dy, z, stats, relu, dz, dgamma, dbeta, scratch, blocks, st)
+                        : bn_backward_tail_t<__nv_bfloat16, 1>(rows, c, dy, z, stats, relu, dz, dgamma, dbeta, scratch, blocks, st);
+    return vec == 4 ? bn_backward_tail_t<float, 4>(rows, c, dy, z, stats, relu, dz, dgamma, dbeta, scratch, blocks, st)
+                    : bn_backward_tail_t<float, 1>(rows, c, dy, z, stats, relu, dz, dgamma, dbeta, scratch, blocks, st);
+}
+
 // ================================================================================================
 // Pooling
 // ================================================================================================
@@ -1035,6 +1063,74 @@ __global__ void __launch_bounds__(256) maxpool2x2_bwd_kernel(const T* __restrict
     }
 }
 
+// The same backward with the batch-norm backward sums of the producer gathered on the way: the window's
+// four raw values z and their gradients g = dx masked by the producer's ReLU are all in registers, so
+// sum g and sum g*z per channel (what bn_partial_stream_kernel<.., 1> would re-read both tensors for) come
+// for free.  Every thread keeps one channel group (grid stride a multiple of the group count); partial
+// rows [block][sum | sum g*z][c] in a fixed order.
+template <typename T, int VEC>
+__global__ void __launch_bounds__(256) maxpool2x2_bwd_sums_kernel(const T* __restrict__ x, const T* __restrict__ dy, T* __restrict__ dx,
+                                                                  int64_t items, int wo, int ho, int cv, int c,
+                                                                  const float* __restrict__ act, float* __restrict__ partial) {
+    __shared__ float red[256][2 * VEC + 1];
+    const int cg = (int)(((int64_t)blockIdx.x * 256 + threadIdx.x) % cv);
+    float sc[VEC], sh[VEC], s0[VEC], s1[VEC];
+#pragma unroll
+    for (int k = 0; k < VEC; ++k) { sc[k] = act[2 * c + cg * VEC + k]; sh[k] = act[3 * c + cg * VEC + k]; s0[k] = 0.f; s1[k] = 0.f; }
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < items; i += (int64_t)gridDim.x * blockDim.x) {
+        int64_t t = i / cv;
+        const int ow = (int)(t % wo); t /= wo;
+        const int oh = (int)(t % ho);
+        const int64_t img = t / ho;
+        const int64_t off = ((img * (2 * ho) + 2 * oh) * (int64_t)(2 * wo) + 2 * ow) * c + cg * VEC;
+        const int64_t down = (int64_t)2 * wo * c;
+        float z[4][VEC], g[VEC], o[4][VEC];
+        load_vec<T, VEC>(x + off, z[0]);
+        load_vec<T, VEC>(x + off + c, z[1]);
+        load_vec<T, VEC>(x + off + down, z[2]);
+        load_vec<T, VEC>(x + off + down + c, z[3]);
+        load_vec<T, VEC>(dy + i * VEC, g);
+#pragma unroll
+        for (int k = 0; k < VEC; ++k) {
+            float a[4];
+#pragma unroll
+            for (int q = 0; q < 4; ++q) a[q] = (float)cvt<T>(fmaxf(fmaf(z[q][k], sc[k], sh[k]), 0.f));
+            const float m = fmaxf(fmaxf(a[0], a[1]), fmaxf(a[2], a[3]));
+            const bool ta = a[0] == m, tb = !ta && a[1] == m, td = !ta && !tb && a[2] == m, te = !ta && !tb && !td;
+            o[0][k] = ta ? g[k] : 0.f; o[1][k] = tb ? g[k] : 0.f; o[2][k] = td ? g[k] : 0.f; o[3][k] = te ? g[k] : 0.f;
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const float gi = a[q] > 0.f ? o[q][k] : 0.f;
+                s0[k] += gi;
+                s1[k] = fmaf(gi, z[q][k], s1[k]);
+            }
+        }
+        store_vec<T, VEC>(dx + off, o[0]);
+        store_vec<T, VEC>(dx + off + c, o[1]);
+        store_vec<T, VEC>(dx + off + down, o[2]);
+        store_vec<T, VEC>(dx + off + down + c, o[3]);
+    }
+#pragma unroll
+    for (int k = 0; k < VEC; ++k) { red[threadIdx.x][k] = s0[k]; red[threadIdx.x][VEC + k] = s1[k]; }
+    __syncthreads();
+    // halving down to one row per channel group: threads t and t + off hold the same group (off a multiple of cv)
+    for (int off = 128; off >= cv; off >>= 1) {
+        if ((int)threadIdx.x < off) {
+#pragma unroll
+            for (int k = 0; k < 2 * VEC; ++k) red[threadIdx.x][k] += red[threadIdx.x + off][k];
+        }
+        __syncthreads();
+    }
+    if ((int)threadIdx.x < cv) {
+        const int chn = (int)(((int64_t)blockIdx.x * 256 + threadIdx.x) % cv) * VEC;
+#pragma unroll
+        for (int k = 0; k < VEC; ++k) {
+            partial[((size_t)blockIdx.x * 2 + 0) * c + chn + k] = red[threadIdx.x][k];
+            partial[((size_t)blockIdx.x * 2 + 1) * c + chn + k] = red[threadIdx.x][VEC + k];
+        }
+    }
+}
+
 bool maxpool_fuses_activation(int dtype, int h, int w, int c, int k, int stride, int pad) {
     const int vec = dtype == CKPT_DTYPE_BF16 ? 8 : 4;
     return k == 2 && stride == 2 && pad == 0 && h % 2 == 0 && w % 2 == 0 && c % vec == 0;
@@ -1149,11 +1245,25 @@ int maxpool_forward(int dtype, int n, int h, int w, int c, int k, int stride, in
     return CKPT_OK;
 }
 
-int maxpool_backward(int dtype, int n, int h, int w, int c, int k, int stride, int pad, const void* x, const void* dy, void* dx, const float* act, void* stream) {
+int maxpool_backward(int dtype, int n, int h, int w, int c, int k, int stride, int pad, const void* x, const void* dy, void* dx, const float* act, void* stream,
+                     float* bn_partial, int* bn_blocks) {
     int ho = (h + 2 * pad - k) / stride + 1, wo = (w + 2 * pad - k) / stride + 1;
+    if (bn_blocks) *bn_blocks = 0;
     if (maxpool_fuses_activation(dtype, h, w, c, k, stride, pad)) {
         const int vec = dtype == CKPT_DTYPE_BF16 ? 8 : 4;
         const int64_t items = (int64_t)n * ho * wo * (c / vec);
+        const int cv = c / vec;
+        if (act && bn_partial && bn_blocks && cv <= 128 && 256 % cv == 0) {
+            // the producer's batch-norm backward sums come out of this pass (one partial row pair per block)
+            const unsigned grid = (unsigned)std::max<int64_t>(1, std::min<int64_t>((items + 255) / 256, BN_MAX_BLOCKS));
+            if (dtype == CKPT_DTYPE_BF16)
+                maxpool2x2_bwd_sums_kernel<__nv_bfloat16, 8><<<grid, 256, 0, (cudaStream_t)stream>>>((const __nv_bfloat16*)x, (const __nv_bfloat16*)dy, (__nv_bfloat16*)dx, items, wo, ho, cv, c, act, bn_partial);
+            else
+                maxpool2x2_bwd_sums_kernel<float, 4><<<grid, 256, 0, (cudaStream_t)stream>>>((const float*)x, (const float*)dy, (float*)dx, items, wo, ho, cv, c, act, bn_partial);
+            CKPT_LAUNCH_CHECK("max-pool 2x2 backward with batch-norm sums");
+            *bn_blocks = (int)grid;
+            return CKPT_OK;
+        }
         if (dtype == CKPT_DTYPE_BF16)
             maxpool2x2_bwd_kernel<__nv_bfloat16, 8><<<elementwise_grid(items), 256, 0, (cudaStream_t)stream>>>((const __nv_bfloat16*)x, (const __nv_bfloat16*)dy, (__nv_bfloat16*)dx, items, wo, ho, c / vec, c, act);
         else
