@@ -1163,7 +1163,16 @@ constexpr int kFirstThreads = 288;
 #endif
 constexpr int kFirstCtasPerSm = FIRST_CTAS;      // each holds 128 of the 512 tensor-memory columns
 
-constexpr uint32_t kFirstSmem = 2 * 16384 + 8192 + 2 * 16384 + 1024;   // operand tiles, filter tile, output tiles, alignment
+constexpr int kFirstSegBytes = 832;                 // one staged input row segment: 130 pixels x 6 bytes plus alignment slack
+constexpr int kFirstSegChunks = kFirstSegBytes / 16;
+// operand tiles, filter tile, output tile, two sets of three staged row segments, alignment: three CTAs fit an SM
+constexpr uint32_t kFirstSmem = 2 * 16384 + 8192 + 16384 + 2 * 3 * kFirstSegBytes + 1024;
+
+__device__ __forceinline__ void cp_async_16(uint32_t dst, const void* src, int src_bytes) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N> __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
 
 __global__ void __launch_bounds__(kFirstThreads, kFirstCtasPerSm)
 tc_conv_first_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __restrict__ w,
@@ -1172,7 +1181,8 @@ tc_conv_first_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* _
     uint8_t* const smem_al = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
     uint8_t (*a_tiles)[128 * 128] = reinterpret_cast<uint8_t (*)[128 * 128]>(smem_al);
     uint8_t* const b_tile = smem_al + 2 * 16384;
-    uint8_t (*o_tiles)[128 * 128] = reinterpret_cast<uint8_t (*)[128 * 128]>(smem_al + 2 * 16384 + 8192);
+    uint8_t* const o_tile = smem_al + 2 * 16384 + 8192;
+    uint8_t* const stage = o_tile + 16384;               // [2][3][kFirstSegBytes]
     __shared__ float stat_red[4][2][64];
     __shared__ __align__(8) uint64_t bar_mem[8];
     __shared__ uint32_t tmem_base_slot;
@@ -1217,48 +1227,67 @@ tc_conv_first_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* _
     const uint32_t tmem_base = tmem_base_slot;
 
     if (warp < 4) {
-        // ---------------- gather: thread t builds row t of the operand tile
+        // ---------------- gather: thread t builds row t of the operand tile.  The 128 pixels of a tile are
+        // consecutive in memory, so the three input rows they touch are three contiguous segments of 130
+        // pixels (pixel p - 1 .. p + 128 of the rows above, at and below): the warps copy them to shared
+        // memory with 16-byte asynchronous copies one tile ahead and pick their 27 values from there.
         const int t = threadIdx.x;
-        const uint16_t* x16 = reinterpret_cast<const uint16_t*>(x);
-        auto gather = [&](int j, uint16_t (&v)[32]) {
-            const long long pix = ((long long)blockIdx.x + (long long)j * gridDim.x) * 128 + t;
+        const long long total_bytes = p.pixels * 6;
+        auto seg_start = [&](long long p0, int r) { return (p0 + (long long)(r - 1) * p.W - 1) * 6; };   // byte offset, may be < 0
+        auto issue = [&](int j) {
+            if (j < my_tiles) {
+                const long long p0 = ((long long)blockIdx.x + (long long)j * gridDim.x) * 128;
+                for (int idx = t; idx < 3 * kFirstSegChunks; idx += 128) {
+                    const int r = idx / kFirstSegChunks, ch = idx % kFirstSegChunks;
+                    const long long b = (seg_start(p0, r) & ~15LL) + ch * 16;
+                    if (b >= 0 && b < total_bytes)
+                        cp_async_16(smem_u32(stage + ((j & 1) * 3 + r) * kFirstSegBytes + ch * 16), reinterpret_cast<const char*>(x) + b,
+                                    (int)min(16LL, total_bytes - b));
+                }
+            }
+            cp_async_commit();
+        };
+        issue(0);
+        bool dead = false;          // after a failed wait the thread keeps walking the barriers, without work
+        for (int j = 0; j < my_tiles; ++j) {
+            const int buf = j & 1;
+            asm volatile("bar.sync 2, 128;" ::: "memory");      // every thread has left the segments of tile j - 1
+            issue(j + 1);
+            cp_async_wait<1>();
+            asm volatile("bar.sync 2, 128;" ::: "memory");      // the segments of tile j are complete
+            const long long p0 = ((long long)blockIdx.x + (long long)j * gridDim.x) * 128;
+            const long long pix = p0 + t;
+            __align__(16) uint16_t v[32];
 #pragma unroll
             for (int e = 0; e < 32; ++e) v[e] = 0;
-            if (j < my_tiles && pix < p.pixels) {
+            if (pix < p.pixels) {
                 const int ow = (int)(pix % p.W);
                 const int oh = (int)((pix / p.W) % p.H);
-                const long long img = pix / ((long long)p.W * p.H);
 #pragma unroll
                 for (int r = 0; r < 3; ++r) {
                     const int ih = oh + r - 1;
                     if (ih < 0 || ih >= p.H) continue;
-                    const uint16_t* row = x16 + ((img * p.H + ih) * p.W + ow) * 3;
+                    const uint8_t* seg = stage + (buf * 3 + r) * kFirstSegBytes + (int)(seg_start(p0, r) & 15LL);
 #pragma unroll
                     for (int s2 = 0; s2 < 3; ++s2) {
                         const int iw = ow + s2 - 1;
                         if (iw < 0 || iw >= p.W) continue;
 #pragma unroll
-                        for (int c = 0; c < 3; ++c) v[(r * 3 + s2) * 3 + c] = __ldg(row + (s2 - 1) * 3 + c);
+                        for (int c = 0; c < 3; ++c)
+                            v[(r * 3 + s2) * 3 + c] = *reinterpret_cast<const uint16_t*>(seg + ((t + s2) * 3 + c) * 2);
                     }
                 }
             }
-        };
-        // the loads of tile j+1 are in flight while tile j is written to shared memory
-        __align__(16) uint16_t cur[32], nxt[32];
-        gather(0, cur);
-        for (int j = 0; j < my_tiles; ++j) {
-            const int buf = j & 1;
-            gather(j + 1, nxt);
-            if (!mbar_wait(a_empty0 + 8 * buf, ((uint32_t)(j >> 1) & 1u) ^ 1u, failed, status, 601)) break;
+            if (!dead && !mbar_wait(a_empty0 + 8 * buf, ((uint32_t)(j >> 1) & 1u) ^ 1u, failed, status, 601)) dead = true;
+            if (dead) continue;
             uint8_t* dst = a_tiles[buf] + t * 128;
 #pragma unroll
             for (int chunk = 0; chunk < 4; ++chunk)
-                *reinterpret_cast<uint4*>(dst + ((chunk ^ (t & 7)) * 16)) = reinterpret_cast<const uint4*>(cur)[chunk];
+                *reinterpret_cast<uint4*>(dst + ((chunk ^ (t & 7)) * 16)) = reinterpret_cast<const uint4*>(v)[chunk];
             fence_proxy_async();
             mbar_arrive(a_full0 + 8 * buf);
-#pragma unroll
-            for (int e = 0; e < 32; ++e) cur[e] = nxt[e];
         }
+        cp_async_wait<0>();
     } else if (warp == 4) {
         if (lane == 0) {
             const uint32_t idesc = instr_desc(128, 64, 0, 0);
@@ -1289,11 +1318,11 @@ tc_conv_first_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* _
             const int buf = j & 1;
             if (!mbar_wait(acc_full0 + 8 * buf, (uint32_t)(j >> 1) & 1u, failed, status, 604)) break;
             tc_fence_after();
-            if (lane == 0) tma_store_wait_read<1>();          // the store that last read this output tile has left it
+            if (lane == 0) tma_store_wait_read<0>();          // the store of the previous tile has left this warp's slab
             __syncwarp();
             const long long pix0 = ((long long)blockIdx.x + (long long)j * gridDim.x) * 128;
             const bool valid = pix0 + row < p.pixels;
-            uint8_t* const orow = o_tiles[buf] + row * 128;
+            uint8_t* const orow = o_tile + row * 128;
 #pragma unroll
             for (int c0 = 0; c0 < 64; c0 += 32) {
                 uint32_t v[32];
@@ -1325,7 +1354,7 @@ tc_conv_first_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* _
             fence_proxy_async();
             __syncwarp();
             if (lane == 0 && pix0 + quarter * 32 < p.pixels) {
-                tma_store_2d(&map_out, smem_u32(o_tiles[buf]) + (uint32_t)(quarter * 4096), co0, (int)(pix0 + quarter * 32));
+                tma_store_2d(&map_out, smem_u32(o_tile) + (uint32_t)(quarter * 4096), co0, (int)(pix0 + quarter * 32));
                 tma_store_commit();
             }
         }
@@ -1732,6 +1761,11 @@ int tc_first_conv_fwd(const ConvGeom& g, const void* x, const void* w, void* z, 
     int sms = 148, dev = 0;
     cudaGetDevice(&dev);
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    if (reinterpret_cast<uintptr_t>(x) & 15u) {
+        // the staged row segments are copied in 16-byte pieces: an input that is not 16-byte aligned takes the CUDA-core kernel
+        if (blocks) *blocks = 0;
+        return small_conv_fwd(g, x, w, z, stream);
+    }
     CUtensorMap map_out;
     int rc = make_mat_map(&map_out, z, p.pixels, g.cout, 32);
     if (rc) return rc;
