@@ -1385,6 +1385,127 @@ tc_conv_first_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* _
     }
 }
 
+// ------------------------------------------------------------------------------------------------
+// Fully connected forward for small batches: out[b][co] = sum_k x[b][k] * W[co][k].  With the batch on M a
+// tile would be mostly padding and every CTA would re-read the activations; here the matrix is the M
+// operand (128 output features x 64 inputs per stage, each element fetched once from HBM), the batch is N,
+// and the long reduction is split over gridDim.y CTAs whose partial sums (float32, [slice][b][co]) are
+// added in a fixed order by fc_reduce_kernel together with bias, ReLU and the rounding.
+// ------------------------------------------------------------------------------------------------
+struct FcParams {
+    int batch, c_in, c_out;
+    int bnb;                     // batch rounded up to a multiple of 16 (the MMA's N)
+    int k_blocks, blocks_per_slice;
+    int stages;
+};
+
+__global__ void __launch_bounds__(kThreads, 1)
+tc_fc_fwd_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_x, float* __restrict__ partial,
+                 FcParams p, int* status) {
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    const uint32_t a_bytes = 128 * 128, b_bytes = (uint32_t)p.bnb * 128, stage_bytes = a_bytes + ((b_bytes + 1023u) & ~1023u);
+    const uint32_t bars = base + (uint32_t)p.stages * stage_bytes;
+    __shared__ uint32_t tmem_base_slot;
+    __shared__ int failed_flag;
+    volatile int* failed = &failed_flag;
+    const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
+    const int m_tile = blockIdx.x, slice = blockIdx.y;
+    const int kb_begin = slice * p.blocks_per_slice;
+    const int iters = max(0, min(p.k_blocks, kb_begin + p.blocks_per_slice) - kb_begin);
+    const uint32_t tmem_cols = p.bnb <= 32 ? 32 : (p.bnb <= 64 ? 64 : (p.bnb <= 128 ? 128 : 256));
+    auto full_bar = [&](int s) { return bars + 8u * s; };
+    auto empty_bar = [&](int s) { return bars + 8u * (kMaxStages + s); };
+    const uint32_t accum_bar = bars + 8u * (2 * kMaxStages);
+
+    if (threadIdx.x == 0) {
+        failed_flag = 0;
+        for (int s = 0; s < p.stages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+        mbar_init(accum_bar, 1);
+        fence_barrier_init();
+        tma_prefetch_desc(&map_w);
+        tma_prefetch_desc(&map_x);
+    }
+    if (warp == 1) tmem_alloc(smem_u32(&tmem_base_slot), tmem_cols);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = tmem_base_slot;
+
+    if (warp == 0 && lane == 0) {
+        int issued = 0;
+        for (int it = 0; it < iters; ++it) {
+            const int s = it % p.stages;
+            if (!mbar_wait(empty_bar(s), ((uint32_t)(it / p.stages) & 1u) ^ 1u, failed, status, 701)) break;
+            const uint32_t a_dst = base + (uint32_t)s * stage_bytes;
+            mbar_expect_tx(full_bar(s), a_bytes + b_bytes);
+            tma_load_2d(a_dst, &map_w, full_bar(s), (kb_begin + it) * 64, m_tile * 128);
+            tma_load_2d(a_dst + a_bytes, &map_x, full_bar(s), (kb_begin + it) * 64, 0);
+            issued = it + 1;
+        }
+        if (*failed) {
+            for (int it = max(0, issued - p.stages); it < issued; ++it)
+                mbar_drain(full_bar(it % p.stages), (uint32_t)(it / p.stages) & 1u);
+        }
+    } else if (warp == 1 && lane == 0) {
+        const uint32_t idesc = instr_desc(128, p.bnb, 0, 0);
+        bool ok = true;
+        for (int it = 0; it < iters && ok; ++it) {
+            const int s = it % p.stages;
+            if (!mbar_wait(full_bar(s), (uint32_t)(it / p.stages) & 1u, failed, status, 702)) { ok = false; break; }
+            tc_fence_after();
+            const uint32_t a_addr = base + (uint32_t)s * stage_bytes;
+            const uint32_t b_addr = a_addr + a_bytes;
+#pragma unroll
+            for (int kk = 0; kk < 4; ++kk)
+                umma_bf16(tmem_base, smem_desc(a_addr + kk * 32, 0, 1024), smem_desc(b_addr + kk * 32, 0, 1024), idesc,
+                          (it > 0 || kk > 0) ? 1u : 0u);
+            umma_commit(empty_bar(s));
+        }
+        if (ok) umma_commit(accum_bar);
+    } else if (warp >= 2) {
+        // thread = accumulator lane = output feature: consecutive lanes write consecutive floats of a row of [b][co]
+        const int quarter = warp % 4;
+        const int co = m_tile * 128 + quarter * 32 + lane;
+        float* dst = partial + (size_t)slice * p.batch * p.c_out + co;
+        const bool have = iters > 0 && mbar_wait(accum_bar, 0, failed, status, 703);
+        if (have) tc_fence_after();
+        for (int c0 = 0; c0 < p.bnb; c0 += 32) {
+            uint32_t v[32];
+            if (have && c0 + 32 <= (int)tmem_cols) {
+                tmem_ld32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)c0, v);
+            } else {
+#pragma unroll
+                for (int e = 0; e < 32; ++e) v[e] = 0u;
+            }
+            if (co < p.c_out && (have || iters == 0)) {
+#pragma unroll
+                for (int e = 0; e < 32; ++e)
+                    if (c0 + e < p.batch) dst[(size_t)(c0 + e) * p.c_out] = __uint_as_float(v[e]);
+            }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        __syncwarp();
+        tc_fence_after();
+        tmem_dealloc(tmem_base, tmem_cols);
+    }
+}
+
+// out[b][co] = round(act(bias[co] + sum over slices, in slice order))
+__global__ void fc_reduce_kernel(const float* __restrict__ partial, int slices, int64_t elems, int c_out, const float* __restrict__ bias,
+                                 int relu, __nv_bfloat16* __restrict__ out) {
+    const int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (e >= elems) return;
+    float sum = 0.f;
+    for (int z = 0; z < slices; ++z) sum += partial[(size_t)z * elems + e];
+    if (bias) sum += bias[e % c_out];
+    if (relu) sum = fmaxf(sum, 0.f);
+    out[e] = __float2bfloat16_rn(sum);
+}
+
 // wt[ci][tap'][co] = w[co][taps-1-tap'][ci]: the matrix of the transposed convolution (stride 1).
 __global__ void transpose_flip_kernel(const __nv_bfloat16* __restrict__ w, __nv_bfloat16* __restrict__ wt, int c_out, int taps, int c_in) {
     const int64_t total = (int64_t)c_out * taps * c_in;
@@ -1617,6 +1738,62 @@ int launch_fwd_like(const void* x, const void* w_mat, void* out, const float* bi
                           stat_blocks);
 }
 
+// Small-batch fully connected forward (see tc_fc_fwd_kernel): worth it when the matrix is large and the batch
+// fills at most one N tile.
+bool fc_applies(const ConvGeom& g) {
+    return g.h == 1 && g.w == 1 && g.k == 1 && g.stride == 1 && g.pad == 0 && g.n <= 256 && g.cin % 64 == 0 && g.cin >= 1024 &&
+           g.cout % 8 == 0;
+}
+void fc_plan(const ConvGeom& g, FcParams* p, int* m_tiles, int* slices) {
+    p->batch = g.n; p->c_in = g.cin; p->c_out = g.cout;
+    p->bnb = (g.n + 15) / 16 * 16;
+    p->k_blocks = g.cin / 64;
+    *m_tiles = (g.cout + 127) / 128;
+    int sms = 148, dev = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    // about two waves of CTAs, at least four 64-wide blocks of the reduction each
+    int want = std::max(1, std::min((2 * sms) / *m_tiles, p->k_blocks / 4));
+    p->blocks_per_slice = (p->k_blocks + want - 1) / want;
+    *slices = (p->k_blocks + p->blocks_per_slice - 1) / p->blocks_per_slice;
+    const uint32_t stage_bytes = 128 * 128 + (((uint32_t)p->bnb * 128 + 1023u) & ~1023u);
+    p->stages = std::min<int>(kMaxStages, kSmemBudget / stage_bytes);
+}
+int64_t fc_scratch_bytes(const ConvGeom& g) {
+    if (!fc_applies(g)) return 0;
+    FcParams p;
+    int m_tiles, slices;
+    fc_plan(g, &p, &m_tiles, &slices);
+    return (int64_t)slices * g.n * g.cout * 4;
+}
+int launch_fc(const ConvGeom& g, const void* x, const void* w, void* z, const float* bias, int relu, void* scratch, int* status,
+              cudaStream_t st) {
+    FcParams p;
+    int m_tiles, slices;
+    fc_plan(g, &p, &m_tiles, &slices);
+    CUtensorMap mw, mx;
+    int rc = make_mat_map(&mw, w, g.cout, g.cin, 128);
+    if (rc) return rc;
+    rc = make_mat_map(&mx, x, g.n, g.cin, p.bnb);
+    if (rc) return rc;
+    const uint32_t stage_bytes = 128 * 128 + (((uint32_t)p.bnb * 128 + 1023u) & ~1023u);
+    const size_t smem = (size_t)p.stages * stage_bytes + 1024 + 256;
+    static bool attr_set = false;
+    if (!attr_set) {
+        cudaError_t e = cudaFuncSetAttribute(tc_fc_fwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget + 2048);
+        if (e != cudaSuccess) return cuda_fail(e, "raising the shared-memory limit");
+        attr_set = true;
+    }
+    dim3 grid(m_tiles, slices);
+    tc_fc_fwd_kernel<<<grid, kThreads, smem, st>>>(mw, mx, (float*)scratch, p, status);
+    CKPT_LAUNCH_CHECK("fully connected forward (tensor cores)");
+    const int64_t elems = (int64_t)g.n * g.cout;
+    fc_reduce_kernel<<<(unsigned)((elems + 255) / 256), 256, 0, st>>>((const float*)scratch, slices, elems, g.cout, bias, relu,
+                                                                      (__nv_bfloat16*)z);
+    CKPT_LAUNCH_CHECK("fully connected slice sum");
+    return CKPT_OK;
+}
+
 void wgrad_plan(const ConvGeom& g, WgradParams* p, int* slices, int* groups, int* co_tiles) {
     p->H = g.ho; p->W = g.wo; p->N = g.n; p->c_out = g.cout; p->c_in = g.cin; p->k = g.k; p->pad = g.pad; p->stride = g.stride;
     choose_tile(64, g.wo, g.ho, g.n, &p->tw, &p->th, &p->tn);
@@ -1720,7 +1897,7 @@ static int64_t tc_conv_stat_bytes(const ConvGeom& g) {
 
 static int64_t tc_conv_work_bytes(const ConvGeom& g);
 int64_t tc_conv_scratch_bytes(const ConvGeom& g) {
-    return std::max(tc_conv_stat_bytes(g), tc_conv_work_bytes(g));
+    return std::max(std::max(tc_conv_stat_bytes(g), tc_conv_work_bytes(g)), fc_scratch_bytes(g));
 }
 
 // partial sums of the split weight gradient, or the transposed filter of the input gradient
@@ -1807,9 +1984,11 @@ int tc_conv_fwd_stats(const ConvGeom& g, const void* x, const void* w, void* z, 
                            "conv forward (tensor cores)", partial, blocks);
 }
 
-int tc_conv_fwd(const ConvGeom& g, const void* x, const void* w, void* z, const float* bias, int relu, void*, int64_t,
-                int* device_status, void* stream) {
+int tc_conv_fwd(const ConvGeom& g, const void* x, const void* w, void* z, const float* bias, int relu, void* scratch,
+                int64_t scratch_bytes, int* device_status, void* stream) {
     if (!device_status) { set_error("no status word"); return CKPT_E_NULL; }
+    if (fc_applies(g) && scratch && scratch_bytes >= fc_scratch_bytes(g))
+        return launch_fc(g, x, w, z, bias, relu, scratch, device_status, (cudaStream_t)stream);
     if (g.stride != 1) {
         if (bias || relu) { set_error("strided tensor-core conv has no bias/ReLU epilogue"); return CKPT_E_UNSUPPORTED; }
         return launch_strided_fwd(g, x, w, z, device_status, (cudaStream_t)stream);

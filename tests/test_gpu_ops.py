@@ -43,6 +43,9 @@ TC_CASES = [
     (5, 30, 30, 128, 64, 1, 0),
     (64, 1, 1, 512, 192, 1, 0),      # fully connected shape
     (48, 1, 1, 256, 1000, 1, 0),     # classifier: output channels not a multiple of 64
+    (64, 1, 1, 2048, 320, 1, 0),     # wide fully connected layer: matrix on M, batch on N, split reduction
+    (5, 1, 1, 1024, 1000, 1, 0),     # the same with a ragged batch and a ragged last tile of output features
+    (200, 1, 1, 4096, 128, 1, 0),    # batch wider than one 128-column accumulator chunk
     (2, 56, 56, 64, 64, 3, 1),
     (2, 16, 16, 128, 128, 3, 1),     # halo-patch kernel, one tile per CTA
     (2, 28, 24, 128, 256, 3, 1),     # halo-patch kernel, 14-row tiles, 256-wide output tile

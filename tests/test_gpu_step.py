@@ -147,6 +147,9 @@ def shallow_chains():
     s = dict(units=[{"kind": "fc", "cin": 2 * 2 * 64, "cout": 128, "relu": True}, {"kind": "fc", "cin": 128, "cout": 64, "relu": False}],
              input_hwc=(2, 2, 64), batch=24, dtype="bf16", loss="softmax_ce", name="fc+fc on tensor cores")
     yield s
+    s = dict(units=[{"kind": "fc", "cin": 4 * 4 * 128, "cout": 200, "relu": True}, {"kind": "fc", "cin": 200, "cout": 16, "relu": False}],
+             input_hwc=(4, 4, 128), batch=40, dtype="bf16", loss="softmax_ce", name="wide fc (matrix on M, split reduction)+fc")
+    yield s
     s = wl.plain_chain(2, 64, 64, (12, 12), 8, "bf16", "softmax_ce", name="conv64+conv64+fc")
     s["units"].append({"kind": "fc", "cin": 12 * 12 * 64, "cout": 10, "relu": False})
     yield s
