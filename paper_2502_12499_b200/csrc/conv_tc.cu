@@ -766,6 +766,7 @@ tc_conv_wgrad_kernel(const __grid_constant__ CUtensorMap map_dz, const __grid_co
     const uint32_t bars = base + (uint32_t)p.stages * stage_bytes;
     __shared__ uint32_t tmem_base_slot;
     __shared__ int failed_flag;
+    __shared__ float turn[4][32][33];                             // per epilogue warp: a 32 x 32 block on its way out
     volatile int* failed = &failed_flag;
 
     const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
@@ -844,24 +845,30 @@ tc_conv_wgrad_kernel(const __grid_constant__ CUtensorMap map_dz, const __grid_co
         }
         if (ok) umma_commit(accum_bar);
     } else if (warp >= 2) {
+        // Thread l of a warp holds row l of each 32 x 32 block; the block is turned through shared memory so
+        // that every store instruction writes 32 consecutive floats of one row (a full line) instead of 16-byte
+        // pieces of 32 rows: the fully connected gradients are hundreds of megabytes of such rows.
         const int quarter = warp % 4;
-        const int co = co_tile * 128 + quarter * 32 + lane;
+        const int co_first = co_tile * 128 + quarter * 32;
+        const int co = co_first + lane;
         const bool valid = co < p.c_out;
         const size_t row_elems = (size_t)p.k * p.k * p.c_in;
         float* dst_row = partial + ((size_t)slice * p.c_out + (valid ? co : 0)) * row_elems;
+        float* dst_first = partial + ((size_t)slice * p.c_out + co_first) * row_elems;
         if (iters > 0 && mbar_wait(accum_bar, 0, failed, status, 203)) {
             tc_fence_after();
             for (int j = 0; j < nb_here; ++j) {
-                float* dst = dst_row + (size_t)(blk_begin + j) * 64;     // column (tap, c_in) = block*64 + c
                 for (int c0 = 0; c0 < 64; c0 += 32) {
                     uint32_t v[32];
                     tmem_ld32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(j * 64 + c0), v);
-                    if (valid) {
+                    __syncwarp();
 #pragma unroll
-                        for (int e = 0; e < 8; ++e)
-                            *reinterpret_cast<float4*>(dst + c0 + 4 * e) =
-                                make_float4(__uint_as_float(v[4 * e]), __uint_as_float(v[4 * e + 1]), __uint_as_float(v[4 * e + 2]), __uint_as_float(v[4 * e + 3]));
-                    }
+                    for (int e = 0; e < 32; ++e) turn[quarter][lane][e] = __uint_as_float(v[e]);
+                    __syncwarp();
+                    float* dst = dst_first + (size_t)(blk_begin + j) * 64 + c0 + lane;     // column (tap, c_in) = block*64 + c
+#pragma unroll 8
+                    for (int r = 0; r < 32; ++r)
+                        if (co_first + r < p.c_out) dst[(size_t)r * row_elems] = turn[quarter][r][lane];
                 }
             }
         } else if (iters == 0 && valid) {
@@ -1802,6 +1809,8 @@ void wgrad_plan(const ConvGeom& g, WgradParams* p, int* slices, int* groups, int
     p->total_blocks = g.k * g.k * g.cin / 64;
     // column blocks per CTA: 4 when that divides evenly or the remainder is small, else 3
     p->nb = p->total_blocks % 4 == 0 ? 4 : (p->total_blocks % 3 == 0 ? 3 : (p->total_blocks >= 4 ? 4 : p->total_blocks));
+    // a reduction of one or two pixel tiles is all stores: narrower CTAs (128 accumulator columns) fit four to an SM
+    if (p->total_tiles <= 2 && p->total_blocks >= 2) p->nb = 2;
     *groups = (p->total_blocks + p->nb - 1) / p->nb;
     *co_tiles = (g.cout + 127) / 128;
     // slices of the pixel range: fill the SMs with whole waves of equally long CTAs (2 to 4 waves),
@@ -1823,7 +1832,9 @@ void wgrad_plan(const ConvGeom& g, WgradParams* p, int* slices, int* groups, int
     p->tiles_per_slice = (int)((p->total_tiles + s - 1) / s);
     *slices = (p->total_tiles + p->tiles_per_slice - 1) / p->tiles_per_slice;
     const uint32_t stage_bytes = (2 + p->nb) * 64 * 128;
-    p->stages = std::min<int>(kMaxStages, kSmemBudget / stage_bytes);
+    // no more stages than pixel tiles per CTA: a short reduction (fully connected layers: one tile) then leaves
+    // room for a second CTA on the SM, whose loads run under the first one's stores
+    p->stages = std::max(1, std::min<int>(std::min<int>(kMaxStages, kSmemBudget / stage_bytes), p->tiles_per_slice));
 }
 
 }  // namespace
