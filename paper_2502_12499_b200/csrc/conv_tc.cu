@@ -236,6 +236,7 @@ struct FwdParams {
     int tw, th, tn;              // pixel tile, tw*th*tn = 128
     int tiles_w, tiles_h, tiles_n;
     int bn, n_tiles;             // output-channel tile and their count
+    int m_tiles, ctas_per_n;     // pixel tiles, and the persistent CTAs that share one output-channel tile
     int stages;
 };
 
@@ -244,34 +245,39 @@ __global__ void __launch_bounds__(kThreads, 1)
 tc_conv_fwd_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w,
                    __nv_bfloat16* __restrict__ out, const float* __restrict__ bias, int relu, float* __restrict__ stat_partial,
                    FwdParams p, int* status) {
+    // Persistent: CTA (first, n_tile) walks the pixel tiles first, first + ctas_per_n, ... of its output-channel
+    // tile.  The operand ring runs on across tile boundaries and the accumulator is double-buffered in tensor
+    // memory (2 x bn columns), so the epilogue of one tile runs under the MMAs of the next.
     extern __shared__ uint8_t smem_raw[];
-    __shared__ float stat_red[4][2][256];        // per-quarter column sums of the tile (batch-norm statistics)
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const uint32_t a_bytes = 128 * 128, b_bytes = (uint32_t)p.bn * 128, stage_bytes = a_bytes + b_bytes;
-    const uint32_t bars = base + (uint32_t)p.stages * stage_bytes;           // full[s], empty[s], accum
+    const uint32_t bars = base + (uint32_t)p.stages * stage_bytes;           // full[s], empty[s], acc_full[2], acc_empty[2]
     __shared__ uint32_t tmem_base_slot;
     __shared__ int failed_flag;
     volatile int* failed = &failed_flag;
 
     const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
     const int n_tile = blockIdx.x % p.n_tiles;
-    int mt = blockIdx.x / p.n_tiles;
-    const int tile_w = mt % p.tiles_w; mt /= p.tiles_w;
-    const int tile_h = mt % p.tiles_h;
-    const int tile_n = mt / p.tiles_h;
-    const int w0 = tile_w * p.tw, h0 = tile_h * p.th, n0 = tile_n * p.tn;
+    const int first = blockIdx.x / p.n_tiles;
+    const int my_tiles = first < p.m_tiles ? (p.m_tiles - first + p.ctas_per_n - 1) / p.ctas_per_n : 0;
     const int blocks = (p.c_red + 63) / 64;      // a ragged last block is zero-filled by the TMA unit
     const int iters = p.taps * blocks;
-    const uint32_t tmem_cols = p.bn < 32 ? 32 : p.bn;
+    const uint32_t tmem_cols = 2 * p.bn <= 32 ? 32 : (2 * p.bn <= 64 ? 64 : (2 * p.bn <= 128 ? 128 : (2 * p.bn <= 256 ? 256 : 512)));
 
     auto full_bar = [&](int s) { return bars + 8u * s; };
     auto empty_bar = [&](int s) { return bars + 8u * (kMaxStages + s); };
-    const uint32_t accum_bar = bars + 8u * (2 * kMaxStages);
+    const uint32_t acc_full0 = bars + 8u * (2 * kMaxStages), acc_empty0 = acc_full0 + 16;
+    auto tile_origin = [&](int j, int& w0, int& h0, int& n0) {
+        int mt = first + j * p.ctas_per_n;
+        w0 = (mt % p.tiles_w) * p.tw; mt /= p.tiles_w;
+        h0 = (mt % p.tiles_h) * p.th;
+        n0 = (mt / p.tiles_h) * p.tn;
+    };
 
     if (threadIdx.x == 0) {
         failed_flag = 0;
         for (int s = 0; s < p.stages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
-        mbar_init(accum_bar, 1);
+        for (int b = 0; b < 2; ++b) { mbar_init(acc_full0 + 8 * b, 1); mbar_init(acc_empty0 + 8 * b, 128); }
         fence_barrier_init();
         tma_prefetch_desc(&map_x);
         tma_prefetch_desc(&map_w);
@@ -286,88 +292,89 @@ tc_conv_fwd_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_const
         // ---------------- TMA producer.  Filter as a [c_out][k*k*c_red] matrix: two copies per stage, measured
         // fastest from a single thread.  Filter read in place for a 1x1 dgrad (B_MN): the tile is bn/64 boxes of
         // 64 reduction channels x 64 output channels, one lane per copy, every lane watching the barrier.
-        int issued = 0;
-        for (int it = 0; it < iters; ++it) {
-            const int s = it % p.stages;
-            const uint32_t phase = (uint32_t)(it / p.stages) & 1u;
-            if (!mbar_wait(empty_bar(s), phase ^ 1u, failed, status, 101)) break;
-            const int tap = it / blocks, blk = it % blocks;
-            const uint32_t a_dst = base + (uint32_t)s * stage_bytes;
-            if (lane == 0) {
-                mbar_expect_tx(full_bar(s), stage_bytes);
-                tma_load_4d(a_dst, &map_x, full_bar(s), blk * 64, w0 * p.in_stride + p.tap_dw[tap], h0 * p.in_stride + p.tap_dh[tap], n0);
-                if (!B_MN) tma_load_2d(a_dst + a_bytes, &map_w, full_bar(s), p.tap_col[tap] * p.c_red + blk * 64, n_tile * p.bn);
+        int g = 0;                                   // stages issued so far (over all tiles)
+        bool ok = true;
+        for (int j = 0; j < my_tiles && ok; ++j) {
+            int w0, h0, n0;
+            tile_origin(j, w0, h0, n0);
+            for (int it = 0; it < iters; ++it, ++g) {
+                const int s = g % p.stages;
+                const uint32_t phase = (uint32_t)(g / p.stages) & 1u;
+                if (!mbar_wait(empty_bar(s), phase ^ 1u, failed, status, 101)) { ok = false; break; }
+                const int tap = it / blocks, blk = it % blocks;
+                const uint32_t a_dst = base + (uint32_t)s * stage_bytes;
+                if (lane == 0) {
+                    mbar_expect_tx(full_bar(s), stage_bytes);
+                    tma_load_4d(a_dst, &map_x, full_bar(s), blk * 64, w0 * p.in_stride + p.tap_dw[tap], h0 * p.in_stride + p.tap_dh[tap], n0);
+                    if (!B_MN) tma_load_2d(a_dst + a_bytes, &map_w, full_bar(s), p.tap_col[tap] * p.c_red + blk * 64, n_tile * p.bn);
+                }
+                if (B_MN) {
+                    __syncwarp();
+                    if (lane >= 1 && lane <= p.bn / 64)
+                        tma_load_2d(a_dst + a_bytes + (lane - 1) * 8192, &map_w, full_bar(s),
+                                    p.tap_col[tap] * p.c_out + n_tile * p.bn + (lane - 1) * 64, blk * 64);
+                }
             }
-            if (B_MN) {
-                __syncwarp();
-                if (lane >= 1 && lane <= p.bn / 64)
-                    tma_load_2d(a_dst + a_bytes + (lane - 1) * 8192, &map_w, full_bar(s),
-                                p.tap_col[tap] * p.c_out + n_tile * p.bn + (lane - 1) * 64, blk * 64);
-            }
-            issued = it + 1;
         }
         if (*failed && lane == 0) {
             // copies that were issued but never consumed must land before the CTA may exit
-            for (int it = max(0, issued - p.stages); it < issued; ++it)
-                mbar_drain(full_bar(it % p.stages), (uint32_t)(it / p.stages) & 1u);
+            for (int q = max(0, g - p.stages); q < g; ++q)
+                mbar_drain(full_bar(q % p.stages), (uint32_t)(q / p.stages) & 1u);
         }
     } else if (warp == 1 && lane == 0) {
         // ---------------- MMA issuer
         const uint32_t idesc = instr_desc(128, p.bn, 0, B_MN ? 1 : 0);
         constexpr uint32_t b_step = B_MN ? 2048u : 32u, b_lbo = B_MN ? 8192u : 0u;
         bool ok = true;
-        for (int it = 0; it < iters && ok; ++it) {
-            const int s = it % p.stages;
-            const uint32_t phase = (uint32_t)(it / p.stages) & 1u;
-            if (!mbar_wait(full_bar(s), phase, failed, status, 102)) { ok = false; break; }
-            tc_fence_after();
-            const uint32_t a_addr = base + (uint32_t)s * stage_bytes;
-            const uint32_t b_addr = a_addr + a_bytes;
+        int g = 0;
+        for (int j = 0; j < my_tiles && ok; ++j) {
+            const int buf = j & 1;
+            if (!mbar_wait(acc_empty0 + 8 * buf, ((uint32_t)(j >> 1) & 1u) ^ 1u, failed, status, 104)) { ok = false; break; }
+            const uint32_t acc = tmem_base + (uint32_t)(buf * p.bn);
+            for (int it = 0; it < iters; ++it, ++g) {
+                const int s = g % p.stages;
+                const uint32_t phase = (uint32_t)(g / p.stages) & 1u;
+                if (!mbar_wait(full_bar(s), phase, failed, status, 102)) { ok = false; break; }
+                tc_fence_after();
+                const uint32_t a_addr = base + (uint32_t)s * stage_bytes;
+                const uint32_t b_addr = a_addr + a_bytes;
 #pragma unroll
-            for (int kk = 0; kk < 4; ++kk) {        // 4 x (K = 16 bf16): 32 bytes along a row, or 16 rows when B_MN
-                umma_bf16(tmem_base, smem_desc(a_addr + kk * 32, 0, 1024), smem_desc(b_addr + kk * b_step, b_lbo, 1024), idesc,
-                          (it > 0 || kk > 0) ? 1u : 0u);
+                for (int kk = 0; kk < 4; ++kk) {        // 4 x (K = 16 bf16): 32 bytes along a row, or 16 rows when B_MN
+                    umma_bf16(acc, smem_desc(a_addr + kk * 32, 0, 1024), smem_desc(b_addr + kk * b_step, b_lbo, 1024), idesc,
+                              (it > 0 || kk > 0) ? 1u : 0u);
+                }
+                umma_commit(empty_bar(s));              // frees the stage when these MMAs have read it
             }
-            umma_commit(empty_bar(s));              // frees the stage when these MMAs have read it
+            if (ok) umma_commit(acc_full0 + 8 * buf);   // accumulator complete
         }
-        if (ok) umma_commit(accum_bar);             // accumulator complete
     } else if (warp >= 2) {
         // ---------------- epilogue: TMEM -> registers -> bf16 -> global
         const int quarter = warp % 4;               // a warp may only touch its own 32 TMEM lanes
         const int row = quarter * 32 + lane;
         const int wl = row % p.tw, hl = (row / p.tw) % p.th, nl = row / (p.tw * p.th);
-        const int oh = (h0 + hl) * p.out_stride + p.out_oh, ow = (w0 + wl) * p.out_stride + p.out_ow;
-        const bool valid = (w0 + wl < p.W) && (h0 + hl < p.H) && (n0 + nl < p.N) && oh < p.out_H && ow < p.out_W;
-        __nv_bfloat16* dst = out + ((((size_t)(n0 + nl) * p.out_H + oh) * p.out_W + ow) * p.c_out + (size_t)n_tile * p.bn);
-        if (stat_partial) {
-            // batch-norm sums of the stored tile: one partial row pair per pixel tile, the four quarters added
-            // in a fixed order (the caller guarantees whole 32-column chunks and no bias/ReLU)
-            if (mbar_wait(accum_bar, 0, failed, status, 103)) {
-                tc_fence_after();
-                for (int c0 = 0; c0 < p.bn; c0 += 32) {
-                    uint32_t v[32];
-                    tmem_ld32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)c0, v);
-                    float sum = 0.f, sumsq = 0.f;
-                    store_chunk(v, valid, dst + c0, true, lane, sum, sumsq);
-                    stat_red[quarter][0][c0 + lane] = sum;
-                    stat_red[quarter][1][c0 + lane] = sumsq;
-                }
-            } else {
-                for (int c0 = 0; c0 < p.bn; c0 += 32) { stat_red[quarter][0][c0 + lane] = 0.f; stat_red[quarter][1][c0 + lane] = 0.f; }
-            }
-            asm volatile("bar.sync 1, 128;" ::: "memory");
-            const size_t m_tile = blockIdx.x / p.n_tiles;
-            for (int col = quarter * 32 + lane; col < p.bn; col += 128) {
+        const bool stats = stat_partial != nullptr;   // the caller guarantees whole 32-column chunks and no bias/ReLU
+        float s_acc[8], q_acc[8];
 #pragma unroll
-                for (int k = 0; k < 2; ++k)
-                    stat_partial[(m_tile * 2 + k) * p.c_out + (size_t)n_tile * p.bn + col] =
-                        (stat_red[0][k][col] + stat_red[1][k][col]) + (stat_red[2][k][col] + stat_red[3][k][col]);
-            }
-        } else if (mbar_wait(accum_bar, 0, failed, status, 103)) {
+        for (int ci = 0; ci < 8; ++ci) { s_acc[ci] = 0.f; q_acc[ci] = 0.f; }
+        for (int j = 0; j < my_tiles; ++j) {
+            const int buf = j & 1;
+            if (!mbar_wait(acc_full0 + 8 * buf, (uint32_t)(j >> 1) & 1u, failed, status, 103)) break;
             tc_fence_after();
-            for (int c0 = 0; c0 < p.bn; c0 += 32) {
+            int w0, h0, n0;
+            tile_origin(j, w0, h0, n0);
+            const int oh = (h0 + hl) * p.out_stride + p.out_oh, ow = (w0 + wl) * p.out_stride + p.out_ow;
+            const bool valid = (w0 + wl < p.W) && (h0 + hl < p.H) && (n0 + nl < p.N) && oh < p.out_H && ow < p.out_W;
+            __nv_bfloat16* dst = out + ((((size_t)(n0 + nl) * p.out_H + oh) * p.out_W + ow) * p.c_out + (size_t)n_tile * p.bn);
+#pragma unroll
+            for (int ci = 0; ci < 8; ++ci) {
+                const int c0 = ci * 32;
+                if (c0 >= p.bn) break;
                 uint32_t v[32];
-                tmem_ld32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)c0, v);
+                tmem_ld32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * p.bn + c0), v);
+                if (stats) {
+                    store_chunk(v, valid, dst + c0, true, lane, s_acc[ci], q_acc[ci]);
+                    continue;
+                }
                 const int col0 = n_tile * p.bn + c0;          // first output channel of this chunk
                 if (valid && col0 < p.c_out) {
                     if (bias) {
@@ -380,14 +387,28 @@ tc_conv_fwd_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_const
                         for (int e = 0; e < 32; ++e) v[e] = __float_as_uint(fmaxf(__uint_as_float(v[e]), 0.f));
                     }
 #pragma unroll
-                    for (int j = 0; j < 4; ++j) {
+                    for (int q = 0; q < 4; ++q) {
                         uint4 pk;
                         __nv_bfloat162* h = reinterpret_cast<__nv_bfloat162*>(&pk);
 #pragma unroll
                         for (int e = 0; e < 4; ++e)
-                            h[e] = __floats2bfloat162_rn(__uint_as_float(v[8 * j + 2 * e]), __uint_as_float(v[8 * j + 2 * e + 1]));
-                        if (col0 + 8 * j + 8 <= p.c_out) *reinterpret_cast<uint4*>(dst + c0 + 8 * j) = pk;
+                            h[e] = __floats2bfloat162_rn(__uint_as_float(v[8 * q + 2 * e]), __uint_as_float(v[8 * q + 2 * e + 1]));
+                        if (col0 + 8 * q + 8 <= p.c_out) *reinterpret_cast<uint4*>(dst + c0 + 8 * q) = pk;
                     }
+                }
+            }
+            tc_fence_before();
+            mbar_arrive(acc_empty0 + 8 * buf);
+        }
+        if (stats) {
+            // one block of partial sums per epilogue warp: [block][sum | sum of squares][channel]
+            const size_t blk = (size_t)first * 4 + quarter;
+#pragma unroll
+            for (int ci = 0; ci < 8; ++ci) {
+                if (ci * 32 < p.bn) {
+                    const int ch = n_tile * p.bn + ci * 32 + lane;
+                    stat_partial[(blk * 2) * p.c_out + ch] = s_acc[ci];
+                    stat_partial[(blk * 2 + 1) * p.c_out + ch] = q_acc[ci];
                 }
             }
         }
@@ -1681,7 +1702,8 @@ int launch_halo(const void* x, const void* w_mat, void* out, float* stat_partial
 int64_t generic_stat_rows(int n, int gh, int gw) {
     int tw, th, tn;
     choose_tile(128, gw, gh, n, &tw, &th, &tn);
-    return (int64_t)((gw + tw - 1) / tw) * ((gh + th - 1) / th) * ((n + tn - 1) / tn);
+    const int64_t m_tiles = (int64_t)((gw + tw - 1) / tw) * ((gh + th - 1) / th) * ((n + tn - 1) / tn);
+    return 4 * std::min<int64_t>(m_tiles, 256);      // one row pair per epilogue warp of each persistent CTA (at most one CTA per SM)
 }
 
 int launch_generic(FwdParams p, const void* a, int a_n, int a_h, int a_w, const void* w_mat, int taps_total, void* out,
@@ -1712,10 +1734,15 @@ int launch_generic(FwdParams p, const void* a, int a_n, int a_h, int a_w, const 
         if (e != cudaSuccess) return cuda_fail(e, "raising the shared-memory limit");
         attr_set = true;
     }
-    const int64_t ctas = (int64_t)p.tiles_w * p.tiles_h * p.tiles_n * p.n_tiles;
+    p.m_tiles = p.tiles_w * p.tiles_h * p.tiles_n;
+    int sms = 148, dev = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    p.ctas_per_n = std::max(1, std::min(p.m_tiles, sms / p.n_tiles));
+    const int64_t ctas = (int64_t)p.ctas_per_n * p.n_tiles;
     // statistics in the epilogue: whole 32-column chunks, plain stores, output written once per pixel
     const bool gather = stat_partial && stat_blocks && !bias && !relu && !b_mn && c_out % 64 == 0 && p.bn >= 32 && p.out_stride == 1;
-    if (gather) *stat_blocks = (int)(ctas / p.n_tiles);
+    if (gather) *stat_blocks = 4 * p.ctas_per_n;
     if (b_mn) tc_conv_fwd_kernel<true><<<(unsigned)ctas, kThreads, smem, st>>>(mx, mw, (__nv_bfloat16*)out, bias, relu, nullptr, p, status);
     else tc_conv_fwd_kernel<false><<<(unsigned)ctas, kThreads, smem, st>>>(mx, mw, (__nv_bfloat16*)out, bias, relu, gather ? stat_partial : nullptr, p, status);
     CKPT_LAUNCH_CHECK(what);
