@@ -1741,7 +1741,10 @@ int launch_generic(FwdParams p, const void* a, int a_n, int a_h, int a_w, const 
     p.ctas_per_n = std::max(1, std::min(p.m_tiles, sms / p.n_tiles));
     const int64_t ctas = (int64_t)p.ctas_per_n * p.n_tiles;
     // statistics in the epilogue: whole 32-column chunks, plain stores, output written once per pixel
-    const bool gather = stat_partial && stat_blocks && !bias && !relu && !b_mn && c_out % 64 == 0 && p.bn >= 32 && p.out_stride == 1;
+    // (a short reduction cannot hide the column sums behind its MMAs: a 64 -> 256 1x1 layer took 172 us with them
+    // against 78 us without, more than the separate pass over the output costs; from 16 stages per tile on they are free)
+    const bool gather = stat_partial && stat_blocks && !bias && !relu && !b_mn && c_out % 64 == 0 && p.bn >= 32 && p.out_stride == 1 &&
+                        p.taps * ((c_red + 63) / 64) >= 16;
     if (gather) *stat_blocks = 4 * p.ctas_per_n;
     if (b_mn) tc_conv_fwd_kernel<true><<<(unsigned)ctas, kThreads, smem, st>>>(mx, mw, (__nv_bfloat16*)out, bias, relu, nullptr, p, status);
     else tc_conv_fwd_kernel<false><<<(unsigned)ctas, kThreads, smem, st>>>(mx, mw, (__nv_bfloat16*)out, bias, relu, gather ? stat_partial : nullptr, p, status);

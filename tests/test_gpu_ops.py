@@ -205,7 +205,8 @@ def test_stem_kernels(n, h, w, cout):
     ((2, 112, 112, 128, 128, 3, 1), True),    # halo-patch kernel, 128-wide output tile
     ((4, 56, 56, 128, 256, 3, 1), True),      # halo-patch kernel, 256-wide output tile
     ((2, 14, 14, 192, 64, 3, 1), True),       # generic tensor-core kernel: one partial row pair per pixel tile
-    ((5, 30, 30, 128, 320, 1, 0), True),      # 1x1, several pixel tiles, 64-wide output tiles
+    ((5, 30, 30, 128, 320, 1, 0), False),     # 1x1 with a short reduction: separate statistics kernel
+    ((5, 30, 30, 1024, 320, 1, 0), True),     # 1x1, long reduction, several pixel tiles, 64-wide output tiles
     ((3, 21, 18, 3, 64, 3, 1), True),         # first-layer kernel, ragged last tile
     ((9, 96, 80, 3, 128, 3, 1), True),        # first-layer kernel, several tiles per CTA, two channel blocks
     ((2, 9, 9, 16, 24, 3, 1), False),         # CUDA-core kernel + separate statistics kernel
