@@ -130,29 +130,49 @@ __global__ void take_paired_columns_kernel(const float* __restrict__ dwp, float*
 // channels.  xcol[output pixel][(r, s, c) padded to WIDTH] so that forward and weight gradient become
 // plain contractions over WIDTH "channels" (a 1x1 convolution) for the tensor cores.
 template <int CIN, int KS, int STRIDE, int PAD, int WIDTH>
-__global__ void __launch_bounds__(256) unfold_stem_kernel(const __nv_bfloat16* __restrict__ x, __nv_bfloat16* __restrict__ xcol,
+__global__ void __launch_bounds__(192) unfold_stem_kernel(const __nv_bfloat16* __restrict__ x, __nv_bfloat16* __restrict__ xcol,
                                                           int n, int h, int wd, int ho, int wo) {
-    // one thread per 16-byte piece of a row: consecutive threads write consecutive pieces (full lines)
-    constexpr int K = KS * KS * CIN, PIECES = WIDTH / 8;
-    const int64_t items = (int64_t)n * ho * wo * PIECES;
+    // A block works on runs of RUN consecutive output pixels of one output row.  The KS input rows under a run are
+    // staged in shared memory with zeros outside the image, so the pieces are built without bounds checks; a
+    // thread always builds the same 16-byte piece j of a row (its eight source offsets are computed once), and 24
+    // consecutive threads write one 384-byte row.
+    constexpr int K = KS * KS * CIN, PIECES = WIDTH / 8, RUN = 32, PX = 192 / PIECES;
+    constexpr int COLS = (RUN - 1) * STRIDE + KS;             // input pixels under a run
+    static_assert(192 % PIECES == 0 && RUN % PX == 0, "thread layout");
+    __shared__ uint16_t rows[KS][COLS * CIN];
     const uint16_t* x16 = reinterpret_cast<const uint16_t*>(x);
-    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < items; i += (int64_t)gridDim.x * blockDim.x) {
-        const int j = (int)(i % PIECES);
-        const int64_t p = i / PIECES;
-        const int ow = (int)(p % wo);
-        const int oh = (int)((p / wo) % ho);
-        const int64_t img = p / ((int64_t)wo * ho);
-        const int ih0 = oh * STRIDE - PAD, iw0 = ow * STRIDE - PAD;
-        const uint16_t* origin = x16 + ((img * h + ih0) * wd + iw0) * CIN;     // may point outside: only dereferenced in bounds
-        __align__(16) uint16_t v[8];
+    const int j = threadIdx.x % PIECES, px0 = threadIdx.x / PIECES;
+    int src[8];                                               // offset of element e in the staged rows, or -1 for padding columns
 #pragma unroll
-        for (int e = 0; e < 8; ++e) {
-            const int idx = j * 8 + e;
-            const int c = idx % CIN, tap = idx / CIN, r = tap / KS, q = tap % KS;
-            const bool in = idx < K && ih0 + r >= 0 && ih0 + r < h && iw0 + q >= 0 && iw0 + q < wd;
-            v[e] = in ? __ldg(origin + ((int64_t)r * wd + q) * CIN + c) : (uint16_t)0;
+    for (int e = 0; e < 8; ++e) {
+        const int idx = j * 8 + e;
+        const int c = idx % CIN, tap = idx / CIN, r = tap / KS, q = tap % KS;
+        src[e] = idx < K ? r * (COLS * CIN) + q * CIN + c : -1;
+    }
+    const int runs_per_row = (wo + RUN - 1) / RUN;
+    const int64_t runs = (int64_t)n * ho * runs_per_row;
+    for (int64_t run = blockIdx.x; run < runs; run += gridDim.x) {
+        const int ow0 = (int)(run % runs_per_row) * RUN;
+        const int oh = (int)((run / runs_per_row) % ho);
+        const int64_t img = run / ((int64_t)runs_per_row * ho);
+        const int ih0 = oh * STRIDE - PAD, iw0 = ow0 * STRIDE - PAD;
+        for (int i = threadIdx.x; i < KS * COLS * CIN; i += 192) {
+            const int r = i / (COLS * CIN), col = i % (COLS * CIN);
+            const int ih = ih0 + r, iw = iw0 + col / CIN;
+            const bool in = ih >= 0 && ih < h && iw >= 0 && iw < wd;
+            rows[r][col] = in ? __ldg(x16 + ((img * h + ih) * wd + iw) * CIN + col % CIN) : (uint16_t)0;
         }
-        reinterpret_cast<uint4*>(xcol)[i] = *reinterpret_cast<const uint4*>(v);
+        __syncthreads();
+        const uint16_t* flat = &rows[0][0];
+        for (int px = px0; px < RUN; px += PX) {
+            if (ow0 + px >= wo) break;
+            __align__(16) uint16_t v[8];
+#pragma unroll
+            for (int e = 0; e < 8; ++e) v[e] = src[e] >= 0 ? flat[src[e] + px * STRIDE * CIN] : (uint16_t)0;
+            const int64_t p = (img * ho + oh) * wo + ow0 + px;
+            reinterpret_cast<uint4*>(xcol)[p * PIECES + j] = *reinterpret_cast<const uint4*>(v);
+        }
+        __syncthreads();
     }
 }
 
@@ -239,9 +259,9 @@ int64_t stem_conv_scratch_bytes(const ConvGeom& g) {
 }
 
 static int stem_unfold(const ConvGeom& g, const void* x, __nv_bfloat16* xcol, cudaStream_t st) {
-    const int64_t items = (int64_t)g.n * g.ho * g.wo * (kStemWidth / 8);
-    const unsigned grid = (unsigned)std::min<int64_t>((items + 255) / 256, 148 * 64);
-    unfold_stem_kernel<3, 7, 2, 3, kStemWidth><<<grid, 256, 0, st>>>((const __nv_bfloat16*)x, xcol, g.n, g.h, g.w, g.ho, g.wo);
+    const int64_t runs = (int64_t)g.n * g.ho * ((g.wo + 31) / 32);
+    const unsigned grid = (unsigned)std::max<int64_t>(1, std::min<int64_t>(runs, 148 * 10));
+    unfold_stem_kernel<3, 7, 2, 3, kStemWidth><<<grid, 192, 0, st>>>((const __nv_bfloat16*)x, xcol, g.n, g.h, g.w, g.ho, g.wo);
     CKPT_LAUNCH_CHECK("stem unfold");
     return CKPT_OK;
 }

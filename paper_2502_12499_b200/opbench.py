@@ -1,6 +1,6 @@
 """Run and time single operations of the library (for profiling and roofline numbers).
 
-    python -m paper_2502_12499_b200.opbench conv fwd|dgrad|wgrad N H W C_IN C_OUT K PAD [--reps R]
+    python -m paper_2502_12499_b200.opbench conv fwd|dgrad|wgrad N H W C_IN C_OUT K PAD [STRIDE] [--reps R]
     python -m paper_2502_12499_b200.opbench bn fwd|bwd ROWS C [--reps R]
     python -m paper_2502_12499_b200.opbench pool fwd|bwd N H W C [--reps R]
     python -m paper_2502_12499_b200.opbench convmix fwd|dgrad|wgrad CONFIG [--reps R]   (all conv layers of a config)
@@ -30,15 +30,16 @@ def _time(fn, reps, warmup=2):
     return e0.elapsed_time(e1) / reps
 
 
-def conv(what, n, h, w, cin, cout, k, pad, reps=3, impl=0):
+def conv(what, n, h, w, cin, cout, k, pad, stride=1, reps=3, impl=0):
     """One convolution operation; returns dict(ms, tflops, flops)."""
     import torch
     dt = ck.DTYPE_BF16
-    shape = ck.ConvShape(n, h, w, cin, cout, k, 1, pad)
+    shape = ck.ConvShape(n, h, w, cin, cout, k, stride, pad)
+    ho, wo = (h + 2 * pad - k) // stride + 1, (w + 2 * pad - k) // stride + 1
     x = torch.randn(n, h, w, cin, device="cuda").bfloat16()
     wt = (torch.randn(cout, k, k, cin, device="cuda") * 0.05).bfloat16()
-    z = torch.empty(n, h, w, cout, device="cuda", dtype=torch.bfloat16)
-    dz = torch.randn(n, h, w, cout, device="cuda").bfloat16()
+    z = torch.empty(n, ho, wo, cout, device="cuda", dtype=torch.bfloat16)
+    dz = torch.randn(n, ho, wo, cout, device="cuda").bfloat16()
     dx = torch.empty_like(x)
     dw = torch.empty(cout, k, k, cin, device="cuda")
     scratch = torch.empty(max(256, ck.conv2d_scratch_bytes(shape, dt)), dtype=torch.uint8, device="cuda")
@@ -46,8 +47,8 @@ def conv(what, n, h, w, cin, cout, k, pad, reps=3, impl=0):
           "dgrad": lambda: ck.conv2d_dgrad(shape, dt, impl, dz, wt, dx, scratch),
           "wgrad": lambda: ck.conv2d_wgrad(shape, dt, impl, dz, x, dw, scratch)}[what]
     ms = _time(fn, reps)
-    flops = 2.0 * n * h * w * cout * k * k * cin
-    return dict(op="conv " + what, shape=[n, h, w, cin, cout, k, pad], ms=ms, flops=flops, tflops=flops / ms / 1e9)
+    flops = 2.0 * n * ho * wo * cout * k * k * cin
+    return dict(op="conv " + what, shape=[n, h, w, cin, cout, k, pad] + ([stride] if stride != 1 else []), ms=ms, flops=flops, tflops=flops / ms / 1e9)
 
 
 def bn(what, rows, c, reps=5):
