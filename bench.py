@@ -276,7 +276,7 @@ def main():
 # DRAM traffic per launch of the conv-forward kernels over the layer mix of config 2, from one ncu pass
 # (profiles/conv_forward_vgg16_b64_dram_traffic.md).  Valid only for the kernel source it was taken
 # on: reported as null when csrc/conv_tc.cu has changed since.
-CONV_FWD_TRAFFIC = {"source_sha256": "54ca8d2386c18caba912e12aa0f447a77e6d25de9928080f6d145483e284be8f", "bytes_per_launch": 165657195}
+CONV_FWD_TRAFFIC = {"source_sha256": "74381a05169829d5fa16b56f3f8549169774a5c107edb455f6920a2c8c5b9e1d", "bytes_per_launch": 165571200}
 
 
 def _kernel_source_sha():
