@@ -423,6 +423,165 @@ tc_conv_fwd_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_const
 }
 
 // ------------------------------------------------------------------------------------------------
+// Forward / dgrad with the roles swapped, for output tiles of 128 channels: D^T[c_out tile 128][256 pixels].
+// An MMA instruction takes about as long at N = 64 or 128 as at N = 256, so with 128 output channels on N
+// (pixels on M) a third of the tensor pipe's time is lost; here the filter box is the M operand (128 output
+// channels x 64 reduction channels per stage), the pixel box the N operand (256 pixels x 64 channels), and
+// every instruction is 128 x 256 x 16.  Persistent CTAs per output-channel tile, operand ring across tile
+// boundaries, double-buffered accumulator (2 x 256 columns: all of tensor memory).
+// Epilogue: a thread owns one output channel (its accumulator lane) and meets 32 pixels per chunk: the 32
+// lanes of a warp store 64 contiguous bytes of one pixel per instruction, and the batch-norm sums of a channel
+// are plain per-thread sums.
+// ------------------------------------------------------------------------------------------------
+struct TParams {
+    int H, W, N;                 // pixel grid walked by the tiles (= the output tensor: stride 1)
+    int c_red, c_out;
+    int taps;
+    int tap_dh[9], tap_dw[9], tap_col[9];
+    int tw_log, th_log;          // pixel tile tw x th x tn = 256, powers of two
+    int tw, th, tn;
+    int tiles_w, tiles_h, tiles_n;
+    int co_tiles, p_tiles, ctas_per_co;
+    int stages;
+};
+
+__global__ void __launch_bounds__(kThreads, 1)
+tc_conv_t_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w,
+                 __nv_bfloat16* __restrict__ out, float* __restrict__ stat_partial, TParams p, int* status) {
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    constexpr uint32_t a_bytes = 128 * 128, b_bytes = 256 * 128, stage_bytes = a_bytes + b_bytes;
+    const uint32_t bars = base + (uint32_t)p.stages * stage_bytes;           // full[s], empty[s], acc_full[2], acc_empty[2]
+    __shared__ uint32_t tmem_base_slot;
+    __shared__ int failed_flag;
+    volatile int* failed = &failed_flag;
+
+    const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
+    const int co_tile = blockIdx.x % p.co_tiles;
+    const int first = blockIdx.x / p.co_tiles;
+    const int my_tiles = first < p.p_tiles ? (p.p_tiles - first + p.ctas_per_co - 1) / p.ctas_per_co : 0;
+    const int blocks = p.c_red / 64;
+    const int iters = p.taps * blocks;
+
+    auto full_bar = [&](int s) { return bars + 8u * s; };
+    auto empty_bar = [&](int s) { return bars + 8u * (kMaxStages + s); };
+    const uint32_t acc_full0 = bars + 8u * (2 * kMaxStages), acc_empty0 = acc_full0 + 16;
+    auto tile_origin = [&](int j, int& w0, int& h0, int& n0) {
+        int t = first + j * p.ctas_per_co;
+        w0 = (t % p.tiles_w) * p.tw; t /= p.tiles_w;
+        h0 = (t % p.tiles_h) * p.th;
+        n0 = (t / p.tiles_h) * p.tn;
+    };
+
+    if (threadIdx.x == 0) {
+        failed_flag = 0;
+        for (int s = 0; s < p.stages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+        for (int b = 0; b < 2; ++b) { mbar_init(acc_full0 + 8 * b, 1); mbar_init(acc_empty0 + 8 * b, 128); }
+        fence_barrier_init();
+        tma_prefetch_desc(&map_x);
+        tma_prefetch_desc(&map_w);
+    }
+    if (warp == 1) tmem_alloc(smem_u32(&tmem_base_slot), 512);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = tmem_base_slot;
+
+    if (warp == 0 && lane == 0) {
+        // ---------------- TMA producer: filter box (M operand) and pixel box (N operand) per stage
+        int g = 0;
+        bool ok = true;
+        for (int j = 0; j < my_tiles && ok; ++j) {
+            int w0, h0, n0;
+            tile_origin(j, w0, h0, n0);
+            for (int it = 0; it < iters; ++it, ++g) {
+                const int s = g % p.stages;
+                if (!mbar_wait(empty_bar(s), ((uint32_t)(g / p.stages) & 1u) ^ 1u, failed, status, 901)) { ok = false; break; }
+                const int tap = it / blocks, blk = it % blocks;
+                const uint32_t a_dst = base + (uint32_t)s * stage_bytes;
+                mbar_expect_tx(full_bar(s), stage_bytes);
+                tma_load_2d(a_dst, &map_w, full_bar(s), p.tap_col[tap] * p.c_red + blk * 64, co_tile * 128);
+                tma_load_4d(a_dst + a_bytes, &map_x, full_bar(s), blk * 64, w0 + p.tap_dw[tap], h0 + p.tap_dh[tap], n0);
+            }
+        }
+        if (*failed) {
+            for (int q = max(0, g - p.stages); q < g; ++q) mbar_drain(full_bar(q % p.stages), (uint32_t)(q / p.stages) & 1u);
+        }
+    } else if (warp == 1 && lane == 0) {
+        // ---------------- MMA issuer
+        const uint32_t idesc = instr_desc(128, 256, 0, 0);
+        bool ok = true;
+        int g = 0;
+        for (int j = 0; j < my_tiles && ok; ++j) {
+            const int buf = j & 1;
+            if (!mbar_wait(acc_empty0 + 8 * buf, ((uint32_t)(j >> 1) & 1u) ^ 1u, failed, status, 904)) { ok = false; break; }
+            const uint32_t acc = tmem_base + (uint32_t)(buf * 256);
+            for (int it = 0; it < iters; ++it, ++g) {
+                const int s = g % p.stages;
+                if (!mbar_wait(full_bar(s), (uint32_t)(g / p.stages) & 1u, failed, status, 902)) { ok = false; break; }
+                tc_fence_after();
+                const uint32_t a_addr = base + (uint32_t)s * stage_bytes;
+                const uint32_t b_addr = a_addr + a_bytes;
+#pragma unroll
+                for (int kk = 0; kk < 4; ++kk)
+                    umma_bf16(acc, smem_desc(a_addr + kk * 32, 0, 1024), smem_desc(b_addr + kk * 32, 0, 1024), idesc,
+                              (it > 0 || kk > 0) ? 1u : 0u);
+                umma_commit(empty_bar(s));
+            }
+            if (ok) umma_commit(acc_full0 + 8 * buf);
+        }
+    } else if (warp >= 2) {
+        // ---------------- epilogue: lane of the accumulator = output channel, column = pixel of the tile
+        const int quarter = warp % 4;
+        const int co = co_tile * 128 + quarter * 32 + lane;
+        const bool stats = stat_partial != nullptr;
+        float sum = 0.f, sumsq = 0.f;
+        for (int j = 0; j < my_tiles; ++j) {
+            const int buf = j & 1;
+            if (!mbar_wait(acc_full0 + 8 * buf, (uint32_t)(j >> 1) & 1u, failed, status, 903)) break;
+            tc_fence_after();
+            int w0, h0, n0;
+            tile_origin(j, w0, h0, n0);
+#pragma unroll 1
+            for (int c0 = 0; c0 < 256; c0 += 32) {
+                // lane e works out where pixel c0 + e of the tile lives (or that it lies outside the tensor)
+                const int idx = c0 + lane;
+                const int wl = idx & (p.tw - 1), hl = (idx >> p.tw_log) & (p.th - 1), nl = idx >> (p.tw_log + p.th_log);
+                const bool inside = (w0 + wl < p.W) && (h0 + hl < p.H) && (n0 + nl < p.N);
+                const int my_pix = inside ? ((n0 + nl) * p.H + (h0 + hl)) * p.W + (w0 + wl) : -1;
+                uint32_t v[32];
+                tmem_ld32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * 256 + c0), v);
+#pragma unroll
+                for (int e = 0; e < 32; ++e) {
+                    const int pix = __shfl_sync(0xffffffffu, my_pix, e);
+                    if (pix >= 0) {
+                        const __nv_bfloat16 r = __float2bfloat16_rn(__uint_as_float(v[e]));
+                        out[(size_t)pix * p.c_out + co] = r;
+                        const float f = __bfloat162float(r);
+                        sum += f;
+                        sumsq = fmaf(f, f, sumsq);
+                    }
+                }
+            }
+            tc_fence_before();
+            mbar_arrive(acc_empty0 + 8 * buf);
+        }
+        if (stats) {
+            // one partial row pair per CTA: [block][sum | sum of squares][channel]
+            stat_partial[((size_t)first * 2) * p.c_out + co] = sum;
+            stat_partial[((size_t)first * 2 + 1) * p.c_out + co] = sumsq;
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        __syncwarp();
+        tc_fence_after();
+        tmem_dealloc(tmem_base, 512);
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
 // Forward / dgrad for 64 reduction channels, 3x3, padding 1 (first layers of VGG-like chains, the
 // whole 64-channel deep chain).  With K = 9*64 the generic kernel is bound by L2->SM traffic (every
 // tap re-fetches the pixel tile) and by the unhidden epilogue.  Here a persistent CTA
@@ -1752,6 +1911,50 @@ int launch_generic(FwdParams p, const void* a, int a_n, int a_h, int a_w, const 
     return CKPT_OK;
 }
 
+// Role-swapped kernel (output channels on M, 256 pixels on N): stride-1 shapes with 128 output channels and a
+// reduction long enough to hide its epilogue.  Measured against the halo-patch kernel: 256 -> 128 channels at 56x56
+// 0.199 -> 0.127 ms, 128 -> 128 at 112x112 0.319 -> 0.307 ms; with 64 reduction channels it loses to the
+// 64-channel kernel (0.155 -> 0.287 ms) and is not used.
+bool t_applies(int c_red, int c_out, int k, int pad) {
+    return c_out == 128 && c_red % 64 == 0 && c_red >= 128 && ((k == 3 && pad == 1) || (k == 1 && pad == 0));
+}
+int launch_t(const void* x, const void* w_mat, void* out, float* stat_partial, int* stat_blocks, int N, int H, int W, int c_red,
+             int c_out, int k, int pad, int* status, cudaStream_t st, const char* what) {
+    TParams p;
+    p.H = H; p.W = W; p.N = N; p.c_red = c_red; p.c_out = c_out;
+    p.taps = k * k;
+    for (int t = 0; t < k * k; ++t) { p.tap_dh[t] = t / k - pad; p.tap_dw[t] = t % k - pad; p.tap_col[t] = t; }
+    choose_tile(256, W, H, N, &p.tw, &p.th, &p.tn);
+    p.tw_log = 0; while ((1 << p.tw_log) < p.tw) ++p.tw_log;
+    p.th_log = 0; while ((1 << p.th_log) < p.th) ++p.th_log;
+    p.tiles_w = (W + p.tw - 1) / p.tw; p.tiles_h = (H + p.th - 1) / p.th; p.tiles_n = (N + p.tn - 1) / p.tn;
+    p.co_tiles = c_out / 128;
+    p.p_tiles = p.tiles_w * p.tiles_h * p.tiles_n;
+    int sms = 148, dev = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    p.ctas_per_co = std::max(1, std::min(p.p_tiles, sms / p.co_tiles));
+    constexpr uint32_t stage_bytes = 128 * 128 + 256 * 128;
+    p.stages = std::min<int>(kMaxStages, kSmemBudget / stage_bytes);
+    CUtensorMap mx, mw;
+    int rc = make_act_map(&mx, x, N, H, W, c_red, p.tw, p.th, p.tn);
+    if (rc) return rc;
+    rc = make_mat_map(&mw, w_mat, c_out, (int64_t)k * k * c_red, 128);
+    if (rc) return rc;
+    const size_t smem = (size_t)p.stages * stage_bytes + 1024 + 256;
+    static bool attr_set = false;
+    if (!attr_set) {
+        cudaError_t e = cudaFuncSetAttribute(tc_conv_t_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget + 2048);
+        if (e != cudaSuccess) return cuda_fail(e, "raising the shared-memory limit");
+        attr_set = true;
+    }
+    if (stat_blocks) *stat_blocks = stat_partial ? p.ctas_per_co : 0;
+    tc_conv_t_kernel<<<p.ctas_per_co * p.co_tiles, kThreads, smem, st>>>(mx, mw, (__nv_bfloat16*)out, stat_blocks ? stat_partial : nullptr, p,
+                                                                         status);
+    CKPT_LAUNCH_CHECK(what);
+    return CKPT_OK;
+}
+
 // stat_partial / stat_blocks: null, or where the kernel leaves the batch-norm partial sums of its output
 // ([block][sum | sum of squares][c_out] floats) and how many blocks it wrote (0 = this kernel does not gather them).
 int launch_fwd_like(const void* x, const void* w_mat, void* out, const float* bias, int relu, int N, int H, int W, int c_red,
@@ -1759,6 +1962,8 @@ int launch_fwd_like(const void* x, const void* w_mat, void* out, const float* bi
                     int* stat_blocks = nullptr, bool b_mn = false) {
     // b_mn (1x1 only): w_mat is the forward filter [c_red][c_out] read in place (c_out a multiple of 64)
     if (stat_blocks) *stat_blocks = 0;
+    if (!bias && !relu && !b_mn && t_applies(c_red, c_out, k, pad))
+        return launch_t(x, w_mat, out, stat_partial, stat_blocks, N, H, W, c_red, c_out, k, pad, status, st, what);
     if (c_red == 64 && k == 3 && pad == 1 && c_out % 64 == 0 && !bias && !relu)
         return launch_c64(x, w_mat, out, stat_partial, stat_blocks, N, H, W, c_out, status, st, what);
     if (!bias && !relu && halo_applies(H, W, c_red, c_out, k, pad))
