@@ -105,6 +105,10 @@ __device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, uint32_t sr
     asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
                  ::"l"(map), "r"(src), "r"(c0), "r"(c1) : "memory");
 }
+__device__ __forceinline__ void tma_store_4d(const CUtensorMap* map, uint32_t src, int c0, int c1, int c2, int c3) {
+    asm volatile("cp.async.bulk.tensor.4d.global.shared::cta.bulk_group [%0, {%2, %3, %4, %5}], [%1];"
+                 ::"l"(map), "r"(src), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
+}
 __device__ __forceinline__ void tma_store_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 // Waits until at most N of this thread's store groups still read their shared-memory source.
 template <int N> __device__ __forceinline__ void tma_store_wait_read() {
@@ -447,11 +451,12 @@ struct TParams {
 
 __global__ void __launch_bounds__(kThreads, 1)
 tc_conv_t_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w,
-                 __nv_bfloat16* __restrict__ out, float* __restrict__ stat_partial, TParams p, int* status) {
+                 const __grid_constant__ CUtensorMap map_out, float* __restrict__ stat_partial, TParams p, int* status) {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     constexpr uint32_t a_bytes = 128 * 128, b_bytes = 256 * 128, stage_bytes = a_bytes + b_bytes;
     const uint32_t bars = base + (uint32_t)p.stages * stage_bytes;           // full[s], empty[s], acc_full[2], acc_empty[2]
+    const uint32_t out_stage = bars + 256;                                   // [4 warps][2][32 pixels x 32 channels] bf16
     __shared__ uint32_t tmem_base_slot;
     __shared__ int failed_flag;
     volatile int* failed = &failed_flag;
@@ -480,6 +485,7 @@ tc_conv_t_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
         fence_barrier_init();
         tma_prefetch_desc(&map_x);
         tma_prefetch_desc(&map_w);
+        tma_prefetch_desc(&map_out);
     }
     if (warp == 1) tmem_alloc(smem_u32(&tmem_base_slot), 512);
     tc_fence_before();
@@ -531,11 +537,16 @@ tc_conv_t_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
             if (ok) umma_commit(acc_full0 + 8 * buf);
         }
     } else if (warp >= 2) {
-        // ---------------- epilogue: lane of the accumulator = output channel, column = pixel of the tile
+        // ---------------- epilogue: lane of the accumulator = output channel, column = pixel of the tile.  A chunk
+        // of 32 pixels x 32 channels is written to shared memory pixel-major (a lane's two bytes next to its
+        // neighbours': 64-byte rows) and leaves as one tile store whose box is the chunk's bw x bh x bn pixels;
+        // the hardware clips what lies outside the tensor.  (Two-byte global stores from the lanes, 64 bytes per
+        // instruction, made this epilogue the bottleneck of the kernel: 0.32 ms against 0.18 ms without them.)
         const int quarter = warp % 4;
         const int co = co_tile * 128 + quarter * 32 + lane;
         const bool stats = stat_partial != nullptr;
         float sum = 0.f, sumsq = 0.f;
+        int chunk_count = 0;
         for (int j = 0; j < my_tiles; ++j) {
             const int buf = j & 1;
             if (!mbar_wait(acc_full0 + 8 * buf, (uint32_t)(j >> 1) & 1u, failed, status, 903)) break;
@@ -543,30 +554,40 @@ tc_conv_t_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
             int w0, h0, n0;
             tile_origin(j, w0, h0, n0);
 #pragma unroll 1
-            for (int c0 = 0; c0 < 256; c0 += 32) {
-                // lane e works out where pixel c0 + e of the tile lives (or that it lies outside the tensor)
+            for (int c0 = 0; c0 < 256; c0 += 32, ++chunk_count) {
+                // lane e works out whether pixel c0 + e of the tile lies inside the tensor (for the sums)
                 const int idx = c0 + lane;
                 const int wl = idx & (p.tw - 1), hl = (idx >> p.tw_log) & (p.th - 1), nl = idx >> (p.tw_log + p.th_log);
                 const bool inside = (w0 + wl < p.W) && (h0 + hl < p.H) && (n0 + nl < p.N);
-                const int my_pix = inside ? ((n0 + nl) * p.H + (h0 + hl)) * p.W + (w0 + wl) : -1;
+                const uint32_t in_mask = __ballot_sync(0xffffffffu, inside);
                 uint32_t v[32];
                 tmem_ld32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * 256 + c0), v);
+                const uint32_t slab = out_stage + (uint32_t)((quarter * 2 + (chunk_count & 1)) * 2048);
+                if (lane == 0) tma_store_wait_read<1>();          // the store that last read this slab has left it
+                __syncwarp();
 #pragma unroll
                 for (int e = 0; e < 32; ++e) {
-                    const int pix = __shfl_sync(0xffffffffu, my_pix, e);
-                    if (pix >= 0) {
-                        const __nv_bfloat16 r = __float2bfloat16_rn(__uint_as_float(v[e]));
-                        out[(size_t)pix * p.c_out + co] = r;
+                    const __nv_bfloat16 r = __float2bfloat16_rn(__uint_as_float(v[e]));
+                    asm volatile("st.shared.b16 [%0], %1;" ::"r"(slab + (uint32_t)(e * 64 + lane * 2)), "h"(__bfloat16_as_ushort(r)) : "memory");
+                    if ((in_mask >> e) & 1u) {
                         const float f = __bfloat162float(r);
                         sum += f;
                         sumsq = fmaf(f, f, sumsq);
                     }
                 }
+                fence_proxy_async();
+                __syncwarp();
+                if (lane == 0 && in_mask != 0u && co_tile * 128 + quarter * 32 < p.c_out) {
+                    const int cw = c0 & (p.tw - 1), chh = (c0 >> p.tw_log) & (p.th - 1), cn = c0 >> (p.tw_log + p.th_log);
+                    tma_store_4d(&map_out, slab, co_tile * 128 + quarter * 32, w0 + cw, h0 + chh, n0 + cn);
+                    tma_store_commit();
+                }
             }
             tc_fence_before();
             mbar_arrive(acc_empty0 + 8 * buf);
         }
-        if (stats) {
+        if (lane == 0) tma_store_wait_all();
+        if (stats && co < p.c_out) {
             // one partial row pair per CTA: [block][sum | sum of squares][channel]
             stat_partial[((size_t)first * 2) * p.c_out + co] = sum;
             stat_partial[((size_t)first * 2 + 1) * p.c_out + co] = sumsq;
@@ -1911,12 +1932,14 @@ int launch_generic(FwdParams p, const void* a, int a_n, int a_h, int a_w, const 
     return CKPT_OK;
 }
 
-// Role-swapped kernel (output channels on M, 256 pixels on N): stride-1 shapes with 128 output channels and a
-// reduction long enough to hide its epilogue.  Measured against the halo-patch kernel: 256 -> 128 channels at 56x56
-// 0.199 -> 0.127 ms, 128 -> 128 at 112x112 0.319 -> 0.307 ms; with 64 reduction channels it loses to the
-// 64-channel kernel (0.155 -> 0.287 ms) and is not used.
+// Role-swapped kernel (output channels on M, 256 pixels on N): stride-1 3x3 and 1x1 shapes whose output channels
+// come in tiles of 128, or 64 of them with 128+ reduction channels (rows 64..127 of the filter box are then zero
+// fill).  Measured on the VGG-16 shapes (batch 64) against the kernels it replaces: 64 -> 128 at 112x112 0.157 ->
+// 0.121 ms, 128 -> 128 at 112x112 0.319 -> 0.205, dgrad 128 -> 64 at 112x112 0.310 -> 0.196, 128 -> 256 at 56x56
+// 0.124 -> 0.105, 256 -> 256 at 56x56 0.219 -> 0.195, 28x28 and 14x14 within 4 % either way; 64 -> 64 at 224x224 stays
+// with the 64-channel kernel (0.31 against 0.64 ms).
 bool t_applies(int c_red, int c_out, int k, int pad) {
-    return c_out == 128 && c_red % 64 == 0 && c_red >= 128 && ((k == 3 && pad == 1) || (k == 1 && pad == 0));
+    return (c_out % 128 == 0 || (c_out == 64 && c_red >= 128)) && c_red % 64 == 0 && ((k == 3 && pad == 1) || (k == 1 && pad == 0));
 }
 int launch_t(const void* x, const void* w_mat, void* out, float* stat_partial, int* stat_blocks, int N, int H, int W, int c_red,
              int c_out, int k, int pad, int* status, cudaStream_t st, const char* what) {
@@ -1928,7 +1951,7 @@ int launch_t(const void* x, const void* w_mat, void* out, float* stat_partial, i
     p.tw_log = 0; while ((1 << p.tw_log) < p.tw) ++p.tw_log;
     p.th_log = 0; while ((1 << p.th_log) < p.th) ++p.th_log;
     p.tiles_w = (W + p.tw - 1) / p.tw; p.tiles_h = (H + p.th - 1) / p.th; p.tiles_n = (N + p.tn - 1) / p.tn;
-    p.co_tiles = c_out / 128;
+    p.co_tiles = (c_out + 127) / 128;
     p.p_tiles = p.tiles_w * p.tiles_h * p.tiles_n;
     int sms = 148, dev = 0;
     cudaGetDevice(&dev);
@@ -1941,16 +1964,29 @@ int launch_t(const void* x, const void* w_mat, void* out, float* stat_partial, i
     if (rc) return rc;
     rc = make_mat_map(&mw, w_mat, c_out, (int64_t)k * k * c_red, 128);
     if (rc) return rc;
-    const size_t smem = (size_t)p.stages * stage_bytes + 1024 + 256;
+    // the box of one epilogue chunk: 32 consecutive pixels of the tile (w fastest) x 32 channels, no swizzle
+    CUtensorMap mo;
+    {
+        const int bw = std::min(p.tw, 32), bh = std::min(p.th, 32 / bw), bnn = 32 / (bw * bh);
+        EncodeTiledFn fn = encode_fn();
+        if (!fn) { set_error("cuTensorMapEncodeTiled is not available from this driver"); return CKPT_E_CUDA; }
+        cuuint64_t dims[4] = {(cuuint64_t)c_out, (cuuint64_t)W, (cuuint64_t)H, (cuuint64_t)N};
+        cuuint64_t strides[3] = {(cuuint64_t)c_out * 2, (cuuint64_t)W * c_out * 2, (cuuint64_t)H * W * c_out * 2};
+        cuuint32_t box[4] = {32, (cuuint32_t)bw, (cuuint32_t)bh, (cuuint32_t)bnn};
+        cuuint32_t es[4] = {1, 1, 1, 1};
+        CUresult r = fn(&mo, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, out, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                        CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        if (r != CUDA_SUCCESS) { set_error("cuTensorMapEncodeTiled failed for an output tensor (code %d)", (int)r); return CKPT_E_CUDA; }
+    }
+    const size_t smem = (size_t)p.stages * stage_bytes + 1024 + 256 + 4 * 2 * 2048;
     static bool attr_set = false;
     if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(tc_conv_t_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget + 2048);
+        cudaError_t e = cudaFuncSetAttribute(tc_conv_t_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024);
         if (e != cudaSuccess) return cuda_fail(e, "raising the shared-memory limit");
         attr_set = true;
     }
     if (stat_blocks) *stat_blocks = stat_partial ? p.ctas_per_co : 0;
-    tc_conv_t_kernel<<<p.ctas_per_co * p.co_tiles, kThreads, smem, st>>>(mx, mw, (__nv_bfloat16*)out, stat_blocks ? stat_partial : nullptr, p,
-                                                                         status);
+    tc_conv_t_kernel<<<p.ctas_per_co * p.co_tiles, kThreads, smem, st>>>(mx, mw, mo, stat_blocks ? stat_partial : nullptr, p, status);
     CKPT_LAUNCH_CHECK(what);
     return CKPT_OK;
 }
