@@ -276,7 +276,7 @@ def main():
 # DRAM traffic per launch of the conv-forward kernels over the layer mix of config 2, from one ncu pass
 # (profiles/conv_forward_vgg16_b64_dram_traffic.md).  Valid only for the kernel source it was taken
 # on: reported as null when csrc/conv_tc.cu has changed since.
-CONV_FWD_TRAFFIC = {"source_sha256": "74381a05169829d5fa16b56f3f8549169774a5c107edb455f6920a2c8c5b9e1d", "bytes_per_launch": 165571200}
+CONV_FWD_TRAFFIC = {"source_sha256": "bd1c0cb9c337ce6505142a85c5260d017d0dfc8e3d805b263e94635fbb804ec5", "bytes_per_launch": 169778666}
 
 
 def _kernel_source_sha():
@@ -286,14 +286,15 @@ def _kernel_source_sha():
 
 
 def dominant_kernel_roofline(config_index, peaks, batch, first_shape):
-    """The convolution-forward kernels (tcgen05) hold the largest share of the step: they run in the
-    forward phase, in segment recomputation and, on the transposed matrix, as dgrad.  Timed here on
+    """The convolution-forward kernels (tcgen05; the role-swapped kernel for every layer but the two
+    64-channel ones) hold the largest share of the step: they run in the forward phase, in segment
+    recomputation and, on the transposed matrix, as dgrad.  Timed here on
     every conv layer shape of the workload with CUDA events; achieved = sum of algorithmic FLOPs /
     sum of launch times, against the measured dense-bf16 peak."""
     from paper_2502_12499_b200 import opbench
     mix = opbench.conv_mix("fwd", config_index, reps=3)
     traffic = CONV_FWD_TRAFFIC["bytes_per_launch"] if CONV_FWD_TRAFFIC["source_sha256"] == _kernel_source_sha() else None
-    out = {"kernel": "tc_conv_fwd_kernel / tc_conv_halo_kernel / tc_conv_c64_kernel (implicit-GEMM conv forward)", "bound": "tensor",
+    out = {"kernel": "tc_conv_t_kernel / tc_conv_c64_kernel (implicit-GEMM conv forward over the layer mix)", "bound": "tensor",
            "achieved": mix["tflops"], "peak": peaks["tflops_burst"], "unit": "TFLOP/s", "frac": mix["tflops"] / peaks["tflops_burst"],
            "peak_source": peaks["source"] + " (burst: kernels timed in isolation)", "traffic": traffic,
            "launch_shapes": mix["launches"], "flops_per_launch": mix["flops"] / mix["launches"],
