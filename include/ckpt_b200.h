@@ -308,12 +308,16 @@ CKPT_API int ckpt_bn_relu_backward(int dtype, int64_t rows, int32_t c, const voi
 CKPT_API int ckpt_bn_relu_forward_noalloc(int dtype, int64_t rows, int32_t c, const void* z, const float* gamma,
                                  const float* beta, int relu, void* y, float* stats, void* stream);
 
-/* Max pooling, NHWC.  backward recomputes the arg-max from x. */
+/* Max pooling, NHWC.  backward recomputes the arg-max from x (first maximum in row-major window order).
+ * scratch (device, may be null): with ckpt_maxpool_backward_scratch_bytes bytes (8-byte aligned) the general
+ * (not 2x2 stride 2) backward records one arg-max byte per output element and gathers from that. */
 CKPT_API int ckpt_maxpool_forward(int dtype, int32_t n, int32_t h, int32_t w, int32_t c, int32_t k,
                          int32_t stride, int32_t pad, const void* x, void* y, void* stream);
+CKPT_API int ckpt_maxpool_backward_scratch_bytes(int dtype, int32_t n, int32_t h, int32_t w, int32_t c, int32_t k,
+                                        int32_t stride, int32_t pad, int64_t* bytes);
 CKPT_API int ckpt_maxpool_backward(int dtype, int32_t n, int32_t h, int32_t w, int32_t c, int32_t k,
                           int32_t stride, int32_t pad, const void* x, const void* dy, void* dx,
-                          void* stream);
+                          void* scratch, int64_t scratch_bytes, void* stream);
 
 /* Softmax cross-entropy, mean over the batch: loss (device float, written), dlogits (chain dtype).
  * labels: device int32. */

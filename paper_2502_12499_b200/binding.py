@@ -341,8 +341,15 @@ def maxpool_forward(dtype, n, h, w, c, k, stride, pad, x, y, stream=None):
     _check(lib().ckpt_maxpool_forward(C.c_int(dtype), n, h, w, c, k, stride, pad, _dev(x), _dev(y), _stream(stream)))
 
 
-def maxpool_backward(dtype, n, h, w, c, k, stride, pad, x, dy, dx, stream=None):
-    _check(lib().ckpt_maxpool_backward(C.c_int(dtype), n, h, w, c, k, stride, pad, _dev(x), _dev(dy), _dev(dx), _stream(stream)))
+def maxpool_backward_scratch_bytes(dtype, n, h, w, c, k, stride, pad):
+    b = C.c_int64(0)
+    _check(lib().ckpt_maxpool_backward_scratch_bytes(C.c_int(dtype), n, h, w, c, k, stride, pad, C.byref(b)))
+    return b.value
+
+
+def maxpool_backward(dtype, n, h, w, c, k, stride, pad, x, dy, dx, scratch=None, stream=None):
+    sp, sb = _scratch_args(scratch)
+    _check(lib().ckpt_maxpool_backward(C.c_int(dtype), n, h, w, c, k, stride, pad, _dev(x), _dev(dy), _dev(dx), sp, sb, _stream(stream)))
 
 
 def softmax_ce(dtype, batch, classes, logits, labels, loss, dlogits, stream=None):

@@ -148,11 +148,19 @@ int ckpt_maxpool_forward(int dtype, int32_t n, int32_t h, int32_t w, int32_t c, 
     return maxpool_forward(dtype, n, h, w, c, k, stride, pad, x, y, nullptr, stream);
 }
 
+int ckpt_maxpool_backward_scratch_bytes(int dtype, int32_t n, int32_t h, int32_t w, int32_t c, int32_t k, int32_t stride, int32_t pad,
+                                        int64_t* bytes) {
+    if (!bytes) { set_error("bytes is null"); return CKPT_E_NULL; }
+    if (n < 1 || c < 1 || k < 1 || stride < 1 || pad < 0 || 2 * pad > k || h + 2 * pad < k || w + 2 * pad < k) { set_error("bad pooling shape"); return CKPT_E_BAD_ARG; }
+    *bytes = maxpool_backward_scratch_bytes(dtype, n, h, w, c, k, stride, pad);
+    return CKPT_OK;
+}
+
 int ckpt_maxpool_backward(int dtype, int32_t n, int32_t h, int32_t w, int32_t c, int32_t k, int32_t stride, int32_t pad,
-                          const void* x, const void* dy, void* dx, void* stream) {
+                          const void* x, const void* dy, void* dx, void* scratch, int64_t scratch_bytes, void* stream) {
     if (!x || !dy || !dx) { set_error("null pointer"); return CKPT_E_NULL; }
     if (n < 1 || c < 1 || k < 1 || stride < 1 || pad < 0 || 2 * pad > k || h + 2 * pad < k || w + 2 * pad < k) { set_error("bad pooling shape"); return CKPT_E_BAD_ARG; }
-    return maxpool_backward(dtype, n, h, w, c, k, stride, pad, x, dy, dx, nullptr, stream);
+    return maxpool_backward(dtype, n, h, w, c, k, stride, pad, x, dy, dx, nullptr, stream, nullptr, nullptr, scratch, scratch_bytes);
 }
 
 int ckpt_softmax_ce(int dtype, int32_t batch, int32_t classes, const void* logits, const int32_t* labels, float* loss,

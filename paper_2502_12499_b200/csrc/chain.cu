@@ -349,7 +349,8 @@ static int unit_backward(StepCtx& c, int64_t i, const void* x_raw, const void* y
                 else if ((rc = activated(c, i - 1, x_raw, &x))) return rc;
             }
             if ((rc = maxpool_backward(dt, (int)c.ch->batch, u.in.h, u.in.w, u.in.c, u.desc.k, u.desc.stride, u.desc.pad, x, g_in,
-                                       g_out, act, c.stream, act ? (float*)(c.ws + c.ch->off_scr) : nullptr, &sum_blocks))) return rc;
+                                       g_out, act, c.stream, act ? (float*)(c.ws + c.ch->off_scr) : nullptr, &sum_blocks,
+                                       c.ws + c.ch->off_scr, c.ch->scr_bytes))) return rc;
             break;
         }
         case CKPT_UNIT_AVGPOOL:
@@ -757,6 +758,7 @@ int ckpt_chain_create(const ckpt_unit_desc* units, int64_t n, int64_t batch, int
                 }
                 u.out = {out_size(cur.h, u.desc.k, u.desc.stride, u.desc.pad),
                          out_size(cur.w, u.desc.k, u.desc.stride, u.desc.pad), cur.c};
+                scr = std::max(scr, maxpool_backward_scratch_bytes(dtype, (int)batch, cur.h, cur.w, cur.c, u.desc.k, u.desc.stride, u.desc.pad));
                 break;
             case CKPT_UNIT_AVGPOOL:
                 u.out = {1, 1, cur.c};

@@ -130,7 +130,9 @@ int maxpool_forward(int dtype, int n, int h, int w, int c, int k, int stride, in
 // sums there ([*bn_blocks][sum g | sum g*z][c] floats; *bn_blocks = 0 when it did not)
 int maxpool_backward(int dtype, int n, int h, int w, int c, int k, int stride, int pad, const void* x,
                      const void* dy, void* dx, const float* act, void* stream, float* bn_partial = nullptr,
-                     int* bn_blocks = nullptr);
+                     int* bn_blocks = nullptr, void* scratch = nullptr, int64_t scratch_bytes = 0);
+// bytes of scratch with which the general (not 2x2) backward runs in two light passes (0: no such path)
+int64_t maxpool_backward_scratch_bytes(int dtype, int n, int h, int w, int c, int k, int stride, int pad);
 int bn_relu_backward_from_partials(int dtype, int64_t rows, int c, const void* dy, const void* z, const float* stats, int relu,
                                    void* dz, float* dgamma, float* dbeta, void* scratch, int blocks, void* stream);
 int avgpool_forward(int dtype, int n, int h, int w, int c, const void* x, void* y, void* stream);

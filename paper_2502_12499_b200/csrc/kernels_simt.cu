@@ -1214,6 +1214,84 @@ __global__ void __launch_bounds__(256) maxpool_bwd_vec_kernel(const T* __restric
     }
 }
 
+// General pooling backward in two passes when scratch is available.  Pass 1, one thread per window and VEC
+// channels: the position (r*k + q) of the first maximum, one byte per channel.  Pass 2, one thread per input
+// pixel and VEC channels: for each of the (at most ceil(k/stride)^2) windows that contain the pixel, take the
+// window's gradient where the recorded position is this pixel's.  Pass 2 never reads x: eight small loads per
+// thread instead of re-scanning up to four whole windows.
+template <typename T, int VEC>
+__global__ void __launch_bounds__(256) maxpool_argmax_kernel(const T* __restrict__ x, uint8_t* __restrict__ arg, int64_t items, int h,
+                                                             int w, int c, int ho, int wo, int k, int stride, int pad) {
+    const int lanes = c / VEC;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < items; i += (int64_t)gridDim.x * blockDim.x) {
+        const int ch = (int)(i % lanes) * VEC;
+        int64_t t = i / lanes;
+        const int ow = (int)(t % wo); t /= wo;
+        const int oh = (int)(t % ho);
+        const int64_t img = t / ho;
+        float best[VEC];
+        uint8_t pos[VEC];
+#pragma unroll
+        for (int e = 0; e < VEC; ++e) { best[e] = -INFINITY; pos[e] = 255; }
+        for (int r = 0; r < k; ++r) {
+            const int ih = oh * stride - pad + r;
+            if (ih < 0 || ih >= h) continue;
+            for (int q = 0; q < k; ++q) {
+                const int iw = ow * stride - pad + q;
+                if (iw < 0 || iw >= w) continue;
+                float v[VEC];
+                load_vec<T, VEC>(x + ((img * h + ih) * w + iw) * c + ch, v);
+#pragma unroll
+                for (int e = 0; e < VEC; ++e)
+                    if (v[e] > best[e] || pos[e] == 255) { best[e] = v[e]; pos[e] = (uint8_t)(r * k + q); }   // strict: the first maximum stays
+            }
+        }
+#pragma unroll
+        for (int e = 0; e < VEC; ++e) arg[i * VEC + e] = pos[e];
+    }
+}
+
+template <typename T, int VEC>
+__global__ void __launch_bounds__(256) maxpool_bwd_arg_kernel(const uint8_t* __restrict__ arg, const T* __restrict__ dy, T* __restrict__ dx,
+                                                              int64_t items, int h, int w, int c, int ho, int wo, int k, int stride,
+                                                              int pad) {
+    const int lanes = c / VEC;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < items; i += (int64_t)gridDim.x * blockDim.x) {
+        const int ch = (int)(i % lanes) * VEC;
+        int64_t t = i / lanes;
+        const int iw = (int)(t % w); t /= w;
+        const int ih = (int)(t % h);
+        const int64_t img = t / h;
+        float acc[VEC];
+#pragma unroll
+        for (int e = 0; e < VEC; ++e) acc[e] = 0.f;
+        const int oh_lo = max(0, (ih + pad - k + stride) / stride), oh_hi = min(ho - 1, (ih + pad) / stride);
+        const int ow_lo = max(0, (iw + pad - k + stride) / stride), ow_hi = min(wo - 1, (iw + pad) / stride);
+        for (int oh = oh_lo; oh <= oh_hi; ++oh) {
+            for (int ow = ow_lo; ow <= ow_hi; ++ow) {
+                const int mine = (ih - (oh * stride - pad)) * k + (iw - (ow * stride - pad));
+                const int64_t o = ((img * ho + oh) * wo + ow) * c + ch;
+                uint8_t pos[VEC];
+                if constexpr (VEC == 8) *reinterpret_cast<uint2*>(pos) = *reinterpret_cast<const uint2*>(arg + o);
+                else *reinterpret_cast<uint32_t*>(pos) = *reinterpret_cast<const uint32_t*>(arg + o);
+                float g[VEC];
+                load_vec<T, VEC>(dy + o, g);
+#pragma unroll
+                for (int e = 0; e < VEC; ++e) acc[e] += pos[e] == mine ? g[e] : 0.f;
+            }
+        }
+        store_vec<T, VEC>(dx + i * VEC, acc);
+    }
+}
+
+int64_t maxpool_backward_scratch_bytes(int dtype, int n, int h, int w, int c, int k, int stride, int pad) {
+    if (maxpool_fuses_activation(dtype, h, w, c, k, stride, pad) || k * k > 250) return 0;
+    const int vec = dtype == CKPT_DTYPE_BF16 ? 8 : 4;
+    if (c % vec) return 0;
+    const int ho = (h + 2 * pad - k) / stride + 1, wo = (w + 2 * pad - k) / stride + 1;
+    return (int64_t)n * ho * wo * c;
+}
+
 int maxpool_forward(int dtype, int n, int h, int w, int c, int k, int stride, int pad, const void* x, void* y, const float* act, void* stream) {
     int ho = (h + 2 * pad - k) / stride + 1, wo = (w + 2 * pad - k) / stride + 1;
     if (maxpool_fuses_activation(dtype, h, w, c, k, stride, pad)) {
@@ -1246,7 +1324,7 @@ int maxpool_forward(int dtype, int n, int h, int w, int c, int k, int stride, in
 }
 
 int maxpool_backward(int dtype, int n, int h, int w, int c, int k, int stride, int pad, const void* x, const void* dy, void* dx, const float* act, void* stream,
-                     float* bn_partial, int* bn_blocks) {
+                     float* bn_partial, int* bn_blocks, void* scratch, int64_t scratch_bytes) {
     int ho = (h + 2 * pad - k) / stride + 1, wo = (w + 2 * pad - k) / stride + 1;
     if (bn_blocks) *bn_blocks = 0;
     if (maxpool_fuses_activation(dtype, h, w, c, k, stride, pad)) {
@@ -1272,6 +1350,23 @@ int maxpool_backward(int dtype, int n, int h, int w, int c, int k, int stride, i
         return CKPT_OK;
     }
     if (act) { set_error("the general pooling kernel takes an activated input"); return CKPT_E_BAD_ARG; }
+    const int64_t arg_bytes = maxpool_backward_scratch_bytes(dtype, n, h, w, c, k, stride, pad);
+    if (arg_bytes > 0 && scratch && scratch_bytes >= arg_bytes && ((uintptr_t)scratch & 7u) == 0) {
+        const int vec = dtype == CKPT_DTYPE_BF16 ? 8 : 4;
+        const int64_t windows = (int64_t)n * ho * wo * (c / vec), pixels = (int64_t)n * h * w * (c / vec);
+        cudaStream_t st = (cudaStream_t)stream;
+        if (dtype == CKPT_DTYPE_BF16) {
+            maxpool_argmax_kernel<__nv_bfloat16, 8><<<elementwise_grid(windows), 256, 0, st>>>((const __nv_bfloat16*)x, (uint8_t*)scratch, windows, h, w, c, ho, wo, k, stride, pad);
+            CKPT_LAUNCH_CHECK("max-pool arg-max");
+            maxpool_bwd_arg_kernel<__nv_bfloat16, 8><<<elementwise_grid(pixels), 256, 0, st>>>((const uint8_t*)scratch, (const __nv_bfloat16*)dy, (__nv_bfloat16*)dx, pixels, h, w, c, ho, wo, k, stride, pad);
+        } else {
+            maxpool_argmax_kernel<float, 4><<<elementwise_grid(windows), 256, 0, st>>>((const float*)x, (uint8_t*)scratch, windows, h, w, c, ho, wo, k, stride, pad);
+            CKPT_LAUNCH_CHECK("max-pool arg-max");
+            maxpool_bwd_arg_kernel<float, 4><<<elementwise_grid(pixels), 256, 0, st>>>((const uint8_t*)scratch, (const float*)dy, (float*)dx, pixels, h, w, c, ho, wo, k, stride, pad);
+        }
+        CKPT_LAUNCH_CHECK("max-pool backward from arg-max");
+        return CKPT_OK;
+    }
     if (c % bn_vec(dtype, c) == 0 && bn_vec(dtype, c) > 1) {
         const int64_t items = (int64_t)n * h * w * (c / bn_vec(dtype, c));
         if (dtype == CKPT_DTYPE_BF16)

@@ -301,7 +301,7 @@ def test_batchnorm_relu(rows, c, relu, dtype):
 
 @pytest.mark.parametrize("dtype", [ck.DTYPE_F32, ck.DTYPE_BF16])
 @pytest.mark.parametrize("n,h,w,c,k,stride,pad", [(2, 8, 6, 5, 2, 2, 0), (3, 13, 11, 8, 3, 2, 1), (2, 32, 32, 16, 2, 2, 0),
-                                                 (2, 20, 18, 64, 3, 2, 1), (2, 9, 9, 6, 3, 2, 1)])
+                                                 (2, 20, 18, 64, 3, 2, 1), (2, 9, 9, 6, 3, 2, 1), (2, 11, 14, 16, 3, 1, 1)])
 def test_maxpool(n, h, w, c, k, stride, pad, dtype):
     import torch
     rng = np.random.default_rng(h * w)
@@ -317,6 +317,14 @@ def test_maxpool(n, h, w, c, k, stride, pad, dtype):
     torch.cuda.synchronize()
     assert np.array_equal(to_host(y), y_ref)
     assert max_rel_err(to_host(dx), dx_ref) <= TIGHT[dtype]
+    # with scratch the general backward records the arg-max positions first and gathers from them: same result
+    sb = ck.maxpool_backward_scratch_bytes(dtype, n, h, w, c, k, stride, pad)
+    if sb > 0:
+        scratch = torch.full((sb,), 0xEE, dtype=torch.uint8, device="cuda")
+        dx2 = torch.full_like(xd, float("nan"))
+        ck.maxpool_backward(dtype, n, h, w, c, k, stride, pad, xd, dyd, dx2, scratch)
+        torch.cuda.synchronize()
+        assert torch.equal(dx2, dx)
 
 
 @pytest.mark.parametrize("dtype", [ck.DTYPE_F32, ck.DTYPE_BF16])
