@@ -449,6 +449,9 @@ struct TParams {
     int stages;
 };
 
+// A_MN (1x1 dgrad): the M operand is the forward filter [c_red][c_out] read in place, output channels contiguous:
+// two boxes of 64 reduction rows x 64 output channels per stage, an MN-major operand for the tensor core.
+template <bool A_MN>
 __global__ void __launch_bounds__(kThreads, 1)
 tc_conv_t_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w,
                  const __grid_constant__ CUtensorMap map_out, float* __restrict__ stat_partial, TParams p, int* status) {
@@ -506,7 +509,12 @@ tc_conv_t_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                 const int tap = it / blocks, blk = it % blocks;
                 const uint32_t a_dst = base + (uint32_t)s * stage_bytes;
                 mbar_expect_tx(full_bar(s), stage_bytes);
-                tma_load_2d(a_dst, &map_w, full_bar(s), p.tap_col[tap] * p.c_red + blk * 64, co_tile * 128);
+                if (A_MN) {
+                    tma_load_2d(a_dst, &map_w, full_bar(s), co_tile * 128, blk * 64);
+                    tma_load_2d(a_dst + 8192, &map_w, full_bar(s), co_tile * 128 + 64, blk * 64);
+                } else {
+                    tma_load_2d(a_dst, &map_w, full_bar(s), p.tap_col[tap] * p.c_red + blk * 64, co_tile * 128);
+                }
                 tma_load_4d(a_dst + a_bytes, &map_x, full_bar(s), blk * 64, w0 + p.tap_dw[tap], h0 + p.tap_dh[tap], n0);
             }
         }
@@ -515,7 +523,8 @@ tc_conv_t_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
         }
     } else if (warp == 1 && lane == 0) {
         // ---------------- MMA issuer
-        const uint32_t idesc = instr_desc(128, 256, 0, 0);
+        const uint32_t idesc = instr_desc(128, 256, A_MN ? 1 : 0, 0);
+        constexpr uint32_t a_step = A_MN ? 2048u : 32u, a_lbo = A_MN ? 8192u : 0u;
         bool ok = true;
         int g = 0;
         for (int j = 0; j < my_tiles && ok; ++j) {
@@ -530,7 +539,7 @@ tc_conv_t_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                 const uint32_t b_addr = a_addr + a_bytes;
 #pragma unroll
                 for (int kk = 0; kk < 4; ++kk)
-                    umma_bf16(acc, smem_desc(a_addr + kk * 32, 0, 1024), smem_desc(b_addr + kk * 32, 0, 1024), idesc,
+                    umma_bf16(acc, smem_desc(a_addr + kk * a_step, a_lbo, 1024), smem_desc(b_addr + kk * 32, 0, 1024), idesc,
                               (it > 0 || kk > 0) ? 1u : 0u);
                 umma_commit(empty_bar(s));
             }
@@ -1942,7 +1951,7 @@ bool t_applies(int c_red, int c_out, int k, int pad) {
     return (c_out % 128 == 0 || (c_out == 64 && c_red >= 128)) && c_red % 64 == 0 && ((k == 3 && pad == 1) || (k == 1 && pad == 0));
 }
 int launch_t(const void* x, const void* w_mat, void* out, float* stat_partial, int* stat_blocks, int N, int H, int W, int c_red,
-             int c_out, int k, int pad, int* status, cudaStream_t st, const char* what) {
+             int c_out, int k, int pad, int* status, cudaStream_t st, const char* what, bool a_mn = false) {
     TParams p;
     p.H = H; p.W = W; p.N = N; p.c_red = c_red; p.c_out = c_out;
     p.taps = k * k;
@@ -1962,7 +1971,7 @@ int launch_t(const void* x, const void* w_mat, void* out, float* stat_partial, i
     CUtensorMap mx, mw;
     int rc = make_act_map(&mx, x, N, H, W, c_red, p.tw, p.th, p.tn);
     if (rc) return rc;
-    rc = make_mat_map(&mw, w_mat, c_out, (int64_t)k * k * c_red, 128);
+    rc = a_mn ? make_mat_map(&mw, w_mat, c_red, c_out, 64) : make_mat_map(&mw, w_mat, c_out, (int64_t)k * k * c_red, 128);
     if (rc) return rc;
     // the box of one epilogue chunk: 32 consecutive pixels of the tile (w fastest) x 32 channels, no swizzle
     CUtensorMap mo;
@@ -1981,12 +1990,14 @@ int launch_t(const void* x, const void* w_mat, void* out, float* stat_partial, i
     const size_t smem = (size_t)p.stages * stage_bytes + 1024 + 256 + 4 * 2 * 2048;
     static bool attr_set = false;
     if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(tc_conv_t_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024);
+        cudaError_t e = cudaFuncSetAttribute(tc_conv_t_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_conv_t_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024);
         if (e != cudaSuccess) return cuda_fail(e, "raising the shared-memory limit");
         attr_set = true;
     }
     if (stat_blocks) *stat_blocks = stat_partial ? p.ctas_per_co : 0;
-    tc_conv_t_kernel<<<p.ctas_per_co * p.co_tiles, kThreads, smem, st>>>(mx, mw, mo, stat_blocks ? stat_partial : nullptr, p, status);
+    if (a_mn) tc_conv_t_kernel<true><<<p.ctas_per_co * p.co_tiles, kThreads, smem, st>>>(mx, mw, mo, stat_blocks ? stat_partial : nullptr, p, status);
+    else tc_conv_t_kernel<false><<<p.ctas_per_co * p.co_tiles, kThreads, smem, st>>>(mx, mw, mo, stat_blocks ? stat_partial : nullptr, p, status);
     CKPT_LAUNCH_CHECK(what);
     return CKPT_OK;
 }
@@ -1998,8 +2009,8 @@ int launch_fwd_like(const void* x, const void* w_mat, void* out, const float* bi
                     int* stat_blocks = nullptr, bool b_mn = false) {
     // b_mn (1x1 only): w_mat is the forward filter [c_red][c_out] read in place (c_out a multiple of 64)
     if (stat_blocks) *stat_blocks = 0;
-    if (!bias && !relu && !b_mn && t_applies(c_red, c_out, k, pad))
-        return launch_t(x, w_mat, out, stat_partial, stat_blocks, N, H, W, c_red, c_out, k, pad, status, st, what);
+    if (!bias && !relu && t_applies(c_red, c_out, k, pad) && (!b_mn || (k == 1 && (int64_t)N * H * W >= 256)))
+        return launch_t(x, w_mat, out, stat_partial, stat_blocks, N, H, W, c_red, c_out, k, pad, status, st, what, b_mn);
     if (c_red == 64 && k == 3 && pad == 1 && c_out % 64 == 0 && !bias && !relu)
         return launch_c64(x, w_mat, out, stat_partial, stat_blocks, N, H, W, c_out, status, st, what);
     if (!bias && !relu && halo_applies(H, W, c_red, c_out, k, pad))
