@@ -449,8 +449,9 @@ struct TParams {
     int stages;
 };
 
-// A_MN (1x1 dgrad): the M operand is the forward filter [c_red][c_out] read in place, output channels contiguous:
-// two boxes of 64 reduction rows x 64 output channels per stage, an MN-major operand for the tensor core.
+// A_MN (dgrad): the M operand is the forward filter [c_red][taps][c_out] read in place, output channels contiguous:
+// two boxes of 64 reduction rows x 64 output channels per stage (at the column block of the mirrored filter
+// position), an MN-major operand for the tensor core.  No transposed copy of the filter is made.
 template <bool A_MN>
 __global__ void __launch_bounds__(kThreads, 1)
 tc_conv_t_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w,
@@ -510,8 +511,10 @@ tc_conv_t_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                 const uint32_t a_dst = base + (uint32_t)s * stage_bytes;
                 mbar_expect_tx(full_bar(s), stage_bytes);
                 if (A_MN) {
-                    tma_load_2d(a_dst, &map_w, full_bar(s), co_tile * 128, blk * 64);
-                    tma_load_2d(a_dst + 8192, &map_w, full_bar(s), co_tile * 128 + 64, blk * 64);
+                    tma_load_2d(a_dst, &map_w, full_bar(s), p.tap_col[tap] * p.c_out + co_tile * 128, blk * 64);
+                    // (with 64 output channels the second box lies past them: it is sent outside the matrix, i.e. zero fill)
+                    tma_load_2d(a_dst + 8192, &map_w, full_bar(s),
+                                co_tile * 128 + 64 < p.c_out ? p.tap_col[tap] * p.c_out + co_tile * 128 + 64 : p.taps * p.c_out, blk * 64);
                 } else {
                     tma_load_2d(a_dst, &map_w, full_bar(s), p.tap_col[tap] * p.c_red + blk * 64, co_tile * 128);
                 }
@@ -1955,7 +1958,7 @@ int launch_t(const void* x, const void* w_mat, void* out, float* stat_partial, i
     TParams p;
     p.H = H; p.W = W; p.N = N; p.c_red = c_red; p.c_out = c_out;
     p.taps = k * k;
-    for (int t = 0; t < k * k; ++t) { p.tap_dh[t] = t / k - pad; p.tap_dw[t] = t % k - pad; p.tap_col[t] = t; }
+    for (int t = 0; t < k * k; ++t) { p.tap_dh[t] = t / k - pad; p.tap_dw[t] = t % k - pad; p.tap_col[t] = a_mn ? k * k - 1 - t : t; }
     choose_tile(256, W, H, N, &p.tw, &p.th, &p.tn);
     p.tw_log = 0; while ((1 << p.tw_log) < p.tw) ++p.tw_log;
     p.th_log = 0; while ((1 << p.th_log) < p.th) ++p.th_log;
@@ -1971,7 +1974,7 @@ int launch_t(const void* x, const void* w_mat, void* out, float* stat_partial, i
     CUtensorMap mx, mw;
     int rc = make_act_map(&mx, x, N, H, W, c_red, p.tw, p.th, p.tn);
     if (rc) return rc;
-    rc = a_mn ? make_mat_map(&mw, w_mat, c_red, c_out, 64) : make_mat_map(&mw, w_mat, c_out, (int64_t)k * k * c_red, 128);
+    rc = a_mn ? make_mat_map(&mw, w_mat, c_red, (int64_t)k * k * c_out, 64) : make_mat_map(&mw, w_mat, c_out, (int64_t)k * k * c_red, 128);
     if (rc) return rc;
     // the box of one epilogue chunk: 32 consecutive pixels of the tile (w fastest) x 32 channels, no swizzle
     CUtensorMap mo;
@@ -2348,6 +2351,9 @@ int tc_conv_dgrad(const ConvGeom& g, const void* dz, const void* w, void* dx, vo
         return launch_fwd_like(dz, w, dx, nullptr, 0, g.n, g.h, g.w, g.cout, g.cin, g.k, g.k - 1 - g.pad, device_status, st,
                                "conv dgrad (tensor cores)", nullptr, nullptr, true);
     }
+    if (t_applies(g.cout, g.cin, g.k, g.k - 1 - g.pad))
+        return launch_t(dz, w, dx, nullptr, nullptr, g.n, g.h, g.w, g.cout, g.cin, g.k, g.k - 1 - g.pad, device_status, st,
+                        "conv dgrad (tensor cores)", true);
     const int64_t elems = (int64_t)g.cout * taps * g.cin;
     if (!scratch || scratch_bytes < elems * 2) { set_error("dgrad scratch too small"); return CKPT_E_WORKSPACE; }
     const unsigned grid = (unsigned)std::min<int64_t>((elems + 255) / 256, 148 * 8);
