@@ -74,7 +74,7 @@ int ckpt_conv2d_bn_statistics(const ckpt_conv_shape* s, int dtype, const void* x
     if (tc_conv_supported(dtype, g)) {
         if (scratch_bytes < tc_conv_scratch_bytes(g)) { set_error("scratch too small for the convolution"); return CKPT_E_WORKSPACE; }
         int blocks = 0;
-        if ((rc = tc_conv_fwd_stats(g, x, w, z, (float*)scratch, &blocks, op_status_word(), stream))) return rc;
+        if ((rc = tc_conv_fwd_stats(g, x, w, z, (float*)scratch, &blocks, op_status_word(), stream, scratch_bytes))) return rc;
         if (blocks > 0) {
             if (fused) *fused = 1;
             return bn_statistics_from_partials((const float*)scratch, blocks, rows, g.cout, gamma, beta, stats, stream);

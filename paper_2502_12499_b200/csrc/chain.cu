@@ -131,7 +131,7 @@ static int conv_with_statistics(StepCtx& c, const ConvGeom& g, const void* x, co
     int rc;
     if (use_tc(c.ch, g) || (c.ch->impl == 0 && tc_first_conv_supported(dt, g))) {
         int blocks = 0;
-        if (use_tc(c.ch, g)) rc = tc_conv_fwd_stats(g, x, w, z, (float*)scr, &blocks, c.status(), c.stream);
+        if (use_tc(c.ch, g)) rc = tc_conv_fwd_stats(g, x, w, z, (float*)scr, &blocks, c.status(), c.stream, c.ch->scr_bytes);
         else rc = tc_first_conv_fwd(g, x, w, z, c.status(), c.stream, (float*)scr, &blocks);
         if (rc) return rc;
         if (blocks > 0) return bn_statistics_from_partials((const float*)scr, blocks, rows, g.cout, gamma, beta, stats, c.stream);

@@ -441,7 +441,9 @@ struct TParams {
     int H, W, N;                 // pixel grid walked by the tiles (= the output tensor: stride 1)
     int c_red, c_out;
     int taps;
-    int tap_dh[9], tap_dw[9], tap_col[9];
+    int tap_dh[12], tap_dw[12], tap_col[12];
+    int tap_xc[12];              // channel offset of a term's pixel box in the input view (pixel pairs: which pixel of the pair)
+    int fold;                    // 0, or 64: the 128 "channels" are (pixel of a pair, 64 channels) and the sums go to block 2*cta + pixel
     int tw_log, th_log;          // pixel tile tw x th x tn = 256, powers of two
     int tw, th, tn;
     int tiles_w, tiles_h, tiles_n;
@@ -518,7 +520,7 @@ tc_conv_t_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                 } else {
                     tma_load_2d(a_dst, &map_w, full_bar(s), p.tap_col[tap] * p.c_red + blk * 64, co_tile * 128);
                 }
-                tma_load_4d(a_dst + a_bytes, &map_x, full_bar(s), blk * 64, w0 + p.tap_dw[tap], h0 + p.tap_dh[tap], n0);
+                tma_load_4d(a_dst + a_bytes, &map_x, full_bar(s), blk * 64 + p.tap_xc[tap], w0 + p.tap_dw[tap], h0 + p.tap_dh[tap], n0);
             }
         }
         if (*failed) {
@@ -601,8 +603,14 @@ tc_conv_t_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
         if (lane == 0) tma_store_wait_all();
         if (stats && co < p.c_out) {
             // one partial row pair per CTA: [block][sum | sum of squares][channel]
-            stat_partial[((size_t)first * 2) * p.c_out + co] = sum;
-            stat_partial[((size_t)first * 2 + 1) * p.c_out + co] = sumsq;
+            if (p.fold) {
+                const size_t blk = (size_t)first * 2 + co / p.fold;
+                stat_partial[(blk * 2) * p.fold + co % p.fold] = sum;
+                stat_partial[(blk * 2 + 1) * p.fold + co % p.fold] = sumsq;
+            } else {
+                stat_partial[((size_t)first * 2) * p.c_out + co] = sum;
+                stat_partial[((size_t)first * 2 + 1) * p.c_out + co] = sumsq;
+            }
         }
     }
     tc_fence_before();
@@ -1726,6 +1734,22 @@ __global__ void fc_reduce_kernel(const float* __restrict__ partial, int slices, 
     out[e] = __float2bfloat16_rn(sum);
 }
 
+// Filter of the pixel-pair form of a 3x3 convolution with 64 output channels (see launch_t_paired):
+//   wp[(p, o)][(r, s'), red] = F[o][r][s' - p][red] for 0 <= s' - p <= 2, else 0,   p = 0, 1; s' = 0..3
+// with F the forward filter w[o][r][s][red] (flip = 0) or the filter of the input gradient
+// F[o][r][s][red] = w[red][2 - r][2 - s][o] (flip = 1; o runs over the forward input channels).
+__global__ void pair_filter_kernel(const __nv_bfloat16* __restrict__ w, __nv_bfloat16* __restrict__ wp, int c_red, int flip) {
+    const int total = 128 * 12 * c_red;
+    for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < total; i += gridDim.x * blockDim.x) {
+        const int red = i % c_red, term = (i / c_red) % 12, row = i / (12 * c_red);
+        const int p = row / 64, o = row % 64, r = term / 4, s = term % 4 - p;
+        __nv_bfloat16 v = __float2bfloat16_rn(0.f);
+        if (s >= 0 && s <= 2)
+            v = flip ? w[((size_t)red * 9 + (2 - r) * 3 + (2 - s)) * 64 + o] : w[((size_t)o * 9 + r * 3 + s) * c_red + red];
+        wp[i] = v;
+    }
+}
+
 // wt[ci][tap'][co] = w[co][taps-1-tap'][ci]: the matrix of the transposed convolution (stride 1).
 __global__ void transpose_flip_kernel(const __nv_bfloat16* __restrict__ w, __nv_bfloat16* __restrict__ wt, int c_out, int taps, int c_in) {
     const int64_t total = (int64_t)c_out * taps * c_in;
@@ -1953,12 +1977,11 @@ int launch_generic(FwdParams p, const void* a, int a_n, int a_h, int a_w, const 
 bool t_applies(int c_red, int c_out, int k, int pad) {
     return (c_out % 128 == 0 || (c_out == 64 && c_red >= 128)) && c_red % 64 == 0 && ((k == 3 && pad == 1) || (k == 1 && pad == 0));
 }
-int launch_t(const void* x, const void* w_mat, void* out, float* stat_partial, int* stat_blocks, int N, int H, int W, int c_red,
-             int c_out, int k, int pad, int* status, cudaStream_t st, const char* what, bool a_mn = false) {
-    TParams p;
+// The role-swapped kernel on prepared terms (p.taps, p.tap_*, p.fold): input [N][H][W][x_channels], output
+// [N][H][W][c_out], filter matrix as given by its tensor map.
+int launch_t_core(TParams p, const void* x, int x_channels, const CUtensorMap& mw, void* out, float* stat_partial, int* stat_blocks,
+                  int N, int H, int W, int c_red, int c_out, int* status, cudaStream_t st, const char* what, bool a_mn) {
     p.H = H; p.W = W; p.N = N; p.c_red = c_red; p.c_out = c_out;
-    p.taps = k * k;
-    for (int t = 0; t < k * k; ++t) { p.tap_dh[t] = t / k - pad; p.tap_dw[t] = t % k - pad; p.tap_col[t] = a_mn ? k * k - 1 - t : t; }
     choose_tile(256, W, H, N, &p.tw, &p.th, &p.tn);
     p.tw_log = 0; while ((1 << p.tw_log) < p.tw) ++p.tw_log;
     p.th_log = 0; while ((1 << p.th_log) < p.th) ++p.th_log;
@@ -1971,10 +1994,8 @@ int launch_t(const void* x, const void* w_mat, void* out, float* stat_partial, i
     p.ctas_per_co = std::max(1, std::min(p.p_tiles, sms / p.co_tiles));
     constexpr uint32_t stage_bytes = 128 * 128 + 256 * 128;
     p.stages = std::min<int>(kMaxStages, kSmemBudget / stage_bytes);
-    CUtensorMap mx, mw;
-    int rc = make_act_map(&mx, x, N, H, W, c_red, p.tw, p.th, p.tn);
-    if (rc) return rc;
-    rc = a_mn ? make_mat_map(&mw, w_mat, c_red, (int64_t)k * k * c_out, 64) : make_mat_map(&mw, w_mat, c_out, (int64_t)k * k * c_red, 128);
+    CUtensorMap mx;
+    int rc = make_act_map(&mx, x, N, H, W, x_channels, p.tw, p.th, p.tn);
     if (rc) return rc;
     // the box of one epilogue chunk: 32 consecutive pixels of the tile (w fastest) x 32 channels, no swizzle
     CUtensorMap mo;
@@ -1998,20 +2019,68 @@ int launch_t(const void* x, const void* w_mat, void* out, float* stat_partial, i
         if (e != cudaSuccess) return cuda_fail(e, "raising the shared-memory limit");
         attr_set = true;
     }
-    if (stat_blocks) *stat_blocks = stat_partial ? p.ctas_per_co : 0;
+    if (stat_blocks) *stat_blocks = stat_partial ? (p.fold ? 2 : 1) * p.ctas_per_co : 0;
     if (a_mn) tc_conv_t_kernel<true><<<p.ctas_per_co * p.co_tiles, kThreads, smem, st>>>(mx, mw, mo, stat_blocks ? stat_partial : nullptr, p, status);
     else tc_conv_t_kernel<false><<<p.ctas_per_co * p.co_tiles, kThreads, smem, st>>>(mx, mw, mo, stat_blocks ? stat_partial : nullptr, p, status);
     CKPT_LAUNCH_CHECK(what);
     return CKPT_OK;
 }
 
+int launch_t(const void* x, const void* w_mat, void* out, float* stat_partial, int* stat_blocks, int N, int H, int W, int c_red,
+             int c_out, int k, int pad, int* status, cudaStream_t st, const char* what, bool a_mn = false) {
+    TParams p;
+    p.taps = k * k;
+    p.fold = 0;
+    for (int t = 0; t < k * k; ++t) {
+        p.tap_dh[t] = t / k - pad; p.tap_dw[t] = t % k - pad; p.tap_col[t] = a_mn ? k * k - 1 - t : t; p.tap_xc[t] = 0;
+    }
+    CUtensorMap mw;
+    int rc = a_mn ? make_mat_map(&mw, w_mat, c_red, (int64_t)k * k * c_out, 64) : make_mat_map(&mw, w_mat, c_out, (int64_t)k * k * c_red, 128);
+    if (rc) return rc;
+    return launch_t_core(p, x, c_red, mw, out, stat_partial, stat_blocks, N, H, W, c_red, c_out, status, st, what, a_mn);
+}
+
+// 3x3, padding 1, 64 output channels, even width: two horizontally adjacent pixels are treated as one pixel with
+// 128 output channels (pixel of the pair, channel), so that the role-swapped kernel's M operand is full.  The pair
+// at column j reads input columns 2j-1 .. 2j+2: per filter row four terms - the odd pixel of pair j-1, both pixels
+// of pair j, the even pixel of pair j+1 - each a plain (aligned) box of the input viewed as [N][H][W/2][2*c_red].
+// A third of the products multiply zeros of the widened filter, but every instruction is 128 x 256 x 16 instead of
+// 128 x 64 x 16 at the same issue interval.  `work`: 128 * 12 * c_red bf16 for the widened filter.
+int64_t paired_work_bytes(int c_red) { return align_up((int64_t)128 * 12 * c_red * 2, 256); }
+// (on small tensors the 64-channel kernel with its resident filter is as fast: 32 x 56 x 56 pixels 0.023 against 0.026 ms)
+bool paired_applies(int c_red, int c_out, int k, int pad, int W, int64_t pixels) {
+    return c_out == 64 && k == 3 && pad == 1 && W % 2 == 0 && c_red % 64 == 0 && pixels >= 262144;
+}
+int launch_t_paired(const void* x, const void* w, int flip, void* out, float* stat_partial, int* stat_blocks, int N, int H, int W,
+                    int c_red, void* work, int* status, cudaStream_t st, const char* what) {
+    __nv_bfloat16* wp = (__nv_bfloat16*)work;
+    pair_filter_kernel<<<std::min(128 * 12 * c_red / 256, 148 * 8), 256, 0, st>>>((const __nv_bfloat16*)w, wp, c_red, flip);
+    CKPT_LAUNCH_CHECK("pixel-pair filter");
+    TParams p;
+    p.taps = 12;
+    p.fold = 64;
+    for (int t = 0; t < 12; ++t) {
+        const int r = t / 4, sp = t % 4;
+        p.tap_dh[t] = r - 1;
+        p.tap_dw[t] = sp == 0 ? -1 : (sp == 3 ? 1 : 0);
+        p.tap_xc[t] = (sp == 0 || sp == 2) ? c_red : 0;
+        p.tap_col[t] = t;
+    }
+    CUtensorMap mw;
+    int rc = make_mat_map(&mw, wp, 128, (int64_t)12 * c_red, 128);
+    if (rc) return rc;
+    return launch_t_core(p, x, 2 * c_red, mw, out, stat_partial, stat_blocks, N, H, W / 2, c_red, 128, status, st, what, false);
+}
+
 // stat_partial / stat_blocks: null, or where the kernel leaves the batch-norm partial sums of its output
 // ([block][sum | sum of squares][c_out] floats) and how many blocks it wrote (0 = this kernel does not gather them).
 int launch_fwd_like(const void* x, const void* w_mat, void* out, const float* bias, int relu, int N, int H, int W, int c_red,
                     int c_out, int k, int pad, int* status, cudaStream_t st, const char* what, float* stat_partial = nullptr,
-                    int* stat_blocks = nullptr, bool b_mn = false) {
+                    int* stat_blocks = nullptr, bool b_mn = false, void* work = nullptr, int64_t work_bytes = 0) {
     // b_mn (1x1 only): w_mat is the forward filter [c_red][c_out] read in place (c_out a multiple of 64)
     if (stat_blocks) *stat_blocks = 0;
+    if (!bias && !relu && !b_mn && paired_applies(c_red, c_out, k, pad, W, (int64_t)N * H * W) && work && work_bytes >= paired_work_bytes(c_red))
+        return launch_t_paired(x, w_mat, 0, out, stat_partial, stat_blocks, N, H, W, c_red, work, status, st, what);
     if (!bias && !relu && t_applies(c_red, c_out, k, pad) && (!b_mn || (k == 1 && (int64_t)N * H * W >= 256)))
         return launch_t(x, w_mat, out, stat_partial, stat_blocks, N, H, W, c_red, c_out, k, pad, status, st, what, b_mn);
     if (c_red == 64 && k == 3 && pad == 1 && c_out % 64 == 0 && !bias && !relu)
@@ -2193,7 +2262,11 @@ static int64_t tc_conv_stat_bytes(const ConvGeom& g) {
 
 static int64_t tc_conv_work_bytes(const ConvGeom& g);
 int64_t tc_conv_scratch_bytes(const ConvGeom& g) {
-    return std::max(std::max(tc_conv_stat_bytes(g), tc_conv_work_bytes(g)), fc_scratch_bytes(g));
+    int64_t b = std::max(std::max(tc_conv_stat_bytes(g), tc_conv_work_bytes(g)), fc_scratch_bytes(g));
+    if (g.stride == 1 && (paired_applies(g.cin, g.cout, g.k, g.pad, g.w, (int64_t)g.n * g.h * g.w) ||
+                          paired_applies(g.cout, g.cin, g.k, g.k - 1 - g.pad, g.w, (int64_t)g.n * g.h * g.w)))
+        b = std::max<int64_t>(b, (1 << 20) + 2 * paired_work_bytes(std::max(g.cin, g.cout)));
+    return b;
 }
 
 // partial sums of the split weight gradient, or the transposed filter of the input gradient
@@ -2268,16 +2341,25 @@ static int launch_strided_fwd(const ConvGeom& g, const void* x, const void* w, v
                           "strided conv forward (tensor cores)", false, stat_partial, stat_blocks);
 }
 
+// The widened filter of the pixel-pair form lives at the end of the caller's scratch region (its start holds
+// the partial sums); null when the region is too small.
+static void* paired_region(void* scratch, int64_t scratch_bytes, int c_red) {
+    const int64_t need = paired_work_bytes(c_red);
+    if (!scratch || scratch_bytes < need + (1 << 20)) return nullptr;
+    return (char*)scratch + ((scratch_bytes - need) & ~(int64_t)255);
+}
+
 // Forward convolution that also leaves the batch-norm partial sums of its output in `partial`
 // (*blocks of them; 0 when the kernel chosen for this shape does not gather them).
 int tc_conv_fwd_stats(const ConvGeom& g, const void* x, const void* w, void* z, float* partial, int* blocks, int* device_status,
-                      void* stream) {
+                      void* stream, int64_t partial_bytes) {
     if (!tc_conv_supported(CKPT_DTYPE_BF16, g)) { set_error("tensor-core conv: unsupported shape"); return CKPT_E_UNSUPPORTED; }
     if (!device_status || !blocks) { set_error("device status word missing"); return CKPT_E_NULL; }
     *blocks = 0;
     if (g.stride != 1) return launch_strided_fwd(g, x, w, z, device_status, (cudaStream_t)stream, partial, blocks);
     return launch_fwd_like(x, w, z, nullptr, 0, g.n, g.h, g.w, g.cin, g.cout, g.k, g.pad, device_status, (cudaStream_t)stream,
-                           "conv forward (tensor cores)", partial, blocks);
+                           "conv forward (tensor cores)", partial, blocks, false, paired_region(partial, partial_bytes, g.cin),
+                           paired_work_bytes(g.cin));
 }
 
 int tc_conv_fwd(const ConvGeom& g, const void* x, const void* w, void* z, const float* bias, int relu, void* scratch,
@@ -2290,7 +2372,8 @@ int tc_conv_fwd(const ConvGeom& g, const void* x, const void* w, void* z, const 
         return launch_strided_fwd(g, x, w, z, device_status, (cudaStream_t)stream);
     }
     return launch_fwd_like(x, w, z, bias, relu, g.n, g.h, g.w, g.cin, g.cout, g.k, g.pad, device_status, (cudaStream_t)stream,
-                           "conv forward (tensor cores)");
+                           "conv forward (tensor cores)", nullptr, nullptr, false, paired_region(scratch, scratch_bytes, g.cin),
+                           paired_work_bytes(g.cin));
 }
 
 int tc_conv_dgrad(const ConvGeom& g, const void* dz, const void* w, void* dx, void* scratch, int64_t scratch_bytes,
@@ -2350,6 +2433,11 @@ int tc_conv_dgrad(const ConvGeom& g, const void* dz, const void* w, void* dx, vo
         // and measured 10-30 % slower than a transposed copy, which costs under 10 us per layer.)
         return launch_fwd_like(dz, w, dx, nullptr, 0, g.n, g.h, g.w, g.cout, g.cin, g.k, g.k - 1 - g.pad, device_status, st,
                                "conv dgrad (tensor cores)", nullptr, nullptr, true);
+    }
+    if (paired_applies(g.cout, g.cin, g.k, g.k - 1 - g.pad, g.w, (int64_t)g.n * g.h * g.w)) {
+        // 64 input channels: the pixel-pair form, its widened filter built straight from the forward filter
+        if (void* work = paired_region(scratch, scratch_bytes, g.cout))
+            return launch_t_paired(dz, w, 1, dx, nullptr, nullptr, g.n, g.h, g.w, g.cout, work, device_status, st, "conv dgrad (tensor cores)");
     }
     if (t_applies(g.cout, g.cin, g.k, g.k - 1 - g.pad))
         return launch_t(dz, w, dx, nullptr, nullptr, g.n, g.h, g.w, g.cout, g.cin, g.k, g.k - 1 - g.pad, device_status, st,

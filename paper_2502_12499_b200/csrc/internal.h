@@ -95,7 +95,8 @@ int tc_conv_fwd(const ConvGeom& g, const void* x, const void* w, void* z, const 
 // Forward that also writes the batch-norm partial sums of its output ([blocks][sum | sum of squares][c_out]
 // floats, at most 4 per SM); *blocks == 0 when the kernel for this shape does not gather them.
 int tc_conv_fwd_stats(const ConvGeom& g, const void* x, const void* w, void* z, float* partial, int* blocks,
-                      int* device_status, void* stream);
+                      int* device_status, void* stream,
+                      int64_t partial_bytes = 0);
 int tc_conv_dgrad(const ConvGeom& g, const void* dz, const void* w, void* dx, void* scratch,
                   int64_t scratch_bytes, int* device_status, void* stream);
 int tc_conv_wgrad(const ConvGeom& g, const void* dz, const void* x, float* dw, void* scratch,

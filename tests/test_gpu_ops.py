@@ -51,6 +51,10 @@ TC_CASES = [
     (2, 28, 24, 128, 256, 3, 1),     # halo-patch kernel, 14-row tiles, 256-wide output tile
     (2, 32, 16, 192, 64, 3, 1),      # halo-patch kernel, three channel blocks, 64-wide output tile
     (2, 112, 112, 128, 128, 3, 1),   # halo-patch kernel, several tiles per persistent CTA
+    # pixel-pair form of 64-channel outputs (large tensors only): forward 64 -> 64 and 128 -> 64, dgrad into 64 channels
+    (5, 232, 228, 64, 64, 3, 1),     # ragged tiles in every dimension, pairs across tile borders
+    (3, 300, 296, 128, 64, 3, 1),    # two reduction blocks per term
+    (3, 300, 296, 64, 128, 3, 1),    # its dgrad: 128 reduction channels, filter widened from the forward filter
     # stride 2 (8th field): strided operand boxes forward and in wgrad, one stride-1 sum per parity class in dgrad
     (2, 28, 28, 128, 128, 3, 1, 2),  # first 3x3 of a residual stage
     (3, 15, 13, 64, 192, 3, 1, 2),   # odd sizes: ragged parity classes
@@ -201,6 +205,7 @@ def test_stem_kernels(n, h, w, cout):
 
 @pytest.mark.parametrize("case,expect_fused", [
     ((8, 56, 56, 64, 64, 3, 1), True),        # 64-channel persistent kernel, two tiles for some CTAs
+    ((5, 232, 228, 64, 64, 3, 1), True),      # pixel-pair form: sums of the two pixels of a pair in separate partial rows
     ((3, 13, 19, 64, 128, 3, 1), True),       # ragged tiles: rows outside the image must not count
     ((2, 112, 112, 128, 128, 3, 1), True),    # halo-patch kernel, 128-wide output tile
     ((4, 56, 56, 128, 256, 3, 1), True),      # halo-patch kernel, 256-wide output tile
