@@ -51,6 +51,11 @@ TC_CASES = [
     (2, 28, 24, 128, 256, 3, 1),     # halo-patch kernel, 14-row tiles, 256-wide output tile
     (2, 32, 16, 192, 64, 3, 1),      # halo-patch kernel, three channel blocks, 64-wide output tile
     (2, 112, 112, 128, 128, 3, 1),   # halo-patch kernel, several tiles per persistent CTA
+    # role-swapped kernel corner cases: a single partial pixel tile, three output-channel tiles, 64 outputs without pairs
+    (1, 5, 7, 128, 128, 3, 1),
+    (2, 9, 11, 192, 384, 1, 0),
+    (3, 10, 6, 256, 64, 3, 1),
+    (1, 515, 510, 64, 64, 3, 1),     # pixel pairs, one image, odd height
     # pixel-pair form of 64-channel outputs (large tensors only): forward 64 -> 64 and 128 -> 64, dgrad into 64 channels
     (5, 232, 228, 64, 64, 3, 1),     # ragged tiles in every dimension, pairs across tile borders
     (3, 300, 296, 128, 64, 3, 1),    # two reduction blocks per term
