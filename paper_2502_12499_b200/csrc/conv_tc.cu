@@ -1253,6 +1253,11 @@ struct WRowsParams {
     int slices;                  // persistent CTAs along the pixel range
     int stages;
     uint32_t dz_box, patch_bytes, stage_bytes;
+    // pixel-pair view (64 input channels, see tc_conv_wgrad): the tensors are read as [N][H][W/2][2C], c_out counts the
+    // rows (pixel of the pair, output channel), and the four columns are the 64-channel halves of the pairs one to the
+    // left, at, and one to the right of the output pair that a 3-wide filter row can reach
+    int pairview;
+    int row_elems;               // floats per partial row: 9 * c_in, or 4 columns * 3 * 64 in the pair view
 };
 
 __global__ void __launch_bounds__(kThreads, 1)
@@ -1303,8 +1308,10 @@ tc_wgrad_rows_kernel(const __grid_constant__ CUtensorMap map_dz, const __grid_co
             if (lane < 2) {
                 tma_load_4d(dst + lane * p.dz_box, &map_dz, full_bar(s), co_tile * 128 + 64 * lane, w0, h0, img);
             } else if (lane < 4) {
-                const int col = 2 * pair + (lane - 2), cib = col / 3, dx = col % 3;
-                tma_load_4d(dst + 2 * p.dz_box + (lane - 2) * p.patch_bytes, &map_x, full_bar(s), cib * 64, w0 + dx - 1, h0 - 1, img);
+                const int col = 2 * pair + (lane - 2);
+                const int ch = p.pairview ? ((col + 1) & 1) * 64 : (col / 3) * 64;
+                const int shift = p.pairview ? (col + 1) / 2 - 1 : col % 3 - 1;
+                tma_load_4d(dst + 2 * p.dz_box + (lane - 2) * p.patch_bytes, &map_x, full_bar(s), ch, w0 + shift, h0 - 1, img);
             }
             issued = j + 1;
         }
@@ -1333,14 +1340,15 @@ tc_wgrad_rows_kernel(const __grid_constant__ CUtensorMap map_dz, const __grid_co
         const int quarter = warp % 4;
         const int co = co_tile * 128 + quarter * 32 + lane;
         const bool valid = co < p.c_out;
-        const size_t row_elems = (size_t)9 * p.c_in;
+        const size_t row_elems = (size_t)p.row_elems;
         float* dst_row = partial + ((size_t)slice * p.c_out + (valid ? co : 0)) * row_elems;
         if (my_tiles > 0 && mbar_wait(accum_bar, 0, failed, status, 703)) {
             tc_fence_after();
             for (int c = 0; c < 2; ++c) {
                 const int col = 2 * pair + c, cib = col / 3, dx = col % 3;
                 for (int dy = 0; dy < 3; ++dy) {
-                    float* dst = dst_row + (size_t)((dy * 3 + dx) * cin_blocks + cib) * 64;   // column (tap, c_in)
+                    float* dst = dst_row + (p.pairview ? (size_t)(col * 3 + dy) * 64
+                                                       : (size_t)((dy * 3 + dx) * cin_blocks + cib) * 64);   // column (tap, c_in)
 #pragma unroll
                     for (int c0 = 0; c0 < 64; c0 += 32) {
                         uint32_t v[32];
@@ -1357,8 +1365,10 @@ tc_wgrad_rows_kernel(const __grid_constant__ CUtensorMap map_dz, const __grid_co
         } else if (my_tiles == 0 && valid) {
             for (int c = 0; c < 2; ++c) {
                 const int col = 2 * pair + c, cib = col / 3, dx = col % 3;
-                for (int dy = 0; dy < 3; ++dy)
-                    for (int e = 0; e < 64; ++e) dst_row[(size_t)((dy * 3 + dx) * cin_blocks + cib) * 64 + e] = 0.f;
+                for (int dy = 0; dy < 3; ++dy) {
+                    float* dst = dst_row + (p.pairview ? (size_t)(col * 3 + dy) * 64 : (size_t)((dy * 3 + dx) * cin_blocks + cib) * 64);
+                    for (int e = 0; e < 64; ++e) dst[e] = 0.f;
+                }
             }
         }
     }
@@ -1759,6 +1769,20 @@ __global__ void transpose_flip_kernel(const __nv_bfloat16* __restrict__ w, __nv_
         const int tap = (int)(t % taps), ci = (int)(t / taps);
         wt[i] = w[((size_t)co * taps + (taps - 1 - tap)) * c_in + ci];
     }
+}
+
+// Pair-view wgrad partials [slice][(q, c_out)][column 4][dy 3][c_in 64] -> dW[c_out][dy][dx][c_in]: pixel q of a pair
+// sees filter column dx in accumulator column dx + q.
+__global__ void pairview_fold_kernel(const float* __restrict__ partial, float* __restrict__ out, int c_out, int slices) {
+    const int idx = blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= c_out * 576) return;
+    const int ci = idx % 64, dx = (idx / 64) % 3, dy = (idx / 192) % 3, co = idx / 576;
+    const float* p0 = partial + (size_t)co * 768 + (dx * 3 + dy) * 64 + ci;
+    const float* p1 = partial + (size_t)(c_out + co) * 768 + ((dx + 1) * 3 + dy) * 64 + ci;
+    const size_t slice_stride = (size_t)2 * c_out * 768;
+    float acc = 0.f;
+    for (int s = 0; s < slices; ++s) acc += p0[s * slice_stride] + p1[s * slice_stride];
+    out[idx] = acc;
 }
 
 __global__ void slice_sum_tc_kernel(const float* __restrict__ partial, float* __restrict__ out, int64_t elems, int slices) {
@@ -2239,6 +2263,30 @@ void wgrad_rows_plan(const ConvGeom& g, WRowsParams* p, int* pairs, int* co_tile
     p->patch_bytes = (uint32_t)(8 * (p->th + 2)) * 128;
     p->stage_bytes = 2 * p->dz_box + 2 * p->patch_bytes;
     p->stages = std::max(2, std::min<int>(kMaxStages, (int)((208 * 1024) / p->stage_bytes)));
+    p->pairview = 0;
+    p->row_elems = 9 * g.cin;
+}
+
+// 64 input channels through the same kernel.  Two horizontally adjacent pixels are read as one pixel of twice the
+// channels (the tensors as [N][H][W/2][2C], no copy), so dz gives 128-row operands even for 64 output channels:
+// row (q, c_out) is output channel c_out at pixel q of the pair.  A 3-wide filter row reaches, from pair j, the
+// second pixel of pair j-1, both pixels of pair j and the first pixel of pair j+1: four columns of 64 input
+// channels, each with its three vertical taps as before.  Row (0, co) uses columns 0..2 as dx = 0..2 and row (1, co)
+// columns 1..3; the other quarter of the accumulator is discarded by the fold that also sums the slices.
+bool wgrad_pairview_applies(const ConvGeom& g) {
+    return g.cin == 64 && g.k == 3 && g.pad == 1 && g.stride == 1 && g.cout % 64 == 0 && g.w % 2 == 0 && g.w >= 2 * WROWS_MIN_W && g.h >= 8;
+}
+void wgrad_pairview_plan(const ConvGeom& g, WRowsParams* p, int* co_tiles) {
+    ConvGeom v = g;
+    v.w = g.w / 2; v.wo = v.w; v.cin = 128; v.cout = 2 * g.cout;
+    int pairs;
+    wgrad_rows_plan(v, p, &pairs, co_tiles);
+    int sms = 148, dev = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    p->slices = std::max(1, std::min(sms / (2 * *co_tiles), p->m_tiles));
+    p->pairview = 1;
+    p->row_elems = 4 * 3 * 64;
 }
 }  // namespace
 
@@ -2271,6 +2319,12 @@ int64_t tc_conv_scratch_bytes(const ConvGeom& g) {
 
 // partial sums of the split weight gradient, or the transposed filter of the input gradient
 static int64_t tc_conv_work_bytes(const ConvGeom& g) {
+    if (wgrad_pairview_applies(g)) {
+        WRowsParams q;
+        int tiles;
+        wgrad_pairview_plan(g, &q, &tiles);
+        return std::max<int64_t>((int64_t)q.slices * 2 * g.cout * q.row_elems * 4, (int64_t)g.cout * 576 * 2);
+    }
     if (wgrad_c64_applies(g)) {
         W64Params q;
         wgrad_c64_plan(g, &q);
@@ -2451,9 +2505,40 @@ int tc_conv_dgrad(const ConvGeom& g, const void* dz, const void* w, void* dx, vo
                            "conv dgrad (tensor cores)");
 }
 
+static int wgrad_rows_attr() {
+    static bool attr_set = false;
+    if (!attr_set) {
+        cudaError_t e = cudaFuncSetAttribute(tc_wgrad_rows_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 222 * 1024);
+        if (e != cudaSuccess) return cuda_fail(e, "raising the shared-memory limit");
+        attr_set = true;
+    }
+    return CKPT_OK;
+}
+
 int tc_conv_wgrad(const ConvGeom& g, const void* dz, const void* x, float* dw, void* scratch, int64_t scratch_bytes,
                   int* device_status, void* stream) {
     if (!device_status) { set_error("no status word"); return CKPT_E_NULL; }
+    if (wgrad_pairview_applies(g)) {
+        WRowsParams p;
+        int co_tiles;
+        wgrad_pairview_plan(g, &p, &co_tiles);
+        if (!scratch || scratch_bytes < (int64_t)p.slices * 2 * g.cout * p.row_elems * 4) { set_error("wgrad scratch too small"); return CKPT_E_WORKSPACE; }
+        CUtensorMap mdz, mx;
+        int rc = make_act_map(&mdz, dz, g.n, g.h, g.w / 2, 2 * g.cout, 8, p.th, 1);
+        if (rc) return rc;
+        rc = make_act_map(&mx, x, g.n, g.h, g.w / 2, 128, 8, p.th + 2, 1);
+        if (rc) return rc;
+        cudaStream_t st = (cudaStream_t)stream;
+        rc = wgrad_rows_attr();
+        if (rc) return rc;
+        const size_t smem = (size_t)p.stages * p.stage_bytes + 1024 + 256;
+        dim3 grid(p.slices, 2, co_tiles);
+        tc_wgrad_rows_kernel<<<grid, kThreads, smem, st>>>(mdz, mx, (float*)scratch, p, device_status);
+        CKPT_LAUNCH_CHECK("conv wgrad, 64 input channels as pixel pairs (tensor cores)");
+        pairview_fold_kernel<<<(unsigned)((g.cout * 576 + 255) / 256), 256, 0, st>>>((const float*)scratch, dw, g.cout, p.slices);
+        CKPT_LAUNCH_CHECK("wgrad pair fold");
+        return CKPT_OK;
+    }
     if (wgrad_c64_applies(g)) {
         W64Params p;
         wgrad_c64_plan(g, &p);
@@ -2491,12 +2576,8 @@ int tc_conv_wgrad(const ConvGeom& g, const void* dz, const void* x, float* dw, v
         rc = make_act_map(&mx, x, g.n, g.h, g.w, g.cin, 8, p.th + 2, 1);
         if (rc) return rc;
         cudaStream_t st = (cudaStream_t)stream;
-        static bool attr_set = false;
-        if (!attr_set) {
-            cudaError_t e = cudaFuncSetAttribute(tc_wgrad_rows_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 222 * 1024);
-            if (e != cudaSuccess) return cuda_fail(e, "raising the shared-memory limit");
-            attr_set = true;
-        }
+        rc = wgrad_rows_attr();
+        if (rc) return rc;
         const size_t smem = (size_t)p.stages * p.stage_bytes + 1024 + 256;
         dim3 grid(p.slices, pairs, co_tiles);
         tc_wgrad_rows_kernel<<<grid, kThreads, smem, st>>>(mdz, mx, (float*)scratch, p, device_status);
