@@ -1771,18 +1771,54 @@ __global__ void transpose_flip_kernel(const __nv_bfloat16* __restrict__ w, __nv_
     }
 }
 
+__device__ __forceinline__ void add4(float4& a, const float4 b) { a.x += b.x; a.y += b.y; a.z += b.z; a.w += b.w; }
+
+// The split kernels leave one partial result per persistent CTA (some tens of MB, mostly still in L2) for a few
+// hundred thousand outputs: a thread per output would leave most SMs idle and one load in flight per thread.  A block
+// is 32 float4 columns x Y slice groups; group y sums slices y, y + Y, ... and the groups are added in a fixed order.
+template <int Y>
+__device__ __forceinline__ void store_group_sum(float4 acc, float4* out, bool ok) {
+    __shared__ float4 red[Y][32];
+    if (Y > 1) {
+        red[threadIdx.y][threadIdx.x] = acc;
+        __syncthreads();
+        if (threadIdx.y == 0)
+            for (int y = 1; y < Y; ++y) add4(acc, red[y][threadIdx.x]);
+    }
+    if (threadIdx.y == 0 && ok) *out = acc;
+}
+
 // Pair-view wgrad partials [slice][(q, c_out)][column 4][dy 3][c_in 64] -> dW[c_out][dy][dx][c_in]: pixel q of a pair
 // sees filter column dx in accumulator column dx + q.
-__global__ void pairview_fold_kernel(const float* __restrict__ partial, float* __restrict__ out, int c_out, int slices) {
-    const int idx = blockIdx.x * blockDim.x + threadIdx.x;
-    if (idx >= c_out * 576) return;
-    const int ci = idx % 64, dx = (idx / 64) % 3, dy = (idx / 192) % 3, co = idx / 576;
+template <int Y>
+__global__ void __launch_bounds__(32 * Y) pairview_fold_kernel(const float* __restrict__ partial, float* __restrict__ out, int c_out, int slices) {
+    const int idx = blockIdx.x * 32 + threadIdx.x;            // one float4 of the output
+    const bool ok = idx < c_out * 144;
+    const int ci = (idx % 16) * 4, dx = (idx / 16) % 3, dy = (idx / 48) % 3, co = ok ? idx / 144 : 0;
     const float* p0 = partial + (size_t)co * 768 + (dx * 3 + dy) * 64 + ci;
     const float* p1 = partial + (size_t)(c_out + co) * 768 + ((dx + 1) * 3 + dy) * 64 + ci;
     const size_t slice_stride = (size_t)2 * c_out * 768;
-    float acc = 0.f;
-    for (int s = 0; s < slices; ++s) acc += p0[s * slice_stride] + p1[s * slice_stride];
-    out[idx] = acc;
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (ok) {
+#pragma unroll 4
+        for (int z = threadIdx.y; z < slices; z += Y) {
+            add4(acc, *reinterpret_cast<const float4*>(p0 + z * slice_stride));
+            add4(acc, *reinterpret_cast<const float4*>(p1 + z * slice_stride));
+        }
+    }
+    store_group_sum<Y>(acc, reinterpret_cast<float4*>(out) + idx, ok);
+}
+
+template <int Y>
+__global__ void __launch_bounds__(32 * Y) slice_sum4_kernel(const float4* __restrict__ partial, float4* __restrict__ out, int64_t elems4, int slices) {
+    const int64_t e = (int64_t)blockIdx.x * 32 + threadIdx.x;
+    const bool ok = e < elems4;
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (ok) {
+#pragma unroll 4
+        for (int z = threadIdx.y; z < slices; z += Y) add4(acc, partial[(size_t)z * elems4 + e]);
+    }
+    store_group_sum<Y>(acc, out + e, ok);
 }
 
 __global__ void slice_sum_tc_kernel(const float* __restrict__ partial, float* __restrict__ out, int64_t elems, int slices) {
@@ -1791,6 +1827,19 @@ __global__ void slice_sum_tc_kernel(const float* __restrict__ partial, float* __
     float s = 0.f;
     for (int z = 0; z < slices; ++z) s += partial[(size_t)z * elems + e];
     out[e] = s;
+}
+
+// sum of the `slices` partial results of a split wgrad into the caller's gradient
+static void launch_slice_sum(const float* partial, float* out, int64_t elems, int slices, cudaStream_t st) {
+    if (elems % 4 || ((uintptr_t)partial | (uintptr_t)out) % 16) {
+        slice_sum_tc_kernel<<<(unsigned)((elems + 255) / 256), 256, 0, st>>>(partial, out, elems, slices);
+        return;
+    }
+    const int64_t elems4 = elems / 4;
+    const unsigned blocks = (unsigned)((elems4 + 31) / 32);
+    if (slices >= 16) slice_sum4_kernel<8><<<blocks, dim3(32, 8), 0, st>>>((const float4*)partial, (float4*)out, elems4, slices);
+    else if (slices >= 4) slice_sum4_kernel<4><<<blocks, dim3(32, 4), 0, st>>>((const float4*)partial, (float4*)out, elems4, slices);
+    else slice_sum4_kernel<1><<<blocks, dim3(32, 1), 0, st>>>((const float4*)partial, (float4*)out, elems4, slices);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -2518,7 +2567,7 @@ static int wgrad_rows_attr() {
 int tc_conv_wgrad(const ConvGeom& g, const void* dz, const void* x, float* dw, void* scratch, int64_t scratch_bytes,
                   int* device_status, void* stream) {
     if (!device_status) { set_error("no status word"); return CKPT_E_NULL; }
-    if (wgrad_pairview_applies(g)) {
+    if (wgrad_pairview_applies(g) && (uintptr_t)dw % 16 == 0) {      // the fold stores float4; otherwise the 64-channel kernel below
         WRowsParams p;
         int co_tiles;
         wgrad_pairview_plan(g, &p, &co_tiles);
@@ -2535,7 +2584,7 @@ int tc_conv_wgrad(const ConvGeom& g, const void* dz, const void* x, float* dw, v
         dim3 grid(p.slices, 2, co_tiles);
         tc_wgrad_rows_kernel<<<grid, kThreads, smem, st>>>(mdz, mx, (float*)scratch, p, device_status);
         CKPT_LAUNCH_CHECK("conv wgrad, 64 input channels as pixel pairs (tensor cores)");
-        pairview_fold_kernel<<<(unsigned)((g.cout * 576 + 255) / 256), 256, 0, st>>>((const float*)scratch, dw, g.cout, p.slices);
+        pairview_fold_kernel<8><<<(unsigned)((g.cout * 144 + 31) / 32), dim3(32, 8), 0, st>>>((const float*)scratch, dw, g.cout, p.slices);
         CKPT_LAUNCH_CHECK("wgrad pair fold");
         return CKPT_OK;
     }
@@ -2560,7 +2609,7 @@ int tc_conv_wgrad(const ConvGeom& g, const void* dz, const void* x, float* dw, v
         dim3 grid(p.slices, g.cout / 64);
         tc_wgrad_c64_kernel<<<grid, kThreads, smem, st>>>(mdz, mx, (float*)scratch, p, device_status);
         CKPT_LAUNCH_CHECK("conv wgrad, 64 input channels (tensor cores)");
-        slice_sum_tc_kernel<<<(unsigned)((elems + 255) / 256), 256, 0, st>>>((const float*)scratch, dw, elems, p.slices);
+        launch_slice_sum((const float*)scratch, dw, elems, p.slices, st);
         CKPT_LAUNCH_CHECK("wgrad slice sum");
         return CKPT_OK;
     }
@@ -2582,7 +2631,7 @@ int tc_conv_wgrad(const ConvGeom& g, const void* dz, const void* x, float* dw, v
         dim3 grid(p.slices, pairs, co_tiles);
         tc_wgrad_rows_kernel<<<grid, kThreads, smem, st>>>(mdz, mx, (float*)scratch, p, device_status);
         CKPT_LAUNCH_CHECK("conv wgrad, shared vertical taps (tensor cores)");
-        slice_sum_tc_kernel<<<(unsigned)((elems + 255) / 256), 256, 0, st>>>((const float*)scratch, dw, elems, p.slices);
+        launch_slice_sum((const float*)scratch, dw, elems, p.slices, st);
         CKPT_LAUNCH_CHECK("wgrad slice sum");
         return CKPT_OK;
     }
@@ -2609,7 +2658,7 @@ int tc_conv_wgrad(const ConvGeom& g, const void* dz, const void* x, float* dw, v
     tc_conv_wgrad_kernel<<<grid, kThreads, smem, st>>>(mdz, mx, target, p, device_status);
     CKPT_LAUNCH_CHECK("conv wgrad (tensor cores)");
     if (slices > 1) {
-        slice_sum_tc_kernel<<<(unsigned)((elems + 255) / 256), 256, 0, st>>>((const float*)scratch, dw, elems, slices);
+        launch_slice_sum((const float*)scratch, dw, elems, slices, st);
         CKPT_LAUNCH_CHECK("wgrad slice sum");
     }
     return CKPT_OK;

@@ -2,7 +2,8 @@
 
 * the tensor-core convolution kernels at the VGG-16 / batch-64 layer shapes, on sampled outputs that
   the oracle computes one by one (a cropped neighbourhood for forward/dgrad, one (c_out, c_in)
-  channel pair over all pixels for wgrad);
+  channel pair over all pixels for wgrad), and the fully connected layers of the VGG-16 head on
+  sampled output rows and input columns;
 * the whole checkpointed step of configurations 2, 3, 4 and 5 through properties that hold at any size:
   arena high-water == highest offset == planner's prediction (arena of exactly that size),
   gradients bit-identical between the checkpointed and the store-all schedule, finite loss."""
@@ -24,7 +25,9 @@ LAYERS = [
     (64, 224, 224, 64, 64),
     (64, 112, 112, 64, 128),
     (64, 112, 112, 128, 128),
+    (64, 56, 56, 128, 256),
     (64, 56, 56, 256, 256),
+    (64, 28, 28, 256, 512),
     (64, 28, 28, 512, 512),
     (64, 14, 14, 512, 512),
     (32, 56, 56, 64, 64),        # the unit of the 1000-layer chain
@@ -76,6 +79,43 @@ def test_conv_kernels_full_size_sampled(layer):
         dzs = bf16_host(dz[..., co:co + 1])
         dw_ref = no.conv2d_bwd(xs, np.zeros((1, 3, 3, 1)), dzs, 1, 1)[1][0, :, :, 0]
         assert np.abs(dw[co, :, :, ci].cpu().numpy().astype(np.float64) - dw_ref).max() <= 2e-5 * max(scale_dw, np.abs(dw_ref).max())
+
+
+FC_LAYERS = [(64, 25088, 4096), (64, 4096, 4096), (64, 4096, 1000)]      # batch, inputs, outputs of the VGG-16 head
+
+
+@pytest.mark.parametrize("layer", FC_LAYERS, ids=lambda l: "x".join(map(str, l)))
+def test_fc_kernels_full_size_sampled(layer):
+    """A fully connected layer is a 1x1 convolution on a 1x1 image: sampled outputs, input gradients and
+    weight gradients against the oracle's convolution on the rows and columns they depend on."""
+    import torch
+    n, cin, cout = layer
+    dt = ck.DTYPE_BF16
+    gen = torch.Generator(device="cuda").manual_seed(cin + cout)
+    x = torch.randn(n, 1, 1, cin, device="cuda", generator=gen).bfloat16()
+    wt = (torch.randn(cout, 1, 1, cin, device="cuda", generator=gen) / cin ** 0.5).bfloat16()
+    dz = torch.randn(n, 1, 1, cout, device="cuda", generator=gen).bfloat16()
+    shape = ck.ConvShape(n, 1, 1, cin, cout, 1, 1, 0)
+    scratch = torch.empty(max(256, ck.conv2d_scratch_bytes(shape, dt)), dtype=torch.uint8, device="cuda")
+    z = torch.empty(n, 1, 1, cout, device="cuda", dtype=torch.bfloat16)
+    dx = torch.empty_like(x)
+    dw = torch.empty(cout, 1, 1, cin, device="cuda")
+    ck.conv2d_forward(shape, dt, 0, x, wt, z, scratch)
+    ck.conv2d_dgrad(shape, dt, 0, dz, wt, dx, scratch)
+    ck.conv2d_wgrad(shape, dt, 0, dz, x, dw, scratch)
+    torch.cuda.synchronize()
+    rng = np.random.default_rng(11)
+    x64, dz64 = bf16_host(x), bf16_host(dz)
+    scale_z, scale_dx, scale_dw = float(z.float().abs().max()), float(dx.float().abs().max()), float(dw.abs().max())
+    outs = sorted({0, cout - 1, 127, 128, *map(int, rng.integers(cout, size=12))})
+    z_ref = no.conv2d_fwd(x64, bf16_host(wt[outs]), 1, 0)                              # [n,1,1,len(outs)]
+    assert np.abs(bf16_host(z[..., outs]) - z_ref).max() <= 6e-3 * scale_z
+    # weight gradient of the sampled output rows (all inputs), and input gradient of sampled input columns
+    dw_ref = no.conv2d_bwd(x64, np.zeros((len(outs), 1, 1, cin)), dz64[..., outs], 1, 0)[1]
+    assert np.abs(dw[outs].cpu().numpy().astype(np.float64) - dw_ref).max() <= 2e-5 * max(scale_dw, np.abs(dw_ref).max())
+    ins = sorted({0, cin - 1, 63, 64, *map(int, rng.integers(cin, size=12))})
+    dx_ref = no.conv2d_bwd(np.zeros((n, 1, 1, len(ins))), bf16_host(wt[..., ins]), dz64, 1, 0)[0]
+    assert np.abs(bf16_host(dx[..., ins]) - dx_ref).max() <= 6e-3 * scale_dx
 
 
 def step_properties(spec, seed=0, finite_last_units=None):
