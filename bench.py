@@ -283,7 +283,7 @@ def main():
 # DRAM traffic per launch of the conv-forward kernels over the layer mix of config 2, from one ncu pass
 # (profiles/conv_forward_vgg16_b64_dram_traffic.md).  Valid only for the kernel source it was taken
 # on: reported as null when csrc/conv_tc.cu has changed since.
-CONV_FWD_TRAFFIC = {"source_sha256": "158c056f06a0e89e7663ddf114cceb82fe9de365767a76ae5c90a3061a99a036", "bytes_per_launch": 170082773}
+CONV_FWD_TRAFFIC = {"source_sha256": "058464cd5165c13afbbe26432d3ef457099db152f3361521d39e034f20747950", "bytes_per_launch": 169688789}
 
 
 def _kernel_source_sha():
@@ -301,7 +301,7 @@ def dominant_kernel_roofline(config_index, peaks, batch, first_shape):
     from paper_2502_12499_b200 import opbench
     mix = opbench.conv_mix("fwd", config_index, reps=3)
     traffic = CONV_FWD_TRAFFIC["bytes_per_launch"] if CONV_FWD_TRAFFIC["source_sha256"] == _kernel_source_sha() else None
-    out = {"kernel": "tc_conv_t_kernel / tc_conv_c64_kernel (implicit-GEMM conv forward over the layer mix)", "bound": "tensor",
+    out = {"kernel": "tc_conv_tp_kernel / tc_conv_t_kernel (implicit-GEMM conv forward over the layer mix)", "bound": "tensor",
            "achieved": mix["tflops"], "peak": peaks["tflops_burst"], "unit": "TFLOP/s", "frac": mix["tflops"] / peaks["tflops_burst"],
            "peak_source": peaks["source"] + " (burst: kernels timed in isolation)", "traffic": traffic,
            "launch_shapes": mix["launches"], "flops_per_launch": mix["flops"] / mix["launches"],

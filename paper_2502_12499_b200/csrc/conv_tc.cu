@@ -449,6 +449,12 @@ struct TParams {
     int tiles_w, tiles_h, tiles_n;
     int co_tiles, p_tiles, ctas_per_co;
     int stages;
+    // halo-patch form (tc_conv_tp_kernel): the terms are grouped in columns of three vertical taps that read one patch
+    int patch_ok;                // the caller filled ncols / col_term
+    int ncols;                   // columns per 64-channel block: (horizontal offset, channel offset) pairs
+    int col_term[4][3];          // term (index into the tap tables) of column c at vertical tap dy; tap_dh = dy - 1
+    int tile_cols;               // pixels per tile = 8 * th
+    uint32_t patch_bytes;        // 8 x (th + 2) pixels x 128 bytes
 };
 
 // A_MN (dgrad): the M operand is the forward filter [c_red][taps][c_out] read in place, output channels contiguous:
@@ -603,6 +609,201 @@ tc_conv_t_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
         if (lane == 0) tma_store_wait_all();
         if (stats && co < p.c_out) {
             // one partial row pair per CTA: [block][sum | sum of squares][channel]
+            if (p.fold) {
+                const size_t blk = (size_t)first * 2 + co / p.fold;
+                stat_partial[(blk * 2) * p.fold + co % p.fold] = sum;
+                stat_partial[(blk * 2 + 1) * p.fold + co % p.fold] = sumsq;
+            } else {
+                stat_partial[((size_t)first * 2) * p.c_out + co] = sum;
+                stat_partial[((size_t)first * 2 + 1) * p.c_out + co] = sumsq;
+            }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        __syncwarp();
+        tc_fence_after();
+        tmem_dealloc(tmem_base, 512);
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// The role-swapped kernel on halo patches, for 3x3 filters on images that tile well into 8-pixel-wide
+// strips.  A pixel tile is 8 wide x th high (th <= 32, one image).  For a column (horizontal offset,
+// 64-channel block) ONE patch of th + 2 rows is loaded; its rows are 1024-byte swizzle atoms, so the
+// pixel operand of vertical tap dy is the same patch read from byte dy * 1024 on.  Per column the
+// SM receives one patch (34 KB) and three filter boxes instead of three pixel boxes of 32 KB: 83 KB
+// for twelve 128 x 256 x 16 instructions instead of 144 KB.  Patches and filter boxes travel in
+// rings of their own (three patches, six boxes) so that the next columns are in flight while the
+// tensor core works on this one.
+// ------------------------------------------------------------------------------------------------
+#ifndef TP_MIN_COVER
+#define TP_MIN_COVER 0.87
+#endif
+constexpr int kTpBoxes = 6, kTpPatches = 3;
+constexpr uint32_t kTpPatchSlot = 34 * 1024;
+constexpr uint32_t kTpSmem = kTpBoxes * 16384 + kTpPatches * kTpPatchSlot + 256 + 4 * 2 * 2048 + 1024;
+
+template <bool A_MN>
+__global__ void __launch_bounds__(kThreads, 1)
+tc_conv_tp_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w,
+                  const __grid_constant__ CUtensorMap map_out, float* __restrict__ stat_partial, TParams p, int* status) {
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    constexpr uint32_t a_bytes = 128 * 128;
+    const uint32_t patches = base + kTpBoxes * a_bytes;
+    const uint32_t bars = patches + kTpPatches * kTpPatchSlot;
+    const uint32_t out_stage = bars + 256;                                   // [4 warps][2][32 pixels x 32 channels] bf16
+    __shared__ uint32_t tmem_base_slot;
+    __shared__ int failed_flag;
+    volatile int* failed = &failed_flag;
+
+    const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
+    const int co_tile = blockIdx.x % p.co_tiles;
+    const int first = blockIdx.x / p.co_tiles;
+    const int my_tiles = first < p.p_tiles ? (p.p_tiles - first + p.ctas_per_co - 1) / p.ctas_per_co : 0;
+    const int blocks = p.c_red / 64;
+    const int cols = p.ncols * blocks;
+
+    auto a_full = [&](int s) { return bars + 8u * s; };
+    auto a_empty = [&](int s) { return bars + 64u + 8u * s; };
+    auto p_full = [&](int s) { return bars + 128u + 8u * s; };
+    auto p_empty = [&](int s) { return bars + 160u + 8u * s; };
+    const uint32_t acc_full0 = bars + 192u, acc_empty0 = bars + 208u;
+    auto tile_origin = [&](int j, int& w0, int& h0, int& n0) {
+        int t = first + j * p.ctas_per_co;
+        w0 = (t % p.tiles_w) * 8; t /= p.tiles_w;
+        h0 = (t % p.tiles_h) * p.th;
+        n0 = t / p.tiles_h;
+    };
+
+    if (threadIdx.x == 0) {
+        failed_flag = 0;
+        for (int s = 0; s < kTpBoxes; ++s) { mbar_init(a_full(s), 1); mbar_init(a_empty(s), 1); }
+        for (int s = 0; s < kTpPatches; ++s) { mbar_init(p_full(s), 1); mbar_init(p_empty(s), 1); }
+        for (int b = 0; b < 2; ++b) { mbar_init(acc_full0 + 8 * b, 1); mbar_init(acc_empty0 + 8 * b, 128); }
+        fence_barrier_init();
+        tma_prefetch_desc(&map_x);
+        tma_prefetch_desc(&map_w);
+        tma_prefetch_desc(&map_out);
+    }
+    if (warp == 1) tmem_alloc(smem_u32(&tmem_base_slot), 512);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = tmem_base_slot;
+
+    if (warp == 0 && lane == 0) {
+        // ---------------- TMA producer: per column one patch, then the filter boxes of its three vertical taps
+        int ga = 0, gp = 0;
+        bool ok = true;
+        for (int j = 0; j < my_tiles && ok; ++j) {
+            int w0, h0, n0;
+            tile_origin(j, w0, h0, n0);
+            for (int c = 0; c < cols && ok; ++c, ++gp) {
+                const int col = c / blocks, blk = c % blocks;
+                const int sp = gp % kTpPatches;
+                if (!mbar_wait(p_empty(sp), ((uint32_t)(gp / kTpPatches) & 1u) ^ 1u, failed, status, 911)) { ok = false; break; }
+                const int t0 = p.col_term[col][0];
+                mbar_expect_tx(p_full(sp), p.patch_bytes);
+                tma_load_4d(patches + (uint32_t)sp * kTpPatchSlot, &map_x, p_full(sp), blk * 64 + p.tap_xc[t0], w0 + p.tap_dw[t0], h0 - 1, n0);
+                for (int dy = 0; dy < 3; ++dy, ++ga) {
+                    const int sa = ga % kTpBoxes;
+                    if (!mbar_wait(a_empty(sa), ((uint32_t)(ga / kTpBoxes) & 1u) ^ 1u, failed, status, 912)) { ok = false; break; }
+                    const int tap = p.col_term[col][dy];
+                    const uint32_t a_dst = base + (uint32_t)sa * a_bytes;
+                    mbar_expect_tx(a_full(sa), a_bytes);
+                    if (A_MN) {
+                        tma_load_2d(a_dst, &map_w, a_full(sa), p.tap_col[tap] * p.c_out + co_tile * 128, blk * 64);
+                        tma_load_2d(a_dst + 8192, &map_w, a_full(sa),
+                                    co_tile * 128 + 64 < p.c_out ? p.tap_col[tap] * p.c_out + co_tile * 128 + 64 : p.taps * p.c_out, blk * 64);
+                    } else {
+                        tma_load_2d(a_dst, &map_w, a_full(sa), p.tap_col[tap] * p.c_red + blk * 64, co_tile * 128);
+                    }
+                }
+                if (!ok) { ++gp; break; }       // this column's patch is in flight: count it for the drain below
+            }
+        }
+        if (*failed) {
+            for (int q = max(0, gp - kTpPatches); q < gp; ++q) mbar_drain(p_full(q % kTpPatches), (uint32_t)(q / kTpPatches) & 1u);
+            for (int q = max(0, ga - kTpBoxes); q < ga; ++q) mbar_drain(a_full(q % kTpBoxes), (uint32_t)(q / kTpBoxes) & 1u);
+        }
+    } else if (warp == 1 && lane == 0) {
+        // ---------------- MMA issuer
+        const uint32_t idesc = instr_desc(128, p.tile_cols, A_MN ? 1 : 0, 0);
+        constexpr uint32_t a_step = A_MN ? 2048u : 32u, a_lbo = A_MN ? 8192u : 0u;
+        bool ok = true;
+        int ga = 0, gp = 0;
+        for (int j = 0; j < my_tiles && ok; ++j) {
+            const int buf = j & 1;
+            if (!mbar_wait(acc_empty0 + 8 * buf, ((uint32_t)(j >> 1) & 1u) ^ 1u, failed, status, 914)) { ok = false; break; }
+            const uint32_t acc = tmem_base + (uint32_t)(buf * 256);
+            for (int c = 0; c < cols && ok; ++c, ++gp) {
+                const int sp = gp % kTpPatches;
+                if (!mbar_wait(p_full(sp), (uint32_t)(gp / kTpPatches) & 1u, failed, status, 915)) { ok = false; break; }
+                const uint32_t patch = patches + (uint32_t)sp * kTpPatchSlot;
+                for (int dy = 0; dy < 3; ++dy, ++ga) {
+                    const int sa = ga % kTpBoxes;
+                    if (!mbar_wait(a_full(sa), (uint32_t)(ga / kTpBoxes) & 1u, failed, status, 916)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint32_t a_addr = base + (uint32_t)sa * a_bytes;
+                    const uint32_t b_addr = patch + (uint32_t)dy * 1024u;
+#pragma unroll
+                    for (int kk = 0; kk < 4; ++kk)
+                        umma_bf16(acc, smem_desc(a_addr + kk * a_step, a_lbo, 1024), smem_desc(b_addr + kk * 32, 0, 1024), idesc,
+                                  (c > 0 || dy > 0 || kk > 0) ? 1u : 0u);
+                    umma_commit(a_empty(sa));
+                }
+                if (ok) umma_commit(p_empty(sp));
+            }
+            if (ok) umma_commit(acc_full0 + 8 * buf);
+        }
+    } else if (warp >= 2) {
+        // ---------------- epilogue, as in tc_conv_t_kernel: lane = output channel, column = pixel hl * 8 + wl of the tile
+        const int quarter = warp % 4;
+        const int co = co_tile * 128 + quarter * 32 + lane;
+        const bool stats = stat_partial != nullptr;
+        float sum = 0.f, sumsq = 0.f;
+        int chunk_count = 0;
+        for (int j = 0; j < my_tiles; ++j) {
+            const int buf = j & 1;
+            if (!mbar_wait(acc_full0 + 8 * buf, (uint32_t)(j >> 1) & 1u, failed, status, 913)) break;
+            tc_fence_after();
+            int w0, h0, n0;
+            tile_origin(j, w0, h0, n0);
+#pragma unroll 1
+            for (int c0 = 0; c0 < p.tile_cols; c0 += 32, ++chunk_count) {
+                const int idx = c0 + lane;
+                const bool inside = (w0 + (idx & 7) < p.W) && (h0 + (idx >> 3) < p.H);
+                const uint32_t in_mask = __ballot_sync(0xffffffffu, inside);
+                uint32_t v[32];
+                tmem_ld32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * 256 + c0), v);
+                const uint32_t slab = out_stage + (uint32_t)((quarter * 2 + (chunk_count & 1)) * 2048);
+                if (lane == 0) tma_store_wait_read<1>();          // the store that last read this slab has left it
+                __syncwarp();
+#pragma unroll
+                for (int e = 0; e < 32; ++e) {
+                    const __nv_bfloat16 r = __float2bfloat16_rn(__uint_as_float(v[e]));
+                    asm volatile("st.shared.b16 [%0], %1;" ::"r"(slab + (uint32_t)(e * 64 + lane * 2)), "h"(__bfloat16_as_ushort(r)) : "memory");
+                    if ((in_mask >> e) & 1u) {
+                        const float f = __bfloat162float(r);
+                        sum += f;
+                        sumsq = fmaf(f, f, sumsq);
+                    }
+                }
+                fence_proxy_async();
+                __syncwarp();
+                if (lane == 0 && in_mask != 0u && co_tile * 128 + quarter * 32 < p.c_out) {
+                    tma_store_4d(&map_out, slab, co_tile * 128 + quarter * 32, w0, h0 + (c0 >> 3), n0);
+                    tma_store_commit();
+                }
+            }
+            tc_fence_before();
+            mbar_arrive(acc_empty0 + 8 * buf);
+        }
+        if (lane == 0) tma_store_wait_all();
+        if (stats && co < p.c_out) {
             if (p.fold) {
                 const size_t blk = (size_t)first * 2 + co / p.fold;
                 stat_partial[(blk * 2) * p.fold + co % p.fold] = sum;
@@ -2056,6 +2257,23 @@ int launch_t_core(TParams p, const void* x, int x_channels, const CUtensorMap& m
                   int N, int H, int W, int c_red, int c_out, int* status, cudaStream_t st, const char* what, bool a_mn) {
     p.H = H; p.W = W; p.N = N; p.c_red = c_red; p.c_out = c_out;
     choose_tile(256, W, H, N, &p.tw, &p.th, &p.tn);
+    bool patch = false;
+#ifndef NO_TP_KERNEL
+    if (p.patch_ok) {
+        // strips of 8 x th pixels, th <= 32 and a multiple of 4 (the epilogue stores chunks of 4 rows): worth it when
+        // they cover the image with little waste, the instructions stay wide and every SM gets several tiles
+        const int nt = (H + 31) / 32;
+        int th = ((H + nt - 1) / nt + 3) / 4 * 4;
+        const int tiles_w = (W + 7) / 8;
+        const double cover = (double)W * H / ((double)tiles_w * 8 * nt * th);
+        if (th <= 32 && th >= 24 && cover >= TP_MIN_COVER && (int64_t)tiles_w * nt * N * ((c_out + 127) / 128) >= 4 * 148) {
+            patch = true;
+            p.tw = 8; p.th = th; p.tn = 1;
+            p.tile_cols = 8 * th;
+            p.patch_bytes = (uint32_t)(8 * (th + 2)) * 128;
+        }
+    }
+#endif
     p.tw_log = 0; while ((1 << p.tw_log) < p.tw) ++p.tw_log;
     p.th_log = 0; while ((1 << p.th_log) < p.th) ++p.th_log;
     p.tiles_w = (W + p.tw - 1) / p.tw; p.tiles_h = (H + p.th - 1) / p.th; p.tiles_n = (N + p.tn - 1) / p.tn;
@@ -2068,7 +2286,7 @@ int launch_t_core(TParams p, const void* x, int x_channels, const CUtensorMap& m
     constexpr uint32_t stage_bytes = 128 * 128 + 256 * 128;
     p.stages = std::min<int>(kMaxStages, kSmemBudget / stage_bytes);
     CUtensorMap mx;
-    int rc = make_act_map(&mx, x, N, H, W, x_channels, p.tw, p.th, p.tn);
+    int rc = make_act_map(&mx, x, N, H, W, x_channels, p.tw, patch ? p.th + 2 : p.th, p.tn);
     if (rc) return rc;
     // the box of one epilogue chunk: 32 consecutive pixels of the tile (w fastest) x 32 channels, no swizzle
     CUtensorMap mo;
@@ -2093,6 +2311,19 @@ int launch_t_core(TParams p, const void* x, int x_channels, const CUtensorMap& m
         attr_set = true;
     }
     if (stat_blocks) *stat_blocks = stat_partial ? (p.fold ? 2 : 1) * p.ctas_per_co : 0;
+    if (patch) {
+        static bool tp_attr_set = false;
+        if (!tp_attr_set) {
+            cudaError_t e = cudaFuncSetAttribute(tc_conv_tp_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kTpSmem);
+            if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_conv_tp_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kTpSmem);
+            if (e != cudaSuccess) return cuda_fail(e, "raising the shared-memory limit");
+            tp_attr_set = true;
+        }
+        if (a_mn) tc_conv_tp_kernel<true><<<p.ctas_per_co * p.co_tiles, kThreads, kTpSmem, st>>>(mx, mw, mo, stat_blocks ? stat_partial : nullptr, p, status);
+        else tc_conv_tp_kernel<false><<<p.ctas_per_co * p.co_tiles, kThreads, kTpSmem, st>>>(mx, mw, mo, stat_blocks ? stat_partial : nullptr, p, status);
+        CKPT_LAUNCH_CHECK(what);
+        return CKPT_OK;
+    }
     if (a_mn) tc_conv_t_kernel<true><<<p.ctas_per_co * p.co_tiles, kThreads, smem, st>>>(mx, mw, mo, stat_blocks ? stat_partial : nullptr, p, status);
     else tc_conv_t_kernel<false><<<p.ctas_per_co * p.co_tiles, kThreads, smem, st>>>(mx, mw, mo, stat_blocks ? stat_partial : nullptr, p, status);
     CKPT_LAUNCH_CHECK(what);
@@ -2104,6 +2335,10 @@ int launch_t(const void* x, const void* w_mat, void* out, float* stat_partial, i
     TParams p;
     p.taps = k * k;
     p.fold = 0;
+    p.patch_ok = k == 3 && pad == 1;
+    p.ncols = 3;
+    for (int dx = 0; dx < 3; ++dx)
+        for (int dy = 0; dy < 3; ++dy) p.col_term[dx][dy] = dy * 3 + dx;
     for (int t = 0; t < k * k; ++t) {
         p.tap_dh[t] = t / k - pad; p.tap_dw[t] = t % k - pad; p.tap_col[t] = a_mn ? k * k - 1 - t : t; p.tap_xc[t] = 0;
     }
@@ -2132,6 +2367,10 @@ int launch_t_paired(const void* x, const void* w, int flip, void* out, float* st
     TParams p;
     p.taps = 12;
     p.fold = 64;
+    p.patch_ok = 1;
+    p.ncols = 4;
+    for (int sp = 0; sp < 4; ++sp)
+        for (int r = 0; r < 3; ++r) p.col_term[sp][r] = r * 4 + sp;
     for (int t = 0; t < 12; ++t) {
         const int r = t / 4, sp = t % 4;
         p.tap_dh[t] = r - 1;
