@@ -444,6 +444,11 @@ struct TParams {
     int tap_dh[12], tap_dw[12], tap_col[12];
     int tap_xc[12];              // channel offset of a term's pixel box in the input view (pixel pairs: which pixel of the pair)
     int fold;                    // 0, or 64: the 128 "channels" are (pixel of a pair, 64 channels) and the sums go to block 2*cta + pixel
+    // pixel pairs: the 128-row filter operand of a term is two 64-row boxes of the caller's filter, one per pixel of the
+    // pair: filter positions tap_col[t] and tap_col2[t], -1 = the term does not reach that pixel (a box outside the
+    // matrix, i.e. zeros)
+    int pair;
+    int tap_col2[12];
     int tw_log, th_log;          // pixel tile tw x th x tn = 256, powers of two
     int tw, th, tn;
     int tiles_w, tiles_h, tiles_n;
@@ -456,6 +461,28 @@ struct TParams {
     int tile_cols;               // pixels per tile = 8 * th
     uint32_t patch_bytes;        // 8 x (th + 2) pixels x 128 bytes
 };
+
+template <bool A_MN>
+__device__ __forceinline__ void load_filter_boxes(const TParams& p, const CUtensorMap* map_w, uint32_t a_dst, uint32_t bar, int tap, int blk,
+                                                  int co_tile) {
+    if (p.pair) {
+        const int c0 = p.tap_col[tap], c1 = p.tap_col2[tap];
+        if (A_MN) {     // forward filter [c_red][9][64]: 64 reduction rows x the 64 output channels of a position
+            tma_load_2d(a_dst, map_w, bar, (c0 < 0 ? 9 : c0) * 64, blk * 64);
+            tma_load_2d(a_dst + 8192, map_w, bar, (c1 < 0 ? 9 : c1) * 64, blk * 64);
+        } else {        // filter [64][9][c_red]: the 64 output channels x 64 reduction channels of a position
+            tma_load_2d(a_dst, map_w, bar, c0 < 0 ? 9 * p.c_red : c0 * p.c_red + blk * 64, 0);
+            tma_load_2d(a_dst + 8192, map_w, bar, c1 < 0 ? 9 * p.c_red : c1 * p.c_red + blk * 64, 0);
+        }
+    } else if (A_MN) {
+        tma_load_2d(a_dst, map_w, bar, p.tap_col[tap] * p.c_out + co_tile * 128, blk * 64);
+        // (with 64 output channels the second box lies past them: it is sent outside the matrix, i.e. zero fill)
+        tma_load_2d(a_dst + 8192, map_w, bar,
+                    co_tile * 128 + 64 < p.c_out ? p.tap_col[tap] * p.c_out + co_tile * 128 + 64 : p.taps * p.c_out, blk * 64);
+    } else {
+        tma_load_2d(a_dst, map_w, bar, p.tap_col[tap] * p.c_red + blk * 64, co_tile * 128);
+    }
+}
 
 // A_MN (dgrad): the M operand is the forward filter [c_red][taps][c_out] read in place, output channels contiguous:
 // two boxes of 64 reduction rows x 64 output channels per stage (at the column block of the mirrored filter
@@ -518,14 +545,7 @@ tc_conv_t_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                 const int tap = it / blocks, blk = it % blocks;
                 const uint32_t a_dst = base + (uint32_t)s * stage_bytes;
                 mbar_expect_tx(full_bar(s), stage_bytes);
-                if (A_MN) {
-                    tma_load_2d(a_dst, &map_w, full_bar(s), p.tap_col[tap] * p.c_out + co_tile * 128, blk * 64);
-                    // (with 64 output channels the second box lies past them: it is sent outside the matrix, i.e. zero fill)
-                    tma_load_2d(a_dst + 8192, &map_w, full_bar(s),
-                                co_tile * 128 + 64 < p.c_out ? p.tap_col[tap] * p.c_out + co_tile * 128 + 64 : p.taps * p.c_out, blk * 64);
-                } else {
-                    tma_load_2d(a_dst, &map_w, full_bar(s), p.tap_col[tap] * p.c_red + blk * 64, co_tile * 128);
-                }
+                load_filter_boxes<A_MN>(p, &map_w, a_dst, full_bar(s), tap, blk, co_tile);
                 tma_load_4d(a_dst + a_bytes, &map_x, full_bar(s), blk * 64 + p.tap_xc[tap], w0 + p.tap_dw[tap], h0 + p.tap_dh[tap], n0);
             }
         }
@@ -641,6 +661,13 @@ tc_conv_t_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
 #ifndef TP_MIN_COVER
 #define TP_MIN_COVER 0.87
 #endif
+#ifndef TP_MIN_TILES
+#define TP_MIN_TILES 200
+#endif
+#ifndef PAIR_MIN_PIXELS
+#define PAIR_MIN_PIXELS 262144
+#define PAIR_MIN_PIXELS_STRIPS 65536
+#endif
 constexpr int kTpBoxes = 6, kTpPatches = 3;
 constexpr uint32_t kTpPatchSlot = 34 * 1024;
 constexpr uint32_t kTpSmem = kTpBoxes * 16384 + kTpPatches * kTpPatchSlot + 256 + 4 * 2 * 2048 + 1024;
@@ -714,13 +741,7 @@ tc_conv_tp_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
                     const int tap = p.col_term[col][dy];
                     const uint32_t a_dst = base + (uint32_t)sa * a_bytes;
                     mbar_expect_tx(a_full(sa), a_bytes);
-                    if (A_MN) {
-                        tma_load_2d(a_dst, &map_w, a_full(sa), p.tap_col[tap] * p.c_out + co_tile * 128, blk * 64);
-                        tma_load_2d(a_dst + 8192, &map_w, a_full(sa),
-                                    co_tile * 128 + 64 < p.c_out ? p.tap_col[tap] * p.c_out + co_tile * 128 + 64 : p.taps * p.c_out, blk * 64);
-                    } else {
-                        tma_load_2d(a_dst, &map_w, a_full(sa), p.tap_col[tap] * p.c_red + blk * 64, co_tile * 128);
-                    }
+                    load_filter_boxes<A_MN>(p, &map_w, a_dst, a_full(sa), tap, blk, co_tile);
                 }
                 if (!ok) { ++gp; break; }       // this column's patch is in flight: count it for the drain below
             }
@@ -843,6 +864,8 @@ struct C64Params {
     int m_tiles;                 // tiles_w * tiles_h * N
     int ctas_per_n;              // persistent CTAs that share one output-channel tile
     uint32_t box_stride;         // bytes between the three shifted copies of a patch
+    int b_mn;                    // dgrad: the filter operand is the forward filter [64][9][c_out] read in place (output
+                                 // channels contiguous, an MN-major operand), tap t from the mirrored position 8 - t
 };
 
 __global__ void __launch_bounds__(kThreads, 1)
@@ -893,7 +916,10 @@ tc_conv_c64_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_const
         // ---------------- producer: the filter once, then the patches; one lane per copy
         if (lane == 0) mbar_expect_tx(w_full, w_bytes);
         __syncwarp();
-        if (lane < 9) tma_load_2d(base + lane * 8192, &map_w, w_full, lane * 64, n_tile * 64);
+        if (lane < 9) {
+            if (p.b_mn) tma_load_2d(base + lane * 8192, &map_w, w_full, (8 - lane) * p.c_out + n_tile * 64, 0);
+            else tma_load_2d(base + lane * 8192, &map_w, w_full, lane * 64, n_tile * 64);
+        }
         int issued = 0;
         for (int j = 0; j < my_tiles; ++j) {
             const int b = j & 1;
@@ -915,7 +941,8 @@ tc_conv_c64_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_const
         }
     } else if (warp == 1 && lane == 0) {
         // ---------------- MMA issuer
-        const uint32_t idesc = instr_desc(128, 64, 0, 0);
+        const uint32_t idesc = instr_desc(128, 64, 0, p.b_mn);
+        const uint32_t b_step = p.b_mn ? 2048u : 32u, b_lbo = p.b_mn ? 8192u : 0u;      // 16 reduction rows, or 32 bytes along a row
         bool ok = mbar_wait(w_full, 0, failed, status, 302);
         for (int j = 0; j < my_tiles && ok; ++j) {
             const int b = j & 1;
@@ -930,7 +957,7 @@ tc_conv_c64_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_const
                 const uint32_t b_addr = base + tap * 8192;
 #pragma unroll
                 for (int kk = 0; kk < 4; ++kk)
-                    umma_bf16(acc, smem_desc(a_addr + kk * 32, 0, 1024), smem_desc(b_addr + kk * 32, 0, 1024), idesc,
+                    umma_bf16(acc, smem_desc(a_addr + kk * 32, 0, 1024), smem_desc(b_addr + kk * b_step, b_lbo, 1024), idesc,
                               (tap > 0 || kk > 0) ? 1u : 0u);
             }
             umma_commit(a_empty0 + 8 * b);
@@ -1945,22 +1972,6 @@ __global__ void fc_reduce_kernel(const float* __restrict__ partial, int slices, 
     out[e] = __float2bfloat16_rn(sum);
 }
 
-// Filter of the pixel-pair form of a 3x3 convolution with 64 output channels (see launch_t_paired):
-//   wp[(p, o)][(r, s'), red] = F[o][r][s' - p][red] for 0 <= s' - p <= 2, else 0,   p = 0, 1; s' = 0..3
-// with F the forward filter w[o][r][s][red] (flip = 0) or the filter of the input gradient
-// F[o][r][s][red] = w[red][2 - r][2 - s][o] (flip = 1; o runs over the forward input channels).
-__global__ void pair_filter_kernel(const __nv_bfloat16* __restrict__ w, __nv_bfloat16* __restrict__ wp, int c_red, int flip) {
-    const int total = 128 * 12 * c_red;
-    for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < total; i += gridDim.x * blockDim.x) {
-        const int red = i % c_red, term = (i / c_red) % 12, row = i / (12 * c_red);
-        const int p = row / 64, o = row % 64, r = term / 4, s = term % 4 - p;
-        __nv_bfloat16 v = __float2bfloat16_rn(0.f);
-        if (s >= 0 && s <= 2)
-            v = flip ? w[((size_t)red * 9 + (2 - r) * 3 + (2 - s)) * 64 + o] : w[((size_t)o * 9 + r * 3 + s) * c_red + red];
-        wp[i] = v;
-    }
-}
-
 // wt[ci][tap'][co] = w[co][taps-1-tap'][ci]: the matrix of the transposed convolution (stride 1).
 __global__ void transpose_flip_kernel(const __nv_bfloat16* __restrict__ w, __nv_bfloat16* __restrict__ wt, int c_out, int taps, int c_in) {
     const int64_t total = (int64_t)c_out * taps * c_in;
@@ -2109,9 +2120,10 @@ void choose_tile(int pixels, int W, int H, int N, int* tw, int* th, int* tn) {
 int pick_bn(int c_out) { return c_out % 256 == 0 ? 256 : (c_out % 128 == 0 ? 128 : 64); }
 
 int launch_c64(const void* x, const void* w_mat, void* out, float* stat_partial, int* stat_blocks, int N, int H, int W,
-               int c_out, int* status, cudaStream_t st, const char* what) {
+               int c_out, int* status, cudaStream_t st, const char* what, bool b_mn = false) {
     C64Params p;
     p.H = H; p.W = W; p.N = N; p.c_out = c_out;
+    p.b_mn = b_mn ? 1 : 0;
     const int nt = (H + 15) / 16;
     p.th = (H + nt - 1) / nt;
     p.tiles_h = (H + p.th - 1) / p.th;
@@ -2127,7 +2139,7 @@ int launch_c64(const void* x, const void* w_mat, void* out, float* stat_partial,
     CUtensorMap mx, mw;
     int rc = make_act_map(&mx, x, N, H, W, 64, 8, p.th + 2, 1);
     if (rc) return rc;
-    rc = make_mat_map(&mw, w_mat, c_out, 9 * 64, 64);
+    rc = b_mn ? make_mat_map(&mw, w_mat, 64, (int64_t)9 * c_out, 64) : make_mat_map(&mw, w_mat, c_out, 9 * 64, 64);
     if (rc) return rc;
     const size_t smem = 9 * 64 * 128 + 2 * 3 * (size_t)p.box_stride + 1024 + 256;
     static bool attr_set = false;
@@ -2253,27 +2265,30 @@ bool t_applies(int c_red, int c_out, int k, int pad) {
 }
 // The role-swapped kernel on prepared terms (p.taps, p.tap_*, p.fold): input [N][H][W][x_channels], output
 // [N][H][W][c_out], filter matrix as given by its tensor map.
+// Strips of 8 x th pixels for tc_conv_tp_kernel, th <= 32 and a multiple of 4 (the epilogue stores chunks of 4 rows):
+// worth it when they cover the image with little waste, the instructions stay wide and the SMs get enough tiles.
+bool tp_strip(int H, int W, int N, int co_tiles, int* th_out) {
+    const int nt = (H + 31) / 32;
+    const int th = ((H + nt - 1) / nt + 3) / 4 * 4;
+    const int tiles_w = (W + 7) / 8;
+    const double cover = (double)W * H / ((double)tiles_w * 8 * nt * th);
+    if (th > 32 || th < 24 || cover < TP_MIN_COVER || (int64_t)tiles_w * nt * N * co_tiles < TP_MIN_TILES) return false;
+    *th_out = th;
+    return true;
+}
+
 int launch_t_core(TParams p, const void* x, int x_channels, const CUtensorMap& mw, void* out, float* stat_partial, int* stat_blocks,
                   int N, int H, int W, int c_red, int c_out, int* status, cudaStream_t st, const char* what, bool a_mn) {
     p.H = H; p.W = W; p.N = N; p.c_red = c_red; p.c_out = c_out;
     choose_tile(256, W, H, N, &p.tw, &p.th, &p.tn);
     bool patch = false;
-#ifndef NO_TP_KERNEL
-    if (p.patch_ok) {
-        // strips of 8 x th pixels, th <= 32 and a multiple of 4 (the epilogue stores chunks of 4 rows): worth it when
-        // they cover the image with little waste, the instructions stay wide and every SM gets several tiles
-        const int nt = (H + 31) / 32;
-        int th = ((H + nt - 1) / nt + 3) / 4 * 4;
-        const int tiles_w = (W + 7) / 8;
-        const double cover = (double)W * H / ((double)tiles_w * 8 * nt * th);
-        if (th <= 32 && th >= 24 && cover >= TP_MIN_COVER && (int64_t)tiles_w * nt * N * ((c_out + 127) / 128) >= 4 * 148) {
-            patch = true;
-            p.tw = 8; p.th = th; p.tn = 1;
-            p.tile_cols = 8 * th;
-            p.patch_bytes = (uint32_t)(8 * (th + 2)) * 128;
-        }
+    int strip_h = 0;
+    if (p.patch_ok && tp_strip(H, W, N, (c_out + 127) / 128, &strip_h)) {
+        patch = true;
+        p.tw = 8; p.th = strip_h; p.tn = 1;
+        p.tile_cols = 8 * strip_h;
+        p.patch_bytes = (uint32_t)(8 * (strip_h + 2)) * 128;
     }
-#endif
     p.tw_log = 0; while ((1 << p.tw_log) < p.tw) ++p.tw_log;
     p.th_log = 0; while ((1 << p.th_log) < p.th) ++p.th_log;
     p.tiles_w = (W + p.tw - 1) / p.tw; p.tiles_h = (H + p.th - 1) / p.th; p.tiles_n = (N + p.tn - 1) / p.tn;
@@ -2335,6 +2350,7 @@ int launch_t(const void* x, const void* w_mat, void* out, float* stat_partial, i
     TParams p;
     p.taps = k * k;
     p.fold = 0;
+    p.pair = 0;
     p.patch_ok = k == 3 && pad == 1;
     p.ncols = 3;
     for (int dx = 0; dx < 3; ++dx)
@@ -2354,19 +2370,23 @@ int launch_t(const void* x, const void* w_mat, void* out, float* stat_partial, i
 // of pair j, the even pixel of pair j+1 - each a plain (aligned) box of the input viewed as [N][H][W/2][2*c_red].
 // A third of the products multiply zeros of the widened filter, but every instruction is 128 x 256 x 16 instead of
 // 128 x 64 x 16 at the same issue interval.  `work`: 128 * 12 * c_red bf16 for the widened filter.
-int64_t paired_work_bytes(int c_red) { return align_up((int64_t)128 * 12 * c_red * 2, 256); }
-// (on small tensors the 64-channel kernel with its resident filter is as fast: 32 x 56 x 56 pixels 0.023 against 0.026 ms)
-bool paired_applies(int c_red, int c_out, int k, int pad, int W, int64_t pixels) {
-    return c_out == 64 && k == 3 && pad == 1 && W % 2 == 0 && c_red % 64 == 0 && pixels >= 262144;
+// Two adjacent pixels as one pixel with 128 outputs.  On small tensors the 64-channel kernel with its resident filter
+// is as fast, unless the pairs tile into strips for the halo-patch kernel.
+bool paired_applies(int c_red, int c_out, int k, int pad, int N, int H, int W) {
+    if (!(c_out == 64 && k == 3 && pad == 1 && W % 2 == 0 && c_red % 64 == 0)) return false;
+    const int64_t pixels = (int64_t)N * H * W;
+    int th;
+    return pixels >= PAIR_MIN_PIXELS || (pixels >= PAIR_MIN_PIXELS_STRIPS && tp_strip(H, W / 2, N, 1, &th));
 }
 int launch_t_paired(const void* x, const void* w, int flip, void* out, float* stat_partial, int* stat_blocks, int N, int H, int W,
-                    int c_red, void* work, int* status, cudaStream_t st, const char* what) {
-    __nv_bfloat16* wp = (__nv_bfloat16*)work;
-    pair_filter_kernel<<<std::min(128 * 12 * c_red / 256, 148 * 8), 256, 0, st>>>((const __nv_bfloat16*)w, wp, c_red, flip);
-    CKPT_LAUNCH_CHECK("pixel-pair filter");
+                    int c_red, int* status, cudaStream_t st, const char* what) {
+    // term t = (filter row r, column sp of the four input columns 2j-1 .. 2j+2 that pair j reaches); pixel q of the
+    // pair sees column sp through filter column s = sp - q.  flip: w is the forward filter [c_red][9][64] and the
+    // input gradient takes the mirrored position.
     TParams p;
     p.taps = 12;
     p.fold = 64;
+    p.pair = 1;
     p.patch_ok = 1;
     p.ncols = 4;
     for (int sp = 0; sp < 4; ++sp)
@@ -2376,12 +2396,14 @@ int launch_t_paired(const void* x, const void* w, int flip, void* out, float* st
         p.tap_dh[t] = r - 1;
         p.tap_dw[t] = sp == 0 ? -1 : (sp == 3 ? 1 : 0);
         p.tap_xc[t] = (sp == 0 || sp == 2) ? c_red : 0;
-        p.tap_col[t] = t;
+        auto position = [&](int s) { return s < 0 || s > 2 ? -1 : (flip ? (2 - r) * 3 + (2 - s) : r * 3 + s); };
+        p.tap_col[t] = position(sp);
+        p.tap_col2[t] = position(sp - 1);
     }
     CUtensorMap mw;
-    int rc = make_mat_map(&mw, wp, 128, (int64_t)12 * c_red, 128);
+    int rc = flip ? make_mat_map(&mw, w, c_red, 9 * 64, 64) : make_mat_map(&mw, w, 64, (int64_t)9 * c_red, 64);
     if (rc) return rc;
-    return launch_t_core(p, x, 2 * c_red, mw, out, stat_partial, stat_blocks, N, H, W / 2, c_red, 128, status, st, what, false);
+    return launch_t_core(p, x, 2 * c_red, mw, out, stat_partial, stat_blocks, N, H, W / 2, c_red, 128, status, st, what, flip != 0);
 }
 
 // stat_partial / stat_blocks: null, or where the kernel leaves the batch-norm partial sums of its output
@@ -2391,8 +2413,8 @@ int launch_fwd_like(const void* x, const void* w_mat, void* out, const float* bi
                     int* stat_blocks = nullptr, bool b_mn = false, void* work = nullptr, int64_t work_bytes = 0) {
     // b_mn (1x1 only): w_mat is the forward filter [c_red][c_out] read in place (c_out a multiple of 64)
     if (stat_blocks) *stat_blocks = 0;
-    if (!bias && !relu && !b_mn && paired_applies(c_red, c_out, k, pad, W, (int64_t)N * H * W) && work && work_bytes >= paired_work_bytes(c_red))
-        return launch_t_paired(x, w_mat, 0, out, stat_partial, stat_blocks, N, H, W, c_red, work, status, st, what);
+    if (!bias && !relu && !b_mn && paired_applies(c_red, c_out, k, pad, N, H, W))
+        return launch_t_paired(x, w_mat, 0, out, stat_partial, stat_blocks, N, H, W, c_red, status, st, what);
     if (!bias && !relu && t_applies(c_red, c_out, k, pad) && (!b_mn || (k == 1 && (int64_t)N * H * W >= 256)))
         return launch_t(x, w_mat, out, stat_partial, stat_blocks, N, H, W, c_red, c_out, k, pad, status, st, what, b_mn);
     if (c_red == 64 && k == 3 && pad == 1 && c_out % 64 == 0 && !bias && !relu)
@@ -2599,9 +2621,6 @@ static int64_t tc_conv_stat_bytes(const ConvGeom& g) {
 static int64_t tc_conv_work_bytes(const ConvGeom& g);
 int64_t tc_conv_scratch_bytes(const ConvGeom& g) {
     int64_t b = std::max(std::max(tc_conv_stat_bytes(g), tc_conv_work_bytes(g)), fc_scratch_bytes(g));
-    if (g.stride == 1 && (paired_applies(g.cin, g.cout, g.k, g.pad, g.w, (int64_t)g.n * g.h * g.w) ||
-                          paired_applies(g.cout, g.cin, g.k, g.k - 1 - g.pad, g.w, (int64_t)g.n * g.h * g.w)))
-        b = std::max<int64_t>(b, (1 << 20) + 2 * paired_work_bytes(std::max(g.cin, g.cout)));
     return b;
 }
 
@@ -2683,14 +2702,6 @@ static int launch_strided_fwd(const ConvGeom& g, const void* x, const void* w, v
                           "strided conv forward (tensor cores)", false, stat_partial, stat_blocks);
 }
 
-// The widened filter of the pixel-pair form lives at the end of the caller's scratch region (its start holds
-// the partial sums); null when the region is too small.
-static void* paired_region(void* scratch, int64_t scratch_bytes, int c_red) {
-    const int64_t need = paired_work_bytes(c_red);
-    if (!scratch || scratch_bytes < need + (1 << 20)) return nullptr;
-    return (char*)scratch + ((scratch_bytes - need) & ~(int64_t)255);
-}
-
 // Forward convolution that also leaves the batch-norm partial sums of its output in `partial`
 // (*blocks of them; 0 when the kernel chosen for this shape does not gather them).
 int tc_conv_fwd_stats(const ConvGeom& g, const void* x, const void* w, void* z, float* partial, int* blocks, int* device_status,
@@ -2700,8 +2711,7 @@ int tc_conv_fwd_stats(const ConvGeom& g, const void* x, const void* w, void* z, 
     *blocks = 0;
     if (g.stride != 1) return launch_strided_fwd(g, x, w, z, device_status, (cudaStream_t)stream, partial, blocks);
     return launch_fwd_like(x, w, z, nullptr, 0, g.n, g.h, g.w, g.cin, g.cout, g.k, g.pad, device_status, (cudaStream_t)stream,
-                           "conv forward (tensor cores)", partial, blocks, false, paired_region(partial, partial_bytes, g.cin),
-                           paired_work_bytes(g.cin));
+                           "conv forward (tensor cores)", partial, blocks);
 }
 
 int tc_conv_fwd(const ConvGeom& g, const void* x, const void* w, void* z, const float* bias, int relu, void* scratch,
@@ -2714,8 +2724,7 @@ int tc_conv_fwd(const ConvGeom& g, const void* x, const void* w, void* z, const 
         return launch_strided_fwd(g, x, w, z, device_status, (cudaStream_t)stream);
     }
     return launch_fwd_like(x, w, z, bias, relu, g.n, g.h, g.w, g.cin, g.cout, g.k, g.pad, device_status, (cudaStream_t)stream,
-                           "conv forward (tensor cores)", nullptr, nullptr, false, paired_region(scratch, scratch_bytes, g.cin),
-                           paired_work_bytes(g.cin));
+                           "conv forward (tensor cores)");
 }
 
 int tc_conv_dgrad(const ConvGeom& g, const void* dz, const void* w, void* dx, void* scratch, int64_t scratch_bytes,
@@ -2776,14 +2785,14 @@ int tc_conv_dgrad(const ConvGeom& g, const void* dz, const void* w, void* dx, vo
         return launch_fwd_like(dz, w, dx, nullptr, 0, g.n, g.h, g.w, g.cout, g.cin, g.k, g.k - 1 - g.pad, device_status, st,
                                "conv dgrad (tensor cores)", nullptr, nullptr, true);
     }
-    if (paired_applies(g.cout, g.cin, g.k, g.k - 1 - g.pad, g.w, (int64_t)g.n * g.h * g.w)) {
-        // 64 input channels: the pixel-pair form, its widened filter built straight from the forward filter
-        if (void* work = paired_region(scratch, scratch_bytes, g.cout))
-            return launch_t_paired(dz, w, 1, dx, nullptr, nullptr, g.n, g.h, g.w, g.cout, work, device_status, st, "conv dgrad (tensor cores)");
-    }
+    // 64 input channels: the pixel-pair form, its filter operand read straight from the forward filter
+    if (paired_applies(g.cout, g.cin, g.k, g.k - 1 - g.pad, g.n, g.h, g.w))
+        return launch_t_paired(dz, w, 1, dx, nullptr, nullptr, g.n, g.h, g.w, g.cout, device_status, st, "conv dgrad (tensor cores)");
     if (t_applies(g.cout, g.cin, g.k, g.k - 1 - g.pad))
         return launch_t(dz, w, dx, nullptr, nullptr, g.n, g.h, g.w, g.cout, g.cin, g.k, g.k - 1 - g.pad, device_status, st,
                         "conv dgrad (tensor cores)", true);
+    if (g.cout == 64 && g.k == 3 && g.pad == 1 && g.cin % 64 == 0)
+        return launch_c64(dz, w, dx, nullptr, nullptr, g.n, g.h, g.w, g.cin, device_status, st, "conv dgrad (tensor cores)", true);
     const int64_t elems = (int64_t)g.cout * taps * g.cin;
     if (!scratch || scratch_bytes < elems * 2) { set_error("dgrad scratch too small"); return CKPT_E_WORKSPACE; }
     const unsigned grid = (unsigned)std::min<int64_t>((elems + 255) / 256, 148 * 8);
