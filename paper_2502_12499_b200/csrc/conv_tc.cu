@@ -1988,9 +1988,9 @@ __device__ __forceinline__ void add4(float4& a, const float4 b) { a.x += b.x; a.
 // The split kernels leave one partial result per persistent CTA (some tens of MB, mostly still in L2) for a few
 // hundred thousand outputs: a thread per output would leave most SMs idle and one load in flight per thread.  A block
 // is 32 float4 columns x Y slice groups; group y sums slices y, y + Y, ... and the groups are added in a fixed order.
-template <int Y>
+template <int X, int Y>
 __device__ __forceinline__ void store_group_sum(float4 acc, float4* out, bool ok) {
-    __shared__ float4 red[Y][32];
+    __shared__ float4 red[Y][X];
     if (Y > 1) {
         red[threadIdx.y][threadIdx.x] = acc;
         __syncthreads();
@@ -2018,19 +2018,19 @@ __global__ void __launch_bounds__(32 * Y) pairview_fold_kernel(const float* __re
             add4(acc, *reinterpret_cast<const float4*>(p1 + z * slice_stride));
         }
     }
-    store_group_sum<Y>(acc, reinterpret_cast<float4*>(out) + idx, ok);
+    store_group_sum<32, Y>(acc, reinterpret_cast<float4*>(out) + idx, ok);
 }
 
-template <int Y>
-__global__ void __launch_bounds__(32 * Y) slice_sum4_kernel(const float4* __restrict__ partial, float4* __restrict__ out, int64_t elems4, int slices) {
-    const int64_t e = (int64_t)blockIdx.x * 32 + threadIdx.x;
+template <int X, int Y>
+__global__ void __launch_bounds__(X * Y) slice_sum4_kernel(const float4* __restrict__ partial, float4* __restrict__ out, int64_t elems4, int slices) {
+    const int64_t e = (int64_t)blockIdx.x * X + threadIdx.x;
     const bool ok = e < elems4;
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
     if (ok) {
 #pragma unroll 4
         for (int z = threadIdx.y; z < slices; z += Y) add4(acc, partial[(size_t)z * elems4 + e]);
     }
-    store_group_sum<Y>(acc, out + e, ok);
+    store_group_sum<X, Y>(acc, out + e, ok);
 }
 
 __global__ void slice_sum_tc_kernel(const float* __restrict__ partial, float* __restrict__ out, int64_t elems, int slices) {
@@ -2049,9 +2049,9 @@ static void launch_slice_sum(const float* partial, float* out, int64_t elems, in
     }
     const int64_t elems4 = elems / 4;
     const unsigned blocks = (unsigned)((elems4 + 31) / 32);
-    if (slices >= 16) slice_sum4_kernel<8><<<blocks, dim3(32, 8), 0, st>>>((const float4*)partial, (float4*)out, elems4, slices);
-    else if (slices >= 4) slice_sum4_kernel<4><<<blocks, dim3(32, 4), 0, st>>>((const float4*)partial, (float4*)out, elems4, slices);
-    else slice_sum4_kernel<1><<<blocks, dim3(32, 1), 0, st>>>((const float4*)partial, (float4*)out, elems4, slices);
+    if (slices >= 16) slice_sum4_kernel<32, 8><<<blocks, dim3(32, 8), 0, st>>>((const float4*)partial, (float4*)out, elems4, slices);
+    else if (slices >= 4) slice_sum4_kernel<32, 4><<<blocks, dim3(32, 4), 0, st>>>((const float4*)partial, (float4*)out, elems4, slices);
+    else slice_sum4_kernel<256, 1><<<(unsigned)((elems4 + 255) / 256), dim3(256, 1), 0, st>>>((const float4*)partial, (float4*)out, elems4, slices);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -2368,10 +2368,11 @@ int launch_t(const void* x, const void* w_mat, void* out, float* stat_partial, i
 // 128 output channels (pixel of the pair, channel), so that the role-swapped kernel's M operand is full.  The pair
 // at column j reads input columns 2j-1 .. 2j+2: per filter row four terms - the odd pixel of pair j-1, both pixels
 // of pair j, the even pixel of pair j+1 - each a plain (aligned) box of the input viewed as [N][H][W/2][2*c_red].
-// A third of the products multiply zeros of the widened filter, but every instruction is 128 x 256 x 16 instead of
-// 128 x 64 x 16 at the same issue interval.  `work`: 128 * 12 * c_red bf16 for the widened filter.
-// Two adjacent pixels as one pixel with 128 outputs.  On small tensors the 64-channel kernel with its resident filter
-// is as fast, unless the pairs tile into strips for the halo-patch kernel.
+// The 128-row filter operand of a term is two 64-row boxes of the caller's filter, one per pixel of the pair; a term
+// that does not reach a pixel takes a box outside the matrix (zeros).  A third of the products therefore multiply
+// zeros, but every instruction is 128 x 256 x 16 instead of 128 x 64 x 16 at the same issue interval.
+// On small tensors the 64-channel kernel with its resident filter is as fast, unless the pairs tile into strips for
+// the halo-patch kernel.
 bool paired_applies(int c_red, int c_out, int k, int pad, int N, int H, int W) {
     if (!(c_out == 64 && k == 3 && pad == 1 && W % 2 == 0 && c_red % 64 == 0)) return false;
     const int64_t pixels = (int64_t)N * H * W;

@@ -56,6 +56,7 @@ TC_CASES = [
     (2, 9, 11, 192, 384, 1, 0),
     (3, 10, 6, 256, 64, 3, 1),
     (1, 515, 510, 64, 64, 3, 1),     # pixel pairs, one image, odd height
+    (4, 48, 104, 128, 256, 3, 1),    # halo-patch strips 24 rows high, two output-channel tiles
     # pixel-pair form of 64-channel outputs (large tensors only): forward 64 -> 64 and 128 -> 64, dgrad into 64 channels
     (5, 232, 228, 64, 64, 3, 1),     # ragged tiles in every dimension, pairs across tile borders
     (3, 300, 296, 128, 64, 3, 1),    # two reduction blocks per term
