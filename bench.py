@@ -203,6 +203,15 @@ def main():
     t0 = time.perf_counter()
     mask, peak = ck.plan(ck.ALGO_DYNAMIC_N, d)
     plan_us = 1e6 * (time.perf_counter() - t0)
+    # the three planners on this chain (host only; median of a few runs): Algorithm 3 is O(n^3), 5 O(n^2), 6 O(n)
+    planner_us = {}
+    for name, algo in (("algorithm_3", ck.ALGO_STATIC_N3), ("algorithm_5", ck.ALGO_DYNAMIC_N2), ("algorithm_6", ck.ALGO_DYNAMIC_N)):
+        runs = []
+        for _ in range(3 if len(d) > 200 else 15):
+            t1 = time.perf_counter()
+            ck.plan(algo, d)
+            runs.append(1e6 * (time.perf_counter() - t1))
+        planner_us[name] = round(sorted(runs)[len(runs) // 2], 1)
     store_all = ck.eval(ck.MODEL_STORE_ALL, d, None)
 
     params_h = wl.make_params(spec, seed=0)
@@ -269,7 +278,7 @@ def main():
                 "gpu_launches": int(rep["launches"]) * args.steps, "clocks": clocks, "roofline": roofline,
                 "peak_bytes": int(rep["peak_bytes"]), "predicted_bytes": int(peak), "store_all_bytes": int(store_all),
                 "peak_gib": rep["peak_bytes"] / 2 ** 30, "workspace_gib": chain.workspace_bytes() / 2 ** 30,
-                "recomputed_units": int(rep["recomputed_units"]), "plan_us": plan_us, "loss": rep["loss"],
+                "recomputed_units": int(rep["recomputed_units"]), "plan_us": plan_us, "planner_us": planner_us, "loss": rep["loss"],
                 "step_tflops": flops / (ms / args.steps * 1e-3) / 1e12,
                 "step_tensor_frac_of_sustained": flops / (ms / args.steps * 1e-3) / 1e12 / peaks["tflops_sustained"],
                 "peaks": peaks}
