@@ -37,6 +37,22 @@ def measured_peaks():
     return dict(hbm_gbs=6650.0, tflops_burst=1590.0, tflops_sustained=1400.0, source="fallback")
 
 
+def max_over_ranks(ms, world, device):
+    """Replicas share nothing but the clock: the job's time per timed region is the slowest rank's."""
+    if world == 1:
+        return ms
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_images_per_s(batch, world, steps, ms):
+    """Every rank runs `steps` steps of `batch` images on its own batch within `ms` milliseconds."""
+    return batch * world * steps / (ms * 1e-3)
+
+
 class ClockSampler:
     """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
     QUERY = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
@@ -244,11 +260,7 @@ def main():
             rep = step(batch, labels)
         e1.record(stream)
         barrier()
-        ms = e0.elapsed_time(e1)
-        if world > 1:
-            t = torch.tensor([ms], device="cuda")
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms = t.item()
+        ms = max_over_ranks(e0.elapsed_time(e1), world, "cuda")
         return ms, rep
 
     for _ in range(max(args.warmup, 3)):
@@ -262,9 +274,8 @@ def main():
     ms_e2e, rep_e2e = timed(x_pinned, labels_pinned, args.steps)
     clocks = sampler.stop() if rank == 0 else None
 
-    images = spec["batch"] * world * args.steps
-    value = images / (ms * 1e-3)
-    e2e_value = images / (ms_e2e * 1e-3)
+    value = whole_job_images_per_s(spec["batch"], world, args.steps, ms)
+    e2e_value = whole_job_images_per_s(spec["batch"], world, args.steps, ms_e2e)
 
     if rank == 0:
         peaks = measured_peaks()
