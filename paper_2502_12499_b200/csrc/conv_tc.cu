@@ -1670,14 +1670,14 @@ tc_conv_first_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* _
         fence_barrier_init();
         tma_prefetch_desc(&map_out);
     }
-    // filter tile: row = output channel, K = (tap, channel) in the first 27 of 64 columns
+    // filter tile: row = output channel, K = filter row r in columns 10 r .. 10 r + 8 (its 3 x 3 values), zeros elsewhere
     for (int i = threadIdx.x; i < 64 * 8; i += blockDim.x) {
         const int co = i / 8, chunk = i % 8;
         __align__(16) uint16_t v[8];
 #pragma unroll
         for (int e = 0; e < 8; ++e) {
-            const int k = chunk * 8 + e;
-            v[e] = k < 27 ? __ldg(reinterpret_cast<const uint16_t*>(w) + (size_t)(co0 + co) * 27 + k) : (uint16_t)0;
+            const int k = chunk * 8 + e, r = k / 10, tt = k % 10;      // filter row r in columns 10 r .. 10 r + 8
+            v[e] = (r < 3 && tt < 9) ? __ldg(reinterpret_cast<const uint16_t*>(w) + (size_t)(co0 + co) * 27 + r * 9 + tt) : (uint16_t)0;
         }
         *reinterpret_cast<uint4*>(b_tile + co * 128 + ((chunk ^ (co & 7)) * 16)) = *reinterpret_cast<const uint4*>(v);
     }
@@ -1723,25 +1723,33 @@ tc_conv_first_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* _
             asm volatile("bar.sync 2, 128;" ::: "memory");      // the segments of tile j are complete
             const long long p0 = ((long long)blockIdx.x + (long long)j * gridDim.x) * 128;
             const long long pix = p0 + t;
-            __align__(16) uint16_t v[32];
+            // The 9 values of a filter row are consecutive in the staged segment, from a 2-byte aligned address: six
+            // word loads from the word below it and five funnel shifts give the row's five words (the tenth value is
+            // padding); the columns outside the image are masked in the words.
+            uint32_t o[16];
 #pragma unroll
-            for (int e = 0; e < 32; ++e) v[e] = 0;
+            for (int e = 0; e < 16; ++e) o[e] = 0u;
             if (pix < p.pixels) {
-                const int ow = (int)(pix % p.W);
-                const int oh = (int)((pix / p.W) % p.H);
+                const uint32_t pp = (uint32_t)pix;                       // the host checks pixels < 2^31
+                const int ow = (int)(pp % (uint32_t)p.W);
+                const int oh = (int)((pp / (uint32_t)p.W) % (uint32_t)p.H);
 #pragma unroll
                 for (int r = 0; r < 3; ++r) {
                     const int ih = oh + r - 1;
                     if (ih < 0 || ih >= p.H) continue;
-                    const uint8_t* seg = stage + (buf * 3 + r) * kFirstSegBytes + (int)(seg_start(p0, r) & 15LL);
+                    const uint32_t a = smem_u32(stage + (buf * 3 + r) * kFirstSegBytes) + (uint32_t)(seg_start(p0, r) & 15LL) + (uint32_t)t * 6u;
+                    const uint32_t a4 = a & ~3u, sh = (a & 2u) * 8u;
+                    uint32_t wv[6];
 #pragma unroll
-                    for (int s2 = 0; s2 < 3; ++s2) {
-                        const int iw = ow + s2 - 1;
-                        if (iw < 0 || iw >= p.W) continue;
+                    for (int q = 0; q < 6; ++q) asm volatile("ld.shared.u32 %0, [%1];" : "=r"(wv[q]) : "r"(a4 + 4u * q));
+                    uint32_t g[5];
 #pragma unroll
-                        for (int c = 0; c < 3; ++c)
-                            v[(r * 3 + s2) * 3 + c] = *reinterpret_cast<const uint16_t*>(seg + ((t + s2) * 3 + c) * 2);
-                    }
+                    for (int q = 0; q < 5; ++q) g[q] = __funnelshift_r(wv[q], wv[q + 1], sh);
+                    g[4] &= 0xffffu;
+                    if (ow == 0) { g[0] = 0u; g[1] &= 0xffff0000u; }
+                    if (ow == p.W - 1) { g[3] = 0u; g[4] = 0u; }
+#pragma unroll
+                    for (int q = 0; q < 5; ++q) o[5 * r + q] = g[q];
                 }
             }
             if (!dead && !mbar_wait(a_empty0 + 8 * buf, ((uint32_t)(j >> 1) & 1u) ^ 1u, failed, status, 601)) dead = true;
@@ -1749,7 +1757,7 @@ tc_conv_first_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* _
             uint8_t* dst = a_tiles[buf] + t * 128;
 #pragma unroll
             for (int chunk = 0; chunk < 4; ++chunk)
-                *reinterpret_cast<uint4*>(dst + ((chunk ^ (t & 7)) * 16)) = reinterpret_cast<const uint4*>(v)[chunk];
+                *reinterpret_cast<uint4*>(dst + ((chunk ^ (t & 7)) * 16)) = make_uint4(o[4 * chunk], o[4 * chunk + 1], o[4 * chunk + 2], o[4 * chunk + 3]);
             fence_proxy_async();
             mbar_arrive(a_full0 + 8 * buf);
         }
@@ -2669,8 +2677,9 @@ int tc_first_conv_fwd(const ConvGeom& g, const void* x, const void* w, void* z, 
     int sms = 148, dev = 0;
     cudaGetDevice(&dev);
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    if (reinterpret_cast<uintptr_t>(x) & 15u) {
-        // the staged row segments are copied in 16-byte pieces: an input that is not 16-byte aligned takes the CUDA-core kernel
+    if ((reinterpret_cast<uintptr_t>(x) & 15u) || p.pixels >= (1LL << 31)) {
+        // the staged row segments are copied in 16-byte pieces and pixels are counted in 32 bits: an input that is not
+        // 16-byte aligned, or larger than that, takes the CUDA-core kernel
         if (blocks) *blocks = 0;
         return small_conv_fwd(g, x, w, z, stream);
     }
