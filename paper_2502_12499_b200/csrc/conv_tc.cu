@@ -1795,32 +1795,19 @@ tc_conv_first_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* _
             if (lane == 0) tma_store_wait_read<0>();          // the store of the previous tile has left this warp's slab
             __syncwarp();
             const long long pix0 = ((long long)blockIdx.x + (long long)j * gridDim.x) * 128;
-            const bool valid = pix0 + row < p.pixels;
             uint8_t* const orow = o_tile + row * 128;
 #pragma unroll
             for (int c0 = 0; c0 < 64; c0 += 32) {
                 uint32_t v[32];
                 tmem_ld32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * 64 + c0), v);
-                float r[32];
 #pragma unroll
                 for (int q = 0; q < 4; ++q) {
                     uint4 pk;
                     __nv_bfloat162* h = reinterpret_cast<__nv_bfloat162*>(&pk);
 #pragma unroll
-                    for (int e = 0; e < 4; ++e) {
+                    for (int e = 0; e < 4; ++e)
                         h[e] = __floats2bfloat162_rn(__uint_as_float(v[8 * q + 2 * e]), __uint_as_float(v[8 * q + 2 * e + 1]));
-                        const float2 f = __bfloat1622float2(h[e]);
-                        r[8 * q + 2 * e] = valid ? f.x : 0.f;
-                        r[8 * q + 2 * e + 1] = valid ? f.y : 0.f;
-                    }
                     *reinterpret_cast<uint4*>(orow + (((c0 / 8 + q) ^ (row & 7)) * 16)) = pk;
-                }
-                if (stats) {
-                    float sq[32];
-#pragma unroll
-                    for (int e = 0; e < 32; ++e) sq[e] = r[e] * r[e];
-                    s_acc[c0 / 32] += warp_column_sum(r, lane);
-                    q_acc[c0 / 32] += warp_column_sum(sq, lane);
                 }
             }
             tc_fence_before();
@@ -1831,12 +1818,26 @@ tc_conv_first_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* _
                 tma_store_2d(&map_out, smem_u32(o_tile) + (uint32_t)(quarter * 4096), co0, (int)(pix0 + quarter * 32));
                 tma_store_commit();
             }
+            if (stats) {
+                // The warp's 32 rounded rows are in its slab: lane l adds up channels 2l and 2l + 1 down the rows that
+                // hold pixels (one word per row, the 32 lanes read the 32 words of a row: no bank conflicts).  A
+                // thread owns a pixel here, so sums taken in registers would need a transposing shuffle reduction.
+                const long long left = p.pixels - (pix0 + quarter * 32);
+                const int rows_here = left < 0 ? 0 : (left > 32 ? 32 : (int)left);
+                const uint8_t* slab = o_tile + quarter * 4096;
+                for (int rr = 0; rr < rows_here; ++rr) {
+                    const uint32_t wv = *reinterpret_cast<const uint32_t*>(slab + rr * 128 + (((lane >> 2) ^ (rr & 7)) * 16) + (lane & 3) * 4);
+                    const float f0 = __uint_as_float(wv << 16), f1 = __uint_as_float(wv & 0xffff0000u);
+                    s_acc[0] += f0; q_acc[0] = fmaf(f0, f0, q_acc[0]);
+                    s_acc[1] += f1; q_acc[1] = fmaf(f1, f1, q_acc[1]);
+                }
+            }
         }
         if (lane == 0) tma_store_wait_all();
         if (stats) {
             // the four quarters of the CTA are added in a fixed order: one partial row per CTA
 #pragma unroll
-            for (int h = 0; h < 2; ++h) { stat_red[quarter][0][h * 32 + lane] = s_acc[h]; stat_red[quarter][1][h * 32 + lane] = q_acc[h]; }
+            for (int h = 0; h < 2; ++h) { stat_red[quarter][0][2 * lane + h] = s_acc[h]; stat_red[quarter][1][2 * lane + h] = q_acc[h]; }
             asm volatile("bar.sync 1, 128;" ::: "memory");
             if (quarter == 0) {
 #pragma unroll
