@@ -80,49 +80,67 @@ __global__ void __launch_bounds__(128) small_fwd_kernel(const __nv_bfloat16* __r
     }
 }
 
-// xcol[p][0..9*CIN) = the 3x3 neighbourhood of pixel p (zero outside the image), [9*CIN..WIDTH) = 0:
-// the first layer's input unfolded to WIDTH "channels" per pixel (64, or 32 when pixels are paired), so
-// that its weight gradient is a plain dz^T * xcol contraction for the tensor cores.
-template <int CIN, int WIDTH>
-__global__ void __launch_bounds__(256) unfold3x3_kernel(const __nv_bfloat16* __restrict__ x, __nv_bfloat16* __restrict__ xcol,
-                                                        int n, int h, int wd) {
-    constexpr int K = 9 * CIN;
+// The first layer's input (3 channels) unfolded to WIDTH "channels" per pixel (64, or 32 when pixels are paired), so
+// that its weight gradient is a plain dz^T * xcol contraction for the tensor cores.  Filter row r occupies columns
+// 10 r .. 10 r + 8: its 3 x 3 values are 9 consecutive values of input row oh + r - 1, fetched with six word loads
+// from the word below them and five funnel shifts; the rest of the row is zero.  Pixels at the left border and the
+// last two of a row (whose words would reach past the row) go value by value.
+template <int WIDTH>
+__global__ void __launch_bounds__(256) unfold3x3_rows_kernel(const __nv_bfloat16* __restrict__ x, uint4* __restrict__ xcol, int n, int h,
+                                                             int wd, int word_aligned) {
+    const uint32_t* x32 = reinterpret_cast<const uint32_t*>(x);
+    const uint16_t* x16 = reinterpret_cast<const uint16_t*>(x);
     const int64_t pixels = (int64_t)n * h * wd;
     for (int64_t p = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; p < pixels; p += (int64_t)gridDim.x * blockDim.x) {
         const int ow = (int)(p % wd);
         const int oh = (int)((p / wd) % h);
         const int64_t img = p / ((int64_t)wd * h);
-        __align__(16) __nv_bfloat16 v[WIDTH];
+        uint32_t o[WIDTH / 2];
 #pragma unroll
-        for (int i = K; i < WIDTH; ++i) v[i] = __float2bfloat16_rn(0.f);
+        for (int q = 0; q < WIDTH / 2; ++q) o[q] = 0u;
 #pragma unroll
         for (int r = 0; r < 3; ++r) {
+            const int ih = oh + r - 1;
+            if (ih < 0 || ih >= h) continue;
+            const int64_t e0 = ((img * h + ih) * wd + (ow - 1)) * 3;          // first of the 9 values
+            if (word_aligned && ow >= 1 && ow + 2 < wd) {
+                const uint32_t* src = x32 + (e0 >> 1);
+                const uint32_t sh = (uint32_t)(e0 & 1) * 16u;
+                uint32_t w[6];
 #pragma unroll
-            for (int s = 0; s < 3; ++s) {
-                const int ih = oh + r - 1, iw = ow + s - 1;
-                const bool in = ih >= 0 && ih < h && iw >= 0 && iw < wd;
-                const __nv_bfloat16* src = x + ((img * h + ih) * wd + iw) * CIN;
+                for (int q = 0; q < 6; ++q) w[q] = __ldg(src + q);
 #pragma unroll
-                for (int c = 0; c < CIN; ++c) v[(r * 3 + s) * CIN + c] = in ? src[c] : __float2bfloat16_rn(0.f);
+                for (int q = 0; q < 5; ++q) o[5 * r + q] = __funnelshift_r(w[q], w[q + 1], sh);
+                o[5 * r + 4] &= 0xffffu;
+            } else {
+#pragma unroll
+                for (int t = 0; t < 9; ++t) {
+                    const int iw = ow - 1 + t / 3;
+                    const uint32_t v = (iw >= 0 && iw < wd) ? (uint32_t)x16[e0 + t] : 0u;
+                    o[5 * r + t / 2] |= v << (16 * (t & 1));
+                }
             }
         }
-        uint4* dst = reinterpret_cast<uint4*>(xcol + p * WIDTH);
+        uint4* dst = xcol + p * (WIDTH / 8);
 #pragma unroll
-        for (int j = 0; j < WIDTH / 8; ++j) dst[j] = reinterpret_cast<const uint4*>(v)[j];
+        for (int q = 0; q < WIDTH / 8; ++q) dst[q] = make_uint4(o[4 * q], o[4 * q + 1], o[4 * q + 2], o[4 * q + 3]);
     }
 }
 
-// dw[co][0..K) = dwp[co][0..K) out of the padded [c_out][64] result
+// column of filter value k = (r, s, c) in an unfolded row
+__device__ __forceinline__ int unfolded_column(int k) { return (k / 9) * 10 + k % 9; }
+
+// dw[co][0..K) out of the padded [c_out][64] result
 __global__ void take_columns_kernel(const float* __restrict__ dwp, float* __restrict__ dw, int cout, int k) {
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
-    if (i < cout * k) dw[i] = dwp[(i / k) * 64 + i % k];
+    if (i < cout * k) dw[i] = dwp[(i / k) * 64 + unfolded_column(i % k)];
 }
-// Paired pixels: dwp is [(parity, co)][(parity, k)]; the gradient is the sum of its two diagonal blocks.
+// Paired pixels: dwp is [(parity, co)][(parity, column)]; the gradient is the sum of its two diagonal blocks.
 __global__ void take_paired_columns_kernel(const float* __restrict__ dwp, float* __restrict__ dw, int cout, int k) {
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i < cout * k) {
-        const int co = i / k, kk = i % k;
-        dw[i] = dwp[(size_t)co * 64 + kk] + dwp[(size_t)(cout + co) * 64 + 32 + kk];
+        const int co = i / k, col = unfolded_column(i % k);
+        dw[i] = dwp[(size_t)co * 64 + col] + dwp[(size_t)(cout + co) * 64 + 32 + col];
     }
 }
 
@@ -227,8 +245,9 @@ int small_conv_wgrad(const ConvGeom& g, const void* dz, const void* x, float* dw
     void* tc_scratch = base + xcol_bytes(g) + dwp_bytes(g);
     const int64_t pixels = (int64_t)g.n * g.h * g.w;
     const unsigned ugrid = (unsigned)std::min<int64_t>((pixels + 255) / 256, 148 * 16);
-    if (paired(g)) unfold3x3_kernel<3, 32><<<ugrid, 256, 0, st>>>((const __nv_bfloat16*)x, xcol, g.n, g.h, g.w);
-    else unfold3x3_kernel<3, 64><<<ugrid, 256, 0, st>>>((const __nv_bfloat16*)x, xcol, g.n, g.h, g.w);
+    const int word_aligned = (uintptr_t)x % 4 == 0 ? 1 : 0;
+    if (paired(g)) unfold3x3_rows_kernel<32><<<ugrid, 256, 0, st>>>((const __nv_bfloat16*)x, (uint4*)xcol, g.n, g.h, g.w, word_aligned);
+    else unfold3x3_rows_kernel<64><<<ugrid, 256, 0, st>>>((const __nv_bfloat16*)x, (uint4*)xcol, g.n, g.h, g.w, word_aligned);
     CKPT_LAUNCH_CHECK("first-layer unfold");
     const ConvGeom u = unfolded_geom(g);
     int rc = tc_conv_wgrad(u, dz, xcol, dwp, tc_scratch, scratch_bytes - xcol_bytes(g) - dwp_bytes(g), device_status, stream);
