@@ -6,7 +6,8 @@
   sampled output rows and input columns;
 * the whole checkpointed step of configurations 2, 3, 4 and 5 through properties that hold at any size:
   arena high-water == highest offset == planner's prediction (arena of exactly that size),
-  gradients bit-identical between the checkpointed and the store-all schedule, finite loss."""
+  gradients bit-identical between the checkpointed and the store-all schedule, finite loss;
+* configuration 2 as bench.py submits it: replayed from its recorded CUDA graph, and fed from pinned host buffers."""
 import time
 
 import numpy as np
@@ -152,6 +153,44 @@ def test_config2_vgg16_full_size_step():
     rep, rep0, peak = step_properties(wl.config(2))
     assert peak < 0.65 * rep0["peak_bytes"]             # 1.17 GiB against 1.82 GiB
     assert abs(rep["loss"] - np.log(1000.0)) < 2.0      # random labels, random weights
+
+
+def test_config2_vgg16_full_size_graph_replay_and_host_batch():
+    """The two submissions bench.py times: the recorded step replayed as a CUDA graph, and the same step fed from
+    pinned host buffers.  Both must reproduce the launch-by-launch step bit for bit."""
+    import torch
+    spec = wl.config(2)
+    params = wl.make_params(spec, seed=0)
+    runner = StepRunner(spec, params)
+    del params
+    mask, peak = ck.plan(ck.ALGO_DYNAMIC_N, runner.d)
+    x, labels = wl.make_batch(spec, seed=1)
+    x_host = torch.from_numpy(x).to(torch.bfloat16).pin_memory()
+    lab_host = torch.from_numpy(np.ascontiguousarray(labels, dtype=np.int32)).pin_memory()
+    xb, lab = x_host.cuda(), lab_host.cuda()
+    arena = torch.empty(peak, dtype=torch.uint8, device="cuda")
+
+    def step(batch, lbl):
+        arena.fill_(0xFF)
+        for g in runner.grads:
+            g.fill_(float("nan"))
+        rep = ck.train_step(runner.chain, mask, ck.POLICY_DYNAMIC, batch, lbl, runner.params, runner.grads, arena, runner.workspace)
+        torch.cuda.synchronize()
+        return rep, [g.detach().cpu().numpy().copy() for g in runner.grads]
+
+    rep0, g0 = step(xb, lab)
+    assert rep0["replayed"] == 0 and rep0["peak_bytes"] == peak and np.isfinite(rep0["loss"])
+    runner.chain.set_graph(True)
+    flags = []
+    for batch, lbl in ((xb, lab), (xb, lab), (xb, lab), (x_host, lab_host), (x_host, lab_host), (x_host, lab_host)):
+        rep, g = step(batch, lbl)
+        flags.append(rep["replayed"])
+        for key in ("peak_bytes", "extent_bytes", "predicted_bytes", "launches", "recomputed_units", "loss", "device_status"):
+            assert rep[key] == rep0[key], key
+        for a, b in zip(g, g0):
+            assert np.array_equal(a, b, equal_nan=True)
+    assert flags == [0, 1, 1, 0, 1, 1]          # each argument set: one plain step, then the recording
+    torch.cuda.empty_cache()
 
 
 def test_config2_vgg16_split_units_full_size_step():
