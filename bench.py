@@ -1,11 +1,19 @@
-"""Benchmark: checkpointed training-step throughput (images/s) of the VGG-16-shaped chain on B200.
+"""Benchmark: checkpointed training-step throughput (images/s) on B200.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--config 2]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--config 2] [--only]
 
 One "step" = one full pass of the hot path over one synthetic batch: forward keeping the planned
 checkpoints, loss, backward with segment recomputation, all weight gradients.  The plan is the
-O(n) dynamic planner's (Algorithm 6) and the schedule is Algorithm 4.  With N > 1 (torchrun) every
+dynamic planner's (Algorithm 6) and the schedule is Algorithm 4.  With N > 1 (torchrun) every
 rank runs an independent replica on its own batch: the step has no exchange between GPUs.
+
+The top-level fields of the JSON line are those of the headline workload (--config, default the VGG-16-shaped
+chain at batch 64).  At N = 1 the line also carries `configs`: the same measurements for every bf16 benchmark
+configuration (VGG-16 b64, ResNet-50 b128, ResNet-152 b256, the 1000-unit chain b32) - checkpointed and
+store-all (Algorithm 1) step times and the recompute overhead between them, end-to-end throughput from pinned
+host batches, device footprint (arena + workspace + parameters) under the plan and under store-all, planner times,
+and the roofline of its kernels: forward, dgrad and wgrad convolution mixes and the launch-weighted batch-norm
+and pooling bandwidth.  `--only` restricts the run to the headline workload.
 
 Prints one JSON line (rank 0).  `--impl reference` times the CPU oracle instead, on rank 0 only.
 """
@@ -127,24 +135,24 @@ def conv_flops(spec, plan_mask, shapes):
     return total, fwd
 
 
-def run_reference(args, spec, steps=None, warmup=None, budget_s=None):
-    """The CPU oracle, as it stands, on a bounded sample of the same workload.  With a time budget the
-    sample (images per step) is sized so that warmup + steps steps fit it (about 1.6 s per image of the
-    VGG-16 chain on 16 cores)."""
-    from oracle import numeric_oracle as no
+def host_cores():
     try:
         from threadpoolctl import threadpool_info
-        cores = max([p.get("num_threads", 1) for p in threadpool_info()] + [1])
+        return int(max([p.get("num_threads", 1) for p in threadpool_info()] + [1]))
     except Exception:
-        cores = os.cpu_count()
-    steps = args.steps_cpu if steps is None else max(1, steps)
-    warmup = args.warmup_cpu if warmup is None else max(0, warmup)
-    sample_batch = min(spec["batch"], args.cpu_batch)
-    if budget_s is not None:
-        sample_batch = int(max(1, min(sample_batch, budget_s / (1.6 * (steps + warmup)))))
+        return int(os.cpu_count() or 1)
+
+
+def run_reference(spec, sample_batch, steps, warmup=0):
+    """The CPU oracle, as it stands (float64 numpy, Algorithm 1 = store-all), on a bounded sample of the same workload:
+    the same chain on the first `sample_batch` images of the batch.  Returns images/s over `steps` timed steps."""
+    from oracle import numeric_oracle as no
+    import numpy  # noqa: F401  (loaded before the thread count is read)
     small = dict(spec, batch=sample_batch)
     params = wl.make_params(small, seed=0)
     x, labels = wl.make_batch(small, seed=1)
+    if spec["loss"] != "softmax_ce":
+        labels = None
     times = []
     for it in range(warmup + steps):
         t0 = time.perf_counter()
@@ -153,73 +161,29 @@ def run_reference(args, spec, steps=None, warmup=None, budget_s=None):
         if it >= warmup:
             times.append(dt)
     t = float(np.mean(times))
-    return dict(value=sample_batch / t, unit=UNIT, cores=int(cores), kind="oracle",
-                sample="store-all step of the same chain on a batch of %d of %d images, float64 numpy, %d timed step(s)"
-                       % (sample_batch, spec["batch"], len(times)), seconds_per_step=t)
+    return dict(value=sample_batch / t, unit=UNIT, cores=host_cores(), kind="oracle",
+                sample="store-all step (Algorithm 1) of the same chain on %d of its %d images, float64 numpy, mean of %d timed step(s)"
+                       % (sample_batch, spec["batch"], len(times)), seconds_per_step=t, steps=len(times))
 
 
-def main():
-    ap = argparse.ArgumentParser()
-    ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=30)
-    ap.add_argument("--warmup", type=int, default=3)
-    ap.add_argument("--impl", default="ours")
-    ap.add_argument("--config", type=int, default=2)
-    ap.add_argument("--batch", type=int, default=0, help="override the batch size (debugging only)")
-    ap.add_argument("--cpu-batch", type=int, default=4)
-    ap.add_argument("--steps-cpu", type=int, default=1)
-    ap.add_argument("--warmup-cpu", type=int, default=0)
-    ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--no-graph", action="store_true", help="launch every kernel of every step from the host")
-    ap.add_argument("--split-units", action="store_true",
-                    help="finer granularity: conv, batch norm and ReLU as chain units of their own")
-    args = ap.parse_args()
+def workload_name(spec):
+    return "%s: %d units, batch %d of %dx%dx%d %s, plan = Algorithm 6, schedule = Algorithm 4" % (
+        spec["name"], len(spec["units"]), spec["batch"], *spec["input_hwc"], spec["dtype"])
 
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
-    spec = wl.config(args.config)
-    if args.batch:
-        spec = dict(spec, batch=args.batch)
-    if args.split_units:
-        spec, _ = wl.split_units(spec)
-    config = {"workload": "%s: %d units, batch %d of %dx%dx%d %s, plan = Algorithm 6, schedule = Algorithm 4"
-                          % (spec["name"], len(spec["units"]), spec["batch"], *spec["input_hwc"], spec["dtype"]),
-              "l2": "inputs larger than L2 (every step streams > 1 GB of activations)",
-              "parallelism": "replicas x%d" % world if world > 1 else "single GPU",
-              "submission": "launch by launch" if args.no_graph else "CUDA graph replay of the recorded step"}
 
-    if args.impl == "reference":
-        if rank != 0:
-            return
-        # the requested step counts, each step a sample of the batch sized so that the run ends within about two minutes
-        cpu = run_reference(args, spec, steps=args.steps, warmup=args.warmup, budget_s=120.0)
-        line = {"impl": "reference", "metric": METRIC, "value": cpu["value"], "unit": UNIT, "n_gpus": args.gpus,
-                "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * cpu["seconds_per_step"],
-                "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-                "config": config, "cpu_baseline": cpu,
-                "e2e": {"value": cpu["value"], "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
-                "gpu_launches": 0}
-        print(json.dumps(line))
-        return
-
+def measure_config(spec, args, rank, world, steps, regions, with_roofline, peaks, sampler=None):
+    """All device measurements of one chain.  Returns a dict; `ms_per_step` is the median over `regions` timed
+    regions of exactly `steps` steps each (barrier + synchronize on both sides, CUDA events, max over ranks)."""
     import torch
     import torch.distributed as dist
     from paper_2502_12499_b200 import binding as ck
-
-    torch.cuda.set_device(local_rank)
-    if world > 1:
-        dist.init_process_group("nccl")
 
     chain = ck.Chain(spec)
     if not args.no_graph:
         chain.set_graph(True)        # a step whose arguments repeat is recorded once and replayed
     d = chain.sizes()
     shapes = [tuple(int(v) for v in s) for s in chain.shapes()]
-    t0 = time.perf_counter()
     mask, peak = ck.plan(ck.ALGO_DYNAMIC_N, d)
-    plan_us = 1e6 * (time.perf_counter() - t0)
-    # the three planners on this chain (host only; median of a few runs): Algorithm 3 is O(n^3), 5 O(n^2), 6 O(n)
     planner_us = {}
     for name, algo in (("algorithm_3", ck.ALGO_STATIC_N3), ("algorithm_5", ck.ALGO_DYNAMIC_N2), ("algorithm_6", ck.ALGO_DYNAMIC_N)):
         runs = []
@@ -233,109 +197,213 @@ def main():
     params_h = wl.make_params(spec, seed=0)
     params, grads, _ = ck.upload_params(chain, params_h)
     del params_h
+    param_bytes = sum(t.numel() * t.element_size() for t in params) + sum(t.numel() * t.element_size() for t in grads)
     x_h, labels_h = wl.make_batch(spec, seed=1 + rank)
     tdt = torch.bfloat16 if spec["dtype"] == "bf16" else torch.float32
     x_pinned = torch.from_numpy(x_h).to(tdt).pin_memory()
     labels_pinned = torch.from_numpy(labels_h).pin_memory()
-    x_dev = x_pinned.cuda()
-    labels_dev = labels_pinned.cuda()
-    arena = torch.empty(peak, dtype=torch.uint8, device="cuda")
-    workspace = torch.empty(chain.workspace_bytes(), dtype=torch.uint8, device="cuda")
+    x_dev, labels_dev = x_pinned.cuda(), labels_pinned.cuda()
+    ws_bytes = chain.workspace_bytes()
+    workspace = torch.empty(ws_bytes, dtype=torch.uint8, device="cuda")
     stream = torch.cuda.current_stream()
-
-    def step(batch, labels):
-        return ck.train_step(chain, mask, ck.POLICY_DYNAMIC, batch, labels, params, grads, arena, workspace, stream)
 
     def barrier():
         if world > 1:
             dist.barrier()
         torch.cuda.synchronize()
 
-    def timed(batch, labels, steps):
-        barrier()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record(stream)
-        rep = None
-        for _ in range(steps):
-            rep = step(batch, labels)
-        e1.record(stream)
-        barrier()
-        ms = max_over_ranks(e0.elapsed_time(e1), world, "cuda")
-        return ms, rep
+    def timed_regions(policy, plan_mask, arena, batch, labels, warm):
+        def step():
+            return ck.train_step(chain, plan_mask, policy, batch, labels, params, grads, arena, workspace, stream)
+        for _ in range(warm):
+            rep = step()
+        out = []
+        for _ in range(regions):
+            barrier()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            for _ in range(steps):
+                rep = step()
+            e1.record(stream)
+            barrier()
+            out.append(max_over_ranks(e0.elapsed_time(e1), world, "cuda"))
+        return out, rep
 
-    for _ in range(max(args.warmup, 3)):
-        rep = step(x_dev, labels_dev)
-    sampler = ClockSampler(local_rank)
-    if rank == 0:
+    warm = max(args.warmup, 3)
+    arena = torch.empty(peak, dtype=torch.uint8, device="cuda")
+    if sampler is not None:
         sampler.start()
-    ms, rep = timed(x_dev, labels_dev, args.steps)
-    for _ in range(3):                       # the end-to-end leg has its own arguments: warm it up (and record it) too
-        step(x_pinned, labels_pinned)
-    ms_e2e, rep_e2e = timed(x_pinned, labels_pinned, args.steps)
-    clocks = sampler.stop() if rank == 0 else None
+    ckpt_ms, rep = timed_regions(ck.POLICY_DYNAMIC, mask, arena, x_dev, labels_dev, warm)
+    e2e_ms, _ = timed_regions(ck.POLICY_DYNAMIC, mask, arena, x_pinned, labels_pinned, 3)
+    clocks = sampler.stop() if sampler is not None else None
+    del arena
+    arena_all = torch.empty(store_all, dtype=torch.uint8, device="cuda")
+    all_ms, rep_all = timed_regions(ck.POLICY_STORE_ALL, None, arena_all, x_dev, labels_dev, warm)
+    del arena_all
 
-    value = whole_job_images_per_s(spec["batch"], world, args.steps, ms)
-    e2e_value = whole_job_images_per_s(spec["batch"], world, args.steps, ms_e2e)
+    med = lambda v: float(sorted(v)[len(v) // 2])  # noqa: E731
+    ms, ms_e2e, ms_all = med(ckpt_ms) / steps, med(e2e_ms) / steps, med(all_ms) / steps
+    flops, _ = conv_flops(spec, mask, shapes)
+    gib = 2.0 ** 30
+    out = {"workload": workload_name(spec), "n_units": len(spec["units"]), "batch": spec["batch"], "steps": steps,
+           "regions_ms": [round(v, 3) for v in ckpt_ms], "ms_per_step": ms,
+           "images_per_s": whole_job_images_per_s(spec["batch"], world, 1, ms),
+           "e2e_images_per_s": whole_job_images_per_s(spec["batch"], world, 1, ms_e2e), "e2e_ms_per_step": ms_e2e,
+           "h2d_bytes_per_step": int(x_pinned.numel() * x_pinned.element_size() + labels_pinned.numel() * 4), "d2h_bytes_per_step": 12,
+           "store_all_ms_per_step": ms_all, "store_all_images_per_s": whole_job_images_per_s(spec["batch"], world, 1, ms_all),
+           "recompute_overhead_pct": 100.0 * (ms / ms_all - 1.0),
+           "recomputed_units": int(rep["recomputed_units"]), "checkpoints": int(mask.sum()),
+           "launches_per_step": int(rep["launches"]), "store_all_launches_per_step": int(rep_all["launches"]),
+           "memory_gib": {"arena_plan": peak / gib, "arena_store_all": store_all / gib, "arena_measured": rep["peak_bytes"] / gib,
+                          "workspace": ws_bytes / gib, "parameters_and_gradients": param_bytes / gib,
+                          "total_plan": (peak + ws_bytes + param_bytes) / gib, "total_store_all": (store_all + ws_bytes + param_bytes) / gib},
+           "peak_bytes": int(rep["peak_bytes"]), "predicted_bytes": int(peak), "store_all_bytes": int(store_all),
+           "planner_us": planner_us, "loss": rep["loss"],
+           "step_tflops": flops / (ms * 1e-3) / 1e12, "step_tensor_frac_of_sustained": flops / (ms * 1e-3) / 1e12 / peaks["tflops_sustained"],
+           "clocks": clocks}
+    assert rep["peak_bytes"] == peak and rep["loss"] == rep_all["loss"]
+    del params, grads, workspace, x_dev, chain
+    torch.cuda.empty_cache()
+    if with_roofline:
+        out["roofline"] = kernel_rooflines(spec, peaks)
+        torch.cuda.empty_cache()
+    return out
+
+
+def kernel_rooflines(spec, peaks):
+    """The step's kernels one at a time on the chain's own layer shapes (CUDA events, buffers rotated beyond the L2,
+    >= 20 launches and >= 10 ms per shape): forward, dgrad and wgrad convolution mixes against the measured dense-bf16
+    peak (burst: kernels timed in isolation) and, per shape, against whichever of the tensor and HBM roofs bounds it;
+    batch norm and 2x2 pooling over every tensor of the chain against the measured copy bandwidth."""
+    import bench_ops
+    out = {}
+    for what in ("fwd", "dgrad", "wgrad"):
+        mix = bench_ops.conv_mix(what, spec, peaks)
+        out["conv_" + what] = {"tflops": mix["tflops"], "frac_of_tensor_peak": mix["frac_of_tensor_peak"], "frac_of_roof": mix["frac_of_roof"],
+                               "launches": mix["launches"], "ms": mix["ms"], "flops": mix["flops"], "per_shape": mix["per_shape"]}
+    tot_f = sum(out["conv_" + w]["flops"] for w in ("fwd", "dgrad", "wgrad"))
+    tot_ms = sum(out["conv_" + w]["ms"] for w in ("fwd", "dgrad", "wgrad"))
+    out["conv_all"] = {"tflops": tot_f / tot_ms / 1e9, "frac_of_tensor_peak": tot_f / tot_ms / 1e9 / peaks["tflops_burst"],
+                       "frac_of_sustained": tot_f / tot_ms / 1e9 / peaks["tflops_sustained"]}
+    out["elementwise"] = bench_ops.elementwise_mix(spec, peaks)
+    return out
+
+
+HEADLINE_STEPS = {2: 30, 3: 20, 4: 8, 5: 6}        # timed steps per region: about a quarter to half a second each
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=0, help="timed steps per region of the headline workload (default: 30 for the VGG-16 chain)")
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours")
+    ap.add_argument("--config", type=int, default=2, help="headline workload: benchmark configuration 2..5")
+    ap.add_argument("--only", action="store_true", help="measure the headline workload only (no `configs` map)")
+    ap.add_argument("--regions", type=int, default=3, help="timed regions per measurement; the median is reported")
+    ap.add_argument("--batch", type=int, default=0, help="override the batch size (debugging only)")
+    ap.add_argument("--cpu-batch", type=int, default=2)
+    ap.add_argument("--steps-cpu", type=int, default=3)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-roofline", action="store_true")
+    ap.add_argument("--no-graph", action="store_true", help="launch every kernel of every step from the host")
+    ap.add_argument("--split-units", action="store_true",
+                    help="finer granularity: conv, batch norm and ReLU as chain units of their own")
+    args = ap.parse_args()
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+
+    def spec_of(index):
+        spec = wl.config(index)
+        if args.batch:
+            spec = dict(spec, batch=args.batch)
+        if args.split_units:
+            spec, _ = wl.split_units(spec)
+        return spec
+
+    spec = spec_of(args.config)
+    steps = args.steps or HEADLINE_STEPS.get(args.config, 10)
+    config = {"workload": workload_name(spec),
+              "l2": "inputs larger than L2 (every step streams > 1 GB of activations); single kernels rotate over buffer sets beyond the L2",
+              "parallelism": "replicas x%d" % world if world > 1 else "single GPU",
+              "submission": "launch by launch" if args.no_graph else "CUDA graph replay of the recorded step",
+              "timing": "median of %d regions of %d steps" % (args.regions, steps)}
+
+    if args.impl == "reference":
+        if rank != 0:
+            return
+        # the requested step counts, each step a sample of the batch sized so that the run ends within about two minutes
+        per_image = 4.5 if args.config == 2 else 2.5
+        sample = int(max(1, min(spec["batch"], 120.0 / (per_image * max(1, args.steps + args.warmup)))))
+        cpu = run_reference(spec, sample, steps=max(1, args.steps), warmup=max(0, args.warmup))
+        config["submission"] = "CPU oracle (float64 numpy), store-all schedule"
+        config["timing"] = "mean of %d steps" % cpu["steps"]
+        line = {"impl": "reference", "metric": METRIC, "value": cpu["value"], "unit": UNIT, "n_gpus": args.gpus,
+                "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * cpu["seconds_per_step"],
+                "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+                "config": config, "cpu_baseline": cpu,
+                "e2e": {"value": cpu["value"], "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+                "gpu_launches": 0}
+        print(json.dumps(line))
+        return
+
+    import torch
+    import torch.distributed as dist
+
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl")
+    peaks = measured_peaks()
+    roofs = rank == 0 and world == 1 and not args.no_roofline
+    sampler = ClockSampler(local_rank) if rank == 0 else None
+    head = measure_config(spec, args, rank, world, steps, args.regions, roofs, peaks, sampler)
+    configs = None
+    if world == 1 and not args.only and not args.batch and not args.split_units:
+        configs = {}
+        for index in (2, 3, 4, 5):
+            name = wl.config(index)["name"]
+            if index == args.config:
+                configs[name] = head
+            else:
+                configs[name] = measure_config(spec_of(index), args, rank, world, HEADLINE_STEPS[index], args.regions, roofs, peaks)
 
     if rank == 0:
-        peaks = measured_peaks()
-        flops, _ = conv_flops(spec, mask, shapes)
-        roofline = dominant_kernel_roofline(args.config, peaks, spec["batch"], shapes[1])
-        line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-                "warmup": max(args.warmup, 3), "ms_per_step": ms / args.steps, "higher_is_better": True,
+        line = {"metric": METRIC, "value": head["images_per_s"], "unit": UNIT, "n_gpus": world, "steps": steps,
+                "warmup": max(args.warmup, 3), "ms_per_step": head["ms_per_step"], "higher_is_better": True,
                 "scaling": "weak", "vs_baseline": None, "dtype": spec["dtype"], "data": "synthetic", "config": config,
-                "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": int(x_pinned.numel() * x_pinned.element_size() + labels_pinned.numel() * 4),
-                        "d2h_bytes_per_step": 12},
-                "gpu_launches": int(rep["launches"]) * args.steps, "clocks": clocks, "roofline": roofline,
-                "peak_bytes": int(rep["peak_bytes"]), "predicted_bytes": int(peak), "store_all_bytes": int(store_all),
-                "peak_gib": rep["peak_bytes"] / 2 ** 30, "workspace_gib": chain.workspace_bytes() / 2 ** 30,
-                "recomputed_units": int(rep["recomputed_units"]), "plan_us": plan_us, "planner_us": planner_us, "loss": rep["loss"],
-                "step_tflops": flops / (ms / args.steps * 1e-3) / 1e12,
-                "step_tensor_frac_of_sustained": flops / (ms / args.steps * 1e-3) / 1e12 / peaks["tflops_sustained"],
-                "peaks": peaks}
+                "e2e": {"value": head["e2e_images_per_s"], "unit": UNIT, "h2d_bytes_per_step": head["h2d_bytes_per_step"],
+                        "d2h_bytes_per_step": head["d2h_bytes_per_step"]},
+                "gpu_launches": head["launches_per_step"] * steps, "clocks": head["clocks"],
+                "peak_bytes": head["peak_bytes"], "predicted_bytes": head["predicted_bytes"], "store_all_bytes": head["store_all_bytes"],
+                "peak_gib": head["memory_gib"]["arena_measured"], "workspace_gib": head["memory_gib"]["workspace"],
+                "memory_gib": head["memory_gib"], "store_all_ms_per_step": head["store_all_ms_per_step"],
+                "recompute_overhead_pct": head["recompute_overhead_pct"], "recomputed_units": head["recomputed_units"],
+                "planner_us": head["planner_us"], "loss": head["loss"], "step_tflops": head["step_tflops"],
+                "step_tensor_frac_of_sustained": head["step_tensor_frac_of_sustained"], "peaks": peaks}
+        if "roofline" in head:
+            line["roofline"] = headline_roofline(head["roofline"], peaks)
+        if configs is not None:
+            line["configs"] = {k: {kk: vv for kk, vv in v.items() if kk != "clocks"} for k, v in configs.items()}
         if not args.no_cpu_baseline and world == 1:
-            line["cpu_baseline"] = run_reference(args, spec)
+            line["cpu_baseline"] = run_reference(spec, min(spec["batch"], args.cpu_batch), steps=args.steps_cpu)
         print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
 
 
-# DRAM traffic per launch of the conv-forward kernels over the layer mix of config 2, from one ncu pass
-# (profiles/conv_forward_vgg16_b64_dram_traffic.md).  Valid only for the kernel source it was taken
-# on: reported as null when csrc/conv_tc.cu has changed since.
-CONV_FWD_TRAFFIC = {"source_sha256": "9fdcfc7547a05b6256d957c5f1e983fb78b6a0d1b4a819e2b4cb5d3a7524a1d5", "bytes_per_launch": 169731242}
-
-
-def _kernel_source_sha():
-    import hashlib
-    path = os.path.join(ROOT, "paper_2502_12499_b200", "csrc", "conv_tc.cu")
-    return hashlib.sha256(open(path, "rb").read()).hexdigest()
-
-
-def dominant_kernel_roofline(config_index, peaks, batch, first_shape):
-    """The convolution-forward kernels (tcgen05; the role-swapped kernel for every layer but the two
-    64-channel ones) hold the largest share of the step: they run in the forward phase, in segment
-    recomputation and, on the transposed matrix, as dgrad.  Timed here on
-    every conv layer shape of the workload with CUDA events; achieved = sum of algorithmic FLOPs /
-    sum of launch times, against the measured dense-bf16 peak."""
-    from paper_2502_12499_b200 import opbench
-    mix = opbench.conv_mix("fwd", config_index, reps=3)
-    traffic = CONV_FWD_TRAFFIC["bytes_per_launch"] if CONV_FWD_TRAFFIC["source_sha256"] == _kernel_source_sha() else None
-    out = {"kernel": "tc_conv_tp_kernel / tc_conv_t_kernel (implicit-GEMM conv forward over the layer mix)", "bound": "tensor",
-           "achieved": mix["tflops"], "peak": peaks["tflops_burst"], "unit": "TFLOP/s", "frac": mix["tflops"] / peaks["tflops_burst"],
-           "peak_source": peaks["source"] + " (burst: kernels timed in isolation)", "traffic": traffic,
-           "launch_shapes": mix["launches"], "flops_per_launch": mix["flops"] / mix["launches"],
-           "ms_per_launch": mix["ms"] / mix["launches"], "per_layer": mix["per_layer"]}
-    # the memory-bound side of the step, for the record: batch-norm and 2x2 pooling passes on the largest
-    # activation of the chain (the output of its first unit)
-    b, (h, w, c) = batch, first_shape
-    f, g = opbench.bn("fwd", b * h * w, c), opbench.bn("bwd", b * h * w, c)
-    pf, pb = opbench.pool("fwd", b, h, w, c), opbench.pool("bwd", b, h, w, c)
-    out["elementwise"] = {"unit": "GB/s", "peak": peaks["hbm_gbs"],
-                          "bn_forward": f["gbs"], "bn_backward": g["gbs"], "maxpool_forward": pf["gbs"], "maxpool_backward": pb["gbs"],
-                          "frac": {"bn_forward": f["gbs"] / peaks["hbm_gbs"], "bn_backward": g["gbs"] / peaks["hbm_gbs"],
-                                   "maxpool_forward": pf["gbs"] / peaks["hbm_gbs"], "maxpool_backward": pb["gbs"] / peaks["hbm_gbs"]}}
-    return out
+def headline_roofline(r, peaks):
+    """The contract's roofline object for the dominant kernels of the headline workload: the implicit-GEMM
+    convolution-forward kernels (they run in the forward phase, in segment recomputation and, on the transposed
+    filter, as dgrad).  achieved = sum of algorithmic FLOPs of the chain's conv layers / sum of their launch times."""
+    f = r["conv_fwd"]
+    return {"kernel": "tc_conv_tp_kernel / tc_conv_t_kernel (implicit-GEMM conv forward over the chain's layer mix)", "bound": "tensor",
+            "achieved": f["tflops"], "peak": peaks["tflops_burst"], "unit": "TFLOP/s", "frac": f["frac_of_tensor_peak"],
+            "peak_source": peaks["source"] + " (burst: kernels timed in isolation)", "traffic": None,
+            "flops_per_launch": f["flops"] / f["launches"], "ms_per_launch": f["ms"] / f["launches"],
+            "conv_fwd": f, "conv_dgrad": r["conv_dgrad"], "conv_wgrad": r["conv_wgrad"], "conv_all": r["conv_all"],
+            "elementwise": r["elementwise"]}
 
 
 if __name__ == "__main__":

@@ -92,6 +92,16 @@ CKPT_API int ckpt_plan_counted(int algo, int64_t n, const int64_t* d, uint8_t* i
 #define CKPT_MODEL_STORE_ALL 2
 CKPT_API int ckpt_eval(int model, int64_t n, const int64_t* d, const uint8_t* is_ckpt, int64_t* peak_bytes);
 
+/* ---------------------------------------------------------------- launch log (host only)
+ *
+ * Which kernels ran.  ckpt_launch_log(1) clears the log and starts counting every kernel the library launches, by
+ * kernel name; ckpt_launch_log(0) stops.  ckpt_launch_log_read writes the counts as text, one "count<TAB>name" line
+ * per kernel, into text (host, capacity bytes, always terminated; may be null) and the size a complete copy needs
+ * into *needed.  A step replayed from its recording (ckpt_chain_set_graph) launches nothing from the host and is
+ * not counted. */
+CKPT_API int ckpt_launch_log(int enable);
+CKPT_API int ckpt_launch_log_read(char* text, int64_t capacity, int64_t* needed);
+
 /* ---------------------------------------------------------------- arena schedule (host only)
  *
  * Execution policies = the paper's three memory schedules:
@@ -204,6 +214,23 @@ CKPT_API int ckpt_chain_set_impl(ckpt_chain* chain, int impl);
  * recordings.  The library holds 64 bytes of pinned host memory per chain while enabled. */
 CKPT_API int ckpt_chain_set_graph(ckpt_chain* chain, int enable);
 
+/* Verification aid (off by default): the backward recursion of Eq. (3) made visible.  With a tap set, every
+ * ckpt_train_step also copies r_i = dL/dd_i, as it enters the backward step of unit i, to
+ * tap + (d_1 + .. + d_{i-1}) for i = n .. 1 (d_i bytes each, chain dtype; for a conv+BN+ReLU unit d_i is the stored
+ * convolution output, so r_i is the gradient with respect to that).  tap: device, at least d_1 + .. + d_n bytes,
+ * or null to switch the copies off.  Together with CKPT_POLICY_STORE_ALL - after which the arena holds d_0 .. d_n at
+ * consecutive offsets, Algorithm 1 freeing nothing - this lets a test check every unit's forward and backward
+ * against a reference on the unit's own inputs.  Costs one device copy per unit. */
+CKPT_API int ckpt_chain_set_gradient_tap(ckpt_chain* chain, void* tap, int64_t tap_bytes);
+
+/* Failure-path self-test (off by default).  With wait_runs_out = 1 every following step launches, after its loss,
+ * one extra single-warp kernel whose only wait has no producer and a limit of 2e5 clock cycles: the wait gives up,
+ * writes its code into the step's status word and the kernel returns, as every bounded wait of the tensor-core
+ * kernels does when its producer never arrives.  The step then finishes normally on the device and returns
+ * CKPT_E_DEVICE_TIMEOUT with report->device_status = 1; the context stays usable.  Nothing faults or spins without
+ * a limit. */
+CKPT_API int ckpt_chain_set_selftest(ckpt_chain* chain, int wait_runs_out);
+
 /* ---------------------------------------------------------------- the training step
  *
  * One pass of Algorithm 1, 2 or 4 (policy) over one batch.  Follows the paper's "Require: weights
@@ -256,6 +283,17 @@ CKPT_API int ckpt_train_step(ckpt_chain* chain, const uint8_t* is_ckpt, int poli
 typedef struct ckpt_conv_shape {
     int32_t n, h, w, c_in, c_out, k, stride, pad;
 } ckpt_conv_shape;
+
+/* Status of the single operations below.  Their tensor-core kernels bound every device-side wait; a wait that
+ * gives up records a code in a status word owned by the library and the kernel returns early, leaving its output
+ * incomplete.  ckpt_op_status waits for the device to go idle, writes that word to *status (host; 0 = every wait was
+ * satisfied), clears it, and returns CKPT_E_DEVICE_TIMEOUT when it was not 0.  Call it after a batch of single
+ * operations whose results matter.  (ckpt_train_step has its own status word and checks it itself.) */
+CKPT_API int ckpt_op_status(int32_t* status);
+/* Launches one single-warp kernel whose only wait has no producer and gives up after limit_cycles (1 .. 2e9) clock
+ * cycles, recording its code (9001) in the status word that ckpt_op_status reads: the failure path of the bounded
+ * waits, exercised without a fault.  Asynchronous on `stream`. */
+CKPT_API int ckpt_selftest_bounded_wait(int64_t limit_cycles, void* stream);
 
 CKPT_API int ckpt_conv2d_scratch_bytes(const ckpt_conv_shape* s, int dtype, int64_t* bytes);
 CKPT_API int ckpt_conv2d_forward(const ckpt_conv_shape* s, int dtype, int impl, const void* x, const void* w,

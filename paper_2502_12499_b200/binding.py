@@ -217,6 +217,14 @@ class Chain:
     def set_impl(self, impl):
         _check(lib().ckpt_chain_set_impl(self._h, C.c_int(impl)))
 
+    def set_gradient_tap(self, tap):
+        """ckpt_chain_set_gradient_tap: a device uint8 tensor of at least d_1 + .. + d_n bytes, or None."""
+        nbytes = 0 if tap is None else tap.numel() * tap.element_size()
+        _check(lib().ckpt_chain_set_gradient_tap(self._h, _dev(tap), C.c_int64(nbytes)))
+
+    def set_selftest(self, wait_runs_out):
+        _check(lib().ckpt_chain_set_selftest(self._h, C.c_int(1 if wait_runs_out else 0)))
+
     def set_graph(self, enable):
         """ckpt_chain_set_graph: record the launch sequence of a repeated step once and replay it."""
         _check(lib().ckpt_chain_set_graph(self._h, C.c_int(1 if enable else 0)))
@@ -272,6 +280,42 @@ def train_step(chain, is_ckpt, policy, batch, labels, params, grads, arena, work
                                C.c_int64(workspace.numel() * workspace.element_size()), _stream(stream), C.byref(rep))
     _check(rc)
     return {name: getattr(rep, name) for name, _ in StepReport._fields_}
+
+
+# ------------------------------------------------------------------------------------------------
+# launch log, status of the single operations
+# ------------------------------------------------------------------------------------------------
+
+def launch_log(enable):
+    _check(lib().ckpt_launch_log(C.c_int(1 if enable else 0)))
+
+
+def launch_log_read():
+    """ckpt_launch_log_read: {kernel name: launches}."""
+    need = C.c_int64(0)
+    _check(lib().ckpt_launch_log_read(None, C.c_int64(0), C.byref(need)))
+    buf = C.create_string_buffer(need.value)
+    _check(lib().ckpt_launch_log_read(buf, C.c_int64(need.value), C.byref(need)))
+    out = {}
+    for line in buf.value.decode().splitlines():
+        count, name = line.split("\t", 1)
+        out[name] = int(count)
+    return out
+
+
+def op_status():
+    """ckpt_op_status: raises CkptError(E_DEVICE_TIMEOUT) when a bounded wait of a single operation gave up."""
+    status = C.c_int32(0)
+    rc = lib().ckpt_op_status(C.byref(status))
+    if rc != 0:
+        err = CkptError(rc, lib().ckpt_last_error().decode())
+        err.status = status.value
+        raise err
+    return status.value
+
+
+def selftest_bounded_wait(limit_cycles, stream=None):
+    _check(lib().ckpt_selftest_bounded_wait(C.c_int64(limit_cycles), _stream(stream)))
 
 
 # ------------------------------------------------------------------------------------------------

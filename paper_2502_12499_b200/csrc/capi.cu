@@ -120,6 +120,24 @@ int ckpt_conv2d_wgrad(const ckpt_conv_shape* s, int dtype, int impl, const void*
     return simt_conv_wgrad(dtype, g, dz, x, dw, scratch, scratch_bytes, stream);
 }
 
+int ckpt_op_status(int32_t* status) {
+    if (!status) { set_error("status is null"); return CKPT_E_NULL; }
+    int* word = op_status_word();
+    if (!word) { set_error("status word unavailable"); return CKPT_E_NO_DEVICE; }
+    int value = 0;
+    cudaError_t e = cudaDeviceSynchronize();
+    if (e == cudaSuccess) e = cudaMemcpy(&value, word, sizeof(int), cudaMemcpyDeviceToHost);
+    if (e == cudaSuccess && value != 0) e = cudaMemset(word, 0, sizeof(int));
+    if (e != cudaSuccess) return cuda_fail(e, "reading the status word of the single operations");
+    *status = value;
+    if (value != 0) { set_error("a device-side wait gave up (status %d)", value); return CKPT_E_DEVICE_TIMEOUT; }
+    return CKPT_OK;
+}
+
+int ckpt_selftest_bounded_wait(int64_t limit_cycles, void* stream) {
+    return tc_selftest_wait((long long)limit_cycles, op_status_word(), stream);
+}
+
 int ckpt_bn_scratch_bytes(int64_t rows, int32_t c, int64_t* bytes) {
     if (!bytes) { set_error("bytes is null"); return CKPT_E_NULL; }
     if (rows < 1 || c < 1) { set_error("bad shape"); return CKPT_E_BAD_ARG; }

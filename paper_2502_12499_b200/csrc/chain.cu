@@ -29,6 +29,7 @@ struct ParamInfo { int64_t unit, elems; int32_t dtype; };
 // One captured step: the launch sequence of run_step for a fixed set of arguments.
 struct StepGraph {
     uint64_t key = 0;
+    std::vector<uint64_t> args;          // the argument set itself: a recording is replayed only for an exact match
     cudaGraph_t graph = nullptr;
     cudaGraphExec_t exec = nullptr;
     int64_t peak = 0, extent = 0, launches = 0, recomputed = 0;
@@ -51,6 +52,11 @@ struct ckpt_chain {
     int use_graph = 0;
     std::vector<ckpt::StepGraph> graphs;
     std::vector<uint64_t> seen_keys;     // argument sets that have run once without capture
+    uint64_t use_clock = 0;              // least-recently-used order of the recordings
+    // verification aids (off by default)
+    char* tap = nullptr;                 // device: where the step leaves every inter-unit gradient (ckpt_chain_set_gradient_tap)
+    int64_t tap_bytes = 0;
+    int selftest_wait = 0;               // the next steps include one kernel whose bounded wait runs out
     void* host_result = nullptr;         // pinned: loss (8 bytes) and status word of the last step
     cudaStream_t capture_stream = nullptr;   // recording happens here (the caller's stream may be the default one,
                                              // which cannot record); replays run on the caller's stream
@@ -390,6 +396,15 @@ static int decode_result(const ckpt_chain* ch, const void* result, double* loss_
     return CKPT_OK;
 }
 
+// Verification aid: r_i = dL/dd_i (Eq. (3)) as it enters unit i's backward, copied to the tap at the offset of d_i
+// among d_1..d_n.
+static int tap_gradient(StepCtx& c, int64_t i, const void* g) {
+    if (c.dry || !c.ch->tap || i < 1) return CKPT_OK;
+    int64_t off = 0;
+    for (int64_t k = 1; k < i; ++k) off += c.ch->d[k];
+    return device_copy(c.ch->tap + off, g, c.ch->d[i], c.stream);
+}
+
 static int run_step(StepCtx& c, double* loss_out) {
     ckpt_chain* ch = c.ch;
     const int64_t n = (int64_t)ch->units.size();
@@ -451,6 +466,8 @@ static int run_step(StepCtx& c, double* loss_out) {
         }
         if (rc) return rc;
         if ((rc = through_pending_act(c, n, ptr(n), g_cur))) return rc;
+        if ((rc = tap_gradient(c, n, g_cur))) return rc;
+        if (ch->selftest_wait && (rc = tc_selftest_wait(200000, c.status(), c.stream))) return rc;
     }
 
     // ---------------- backward phase
@@ -502,7 +519,10 @@ static int run_step(StepCtx& c, double* loss_out) {
         bypass_r_once = false;
         const bool need_dx = i > 1;   // the gradient w.r.t. the input batch is never used
         if ((rc = unit_backward(c, i, ptr(i - 1), ptr(i), g_cur, need_dx ? g_next : nullptr))) return rc;
-        if (need_dx) { g_cur = g_next; g_in_r = next_in_r; }
+        if (need_dx) {
+            g_cur = g_next; g_in_r = next_in_r;
+            if ((rc = tap_gradient(c, i - 1, g_cur))) return rc;
+        }
         if (c.policy == CKPT_POLICY_DYNAMIC) if ((rc = A.release(i))) return rc;
         if (c.stage_trace) c.stage_trace[2 * n + 1 - i] = A.live_bytes();
     }
@@ -544,15 +564,20 @@ static uint64_t mix(uint64_t h, uint64_t v) {
     h ^= v + 0x9E3779B97F4A7C15ull + (h << 6) + (h >> 2);
     return h * 0xFF51AFD7ED558CCDull;
 }
+// Everything a step's launch sequence depends on, as a list of words, and a hash of it.
 static uint64_t step_key(const ckpt_chain* ch, const uint8_t* is_ckpt, int policy, const void* batch, const int32_t* labels,
-                         void* const* params, void* const* grads, const void* arena, const void* ws) {
-    uint64_t h = mix(0x1234567ull, (uint64_t)policy);
-    h = mix(h, (uint64_t)(uintptr_t)batch); h = mix(h, (uint64_t)(uintptr_t)labels);
-    h = mix(h, (uint64_t)(uintptr_t)arena); h = mix(h, (uint64_t)(uintptr_t)ws);
-    h = mix(h, (uint64_t)ch->impl);
-    for (size_t p = 0; p < ch->params.size(); ++p) { h = mix(h, (uint64_t)(uintptr_t)params[p]); h = mix(h, (uint64_t)(uintptr_t)grads[p]); }
+                         void* const* params, void* const* grads, const void* arena, const void* ws, std::vector<uint64_t>* args) {
+    args->clear();
+    args->push_back((uint64_t)policy);
+    args->push_back((uint64_t)(uintptr_t)batch); args->push_back((uint64_t)(uintptr_t)labels);
+    args->push_back((uint64_t)(uintptr_t)arena); args->push_back((uint64_t)(uintptr_t)ws);
+    args->push_back((uint64_t)ch->impl);
+    args->push_back((uint64_t)(uintptr_t)ch->tap); args->push_back((uint64_t)ch->selftest_wait);
+    for (size_t p = 0; p < ch->params.size(); ++p) { args->push_back((uint64_t)(uintptr_t)params[p]); args->push_back((uint64_t)(uintptr_t)grads[p]); }
     if (policy != CKPT_POLICY_STORE_ALL)
-        for (size_t i = 0; i <= ch->units.size(); ++i) h = mix(h, (uint64_t)is_ckpt[i] + 3 * i);
+        for (size_t i = 0; i <= ch->units.size(); ++i) args->push_back((uint64_t)is_ckpt[i]);
+    uint64_t h = 0x1234567ull;
+    for (uint64_t v : *args) h = mix(h, v);
     return h;
 }
 // A copy from pageable host memory cannot be part of a captured sequence.
@@ -566,10 +591,9 @@ static bool graph_eligible(const void* batch, const int32_t* labels) {
     }
     return true;
 }
-static StepGraph* find_graph(ckpt_chain* ch, uint64_t key) {
-    static uint64_t clock = 0;
+static StepGraph* find_graph(ckpt_chain* ch, uint64_t key, const std::vector<uint64_t>& args) {
     for (StepGraph& g : ch->graphs)
-        if (g.key == key) { g.last_use = ++clock; return &g; }
+        if (g.key == key && g.args == args) { g.last_use = ++ch->use_clock; return &g; }
     return nullptr;
 }
 static void destroy_graph(StepGraph& g) {
@@ -582,7 +606,7 @@ static void drop_graphs(ckpt_chain* ch) {
     ch->graphs.clear();
     ch->seen_keys.clear();
 }
-static int capture_step(ckpt_chain* ch, StepCtx c, uint64_t key, StepGraph** out) {
+static int capture_step(ckpt_chain* ch, StepCtx c, uint64_t key, const std::vector<uint64_t>& args, StepGraph** out) {
     Arena ar(c.arena->capacity());
     c.arena = &ar;
     c.host_result = ch->host_result;
@@ -608,6 +632,7 @@ static int capture_step(ckpt_chain* ch, StepCtx c, uint64_t key, StepGraph** out
     e = cudaGraphInstantiate(&g.exec, g.graph, 0);
     if (e != cudaSuccess) { cudaGraphDestroy(g.graph); return cuda_fail(e, "instantiating the captured step"); }
     g.key = key;
+    g.args = args;
     g.peak = ar.high_water(); g.extent = ar.extent();
     g.launches = g_launches - launches0; g.recomputed = c.recomputed;
     if (ch->graphs.size() >= kMaxGraphs) {
@@ -617,7 +642,7 @@ static int capture_step(ckpt_chain* ch, StepCtx c, uint64_t key, StepGraph** out
         ch->graphs.erase(ch->graphs.begin() + victim);
     }
     ch->graphs.push_back(g);
-    *out = find_graph(ch, key);
+    *out = find_graph(ch, key, args);
     return CKPT_OK;
 }
 
@@ -908,12 +933,13 @@ int ckpt_train_step(ckpt_chain* chain, const uint8_t* is_ckpt, int policy, const
     c.batch = batch; c.labels = labels; c.stream = (cudaStream_t)stream; c.arena = &ar;
     double loss = 0;
     if (chain->use_graph && graph_eligible(batch, labels)) {
-        const uint64_t key = step_key(chain, is_ckpt, policy, batch, labels, params, grads, arena, workspace);
-        StepGraph* g = find_graph(chain, key);
+        std::vector<uint64_t> args;
+        const uint64_t key = step_key(chain, is_ckpt, policy, batch, labels, params, grads, arena, workspace, &args);
+        StepGraph* g = find_graph(chain, key, args);
         const bool seen = std::find(chain->seen_keys.begin(), chain->seen_keys.end(), key) != chain->seen_keys.end();
         if (!g && seen) {
             // second step with these arguments: record its launch sequence
-            rc = capture_step(chain, c, key, &g);
+            rc = capture_step(chain, c, key, args, &g);
             if (rc) return rc;
         }
         if (g) {
@@ -954,6 +980,22 @@ int ckpt_chain_set_graph(ckpt_chain* chain, int enable) {
     }
     chain->use_graph = enable ? 1 : 0;
     if (!enable) drop_graphs(chain);
+    return CKPT_OK;
+}
+
+int ckpt_chain_set_gradient_tap(ckpt_chain* chain, void* tap, int64_t tap_bytes) {
+    if (!chain) { set_error("null pointer"); return CKPT_E_NULL; }
+    int64_t need = 0;
+    for (size_t i = 1; i < chain->d.size(); ++i) need += chain->d[i];
+    if (tap && tap_bytes < need) { set_error("gradient tap of %lld bytes, %lld needed", (long long)tap_bytes, (long long)need); return CKPT_E_WORKSPACE; }
+    chain->tap = (char*)tap;
+    chain->tap_bytes = tap ? tap_bytes : 0;
+    return CKPT_OK;
+}
+
+int ckpt_chain_set_selftest(ckpt_chain* chain, int wait_runs_out) {
+    if (!chain) { set_error("null pointer"); return CKPT_E_NULL; }
+    chain->selftest_wait = wait_runs_out ? 1 : 0;
     return CKPT_OK;
 }
 

@@ -17,13 +17,6 @@
 
 namespace ckpt {
 
-#define CKPT_LAUNCH_CHECK(what)                                   \
-    do {                                                          \
-        ++g_launches;                                             \
-        cudaError_t e__ = cudaGetLastError();                     \
-        if (e__ != cudaSuccess) return cuda_fail(e__, what);      \
-    } while (0)
-
 namespace {
 
 template <int CIN>

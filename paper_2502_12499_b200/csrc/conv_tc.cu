@@ -28,13 +28,6 @@
 
 namespace ckpt {
 
-#define CKPT_LAUNCH_CHECK(what)                                   \
-    do {                                                          \
-        ++g_launches;                                             \
-        cudaError_t e__ = cudaGetLastError();                     \
-        if (e__ != cudaSuccess) return cuda_fail(e__, what);      \
-    } while (0)
-
 namespace {
 
 constexpr int kThreads = 192;
@@ -658,16 +651,11 @@ tc_conv_t_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
 // rings of their own (three patches, six boxes) so that the next columns are in flight while the
 // tensor core works on this one.
 // ------------------------------------------------------------------------------------------------
-#ifndef TP_MIN_COVER
-#define TP_MIN_COVER 0.87
-#endif
-#ifndef TP_MIN_TILES
-#define TP_MIN_TILES 200
-#endif
-#ifndef PAIR_MIN_PIXELS
-#define PAIR_MIN_PIXELS 262144
-#define PAIR_MIN_PIXELS_STRIPS 65536
-#endif
+// Dispatch thresholds of the halo-patch and pixel-pair forms (measured on the VGG-16 and 1000-unit chains).
+constexpr double TP_MIN_COVER = 0.87;              // share of a strip tiling that is real pixels
+constexpr long long TP_MIN_TILES = 200;            // (strip, channel tile) items: below that the SMs do not fill
+constexpr long long PAIR_MIN_PIXELS = 262144;      // pixel pairs on the plain role-swapped kernel from this size on,
+constexpr long long PAIR_MIN_PIXELS_STRIPS = 65536;    // from this size when the pairs tile into strips
 constexpr int kTpBoxes = 6, kTpPatches = 3;
 constexpr uint32_t kTpPatchSlot = 34 * 1024;
 constexpr uint32_t kTpSmem = kTpBoxes * 16384 + kTpPatches * kTpPatchSlot + 256 + 4 * 2 * 2048 + 1024;
@@ -1624,10 +1612,7 @@ struct FirstParams {
     int m_tiles;
 };
 constexpr int kFirstThreads = 288;
-#ifndef FIRST_CTAS
-#define FIRST_CTAS 3
-#endif
-constexpr int kFirstCtasPerSm = FIRST_CTAS;      // each holds 128 of the 512 tensor-memory columns
+constexpr int kFirstCtasPerSm = 3;      // each holds 128 of the 512 tensor-memory columns
 
 constexpr int kFirstSegBytes = 832;                 // one staged input row segment: 130 pixels x 6 bytes plus alignment slack
 constexpr int kFirstSegChunks = kFirstSegBytes / 16;
@@ -2158,7 +2143,7 @@ int launch_c64(const void* x, const void* w_mat, void* out, float* stat_partial,
         attr_set = true;
     }
     tc_conv_c64_kernel<<<p.ctas_per_n * p.n_tiles, kThreads, smem, st>>>(mx, mw, (__nv_bfloat16*)out, stat_partial, p, status);
-    CKPT_LAUNCH_CHECK(what);
+    CKPT_LAUNCH_CHECK_NAMED("tc_conv_c64_kernel", what);
     if (stat_blocks) *stat_blocks = 4 * p.ctas_per_n;
     return CKPT_OK;
 }
@@ -2202,7 +2187,7 @@ int launch_halo(const void* x, const void* w_mat, void* out, float* stat_partial
         attr_set = true;
     }
     tc_conv_halo_kernel<<<p.ctas_per_n * p.n_tiles, kThreads, smem, st>>>(mx, mw, (__nv_bfloat16*)out, stat_partial, p, status);
-    CKPT_LAUNCH_CHECK(what);
+    CKPT_LAUNCH_CHECK_NAMED("tc_conv_halo_kernel", what);
     if (stat_blocks) *stat_blocks = 4 * p.ctas_per_n;
     return CKPT_OK;
 }
@@ -2259,7 +2244,7 @@ int launch_generic(FwdParams p, const void* a, int a_n, int a_h, int a_w, const 
     if (gather) *stat_blocks = 4 * p.ctas_per_n;
     if (b_mn) tc_conv_fwd_kernel<true><<<(unsigned)ctas, kThreads, smem, st>>>(mx, mw, (__nv_bfloat16*)out, bias, relu, nullptr, p, status);
     else tc_conv_fwd_kernel<false><<<(unsigned)ctas, kThreads, smem, st>>>(mx, mw, (__nv_bfloat16*)out, bias, relu, gather ? stat_partial : nullptr, p, status);
-    CKPT_LAUNCH_CHECK(what);
+    CKPT_LAUNCH_CHECK_NAMED("tc_conv_fwd_kernel", what);
     return CKPT_OK;
 }
 
@@ -2345,12 +2330,12 @@ int launch_t_core(TParams p, const void* x, int x_channels, const CUtensorMap& m
         }
         if (a_mn) tc_conv_tp_kernel<true><<<p.ctas_per_co * p.co_tiles, kThreads, kTpSmem, st>>>(mx, mw, mo, stat_blocks ? stat_partial : nullptr, p, status);
         else tc_conv_tp_kernel<false><<<p.ctas_per_co * p.co_tiles, kThreads, kTpSmem, st>>>(mx, mw, mo, stat_blocks ? stat_partial : nullptr, p, status);
-        CKPT_LAUNCH_CHECK(what);
+        CKPT_LAUNCH_CHECK_NAMED("tc_conv_tp_kernel", what);
         return CKPT_OK;
     }
     if (a_mn) tc_conv_t_kernel<true><<<p.ctas_per_co * p.co_tiles, kThreads, smem, st>>>(mx, mw, mo, stat_blocks ? stat_partial : nullptr, p, status);
     else tc_conv_t_kernel<false><<<p.ctas_per_co * p.co_tiles, kThreads, smem, st>>>(mx, mw, mo, stat_blocks ? stat_partial : nullptr, p, status);
-    CKPT_LAUNCH_CHECK(what);
+    CKPT_LAUNCH_CHECK_NAMED("tc_conv_t_kernel", what);
     return CKPT_OK;
 }
 
@@ -2491,11 +2476,11 @@ int launch_fc(const ConvGeom& g, const void* x, const void* w, void* z, const fl
     }
     dim3 grid(m_tiles, slices);
     tc_fc_fwd_kernel<<<grid, kThreads, smem, st>>>(mw, mx, (float*)scratch, p, status);
-    CKPT_LAUNCH_CHECK("fully connected forward (tensor cores)");
+    CKPT_LAUNCH_CHECK_NAMED("tc_fc_fwd_kernel", "fully connected forward (tensor cores)");
     const int64_t elems = (int64_t)g.n * g.cout;
     fc_reduce_kernel<<<(unsigned)((elems + 255) / 256), 256, 0, st>>>((const float*)scratch, slices, elems, g.cout, bias, relu,
                                                                       (__nv_bfloat16*)z);
-    CKPT_LAUNCH_CHECK("fully connected slice sum");
+    CKPT_LAUNCH_CHECK_NAMED("fc_reduce_kernel", "fully connected slice sum");
     return CKPT_OK;
 }
 
@@ -2559,9 +2544,7 @@ void wgrad_c64_plan(const ConvGeom& g, W64Params* p) {
 }  // namespace
 
 namespace {
-#ifndef WROWS_MIN_W
-#define WROWS_MIN_W 14
-#endif
+constexpr int WROWS_MIN_W = 14;
 bool wgrad_rows_applies(const ConvGeom& g) {
     return g.k == 3 && g.pad == 1 && g.stride == 1 && g.cin % 128 == 0 && g.cout % 64 == 0 && g.w >= WROWS_MIN_W && g.h >= 8;
 }
@@ -2697,7 +2680,7 @@ int tc_first_conv_fwd(const ConvGeom& g, const void* x, const void* w, void* z, 
     if (blocks) *blocks = partial ? (int)grid.x : 0;
     tc_conv_first_kernel<<<grid, kFirstThreads, kFirstSmem, (cudaStream_t)stream>>>((const __nv_bfloat16*)x, (const __nv_bfloat16*)w,
                                                                                    map_out, partial, p, device_status);
-    CKPT_LAUNCH_CHECK("first-layer conv forward (tensor cores)");
+    CKPT_LAUNCH_CHECK_NAMED("tc_conv_first_kernel", "first-layer conv forward (tensor cores)");
     return CKPT_OK;
 }
 
@@ -2754,7 +2737,7 @@ int tc_conv_dgrad(const ConvGeom& g, const void* dz, const void* w, void* dx, vo
             if (!scratch || scratch_bytes < elems * 2) { set_error("dgrad scratch too small"); return CKPT_E_WORKSPACE; }
             const unsigned grid = (unsigned)std::min<int64_t>((elems + 255) / 256, 148 * 8);
             transpose_flip_kernel<<<grid, 256, 0, st>>>((const __nv_bfloat16*)w, (__nv_bfloat16*)scratch, g.cout, taps, g.cin);
-            CKPT_LAUNCH_CHECK("dgrad matrix transpose");
+            CKPT_LAUNCH_CHECK_NAMED("transpose_flip_kernel", "dgrad matrix transpose");
             w_mat = scratch;
         }
         // a filter narrower than the stride leaves whole classes without a term: their gradient is zero
@@ -2808,7 +2791,7 @@ int tc_conv_dgrad(const ConvGeom& g, const void* dz, const void* w, void* dx, vo
     if (!scratch || scratch_bytes < elems * 2) { set_error("dgrad scratch too small"); return CKPT_E_WORKSPACE; }
     const unsigned grid = (unsigned)std::min<int64_t>((elems + 255) / 256, 148 * 8);
     transpose_flip_kernel<<<grid, 256, 0, st>>>((const __nv_bfloat16*)w, (__nv_bfloat16*)scratch, g.cout, taps, g.cin);
-    CKPT_LAUNCH_CHECK("dgrad matrix transpose");
+    CKPT_LAUNCH_CHECK_NAMED("transpose_flip_kernel", "dgrad matrix transpose");
     return launch_fwd_like(dz, scratch, dx, nullptr, 0, g.n, g.h, g.w, g.cout, g.cin, g.k, g.k - 1 - g.pad, device_status, st,
                            "conv dgrad (tensor cores)");
 }
@@ -2842,9 +2825,9 @@ int tc_conv_wgrad(const ConvGeom& g, const void* dz, const void* x, float* dw, v
         const size_t smem = (size_t)p.stages * p.stage_bytes + 1024 + 256;
         dim3 grid(p.slices, 2, co_tiles);
         tc_wgrad_rows_kernel<<<grid, kThreads, smem, st>>>(mdz, mx, (float*)scratch, p, device_status);
-        CKPT_LAUNCH_CHECK("conv wgrad, 64 input channels as pixel pairs (tensor cores)");
+        CKPT_LAUNCH_CHECK_NAMED("tc_wgrad_rows_kernel (pixel pairs)", "conv wgrad, 64 input channels as pixel pairs (tensor cores)");
         pairview_fold_kernel<8><<<(unsigned)((g.cout * 144 + 31) / 32), dim3(32, 8), 0, st>>>((const float*)scratch, dw, g.cout, p.slices);
-        CKPT_LAUNCH_CHECK("wgrad pair fold");
+        CKPT_LAUNCH_CHECK_NAMED("pairview_fold_kernel", "wgrad pair fold");
         return CKPT_OK;
     }
     if (wgrad_c64_applies(g)) {
@@ -2867,9 +2850,9 @@ int tc_conv_wgrad(const ConvGeom& g, const void* dz, const void* x, float* dw, v
         const size_t smem = (size_t)p.stages * p.stage_bytes + 1024 + 256;
         dim3 grid(p.slices, g.cout / 64);
         tc_wgrad_c64_kernel<<<grid, kThreads, smem, st>>>(mdz, mx, (float*)scratch, p, device_status);
-        CKPT_LAUNCH_CHECK("conv wgrad, 64 input channels (tensor cores)");
+        CKPT_LAUNCH_CHECK_NAMED("tc_wgrad_c64_kernel", "conv wgrad, 64 input channels (tensor cores)");
         launch_slice_sum((const float*)scratch, dw, elems, p.slices, st);
-        CKPT_LAUNCH_CHECK("wgrad slice sum");
+        CKPT_LAUNCH_CHECK_NAMED("slice_sum_kernel", "wgrad slice sum");
         return CKPT_OK;
     }
     if (wgrad_rows_applies(g)) {
@@ -2889,9 +2872,9 @@ int tc_conv_wgrad(const ConvGeom& g, const void* dz, const void* x, float* dw, v
         const size_t smem = (size_t)p.stages * p.stage_bytes + 1024 + 256;
         dim3 grid(p.slices, pairs, co_tiles);
         tc_wgrad_rows_kernel<<<grid, kThreads, smem, st>>>(mdz, mx, (float*)scratch, p, device_status);
-        CKPT_LAUNCH_CHECK("conv wgrad, shared vertical taps (tensor cores)");
+        CKPT_LAUNCH_CHECK_NAMED("tc_wgrad_rows_kernel", "conv wgrad, shared vertical taps (tensor cores)");
         launch_slice_sum((const float*)scratch, dw, elems, p.slices, st);
-        CKPT_LAUNCH_CHECK("wgrad slice sum");
+        CKPT_LAUNCH_CHECK_NAMED("slice_sum_kernel", "wgrad slice sum");
         return CKPT_OK;
     }
     WgradParams p;
@@ -2915,11 +2898,37 @@ int tc_conv_wgrad(const ConvGeom& g, const void* dz, const void* x, float* dw, v
     float* target = slices > 1 ? (float*)scratch : dw;
     dim3 grid(slices, groups, co_tiles);
     tc_conv_wgrad_kernel<<<grid, kThreads, smem, st>>>(mdz, mx, target, p, device_status);
-    CKPT_LAUNCH_CHECK("conv wgrad (tensor cores)");
+    CKPT_LAUNCH_CHECK_NAMED("tc_conv_wgrad_kernel", "conv wgrad (tensor cores)");
     if (slices > 1) {
         launch_slice_sum((const float*)scratch, dw, elems, slices, st);
-        CKPT_LAUNCH_CHECK("wgrad slice sum");
+        CKPT_LAUNCH_CHECK_NAMED("slice_sum_kernel", "wgrad slice sum");
     }
+    return CKPT_OK;
+}
+
+// A wait that nothing will ever satisfy, with a short limit: the barrier is initialised for one arrival and no
+// thread arrives.  The wait gives up after `limit_cycles`, records its code in the status word like every other
+// bounded wait of this file, and the kernel returns.  Used to exercise the status path end to end.
+namespace {
+constexpr int kSelftestCode = 9001;
+__global__ void selftest_wait_kernel(long long limit_cycles, int* status) {
+    __shared__ __align__(8) uint64_t bar;
+    __shared__ int failed;
+    if (threadIdx.x == 0) {
+        failed = 0;
+        mbar_init(smem_u32(&bar), 1);
+        fence_barrier_init();
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) mbar_wait(smem_u32(&bar), 0, &failed, status, kSelftestCode, limit_cycles);
+}
+}  // namespace
+
+int tc_selftest_wait(long long limit_cycles, int* device_status, void* stream) {
+    if (!device_status) { set_error("no status word"); return CKPT_E_NULL; }
+    if (limit_cycles < 1 || limit_cycles > 2000000000LL) { set_error("wait limit must be 1 .. 2e9 cycles"); return CKPT_E_BAD_ARG; }
+    selftest_wait_kernel<<<1, 32, 0, (cudaStream_t)stream>>>(limit_cycles, device_status);
+    CKPT_LAUNCH_CHECK_NAMED("selftest_wait_kernel", "bounded-wait self-test");
     return CKPT_OK;
 }
 

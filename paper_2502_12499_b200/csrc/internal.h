@@ -17,6 +17,17 @@ inline int64_t dtype_size(int dtype) { return dtype == CKPT_DTYPE_BF16 ? 2 : 4; 
 
 // Number of kernels launched since the library was loaded (incremented by every launcher).
 extern int64_t g_launches;
+// Counts one launch and, while the launch log is on, files it under `kernel` (see ckpt_launch_log).
+void note_launch(const char* kernel);
+
+// After a kernel launch: count it under `kernel` and turn a launch error into CKPT_E_CUDA (message `what`).
+#define CKPT_LAUNCH_CHECK_NAMED(kernel, what)                     \
+    do {                                                          \
+        ::ckpt::note_launch(kernel);                              \
+        cudaError_t e__ = cudaGetLastError();                     \
+        if (e__ != cudaSuccess) return ::ckpt::cuda_fail(e__, what); \
+    } while (0)
+#define CKPT_LAUNCH_CHECK(what) CKPT_LAUNCH_CHECK_NAMED(what, what)
 
 // ------------------------------------------------------------------ host planners (planner.cpp)
 int validate_sizes(int64_t n, const int64_t* d);
@@ -101,6 +112,10 @@ int tc_conv_dgrad(const ConvGeom& g, const void* dz, const void* w, void* dx, vo
                   int64_t scratch_bytes, int* device_status, void* stream);
 int tc_conv_wgrad(const ConvGeom& g, const void* dz, const void* x, float* dw, void* scratch,
                   int64_t scratch_bytes, int* device_status, void* stream);
+
+// One tiny kernel whose only wait has no producer and gives up after `limit_cycles` (1 .. 2e9), writing its code
+// into the status word: the bounded-wait path, run to its limit on purpose.
+int tc_selftest_wait(long long limit_cycles, int* device_status, void* stream);
 
 int64_t bn_scratch_bytes(int64_t rows, int c);
 int bn_relu_forward(int dtype, int64_t rows, int c, const void* z, const float* gamma, const float* beta,

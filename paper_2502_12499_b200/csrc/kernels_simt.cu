@@ -20,13 +20,6 @@ int cuda_fail(int err, const char* what) {
     return CKPT_E_CUDA;
 }
 
-#define CKPT_LAUNCH_CHECK(what)                                   \
-    do {                                                          \
-        ++g_launches;                                             \
-        cudaError_t e__ = cudaGetLastError();                     \
-        if (e__ != cudaSuccess) return cuda_fail(e__, what);      \
-    } while (0)
-
 ConvGeom make_geom(const ckpt_conv_shape& s) {
     ConvGeom g;
     g.n = s.n; g.h = s.h; g.w = s.w; g.cin = s.c_in; g.cout = s.c_out; g.k = s.k; g.stride = s.stride; g.pad = s.pad;

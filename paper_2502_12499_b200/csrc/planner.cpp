@@ -7,7 +7,11 @@
 #include <algorithm>
 #include <cstdarg>
 #include <cstdio>
+#include <cstring>
 #include <limits>
+#include <map>
+#include <mutex>
+#include <string>
 
 #include "internal.h"
 
@@ -15,6 +19,18 @@ namespace ckpt {
 
 static thread_local char g_error[512] = "";
 int64_t g_launches = 0;
+
+// Launch log: kernel name -> launches since the log was switched on.
+static std::mutex g_log_mutex;
+static bool g_log_on = false;
+static std::map<std::string, int64_t> g_log;
+
+void note_launch(const char* kernel) {
+    ++g_launches;
+    if (!g_log_on) return;
+    std::lock_guard<std::mutex> lock(g_log_mutex);
+    ++g_log[kernel ? kernel : "?"];
+}
 
 void set_error(const char* fmt, ...) {
     va_list ap;
@@ -294,6 +310,33 @@ int ckpt_plan(int algo, int64_t n, const int64_t* d, uint8_t* is_ckpt, int64_t* 
 
 int ckpt_eval(int model, int64_t n, const int64_t* d, const uint8_t* is_ckpt, int64_t* peak_bytes) {
     return ckpt::eval_model(model, n, d, is_ckpt, peak_bytes);
+}
+
+}  // extern "C"
+
+extern "C" {
+
+int ckpt_launch_log(int enable) {
+    std::lock_guard<std::mutex> lock(ckpt::g_log_mutex);
+    if (enable) ckpt::g_log.clear();
+    ckpt::g_log_on = enable != 0;
+    return CKPT_OK;
+}
+
+int ckpt_launch_log_read(char* text, int64_t capacity, int64_t* needed) {
+    if (!needed) { ckpt::set_error("needed is null"); return CKPT_E_NULL; }
+    std::string out;
+    {
+        std::lock_guard<std::mutex> lock(ckpt::g_log_mutex);
+        for (const auto& kv : ckpt::g_log) out += std::to_string(kv.second) + "\t" + kv.first + "\n";
+    }
+    *needed = (int64_t)out.size() + 1;
+    if (text && capacity > 0) {
+        const size_t m = std::min<size_t>(out.size(), (size_t)capacity - 1);
+        memcpy(text, out.data(), m);
+        text[m] = 0;
+    }
+    return CKPT_OK;
 }
 
 }  // extern "C"

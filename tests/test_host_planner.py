@@ -278,3 +278,9 @@ def test_split_units_chain_and_plan():
     flat_f = ck.flatten_params(fine, wl.split_params(origin, shapes))
     assert [(origin[fi][0], name) for fi, name, _ in flat_f] == [(ui, name) for ui, name, _ in flat_c]
     assert chain.num_params() == len(flat_f)
+
+
+def test_launch_log_is_empty_without_launches():
+    ck.launch_log(True)
+    assert ck.launch_log_read() == {}
+    ck.launch_log(False)
