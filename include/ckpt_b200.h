@@ -92,6 +92,25 @@ CKPT_API int ckpt_plan_counted(int algo, int64_t n, const int64_t* d, uint8_t* i
 #define CKPT_MODEL_STORE_ALL 2
 CKPT_API int ckpt_eval(int model, int64_t n, const int64_t* d, const uint8_t* is_ckpt, int64_t* peak_bytes);
 
+/* Eq. (memory) with three sizes per tensor instead of one - the more faithful model of what a framework holds that
+ * Section 6 leaves as future work, built on Observations (1)-(2) of Section 4.  Tensor t occupies kept[t] bytes while
+ * it is a checkpoint, live[t] bytes while it is an interior tensor of the segment being processed (a unit's backward
+ * may need more than its output: a pre-normalisation copy, the interior tensors of a residual block), and its
+ * gradient r_t occupies grad[t] bytes.  Backward at checkpoint i with previous checkpoint h then holds
+ *     sum of kept[c], c in C, c <= i  +  sum of live[t], h < t < i  +  max grad[t], h <= t < i
+ *     (+ max grad[t], h < t <= i, when incoming != 0: the buffer of the gradient each step reads, which Eq. (memory)
+ *     leaves out),
+ * and the objective is the maximum over i.  kept = live = grad = d with incoming = 0 is Eq. (memory) itself.
+ *   ckpt_plan_sizes: CKPT_ALGO_DYNAMIC_N2 (the recursion of Algorithm 5, any sizes) or CKPT_ALGO_DYNAMIC_N (the
+ *     queue-based search of Algorithm 6; its Lemma 1, U(i,j) increasing in j, holds when live[t] >= kept[t] for
+ *     0 < t < n, otherwise CKPT_E_BAD_ARG).  Same tie rule and outputs as ckpt_plan.
+ *   ckpt_eval_sizes: the objective of a given set.
+ * All arrays: host, n+1 entries, every entry >= 1. */
+CKPT_API int ckpt_plan_sizes(int algo, int64_t n, const int64_t* kept, const int64_t* live, const int64_t* grad, int incoming,
+                    uint8_t* is_ckpt, int64_t* peak_bytes);
+CKPT_API int ckpt_eval_sizes(int64_t n, const int64_t* kept, const int64_t* live, const int64_t* grad, int incoming,
+                    const uint8_t* is_ckpt, int64_t* peak_bytes);
+
 /* ---------------------------------------------------------------- launch log (host only)
  *
  * Which kernels ran.  ckpt_launch_log(1) clears the log and starts counting every kernel the library launches, by

@@ -29,6 +29,13 @@ Functions and the passage each one restates:
                          contiguous range sums of d_1..d_{n-1} plus 0, output d_n forced.
 * ``dp_dynamic_reference`` - Algorithm 5 (the O(n^2) recursion of Eq. (T-rec)) with i running down
                          to 0 and j up to n inclusive.
+* ``eval_two_size`` / ``brute_force_two_size`` / ``dp_two_size_reference`` - Eq. (memory) with three sizes per
+                         tensor instead of one (the more faithful allocator model the paper's Section 6 leaves as
+                         future work, following Observations (1)-(2) of Section 4): what d_t occupies as a
+                         checkpoint, what it occupies inside the segment being processed, and the size of its
+                         gradient; optionally with the buffer of the *incoming* gradient counted next to the
+                         paper's output-gradient buffer.  With all three sizes equal to d and no incoming buffer
+                         it is Eq. (memory) itself.
 
 Tie rule (the paper gives none; several optimal sets usually exist):
 
@@ -390,6 +397,83 @@ def dp_dynamic_reference(d):
     while C[-1] != n:
         C.append(nxt[C[-1]])
     return M[0], C, M
+
+
+# --------------------------------------------------------------------------------------------
+# Eq. (memory) with separate sizes for a checkpoint, a segment tensor and a gradient
+# --------------------------------------------------------------------------------------------
+
+def _check_three(kept, live, grad):
+    n = _check_sizes(kept)
+    if len(live) != n + 1 or len(grad) != n + 1:
+        raise ValueError("kept, live and grad must have n+1 entries each")
+    _check_sizes(live)
+    _check_sizes(grad)
+    return n
+
+
+def s_term_two_size(live, grad, h, i, incoming):
+    """Eq. (s) with the segment tensors at their live size, the output-gradient buffer sized by the gradients
+    r_h .. r_{i-1} it holds and, when `incoming`, a second buffer for the gradients r_{h+1} .. r_i the steps read."""
+    s = sum(live[t] for t in range(h + 1, i)) + max(grad[t] for t in range(h, i))
+    if incoming:
+        s += max(grad[t] for t in range(h + 1, i + 1))
+    return s
+
+
+def eval_two_size(kept, live, grad, C, incoming=False):
+    """max over checkpoints i > 0 of [checkpoints up to i at their kept size + s_term_two_size(h, i)]."""
+    n = _check_three(kept, live, grad)
+    cs = _check_set(n, C)
+    worst = 0
+    for pos in range(1, len(cs)):
+        h, i = cs[pos - 1], cs[pos]
+        worst = max(worst, sum(kept[c] for c in cs[: pos + 1]) + s_term_two_size(live, grad, h, i, incoming))
+    return worst
+
+
+def brute_force_two_size(kept, live, grad, incoming=False):
+    """Optimum of eval_two_size over every feasible set, and the canonical optimal set under the dynamic tie rule
+    (from checkpoint i the smallest next checkpoint that starts an optimal solution of the suffix problem)."""
+    n = _check_three(kept, live, grad)
+
+    def suffix_value(C):
+        worst = kept[C[0]] if len(C) == 1 else 0
+        for pos in range(1, len(C)):
+            worst = max(worst, sum(kept[c] for c in C[: pos + 1]) + s_term_two_size(live, grad, C[pos - 1], C[pos], incoming))
+        return worst
+
+    best_of, first = {n: kept[n]}, {}
+    for i in range(n - 1, -1, -1):
+        best = best_first = None
+        for inner in _all_sets(i, n):
+            C = (i,) + inner + (n,)
+            v = suffix_value(C)
+            if best is None or v < best or (v == best and C[1] < best_first):
+                best, best_first = v, C[1]
+        best_of[i], first[i] = best, best_first
+    C = [0]
+    while C[-1] != n:
+        C.append(first[C[-1]])
+    return dict(value=best_of[0], set=C)
+
+
+def dp_two_size_reference(kept, live, grad, incoming=False):
+    """Algorithm 5 on the three-size objective: M(n) = kept_n; M(i) = min over i < j <= n of
+    max(kept_i + M(j), kept_i + s(i,j) + kept_j), first minimiser wins.  Returns (value, set)."""
+    n = _check_three(kept, live, grad)
+    M = [None] * (n + 1)
+    nxt = [None] * (n + 1)
+    M[n] = kept[n]
+    for i in range(n - 1, -1, -1):
+        for j in range(i + 1, n + 1):
+            v = max(kept[i] + M[j], kept[i] + s_term_two_size(live, grad, i, j, incoming) + kept[j])
+            if M[i] is None or v < M[i]:
+                M[i], nxt[i] = v, j
+    C = [0]
+    while C[-1] != n:
+        C.append(nxt[C[-1]])
+    return M[0], C
 
 
 def sqrt_n_plan(n):

@@ -123,6 +123,27 @@ def eval(model, d, is_ckpt):  # noqa: A001 - named after ckpt_eval
     return peak.value
 
 
+def plan_sizes(algo, kept, live, grad, incoming=False):
+    """ckpt_plan_sizes: returns (is_ckpt uint8[n+1], peak_bytes)."""
+    kept, live, grad = _i64(kept), _i64(live), _i64(grad)
+    n = len(kept) - 1
+    mask = np.zeros(max(n + 1, 1), dtype=np.uint8)
+    peak = C.c_int64(0)
+    _check(lib().ckpt_plan_sizes(C.c_int(algo), C.c_int64(n), _ptr(kept, C.c_int64), _ptr(live, C.c_int64), _ptr(grad, C.c_int64),
+                                 C.c_int(1 if incoming else 0), _ptr(mask, C.c_uint8), C.byref(peak)))
+    return mask, peak.value
+
+
+def eval_sizes(kept, live, grad, is_ckpt, incoming=False):
+    kept, live, grad = _i64(kept), _i64(live), _i64(grad)
+    n = len(kept) - 1
+    mask = np.ascontiguousarray(is_ckpt, dtype=np.uint8)
+    peak = C.c_int64(0)
+    _check(lib().ckpt_eval_sizes(C.c_int64(n), _ptr(kept, C.c_int64), _ptr(live, C.c_int64), _ptr(grad, C.c_int64),
+                                 C.c_int(1 if incoming else 0), _ptr(mask, C.c_uint8), C.byref(peak)))
+    return peak.value
+
+
 def arena_dry_run(policy, d, is_ckpt):
     """ckpt_arena_dry_run: returns dict(events=int64[k,4], high_water, extent)."""
     d = _i64(d)

@@ -178,18 +178,31 @@ static void walk_next(int64_t n, const std::vector<int64_t>& nxt, uint8_t* is_ck
     is_ckpt[n] = 1;
 }
 
-int plan_dynamic_n2(int64_t n, const int64_t* d, uint8_t* is_ckpt, int64_t* peak, int64_t* work) {
+// Sizes of the generalised Eq. (memory): what tensor t occupies as a checkpoint (kept), inside the segment being
+// processed (live), and the size of its gradient (grad); `incoming` adds a second buffer for the gradients
+// r_{h+1} .. r_i that the steps of a segment read.  kept = live = grad = d without `incoming` is the paper's objective.
+struct Sizes3 {
+    const int64_t* kept;
+    const int64_t* live;
+    const int64_t* grad;
+    int incoming;
+};
+
+// Algorithm 5 on the generalised sizes: M(n) = kept_n, M(i) = min over j > i of kept_i + max(M(j), U(i,j)),
+// U(i,j) = s(i,j) + kept_j, s(i,j) = sum of live_{i+1..j-1} + max grad_{i..j-1} (+ max grad_{i+1..j}).
+static int plan_dynamic_n2_sizes(int64_t n, const Sizes3& z, uint8_t* is_ckpt, int64_t* peak, int64_t* work) {
     std::vector<int64_t> M(n + 1), nxt(n + 1, -1);
-    M[n] = d[n];
+    M[n] = z.kept[n];
     int64_t steps = 0;
     for (int64_t i = n - 1; i >= 0; --i) {
-        int64_t seg_sum = 0, seg_max = d[i], best = -1, best_j = -1;
+        int64_t seg_sum = 0, out_max = z.grad[i], in_max = 0, best = -1, best_j = -1;
         for (int64_t j = i + 1; j <= n; ++j) {
-            int64_t u = seg_sum + seg_max + d[j];              // U(i,j) = s(i,j) + d_j
-            int64_t v = d[i] + std::max(M[j], u);
+            in_max = std::max(in_max, z.grad[j]);
+            int64_t u = seg_sum + out_max + (z.incoming ? in_max : 0) + z.kept[j];
+            int64_t v = z.kept[i] + std::max(M[j], u);
             if (best < 0 || v < best) { best = v; best_j = j; }
-            seg_sum += d[j];
-            seg_max = std::max(seg_max, d[j]);
+            seg_sum += z.live[j];
+            out_max = std::max(out_max, z.grad[j]);
             ++steps;
         }
         M[i] = best;
@@ -201,45 +214,61 @@ int plan_dynamic_n2(int64_t n, const int64_t* d, uint8_t* is_ckpt, int64_t* peak
     return CKPT_OK;
 }
 
+int plan_dynamic_n2(int64_t n, const int64_t* d, uint8_t* is_ckpt, int64_t* peak, int64_t* work) {
+    const Sizes3 z{d, d, d, 0};
+    return plan_dynamic_n2_sizes(n, z, is_ckpt, peak, work);
+}
+
 // ------------------------------------------------------------------------------------------------
 // Algorithm 6.  Q holds indices with strictly decreasing M as the index grows (Lemma 2); only Q has
 // to be searched (Lemma 3); U(i,.) increases along Q while M decreases, so max(M(j),U(i,j)) is
 // unimodal along Q and its minimum sits at the crossover; the crossover only moves towards smaller
 // j as i decreases (Lemma 4), so a pointer that walks along Q finds it in amortised O(1) moves.
 // U(i,j) is evaluated exactly from prefix sums and a range maximum: the record-maxima stack of the
-// suffix d_i, d_{i+1}, ... (maintained as i decreases) searched by bisection, O(log n) per value.
+// suffix grad_i, grad_{i+1}, ... (maintained as i decreases) searched by bisection, O(log n) per value.
+// On the generalised sizes Lemma 1 (U increasing in j) needs live_t >= kept_t for every interior t:
+// U(i,j+1) - U(i,j) >= live_j - kept_j + kept_{j+1} > 0; the caller checks that.
 // ------------------------------------------------------------------------------------------------
-int plan_dynamic_n(int64_t n, const int64_t* d, uint8_t* is_ckpt, int64_t* peak, int64_t* work) {
-    std::vector<int64_t> prefix(n + 1), M(n + 1), nxt(n + 1, -1), q(n + 1), rec(n + 1);
-    prefix[0] = 0;
-    for (int64_t i = 1; i <= n; ++i) prefix[i] = prefix[i - 1] + d[i];
-    int64_t steps = 0;
-
-    // rec[0..nrec): indices k with d_k larger than every d between the current i and k; stored with
-    // the largest index first, so indices decrease and values decrease along the array.
-    int64_t nrec = 0;
-    int64_t cur_i = 0;
-    auto range_max = [&](int64_t last) -> int64_t {   // max d[cur_i..last], last >= cur_i
-        // first position (from the front) whose index <= last
-        int64_t lo = 0, hi = nrec - 1;
+struct RecordStack {                 // indices t with grad_t larger than every grad between the start of the suffix and t;
+    std::vector<int64_t> idx;        // stored with the largest index first, so indices and values decrease along the array
+    int64_t count = 0;
+    void push(const int64_t* g, int64_t i) {
+        while (count > 0 && g[idx[count - 1]] <= g[i]) --count;
+        idx[count++] = i;
+    }
+    int64_t max_up_to(const int64_t* g, int64_t last) const {   // max of g over [start of the suffix, last]
+        int64_t lo = 0, hi = count - 1;
         while (lo < hi) {
             int64_t mid = (lo + hi) / 2;
-            if (rec[mid] <= last) hi = mid; else lo = mid + 1;
+            if (idx[mid] <= last) hi = mid; else lo = mid + 1;
         }
-        return d[rec[lo]];
-    };
+        return g[idx[lo]];
+    }
+};
+
+static int plan_dynamic_n_sizes(int64_t n, const Sizes3& z, uint8_t* is_ckpt, int64_t* peak, int64_t* work) {
+    std::vector<int64_t> prefix(n + 1), M(n + 1), nxt(n + 1, -1), q(n + 1);
+    prefix[0] = 0;
+    for (int64_t i = 1; i <= n; ++i) prefix[i] = prefix[i - 1] + z.live[i];
+    int64_t steps = 0;
+    RecordStack out_rec, in_rec;     // suffixes that start at i (output gradients) and at i + 1 (incoming gradients)
+    out_rec.idx.resize(n + 1);
+    in_rec.idx.resize(n + 1);
+    int64_t cur_i = 0;
     auto U = [&](int64_t j) -> int64_t {               // U(cur_i, j), j > cur_i
-        return prefix[j - 1] - prefix[cur_i] + range_max(j - 1) + d[j];
+        int64_t u = prefix[j - 1] - prefix[cur_i] + out_rec.max_up_to(z.grad, j - 1) + z.kept[j];
+        if (z.incoming) u += in_rec.max_up_to(z.grad, j);
+        return u;
     };
 
-    M[n] = d[n];
+    M[n] = z.kept[n];
     int64_t top = 0;      // q[0..top]: q[0] = n (largest index), q[top] = head (smallest index)
     q[0] = n;
     int64_t p = 0;        // position in q of the current minimiser
     for (int64_t i = n - 1; i >= 0; --i) {
         cur_i = i;
-        while (nrec > 0 && d[rec[nrec - 1]] <= d[i]) --nrec;
-        rec[nrec++] = i;
+        out_rec.push(z.grad, i);
+        in_rec.push(z.grad, i + 1);
 
         auto f = [&](int64_t t) -> int64_t { ++steps; return std::max(M[q[t]], U(q[t])); };
         if (p > top) p = top;
@@ -254,7 +283,7 @@ int plan_dynamic_n(int64_t n, const int64_t* d, uint8_t* is_ckpt, int64_t* peak,
             int64_t fn = f(p - 1);
             if (fn < fp) { --p; fp = fn; } else break;
         }
-        M[i] = d[i] + fp;
+        M[i] = z.kept[i] + fp;
         nxt[i] = q[p];
         while (top >= 0 && M[q[top]] >= M[i]) { --top; ++steps; }
         q[++top] = i;
@@ -263,6 +292,40 @@ int plan_dynamic_n(int64_t n, const int64_t* d, uint8_t* is_ckpt, int64_t* peak,
     walk_next(n, nxt, is_ckpt);
     *peak = M[0];
     if (work) *work += steps;
+    return CKPT_OK;
+}
+
+int plan_dynamic_n(int64_t n, const int64_t* d, uint8_t* is_ckpt, int64_t* peak, int64_t* work) {
+    const Sizes3 z{d, d, d, 0};
+    return plan_dynamic_n_sizes(n, z, is_ckpt, peak, work);
+}
+
+// Generalised Eq. (memory) of a given set.
+static int64_t eval_sizes(int64_t n, const Sizes3& z, const uint8_t* is_ckpt) {
+    int64_t worst = 0, kept_sum = z.kept[0], h = 0;
+    for (int64_t i = 1; i <= n; ++i) {
+        if (!is_ckpt[i]) continue;
+        kept_sum += z.kept[i];
+        int64_t seg = 0, out_max = 0, in_max = 0;
+        for (int64_t t = h + 1; t < i; ++t) seg += z.live[t];
+        for (int64_t t = h; t < i; ++t) out_max = std::max(out_max, z.grad[t]);
+        for (int64_t t = h + 1; t <= i; ++t) in_max = std::max(in_max, z.grad[t]);
+        worst = std::max(worst, kept_sum + seg + out_max + (z.incoming ? in_max : 0));
+        h = i;
+    }
+    return worst;
+}
+
+static int validate_three(int64_t n, const int64_t* kept, const int64_t* live, const int64_t* grad) {
+    int rc = validate_sizes(n, kept);
+    if (!rc) rc = validate_sizes(n, live);
+    if (!rc) rc = validate_sizes(n, grad);
+    if (rc) return rc;
+    // the worst case adds kept, live and two gradient buffers
+    const int64_t limit = std::numeric_limits<int64_t>::max() / 4;
+    int64_t a = 0, b = 0, c = 0;
+    for (int64_t i = 0; i <= n; ++i) { a += kept[i]; b += live[i]; c = std::max(c, grad[i]); }
+    if (a > limit || b > limit || c > limit) { set_error("sizes overflow int64"); return CKPT_E_OVERFLOW; }
     return CKPT_OK;
 }
 
@@ -336,6 +399,42 @@ int ckpt_launch_log_read(char* text, int64_t capacity, int64_t* needed) {
         memcpy(text, out.data(), m);
         text[m] = 0;
     }
+    return CKPT_OK;
+}
+
+}  // extern "C"
+
+extern "C" {
+
+int ckpt_plan_sizes(int algo, int64_t n, const int64_t* kept, const int64_t* live, const int64_t* grad, int incoming,
+                    uint8_t* is_ckpt, int64_t* peak_bytes) {
+    int rc = ckpt::validate_three(n, kept, live, grad);
+    if (rc) return rc;
+    if (!is_ckpt || !peak_bytes) { ckpt::set_error("output pointer is null"); return CKPT_E_NULL; }
+    const ckpt::Sizes3 z{kept, live, grad, incoming ? 1 : 0};
+    if (algo == CKPT_ALGO_DYNAMIC_N2) return ckpt::plan_dynamic_n2_sizes(n, z, is_ckpt, peak_bytes, nullptr);
+    if (algo == CKPT_ALGO_DYNAMIC_N) {
+        for (int64_t t = 1; t < n; ++t)
+            if (live[t] < kept[t]) {
+                ckpt::set_error("live[%lld] < kept[%lld]: the queue-based search needs live >= kept (use CKPT_ALGO_DYNAMIC_N2)",
+                                (long long)t, (long long)t);
+                return CKPT_E_BAD_ARG;
+            }
+        return ckpt::plan_dynamic_n_sizes(n, z, is_ckpt, peak_bytes, nullptr);
+    }
+    ckpt::set_error("algorithm %d does not take separate sizes", algo);
+    return CKPT_E_BAD_ARG;
+}
+
+int ckpt_eval_sizes(int64_t n, const int64_t* kept, const int64_t* live, const int64_t* grad, int incoming,
+                    const uint8_t* is_ckpt, int64_t* peak_bytes) {
+    int rc = ckpt::validate_three(n, kept, live, grad);
+    if (rc) return rc;
+    if (!peak_bytes) { ckpt::set_error("peak_bytes is null"); return CKPT_E_NULL; }
+    rc = ckpt::validate_plan(n, is_ckpt);
+    if (rc) return rc;
+    const ckpt::Sizes3 z{kept, live, grad, incoming ? 1 : 0};
+    *peak_bytes = ckpt::eval_sizes(n, z, is_ckpt);
     return CKPT_OK;
 }
 
