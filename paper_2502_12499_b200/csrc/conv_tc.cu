@@ -31,6 +31,7 @@ namespace ckpt {
 namespace {
 
 constexpr int kThreads = 192;
+constexpr int kThreadsT = 320;                        // role-swapped kernel: TMA warp, MMA warp, eight epilogue warps
 constexpr int kMaxStages = 8;
 constexpr uint32_t kSmemBudget = 200 * 1024;          // operand stages; barriers live behind them
 constexpr long long kWaitCycles = 4000000000LL;       // ~2 s at 2 GHz: far beyond any legitimate wait
@@ -430,6 +431,34 @@ tc_conv_fwd_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_const
 // lanes of a warp store 64 contiguous bytes of one pixel per instruction, and the batch-norm sums of a channel
 // are plain per-thread sums.
 // ------------------------------------------------------------------------------------------------
+// Epilogue of the role-swapped kernels for one chunk of 32 pixels x 32 output channels: the lane owns a channel and
+// holds that channel's accumulators of the 32 pixels.  Rounds them to bf16, writes them pixel-major into the slab
+// (64-byte rows: a lane's two bytes next to its neighbours') and adds the rounded values of the pixels inside the
+// tensor to the lane's batch-norm sums, kept in four interleaved partial sums so that consecutive additions do not
+// wait on one another.
+__device__ __forceinline__ void t_chunk_to_slab(const uint32_t (&v)[32], uint32_t in_mask, uint32_t slab_lane, float (&sum)[4],
+                                                float (&sumsq)[4]) {
+    if (in_mask == 0xffffffffu) {
+#pragma unroll
+        for (int e = 0; e < 32; ++e) {
+            const __nv_bfloat16 r = __float2bfloat16_rn(__uint_as_float(v[e]));
+            asm volatile("st.shared.b16 [%0], %1;" ::"r"(slab_lane + (uint32_t)(e * 64)), "h"(__bfloat16_as_ushort(r)) : "memory");
+            const float f = __bfloat162float(r);
+            sum[e & 3] += f;
+            sumsq[e & 3] = fmaf(f, f, sumsq[e & 3]);
+        }
+    } else {
+#pragma unroll
+        for (int e = 0; e < 32; ++e) {
+            const __nv_bfloat16 r = __float2bfloat16_rn(__uint_as_float(v[e]));
+            asm volatile("st.shared.b16 [%0], %1;" ::"r"(slab_lane + (uint32_t)(e * 64)), "h"(__bfloat16_as_ushort(r)) : "memory");
+            const float f = ((in_mask >> e) & 1u) ? __bfloat162float(r) : 0.f;
+            sum[e & 3] += f;
+            sumsq[e & 3] = fmaf(f, f, sumsq[e & 3]);
+        }
+    }
+}
+
 struct TParams {
     int H, W, N;                 // pixel grid walked by the tiles (= the output tensor: stride 1)
     int c_red, c_out;
@@ -481,14 +510,14 @@ __device__ __forceinline__ void load_filter_boxes(const TParams& p, const CUtens
 // two boxes of 64 reduction rows x 64 output channels per stage (at the column block of the mirrored filter
 // position), an MN-major operand for the tensor core.  No transposed copy of the filter is made.
 template <bool A_MN>
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__(kThreadsT, 1)
 tc_conv_t_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w,
                  const __grid_constant__ CUtensorMap map_out, float* __restrict__ stat_partial, TParams p, int* status) {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     constexpr uint32_t a_bytes = 128 * 128, b_bytes = 256 * 128, stage_bytes = a_bytes + b_bytes;
     const uint32_t bars = base + (uint32_t)p.stages * stage_bytes;           // full[s], empty[s], acc_full[2], acc_empty[2]
-    const uint32_t out_stage = bars + 256;                                   // [4 warps][2][32 pixels x 32 channels] bf16
+    const uint32_t out_stage = bars + 256;                                   // [8 warps][2][32 pixels x 32 channels] bf16
     __shared__ uint32_t tmem_base_slot;
     __shared__ int failed_flag;
     volatile int* failed = &failed_flag;
@@ -513,7 +542,7 @@ tc_conv_t_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
     if (threadIdx.x == 0) {
         failed_flag = 0;
         for (int s = 0; s < p.stages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
-        for (int b = 0; b < 2; ++b) { mbar_init(acc_full0 + 8 * b, 1); mbar_init(acc_empty0 + 8 * b, 128); }
+        for (int b = 0; b < 2; ++b) { mbar_init(acc_full0 + 8 * b, 1); mbar_init(acc_empty0 + 8 * b, 256); }
         fence_barrier_init();
         tma_prefetch_desc(&map_x);
         tma_prefetch_desc(&map_w);
@@ -575,10 +604,14 @@ tc_conv_t_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
         // neighbours': 64-byte rows) and leaves as one tile store whose box is the chunk's bw x bh x bn pixels;
         // the hardware clips what lies outside the tensor.  (Two-byte global stores from the lanes, 64 bytes per
         // instruction, made this epilogue the bottleneck of the kernel: 0.32 ms against 0.18 ms without them.)
-        const int quarter = warp % 4;
+        // Eight epilogue warps: two per quarter of the accumulator's lanes (a warp reaches the 32 lanes of quarter
+        // warp % 4 only), the two taking alternate chunks.  With one warp per scheduler the chain round - store - add of
+        // a chunk ran at the latency of its instructions (issue slots 30 % used, 9 B/clk of output per SM on a
+        // 64 -> 256 1x1 layer); two warps per scheduler overlap them.
+        const int quarter = warp % 4, half = (warp - 2) / 4;
         const int co = co_tile * 128 + quarter * 32 + lane;
         const bool stats = stat_partial != nullptr;
-        float sum = 0.f, sumsq = 0.f;
+        float sum[4] = {0.f, 0.f, 0.f, 0.f}, sumsq[4] = {0.f, 0.f, 0.f, 0.f};
         int chunk_count = 0;
         for (int j = 0; j < my_tiles; ++j) {
             const int buf = j & 1;
@@ -587,7 +620,7 @@ tc_conv_t_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
             int w0, h0, n0;
             tile_origin(j, w0, h0, n0);
 #pragma unroll 1
-            for (int c0 = 0; c0 < 256; c0 += 32, ++chunk_count) {
+            for (int c0 = half * 32; c0 < 256; c0 += 64, ++chunk_count) {
                 // lane e works out whether pixel c0 + e of the tile lies inside the tensor (for the sums)
                 const int idx = c0 + lane;
                 const int wl = idx & (p.tw - 1), hl = (idx >> p.tw_log) & (p.th - 1), nl = idx >> (p.tw_log + p.th_log);
@@ -595,19 +628,10 @@ tc_conv_t_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                 const uint32_t in_mask = __ballot_sync(0xffffffffu, inside);
                 uint32_t v[32];
                 tmem_ld32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * 256 + c0), v);
-                const uint32_t slab = out_stage + (uint32_t)((quarter * 2 + (chunk_count & 1)) * 2048);
+                const uint32_t slab = out_stage + (uint32_t)(((warp - 2) * 2 + (chunk_count & 1)) * 2048);
                 if (lane == 0) tma_store_wait_read<1>();          // the store that last read this slab has left it
                 __syncwarp();
-#pragma unroll
-                for (int e = 0; e < 32; ++e) {
-                    const __nv_bfloat16 r = __float2bfloat16_rn(__uint_as_float(v[e]));
-                    asm volatile("st.shared.b16 [%0], %1;" ::"r"(slab + (uint32_t)(e * 64 + lane * 2)), "h"(__bfloat16_as_ushort(r)) : "memory");
-                    if ((in_mask >> e) & 1u) {
-                        const float f = __bfloat162float(r);
-                        sum += f;
-                        sumsq = fmaf(f, f, sumsq);
-                    }
-                }
+                t_chunk_to_slab(v, in_mask, slab + (uint32_t)(lane * 2), sum, sumsq);
                 fence_proxy_async();
                 __syncwarp();
                 if (lane == 0 && in_mask != 0u && co_tile * 128 + quarter * 32 < p.c_out) {
@@ -621,14 +645,16 @@ tc_conv_t_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
         }
         if (lane == 0) tma_store_wait_all();
         if (stats && co < p.c_out) {
-            // one partial row pair per CTA: [block][sum | sum of squares][channel]
+            // two partial row pairs per CTA (one per warp of the channel's quarter): [block][sum | sum of squares][channel]
+            const float s1 = (sum[0] + sum[1]) + (sum[2] + sum[3]), s2 = (sumsq[0] + sumsq[1]) + (sumsq[2] + sumsq[3]);
+            const size_t row = (size_t)first * 2 + half;
             if (p.fold) {
-                const size_t blk = (size_t)first * 2 + co / p.fold;
-                stat_partial[(blk * 2) * p.fold + co % p.fold] = sum;
-                stat_partial[(blk * 2 + 1) * p.fold + co % p.fold] = sumsq;
+                const size_t blk = row * 2 + co / p.fold;
+                stat_partial[(blk * 2) * p.fold + co % p.fold] = s1;
+                stat_partial[(blk * 2 + 1) * p.fold + co % p.fold] = s2;
             } else {
-                stat_partial[((size_t)first * 2) * p.c_out + co] = sum;
-                stat_partial[((size_t)first * 2 + 1) * p.c_out + co] = sumsq;
+                stat_partial[(row * 2) * p.c_out + co] = s1;
+                stat_partial[(row * 2 + 1) * p.c_out + co] = s2;
             }
         }
     }
@@ -773,7 +799,7 @@ tc_conv_tp_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
         const int quarter = warp % 4;
         const int co = co_tile * 128 + quarter * 32 + lane;
         const bool stats = stat_partial != nullptr;
-        float sum = 0.f, sumsq = 0.f;
+        float sum[4] = {0.f, 0.f, 0.f, 0.f}, sumsq[4] = {0.f, 0.f, 0.f, 0.f};
         int chunk_count = 0;
         for (int j = 0; j < my_tiles; ++j) {
             const int buf = j & 1;
@@ -791,16 +817,7 @@ tc_conv_tp_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
                 const uint32_t slab = out_stage + (uint32_t)((quarter * 2 + (chunk_count & 1)) * 2048);
                 if (lane == 0) tma_store_wait_read<1>();          // the store that last read this slab has left it
                 __syncwarp();
-#pragma unroll
-                for (int e = 0; e < 32; ++e) {
-                    const __nv_bfloat16 r = __float2bfloat16_rn(__uint_as_float(v[e]));
-                    asm volatile("st.shared.b16 [%0], %1;" ::"r"(slab + (uint32_t)(e * 64 + lane * 2)), "h"(__bfloat16_as_ushort(r)) : "memory");
-                    if ((in_mask >> e) & 1u) {
-                        const float f = __bfloat162float(r);
-                        sum += f;
-                        sumsq = fmaf(f, f, sumsq);
-                    }
-                }
+                t_chunk_to_slab(v, in_mask, slab + (uint32_t)(lane * 2), sum, sumsq);
                 fence_proxy_async();
                 __syncwarp();
                 if (lane == 0 && in_mask != 0u && co_tile * 128 + quarter * 32 < p.c_out) {
@@ -813,13 +830,14 @@ tc_conv_tp_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
         }
         if (lane == 0) tma_store_wait_all();
         if (stats && co < p.c_out) {
+            const float s1 = (sum[0] + sum[1]) + (sum[2] + sum[3]), s2 = (sumsq[0] + sumsq[1]) + (sumsq[2] + sumsq[3]);
             if (p.fold) {
                 const size_t blk = (size_t)first * 2 + co / p.fold;
-                stat_partial[(blk * 2) * p.fold + co % p.fold] = sum;
-                stat_partial[(blk * 2 + 1) * p.fold + co % p.fold] = sumsq;
+                stat_partial[(blk * 2) * p.fold + co % p.fold] = s1;
+                stat_partial[(blk * 2 + 1) * p.fold + co % p.fold] = s2;
             } else {
-                stat_partial[((size_t)first * 2) * p.c_out + co] = sum;
-                stat_partial[((size_t)first * 2 + 1) * p.c_out + co] = sumsq;
+                stat_partial[((size_t)first * 2) * p.c_out + co] = s1;
+                stat_partial[((size_t)first * 2 + 1) * p.c_out + co] = s2;
             }
         }
     }
@@ -2199,7 +2217,7 @@ int64_t generic_stat_rows(int n, int gh, int gw) {
     int tw, th, tn;
     choose_tile(128, gw, gh, n, &tw, &th, &tn);
     const int64_t m_tiles = (int64_t)((gw + tw - 1) / tw) * ((gh + th - 1) / th) * ((n + tn - 1) / tn);
-    return 4 * std::min<int64_t>(m_tiles, 256);      // one row pair per epilogue warp of each persistent CTA (at most one CTA per SM)
+    return 8 * std::min<int64_t>(m_tiles, 256);      // up to four row pairs per persistent CTA (at most one CTA per SM), with room to spare
 }
 
 int launch_generic(FwdParams p, const void* a, int a_n, int a_h, int a_w, const void* w_mat, int taps_total, void* out,
@@ -2293,7 +2311,8 @@ int launch_t_core(TParams p, const void* x, int x_channels, const CUtensorMap& m
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     p.ctas_per_co = std::max(1, std::min(p.p_tiles, sms / p.co_tiles));
     constexpr uint32_t stage_bytes = 128 * 128 + 256 * 128;
-    p.stages = std::min<int>(kMaxStages, kSmemBudget / stage_bytes);
+    constexpr uint32_t t_slabs = 8 * 2 * 2048;          // two chunk slabs for each of the eight epilogue warps
+    p.stages = std::min<int>(kMaxStages, (227 * 1024 - 1024 - 256 - t_slabs - 64) / stage_bytes);
     CUtensorMap mx;
     int rc = make_act_map(&mx, x, N, H, W, x_channels, p.tw, patch ? p.th + 2 : p.th, p.tn);
     if (rc) return rc;
@@ -2311,15 +2330,17 @@ int launch_t_core(TParams p, const void* x, int x_channels, const CUtensorMap& m
                         CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
         if (r != CUDA_SUCCESS) { set_error("cuTensorMapEncodeTiled failed for an output tensor (code %d)", (int)r); return CKPT_E_CUDA; }
     }
-    const size_t smem = (size_t)p.stages * stage_bytes + 1024 + 256 + 4 * 2 * 2048;
+    const size_t smem = (size_t)p.stages * stage_bytes + 1024 + 256 + t_slabs;
     static bool attr_set = false;
     if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(tc_conv_t_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024);
-        if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_conv_t_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024);
+        cudaError_t e = cudaFuncSetAttribute(tc_conv_t_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024 - 64);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_conv_t_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024 - 64);
         if (e != cudaSuccess) return cuda_fail(e, "raising the shared-memory limit");
         attr_set = true;
     }
-    if (stat_blocks) *stat_blocks = stat_partial ? (p.fold ? 2 : 1) * p.ctas_per_co : 0;
+    // partial row pairs per CTA: one per epilogue warp of a channel's quarter (the plain kernel has two), twice that
+    // in the pixel-pair form
+    if (stat_blocks) *stat_blocks = stat_partial ? (p.fold ? 2 : 1) * (patch ? 1 : 2) * p.ctas_per_co : 0;
     if (patch) {
         static bool tp_attr_set = false;
         if (!tp_attr_set) {
@@ -2333,8 +2354,8 @@ int launch_t_core(TParams p, const void* x, int x_channels, const CUtensorMap& m
         CKPT_LAUNCH_CHECK_NAMED("tc_conv_tp_kernel", what);
         return CKPT_OK;
     }
-    if (a_mn) tc_conv_t_kernel<true><<<p.ctas_per_co * p.co_tiles, kThreads, smem, st>>>(mx, mw, mo, stat_blocks ? stat_partial : nullptr, p, status);
-    else tc_conv_t_kernel<false><<<p.ctas_per_co * p.co_tiles, kThreads, smem, st>>>(mx, mw, mo, stat_blocks ? stat_partial : nullptr, p, status);
+    if (a_mn) tc_conv_t_kernel<true><<<p.ctas_per_co * p.co_tiles, kThreadsT, smem, st>>>(mx, mw, mo, stat_blocks ? stat_partial : nullptr, p, status);
+    else tc_conv_t_kernel<false><<<p.ctas_per_co * p.co_tiles, kThreadsT, smem, st>>>(mx, mw, mo, stat_blocks ? stat_partial : nullptr, p, status);
     CKPT_LAUNCH_CHECK_NAMED("tc_conv_t_kernel", what);
     return CKPT_OK;
 }
