@@ -242,6 +242,16 @@ CKPT_API int ckpt_chain_set_graph(ckpt_chain* chain, int enable);
  * against a reference on the unit's own inputs.  Costs one device copy per unit. */
 CKPT_API int ckpt_chain_set_gradient_tap(ckpt_chain* chain, void* tap, int64_t tap_bytes);
 
+/* "Update w_i with g_i" - the last line of the backward loop of Algorithms 1, 2 and 4 - as plain gradient descent
+ * (the paper names no rule): with learning_rate > 0 every following ckpt_train_step also overwrites each parameter
+ * tensor with w - learning_rate * g, in the parameter's storage type (bf16 filters: float32 arithmetic, rounded to
+ * nearest even), as soon as its gradient g is complete and nothing in the step reads the parameter any more; the
+ * gradients are still written to `grads`.  For convolution filters on the tensor-core path the update happens in
+ * the pass that sums the slices of the split weight gradient (no extra pass over the filter), and the input gradient
+ * of the unit, which reads the filter, is computed before it.  params then point to memory the step writes.
+ * learning_rate = 0 (default) leaves the parameters untouched.  NaN or negative values: CKPT_E_BAD_ARG. */
+CKPT_API int ckpt_chain_set_sgd(ckpt_chain* chain, double learning_rate);
+
 /* Failure-path self-test (off by default).  With wait_runs_out = 1 every following step launches, after its loss,
  * one extra single-warp kernel whose only wait has no producer and a limit of 2e5 clock cycles: the wait gives up,
  * writes its code into the step's status word and the kernel returns, as every bounded wait of the tensor-core

@@ -297,6 +297,20 @@ def chain_forward_backward(chain, params, x, labels=None, storage="exact"):
     return dict(loss=loss, grads=grads, d=d, input_grad=r)
 
 
+def sgd_update(params, grads, lr, storage="exact"):
+    """Last line of the backward loop of Algorithm 1, "update w_i with g_i", read as plain gradient descent:
+    w_i <- w_i - lr * g_i for every parameter of every unit.  With storage="bf16" the matrices (names starting with
+    "w"), which a low-precision executor keeps in bfloat16, are rounded after the update."""
+    out = []
+    for p, g in zip(params, grads):
+        q = {}
+        for name, w in p.items():
+            new = np.asarray(w, dtype=np.float64) - lr * np.asarray(g[name], dtype=np.float64)
+            q[name] = _store(new, storage) if name.startswith("w") else new
+        out.append(q)
+    return out
+
+
 def output_shapes(chain):
     """(H, W, C) of d_0..d_n by running shapes through the layer definitions."""
     h, w, c = chain["input_hwc"]

@@ -243,6 +243,10 @@ class Chain:
         nbytes = 0 if tap is None else tap.numel() * tap.element_size()
         _check(lib().ckpt_chain_set_gradient_tap(self._h, _dev(tap), C.c_int64(nbytes)))
 
+    def set_sgd(self, learning_rate):
+        """ckpt_chain_set_sgd: steps also apply w <- w - learning_rate * g to every parameter (0 switches it off)."""
+        _check(lib().ckpt_chain_set_sgd(self._h, C.c_double(learning_rate)))
+
     def set_selftest(self, wait_runs_out):
         _check(lib().ckpt_chain_set_selftest(self._h, C.c_int(1 if wait_runs_out else 0)))
 

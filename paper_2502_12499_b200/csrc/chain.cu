@@ -57,6 +57,7 @@ struct ckpt_chain {
     char* tap = nullptr;                 // device: where the step leaves every inter-unit gradient (ckpt_chain_set_gradient_tap)
     int64_t tap_bytes = 0;
     int selftest_wait = 0;               // the next steps include one kernel whose bounded wait runs out
+    float sgd_lr = 0.f;                  // != 0: every parameter takes w - lr * g as soon as its gradient is complete
     void* host_result = nullptr;         // pinned: loss (8 bytes) and status word of the last step
     cudaStream_t capture_stream = nullptr;   // recording happens here (the caller's stream may be the default one,
                                              // which cannot record); replays run on the caller's stream
@@ -125,6 +126,35 @@ static int conv_wgrad_any(StepCtx& c, const ConvGeom& g, const void* dz, const v
     if (use_tc(c.ch, g))
         return tc_conv_wgrad(g, dz, x, dw, c.ws + c.ch->off_scr, c.ch->scr_bytes, c.status(), c.stream);
     return simt_conv_wgrad(c.ch->dtype, g, dz, x, dw, c.ws + c.ch->off_scr, c.ch->scr_bytes, c.stream);
+}
+
+// "Update w_i with g_i" (Algorithms 1, 2, 4), when a learning rate is set.  param = index of the parameter tensor.
+static SgdUpdate sgd_of(StepCtx& c, int param) {
+    SgdUpdate u;
+    if (c.ch->sgd_lr != 0.f) { u.w = c.params[param]; u.lr = c.ch->sgd_lr; u.dtype = c.ch->params[param].dtype; }
+    return u;
+}
+static int sgd_step(StepCtx& c, int param) {
+    if (c.ch->sgd_lr == 0.f) return CKPT_OK;
+    return sgd_update(sgd_of(c, param), (const float*)c.grads[param], c.ch->params[param].elems, c.stream);
+}
+// Weight gradient and input gradient of one convolution.  Without an update: wgrad, then dgrad.  With one the filter
+// changes as soon as its gradient is summed, so the input gradient (which reads the filter) runs first.
+static int conv_backward_pair(StepCtx& c, const ConvGeom& g, const void* dz, const void* x, const void* w, int param, void* dx) {
+    int rc;
+    const bool sgd = c.ch->sgd_lr != 0.f;
+    if (sgd && dx && (rc = conv_dgrad_any(c, g, dz, w, dx))) return rc;
+    const bool tc_path = !(c.ch->impl == 0 && small_conv_supported(c.ch->dtype, g)) && !(c.ch->impl == 0 && stem_conv_supported(c.ch->dtype, g)) &&
+                         use_tc(c.ch, g);
+    if (sgd && tc_path) {
+        rc = tc_conv_wgrad(g, dz, x, (float*)c.grads[param], c.ws + c.ch->off_scr, c.ch->scr_bytes, c.status(), c.stream, sgd_of(c, param));
+        if (rc) return rc;
+    } else {
+        if ((rc = conv_wgrad_any(c, g, dz, x, (float*)c.grads[param]))) return rc;
+        if ((rc = sgd_step(c, param))) return rc;
+    }
+    if (!sgd && dx && (rc = conv_dgrad_any(c, g, dz, w, dx))) return rc;
+    return CKPT_OK;
 }
 
 // Convolution followed by the batch statistics of its stored output.  The tensor-core kernels gather the
@@ -227,6 +257,7 @@ static int block_backward(StepCtx& c, const Unit& u, const void* x, const void* 
     const BlockBuffers B = block_buffers(c, u);
     void* const* p = c.params + u.param_first;
     void* const* g = c.grads + u.param_first;
+    const int pf = u.param_first;
     char* scr = c.ws + c.ch->off_scr;
     const int64_t in_px = c.ch->batch * u.in.h * u.in.w, out_px = c.ch->batch * u.out.h * u.out.w;
     const int mid = u.desc.mid, co = u.out.c;
@@ -238,20 +269,20 @@ static int block_backward(StepCtx& c, const Unit& u, const void* x, const void* 
     const void* dx_shortcut = g_in;                       // identity shortcut: the same gradient flows to x
     if (project) {
         if ((rc = bn_relu_backward(dt, out_px, co, g_in, B.zp, (const float*)p[10], B.sp, 0, B.t0, (float*)g[10], (float*)g[11], scr, c.stream))) return rc;
-        if ((rc = conv_wgrad_any(c, u.gp, B.t0, x, (float*)g[9]))) return rc;
-        if (g_out) { if ((rc = conv_dgrad_any(c, u.gp, B.t0, p[9], B.dxs))) return rc; }
+        if ((rc = sgd_step(c, pf + 10)) || (rc = sgd_step(c, pf + 11))) return rc;
+        if ((rc = conv_backward_pair(c, u.gp, B.t0, x, p[9], pf + 9, g_out ? B.dxs : nullptr))) return rc;
         dx_shortcut = B.dxs;
     }
     if ((rc = bn_relu_backward(dt, out_px, co, g_in, B.z3, (const float*)p[7], B.s3, 0, B.t1, (float*)g[7], (float*)g[8], scr, c.stream))) return rc;
-    if ((rc = conv_wgrad_any(c, u.g3, B.t1, B.b, (float*)g[6]))) return rc;
-    if ((rc = conv_dgrad_any(c, u.g3, B.t1, p[6], B.db))) return rc;
+    if ((rc = sgd_step(c, pf + 7)) || (rc = sgd_step(c, pf + 8))) return rc;
+    if ((rc = conv_backward_pair(c, u.g3, B.t1, B.b, p[6], pf + 6, B.db))) return rc;
     if ((rc = bn_relu_backward(dt, out_px, mid, B.db, B.z2, (const float*)p[4], B.s2, 1, B.db, (float*)g[4], (float*)g[5], scr, c.stream))) return rc;
-    if ((rc = conv_wgrad_any(c, u.g2, B.db, B.a, (float*)g[3]))) return rc;
-    if ((rc = conv_dgrad_any(c, u.g2, B.db, p[3], B.da))) return rc;
+    if ((rc = sgd_step(c, pf + 4)) || (rc = sgd_step(c, pf + 5))) return rc;
+    if ((rc = conv_backward_pair(c, u.g2, B.db, B.a, p[3], pf + 3, B.da))) return rc;
     if ((rc = bn_relu_backward(dt, in_px, mid, B.da, B.z1, (const float*)p[1], B.s1, 1, B.da, (float*)g[1], (float*)g[2], scr, c.stream))) return rc;
-    if ((rc = conv_wgrad_any(c, u.g1, B.da, x, (float*)g[0]))) return rc;
+    if ((rc = sgd_step(c, pf + 1)) || (rc = sgd_step(c, pf + 2))) return rc;
+    if ((rc = conv_backward_pair(c, u.g1, B.da, x, p[0], pf, g_out))) return rc;
     if (!g_out) return CKPT_OK;
-    if ((rc = conv_dgrad_any(c, u.g1, B.da, p[0], g_out))) return rc;
     return add_tensors(dt, in_px * u.in.c, g_out, dx_shortcut, g_out, c.stream);
 }
 
@@ -311,11 +342,18 @@ static int through_pending_act(StepCtx& c, int64_t j, const void* d_j, void* g, 
     const Unit& uj = c.ch->units[j - 1];
     void* const* p = c.params + uj.param_first;
     void* const* gr = c.grads + uj.param_first;
+    int rc;
     if (sum_blocks > 0)
-        return bn_relu_backward_from_partials(c.ch->dtype, rows_of(c.ch, j), uj.out.c, g, d_j, stats_of(c, j), 1, g,
-                                              (float*)gr[1], (float*)gr[2], c.ws + c.ch->off_scr, sum_blocks, c.stream);
-    return bn_relu_backward(c.ch->dtype, rows_of(c.ch, j), uj.out.c, g, d_j, (const float*)p[1], stats_of(c, j), 1, g,
-                            (float*)gr[1], (float*)gr[2], c.ws + c.ch->off_scr, c.stream);
+        rc = bn_relu_backward_from_partials(c.ch->dtype, rows_of(c.ch, j), uj.out.c, g, d_j, stats_of(c, j), 1, g,
+                                            (float*)gr[1], (float*)gr[2], c.ws + c.ch->off_scr, sum_blocks, c.stream);
+    else
+        rc = bn_relu_backward(c.ch->dtype, rows_of(c.ch, j), uj.out.c, g, d_j, (const float*)p[1], stats_of(c, j), 1, g,
+                              (float*)gr[1], (float*)gr[2], c.ws + c.ch->off_scr, c.stream);
+    // scale and shift of unit j are not read again in this step: the saved statistics block holds what forward and
+    // backward need of them
+    if (!rc) rc = sgd_step(c, uj.param_first + 1);
+    if (!rc) rc = sgd_step(c, uj.param_first + 2);
+    return rc;
 }
 
 // r_i and g_i (Eqs. (3) and (5)): g_in = dL/dd_i (may be overwritten), g_out = dL/dd_{i-1} or null.
@@ -329,20 +367,16 @@ static int unit_backward(StepCtx& c, int64_t i, const void* x_raw, const void* y
     int rc, sum_blocks = 0;
     switch (u.desc.kind) {
         case CKPT_UNIT_CONV_BN_RELU:
-            if ((rc = activated(c, i - 1, x_raw, &x))) return rc;
-            if ((rc = conv_wgrad_any(c, u.geom, g_in, x, (float*)g[0]))) return rc;
-            if (g_out && (rc = conv_dgrad_any(c, u.geom, g_in, p[0], g_out))) return rc;
-            break;
         case CKPT_UNIT_CONV:
             if ((rc = activated(c, i - 1, x_raw, &x))) return rc;
-            if ((rc = conv_wgrad_any(c, u.geom, g_in, x, (float*)g[0]))) return rc;
-            if (g_out && (rc = conv_dgrad_any(c, u.geom, g_in, p[0], g_out))) return rc;
+            if ((rc = conv_backward_pair(c, u.geom, g_in, x, p[0], u.param_first, g_out))) return rc;
             break;
         case CKPT_UNIT_BN:
             // the statistics saved by this unit's (re)computed forward are those of its input
             if ((rc = activated(c, i - 1, x_raw, &x))) return rc;
             if ((rc = bn_relu_backward(dt, rows_of(c.ch, i), u.out.c, g_in, x, (const float*)p[0], stats_of(c, i), 0,
                                        g_out ? g_out : g_in, (float*)g[0], (float*)g[1], c.ws + c.ch->off_scr, c.stream))) return rc;
+            if ((rc = sgd_step(c, u.param_first)) || (rc = sgd_step(c, u.param_first + 1))) return rc;
             break;
         case CKPT_UNIT_RELU:
             if (g_out && (rc = relu_backward(dt, rows_of(c.ch, i) * u.out.c, g_in, y, g_out, c.stream))) return rc;
@@ -369,8 +403,8 @@ static int unit_backward(StepCtx& c, int64_t i, const void* x_raw, const void* y
             if (u.desc.flags & 1)
                 if ((rc = relu_mask_inplace(dt, elems, g_in, y, c.stream))) return rc;
             if ((rc = column_sums(dt, c.ch->batch, u.out.c, g_in, (float*)g[1], c.stream))) return rc;
-            if ((rc = conv_wgrad_any(c, u.geom, g_in, x, (float*)g[0]))) return rc;
-            if (g_out && (rc = conv_dgrad_any(c, u.geom, g_in, p[0], g_out))) return rc;
+            if ((rc = sgd_step(c, u.param_first + 1))) return rc;
+            if ((rc = conv_backward_pair(c, u.geom, g_in, x, p[0], u.param_first, g_out))) return rc;
             break;
         }
         case CKPT_UNIT_BOTTLENECK:
@@ -573,6 +607,7 @@ static uint64_t step_key(const ckpt_chain* ch, const uint8_t* is_ckpt, int polic
     args->push_back((uint64_t)(uintptr_t)arena); args->push_back((uint64_t)(uintptr_t)ws);
     args->push_back((uint64_t)ch->impl);
     args->push_back((uint64_t)(uintptr_t)ch->tap); args->push_back((uint64_t)ch->selftest_wait);
+    { uint32_t bits; memcpy(&bits, &ch->sgd_lr, sizeof(bits)); args->push_back((uint64_t)bits); }
     for (size_t p = 0; p < ch->params.size(); ++p) { args->push_back((uint64_t)(uintptr_t)params[p]); args->push_back((uint64_t)(uintptr_t)grads[p]); }
     if (policy != CKPT_POLICY_STORE_ALL)
         for (size_t i = 0; i <= ch->units.size(); ++i) args->push_back((uint64_t)is_ckpt[i]);
@@ -990,6 +1025,13 @@ int ckpt_chain_set_gradient_tap(ckpt_chain* chain, void* tap, int64_t tap_bytes)
     if (tap && tap_bytes < need) { set_error("gradient tap of %lld bytes, %lld needed", (long long)tap_bytes, (long long)need); return CKPT_E_WORKSPACE; }
     chain->tap = (char*)tap;
     chain->tap_bytes = tap ? tap_bytes : 0;
+    return CKPT_OK;
+}
+
+int ckpt_chain_set_sgd(ckpt_chain* chain, double learning_rate) {
+    if (!chain) { set_error("null pointer"); return CKPT_E_NULL; }
+    if (!(learning_rate == learning_rate) || learning_rate < 0) { set_error("learning rate must be >= 0"); return CKPT_E_BAD_ARG; }
+    chain->sgd_lr = (float)learning_rate;
     return CKPT_OK;
 }
 

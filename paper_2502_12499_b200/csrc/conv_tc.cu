@@ -2000,8 +2000,24 @@ __device__ __forceinline__ void add4(float4& a, const float4 b) { a.x += b.x; a.
 // The split kernels leave one partial result per persistent CTA (some tens of MB, mostly still in L2) for a few
 // hundred thousand outputs: a thread per output would leave most SMs idle and one load in flight per thread.  A block
 // is 32 float4 columns x Y slice groups; group y sums slices y, y + Y, ... and the groups are added in a fixed order.
+// Parameter update fused into a gradient store: elements 4*e4 .. 4*e4+3 of the parameter take w - lr * g.
+__device__ __forceinline__ void sgd_apply4(const SgdUpdate& u, int64_t e4, float4 g) {
+    if (!u.w) return;
+    if (u.dtype == CKPT_DTYPE_BF16) {
+        __nv_bfloat162* p = reinterpret_cast<__nv_bfloat162*>(u.w) + 2 * e4;
+        const float2 a = __bfloat1622float2(p[0]), b = __bfloat1622float2(p[1]);
+        p[0] = __floats2bfloat162_rn(fmaf(-u.lr, g.x, a.x), fmaf(-u.lr, g.y, a.y));
+        p[1] = __floats2bfloat162_rn(fmaf(-u.lr, g.z, b.x), fmaf(-u.lr, g.w, b.y));
+    } else {
+        float4* p = reinterpret_cast<float4*>(u.w) + e4;
+        float4 w = *p;
+        w.x = fmaf(-u.lr, g.x, w.x); w.y = fmaf(-u.lr, g.y, w.y); w.z = fmaf(-u.lr, g.z, w.z); w.w = fmaf(-u.lr, g.w, w.w);
+        *p = w;
+    }
+}
+
 template <int X, int Y>
-__device__ __forceinline__ void store_group_sum(float4 acc, float4* out, bool ok) {
+__device__ __forceinline__ void store_group_sum(float4 acc, float4* out, bool ok, const SgdUpdate& upd, int64_t e4) {
     __shared__ float4 red[Y][X];
     if (Y > 1) {
         red[threadIdx.y][threadIdx.x] = acc;
@@ -2009,13 +2025,16 @@ __device__ __forceinline__ void store_group_sum(float4 acc, float4* out, bool ok
         if (threadIdx.y == 0)
             for (int y = 1; y < Y; ++y) add4(acc, red[y][threadIdx.x]);
     }
-    if (threadIdx.y == 0 && ok) *out = acc;
+    if (threadIdx.y == 0 && ok) {
+        *out = acc;
+        sgd_apply4(upd, e4, acc);
+    }
 }
 
 // Pair-view wgrad partials [slice][(q, c_out)][column 4][dy 3][c_in 64] -> dW[c_out][dy][dx][c_in]: pixel q of a pair
 // sees filter column dx in accumulator column dx + q.
 template <int Y>
-__global__ void __launch_bounds__(32 * Y) pairview_fold_kernel(const float* __restrict__ partial, float* __restrict__ out, int c_out, int slices) {
+__global__ void __launch_bounds__(32 * Y) pairview_fold_kernel(const float* __restrict__ partial, float* __restrict__ out, int c_out, int slices, SgdUpdate upd) {
     const int idx = blockIdx.x * 32 + threadIdx.x;            // one float4 of the output
     const bool ok = idx < c_out * 144;
     const int ci = (idx % 16) * 4, dx = (idx / 16) % 3, dy = (idx / 48) % 3, co = ok ? idx / 144 : 0;
@@ -2030,11 +2049,11 @@ __global__ void __launch_bounds__(32 * Y) pairview_fold_kernel(const float* __re
             add4(acc, *reinterpret_cast<const float4*>(p1 + z * slice_stride));
         }
     }
-    store_group_sum<32, Y>(acc, reinterpret_cast<float4*>(out) + idx, ok);
+    store_group_sum<32, Y>(acc, reinterpret_cast<float4*>(out) + idx, ok, upd, idx);
 }
 
 template <int X, int Y>
-__global__ void __launch_bounds__(X * Y) slice_sum4_kernel(const float4* __restrict__ partial, float4* __restrict__ out, int64_t elems4, int slices) {
+__global__ void __launch_bounds__(X * Y) slice_sum4_kernel(const float4* __restrict__ partial, float4* __restrict__ out, int64_t elems4, int slices, SgdUpdate upd) {
     const int64_t e = (int64_t)blockIdx.x * X + threadIdx.x;
     const bool ok = e < elems4;
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -2042,7 +2061,7 @@ __global__ void __launch_bounds__(X * Y) slice_sum4_kernel(const float4* __restr
 #pragma unroll 4
         for (int z = threadIdx.y; z < slices; z += Y) add4(acc, partial[(size_t)z * elems4 + e]);
     }
-    store_group_sum<X, Y>(acc, out + e, ok);
+    store_group_sum<X, Y>(acc, out + e, ok, upd, e);
 }
 
 __global__ void slice_sum_tc_kernel(const float* __restrict__ partial, float* __restrict__ out, int64_t elems, int slices) {
@@ -2054,16 +2073,18 @@ __global__ void slice_sum_tc_kernel(const float* __restrict__ partial, float* __
 }
 
 // sum of the `slices` partial results of a split wgrad into the caller's gradient
-static void launch_slice_sum(const float* partial, float* out, int64_t elems, int slices, cudaStream_t st) {
-    if (elems % 4 || ((uintptr_t)partial | (uintptr_t)out) % 16) {
+static void launch_slice_sum(const float* partial, float* out, int64_t elems, int slices, cudaStream_t st,
+                             const SgdUpdate& upd = SgdUpdate()) {
+    if (elems % 4 || ((uintptr_t)partial | (uintptr_t)out) % 16 || (upd.w && (uintptr_t)upd.w % 16)) {
         slice_sum_tc_kernel<<<(unsigned)((elems + 255) / 256), 256, 0, st>>>(partial, out, elems, slices);
+        if (upd.w) sgd_update(upd, out, elems, st);
         return;
     }
     const int64_t elems4 = elems / 4;
     const unsigned blocks = (unsigned)((elems4 + 31) / 32);
-    if (slices >= 16) slice_sum4_kernel<32, 8><<<blocks, dim3(32, 8), 0, st>>>((const float4*)partial, (float4*)out, elems4, slices);
-    else if (slices >= 4) slice_sum4_kernel<32, 4><<<blocks, dim3(32, 4), 0, st>>>((const float4*)partial, (float4*)out, elems4, slices);
-    else slice_sum4_kernel<256, 1><<<(unsigned)((elems4 + 255) / 256), dim3(256, 1), 0, st>>>((const float4*)partial, (float4*)out, elems4, slices);
+    if (slices >= 16) slice_sum4_kernel<32, 8><<<blocks, dim3(32, 8), 0, st>>>((const float4*)partial, (float4*)out, elems4, slices, upd);
+    else if (slices >= 4) slice_sum4_kernel<32, 4><<<blocks, dim3(32, 4), 0, st>>>((const float4*)partial, (float4*)out, elems4, slices, upd);
+    else slice_sum4_kernel<256, 1><<<(unsigned)((elems4 + 255) / 256), dim3(256, 1), 0, st>>>((const float4*)partial, (float4*)out, elems4, slices, upd);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -2828,9 +2849,9 @@ static int wgrad_rows_attr() {
 }
 
 int tc_conv_wgrad(const ConvGeom& g, const void* dz, const void* x, float* dw, void* scratch, int64_t scratch_bytes,
-                  int* device_status, void* stream) {
+                  int* device_status, void* stream, const SgdUpdate& upd) {
     if (!device_status) { set_error("no status word"); return CKPT_E_NULL; }
-    if (wgrad_pairview_applies(g) && (uintptr_t)dw % 16 == 0) {      // the fold stores float4; otherwise the 64-channel kernel below
+    if (wgrad_pairview_applies(g) && (uintptr_t)dw % 16 == 0 && (uintptr_t)upd.w % 16 == 0) {      // the fold stores float4; otherwise the 64-channel kernel below
         WRowsParams p;
         int co_tiles;
         wgrad_pairview_plan(g, &p, &co_tiles);
@@ -2847,7 +2868,7 @@ int tc_conv_wgrad(const ConvGeom& g, const void* dz, const void* x, float* dw, v
         dim3 grid(p.slices, 2, co_tiles);
         tc_wgrad_rows_kernel<<<grid, kThreads, smem, st>>>(mdz, mx, (float*)scratch, p, device_status);
         CKPT_LAUNCH_CHECK_NAMED("tc_wgrad_rows_kernel (pixel pairs)", "conv wgrad, 64 input channels as pixel pairs (tensor cores)");
-        pairview_fold_kernel<8><<<(unsigned)((g.cout * 144 + 31) / 32), dim3(32, 8), 0, st>>>((const float*)scratch, dw, g.cout, p.slices);
+        pairview_fold_kernel<8><<<(unsigned)((g.cout * 144 + 31) / 32), dim3(32, 8), 0, st>>>((const float*)scratch, dw, g.cout, p.slices, upd);
         CKPT_LAUNCH_CHECK_NAMED("pairview_fold_kernel", "wgrad pair fold");
         return CKPT_OK;
     }
@@ -2872,7 +2893,7 @@ int tc_conv_wgrad(const ConvGeom& g, const void* dz, const void* x, float* dw, v
         dim3 grid(p.slices, g.cout / 64);
         tc_wgrad_c64_kernel<<<grid, kThreads, smem, st>>>(mdz, mx, (float*)scratch, p, device_status);
         CKPT_LAUNCH_CHECK_NAMED("tc_wgrad_c64_kernel", "conv wgrad, 64 input channels (tensor cores)");
-        launch_slice_sum((const float*)scratch, dw, elems, p.slices, st);
+        launch_slice_sum((const float*)scratch, dw, elems, p.slices, st, upd);
         CKPT_LAUNCH_CHECK_NAMED("slice_sum_kernel", "wgrad slice sum");
         return CKPT_OK;
     }
@@ -2894,7 +2915,7 @@ int tc_conv_wgrad(const ConvGeom& g, const void* dz, const void* x, float* dw, v
         dim3 grid(p.slices, pairs, co_tiles);
         tc_wgrad_rows_kernel<<<grid, kThreads, smem, st>>>(mdz, mx, (float*)scratch, p, device_status);
         CKPT_LAUNCH_CHECK_NAMED("tc_wgrad_rows_kernel", "conv wgrad, shared vertical taps (tensor cores)");
-        launch_slice_sum((const float*)scratch, dw, elems, p.slices, st);
+        launch_slice_sum((const float*)scratch, dw, elems, p.slices, st, upd);
         CKPT_LAUNCH_CHECK_NAMED("slice_sum_kernel", "wgrad slice sum");
         return CKPT_OK;
     }
@@ -2921,8 +2942,10 @@ int tc_conv_wgrad(const ConvGeom& g, const void* dz, const void* x, float* dw, v
     tc_conv_wgrad_kernel<<<grid, kThreads, smem, st>>>(mdz, mx, target, p, device_status);
     CKPT_LAUNCH_CHECK_NAMED("tc_conv_wgrad_kernel", "conv wgrad (tensor cores)");
     if (slices > 1) {
-        launch_slice_sum((const float*)scratch, dw, elems, slices, st);
+        launch_slice_sum((const float*)scratch, dw, elems, slices, st, upd);
         CKPT_LAUNCH_CHECK_NAMED("slice_sum_kernel", "wgrad slice sum");
+    } else if (upd.w) {
+        return sgd_update(upd, dw, elems, st);       // the gradient went straight to the caller's buffer
     }
     return CKPT_OK;
 }

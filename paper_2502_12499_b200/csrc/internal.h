@@ -65,6 +65,17 @@ private:
     int64_t capacity_, live_bytes_ = 0, high_water_ = 0, extent_ = 0;
 };
 
+// "Update w_i with g_i" (last line of the backward loop of Algorithms 1, 2 and 4) as plain gradient descent,
+// w <- w - lr * g, applied to a parameter in its storage type (bf16 parameters: float32 arithmetic, rounded to nearest
+// even).  w == nullptr means no update.  The tensor-core wgrad applies it in the pass that sums its slices; every other
+// gradient takes the stand-alone kernel.
+struct SgdUpdate {
+    void* w = nullptr;
+    float lr = 0.f;
+    int dtype = CKPT_DTYPE_F32;
+};
+int sgd_update(const SgdUpdate& u, const float* g, int64_t elems, void* stream);
+
 // ------------------------------------------------------------------ kernel launchers (kernels_simt.cu)
 struct ConvGeom {
     int n, h, w, cin, ho, wo, cout, k, stride, pad;
@@ -110,8 +121,9 @@ int tc_conv_fwd_stats(const ConvGeom& g, const void* x, const void* w, void* z, 
                       int64_t partial_bytes = 0);
 int tc_conv_dgrad(const ConvGeom& g, const void* dz, const void* w, void* dx, void* scratch,
                   int64_t scratch_bytes, int* device_status, void* stream);
+// upd: optional parameter update applied together with the gradient (the filter must no longer be needed by this step)
 int tc_conv_wgrad(const ConvGeom& g, const void* dz, const void* x, float* dw, void* scratch,
-                  int64_t scratch_bytes, int* device_status, void* stream);
+                  int64_t scratch_bytes, int* device_status, void* stream, const SgdUpdate& upd = SgdUpdate());
 
 // One tiny kernel whose only wait has no producer and gives up after `limit_cycles` (1 .. 2e9), writing its code
 // into the status word: the bounded-wait path, run to its limit on purpose.
@@ -167,5 +179,6 @@ int sum_loss(int dtype, int64_t elems, const void* y, double* loss, void* grad, 
              void* stream);
 int64_t sum_loss_scratch_bytes();
 int device_copy(void* dst, const void* src, int64_t bytes, void* stream);
+
 
 }  // namespace ckpt

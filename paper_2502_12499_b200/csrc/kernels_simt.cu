@@ -1610,4 +1610,20 @@ int device_copy(void* dst, const void* src, int64_t bytes, void* stream) {
     return CKPT_OK;
 }
 
+// w <- w - lr * g, element by element (float32 arithmetic; bf16 parameters rounded to nearest even).
+template <typename T>
+__global__ void sgd_update_kernel(T* __restrict__ w, const float* __restrict__ g, int64_t elems, float lr) {
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < elems; i += (int64_t)gridDim.x * blockDim.x) {
+        if constexpr (sizeof(T) == 2) w[i] = __float2bfloat16_rn(fmaf(-lr, g[i], __bfloat162float(w[i])));
+        else w[i] = fmaf(-lr, g[i], w[i]);
+    }
+}
+int sgd_update(const SgdUpdate& u, const float* g, int64_t elems, void* stream) {
+    if (!u.w || elems <= 0) return CKPT_OK;
+    if (u.dtype == CKPT_DTYPE_BF16) sgd_update_kernel<__nv_bfloat16><<<elementwise_grid(elems), 256, 0, (cudaStream_t)stream>>>((__nv_bfloat16*)u.w, g, elems, u.lr);
+    else sgd_update_kernel<float><<<elementwise_grid(elems), 256, 0, (cudaStream_t)stream>>>((float*)u.w, g, elems, u.lr);
+    CKPT_LAUNCH_CHECK("parameter update");
+    return CKPT_OK;
+}
+
 }  // namespace ckpt

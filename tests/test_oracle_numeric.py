@@ -226,3 +226,24 @@ def test_split_chain_equals_fused_chain():
                 assert np.array_equal(b["d"][fi + 1], np.maximum(b["d"][fi], 0))
             if u["kind"] == "bn":
                 np.testing.assert_allclose(b["d"][fi + 1].mean(axis=(0, 1, 2)), fparams[fi]["beta"], atol=1e-12)
+
+
+def test_sgd_update_is_a_descent_step():
+    """"Update w_i with g_i" as w - lr*g: hand values, and along -g the float64 loss of a tiny chain goes down by
+    lr * |g|^2 to first order."""
+    new = no.sgd_update([{"w": np.array([1.0, -2.0]), "b": np.array([0.5])}], [{"w": np.array([0.5, 0.25]), "b": np.array([-1.0])}], 0.1)
+    assert np.allclose(new[0]["w"], [0.95, -2.025]) and np.allclose(new[0]["b"], [0.6])
+    rounded = no.sgd_update([{"w": np.array([1.0 + 2.0 ** -9]), "gamma": np.array([1.0 + 2.0 ** -9])}],
+                            [{"w": np.array([0.0]), "gamma": np.array([0.0])}], 0.1, storage="bf16")
+    assert rounded[0]["w"][0] == 1.0 and rounded[0]["gamma"][0] == 1.0 + 2.0 ** -9      # only matrices are stored in bf16
+    from paper_2502_12499_b200 import workloads as wl
+    spec = wl.plain_chain(2, 4, 3, (6, 6), 2, "f32", "softmax_ce", name="tiny")
+    spec["units"].append({"kind": "fc", "cin": 6 * 6 * 4, "cout": 5, "relu": False})
+    params = [{k: v.astype(np.float64) for k, v in p.items()} for p in wl.make_params(spec, seed=2, bn_affine="random")]
+    x, labels = wl.make_batch(spec, seed=3)
+    ref = no.chain_forward_backward(spec, params, x.astype(np.float64), labels)
+    lr = 1e-4
+    after = no.chain_forward_backward(spec, no.sgd_update(params, ref["grads"], lr), x.astype(np.float64), labels)
+    g2 = sum(float((g ** 2).sum()) for unit in ref["grads"] for g in unit.values())
+    assert after["loss"] < ref["loss"]
+    assert abs((ref["loss"] - after["loss"]) - lr * g2) <= 0.05 * lr * g2
