@@ -1202,7 +1202,8 @@ struct WgradParams {
     int H, W, N;                 // the dz pixel grid
     int c_out, c_in;
     int k, pad, stride;          // input pixel of a term = dz pixel * stride + filter position - pad
-    int tw, th, tn;              // pixel tile, tw*th*tn = 64
+    int tw, th, tn;              // pixel tile, tw*th*tn = px
+    int px;                      // pixels per operand box and stage: 64, 128 or 256
     int tiles_w, tiles_h, tiles_n;
     int nb;                      // column blocks per CTA (1..4)
     int total_blocks;            // k*k*c_in/64
@@ -1216,7 +1217,12 @@ tc_conv_wgrad_kernel(const __grid_constant__ CUtensorMap map_dz, const __grid_co
                      float* __restrict__ partial, WgradParams p, int* status) {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-    constexpr uint32_t box_bytes = 64 * 128;                      // 64 pixels x 64 channels
+    // One copy brings px pixels x 64 channels (px = 64, 128 or 256: as many as leave two stages in shared memory, so
+    // that a stage is 8 to 16 MMAs and the barrier rounds are few).  Measured with clock64 on the ResNet-50 1x1 layers
+    // (batch 128): the main loop runs at 23-30 bytes per clock and SM of operand feed from the L2 with every SM
+    // loading (8 TB/s in total: that, not the tensor core, bounds it), and the 128 x 256 float accumulator takes as
+    // long to leave as six such stages take to load when all CTAs of a wave store at once.
+    const uint32_t box_bytes = (uint32_t)p.px * 128;              // px pixels x 64 channels
     const uint32_t stage_bytes = (2 + (uint32_t)p.nb) * box_bytes;
     const uint32_t bars = base + (uint32_t)p.stages * stage_bytes;
     __shared__ uint32_t tmem_base_slot;
@@ -1268,12 +1274,16 @@ tc_conv_wgrad_kernel(const __grid_constant__ CUtensorMap map_dz, const __grid_co
             const int h0 = (t % p.tiles_h) * p.th;
             const int n0 = (t / p.tiles_h) * p.tn;
             const uint32_t dst = base + (uint32_t)s * stage_bytes;
-            if (lane < 2) {
-                tma_load_4d(dst + lane * box_bytes, &map_dz, full_bar(s), co_tile * 128 + 64 * lane, w0, h0, n0);
-            } else if (lane < 2 + nb_here) {
-                const int j = lane - 2;
+            if (lane < 2 + nb_here) {
+                // one instruction for all copies of the stage: the lanes differ in tensor map, coordinates and target only
+                const bool is_dz = lane < 2;
+                const int j = is_dz ? 0 : lane - 2;
                 const int b = blk_begin + j, tap = b / cin_blocks, cib = b % cin_blocks;
-                tma_load_4d(dst + (2 + j) * box_bytes, &map_x, full_bar(s), cib * 64, w0 * p.stride + tap % p.k - p.pad, h0 * p.stride + tap / p.k - p.pad, n0);
+                const CUtensorMap* map = is_dz ? &map_dz : &map_x;
+                const int c0 = is_dz ? co_tile * 128 + 64 * lane : cib * 64;
+                const int c1 = is_dz ? w0 : w0 * p.stride + tap % p.k - p.pad;
+                const int c2 = is_dz ? h0 : h0 * p.stride + tap / p.k - p.pad;
+                tma_load_4d(dst + (uint32_t)lane * box_bytes, map, full_bar(s), c0, c1, c2, n0);
             }
             issued = it + 1;
         }
@@ -1291,8 +1301,9 @@ tc_conv_wgrad_kernel(const __grid_constant__ CUtensorMap map_dz, const __grid_co
             tc_fence_after();
             const uint32_t a_addr = base + (uint32_t)s * stage_bytes;
             const uint32_t b_addr = a_addr + 2 * box_bytes;
-#pragma unroll
-            for (int kk = 0; kk < 4; ++kk) {        // 4 x (K = 16 pixels = 2 groups of 8 rows = 2048 bytes)
+            const int k_steps = p.px / 16;
+#pragma unroll 4
+            for (int kk = 0; kk < k_steps; ++kk) {  // K = 16 pixels = 2 groups of 8 rows = 2048 bytes per step
                 umma_bf16(tmem_base, smem_desc(a_addr + kk * 2048, box_bytes, 1024), smem_desc(b_addr + kk * 2048, box_bytes, 1024),
                           idesc, (it > 0 || kk > 0) ? 1u : 0u);
             }
@@ -2528,35 +2539,40 @@ int launch_fc(const ConvGeom& g, const void* x, const void* w, void* z, const fl
 
 void wgrad_plan(const ConvGeom& g, WgradParams* p, int* slices, int* groups, int* co_tiles) {
     p->H = g.ho; p->W = g.wo; p->N = g.n; p->c_out = g.cout; p->c_in = g.cin; p->k = g.k; p->pad = g.pad; p->stride = g.stride;
-    choose_tile(64, g.wo, g.ho, g.n, &p->tw, &p->th, &p->tn);
-    p->tiles_w = (g.wo + p->tw - 1) / p->tw; p->tiles_h = (g.ho + p->th - 1) / p->th; p->tiles_n = (g.n + p->tn - 1) / p->tn;
-    p->total_tiles = p->tiles_w * p->tiles_h * p->tiles_n;
     p->total_blocks = g.k * g.k * g.cin / 64;
     // column blocks per CTA: 4 when that divides evenly or the remainder is small, else 3
     p->nb = p->total_blocks % 4 == 0 ? 4 : (p->total_blocks % 3 == 0 ? 3 : (p->total_blocks >= 4 ? 4 : p->total_blocks));
+    // pixels per stage: as many as leave two stages in shared memory (96 KB per stage at most), for reductions long
+    // enough to use them; short ones - the fully connected layers - keep 64: they are bound by their stores, see below
+    const int64_t pixels = (int64_t)g.n * g.ho * g.wo;
+    p->px = 64;
+    if (g.stride == 1 && pixels >= 4096) p->px = p->nb == 1 ? 256 : 128;
+    choose_tile(p->px, g.wo, g.ho, g.n, &p->tw, &p->th, &p->tn);
+    p->tiles_w = (g.wo + p->tw - 1) / p->tw; p->tiles_h = (g.ho + p->th - 1) / p->th; p->tiles_n = (g.n + p->tn - 1) / p->tn;
+    p->total_tiles = p->tiles_w * p->tiles_h * p->tiles_n;
     // a reduction of one or two pixel tiles is all stores: narrower CTAs (128 accumulator columns) fit four to an SM
     if (p->total_tiles <= 2 && p->total_blocks >= 2) p->nb = 2;
     *groups = (p->total_blocks + p->nb - 1) / p->nb;
     *co_tiles = (g.cout + 127) / 128;
-    // slices of the pixel range: fill the SMs with whole waves of equally long CTAs (2 to 4 waves),
-    // keeping at least 8 pixel tiles per slice
+    // slices of the pixel range: one wave of equally long CTAs that fills the SMs as far as it can (every CTA pays
+    // for its accumulator's way out - 128 KB of partial sums - once, so fewer and longer CTAs win: 256 -> 1024 at
+    // 14 x 14, batch 128: 35 us in one wave of 144 against 49 us in two waves of 288), at least 512 pixels per slice
     const int64_t base_ctas = (int64_t)*groups * *co_tiles;
     int sms = 148, dev = 0;
     cudaGetDevice(&dev);
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    int64_t by_k = std::max<int64_t>(1, p->total_tiles / 8);
+    int64_t by_k = std::max<int64_t>(1, (int64_t)p->total_tiles * p->px / 512);
     int64_t s = 1;
     double best_eff = -1.0;
     for (int64_t cand = 1; cand <= std::min<int64_t>(by_k, 256); ++cand) {
         const int64_t ctas = cand * base_ctas;
-        const int64_t waves = (ctas + sms - 1) / sms;
-        if (waves > 4 && cand > 1) break;
-        const double eff = (double)ctas / (double)(waves * sms) * (waves >= 2 ? 1.0 : 0.9);
+        if (ctas > sms && cand > 1) break;
+        const double eff = (double)ctas / (double)sms;
         if (eff > best_eff + 1e-9) { best_eff = eff; s = cand; }
     }
     p->tiles_per_slice = (int)((p->total_tiles + s - 1) / s);
     *slices = (p->total_tiles + p->tiles_per_slice - 1) / p->tiles_per_slice;
-    const uint32_t stage_bytes = (2 + p->nb) * 64 * 128;
+    const uint32_t stage_bytes = (2 + p->nb) * (uint32_t)p->px * 128;
     // no more stages than pixel tiles per CTA: a short reduction (fully connected layers: one tile) then leaves
     // room for a second CTA on the SM, whose loads run under the first one's stores
     p->stages = std::max(1, std::min<int>(std::min<int>(kMaxStages, kSmemBudget / stage_bytes), p->tiles_per_slice));
@@ -2936,7 +2952,7 @@ int tc_conv_wgrad(const ConvGeom& g, const void* dz, const void* x, float* dw, v
         if (e != cudaSuccess) return cuda_fail(e, "raising the shared-memory limit");
         attr_set = true;
     }
-    const size_t smem = (size_t)p.stages * (2 + p.nb) * 64 * 128 + 1024 + 256;
+    const size_t smem = (size_t)p.stages * (2 + p.nb) * p.px * 128 + 1024 + 256;
     float* target = slices > 1 ? (float*)scratch : dw;
     dim3 grid(slices, groups, co_tiles);
     tc_conv_wgrad_kernel<<<grid, kThreads, smem, st>>>(mdz, mx, target, p, device_status);
