@@ -1503,6 +1503,7 @@ struct WRowsParams {
     // left, at, and one to the right of the output pair that a 3-wide filter row can reach
     int pairview;
     int row_elems;               // floats per partial row: 9 * c_in, or 4 columns * 3 * 64 in the pair view
+    int cols;                    // columns per CTA: 2, or 1 for short reductions (half the partial sums per CTA)
 };
 
 __global__ void __launch_bounds__(kThreads, 1)
@@ -1520,6 +1521,7 @@ tc_wgrad_rows_kernel(const __grid_constant__ CUtensorMap map_dz, const __grid_co
 
     const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
     const int slice = blockIdx.x, pair = blockIdx.y, co_tile = blockIdx.z;
+    const int ncols = p.cols;
     const int my_tiles = slice < p.m_tiles ? (p.m_tiles - slice + p.slices - 1) / p.slices : 0;
     const int cin_blocks = p.c_in / 64;
 
@@ -1547,13 +1549,13 @@ tc_wgrad_rows_kernel(const __grid_constant__ CUtensorMap map_dz, const __grid_co
             const int w0 = (t % p.tiles_w) * 8; t /= p.tiles_w;
             const int h0 = (t % p.tiles_h) * p.th;
             const int img = t / p.tiles_h;
-            if (lane == 0) mbar_expect_tx(full_bar(s), 2 * p.dz_box + 2 * p.patch_bytes);
+            if (lane == 0) mbar_expect_tx(full_bar(s), 2 * p.dz_box + (uint32_t)ncols * p.patch_bytes);
             __syncwarp();
             const uint32_t dst = base + (uint32_t)s * p.stage_bytes;
             if (lane < 2) {
                 tma_load_4d(dst + lane * p.dz_box, &map_dz, full_bar(s), co_tile * 128 + 64 * lane, w0, h0, img);
-            } else if (lane < 4) {
-                const int col = 2 * pair + (lane - 2);
+            } else if (lane < 2 + ncols) {
+                const int col = ncols * pair + (lane - 2);
                 const int ch = p.pairview ? ((col + 1) & 1) * 64 : (col / 3) * 64;
                 const int shift = p.pairview ? (col + 1) / 2 - 1 : col % 3 - 1;
                 tma_load_4d(dst + 2 * p.dz_box + (lane - 2) * p.patch_bytes, &map_x, full_bar(s), ch, w0 + shift, h0 - 1, img);
@@ -1572,7 +1574,7 @@ tc_wgrad_rows_kernel(const __grid_constant__ CUtensorMap map_dz, const __grid_co
             tc_fence_after();
             const uint32_t dz_addr = base + (uint32_t)s * p.stage_bytes;
 #pragma unroll 1
-            for (int c = 0; c < 2; ++c) {
+            for (int c = 0; c < ncols; ++c) {
                 const uint32_t x_addr = dz_addr + 2 * p.dz_box + (uint32_t)c * p.patch_bytes;
                 for (int kk = 0; kk < ksteps; ++kk)
                     umma_bf16(tmem_base + (uint32_t)c * 192, smem_desc(dz_addr + kk * 2048, p.dz_box, 1024),
@@ -1582,6 +1584,9 @@ tc_wgrad_rows_kernel(const __grid_constant__ CUtensorMap map_dz, const __grid_co
         }
         if (ok) umma_commit(accum_bar);
     } else if (warp >= 2) {
+        // Thread l of a warp holds row l (an output channel) of the accumulator and writes its 64 floats of a (column,
+        // dy) block as 16-byte pieces.  (Turning 32 x 32 blocks through shared memory for full-line stores, as the
+        // generic wgrad kernel does for its much wider rows, measured 10-25 % slower here.)
         const int quarter = warp % 4;
         const int co = co_tile * 128 + quarter * 32 + lane;
         const bool valid = co < p.c_out;
@@ -1589,8 +1594,8 @@ tc_wgrad_rows_kernel(const __grid_constant__ CUtensorMap map_dz, const __grid_co
         float* dst_row = partial + ((size_t)slice * p.c_out + (valid ? co : 0)) * row_elems;
         if (my_tiles > 0 && mbar_wait(accum_bar, 0, failed, status, 703)) {
             tc_fence_after();
-            for (int c = 0; c < 2; ++c) {
-                const int col = 2 * pair + c, cib = col / 3, dx = col % 3;
+            for (int c = 0; c < ncols; ++c) {
+                const int col = ncols * pair + c, cib = col / 3, dx = col % 3;
                 for (int dy = 0; dy < 3; ++dy) {
                     float* dst = dst_row + (p.pairview ? (size_t)(col * 3 + dy) * 64
                                                        : (size_t)((dy * 3 + dx) * cin_blocks + cib) * 64);   // column (tap, c_in)
@@ -1608,8 +1613,8 @@ tc_wgrad_rows_kernel(const __grid_constant__ CUtensorMap map_dz, const __grid_co
                 }
             }
         } else if (my_tiles == 0 && valid) {
-            for (int c = 0; c < 2; ++c) {
-                const int col = 2 * pair + c, cib = col / 3, dx = col % 3;
+            for (int c = 0; c < ncols; ++c) {
+                const int col = ncols * pair + c, cib = col / 3, dx = col % 3;
                 for (int dy = 0; dy < 3; ++dy) {
                     float* dst = dst_row + (p.pairview ? (size_t)(col * 3 + dy) * 64 : (size_t)((dy * 3 + dx) * cin_blocks + cib) * 64);
                     for (int e = 0; e < 64; ++e) dst[e] = 0.f;
@@ -2626,6 +2631,7 @@ void wgrad_rows_plan(const ConvGeom& g, WRowsParams* p, int* pairs, int* co_tile
     p->stages = std::max(2, std::min<int>(kMaxStages, (int)((208 * 1024) / p->stage_bytes)));
     p->pairview = 0;
     p->row_elems = 9 * g.cin;
+    p->cols = 2;
 }
 
 // 64 input channels through the same kernel.  Two horizontally adjacent pixels are read as one pixel of twice the
@@ -2648,6 +2654,14 @@ void wgrad_pairview_plan(const ConvGeom& g, WRowsParams* p, int* co_tiles) {
     p->slices = std::max(1, std::min(sms / (2 * *co_tiles), p->m_tiles));
     p->pairview = 1;
     p->row_elems = 4 * 3 * 64;
+    // A short reduction is dominated by what every CTA writes and the fold reads back (128 x 192 floats per column):
+    // with one column per CTA and half as many slices the same SMs are busy with half the partial sums.
+    if (p->m_tiles / p->slices < 16 && p->slices >= 2) {
+        p->cols = 1;
+        p->slices = std::max(1, std::min(sms / (4 * *co_tiles), p->m_tiles));
+        p->stage_bytes = 2 * p->dz_box + p->patch_bytes;
+        p->stages = std::max(2, std::min<int>(kMaxStages, (int)((208 * 1024) / p->stage_bytes)));
+    }
 }
 }  // namespace
 
@@ -2881,7 +2895,7 @@ int tc_conv_wgrad(const ConvGeom& g, const void* dz, const void* x, float* dw, v
         rc = wgrad_rows_attr();
         if (rc) return rc;
         const size_t smem = (size_t)p.stages * p.stage_bytes + 1024 + 256;
-        dim3 grid(p.slices, 2, co_tiles);
+        dim3 grid(p.slices, 4 / p.cols, co_tiles);
         tc_wgrad_rows_kernel<<<grid, kThreads, smem, st>>>(mdz, mx, (float*)scratch, p, device_status);
         CKPT_LAUNCH_CHECK_NAMED("tc_wgrad_rows_kernel (pixel pairs)", "conv wgrad, 64 input channels as pixel pairs (tensor cores)");
         pairview_fold_kernel<8><<<(unsigned)((g.cout * 144 + 31) / 32), dim3(32, 8), 0, st>>>((const float*)scratch, dw, g.cout, p.slices, upd);
