@@ -107,9 +107,11 @@ class ClockSampler:
 
 
 def conv_flops(spec, plan_mask, shapes):
-    """Algorithmic FLOPs of one step: 2*MAC x (forward + recompute of non-checkpoints + dgrad
-    (units 2..n) + wgrad)."""
+    """FLOPs of one step as executed: 2*MAC x (forward + recompute of non-checkpoints + dgrad (units 2..n) + wgrad),
+    plus one more forward of every residual block: only a block's output is chain data, so its backward re-derives
+    the interior tensors under every schedule, store-all included."""
     fwd = []
+    rederived = []          # 1-based indices of units whose backward re-derives its interior tensors (one more forward)
     h, w, c = spec["input_hwc"]
     for u, (ho, wo, co) in zip(spec["units"], shapes[1:]):
         if u["kind"] in ("conv_bn_relu", "conv"):
@@ -120,6 +122,7 @@ def conv_flops(spec, plan_mask, shapes):
             if u["project"]:
                 macs += ho * wo * u["cin"] * co
             fwd.append(2.0 * spec["batch"] * macs)
+            rederived.append(len(fwd))
         elif u["kind"] == "fc":
             fwd.append(2.0 * spec["batch"] * u["cin"] * u["cout"])
         else:
@@ -132,6 +135,8 @@ def conv_flops(spec, plan_mask, shapes):
         total += f                                   # wgrad
         if i > 1:
             total += f                               # dgrad
+        if i in rederived:
+            total += f                               # a residual block's backward re-runs its convolutions (any schedule)
     return total, fwd
 
 
@@ -252,6 +257,7 @@ def measure_config(spec, args, rank, world, steps, regions, with_roofline, peaks
            "h2d_bytes_per_step": int(x_pinned.numel() * x_pinned.element_size() + labels_pinned.numel() * 4), "d2h_bytes_per_step": 12,
            "store_all_ms_per_step": ms_all, "store_all_images_per_s": whole_job_images_per_s(spec["batch"], world, 1, ms_all),
            "recompute_overhead_pct": 100.0 * (ms / ms_all - 1.0),
+           "store_all_note": "residual blocks re-derive their interior tensors in the backward under every schedule, store-all included",
            "recomputed_units": int(rep["recomputed_units"]), "checkpoints": int(mask.sum()),
            "launches_per_step": int(rep["launches"]), "store_all_launches_per_step": int(rep_all["launches"]),
            "memory_gib": {"arena_plan": peak / gib, "arena_store_all": store_all / gib, "arena_measured": rep["peak_bytes"] / gib,

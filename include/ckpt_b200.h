@@ -60,7 +60,10 @@ CKPT_API const char* ckpt_last_error(void);
  *   CKPT_ALGO_DYNAMIC_N2 - Algorithm 5 (Section 4.1): minimises max_i m(i) of Eq. (memory) by the
  *                          O(n^2) recursion Eq. (T-rec).
  *   CKPT_ALGO_DYNAMIC_N  - Algorithm 6 (Section 4.2): same optimum by the monotone-queue /
- *                          two-pointer search.
+ *                          two-pointer search.  Queue pushes, pops and pointer moves are O(n) in total as in
+ *                          the paper; each U(i,j) is evaluated exactly from prefix sums and a range maximum found
+ *                          by bisection (the paper's incremental update of a running maximum cannot be undone when
+ *                          the pointer moves back), so the implementation is O(n log n).
  * Readings of the printed algorithms: data are d_0..d_n and the dynamic recursion runs down to
  * i = 0 (answer M(0)); j ranges up to n inclusive; M(n) = d_n is the base case; Algorithm 3 forces
  * d_n as a checkpoint (answer min_s s + d_n + M(n-1,s)) and inserts candidate i before reading the

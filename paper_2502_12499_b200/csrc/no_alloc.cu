@@ -20,6 +20,9 @@ static __device__ __align__(256) unsigned char g_bn_static_scratch[kStaticScratc
 
 // In host code the array's name is only a handle for the runtime; the address a kernel can use has
 // to be looked up, once per device, while that device is current.
+// The looked-up addresses are cached per device ordinal for the life of the process: they are valid as long as the
+// device's primary context is (a cudaDeviceReset by the caller invalidates them - do not reset a device between calls),
+// and the cache is not locked: the calls are serialised by their callers anyway (they share the one array).
 constexpr int kMaxDevices = 64;
 void* g_scratch_address[kMaxDevices] = {};
 
