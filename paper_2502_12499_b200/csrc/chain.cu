@@ -225,19 +225,27 @@ static BlockBuffers block_buffers(StepCtx& c, const Unit& u) {
 }
 
 // z1, a, z2, b, z3 (and zp) with their statistics; the residual join is left to the caller.
-static int block_interiors(StepCtx& c, const Unit& u, const void* x, const BlockBuffers& B) {
+// have_stats: the block's four statistics blocks are those of this very input (they were written by the unit's last
+// forward, original or recomputed, and every unit has a block of its own), so the backward's re-derivation of the
+// interior tensors runs the convolutions without gathering sums and skips the finalize steps; the tensors come out
+// bit-identical (same kernels, same reduction order).
+static int block_interiors(StepCtx& c, const Unit& u, const void* x, const BlockBuffers& B, bool have_stats = false) {
     const int dt = c.ch->dtype;
     void* const* p = c.params + u.param_first;
     const int64_t in_px = c.ch->batch * u.in.h * u.in.w, out_px = c.ch->batch * u.out.h * u.out.w;
     const int mid = u.desc.mid;
     int rc;
-    if ((rc = conv_with_statistics(c, u.g1, x, p[0], B.z1, (const float*)p[1], (const float*)p[2], B.s1))) return rc;
+    auto conv = [&](const ConvGeom& g, const void* in, int w_index, void* z, float* stats) {
+        if (have_stats) return conv_forward_any(c, g, in, p[w_index], z, nullptr, 0);
+        return conv_with_statistics(c, g, in, p[w_index], z, (const float*)p[w_index + 1], (const float*)p[w_index + 2], stats);
+    };
+    if ((rc = conv(u.g1, x, 0, B.z1, B.s1))) return rc;
     if ((rc = bn_apply(dt, in_px, mid, B.z1, B.s1, 1, B.a, c.stream))) return rc;
-    if ((rc = conv_with_statistics(c, u.g2, B.a, p[3], B.z2, (const float*)p[4], (const float*)p[5], B.s2))) return rc;
+    if ((rc = conv(u.g2, B.a, 3, B.z2, B.s2))) return rc;
     if ((rc = bn_apply(dt, out_px, mid, B.z2, B.s2, 1, B.b, c.stream))) return rc;
-    if ((rc = conv_with_statistics(c, u.g3, B.b, p[6], B.z3, (const float*)p[7], (const float*)p[8], B.s3))) return rc;
+    if ((rc = conv(u.g3, B.b, 6, B.z3, B.s3))) return rc;
     if (u.desc.flags & 2) {
-        if ((rc = conv_with_statistics(c, u.gp, x, p[9], B.zp, (const float*)p[10], (const float*)p[11], B.sp))) return rc;
+        if ((rc = conv(u.gp, x, 9, B.zp, B.sp))) return rc;
     }
     return CKPT_OK;
 }
@@ -263,7 +271,7 @@ static int block_backward(StepCtx& c, const Unit& u, const void* x, const void* 
     const int mid = u.desc.mid, co = u.out.c;
     const bool project = (u.desc.flags & 2) != 0;
     int rc;
-    if ((rc = block_interiors(c, u, x, B))) return rc;
+    if ((rc = block_interiors(c, u, x, B, true))) return rc;
     // through the final ReLU: g_in <- dL/d(bn3 + shortcut)
     if ((rc = relu_mask_inplace(dt, out_px * co, g_in, y, c.stream))) return rc;
     const void* dx_shortcut = g_in;                       // identity shortcut: the same gradient flows to x
