@@ -3,7 +3,7 @@
     python bench_ops.py conv fwd|dgrad|wgrad N H W C_IN C_OUT K PAD [STRIDE] [--reps R]
     python bench_ops.py bn fwd|bwd ROWS C [--reps R]
     python bench_ops.py pool fwd|bwd N H W C [--reps R]
-    python bench_ops.py convmix fwd|dgrad|wgrad CONFIG        (all conv layers of a benchmark configuration)
+    python bench_ops.py convmix fwd|dgrad|wgrad CONFIG [--batch B]   (all conv layers of a benchmark configuration)
 
 Prints one JSON line with the CUDA-event time per launch and the algorithmic throughput (TFLOP/s for convolutions,
 GB/s for the memory-bound operations).  bf16 storage throughout.  Everything goes through the C ABI; torch only
@@ -239,6 +239,7 @@ def main():
     ap.add_argument("dims", type=int, nargs="+")
     ap.add_argument("--reps", type=int, default=None)
     ap.add_argument("--impl", type=int, default=0)
+    ap.add_argument("--batch", type=int, default=0, help="convmix: run the configuration's layers at this batch (small profiler captures)")
     a = ap.parse_args()
     if a.kind == "convmix":
         from paper_2502_12499_b200 import workloads as wl
@@ -247,7 +248,10 @@ def main():
         if os.path.exists(path):
             p = json.load(open(path))
             peaks = dict(tflops_burst=p["bf16_tflops"], hbm_gbs=p["hbm_gbs"])
-        out = conv_mix(a.what, wl.config(a.dims[0]), peaks, reps=a.reps)
+        spec = wl.config(a.dims[0])
+        if a.batch:
+            spec = dict(spec, batch=a.batch)
+        out = conv_mix(a.what, spec, peaks, reps=a.reps)
     elif a.kind == "conv":
         out = conv(a.what, *a.dims, reps=a.reps, impl=a.impl)
     elif a.kind == "bn":
