@@ -480,8 +480,13 @@ struct TParams {
     int patch_ok;                // the caller filled ncols / col_term
     int ncols;                   // columns per 64-channel block: (horizontal offset, channel offset) pairs
     int col_term[4][3];          // term (index into the tap tables) of column c at vertical tap dy; tap_dh = dy - 1
-    int tile_cols;               // pixels per tile = 8 * th
-    uint32_t patch_bytes;        // 8 x (th + 2) pixels x 128 bytes
+    int tile_cols;               // pixels per tile = 8 * th * stack
+    uint32_t patch_bytes;        // 8 x (th + 2) pixels x 128 bytes; stacked: 8 x th x stack
+    // stacked form for small images (tc_conv_tp_kernel): a tile is the strip of `stack` whole images, each taking th
+    // rows of the accumulator (its H rows and th - H idle ones) and th rows of the patch (rows -1 .. th - 2: the image,
+    // its halo and zero fill), so that image i's patch starts exactly th rows after image i-1's and the operand of
+    // vertical tap dy is still the patch read from byte dy * 1024 on
+    int stack;                   // 0 = one image per tile with a halo of its own (th + 2 patch rows)
 };
 
 template <bool A_MN>
@@ -715,8 +720,8 @@ tc_conv_tp_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
     auto tile_origin = [&](int j, int& w0, int& h0, int& n0) {
         int t = first + j * p.ctas_per_co;
         w0 = (t % p.tiles_w) * 8; t /= p.tiles_w;
-        h0 = (t % p.tiles_h) * p.th;
-        n0 = t / p.tiles_h;
+        if (p.stack) { h0 = 0; n0 = t * p.stack; }
+        else { h0 = (t % p.tiles_h) * p.th; n0 = t / p.tiles_h; }
     };
 
     if (threadIdx.x == 0) {
@@ -810,7 +815,9 @@ tc_conv_tp_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
 #pragma unroll 1
             for (int c0 = 0; c0 < p.tile_cols; c0 += 32, ++chunk_count) {
                 const int idx = c0 + lane;
-                const bool inside = (w0 + (idx & 7) < p.W) && (h0 + (idx >> 3) < p.H);
+                // accumulator row (idx / 8) -> image of the stack and row of that image
+                const int arow = idx >> 3, img = p.stack ? arow / p.th : 0, hrow = p.stack ? arow % p.th : arow;
+                const bool inside = (w0 + (idx & 7) < p.W) && (h0 + hrow < p.H) && (n0 + img < p.N);
                 const uint32_t in_mask = __ballot_sync(0xffffffffu, inside);
                 uint32_t v[32];
                 tmem_ld32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * 256 + c0), v);
@@ -821,7 +828,9 @@ tc_conv_tp_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
                 fence_proxy_async();
                 __syncwarp();
                 if (lane == 0 && in_mask != 0u && co_tile * 128 + quarter * 32 < p.c_out) {
-                    tma_store_4d(&map_out, slab, co_tile * 128 + quarter * 32, w0, h0 + (c0 >> 3), n0);
+                    const int crow = c0 >> 3;                    // a chunk is four accumulator rows of one image (th % 4 == 0)
+                    tma_store_4d(&map_out, slab, co_tile * 128 + quarter * 32, w0, p.stack ? crow % p.th : h0 + crow,
+                                 p.stack ? n0 + crow / p.th : n0);
                     tma_store_commit();
                 }
             }
@@ -2326,21 +2335,48 @@ bool tp_strip(int H, int W, int N, int co_tiles, int* th_out) {
     return true;
 }
 
+// Small images (H + 2 <= 16: the 14 x 14 layers): strips of `stack` whole images, th = 16 accumulator and patch rows
+// each.  Three quarters of such a tile are real pixels at 14 x 14; still better than one pixel box per tap (the plain
+// role-swapped kernel) while that kernel has fewer than two tiles per SM to run.
+bool tp_stack(int H, int W, int N, int co_tiles, int* th_out, int* stack_out) {
+    const int th = (H + 2 + 3) / 4 * 4;
+    if (th > 16 || H < 8) return false;
+    const int stack = 32 / th, tiles_w = (W + 7) / 8;
+    const double cover = (double)W * H / ((double)tiles_w * 8 * th);
+    if (cover < 0.7 || (int64_t)tiles_w * ((N + stack - 1) / stack) * co_tiles < TP_MIN_TILES) return false;
+    // with many tiles per SM the plain kernel's full tiles win again (measured, 256 -> 256 at 14 x 14: batch 128
+    // 0.037 -> 0.035 ms stacked, batch 256 0.053 -> 0.060 ms; 512 -> 512 at batch 64 0.064 -> 0.058 ms)
+    int sms = 148, dev = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    if (((int64_t)N * H * W + 255) / 256 * co_tiles >= 2 * (int64_t)sms) return false;
+    *th_out = th; *stack_out = stack;
+    return true;
+}
+
 int launch_t_core(TParams p, const void* x, int x_channels, const CUtensorMap& mw, void* out, float* stat_partial, int* stat_blocks,
                   int N, int H, int W, int c_red, int c_out, int* status, cudaStream_t st, const char* what, bool a_mn) {
     p.H = H; p.W = W; p.N = N; p.c_red = c_red; p.c_out = c_out;
     choose_tile(256, W, H, N, &p.tw, &p.th, &p.tn);
     bool patch = false;
-    int strip_h = 0;
+    int strip_h = 0, stack = 0;
+    p.stack = 0;
     if (p.patch_ok && tp_strip(H, W, N, (c_out + 127) / 128, &strip_h)) {
         patch = true;
         p.tw = 8; p.th = strip_h; p.tn = 1;
         p.tile_cols = 8 * strip_h;
         p.patch_bytes = (uint32_t)(8 * (strip_h + 2)) * 128;
+    } else if (p.patch_ok && tp_stack(H, W, N, (c_out + 127) / 128, &strip_h, &stack)) {
+        patch = true;
+        p.stack = stack;
+        p.tw = 8; p.th = strip_h; p.tn = stack;
+        p.tile_cols = 8 * strip_h * stack;
+        p.patch_bytes = (uint32_t)(8 * strip_h * stack) * 128;
     }
     p.tw_log = 0; while ((1 << p.tw_log) < p.tw) ++p.tw_log;
     p.th_log = 0; while ((1 << p.th_log) < p.th) ++p.th_log;
     p.tiles_w = (W + p.tw - 1) / p.tw; p.tiles_h = (H + p.th - 1) / p.th; p.tiles_n = (N + p.tn - 1) / p.tn;
+    if (p.stack) p.tiles_h = 1;
     p.co_tiles = (c_out + 127) / 128;
     p.p_tiles = p.tiles_w * p.tiles_h * p.tiles_n;
     int sms = 148, dev = 0;
@@ -2351,7 +2387,7 @@ int launch_t_core(TParams p, const void* x, int x_channels, const CUtensorMap& m
     constexpr uint32_t t_slabs = 8 * 2 * 2048;          // two chunk slabs for each of the eight epilogue warps
     p.stages = std::min<int>(kMaxStages, (227 * 1024 - 1024 - 256 - t_slabs - 64) / stage_bytes);
     CUtensorMap mx;
-    int rc = make_act_map(&mx, x, N, H, W, x_channels, p.tw, patch ? p.th + 2 : p.th, p.tn);
+    int rc = make_act_map(&mx, x, N, H, W, x_channels, p.tw, patch && !p.stack ? p.th + 2 : p.th, p.tn);
     if (rc) return rc;
     // the box of one epilogue chunk: 32 consecutive pixels of the tile (w fastest) x 32 channels, no swizzle
     CUtensorMap mo;
