@@ -278,7 +278,8 @@ def measure_config(spec, args, rank, world, steps, regions, with_roofline, peaks
 
 def kernel_rooflines(spec, peaks):
     """The step's kernels one at a time on the chain's own layer shapes (CUDA events, buffers rotated beyond the L2,
-    >= 20 launches and >= 10 ms per shape): forward, dgrad and wgrad convolution mixes against the measured dense-bf16
+    >= 20 launches and >= 10 ms per shape): forward, dgrad and wgrad mixes over the chain's convolutions (the fully
+    connected layers, HBM-bound matrix-streaming kernels, are listed apart as fc_*) against the measured dense-bf16
     peak (burst: kernels timed in isolation) and, per shape, against whichever of the tensor and HBM roofs bounds it;
     batch norm and 2x2 pooling over every tensor of the chain against the measured copy bandwidth."""
     import bench_ops
@@ -287,6 +288,11 @@ def kernel_rooflines(spec, peaks):
         mix = bench_ops.conv_mix(what, spec, peaks)
         out["conv_" + what] = {"tflops": mix["tflops"], "frac_of_tensor_peak": mix["frac_of_tensor_peak"], "frac_of_roof": mix["frac_of_roof"],
                                "launches": mix["launches"], "ms": mix["ms"], "flops": mix["flops"], "per_shape": mix["per_shape"]}
+    for what in ("fwd", "dgrad", "wgrad"):           # fully connected layers: kernels of their own, bound by the matrix traffic
+        mix = bench_ops.conv_mix(what, spec, peaks, layers="fc")
+        if mix is not None:
+            out["fc_" + what] = {"gbs": sum(r["gbs"] * r["ms"] for r in mix["per_shape"]) / mix["ms"], "frac_of_roof": mix["frac_of_roof"],
+                                 "launches": mix["launches"], "ms": mix["ms"], "per_shape": mix["per_shape"]}
     tot_f = sum(out["conv_" + w]["flops"] for w in ("fwd", "dgrad", "wgrad"))
     tot_ms = sum(out["conv_" + w]["ms"] for w in ("fwd", "dgrad", "wgrad"))
     out["conv_all"] = {"tflops": tot_f / tot_ms / 1e9, "frac_of_tensor_peak": tot_f / tot_ms / 1e9 / peaks["tflops_burst"],
@@ -402,14 +408,14 @@ def main():
 def headline_roofline(r, peaks):
     """The contract's roofline object for the dominant kernels of the headline workload: the implicit-GEMM
     convolution-forward kernels (they run in the forward phase, in segment recomputation and, on the transposed
-    filter, as dgrad).  achieved = sum of algorithmic FLOPs of the chain's conv layers / sum of their launch times."""
+    filter, as dgrad).  achieved = sum of algorithmic FLOPs of the chain's convolution layers / sum of their launch times."""
     f = r["conv_fwd"]
     return {"kernel": "tc_conv_tp_kernel / tc_conv_t_kernel (implicit-GEMM conv forward over the chain's layer mix)", "bound": "tensor",
             "achieved": f["tflops"], "peak": peaks["tflops_burst"], "unit": "TFLOP/s", "frac": f["frac_of_tensor_peak"],
             "peak_source": peaks["source"] + " (burst: kernels timed in isolation)", "traffic": None,
             "flops_per_launch": f["flops"] / f["launches"], "ms_per_launch": f["ms"] / f["launches"],
             "conv_fwd": f, "conv_dgrad": r["conv_dgrad"], "conv_wgrad": r["conv_wgrad"], "conv_all": r["conv_all"],
-            "elementwise": r["elementwise"]}
+            "fc": {k: v for k, v in r.items() if k.startswith("fc_")}, "elementwise": r["elementwise"]}
 
 
 if __name__ == "__main__":

@@ -134,9 +134,9 @@ def pool(what, n, h, w, c, reps=None):
 
 def chain_layers(spec):
     """Walks a chain description and lists what its step runs, with input sizes:
-    convs = (n, h, w, c_in, c_out, k, pad, stride) of every convolution (units and bottleneck interiors; fully
-    connected layers as 1x1 convolutions on a 1x1 image), norms = (rows, channels) of every batch normalisation,
-    pools = (n, h, w, c) of every 2x2 max-pool."""
+    convs = (n, h, w, c_in, c_out, k, pad, stride) of every convolution (units and bottleneck interiors), followed by
+    the fully connected layers as 1x1 convolutions on a 1x1 image (h = w = 1), norms = (rows, channels) of every batch
+    normalisation, pools = (n, h, w, c) of every 2x2 max-pool."""
     convs, norms, pools = [], [], []
     h, w, c = spec["input_hwc"]
     b = spec["batch"]
@@ -180,12 +180,19 @@ def chain_layers(spec):
     return convs, norms, pools
 
 
-def conv_mix(what, spec, peaks, reps=None, min_cin=16):
-    """The conv kernels `what` over every convolution of a chain with at least `min_cin` input channels (the 3-channel
-    first layers are gather kernels of their own): per-shape numbers and the launch-weighted totals.
+def is_fc(shape):
+    return shape[1] == 1 and shape[2] == 1 and shape[5] == 1
+
+
+def conv_mix(what, spec, peaks, reps=None, min_cin=16, layers="conv"):
+    """The kernels `what` over every convolution of a chain with at least `min_cin` input channels (the 3-channel
+    first layers are gather kernels of their own), or over its fully connected layers (layers="fc": matrix-streaming
+    kernels of their own, bound by HBM): per-shape numbers and the launch-weighted totals.
     Each shape is held against the roof that bounds it: time_roof = max(FLOPs / tensor peak, bytes / HBM bandwidth)
     with bytes = its operands and result once; frac = time_roof / measured time."""
-    layers = [s for s in chain_layers(spec)[0] if s[3] >= min_cin]
+    layers = [s for s in chain_layers(spec)[0] if s[3] >= min_cin and is_fc(s) == (layers == "fc")]
+    if not layers:
+        return None
     seen, per_layer = {}, []
     for s in layers:
         if s not in seen:
