@@ -284,3 +284,23 @@ def test_launch_log_is_empty_without_launches():
     ck.launch_log(True)
     assert ck.launch_log_read() == {}
     ck.launch_log(False)
+
+
+def test_chain_option_errors_need_no_device():
+    """Argument checks of the chain options (host only: nothing is launched or dereferenced)."""
+    import ctypes as C
+    from paper_2502_12499_b200 import workloads as wl
+    chain = ck.Chain(wl.config(1))
+    need = int(sum(chain.sizes()[1:]))
+    lib = ck.lib()
+    fake = C.c_void_p(0x1000)                       # never dereferenced: the call only records the address
+    assert lib.ckpt_chain_set_gradient_tap(chain._h, fake, C.c_int64(need - 1)) == -8       # E_WORKSPACE: tap too small
+    assert "tap" in lib.ckpt_last_error().decode()
+    assert lib.ckpt_chain_set_gradient_tap(chain._h, fake, C.c_int64(need)) == 0
+    assert lib.ckpt_chain_set_gradient_tap(chain._h, None, C.c_int64(0)) == 0
+    assert lib.ckpt_chain_set_sgd(chain._h, C.c_double(-1.0)) == -6
+    assert lib.ckpt_chain_set_sgd(chain._h, C.c_double(float("nan"))) == -6
+    assert lib.ckpt_chain_set_sgd(chain._h, C.c_double(0.01)) == 0
+    assert lib.ckpt_chain_set_sgd(None, C.c_double(0.01)) == -1
+    assert lib.ckpt_chain_set_selftest(None, 1) == -1
+    assert lib.ckpt_selftest_bounded_wait(C.c_int64(0), None) in (-6, -1)                   # limit out of range (or no status word)
