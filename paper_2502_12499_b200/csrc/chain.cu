@@ -217,7 +217,10 @@ static BlockBuffers block_buffers(StepCtx& c, const Unit& u) {
     char* p = c.ws + c.ch->off_blk;
     B.z1 = p; p += m_in; B.a = p; p += m_in; B.da = p; p += m_in;
     B.z2 = p; p += m_out; B.b = p; p += m_out; B.db = p; p += m_out;
-    B.z3 = p; p += c_out; B.zp = p; p += c_out; B.t0 = p; p += c_out; B.t1 = p; p += c_out;
+    B.z3 = p; p += c_out; B.zp = p; p += c_out;
+    // the gradients with respect to z3 and zp are written over z3 and zp themselves (the batch-norm backward reads an
+    // element of z and of the incoming gradient and writes the same element; nothing reads z3 or zp afterwards)
+    B.t1 = B.z3; B.t0 = B.zp;
     B.dxs = p;
     float* st = (float*)(c.ws + c.ch->off_stats) + u.stats_off;
     B.s1 = st; B.s2 = st + 4 * u.desc.mid; B.s3 = st + 8 * u.desc.mid; B.sp = B.s3 + 4 * u.out.c;
@@ -873,7 +876,7 @@ int ckpt_chain_create(const ckpt_unit_desc* units, int64_t n, int64_t batch, int
                 // interiors and gradient temporaries of one block (see block_buffers)
                 const int64_t in_px = batch * cur.h * cur.w, out_px = batch * ho * wo;
                 const int64_t blk = 3 * align_up(in_px * mid * es, 256) + 3 * align_up(out_px * mid * es, 256) +
-                                    4 * align_up(out_px * co * es, 256) + align_up(in_px * cur.c * es, 256);
+                                    2 * align_up(out_px * co * es, 256) + align_up(in_px * cur.c * es, 256);
                 ch->blk_bytes = std::max(ch->blk_bytes, blk);
                 break;
             }
