@@ -55,7 +55,7 @@ int ckpt_conv2d_forward(const ckpt_conv_shape* s, int dtype, int impl, const voi
     if (!x || !w || !z) { set_error("null tensor"); return CKPT_E_NULL; }
     ConvGeom g = make_geom(*s);
     if (impl != 1 && tc_first_conv_supported(dtype, g)) return tc_first_conv_fwd(g, x, w, z, op_status_word(), stream);
-    if (impl != 1 && stem_conv_supported(dtype, g)) return stem_conv_fwd(g, x, w, z, scratch, scratch_bytes, op_status_word(), stream);
+    if (impl != 1 && stem_conv_supported(dtype, g)) return stem_conv_fwd(g, x, w, z, op_status_word(), stream);
     if (want_tc(impl, dtype, g, &rc)) return tc_conv_fwd(g, x, w, z, nullptr, 0, scratch, scratch_bytes, op_status_word(), stream);
     if (rc) return rc;
     return simt_conv_fwd(dtype, g, x, w, z, nullptr, 0, stream);
@@ -79,11 +79,15 @@ int ckpt_conv2d_bn_statistics(const ckpt_conv_shape* s, int dtype, const void* x
             if (fused) *fused = 1;
             return bn_statistics_from_partials((const float*)scratch, blocks, rows, g.cout, gamma, beta, stats, stream);
         }
-    } else if (stem_conv_supported(dtype, g) && scratch_bytes >= stem_conv_scratch_bytes(g)) {
-        if ((rc = stem_conv_fwd(g, x, w, z, scratch, scratch_bytes, op_status_word(), stream))) return rc;
-    } else if (tc_first_conv_supported(dtype, g)) {
+    } else if (stem_conv_supported(dtype, g) || tc_first_conv_supported(dtype, g)) {
         int blocks = 0;
-        if ((rc = tc_first_conv_fwd(g, x, w, z, op_status_word(), stream, (float*)scratch, &blocks))) return rc;
+        if (stem_conv_supported(dtype, g)) {
+            if (scratch_bytes < stem_conv_scratch_bytes(g)) { set_error("scratch too small for the convolution"); return CKPT_E_WORKSPACE; }
+            rc = stem_conv_fwd(g, x, w, z, op_status_word(), stream, (float*)scratch, &blocks);
+        } else {
+            rc = tc_first_conv_fwd(g, x, w, z, op_status_word(), stream, (float*)scratch, &blocks);
+        }
+        if (rc) return rc;
         if (blocks > 0) {
             if (fused) *fused = 1;
             return bn_statistics_from_partials((const float*)scratch, blocks, rows, g.cout, gamma, beta, stats, stream);

@@ -110,7 +110,7 @@ static int conv_forward_any(StepCtx& c, const ConvGeom& g, const void* x, const 
     if (c.ch->impl == 0 && !bias && !relu && tc_first_conv_supported(c.ch->dtype, g))
         return tc_first_conv_fwd(g, x, w, z, c.status(), c.stream);
     if (c.ch->impl == 0 && !bias && !relu && stem_conv_supported(c.ch->dtype, g))
-        return stem_conv_fwd(g, x, w, z, c.ws + c.ch->off_scr, c.ch->scr_bytes, c.status(), c.stream);
+        return stem_conv_fwd(g, x, w, z, c.status(), c.stream);
     return simt_conv_fwd(c.ch->dtype, g, x, w, z, bias, relu, c.stream);
 }
 static int conv_dgrad_any(StepCtx& c, const ConvGeom& g, const void* dz, const void* w, void* dx) {
@@ -144,9 +144,12 @@ static int conv_backward_pair(StepCtx& c, const ConvGeom& g, const void* dz, con
     int rc;
     const bool sgd = c.ch->sgd_lr != 0.f;
     if (sgd && dx && (rc = conv_dgrad_any(c, g, dz, w, dx))) return rc;
-    const bool tc_path = !(c.ch->impl == 0 && small_conv_supported(c.ch->dtype, g)) && !(c.ch->impl == 0 && stem_conv_supported(c.ch->dtype, g)) &&
-                         use_tc(c.ch, g);
-    if (sgd && tc_path) {
+    const bool stem = c.ch->impl == 0 && stem_conv_supported(c.ch->dtype, g);
+    const bool tc_path = !(c.ch->impl == 0 && small_conv_supported(c.ch->dtype, g)) && !stem && use_tc(c.ch, g);
+    if (sgd && stem) {
+        rc = stem_conv_wgrad(g, dz, x, (float*)c.grads[param], c.ws + c.ch->off_scr, c.ch->scr_bytes, c.status(), c.stream, sgd_of(c, param));
+        if (rc) return rc;
+    } else if (sgd && tc_path) {
         rc = tc_conv_wgrad(g, dz, x, (float*)c.grads[param], c.ws + c.ch->off_scr, c.ch->scr_bytes, c.status(), c.stream, sgd_of(c, param));
         if (rc) return rc;
     } else {
@@ -165,9 +168,10 @@ static int conv_with_statistics(StepCtx& c, const ConvGeom& g, const void* x, co
     const int64_t rows = (int64_t)g.n * g.ho * g.wo;
     char* scr = c.ws + c.ch->off_scr;
     int rc;
-    if (use_tc(c.ch, g) || (c.ch->impl == 0 && tc_first_conv_supported(dt, g))) {
+    if (use_tc(c.ch, g) || (c.ch->impl == 0 && (tc_first_conv_supported(dt, g) || stem_conv_supported(dt, g)))) {
         int blocks = 0;
         if (use_tc(c.ch, g)) rc = tc_conv_fwd_stats(g, x, w, z, (float*)scr, &blocks, c.status(), c.stream, c.ch->scr_bytes);
+        else if (stem_conv_supported(dt, g)) rc = stem_conv_fwd(g, x, w, z, c.status(), c.stream, (float*)scr, &blocks);
         else rc = tc_first_conv_fwd(g, x, w, z, c.status(), c.stream, (float*)scr, &blocks);
         if (rc) return rc;
         if (blocks > 0) return bn_statistics_from_partials((const float*)scr, blocks, rows, g.cout, gamma, beta, stats, c.stream);

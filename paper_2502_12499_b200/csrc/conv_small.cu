@@ -137,68 +137,6 @@ __global__ void take_paired_columns_kernel(const float* __restrict__ dwp, float*
     }
 }
 
-// Stem of the residual networks: 7x7 filter, stride 2, padding 3, 3 input channels.  xcol[output pixel][192]: filter
-// row r occupies elements 24 r .. 24 r + 20 (its 7 x 3 values, which are 21 consecutive values of input row
-// 2 oh - 3 + r), the rest is zero; forward and weight gradient become plain contractions over 192 "channels" (a 1x1
-// convolution) for the tensor cores.  One thread builds one 48-byte segment: the 21 values start at an odd element of a
-// word-aligned row, so it loads the 11 words from one element earlier and shifts each pair by 16 bits.  Pixels whose
-// window crosses the left or right border (and tensors that are not word-aligned) go element by element.
-__global__ void __launch_bounds__(256) unfold_stem7_kernel(const __nv_bfloat16* __restrict__ x, uint4* __restrict__ xcol, int n, int h,
-                                                           int wd, int ho, int wo, int aligned) {
-    const uint32_t* x32 = reinterpret_cast<const uint32_t*>(x);
-    const uint16_t* x16 = reinterpret_cast<const uint16_t*>(x);
-    const int64_t total = (int64_t)n * ho * wo * 8;
-    for (int64_t idx = (int64_t)blockIdx.x * 256 + threadIdx.x; idx < total; idx += (int64_t)gridDim.x * 256) {
-        const int r = (int)(idx & 7);
-        const int64_t p = idx >> 3;
-        const int ow = (int)(p % wo), oh = (int)((p / wo) % ho);
-        const int64_t img = p / ((int64_t)wo * ho);
-        uint32_t o[12];
-#pragma unroll
-        for (int q = 0; q < 12; ++q) o[q] = 0u;
-        const int ih = 2 * oh - 3 + r;
-        if (r < 7 && ih >= 0 && ih < h) {
-            const int iw0 = 2 * ow - 3;
-            const int64_t row_e = ((img * h + ih) * wd) * 3;            // first element of the input row
-            if (aligned && iw0 >= 1 && iw0 + 6 < wd) {
-                const uint32_t* src = x32 + (row_e + iw0 * 3 - 1) / 2;   // the word that ends with the first value
-                uint32_t w[11];
-#pragma unroll
-                for (int q = 0; q < 11; ++q) w[q] = __ldg(src + q);
-#pragma unroll
-                for (int q = 0; q < 10; ++q) o[q] = __funnelshift_r(w[q], w[q + 1], 16);
-                o[10] = w[10] >> 16;
-            } else {
-#pragma unroll
-                for (int t = 0; t < 21; ++t) {
-                    const int iw = iw0 + t / 3;
-                    const uint32_t v = (iw >= 0 && iw < wd) ? (uint32_t)x16[row_e + iw * 3 + t % 3] : 0u;
-                    o[t / 2] |= v << (16 * (t & 1));
-                }
-            }
-        }
-        uint4* dst = xcol + p * 24 + r * 3;
-        dst[0] = make_uint4(o[0], o[1], o[2], o[3]);
-        dst[1] = make_uint4(o[4], o[5], o[6], o[7]);
-        dst[2] = make_uint4(o[8], o[9], o[10], o[11]);
-    }
-}
-
-// wp[co][24 r + t] = w[co][r][t] for the 21 values t of filter row r, zeros elsewhere (192 per output channel)
-__global__ void stem_filter_rows_kernel(const __nv_bfloat16* __restrict__ w, __nv_bfloat16* __restrict__ wp, int cout) {
-    const int i = blockIdx.x * blockDim.x + threadIdx.x;
-    if (i >= cout * 192) return;
-    const int co = i / 192, r = (i % 192) / 24, t = i % 24;
-    wp[i] = (r < 7 && t < 21) ? w[(size_t)co * 147 + r * 21 + t] : __float2bfloat16_rn(0.f);
-}
-// dw[co][r][t] = dwp[co][24 r + t]
-__global__ void stem_take_rows_kernel(const float* __restrict__ dwp, float* __restrict__ dw, int cout) {
-    const int i = blockIdx.x * blockDim.x + threadIdx.x;
-    if (i >= cout * 147) return;
-    const int co = i / 147, r = (i % 147) / 21, t = i % 21;
-    dw[i] = dwp[(size_t)co * 192 + r * 24 + t];
-}
-
 }  // namespace
 
 bool small_conv_supported(int dtype, const ConvGeom& g) {
@@ -248,67 +186,6 @@ int small_conv_wgrad(const ConvGeom& g, const void* dz, const void* x, float* dw
     if (paired(g)) take_paired_columns_kernel<<<(g.cout * 27 + 255) / 256, 256, 0, st>>>(dwp, dw, g.cout, 27);
     else take_columns_kernel<<<(g.cout * 27 + 255) / 256, 256, 0, st>>>(dwp, dw, g.cout, 27);
     CKPT_LAUNCH_CHECK("first-layer wgrad column pick");
-    return CKPT_OK;
-}
-
-// ------------------------------------------------------------------------------------------------
-// 7x7 stride-2 padding-3 stem on 3 input channels: unfold, then the tensor-core 1x1 kernels.
-// ------------------------------------------------------------------------------------------------
-constexpr int kStemWidth = 192;      // 7 filter rows of 21 values, each padded to 24, plus one block of zeros: whole 64-channel blocks
-
-bool stem_conv_supported(int dtype, const ConvGeom& g) {
-    return dtype == CKPT_DTYPE_BF16 && g.cin == 3 && g.k == 7 && g.stride == 2 && g.pad == 3 && g.cout % 64 == 0;
-}
-static ConvGeom stem_unfolded_geom(const ConvGeom& g) {
-    ConvGeom u = g;
-    u.h = g.ho; u.w = g.wo; u.cin = kStemWidth; u.k = 1; u.stride = 1; u.pad = 0;
-    return u;
-}
-static int64_t stem_xcol_bytes(const ConvGeom& g) { return align_up((int64_t)g.n * g.ho * g.wo * kStemWidth * 2, 256); }
-static int64_t stem_mat_bytes(const ConvGeom& g) { return align_up((int64_t)g.cout * kStemWidth * 4, 256); }
-
-int64_t stem_conv_scratch_bytes(const ConvGeom& g) {
-    return stem_xcol_bytes(g) + stem_mat_bytes(g) + tc_conv_scratch_bytes(stem_unfolded_geom(g));
-}
-
-static int stem_unfold(const ConvGeom& g, const void* x, __nv_bfloat16* xcol, cudaStream_t st) {
-    const int64_t threads = (int64_t)g.n * g.ho * g.wo * 8;
-    const unsigned grid = (unsigned)std::max<int64_t>(1, std::min<int64_t>((threads + 255) / 256, 148 * 64));
-    const int aligned = ((uintptr_t)x % 4 == 0 && g.w % 2 == 0) ? 1 : 0;      // every input row starts on a word
-    unfold_stem7_kernel<<<grid, 256, 0, st>>>((const __nv_bfloat16*)x, (uint4*)xcol, g.n, g.h, g.w, g.ho, g.wo, aligned);
-    CKPT_LAUNCH_CHECK("stem unfold");
-    return CKPT_OK;
-}
-
-int stem_conv_fwd(const ConvGeom& g, const void* x, const void* w, void* z, void* scratch, int64_t scratch_bytes,
-                  int* device_status, void* stream) {
-    if (!scratch || scratch_bytes < stem_conv_scratch_bytes(g)) { set_error("stem conv scratch too small"); return CKPT_E_WORKSPACE; }
-    cudaStream_t st = (cudaStream_t)stream;
-    char* base = (char*)scratch;
-    __nv_bfloat16* xcol = (__nv_bfloat16*)base;
-    __nv_bfloat16* wp = (__nv_bfloat16*)(base + stem_xcol_bytes(g));
-    int rc = stem_unfold(g, x, xcol, st);
-    if (rc) return rc;
-    stem_filter_rows_kernel<<<(g.cout * kStemWidth + 255) / 256, 256, 0, st>>>((const __nv_bfloat16*)w, wp, g.cout);
-    CKPT_LAUNCH_CHECK("stem filter layout");
-    return tc_conv_fwd(stem_unfolded_geom(g), xcol, wp, z, nullptr, 0, nullptr, 0, device_status, stream);
-}
-
-int stem_conv_wgrad(const ConvGeom& g, const void* dz, const void* x, float* dw, void* scratch, int64_t scratch_bytes,
-                    int* device_status, void* stream) {
-    if (!scratch || scratch_bytes < stem_conv_scratch_bytes(g)) { set_error("stem conv scratch too small"); return CKPT_E_WORKSPACE; }
-    cudaStream_t st = (cudaStream_t)stream;
-    char* base = (char*)scratch;
-    __nv_bfloat16* xcol = (__nv_bfloat16*)base;
-    float* dwp = (float*)(base + stem_xcol_bytes(g));
-    void* tc_scratch = base + stem_xcol_bytes(g) + stem_mat_bytes(g);
-    int rc = stem_unfold(g, x, xcol, st);
-    if (rc) return rc;
-    rc = tc_conv_wgrad(stem_unfolded_geom(g), dz, xcol, dwp, tc_scratch, scratch_bytes - stem_xcol_bytes(g) - stem_mat_bytes(g),
-                       device_status, stream);
-    if (rc) return rc;
-    stem_take_rows_kernel<<<(g.cout * 147 + 255) / 256, 256, 0, st>>>(dwp, dw, g.cout);
-    CKPT_LAUNCH_CHECK("stem wgrad column pick");
     return CKPT_OK;
 }
 

@@ -1889,6 +1889,410 @@ tc_conv_first_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* _
 }
 
 // ------------------------------------------------------------------------------------------------
+// Stem of the residual networks: 3 input channels, 7x7, stride 2, padding 3.  The 21 values of a filter
+// row (7 pixels x 3 channels) are consecutive in memory, so the reduction is laid out as seven segments
+// of 24 (21 values + 3 zeros): K = 168, run as 11 MMAs of K = 16 over three 64-element swizzle atoms
+// whose last chunks stay zero.  A tile is 128 consecutive pixels of one output row: the seven input rows
+// it touches are seven contiguous segments of 261 pixels, staged in shared memory by 16-byte
+// asynchronous copies one tile ahead; thread t then picks the 21 values of each filter row of its pixel
+// (12 word loads from the word below them, 11 funnel shifts) and writes them into the operand tile in
+// the layout the other kernels get from TMA.  Columns outside the image are masked in the words, rows
+// outside it and pixels past the end of the output row are written as zeros.  The same tile serves the
+// forward kernel (K-major A operand) and the weight-gradient kernel (MN-major A operand, the pixels being
+// the reduction), which is why the atoms sit in the order 2, 0, 1: an MN-major operand of 128 rows is a
+// pair of atoms a fixed distance apart, (0, 1) and (2, 0) here.
+// ------------------------------------------------------------------------------------------------
+struct StemParams {
+    int H, W, ho, wo, c_out;
+    int chunks;                  // 128-pixel pieces of an output row
+    int m_tiles;                 // N * ho * chunks
+    long long in_bytes;
+    int slices;                  // weight gradient: persistent CTAs along the tile range
+};
+constexpr int kStemThreads = 288;
+constexpr int kStemSegBytes = 1600;                 // 261 pixels x 6 bytes, alignment slack, the word pair read past the last value
+constexpr int kStemSegChunks = kStemSegBytes / 16;
+constexpr uint32_t kStemATile = 3 * 16384;
+constexpr uint32_t kStemStage = 7 * kStemSegBytes;
+constexpr uint32_t kStemFwdSmem = 2 * kStemATile + 3 * 8192 + 16384 + 2 * kStemStage + 1024;
+constexpr uint32_t kStemWgradSmem = 2 * kStemATile + 2 * 16384 + 2 * kStemStage + 1024;
+
+struct StemTile { int img, oh, ow0; };
+__device__ __forceinline__ StemTile stem_tile(const StemParams& p, int t) {
+    StemTile s;
+    s.ow0 = (t % p.chunks) * 128; t /= p.chunks;
+    s.oh = t % p.ho;
+    s.img = t / p.ho;
+    return s;
+}
+__device__ __forceinline__ uint32_t stem_atom_offset(int atom) { return atom == 2 ? 0u : (uint32_t)(atom + 1) * 16384u; }
+// byte offset of the first value filter row r needs for the tile's first pixel (negative or past the row at the borders)
+__device__ __forceinline__ long long stem_seg_start(const StemParams& p, const StemTile& s, int r) {
+    return (((long long)s.img * p.H + (2 * s.oh - 3 + r)) * p.W + (2 * s.ow0 - 3)) * 6;
+}
+__device__ __forceinline__ void stem_stage_issue(const StemParams& p, const __nv_bfloat16* x, uint8_t* stage_buf, const StemTile& s, int t) {
+    for (int idx = t; idx < 7 * kStemSegChunks; idx += 128) {
+        const int r = idx / kStemSegChunks, ch = idx % kStemSegChunks;
+        const int ih = 2 * s.oh - 3 + r;
+        if (ih < 0 || ih >= p.H) continue;
+        const long long b = (stem_seg_start(p, s, r) & ~15LL) + ch * 16;
+        if (b >= 0 && b < p.in_bytes)
+            cp_async_16(smem_u32(stage_buf + r * kStemSegBytes + ch * 16), reinterpret_cast<const char*>(x) + b, (int)min(16LL, p.in_bytes - b));
+    }
+}
+// row t of the operand tile from the staged segments
+__device__ __forceinline__ void stem_gather_row(const StemParams& p, const StemTile& s, const uint8_t* stage_buf, uint8_t* a_tile, int t) {
+    const int ow = s.ow0 + t;
+    const bool pixel = ow < p.wo;
+    // the values [lo, hi) of a filter row's 21 lie inside the image
+    const int lo = max(0, 3 - 2 * ow) * 3, hi = min(7, p.W + 3 - 2 * ow) * 3;
+#pragma unroll
+    for (int r = 0; r < 7; ++r) {
+        uint32_t o[12];
+#pragma unroll
+        for (int q = 0; q < 12; ++q) o[q] = 0u;
+        const int ih = 2 * s.oh - 3 + r;
+        if (pixel && ih >= 0 && ih < p.H) {
+            const uint32_t a = smem_u32(stage_buf + r * kStemSegBytes) + (uint32_t)(stem_seg_start(p, s, r) & 15LL) + (uint32_t)t * 12u;
+            const uint32_t a4 = a & ~3u, sh = (a & 2u) * 8u;
+            uint32_t wv[12];
+#pragma unroll
+            for (int q = 0; q < 12; ++q) asm volatile("ld.shared.u32 %0, [%1];" : "=r"(wv[q]) : "r"(a4 + 4u * q));
+#pragma unroll
+            for (int q = 0; q < 11; ++q) o[q] = __funnelshift_r(wv[q], wv[q + 1], sh);
+            o[10] &= 0xffffu;
+            if (lo > 0 || hi < 21) {
+#pragma unroll
+                for (int q = 0; q < 11; ++q) {
+                    const uint32_t m = ((2 * q >= lo && 2 * q < hi) ? 0xffffu : 0u) | ((2 * q + 1 >= lo && 2 * q + 1 < hi) ? 0xffff0000u : 0u);
+                    o[q] &= m;
+                }
+            }
+        }
+#pragma unroll
+        for (int q = 0; q < 3; ++q) {
+            const int c = 3 * r + q;
+            *reinterpret_cast<uint4*>(a_tile + stem_atom_offset(c >> 3) + t * 128 + (((c & 7) ^ (t & 7)) * 16)) =
+                make_uint4(o[4 * q], o[4 * q + 1], o[4 * q + 2], o[4 * q + 3]);
+        }
+    }
+}
+// chunks 21-23 of every row (K = 168 .. 191) are never written by the gather: zero them once
+__device__ __forceinline__ void stem_zero_padding(uint8_t* a_tiles) {
+    for (int i = threadIdx.x; i < 2 * 128 * 3; i += blockDim.x) {
+        const int buf = i / 384, row = (i % 384) / 3, c = 21 + i % 3;
+        *reinterpret_cast<uint4*>(a_tiles + buf * kStemATile + stem_atom_offset(2) + row * 128 + (((c & 7) ^ (row & 7)) * 16)) = make_uint4(0u, 0u, 0u, 0u);
+    }
+}
+
+// Forward: persistent CTAs, two operand tiles and two 64-column accumulators.  Warps 0-3 gather, warp 4 owns tensor
+// memory and issues the MMAs, warps 5-8 round, store (one tile store per warp) and take the batch-norm sums.
+__global__ void __launch_bounds__(kStemThreads, 1)
+tc_conv_stem_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __restrict__ w,
+                    const __grid_constant__ CUtensorMap map_out, float* __restrict__ stat_partial, StemParams p, int* status) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* const smem_al = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
+    uint8_t* const a_tiles = smem_al;                       // [2][atoms 2, 0, 1][128 rows][128 bytes]
+    uint8_t* const b_tile = smem_al + 2 * kStemATile;       // [atoms 0, 1, 2][64 rows][128 bytes]
+    uint8_t* const o_tile = b_tile + 3 * 8192;
+    uint8_t* const stage = o_tile + 16384;                  // [2][7][kStemSegBytes]
+    __shared__ float stat_red[4][2][64];
+    __shared__ __align__(8) uint64_t bar_mem[8];
+    __shared__ uint32_t tmem_base_slot;
+    __shared__ int failed_flag;
+    volatile int* failed = &failed_flag;
+    const uint32_t bars = smem_u32(bar_mem);
+    const uint32_t a_full0 = bars, a_empty0 = bars + 16, acc_full0 = bars + 32, acc_empty0 = bars + 48;
+
+    const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
+    const int co0 = blockIdx.y * 64;
+    const int my_tiles = (int)blockIdx.x < p.m_tiles ? (p.m_tiles - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x : 0;
+
+    if (threadIdx.x == 0) {
+        failed_flag = 0;
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(a_full0 + 8 * b, 128); mbar_init(a_empty0 + 8 * b, 1);
+            mbar_init(acc_full0 + 8 * b, 1); mbar_init(acc_empty0 + 8 * b, 128);
+        }
+        fence_barrier_init();
+        tma_prefetch_desc(&map_out);
+    }
+    // filter tile: row = output channel, K = filter row r in columns 24 r .. 24 r + 20, zeros elsewhere
+    for (int i = threadIdx.x; i < 64 * 24; i += blockDim.x) {
+        const int co = i / 24, chunk = i % 24;
+        __align__(16) uint16_t v[8];
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+            const int k = chunk * 8 + e, r = k / 24, tt = k % 24;
+            v[e] = (r < 7 && tt < 21) ? __ldg(reinterpret_cast<const uint16_t*>(w) + (size_t)(co0 + co) * 147 + r * 21 + tt) : (uint16_t)0;
+        }
+        *reinterpret_cast<uint4*>(b_tile + (chunk >> 3) * 8192 + co * 128 + (((chunk & 7) ^ (co & 7)) * 16)) = *reinterpret_cast<const uint4*>(v);
+    }
+    stem_zero_padding(a_tiles);
+    fence_proxy_async();
+    if ((smem_u32(a_tiles) | smem_u32(b_tile)) & 1023u) {       // the swizzle pattern assumes 1024-byte aligned tiles
+        if (threadIdx.x == 0) atomicCAS(status, 0, 610);
+        return;
+    }
+    if (warp == 4) tmem_alloc(smem_u32(&tmem_base_slot), 128);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = tmem_base_slot;
+
+    if (warp < 4) {
+        const int t = threadIdx.x;
+        auto issue = [&](int j) {
+            if (j < my_tiles) stem_stage_issue(p, x, stage + (j & 1) * kStemStage, stem_tile(p, (int)blockIdx.x + j * (int)gridDim.x), t);
+            cp_async_commit();
+        };
+        issue(0);
+        bool dead = false;          // after a failed wait the thread keeps walking the barriers, without work
+        for (int j = 0; j < my_tiles; ++j) {
+            const int buf = j & 1;
+            asm volatile("bar.sync 2, 128;" ::: "memory");      // every thread has left the segments of tile j - 1
+            issue(j + 1);
+            cp_async_wait<1>();
+            asm volatile("bar.sync 2, 128;" ::: "memory");      // the segments of tile j are complete
+            if (!dead && !mbar_wait(a_empty0 + 8 * buf, ((uint32_t)(j >> 1) & 1u) ^ 1u, failed, status, 611)) dead = true;
+            if (dead) continue;
+            stem_gather_row(p, stem_tile(p, (int)blockIdx.x + j * (int)gridDim.x), stage + buf * kStemStage, a_tiles + buf * kStemATile, t);
+            fence_proxy_async();
+            mbar_arrive(a_full0 + 8 * buf);
+        }
+        cp_async_wait<0>();
+    } else if (warp == 4) {
+        if (lane == 0) {
+            const uint32_t idesc = instr_desc(128, 64, 0, 0);
+            const uint32_t b_addr = smem_u32(b_tile);
+            for (int j = 0; j < my_tiles; ++j) {
+                const int buf = j & 1;
+                if (!mbar_wait(acc_empty0 + 8 * buf, ((uint32_t)(j >> 1) & 1u) ^ 1u, failed, status, 612)) break;
+                if (!mbar_wait(a_full0 + 8 * buf, (uint32_t)(j >> 1) & 1u, failed, status, 613)) break;
+                tc_fence_after();
+                const uint32_t a_addr = smem_u32(a_tiles + buf * kStemATile);
+#pragma unroll
+                for (int kk = 0; kk < 11; ++kk)
+                    umma_bf16(tmem_base + (uint32_t)(buf * 64), smem_desc(a_addr + stem_atom_offset(kk >> 2) + (kk & 3) * 32, 0, 1024),
+                              smem_desc(b_addr + (kk >> 2) * 8192 + (kk & 3) * 32, 0, 1024), idesc, kk > 0 ? 1u : 0u);
+                umma_commit(a_empty0 + 8 * buf);
+                umma_commit(acc_full0 + 8 * buf);
+            }
+        }
+    } else {
+        // thread = accumulator lane = pixel of the tile; rounded rows go through a swizzled tile in shared memory
+        const int quarter = warp % 4;
+        const int row = quarter * 32 + lane;
+        const bool stats = stat_partial != nullptr;
+        float s_acc[2] = {0.f, 0.f}, q_acc[2] = {0.f, 0.f};
+        for (int j = 0; j < my_tiles; ++j) {
+            const int buf = j & 1;
+            if (!mbar_wait(acc_full0 + 8 * buf, (uint32_t)(j >> 1) & 1u, failed, status, 614)) break;
+            tc_fence_after();
+            if (lane == 0) tma_store_wait_read<0>();          // the store of the previous tile has left this warp's slab
+            __syncwarp();
+            const StemTile tile = stem_tile(p, (int)blockIdx.x + j * (int)gridDim.x);
+            uint8_t* const orow = o_tile + row * 128;
+#pragma unroll
+            for (int c0 = 0; c0 < 64; c0 += 32) {
+                uint32_t v[32];
+                tmem_ld32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * 64 + c0), v);
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    uint4 pk;
+                    __nv_bfloat162* h = reinterpret_cast<__nv_bfloat162*>(&pk);
+#pragma unroll
+                    for (int e = 0; e < 4; ++e)
+                        h[e] = __floats2bfloat162_rn(__uint_as_float(v[8 * q + 2 * e]), __uint_as_float(v[8 * q + 2 * e + 1]));
+                    *reinterpret_cast<uint4*>(orow + (((c0 / 8 + q) ^ (row & 7)) * 16)) = pk;
+                }
+            }
+            tc_fence_before();
+            mbar_arrive(acc_empty0 + 8 * buf);
+            fence_proxy_async();
+            __syncwarp();
+            const int first = tile.ow0 + quarter * 32;
+            const int rows_here = min(32, max(0, p.wo - first));
+            if (lane == 0 && rows_here > 0) {
+                tma_store_4d(&map_out, smem_u32(o_tile) + (uint32_t)(quarter * 4096), co0, first, tile.oh, tile.img);
+                tma_store_commit();
+            }
+            if (stats) {
+                // lane l adds up channels 2l and 2l + 1 down the rows of the warp's slab that hold pixels
+                const uint8_t* slab = o_tile + quarter * 4096;
+                for (int rr = 0; rr < rows_here; ++rr) {
+                    const uint32_t wv = *reinterpret_cast<const uint32_t*>(slab + rr * 128 + (((lane >> 2) ^ (rr & 7)) * 16) + (lane & 3) * 4);
+                    const float f0 = __uint_as_float(wv << 16), f1 = __uint_as_float(wv & 0xffff0000u);
+                    s_acc[0] += f0; q_acc[0] = fmaf(f0, f0, q_acc[0]);
+                    s_acc[1] += f1; q_acc[1] = fmaf(f1, f1, q_acc[1]);
+                }
+            }
+        }
+        if (lane == 0) tma_store_wait_all();
+        if (stats) {
+            // the four quarters of the CTA are added in a fixed order: one partial row pair per CTA
+#pragma unroll
+            for (int h = 0; h < 2; ++h) { stat_red[quarter][0][2 * lane + h] = s_acc[h]; stat_red[quarter][1][2 * lane + h] = q_acc[h]; }
+            asm volatile("bar.sync 1, 128;" ::: "memory");
+            if (quarter == 0) {
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    const int col = h * 32 + lane;
+#pragma unroll
+                    for (int k = 0; k < 2; ++k)
+                        stat_partial[((size_t)blockIdx.x * 2 + k) * p.c_out + co0 + col] =
+                            (stat_red[0][k][col] + stat_red[1][k][col]) + (stat_red[2][k][col] + stat_red[3][k][col]);
+                }
+            }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 4) {
+        __syncwarp();
+        tc_fence_after();
+        tmem_dealloc(tmem_base, 128);
+    }
+}
+
+// Weight gradient of the stem: D[(filter row, value) = 128 rows][c_out tile = 64 columns] += Xtile^T * dZtile over the
+// pixels of a tile, for the two atom pairs (0, 1) and (2, 0) of the gathered operand tile (the second half of the
+// second accumulator repeats atom 0 and is not read back).  The dz tile of the same 128 pixels arrives by TMA (pixels
+// past the end of the row are zero-filled, and the gathered rows there are zeros too).  Each CTA keeps its two
+// accumulators over all its tiles and leaves partial[slice][c_out][147]; the slices are added in a fixed order.
+__global__ void __launch_bounds__(kStemThreads, 1)
+tc_wgrad_stem_kernel(const __nv_bfloat16* __restrict__ x, const __grid_constant__ CUtensorMap map_dz, float* __restrict__ partial,
+                     StemParams p, int* status) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* const smem_al = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
+    uint8_t* const a_tiles = smem_al;                       // [2][atoms 2, 0, 1][128 pixels][128 bytes]
+    uint8_t* const dz_tiles = smem_al + 2 * kStemATile;     // [2][128 pixels][64 channels]
+    uint8_t* const stage = dz_tiles + 2 * 16384;            // [2][7][kStemSegBytes]
+    __shared__ __align__(8) uint64_t bar_mem[10];
+    __shared__ uint32_t tmem_base_slot;
+    __shared__ int failed_flag;
+    volatile int* failed = &failed_flag;
+    const uint32_t bars = smem_u32(bar_mem);
+    const uint32_t a_full0 = bars, a_empty0 = bars + 16, dz_full0 = bars + 32, dz_empty0 = bars + 48, accum_bar = bars + 64;
+
+    const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
+    const int slice = blockIdx.x, co_tile = blockIdx.y;
+    const int my_tiles = slice < p.m_tiles ? (p.m_tiles - slice + p.slices - 1) / p.slices : 0;
+
+    if (threadIdx.x == 0) {
+        failed_flag = 0;
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(a_full0 + 8 * b, 128); mbar_init(a_empty0 + 8 * b, 1);
+            mbar_init(dz_full0 + 8 * b, 1); mbar_init(dz_empty0 + 8 * b, 1);
+        }
+        mbar_init(accum_bar, 1);
+        fence_barrier_init();
+        tma_prefetch_desc(&map_dz);
+    }
+    stem_zero_padding(a_tiles);
+    fence_proxy_async();
+    if ((smem_u32(a_tiles) | smem_u32(dz_tiles)) & 1023u) {
+        if (threadIdx.x == 0) atomicCAS(status, 0, 620);
+        return;
+    }
+    if (warp == 4) tmem_alloc(smem_u32(&tmem_base_slot), 128);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = tmem_base_slot;
+
+    if (warp < 4) {
+        const int t = threadIdx.x;
+        bool dead = false;
+        auto issue = [&](int j) {
+            if (j < my_tiles) {
+                const StemTile tile = stem_tile(p, slice + j * p.slices);
+                stem_stage_issue(p, x, stage + (j & 1) * kStemStage, tile, t);
+                if (t == 0 && !dead) {
+                    // the dz tile of the same pixels, one tile ahead like the segments
+                    if (mbar_wait(dz_empty0 + 8 * (j & 1), ((uint32_t)(j >> 1) & 1u) ^ 1u, failed, status, 621)) {
+                        mbar_expect_tx(dz_full0 + 8 * (j & 1), 16384u);
+                        tma_load_4d(smem_u32(dz_tiles + (j & 1) * 16384), &map_dz, dz_full0 + 8 * (j & 1), co_tile * 64, tile.ow0, tile.oh, tile.img);
+                    }
+                }
+            }
+            cp_async_commit();
+        };
+        issue(0);
+        for (int j = 0; j < my_tiles; ++j) {
+            const int buf = j & 1;
+            asm volatile("bar.sync 2, 128;" ::: "memory");      // every thread has left the segments of tile j - 1
+            issue(j + 1);
+            cp_async_wait<1>();
+            asm volatile("bar.sync 2, 128;" ::: "memory");      // the segments of tile j are complete
+            if (!dead && !mbar_wait(a_empty0 + 8 * buf, ((uint32_t)(j >> 1) & 1u) ^ 1u, failed, status, 622)) dead = true;
+            if (dead) continue;
+            stem_gather_row(p, stem_tile(p, slice + j * p.slices), stage + buf * kStemStage, a_tiles + buf * kStemATile, t);
+            fence_proxy_async();
+            mbar_arrive(a_full0 + 8 * buf);
+        }
+        cp_async_wait<0>();
+        // copies that were issued but never consumed after a failure get a bounded time to land
+        if (*failed && t == 0)
+            for (int b = 0; b < 2; ++b) mbar_drain(dz_full0 + 8 * b, 0);
+    } else if (warp == 4) {
+        if (lane == 0) {
+            const uint32_t idesc = instr_desc(128, 64, 1, 1);
+            bool ok = true;
+            for (int j = 0; j < my_tiles && ok; ++j) {
+                const int buf = j & 1;
+                const uint32_t phase = (uint32_t)(j >> 1) & 1u;
+                if (!mbar_wait(a_full0 + 8 * buf, phase, failed, status, 623)) { ok = false; break; }
+                if (!mbar_wait(dz_full0 + 8 * buf, phase, failed, status, 624)) { ok = false; break; }
+                tc_fence_after();
+                const uint32_t a_addr = smem_u32(a_tiles + buf * kStemATile);
+                const uint32_t dz_addr = smem_u32(dz_tiles + buf * 16384);
+#pragma unroll
+                for (int kk = 0; kk < 8; ++kk) {            // 16 pixels per MMA
+                    const uint64_t bd = smem_desc(dz_addr + kk * 2048, 8192, 1024);
+                    umma_bf16(tmem_base, smem_desc(a_addr + stem_atom_offset(0) + kk * 2048, 16384, 1024), bd, idesc, (j > 0 || kk > 0) ? 1u : 0u);
+                    umma_bf16(tmem_base + 64u, smem_desc(a_addr + stem_atom_offset(2) + kk * 2048, 16384, 1024), bd, idesc, (j > 0 || kk > 0) ? 1u : 0u);
+                }
+                umma_commit(a_empty0 + 8 * buf);
+                umma_commit(dz_empty0 + 8 * buf);
+            }
+            if (ok) umma_commit(accum_bar);
+        }
+    } else {
+        const int quarter = warp % 4;
+        const int row = quarter * 32 + lane;
+        float* const base = partial + ((size_t)slice * p.c_out + (size_t)co_tile * 64) * 147;
+        if (my_tiles > 0 && mbar_wait(accum_bar, 0, failed, status, 625)) {
+            tc_fence_after();
+#pragma unroll
+            for (int half = 0; half < 2; ++half) {
+                const int k = half * 128 + row, r = k / 24, tt = k % 24;
+                const bool valid = (half == 0 || row < 64) && r < 7 && tt < 21;
+                float* dst = base + r * 21 + tt;
+#pragma unroll
+                for (int c0 = 0; c0 < 64; c0 += 32) {
+                    uint32_t v[32];
+                    tmem_ld32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(half * 64 + c0), v);
+                    if (valid) {
+#pragma unroll
+                        for (int e = 0; e < 32; ++e) dst[(size_t)(c0 + e) * 147] = __uint_as_float(v[e]);
+                    }
+                }
+            }
+        } else if (my_tiles == 0) {
+            for (int i = threadIdx.x - 160; i < 64 * 147; i += 128) base[i] = 0.f;
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 4) {
+        __syncwarp();
+        tc_fence_after();
+        tmem_dealloc(tmem_base, 128);
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
 // Fully connected forward for small batches: out[b][co] = sum_k x[b][k] * W[co][k].  With the batch on M a
 // tile would be mostly padding and every CTA would re-read the activations; here the matrix is the M
 // operand (128 output features x 64 inputs per stage, each element fetched once from HBM), the batch is N,
@@ -2789,6 +3193,97 @@ int tc_first_conv_fwd(const ConvGeom& g, const void* x, const void* w, void* z, 
     tc_conv_first_kernel<<<grid, kFirstThreads, kFirstSmem, (cudaStream_t)stream>>>((const __nv_bfloat16*)x, (const __nv_bfloat16*)w,
                                                                                    map_out, partial, p, device_status);
     CKPT_LAUNCH_CHECK_NAMED("tc_conv_first_kernel", "first-layer conv forward (tensor cores)");
+    return CKPT_OK;
+}
+
+// ------------------------------------------------------------------------------------------------
+// 7x7 stride-2 padding-3 stem on 3 input channels
+// ------------------------------------------------------------------------------------------------
+bool stem_conv_supported(int dtype, const ConvGeom& g) {
+    return dtype == CKPT_DTYPE_BF16 && g.cin == 3 && g.k == 7 && g.stride == 2 && g.pad == 3 && g.cout % 64 == 0;
+}
+static int sm_count() {
+    int sms = 148, dev = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    return sms;
+}
+static StemParams stem_params(const ConvGeom& g) {
+    StemParams p;
+    p.H = g.h; p.W = g.w; p.ho = g.ho; p.wo = g.wo; p.c_out = g.cout;
+    p.chunks = (g.wo + 127) / 128;
+    p.m_tiles = (int)std::min<int64_t>((int64_t)g.n * g.ho * p.chunks, INT32_MAX);
+    p.in_bytes = (long long)g.n * g.h * g.w * 6;
+    p.slices = 1;
+    return p;
+}
+// The staged segments are copied in 16-byte pieces and tiles are counted in 32 bits; anything else takes the CUDA cores.
+static bool stem_direct(const ConvGeom& g, const void* x) {
+    return (reinterpret_cast<uintptr_t>(x) & 15u) == 0 && (int64_t)g.n * g.ho * ((g.wo + 127) / 128) < (1LL << 30);
+}
+static int stem_wgrad_slices(const ConvGeom& g) {
+    const StemParams p = stem_params(g);
+    return std::max(1, std::min(p.m_tiles, sm_count() / std::max(1, g.cout / 64)));
+}
+int64_t stem_conv_scratch_bytes(const ConvGeom& g) {
+    const int64_t partial = (int64_t)stem_wgrad_slices(g) * g.cout * 147 * 4;
+    const int64_t stat = (int64_t)sm_count() * 2 * g.cout * 4;
+    return align_up(std::max(std::max(partial, stat), simt_wgrad_scratch_bytes(g)), 256);
+}
+
+// partial / blocks: null, or where the kernel leaves the batch-norm partial sums of its output
+// ([*blocks][sum | sum of squares][c_out] floats, one row pair per CTA).
+int stem_conv_fwd(const ConvGeom& g, const void* x, const void* w, void* z, int* device_status, void* stream, float* partial, int* blocks) {
+    if (!stem_conv_supported(CKPT_DTYPE_BF16, g)) { set_error("stem kernel: unsupported shape"); return CKPT_E_UNSUPPORTED; }
+    if (!device_status) { set_error("device status word missing"); return CKPT_E_NULL; }
+    if (blocks) *blocks = 0;
+    if (!stem_direct(g, x)) return simt_conv_fwd(CKPT_DTYPE_BF16, g, x, w, z, nullptr, 0, stream);
+    const StemParams p = stem_params(g);
+    CUtensorMap map_out;
+    int rc = make_act_map(&map_out, z, g.n, g.ho, g.wo, g.cout, 32, 1, 1);
+    if (rc) return rc;
+    static bool attr_set = false;
+    if (!attr_set) {
+        cudaError_t e = cudaFuncSetAttribute(tc_conv_stem_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kStemFwdSmem);
+        if (e != cudaSuccess) return cuda_fail(e, "shared-memory opt-in of the stem kernel");
+        attr_set = true;
+    }
+    const int co_tiles = g.cout / 64;
+    dim3 grid((unsigned)std::min(p.m_tiles, std::max(1, sm_count() / co_tiles)), (unsigned)co_tiles);
+    if (blocks) *blocks = partial ? (int)grid.x : 0;
+    tc_conv_stem_kernel<<<grid, kStemThreads, kStemFwdSmem, (cudaStream_t)stream>>>((const __nv_bfloat16*)x, (const __nv_bfloat16*)w,
+                                                                                  map_out, partial, p, device_status);
+    CKPT_LAUNCH_CHECK_NAMED("tc_conv_stem_kernel", "stem conv forward (tensor cores)");
+    return CKPT_OK;
+}
+
+int stem_conv_wgrad(const ConvGeom& g, const void* dz, const void* x, float* dw, void* scratch, int64_t scratch_bytes,
+                    int* device_status, void* stream, const SgdUpdate& upd) {
+    if (!stem_conv_supported(CKPT_DTYPE_BF16, g)) { set_error("stem kernel: unsupported shape"); return CKPT_E_UNSUPPORTED; }
+    if (!device_status) { set_error("device status word missing"); return CKPT_E_NULL; }
+    if (!scratch || scratch_bytes < stem_conv_scratch_bytes(g)) { set_error("stem wgrad scratch too small"); return CKPT_E_WORKSPACE; }
+    cudaStream_t st = (cudaStream_t)stream;
+    if (!stem_direct(g, x)) {
+        int rc = simt_conv_wgrad(CKPT_DTYPE_BF16, g, dz, x, dw, scratch, scratch_bytes, stream);
+        if (rc == CKPT_OK && upd.w) rc = sgd_update(upd, dw, (int64_t)g.cout * 147, stream);
+        return rc;
+    }
+    StemParams p = stem_params(g);
+    p.slices = stem_wgrad_slices(g);
+    CUtensorMap map_dz;
+    int rc = make_act_map(&map_dz, dz, g.n, g.ho, g.wo, g.cout, 128, 1, 1);
+    if (rc) return rc;
+    static bool attr_set = false;
+    if (!attr_set) {
+        cudaError_t e = cudaFuncSetAttribute(tc_wgrad_stem_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kStemWgradSmem);
+        if (e != cudaSuccess) return cuda_fail(e, "shared-memory opt-in of the stem wgrad kernel");
+        attr_set = true;
+    }
+    dim3 grid((unsigned)p.slices, (unsigned)(g.cout / 64));
+    tc_wgrad_stem_kernel<<<grid, kStemThreads, kStemWgradSmem, st>>>((const __nv_bfloat16*)x, map_dz, (float*)scratch, p, device_status);
+    CKPT_LAUNCH_CHECK_NAMED("tc_wgrad_stem_kernel", "stem conv wgrad (tensor cores)");
+    launch_slice_sum((const float*)scratch, dw, (int64_t)g.cout * 147, p.slices, st, upd);
+    CKPT_LAUNCH_CHECK("stem wgrad slice sum");
     return CKPT_OK;
 }
 

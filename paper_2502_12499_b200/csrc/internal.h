@@ -97,14 +97,16 @@ int small_conv_fwd(const ConvGeom& g, const void* x, const void* w, void* z, voi
 int small_conv_wgrad(const ConvGeom& g, const void* dz, const void* x, float* dw, void* scratch,
                      int64_t scratch_bytes, int* device_status, void* stream);
 
-// First layer on the tensor cores (operand tiles gathered by threads, K = 27 padded to 32).
-// 7x7 stride-2 stem on 3 input channels: unfolded input + tensor-core 1x1 kernels
+// 7x7 stride-2 padding-3 stem on 3 input channels (bf16): operand tiles gathered by threads from staged input rows,
+// forward with the batch-norm partial sums of its output (partial / blocks as for the first layer), weight gradient
+// with an optional fused parameter update.  Unaligned inputs take the CUDA-core kernels.
 bool stem_conv_supported(int dtype, const ConvGeom& g);
 int64_t stem_conv_scratch_bytes(const ConvGeom& g);
-int stem_conv_fwd(const ConvGeom& g, const void* x, const void* w, void* z, void* scratch, int64_t scratch_bytes,
-                  int* device_status, void* stream);
+int stem_conv_fwd(const ConvGeom& g, const void* x, const void* w, void* z, int* device_status, void* stream,
+                  float* partial = nullptr, int* blocks = nullptr);
 int stem_conv_wgrad(const ConvGeom& g, const void* dz, const void* x, float* dw, void* scratch, int64_t scratch_bytes,
-                    int* device_status, void* stream);
+                    int* device_status, void* stream, const SgdUpdate& upd = SgdUpdate());
+// First layer on the tensor cores (operand tiles gathered by threads, K = 27 padded to 32).
 bool tc_first_conv_supported(int dtype, const ConvGeom& g);
 int tc_first_conv_fwd(const ConvGeom& g, const void* x, const void* w, void* z, int* device_status, void* stream,
                       float* partial = nullptr, int* blocks = nullptr);

@@ -115,11 +115,11 @@ def test_config2_vgg16_chain():
 
 
 def test_config3_resnet50_chain():
-    """The ResNet-50 chain unchanged at batch 16: stem through its unfolded input, 3x3 stride-2 max-pool, all 16
+    """The ResNet-50 chain unchanged at batch 16: stem on its own gather kernels, 3x3 stride-2 max-pool, all 16
     bottleneck blocks (projection, stride 2, identity), average pool, classifier."""
     spec = dict(wl.config(3), batch=16)
     params, x, labels, step = run_case(spec)
-    assert_tensor_core_dispatch(step, ["stem unfold", "tc_conv_t_kernel", "tc_conv_fwd_kernel", "tc_conv_c64_kernel",
+    assert_tensor_core_dispatch(step, ["tc_conv_stem_kernel", "tc_wgrad_stem_kernel", "tc_conv_t_kernel", "tc_conv_fwd_kernel", "tc_conv_c64_kernel",
                                        "tc_conv_wgrad_kernel", "tc_wgrad_rows_kernel", "residual join", "gradient join",
                                        "max-pool backward from arg-max"])
     assert_units_match_locally(step, params, labels)

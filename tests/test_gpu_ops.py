@@ -174,10 +174,12 @@ def test_first_layer_kernels(n, h, w, cout):
     assert not torch.isnan(z.float()).any()
 
 
-@pytest.mark.parametrize("n,h,w,cout", [(2, 23, 19, 64), (3, 64, 64, 64), (1, 224, 224, 64), (2, 30, 37, 128)])
+@pytest.mark.parametrize("n,h,w,cout", [(2, 23, 19, 64), (3, 64, 64, 64), (1, 224, 224, 64), (2, 30, 37, 128), (1, 7, 520, 64),
+                                        (40, 32, 32, 64)])
 def test_stem_kernels(n, h, w, cout):
-    """7x7 stride-2 padding-3 convolution on 3 input channels, bf16, automatic kernel choice: unfolded input and
-    the tensor-core 1x1 kernels for forward and wgrad, against the oracle and the CUDA-core kernels."""
+    """7x7 stride-2 padding-3 convolution on 3 input channels, bf16, automatic kernel choice: the stem kernels that
+    gather their operand tiles from staged input rows (forward and wgrad), against the oracle and the CUDA-core
+    kernels.  Odd widths (rows that start on an odd element), rows of several 128-pixel pieces, more tiles than CTAs."""
     import torch
     dtype = ck.DTYPE_BF16
     rng = np.random.default_rng(n * h + w + cout)
@@ -190,15 +192,22 @@ def test_stem_kernels(n, h, w, cout):
     xd, wd, dzd = to_dev(x, dtype), to_dev(wt, dtype), to_dev(dz, dtype)
     scratch = torch.empty(max(ck.conv2d_scratch_bytes(shape, dtype), 256), dtype=torch.uint8, device="cuda")
     outs = []
-    for rep in range(2):
-        z = torch.full(z_ref.shape, float("nan"), device="cuda").to(xd.dtype)
-        dw = torch.full(wt.shape, float("nan"), device="cuda", dtype=torch.float32)
-        scratch.fill_(0xFF)
-        ck.conv2d_forward(shape, dtype, 0, xd, wd, z, scratch)
-        scratch.fill_(0xFF)
-        ck.conv2d_wgrad(shape, dtype, 0, dzd, xd, dw, scratch)
-        torch.cuda.synchronize()
-        outs.append((z, dw))
+    ck.launch_log(True)
+    try:
+        for rep in range(2):
+            z = torch.full(z_ref.shape, float("nan"), device="cuda").to(xd.dtype)
+            dw = torch.full(wt.shape, float("nan"), device="cuda", dtype=torch.float32)
+            scratch.fill_(0xFF)
+            ck.conv2d_forward(shape, dtype, 0, xd, wd, z, scratch)
+            scratch.fill_(0xFF)
+            ck.conv2d_wgrad(shape, dtype, 0, dzd, xd, dw, scratch)
+            torch.cuda.synchronize()
+            outs.append((z, dw))
+    finally:
+        kernels = ck.launch_log_read()
+        ck.launch_log(False)
+    assert kernels.get("tc_conv_stem_kernel") == 2 and kernels.get("tc_wgrad_stem_kernel") == 2, kernels
+    assert ck.op_status() == 0
     z, dw = outs[0]
     assert max_rel_err(to_host(z), z_ref) <= TIGHT[dtype]
     assert max_rel_err(to_host(dw), dw_ref) <= 2e-5
@@ -221,23 +230,26 @@ def test_stem_kernels(n, h, w, cout):
     ((3, 21, 18, 3, 64, 3, 1), True),         # first-layer kernel, ragged last tile
     ((9, 96, 80, 3, 128, 3, 1), True),        # first-layer kernel, several tiles per CTA, two channel blocks
     ((2, 9, 9, 16, 24, 3, 1), False),         # CUDA-core kernel + separate statistics kernel
+    ((3, 50, 46, 3, 64, 7, 3, 2), True),      # stem kernel: several tiles per CTA, short output rows
+    ((2, 300, 290, 3, 128, 7, 3, 2), True),   # stem kernel: output rows of two 128-pixel pieces, two channel blocks
 ])
 def test_conv_bn_statistics(case, expect_fused):
     """Convolution + batch statistics of its stored output (gathered in the epilogue of the persistent
     tensor-core kernels) against the oracle's convolution, bf16 rounding and batch norm."""
     import torch
     dtype = ck.DTYPE_BF16
-    n, h, w, cin, cout, k, pad = case
+    n, h, w, cin, cout, k, pad = case[:7]
+    stride = case[7] if len(case) > 7 else 1
     rng = np.random.default_rng(sum(case))
     x = rounded(rng.standard_normal((n, h, w, cin)) + 0.3, dtype)
     wt = rounded(rng.standard_normal((cout, k, k, cin)) / np.sqrt(k * k * cin), dtype)
     gamma = rng.uniform(0.5, 1.5, cout).astype(np.float32)
     beta = (rng.standard_normal(cout) * 0.3).astype(np.float32)
-    z_ref = no.round_bf16(no.conv2d_fwd(x.astype(np.float64), wt.astype(np.float64), 1, pad))
+    z_ref = no.round_bf16(no.conv2d_fwd(x.astype(np.float64), wt.astype(np.float64), stride, pad))
     y_ref, (xhat, inv_std) = no.bn_fwd(z_ref, gamma.astype(np.float64), beta.astype(np.float64))
     mean_ref = z_ref.mean(axis=(0, 1, 2))
-    shape = ck.ConvShape(n, h, w, cin, cout, k, 1, pad)
-    rows = n * h * w
+    shape = ck.ConvShape(n, h, w, cin, cout, k, stride, pad)
+    rows = int(np.prod(z_ref.shape[:3]))
     xd, wd = to_dev(x, dtype), to_dev(wt, dtype)
     gd, bd = torch.from_numpy(gamma).cuda(), torch.from_numpy(beta).cuda()
     scratch = torch.empty(max(ck.conv2d_scratch_bytes(shape, dtype), ck.bn_scratch_bytes(rows, cout)), dtype=torch.uint8, device="cuda")
