@@ -1909,13 +1909,15 @@ struct StemParams {
     long long in_bytes;
     int slices;                  // weight gradient: persistent CTAs along the tile range
 };
-constexpr int kStemThreads = 288;
+constexpr int kStemGather = 256;                    // gather threads: two per operand row (filter rows 0-3 and 4-6)
+constexpr int kStemFwdThreads = kStemGather + 64 + 256;     // + MMA warp, copy warp, eight epilogue warps
+constexpr int kStemWgradThreads = kStemGather + 64 + 128;
+constexpr int kStemStages = 4;                      // staged tiles in flight
 constexpr int kStemSegBytes = 1600;                 // 261 pixels x 6 bytes, alignment slack, the word pair read past the last value
-constexpr int kStemSegChunks = kStemSegBytes / 16;
 constexpr uint32_t kStemATile = 3 * 16384;
 constexpr uint32_t kStemStage = 7 * kStemSegBytes;
-constexpr uint32_t kStemFwdSmem = 2 * kStemATile + 3 * 8192 + 16384 + 2 * kStemStage + 1024;
-constexpr uint32_t kStemWgradSmem = 2 * kStemATile + 2 * 16384 + 2 * kStemStage + 1024;
+constexpr uint32_t kStemFwdSmem = 2 * kStemATile + 3 * 8192 + 2 * 16384 + kStemStages * kStemStage + 1024;
+constexpr uint32_t kStemWgradSmem = 2 * kStemATile + kStemStages * 16384 + kStemStages * kStemStage + 1024;
 
 struct StemTile { int img, oh, ow0; };
 __device__ __forceinline__ StemTile stem_tile(const StemParams& p, int t) {
@@ -1926,40 +1928,72 @@ __device__ __forceinline__ StemTile stem_tile(const StemParams& p, int t) {
     return s;
 }
 __device__ __forceinline__ uint32_t stem_atom_offset(int atom) { return atom == 2 ? 0u : (uint32_t)(atom + 1) * 16384u; }
-// byte offset of the first value filter row r needs for the tile's first pixel (negative or past the row at the borders)
-__device__ __forceinline__ long long stem_seg_start(const StemParams& p, const StemTile& s, int r) {
-    return (((long long)s.img * p.H + (2 * s.oh - 3 + r)) * p.W + (2 * s.ow0 - 3)) * 6;
+// byte offset of the first value filter row 0 needs for the tile's first pixel (negative or past the row at the borders);
+// filter row r starts W * 6 bytes per row further
+__device__ __forceinline__ long long stem_seg_start(const StemParams& p, const StemTile& s) {
+    return (((long long)s.img * p.H + (2 * s.oh - 3)) * p.W + (2 * s.ow0 - 3)) * 6;
 }
-__device__ __forceinline__ void stem_stage_issue(const StemParams& p, const __nv_bfloat16* x, uint8_t* stage_buf, const StemTile& s, int t) {
-    for (int idx = t; idx < 7 * kStemSegChunks; idx += 128) {
-        const int r = idx / kStemSegChunks, ch = idx % kStemSegChunks;
-        const int ih = 2 * s.oh - 3 + r;
-        if (ih < 0 || ih >= p.H) continue;
-        const long long b = (stem_seg_start(p, s, r) & ~15LL) + ch * 16;
-        if (b >= 0 && b < p.in_bytes)
-            cp_async_16(smem_u32(stage_buf + r * kStemSegBytes + ch * 16), reinterpret_cast<const char*>(x) + b, (int)min(16LL, p.in_bytes - b));
+__device__ __forceinline__ void bulk_copy_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+// The seven segments of a tile, one bulk copy each (lane r of the copy warp takes filter row r); the barrier gets the
+// warp's one arrival with the byte count.  A segment starts at the 16-byte boundary below its first value and is cut
+// at the ends of the tensor; when the tensor does not end on a 16-byte boundary its last bytes are copied by the lane.
+// Sixteen-byte cp.async copies from the gather threads kept a few hundred small requests in flight per SM and ran a
+// tile in 4100 clocks, at the latency of the memory system.
+__device__ __forceinline__ void stem_stage_tile(const StemParams& p, const __nv_bfloat16* x, uint8_t* stage_buf, const StemTile& s, uint32_t bar, int lane) {
+    const long long whole = p.in_bytes & ~15LL;
+    const int ih = 2 * s.oh - 3 + lane;
+    const long long b0 = (stem_seg_start(p, s) + (long long)lane * (p.W * 6)) & ~15LL;
+    long long lo = 0, hi = 0;
+    if (lane < 7 && ih >= 0 && ih < p.H) {
+        lo = max(b0, 0LL);
+        hi = min(b0 + kStemSegBytes, whole);
+        if (hi < lo) hi = lo;
+        const long long tail_end = min(b0 + (long long)kStemSegBytes, p.in_bytes);
+        for (long long b = max(whole, lo); b < tail_end; ++b)
+            stage_buf[lane * kStemSegBytes + (int)(b - b0)] = reinterpret_cast<const uint8_t*>(x)[b];
     }
+    const uint32_t bytes = (uint32_t)(hi - lo);
+    const uint32_t total = __reduce_add_sync(0xffffffffu, bytes);
+    if (lane == 0) mbar_expect_tx(bar, total);
+    __syncwarp();
+    if (bytes) bulk_copy_g2s(smem_u32(stage_buf + lane * kStemSegBytes) + (uint32_t)(lo - b0), reinterpret_cast<const char*>(x) + lo, bytes, bar);
 }
-// row t of the operand tile from the staged segments
-__device__ __forceinline__ void stem_gather_row(const StemParams& p, const StemTile& s, const uint8_t* stage_buf, uint8_t* a_tile, int t) {
+// Filter rows R0 .. R0 + RN - 1 of row t of the operand tile, from the staged segments: every load first (they are
+// independent), then the shifts, the border masks and the stores.
+template <int R0, int RN>
+__device__ __forceinline__ void stem_gather_rows(const StemParams& p, const StemTile& s, const uint8_t* stage_buf, uint8_t* a_tile, int t) {
     const int ow = s.ow0 + t;
     const bool pixel = ow < p.wo;
     // the values [lo, hi) of a filter row's 21 lie inside the image
     const int lo = max(0, 3 - 2 * ow) * 3, hi = min(7, p.W + 3 - 2 * ow) * 3;
+    const long long start0 = stem_seg_start(p, s);
+    const int row_bytes = p.W * 6;
+    uint32_t wv[RN][12], sh[RN];
+    bool live[RN];
 #pragma unroll
-    for (int r = 0; r < 7; ++r) {
+    for (int i = 0; i < RN; ++i) {
+        const int r = R0 + i, ih = 2 * s.oh - 3 + r;
+        live[i] = pixel && ih >= 0 && ih < p.H;
+        const uint32_t a = smem_u32(stage_buf + r * kStemSegBytes) + (uint32_t)((start0 + (long long)r * row_bytes) & 15LL) + (uint32_t)t * 12u;
+        const uint32_t a4 = a & ~3u;
+        sh[i] = (a & 2u) * 8u;
+        if (live[i]) {
+#pragma unroll
+            for (int q = 0; q < 12; ++q) asm volatile("ld.shared.u32 %0, [%1];" : "=r"(wv[i][q]) : "r"(a4 + 4u * q));
+        }
+    }
+#pragma unroll
+    for (int i = 0; i < RN; ++i) {
+        const int r = R0 + i;
         uint32_t o[12];
 #pragma unroll
         for (int q = 0; q < 12; ++q) o[q] = 0u;
-        const int ih = 2 * s.oh - 3 + r;
-        if (pixel && ih >= 0 && ih < p.H) {
-            const uint32_t a = smem_u32(stage_buf + r * kStemSegBytes) + (uint32_t)(stem_seg_start(p, s, r) & 15LL) + (uint32_t)t * 12u;
-            const uint32_t a4 = a & ~3u, sh = (a & 2u) * 8u;
-            uint32_t wv[12];
+        if (live[i]) {
 #pragma unroll
-            for (int q = 0; q < 12; ++q) asm volatile("ld.shared.u32 %0, [%1];" : "=r"(wv[q]) : "r"(a4 + 4u * q));
-#pragma unroll
-            for (int q = 0; q < 11; ++q) o[q] = __funnelshift_r(wv[q], wv[q + 1], sh);
+            for (int q = 0; q < 11; ++q) o[q] = __funnelshift_r(wv[i][q], wv[i][q + 1], sh[i]);
             o[10] &= 0xffffu;
             if (lo > 0 || hi < 21) {
 #pragma unroll
@@ -1984,25 +2018,48 @@ __device__ __forceinline__ void stem_zero_padding(uint8_t* a_tiles) {
         *reinterpret_cast<uint4*>(a_tiles + buf * kStemATile + stem_atom_offset(2) + row * 128 + (((c & 7) ^ (row & 7)) * 16)) = make_uint4(0u, 0u, 0u, 0u);
     }
 }
+// The gather role of both kernels: tile j is built from stage j % kStemStages into operand tile j % 2.
+__device__ __forceinline__ void stem_gather_role(const StemParams& p, const uint8_t* stage, uint8_t* a_tiles, int first_tile, int tile_step,
+                                                 int my_tiles, uint32_t seg_full0, uint32_t seg_empty0, uint32_t a_full0, uint32_t a_empty0,
+                                                 volatile int* failed, int* status, int code) {
+    const int tid = threadIdx.x, t = tid & 127;
+    for (int j = 0; j < my_tiles; ++j) {
+        const int buf = j & 1, st = j % kStemStages;
+        if (!mbar_wait(seg_full0 + 8 * st, (uint32_t)(j / kStemStages) & 1u, failed, status, code)) break;
+        if (!mbar_wait(a_empty0 + 8 * buf, ((uint32_t)(j >> 1) & 1u) ^ 1u, failed, status, code + 1)) break;
+        const StemTile tile = stem_tile(p, first_tile + j * tile_step);
+        const uint8_t* seg = stage + st * kStemStage;
+        uint8_t* a_tile = a_tiles + buf * kStemATile;
+        if (tid < 128) { stem_gather_rows<0, 2>(p, tile, seg, a_tile, t); stem_gather_rows<2, 2>(p, tile, seg, a_tile, t); }
+        else { stem_gather_rows<4, 2>(p, tile, seg, a_tile, t); stem_gather_rows<6, 1>(p, tile, seg, a_tile, t); }
+        fence_proxy_async();
+        mbar_arrive(a_full0 + 8 * buf);
+        mbar_arrive(seg_empty0 + 8 * st);
+    }
+}
 
-// Forward: persistent CTAs, two operand tiles and two 64-column accumulators.  Warps 0-3 gather, warp 4 owns tensor
-// memory and issues the MMAs, warps 5-8 round, store (one tile store per warp) and take the batch-norm sums.
-__global__ void __launch_bounds__(kStemThreads, 1)
+// Forward: persistent CTAs, a ring of staged tiles, two operand tiles and two 64-column accumulators.  Warps 0-7
+// gather, warp 8 owns tensor memory and issues the MMAs, warp 9 copies the segments, warps 10-13 and 14-17 take the
+// even and the odd tiles' accumulators: round, store (one tile store per warp) and take the batch-norm sums.  Every
+// role runs at instruction latency, hence the many warps: four epilogue warps needed 1600 clocks per tile against
+// 1000 of MMAs.
+__global__ void __launch_bounds__(kStemFwdThreads, 1)
 tc_conv_stem_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __restrict__ w,
                     const __grid_constant__ CUtensorMap map_out, float* __restrict__ stat_partial, StemParams p, int* status) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* const smem_al = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
     uint8_t* const a_tiles = smem_al;                       // [2][atoms 2, 0, 1][128 rows][128 bytes]
     uint8_t* const b_tile = smem_al + 2 * kStemATile;       // [atoms 0, 1, 2][64 rows][128 bytes]
-    uint8_t* const o_tile = b_tile + 3 * 8192;
-    uint8_t* const stage = o_tile + 16384;                  // [2][7][kStemSegBytes]
-    __shared__ float stat_red[4][2][64];
-    __shared__ __align__(8) uint64_t bar_mem[8];
+    uint8_t* const o_tiles = b_tile + 3 * 8192;             // [2][128 rows][128 bytes]
+    uint8_t* const stage = o_tiles + 2 * 16384;             // [kStemStages][7][kStemSegBytes]
+    __shared__ float stat_red[8][2][64];
+    __shared__ __align__(8) uint64_t bar_mem[8 + 2 * kStemStages];
     __shared__ uint32_t tmem_base_slot;
     __shared__ int failed_flag;
     volatile int* failed = &failed_flag;
     const uint32_t bars = smem_u32(bar_mem);
     const uint32_t a_full0 = bars, a_empty0 = bars + 16, acc_full0 = bars + 32, acc_empty0 = bars + 48;
+    const uint32_t seg_full0 = bars + 64, seg_empty0 = seg_full0 + 8 * kStemStages;
 
     const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
     const int co0 = blockIdx.y * 64;
@@ -2011,9 +2068,10 @@ tc_conv_stem_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __
     if (threadIdx.x == 0) {
         failed_flag = 0;
         for (int b = 0; b < 2; ++b) {
-            mbar_init(a_full0 + 8 * b, 128); mbar_init(a_empty0 + 8 * b, 1);
+            mbar_init(a_full0 + 8 * b, kStemGather); mbar_init(a_empty0 + 8 * b, 1);
             mbar_init(acc_full0 + 8 * b, 1); mbar_init(acc_empty0 + 8 * b, 128);
         }
+        for (int b = 0; b < kStemStages; ++b) { mbar_init(seg_full0 + 8 * b, 1); mbar_init(seg_empty0 + 8 * b, kStemGather); }
         fence_barrier_init();
         tma_prefetch_desc(&map_out);
     }
@@ -2034,34 +2092,26 @@ tc_conv_stem_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __
         if (threadIdx.x == 0) atomicCAS(status, 0, 610);
         return;
     }
-    if (warp == 4) tmem_alloc(smem_u32(&tmem_base_slot), 128);
+    if (warp == 8) tmem_alloc(smem_u32(&tmem_base_slot), 128);
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = tmem_base_slot;
 
-    if (warp < 4) {
-        const int t = threadIdx.x;
-        auto issue = [&](int j) {
-            if (j < my_tiles) stem_stage_issue(p, x, stage + (j & 1) * kStemStage, stem_tile(p, (int)blockIdx.x + j * (int)gridDim.x), t);
-            cp_async_commit();
-        };
-        issue(0);
-        bool dead = false;          // after a failed wait the thread keeps walking the barriers, without work
+    if (warp < 8) {
+        stem_gather_role(p, stage, a_tiles, (int)blockIdx.x, (int)gridDim.x, my_tiles, seg_full0, seg_empty0, a_full0, a_empty0, failed, status, 615);
+    } else if (warp == 9) {
+        int issued = 0;
         for (int j = 0; j < my_tiles; ++j) {
-            const int buf = j & 1;
-            asm volatile("bar.sync 2, 128;" ::: "memory");      // every thread has left the segments of tile j - 1
-            issue(j + 1);
-            cp_async_wait<1>();
-            asm volatile("bar.sync 2, 128;" ::: "memory");      // the segments of tile j are complete
-            if (!dead && !mbar_wait(a_empty0 + 8 * buf, ((uint32_t)(j >> 1) & 1u) ^ 1u, failed, status, 611)) dead = true;
-            if (dead) continue;
-            stem_gather_row(p, stem_tile(p, (int)blockIdx.x + j * (int)gridDim.x), stage + buf * kStemStage, a_tiles + buf * kStemATile, t);
-            fence_proxy_async();
-            mbar_arrive(a_full0 + 8 * buf);
+            const int st = j % kStemStages;
+            if (!mbar_wait(seg_empty0 + 8 * st, ((uint32_t)(j / kStemStages) & 1u) ^ 1u, failed, status, 611)) break;
+            stem_stage_tile(p, x, stage + st * kStemStage, stem_tile(p, (int)blockIdx.x + j * (int)gridDim.x), seg_full0 + 8 * st, lane);
+            issued = j + 1;
         }
-        cp_async_wait<0>();
-    } else if (warp == 4) {
+        // after a failure: copies still in flight get a bounded time to land
+        if (*failed && lane == 0)
+            for (int j = max(0, issued - kStemStages); j < issued; ++j) mbar_drain(seg_full0 + 8 * (j % kStemStages), (uint32_t)(j / kStemStages) & 1u);
+    } else if (warp == 8) {
         if (lane == 0) {
             const uint32_t idesc = instr_desc(128, 64, 0, 0);
             const uint32_t b_addr = smem_u32(b_tile);
@@ -2080,23 +2130,24 @@ tc_conv_stem_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __
             }
         }
     } else {
-        // thread = accumulator lane = pixel of the tile; rounded rows go through a swizzled tile in shared memory
-        const int quarter = warp % 4;
+        // thread = accumulator lane = pixel of the tile; rounded rows go through a swizzled tile in shared memory.
+        // Group g takes the tiles j = g, g + 2, ... (accumulator g, output tile g).
+        const int quarter = warp % 4, group = (warp - 10) / 4;
         const int row = quarter * 32 + lane;
         const bool stats = stat_partial != nullptr;
+        uint8_t* const o_tile = o_tiles + group * 16384;
         float s_acc[2] = {0.f, 0.f}, q_acc[2] = {0.f, 0.f};
-        for (int j = 0; j < my_tiles; ++j) {
-            const int buf = j & 1;
-            if (!mbar_wait(acc_full0 + 8 * buf, (uint32_t)(j >> 1) & 1u, failed, status, 614)) break;
+        for (int j = group; j < my_tiles; j += 2) {
+            if (!mbar_wait(acc_full0 + 8 * group, (uint32_t)(j >> 1) & 1u, failed, status, 614)) break;
             tc_fence_after();
-            if (lane == 0) tma_store_wait_read<0>();          // the store of the previous tile has left this warp's slab
+            if (lane == 0) tma_store_wait_read<0>();          // the store of this group's previous tile has left the warp's slab
             __syncwarp();
             const StemTile tile = stem_tile(p, (int)blockIdx.x + j * (int)gridDim.x);
             uint8_t* const orow = o_tile + row * 128;
 #pragma unroll
             for (int c0 = 0; c0 < 64; c0 += 32) {
                 uint32_t v[32];
-                tmem_ld32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * 64 + c0), v);
+                tmem_ld32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(group * 64 + c0), v);
 #pragma unroll
                 for (int q = 0; q < 4; ++q) {
                     uint4 pk;
@@ -2108,7 +2159,7 @@ tc_conv_stem_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __
                 }
             }
             tc_fence_before();
-            mbar_arrive(acc_empty0 + 8 * buf);
+            mbar_arrive(acc_empty0 + 8 * group);
             fence_proxy_async();
             __syncwarp();
             const int first = tile.ow0 + quarter * 32;
@@ -2130,25 +2181,29 @@ tc_conv_stem_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __
         }
         if (lane == 0) tma_store_wait_all();
         if (stats) {
-            // the four quarters of the CTA are added in a fixed order: one partial row pair per CTA
+            // the eight warps' sums are added in a fixed order: one partial row pair per CTA
+            const int slot = group * 4 + quarter;
 #pragma unroll
-            for (int h = 0; h < 2; ++h) { stat_red[quarter][0][2 * lane + h] = s_acc[h]; stat_red[quarter][1][2 * lane + h] = q_acc[h]; }
-            asm volatile("bar.sync 1, 128;" ::: "memory");
-            if (quarter == 0) {
+            for (int h = 0; h < 2; ++h) { stat_red[slot][0][2 * lane + h] = s_acc[h]; stat_red[slot][1][2 * lane + h] = q_acc[h]; }
+            asm volatile("bar.sync 1, 256;" ::: "memory");
+            if (slot == 0) {
 #pragma unroll
                 for (int h = 0; h < 2; ++h) {
                     const int col = h * 32 + lane;
 #pragma unroll
-                    for (int k = 0; k < 2; ++k)
-                        stat_partial[((size_t)blockIdx.x * 2 + k) * p.c_out + co0 + col] =
-                            (stat_red[0][k][col] + stat_red[1][k][col]) + (stat_red[2][k][col] + stat_red[3][k][col]);
+                    for (int k = 0; k < 2; ++k) {
+                        float acc = 0.f;
+#pragma unroll
+                        for (int u = 0; u < 8; u += 2) acc += stat_red[u][k][col] + stat_red[u + 1][k][col];
+                        stat_partial[((size_t)blockIdx.x * 2 + k) * p.c_out + co0 + col] = acc;
+                    }
                 }
             }
         }
     }
     tc_fence_before();
     __syncthreads();
-    if (warp == 4) {
+    if (warp == 8) {
         __syncwarp();
         tc_fence_after();
         tmem_dealloc(tmem_base, 128);
@@ -2160,20 +2215,23 @@ tc_conv_stem_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __
 // second accumulator repeats atom 0 and is not read back).  The dz tile of the same 128 pixels arrives by TMA (pixels
 // past the end of the row are zero-filled, and the gathered rows there are zeros too).  Each CTA keeps its two
 // accumulators over all its tiles and leaves partial[slice][c_out][147]; the slices are added in a fixed order.
-__global__ void __launch_bounds__(kStemThreads, 1)
+// Warps 0-7 gather, warp 8 issues the MMAs, warp 9 copies segments and dz tiles, warps 10-13 write the partial sums at the end.
+__global__ void __launch_bounds__(kStemWgradThreads, 1)
 tc_wgrad_stem_kernel(const __nv_bfloat16* __restrict__ x, const __grid_constant__ CUtensorMap map_dz, float* __restrict__ partial,
                      StemParams p, int* status) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* const smem_al = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
     uint8_t* const a_tiles = smem_al;                       // [2][atoms 2, 0, 1][128 pixels][128 bytes]
-    uint8_t* const dz_tiles = smem_al + 2 * kStemATile;     // [2][128 pixels][64 channels]
-    uint8_t* const stage = dz_tiles + 2 * 16384;            // [2][7][kStemSegBytes]
-    __shared__ __align__(8) uint64_t bar_mem[10];
+    uint8_t* const dz_tiles = smem_al + 2 * kStemATile;     // [kStemStages][128 pixels][64 channels]
+    uint8_t* const stage = dz_tiles + kStemStages * 16384;  // [kStemStages][7][kStemSegBytes]
+    __shared__ __align__(8) uint64_t bar_mem[5 + 4 * kStemStages];
     __shared__ uint32_t tmem_base_slot;
     __shared__ int failed_flag;
     volatile int* failed = &failed_flag;
     const uint32_t bars = smem_u32(bar_mem);
-    const uint32_t a_full0 = bars, a_empty0 = bars + 16, dz_full0 = bars + 32, dz_empty0 = bars + 48, accum_bar = bars + 64;
+    const uint32_t a_full0 = bars, a_empty0 = bars + 16, accum_bar = bars + 32;
+    const uint32_t seg_full0 = bars + 40, seg_empty0 = seg_full0 + 8 * kStemStages;
+    const uint32_t dz_full0 = seg_empty0 + 8 * kStemStages, dz_empty0 = dz_full0 + 8 * kStemStages;
 
     const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
     const int slice = blockIdx.x, co_tile = blockIdx.y;
@@ -2181,8 +2239,9 @@ tc_wgrad_stem_kernel(const __nv_bfloat16* __restrict__ x, const __grid_constant_
 
     if (threadIdx.x == 0) {
         failed_flag = 0;
-        for (int b = 0; b < 2; ++b) {
-            mbar_init(a_full0 + 8 * b, 128); mbar_init(a_empty0 + 8 * b, 1);
+        for (int b = 0; b < 2; ++b) { mbar_init(a_full0 + 8 * b, kStemGather); mbar_init(a_empty0 + 8 * b, 1); }
+        for (int b = 0; b < kStemStages; ++b) {
+            mbar_init(seg_full0 + 8 * b, 1); mbar_init(seg_empty0 + 8 * b, kStemGather);
             mbar_init(dz_full0 + 8 * b, 1); mbar_init(dz_empty0 + 8 * b, 1);
         }
         mbar_init(accum_bar, 1);
@@ -2195,58 +2254,46 @@ tc_wgrad_stem_kernel(const __nv_bfloat16* __restrict__ x, const __grid_constant_
         if (threadIdx.x == 0) atomicCAS(status, 0, 620);
         return;
     }
-    if (warp == 4) tmem_alloc(smem_u32(&tmem_base_slot), 128);
+    if (warp == 8) tmem_alloc(smem_u32(&tmem_base_slot), 128);
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = tmem_base_slot;
 
-    if (warp < 4) {
-        const int t = threadIdx.x;
-        bool dead = false;
-        auto issue = [&](int j) {
-            if (j < my_tiles) {
-                const StemTile tile = stem_tile(p, slice + j * p.slices);
-                stem_stage_issue(p, x, stage + (j & 1) * kStemStage, tile, t);
-                if (t == 0 && !dead) {
-                    // the dz tile of the same pixels, one tile ahead like the segments
-                    if (mbar_wait(dz_empty0 + 8 * (j & 1), ((uint32_t)(j >> 1) & 1u) ^ 1u, failed, status, 621)) {
-                        mbar_expect_tx(dz_full0 + 8 * (j & 1), 16384u);
-                        tma_load_4d(smem_u32(dz_tiles + (j & 1) * 16384), &map_dz, dz_full0 + 8 * (j & 1), co_tile * 64, tile.ow0, tile.oh, tile.img);
-                    }
-                }
-            }
-            cp_async_commit();
-        };
-        issue(0);
+    if (warp < 8) {
+        stem_gather_role(p, stage, a_tiles, slice, p.slices, my_tiles, seg_full0, seg_empty0, a_full0, a_empty0, failed, status, 626);
+    } else if (warp == 9) {
+        int issued = 0;
         for (int j = 0; j < my_tiles; ++j) {
-            const int buf = j & 1;
-            asm volatile("bar.sync 2, 128;" ::: "memory");      // every thread has left the segments of tile j - 1
-            issue(j + 1);
-            cp_async_wait<1>();
-            asm volatile("bar.sync 2, 128;" ::: "memory");      // the segments of tile j are complete
-            if (!dead && !mbar_wait(a_empty0 + 8 * buf, ((uint32_t)(j >> 1) & 1u) ^ 1u, failed, status, 622)) dead = true;
-            if (dead) continue;
-            stem_gather_row(p, stem_tile(p, slice + j * p.slices), stage + buf * kStemStage, a_tiles + buf * kStemATile, t);
-            fence_proxy_async();
-            mbar_arrive(a_full0 + 8 * buf);
+            const int st = j % kStemStages;
+            const uint32_t phase = (uint32_t)(j / kStemStages) & 1u;
+            if (!mbar_wait(seg_empty0 + 8 * st, phase ^ 1u, failed, status, 621)) break;
+            if (!mbar_wait(dz_empty0 + 8 * st, phase ^ 1u, failed, status, 622)) break;
+            const StemTile tile = stem_tile(p, slice + j * p.slices);
+            stem_stage_tile(p, x, stage + st * kStemStage, tile, seg_full0 + 8 * st, lane);
+            if (lane == 0) {
+                mbar_expect_tx(dz_full0 + 8 * st, 16384u);
+                tma_load_4d(smem_u32(dz_tiles + st * 16384), &map_dz, dz_full0 + 8 * st, co_tile * 64, tile.ow0, tile.oh, tile.img);
+            }
+            issued = j + 1;
         }
-        cp_async_wait<0>();
-        // copies that were issued but never consumed after a failure get a bounded time to land
-        if (*failed && t == 0)
-            for (int b = 0; b < 2; ++b) mbar_drain(dz_full0 + 8 * b, 0);
-    } else if (warp == 4) {
+        // after a failure: copies still in flight get a bounded time to land
+        if (*failed && lane == 0)
+            for (int j = max(0, issued - kStemStages); j < issued; ++j) {
+                mbar_drain(seg_full0 + 8 * (j % kStemStages), (uint32_t)(j / kStemStages) & 1u);
+                mbar_drain(dz_full0 + 8 * (j % kStemStages), (uint32_t)(j / kStemStages) & 1u);
+            }
+    } else if (warp == 8) {
         if (lane == 0) {
             const uint32_t idesc = instr_desc(128, 64, 1, 1);
             bool ok = true;
             for (int j = 0; j < my_tiles && ok; ++j) {
-                const int buf = j & 1;
-                const uint32_t phase = (uint32_t)(j >> 1) & 1u;
-                if (!mbar_wait(a_full0 + 8 * buf, phase, failed, status, 623)) { ok = false; break; }
-                if (!mbar_wait(dz_full0 + 8 * buf, phase, failed, status, 624)) { ok = false; break; }
+                const int buf = j & 1, st = j % kStemStages;
+                if (!mbar_wait(a_full0 + 8 * buf, (uint32_t)(j >> 1) & 1u, failed, status, 623)) { ok = false; break; }
+                if (!mbar_wait(dz_full0 + 8 * st, (uint32_t)(j / kStemStages) & 1u, failed, status, 624)) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t a_addr = smem_u32(a_tiles + buf * kStemATile);
-                const uint32_t dz_addr = smem_u32(dz_tiles + buf * 16384);
+                const uint32_t dz_addr = smem_u32(dz_tiles + st * 16384);
 #pragma unroll
                 for (int kk = 0; kk < 8; ++kk) {            // 16 pixels per MMA
                     const uint64_t bd = smem_desc(dz_addr + kk * 2048, 8192, 1024);
@@ -2254,7 +2301,7 @@ tc_wgrad_stem_kernel(const __nv_bfloat16* __restrict__ x, const __grid_constant_
                     umma_bf16(tmem_base + 64u, smem_desc(a_addr + stem_atom_offset(2) + kk * 2048, 16384, 1024), bd, idesc, (j > 0 || kk > 0) ? 1u : 0u);
                 }
                 umma_commit(a_empty0 + 8 * buf);
-                umma_commit(dz_empty0 + 8 * buf);
+                umma_commit(dz_empty0 + 8 * st);
             }
             if (ok) umma_commit(accum_bar);
         }
@@ -2280,12 +2327,12 @@ tc_wgrad_stem_kernel(const __nv_bfloat16* __restrict__ x, const __grid_constant_
                 }
             }
         } else if (my_tiles == 0) {
-            for (int i = threadIdx.x - 160; i < 64 * 147; i += 128) base[i] = 0.f;
+            for (int i = threadIdx.x - (kStemGather + 64); i < 64 * 147; i += 128) base[i] = 0.f;
         }
     }
     tc_fence_before();
     __syncthreads();
-    if (warp == 4) {
+    if (warp == 8) {
         __syncwarp();
         tc_fence_after();
         tmem_dealloc(tmem_base, 128);
@@ -3251,7 +3298,7 @@ int stem_conv_fwd(const ConvGeom& g, const void* x, const void* w, void* z, int*
     const int co_tiles = g.cout / 64;
     dim3 grid((unsigned)std::min(p.m_tiles, std::max(1, sm_count() / co_tiles)), (unsigned)co_tiles);
     if (blocks) *blocks = partial ? (int)grid.x : 0;
-    tc_conv_stem_kernel<<<grid, kStemThreads, kStemFwdSmem, (cudaStream_t)stream>>>((const __nv_bfloat16*)x, (const __nv_bfloat16*)w,
+    tc_conv_stem_kernel<<<grid, kStemFwdThreads, kStemFwdSmem, (cudaStream_t)stream>>>((const __nv_bfloat16*)x, (const __nv_bfloat16*)w,
                                                                                   map_out, partial, p, device_status);
     CKPT_LAUNCH_CHECK_NAMED("tc_conv_stem_kernel", "stem conv forward (tensor cores)");
     return CKPT_OK;
@@ -3280,7 +3327,7 @@ int stem_conv_wgrad(const ConvGeom& g, const void* dz, const void* x, float* dw,
         attr_set = true;
     }
     dim3 grid((unsigned)p.slices, (unsigned)(g.cout / 64));
-    tc_wgrad_stem_kernel<<<grid, kStemThreads, kStemWgradSmem, st>>>((const __nv_bfloat16*)x, map_dz, (float*)scratch, p, device_status);
+    tc_wgrad_stem_kernel<<<grid, kStemWgradThreads, kStemWgradSmem, st>>>((const __nv_bfloat16*)x, map_dz, (float*)scratch, p, device_status);
     CKPT_LAUNCH_CHECK_NAMED("tc_wgrad_stem_kernel", "stem conv wgrad (tensor cores)");
     launch_slice_sum((const float*)scratch, dw, (int64_t)g.cout * 147, p.slices, st, upd);
     CKPT_LAUNCH_CHECK("stem wgrad slice sum");
