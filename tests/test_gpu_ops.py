@@ -14,6 +14,15 @@ from tests.gpu_util import max_rel_err, to_dev, to_host
 
 pytestmark = pytest.mark.gpu
 TOL = {ck.DTYPE_F32: 1e-3, ck.DTYPE_BF16: 3e-2}
+
+
+@pytest.fixture(autouse=True)
+def no_device_timeout():
+    """Every operation of a test must leave the library's device status word at zero: a bounded wait that gave up inside
+    a kernel would otherwise look like a numeric error (or pass, on a tensor the test does not read)."""
+    yield
+    assert ck.op_status() == 0
+
 # pure rounding of one bf16 output is 2^-9 relative; anything above a few of those is a bug
 TIGHT = {ck.DTYPE_F32: 2e-5, ck.DTYPE_BF16: 6e-3}
 
