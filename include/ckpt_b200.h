@@ -235,6 +235,19 @@ CKPT_API int ckpt_chain_set_impl(ckpt_chain* chain, int impl);
  * label pointer in pageable host memory disables recording for that call.  enable = 0 drops the
  * recordings.  The library holds 64 bytes of pinned host memory per chain while enabled. */
 CKPT_API int ckpt_chain_set_graph(ckpt_chain* chain, int enable);
+/* Input staging: overlaps the host-to-device copy of the next step's batch with the current step (the training loop
+ * of Algorithms 1, 2 and 4 reads one batch per step; ckpt_train_step itself copies a host batch at its start, on the
+ * step's stream).  ckpt_chain_stage_batch starts an asynchronous copy of batch (host; pinned memory for a copy that
+ * really overlaps) and labels (host, or null for the sum loss) into slot 0 or 1 of staging (device, caller-owned,
+ * ckpt_chain_staging_bytes bytes, 256-byte aligned) on a stream the chain owns, and returns the device addresses of the
+ * staged batch and labels.  Passing that batch address to ckpt_train_step makes the step wait, on its own stream, for
+ * the copy before it reads the batch.  A slot may be staged again once the step that was given it has returned
+ * (ckpt_train_step returns after its step has finished).  Typical loop: stage(slot 0, batch 0); for k: stage(slot
+ * (k+1) % 2, batch k+1); train_step(staged slot k % 2).
+ * Errors: CKPT_E_NULL, CKPT_E_BAD_ARG (slot), CKPT_E_WORKSPACE (staging too small), CKPT_E_NO_DEVICE, CKPT_E_CUDA. */
+CKPT_API int ckpt_chain_staging_bytes(const ckpt_chain* chain, int64_t* bytes);
+CKPT_API int ckpt_chain_stage_batch(ckpt_chain* chain, int slot, const void* batch, const int32_t* labels, void* staging,
+                           int64_t staging_bytes, const void** batch_dev, const int32_t** labels_dev);
 
 /* Verification aid (off by default): the backward recursion of Eq. (3) made visible.  With a tap set, every
  * ckpt_train_step also copies r_i = dL/dd_i, as it enters the backward step of unit i, to

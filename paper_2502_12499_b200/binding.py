@@ -254,6 +254,25 @@ class Chain:
         """ckpt_chain_set_graph: record the launch sequence of a repeated step once and replay it."""
         _check(lib().ckpt_chain_set_graph(self._h, C.c_int(1 if enable else 0)))
 
+    def staging_bytes(self):
+        """ckpt_chain_staging_bytes: size of the two-slot staging buffer of ckpt_chain_stage_batch."""
+        b = C.c_int64(0)
+        _check(lib().ckpt_chain_staging_bytes(self._h, C.byref(b)))
+        return b.value
+
+    def stage_batch(self, slot, batch, labels, staging):
+        """ckpt_chain_stage_batch: starts the copy of a host batch (torch tensor or numpy array in the chain's storage
+        layout) and its labels into a slot of the device tensor ``staging``; returns the device addresses (ints; the
+        second is None without labels) to hand to train_step as ``batch`` and ``labels``."""
+        def addr(a):
+            if a is None:
+                return C.c_void_p(0)
+            return C.c_void_p(a.ctypes.data if isinstance(a, np.ndarray) else a.data_ptr())
+        b_dev, l_dev = C.c_void_p(0), C.c_void_p(0)
+        _check(lib().ckpt_chain_stage_batch(self._h, C.c_int(slot), addr(batch), addr(labels), _dev(staging),
+                                            C.c_int64(staging.numel() * staging.element_size()), C.byref(b_dev), C.byref(l_dev)))
+        return b_dev.value, l_dev.value
+
 
 def flatten_params(chain_spec, params):
     """List of (unit index, name, array) in the library's parameter order."""
@@ -282,8 +301,9 @@ def upload_params(chain, params, device="cuda"):
 
 
 def train_step(chain, is_ckpt, policy, batch, labels, params, grads, arena, workspace, stream=None):
-    """ckpt_train_step.  ``batch``/``labels``: torch tensors (device, or pinned/pageable host) or
-    numpy arrays already in the chain's storage layout; everything else: device torch tensors."""
+    """ckpt_train_step.  ``batch``/``labels``: torch tensors (device, or pinned/pageable host), numpy arrays already
+    in the chain's storage layout, or the device addresses Chain.stage_batch returned; everything else: device torch
+    tensors."""
     n_p = chain.num_params()
     p_arr = (C.c_void_p * n_p)(*[t.data_ptr() for t in params])
     g_arr = (C.c_void_p * n_p)(*[t.data_ptr() for t in grads])
@@ -295,6 +315,8 @@ def train_step(chain, is_ckpt, policy, batch, labels, params, grads, arena, work
     def addr(a):
         if a is None:
             return C.c_void_p(0)
+        if isinstance(a, int):                  # a device address from Chain.stage_batch
+            return C.c_void_p(a)
         if isinstance(a, np.ndarray):
             return C.c_void_p(a.ctypes.data)
         return C.c_void_p(a.data_ptr())

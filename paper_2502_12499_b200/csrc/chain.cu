@@ -61,6 +61,12 @@ struct ckpt_chain {
     void* host_result = nullptr;         // pinned: loss (8 bytes) and status word of the last step
     cudaStream_t capture_stream = nullptr;   // recording happens here (the caller's stream may be the default one,
                                              // which cannot record); replays run on the caller's stream
+    // input staging (ckpt_chain_stage_batch): copies run on a stream of the chain's own, the step that is given a
+    // staged batch waits for the copy's event on its stream
+    cudaStream_t copy_stream = nullptr;
+    cudaEvent_t stage_event[2] = {nullptr, nullptr};
+    const void* stage_batch[2] = {nullptr, nullptr};
+    bool stage_pending[2] = {false, false};
     ~ckpt_chain();
 };
 
@@ -702,6 +708,8 @@ ckpt_chain::~ckpt_chain() {
     ckpt::drop_graphs(this);
     if (host_result) cudaFreeHost(host_result);
     if (capture_stream) cudaStreamDestroy(capture_stream);
+    for (cudaEvent_t e : stage_event) if (e) cudaEventDestroy(e);
+    if (copy_stream) cudaStreamDestroy(copy_stream);
 }
 
 using namespace ckpt;
@@ -982,6 +990,14 @@ int ckpt_train_step(ckpt_chain* chain, const uint8_t* is_ckpt, int policy, const
     c.arena_base = (char*)arena; c.ws = (char*)workspace; c.params = params; c.grads = grads;
     c.batch = batch; c.labels = labels; c.stream = (cudaStream_t)stream; c.arena = &ar;
     double loss = 0;
+    for (int slot = 0; slot < 2; ++slot) {
+        if (chain->stage_pending[slot] && chain->stage_batch[slot] == batch) {
+            // the batch was staged by ckpt_chain_stage_batch: its copy has to land before the step reads it
+            cudaError_t se = cudaStreamWaitEvent(c.stream, chain->stage_event[slot], 0);
+            if (se != cudaSuccess) return cuda_fail(se, "waiting for the staged batch");
+            chain->stage_pending[slot] = false;
+        }
+    }
     if (chain->use_graph && graph_eligible(batch, labels)) {
         std::vector<uint64_t> args;
         const uint64_t key = step_key(chain, is_ckpt, policy, batch, labels, params, grads, arena, workspace, &args);
@@ -1030,6 +1046,49 @@ int ckpt_chain_set_graph(ckpt_chain* chain, int enable) {
     }
     chain->use_graph = enable ? 1 : 0;
     if (!enable) drop_graphs(chain);
+    return CKPT_OK;
+}
+
+static int64_t staging_slot_bytes(const ckpt_chain* chain) {
+    return align_up(chain->d[0], 256) + align_up(chain->batch * (int64_t)sizeof(int32_t), 256);
+}
+
+int ckpt_chain_staging_bytes(const ckpt_chain* chain, int64_t* bytes) {
+    if (!chain || !bytes) { set_error("null pointer"); return CKPT_E_NULL; }
+    *bytes = 2 * staging_slot_bytes(chain);
+    return CKPT_OK;
+}
+
+int ckpt_chain_stage_batch(ckpt_chain* chain, int slot, const void* batch, const int32_t* labels, void* staging, int64_t staging_bytes,
+                           const void** batch_dev, const int32_t** labels_dev) {
+    if (!chain || !batch || !staging || !batch_dev || !labels_dev) { set_error("null pointer"); return CKPT_E_NULL; }
+    if (slot < 0 || slot > 1) { set_error("staging slot %d: 0 or 1", slot); return CKPT_E_BAD_ARG; }
+    if (chain->loss == CKPT_LOSS_SOFTMAX_CE && !labels) { set_error("labels are null"); return CKPT_E_NULL; }
+    if (staging_bytes < 2 * staging_slot_bytes(chain)) {
+        set_error("staging buffer of %lld bytes, %lld needed", (long long)staging_bytes, (long long)(2 * staging_slot_bytes(chain)));
+        return CKPT_E_WORKSPACE;
+    }
+    int ndev = 0;
+    if (cudaGetDeviceCount(&ndev) != cudaSuccess || ndev == 0) { set_error("no CUDA device"); return CKPT_E_NO_DEVICE; }
+    cudaError_t e = cudaSuccess;
+    if (!chain->copy_stream) {
+        e = cudaStreamCreateWithFlags(&chain->copy_stream, cudaStreamNonBlocking);
+        if (e != cudaSuccess) { chain->copy_stream = nullptr; return cuda_fail(e, "creating the copy stream"); }
+    }
+    if (!chain->stage_event[slot]) {
+        e = cudaEventCreateWithFlags(&chain->stage_event[slot], cudaEventDisableTiming);
+        if (e != cudaSuccess) { chain->stage_event[slot] = nullptr; return cuda_fail(e, "creating the staging event"); }
+    }
+    char* base = (char*)staging + (int64_t)slot * staging_slot_bytes(chain);
+    int32_t* lab = (int32_t*)(base + align_up(chain->d[0], 256));
+    e = cudaMemcpyAsync(base, batch, (size_t)chain->d[0], cudaMemcpyDefault, chain->copy_stream);
+    if (e == cudaSuccess && labels) e = cudaMemcpyAsync(lab, labels, (size_t)chain->batch * sizeof(int32_t), cudaMemcpyDefault, chain->copy_stream);
+    if (e == cudaSuccess) e = cudaEventRecord(chain->stage_event[slot], chain->copy_stream);
+    if (e != cudaSuccess) return cuda_fail(e, "staging a batch");
+    chain->stage_batch[slot] = base;
+    chain->stage_pending[slot] = true;
+    *batch_dev = base;
+    *labels_dev = labels ? lab : nullptr;
     return CKPT_OK;
 }
 

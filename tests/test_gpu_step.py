@@ -350,3 +350,47 @@ def test_graph_replay_is_bit_identical(dtype):
     assert rep["replayed"] == 0
     for a, b in zip(g_two, graphed.grads):
         assert np.array_equal(a, b.detach().cpu().numpy())
+
+
+@pytest.mark.parametrize("graph", [False, True])
+def test_staged_batches_equal_direct_steps(graph):
+    """ckpt_chain_stage_batch: batches copied from pinned host memory on the chain's copy stream, one step ahead, give
+    the gradients, loss and report of steps that are handed the same batches directly - launch by launch and through
+    graph replay (one recording per staging slot)."""
+    import torch
+    spec = mini_vgg("bf16")
+    params = wl.make_params(spec, seed=43, bn_affine="random")
+    direct, staged = StepRunner(spec, params), StepRunner(spec, params)
+    staged.chain.set_graph(graph)
+    mask = ck.plan(ck.ALGO_DYNAMIC_N, direct.d)[0]
+    peak = ck.eval(ck.MODEL_DYNAMIC, direct.d, mask)
+    arenas = [torch.empty(peak, dtype=torch.uint8, device="cuda") for _ in range(2)]
+    staging = torch.empty(staged.chain.staging_bytes(), dtype=torch.uint8, device="cuda")
+    staging.fill_(0xFF)
+    batches = []
+    for step in range(6):
+        x, labels = wl.make_batch(spec, seed=70 + step)
+        batches.append((torch.from_numpy(x).to(torch.bfloat16).pin_memory(),
+                        torch.from_numpy(np.ascontiguousarray(labels, dtype=np.int32)).pin_memory()))
+    nxt = staged.chain.stage_batch(0, batches[0][0], batches[0][1], staging)
+    replayed = []
+    for step in range(6):
+        cur = nxt
+        if step + 1 < 6:
+            nxt = staged.chain.stage_batch((step + 1) % 2, batches[step + 1][0], batches[step + 1][1], staging)
+        for g in staged.grads + direct.grads:
+            g.fill_(float("nan"))
+        rep_s = ck.train_step(staged.chain, mask, ck.POLICY_DYNAMIC, cur[0], cur[1], staged.params, staged.grads, arenas[0], staged.workspace)
+        rep_d = ck.train_step(direct.chain, mask, ck.POLICY_DYNAMIC, batches[step][0].cuda(), batches[step][1].cuda(), direct.params,
+                              direct.grads, arenas[1], direct.workspace)
+        torch.cuda.synchronize()
+        replayed.append(rep_s["replayed"])
+        for key in ("peak_bytes", "extent_bytes", "predicted_bytes", "recomputed_units", "loss", "device_status"):
+            assert rep_s[key] == rep_d[key], (step, key)
+        assert np.isfinite(rep_s["loss"])
+        for a, b in zip(staged.grads, direct.grads):
+            assert torch.equal(a, b)
+    assert replayed == ([0, 0, 1, 1, 1, 1] if graph else [0] * 6)
+    with pytest.raises(ck.CkptError) as e:
+        staged.chain.stage_batch(0, batches[0][0], batches[0][1], staging[:-256])
+    assert e.value.code == -8

@@ -304,3 +304,16 @@ def test_chain_option_errors_need_no_device():
     assert lib.ckpt_chain_set_sgd(None, C.c_double(0.01)) == -1
     assert lib.ckpt_chain_set_selftest(None, 1) == -1
     assert lib.ckpt_selftest_bounded_wait(C.c_int64(0), None) in (-6, -1)                   # limit out of range (or no status word)
+    # input staging: null pointers, slot, labels and buffer size are checked before any device call
+    need_stage = chain.staging_bytes()
+    assert need_stage >= 2 * (int(chain.sizes()[0]) + 4 * wl.config(1)["batch"])
+    out_b, out_l = C.c_void_p(0), C.c_void_p(0)
+    args = lambda slot, batch, labels, size: lib.ckpt_chain_stage_batch(  # noqa: E731
+        chain._h, C.c_int(slot), batch, labels, fake, C.c_int64(size), C.byref(out_b), C.byref(out_l))
+    assert args(0, None, fake, need_stage) == -1
+    assert args(2, fake, fake, need_stage) == -6 and "slot" in lib.ckpt_last_error().decode()
+    labelled = ck.Chain(wl.config(2))               # softmax loss: labels are required
+    assert lib.ckpt_chain_stage_batch(labelled._h, C.c_int(0), fake, None, fake, C.c_int64(labelled.staging_bytes()), C.byref(out_b),
+                                      C.byref(out_l)) == -1 and "labels" in lib.ckpt_last_error().decode()
+    assert args(1, fake, fake, need_stage - 1) == -8 and "staging" in lib.ckpt_last_error().decode()
+    assert lib.ckpt_chain_staging_bytes(chain._h, None) == -1
