@@ -3,7 +3,8 @@
 * the tensor-core convolution kernels at the VGG-16 / batch-64 layer shapes, on sampled outputs that
   the oracle computes one by one (a cropped neighbourhood for forward/dgrad, one (c_out, c_in)
   channel pair over all pixels for wgrad), and the fully connected layers of the VGG-16 head on
-  sampled output rows and input columns;
+  sampled output rows and input columns; the same for the layer shapes of the residual networks at their
+  benchmark batches (7x7 stride-2 stem, 1x1 layers, strided 3x3 and 1x1 layers);
 * the whole checkpointed step of configurations 2, 3, 4 and 5 through properties that hold at any size:
   arena high-water == highest offset == planner's prediction (arena of exactly that size),
   gradients bit-identical between the checkpointed and the store-all schedule, finite loss;
@@ -119,7 +120,113 @@ def test_fc_kernels_full_size_sampled(layer):
     assert np.abs(bf16_host(dx[..., ins]) - dx_ref).max() <= 6e-3 * scale_dx
 
 
+RESNET_LAYERS = [
+    # n, h, w, cin, cout, k, stride, pad: layer shapes of the residual networks at their benchmark batches
+    (128, 224, 224, 3, 64, 7, 2, 3),     # stem: operand tiles gathered from staged input rows
+    (128, 56, 56, 64, 256, 1, 1, 0),     # 1x1, short reduction (role-swapped kernel, epilogue-bound)
+    (128, 56, 56, 256, 64, 1, 1, 0),     # 1x1, 64 output channels
+    (128, 56, 56, 128, 128, 3, 2, 1),    # 3x3 stride 2: strided boxes forward, parity classes for dgrad
+    (128, 56, 56, 256, 512, 1, 2, 0),    # 1x1 stride-2 projection
+    (256, 14, 14, 256, 1024, 1, 1, 0),   # the layers ResNet-152 spends its time in
+    (256, 14, 14, 1024, 256, 1, 1, 0),
+    (256, 14, 14, 256, 256, 3, 1, 1),
+    (128, 7, 7, 512, 512, 3, 1, 1),
+]
+
+
+def crop_range(o, size_out, size_in, k, stride, pad, lo_out, hi_out):
+    """Output rows [a, b) around [lo_out, hi_out] and the input rows [a * stride, end) such that the oracle's
+    convolution of the cropped input (same stride and padding) has exactly the output rows a .. b - 1 of the full
+    convolution, and is exact on rows lo_out .. hi_out: the crop starts on a multiple of the stride (or at the image
+    border, where the oracle's zero padding is the real one) far enough above, and ends at the image border or after
+    the last row the window of output b - 1 reads."""
+    margin = -(-pad // stride) + 1
+    a = max(0, lo_out - margin)
+    b = min(size_out, hi_out + margin + 1)
+    start = a * stride
+    end = size_in if b == size_out else start + (b - a - 1) * stride + k - 2 * pad
+    # rows the oracle pads below the crop stand for real rows: keep output hi_out's window inside the crop
+    while b < size_out and hi_out * stride - pad + k > end:
+        b += 1
+        end = size_in if b == size_out else start + (b - a - 1) * stride + k - 2 * pad
+    assert (end - start + 2 * pad - k) // stride + 1 == b - a
+    return a, b, start, end
+
+
+@pytest.mark.parametrize("layer", RESNET_LAYERS, ids=lambda l: "x".join(map(str, l)))
+def test_resnet_conv_kernels_full_size_sampled(layer):
+    """The convolution kernels at the residual networks' layer shapes and batches (7x7 stem, 1x1, strided 3x3 and
+    1x1): sampled output pixels and input-gradient pixels against the oracle's convolution of a cropped neighbourhood,
+    sampled (c_out, c_in) pairs of the weight gradient against the oracle over all pixels."""
+    import torch
+    n, h, w, cin, cout, k, stride, pad = layer
+    ho, wo = (h + 2 * pad - k) // stride + 1, (w + 2 * pad - k) // stride + 1
+    dt = ck.DTYPE_BF16
+    gen = torch.Generator(device="cuda").manual_seed(n * h + cin + k)
+    x = torch.randn(n, h, w, cin, device="cuda", generator=gen).bfloat16()
+    wt = (torch.randn(cout, k, k, cin, device="cuda", generator=gen) / (k * cin ** 0.5)).bfloat16()
+    dz = torch.randn(n, ho, wo, cout, device="cuda", generator=gen).bfloat16()
+    shape = ck.ConvShape(n, h, w, cin, cout, k, stride, pad)
+    scratch = torch.empty(max(256, ck.conv2d_scratch_bytes(shape, dt)), dtype=torch.uint8, device="cuda")
+    z = torch.empty(n, ho, wo, cout, device="cuda", dtype=torch.bfloat16)
+    dx = torch.empty_like(x)
+    dw = torch.empty(cout, k, k, cin, device="cuda")
+    ck.launch_log(True)
+    try:
+        ck.conv2d_forward(shape, dt, 0, x, wt, z, scratch)
+        if cin > 3:
+            ck.conv2d_dgrad(shape, dt, 0, dz, wt, dx, scratch)
+        ck.conv2d_wgrad(shape, dt, 0, dz, x, dw, scratch)
+        torch.cuda.synchronize()
+    finally:
+        kernels = ck.launch_log_read()
+        ck.launch_log(False)
+    assert ck.op_status() == 0
+    assert not [name for name in kernels if "CUDA cores" in name or "conv_gemm" in name], kernels
+    w64 = bf16_host(wt)
+    rng = np.random.default_rng(13)
+    scale_z = float(z.float().abs().max())
+    # forward: corners, borders and random output pixels
+    picks = [(0, 0, 0), (n - 1, ho - 1, wo - 1), (n // 2, 0, wo - 1), (n - 1, ho - 1, 0), (1, ho // 2, wo // 2)]
+    picks += [(int(rng.integers(n)), int(rng.integers(ho)), int(rng.integers(wo))) for _ in range(9)]
+    for (b, oi, oj) in picks:
+        a_i, b_i, s_i, e_i = crop_range(oi, ho, h, k, stride, pad, oi, oi)
+        a_j, b_j, s_j, e_j = crop_range(oj, wo, w, k, stride, pad, oj, oj)
+        z_crop = no.conv2d_fwd(bf16_host(x[b:b + 1, s_i:e_i, s_j:e_j, :]), w64, stride, pad)
+        assert z_crop.shape[1:3] == (b_i - a_i, b_j - a_j)
+        assert np.abs(bf16_host(z[b, oi, oj, :]) - z_crop[0, oi - a_i, oj - a_j, :]).max() <= 6e-3 * scale_z, (b, oi, oj)
+    # input gradient: every output pixel whose window reaches the input pixel lies inside the crop
+    if cin > 3:
+        scale_dx = float(dx.float().abs().max())
+        picks = [(0, 0, 0), (n - 1, h - 1, w - 1), (n // 2, 0, w - 1), (n - 1, h - 1, 0), (1, h // 2 + 1, w // 2)]
+        picks += [(int(rng.integers(n)), int(rng.integers(h)), int(rng.integers(w))) for _ in range(9)]
+        for (b, i, j) in picks:
+            rng_o = []
+            for pos, size_o in ((i, ho), (j, wo)):
+                lo = max(0, -(-(pos + pad - k + 1) // stride))
+                hi = min(size_o - 1, (pos + pad) // stride)
+                rng_o.append((lo, max(lo, hi)))
+            a_i, b_i, s_i, e_i = crop_range(i, ho, h, k, stride, pad, *rng_o[0])
+            a_j, b_j, s_j, e_j = crop_range(j, wo, w, k, stride, pad, *rng_o[1])
+            if not (s_i <= i < e_i and s_j <= j < e_j):
+                continue                                    # an input pixel no window reaches (stride-2 1x1): checked below
+            xc = np.zeros((1, e_i - s_i, e_j - s_j, cin))
+            dx_crop = no.conv2d_bwd(xc, w64, bf16_host(dz[b:b + 1, a_i:b_i, a_j:b_j, :]), stride, pad)[0]
+            assert np.abs(bf16_host(dx[b, i, j, :]) - dx_crop[0, i - s_i, j - s_j, :]).max() <= 6e-3 * scale_dx, (b, i, j)
+        if k == 1 and stride == 2:
+            assert float(dx[:, 1::2, :, :].float().abs().max()) == 0.0 and float(dx[:, :, 1::2, :].float().abs().max()) == 0.0
+    # weight gradient: sampled (c_out, c_in) pairs over all pixels
+    scale_dw = float(dw.abs().max())
+    for _ in range(2):
+        co, ci = int(rng.integers(cout)), int(rng.integers(cin))
+        dw_ref = no.conv2d_bwd(bf16_host(x[..., ci:ci + 1]), np.zeros((1, k, k, 1)), bf16_host(dz[..., co:co + 1]), stride, pad)[1][0, :, :, 0]
+        assert np.abs(dw[co, :, :, ci].cpu().numpy().astype(np.float64) - dw_ref).max() <= 2e-5 * max(scale_dw, np.abs(dw_ref).max()), (co, ci)
+    del x, z, dx, dz, dw, scratch
+    torch.cuda.empty_cache()
+
+
 def step_properties(spec, seed=0, finite_last_units=None):
+
     import torch
     params = wl.make_params(spec, seed=seed)
     x, labels = wl.make_batch(spec, seed=seed + 1)
