@@ -67,7 +67,7 @@ def conv(what, n, h, w, cin, cout, k, pad, stride=1, reps=None, impl=0):
     ho, wo = (h + 2 * pad - k) // stride + 1, (w + 2 * pad - k) // stride + 1
     x_b, z_b, w_b = n * h * w * cin * 2.0, n * ho * wo * cout * 2.0, cout * k * k * cin * 2.0
     nbytes = x_b + z_b + (2 * w_b if what == "wgrad" else w_b)
-    scratch = torch.empty(max(256, ck.conv2d_scratch_bytes(shape, dt)), dtype=torch.uint8, device="cuda")
+    scratch = torch.empty(max(256, ck.conv2d_scratch_bytes(shape, dt), ck.bn_scratch_bytes(n * ho * wo, cout)), dtype=torch.uint8, device="cuda")
     fns = []
     for _ in range(1 if reps == 1 else sets_beyond_l2(nbytes)):
         x = torch.randn(n, h, w, cin, device="cuda").bfloat16()
@@ -75,6 +75,12 @@ def conv(what, n, h, w, cin, cout, k, pad, stride=1, reps=None, impl=0):
         z = torch.empty(n, ho, wo, cout, device="cuda", dtype=torch.bfloat16)
         if what == "fwd":
             fns.append(lambda x=x, wt=wt, z=z: ck.conv2d_forward(shape, dt, impl, x, wt, z, scratch))
+        elif what == "fwd_stats":
+            # as a conv+BN+ReLU unit runs it: the batch-norm sums of the stored output gathered in the epilogue, then
+            # the per-channel finalize
+            gamma, beta = torch.ones(cout, device="cuda"), torch.zeros(cout, device="cuda")
+            stats = torch.empty(4 * cout, device="cuda")
+            fns.append(lambda x=x, wt=wt, z=z, g=gamma, b=beta, st=stats: ck.conv2d_bn_statistics(shape, dt, x, wt, z, g, b, st, scratch))
         elif what == "dgrad":
             z.normal_()
             dx = torch.empty_like(x)
