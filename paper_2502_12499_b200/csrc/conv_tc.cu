@@ -703,10 +703,12 @@ constexpr long long PAIR_MIN_PIXELS = 262144;      // pixel pairs on the plain r
 constexpr long long PAIR_MIN_PIXELS_STRIPS = 65536;    // from this size when the pairs tile into strips
 constexpr int kTpBoxes = 6, kTpPatches = 3;
 constexpr uint32_t kTpPatchSlot = 34 * 1024;
-constexpr uint32_t kTpSmem = kTpBoxes * 16384 + kTpPatches * kTpPatchSlot + 256 + 4 * 2 * 2048 + 1024;
+constexpr int kTpEpi = 2;                          // epilogue warps per quarter of the accumulator's lanes, one chunk slab each
+constexpr int kTpThreads = 64 + 128 * kTpEpi;
+constexpr uint32_t kTpSmem = kTpBoxes * 16384 + kTpPatches * kTpPatchSlot + 256 + 4 * kTpEpi * 2048 + 1024;
 
 template <bool A_MN>
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__(kTpThreads, 1)
 tc_conv_tp_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w,
                   const __grid_constant__ CUtensorMap map_out, float* __restrict__ stat_partial, TParams p, int* status) {
     extern __shared__ uint8_t smem_raw[];
@@ -714,7 +716,7 @@ tc_conv_tp_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
     constexpr uint32_t a_bytes = 128 * 128;
     const uint32_t patches = base + kTpBoxes * a_bytes;
     const uint32_t bars = patches + kTpPatches * kTpPatchSlot;
-    const uint32_t out_stage = bars + 256;                                   // [4 warps][2][32 pixels x 32 channels] bf16
+    const uint32_t out_stage = bars + 256;                                   // [epilogue warps][32 pixels x 32 channels] bf16
     __shared__ uint32_t tmem_base_slot;
     __shared__ int failed_flag;
     volatile int* failed = &failed_flag;
@@ -742,7 +744,7 @@ tc_conv_tp_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
         failed_flag = 0;
         for (int s = 0; s < kTpBoxes; ++s) { mbar_init(a_full(s), 1); mbar_init(a_empty(s), 1); }
         for (int s = 0; s < kTpPatches; ++s) { mbar_init(p_full(s), 1); mbar_init(p_empty(s), 1); }
-        for (int b = 0; b < 2; ++b) { mbar_init(acc_full0 + 8 * b, 1); mbar_init(acc_empty0 + 8 * b, 128); }
+        for (int b = 0; b < 2; ++b) { mbar_init(acc_full0 + 8 * b, 1); mbar_init(acc_empty0 + 8 * b, 128 * kTpEpi); }
         fence_barrier_init();
         tma_prefetch_desc(&map_x);
         tma_prefetch_desc(&map_w);
@@ -815,11 +817,10 @@ tc_conv_tp_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
         }
     } else if (warp >= 2) {
         // ---------------- epilogue, as in tc_conv_t_kernel: lane = output channel, column = pixel hl * 8 + wl of the tile
-        const int quarter = warp % 4;
+        const int quarter = warp % 4, half = (warp - 2) / 4;      // the warps of a quarter take alternate chunks
         const int co = co_tile * 128 + quarter * 32 + lane;
         const bool stats = stat_partial != nullptr;
         float sum[4] = {0.f, 0.f, 0.f, 0.f}, sumsq[4] = {0.f, 0.f, 0.f, 0.f};
-        int chunk_count = 0;
         for (int j = 0; j < my_tiles; ++j) {
             const int buf = j & 1;
             if (!mbar_wait(acc_full0 + 8 * buf, (uint32_t)(j >> 1) & 1u, failed, status, 913)) break;
@@ -827,7 +828,7 @@ tc_conv_tp_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
             int w0, h0, n0;
             tile_origin(j, w0, h0, n0);
 #pragma unroll 1
-            for (int c0 = 0; c0 < p.tile_cols; c0 += 32, ++chunk_count) {
+            for (int c0 = half * 32; c0 < p.tile_cols; c0 += 32 * kTpEpi) {
                 const int idx = c0 + lane;
                 // accumulator row (idx / 8) -> image of the stack and row of that image
                 const int arow = idx >> 3, img = p.stack ? arow / p.th : 0, hrow = p.stack ? arow % p.th : arow;
@@ -835,8 +836,8 @@ tc_conv_tp_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
                 const uint32_t in_mask = __ballot_sync(0xffffffffu, inside);
                 uint32_t v[32];
                 tmem_ld32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * 256 + c0), v);
-                const uint32_t slab = out_stage + (uint32_t)((quarter * 2 + (chunk_count & 1)) * 2048);
-                if (lane == 0) tma_store_wait_read<1>();          // the store that last read this slab has left it
+                const uint32_t slab = out_stage + (uint32_t)((warp - 2) * 2048);
+                if (lane == 0) tma_store_wait_read<0>();          // the store that last read this slab has left it
                 __syncwarp();
                 t_chunk_to_slab(v, in_mask, slab + (uint32_t)(lane * 2), stats, sum, sumsq);
                 fence_proxy_async();
@@ -855,12 +856,13 @@ tc_conv_tp_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
         if (stats && co < p.c_out) {
             const float s1 = (sum[0] + sum[1]) + (sum[2] + sum[3]), s2 = (sumsq[0] + sumsq[1]) + (sumsq[2] + sumsq[3]);
             if (p.fold) {
-                const size_t blk = (size_t)first * 2 + co / p.fold;
+                const size_t blk = ((size_t)first * kTpEpi + half) * 2 + co / p.fold;
                 stat_partial[(blk * 2) * p.fold + co % p.fold] = s1;
                 stat_partial[(blk * 2 + 1) * p.fold + co % p.fold] = s2;
             } else {
-                stat_partial[((size_t)first * 2) * p.c_out + co] = s1;
-                stat_partial[((size_t)first * 2 + 1) * p.c_out + co] = s2;
+                const size_t row = (size_t)first * kTpEpi + half;
+                stat_partial[(row * 2) * p.c_out + co] = s1;
+                stat_partial[(row * 2 + 1) * p.c_out + co] = s2;
             }
         }
     }
@@ -2878,7 +2880,7 @@ int launch_t_core(TParams p, const void* x, int x_channels, const CUtensorMap& m
     }
     // partial row pairs per CTA: one per epilogue warp of a channel's quarter (the plain kernel has two), twice that
     // in the pixel-pair form
-    if (stat_blocks) *stat_blocks = stat_partial ? (p.fold ? 2 : 1) * (patch ? 1 : kTEpi) * p.ctas_per_co : 0;
+    if (stat_blocks) *stat_blocks = stat_partial ? (p.fold ? 2 : 1) * (patch ? kTpEpi : kTEpi) * p.ctas_per_co : 0;
     if (patch) {
         static bool tp_attr_set = false;
         if (!tp_attr_set) {
@@ -2887,8 +2889,8 @@ int launch_t_core(TParams p, const void* x, int x_channels, const CUtensorMap& m
             if (e != cudaSuccess) return cuda_fail(e, "raising the shared-memory limit");
             tp_attr_set = true;
         }
-        if (a_mn) tc_conv_tp_kernel<true><<<p.ctas_per_co * p.co_tiles, kThreads, kTpSmem, st>>>(mx, mw, mo, stat_blocks ? stat_partial : nullptr, p, status);
-        else tc_conv_tp_kernel<false><<<p.ctas_per_co * p.co_tiles, kThreads, kTpSmem, st>>>(mx, mw, mo, stat_blocks ? stat_partial : nullptr, p, status);
+        if (a_mn) tc_conv_tp_kernel<true><<<p.ctas_per_co * p.co_tiles, kTpThreads, kTpSmem, st>>>(mx, mw, mo, stat_blocks ? stat_partial : nullptr, p, status);
+        else tc_conv_tp_kernel<false><<<p.ctas_per_co * p.co_tiles, kTpThreads, kTpSmem, st>>>(mx, mw, mo, stat_blocks ? stat_partial : nullptr, p, status);
         CKPT_LAUNCH_CHECK_NAMED("tc_conv_tp_kernel", what);
         return CKPT_OK;
     }
