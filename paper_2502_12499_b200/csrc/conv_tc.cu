@@ -442,6 +442,9 @@ tc_conv_fwd_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_const
 // (64-byte rows: a lane's two bytes next to its neighbours') and adds the rounded values of the pixels inside the
 // tensor to the lane's batch-norm sums, kept in four interleaved partial sums so that consecutive additions do not
 // wait on one another.
+// PACKED: two values per conversion in the path with sums too (10 % on the epilogue-bound 1x1 layers; the halo-patch
+// kernel, whose epilogue hides under the MMAs, measured 3-8 % slower with it on its wide layers and keeps one each).
+template <bool PACKED>
 __device__ __forceinline__ void t_chunk_to_slab(const uint32_t (&v)[32], uint32_t in_mask, uint32_t slab_lane, bool stats, float (&sum)[4],
                                                 float (&sumsq)[4]) {
     if (!stats) {
@@ -451,6 +454,20 @@ __device__ __forceinline__ void t_chunk_to_slab(const uint32_t (&v)[32], uint32_
             const __nv_bfloat162 r = __floats2bfloat162_rn(__uint_as_float(v[e]), __uint_as_float(v[e + 1]));
             asm volatile("st.shared.b16 [%0], %1;" ::"r"(slab_lane + (uint32_t)(e * 64)), "h"(__bfloat16_as_ushort(r.x)) : "memory");
             asm volatile("st.shared.b16 [%0], %1;" ::"r"(slab_lane + (uint32_t)((e + 1) * 64)), "h"(__bfloat16_as_ushort(r.y)) : "memory");
+        }
+    } else if (in_mask == 0xffffffffu && PACKED) {
+#pragma unroll
+        for (int e = 0; e < 32; e += 2) {
+            // one conversion for two values; the rounded values come back as the two halves of the packed word
+            const __nv_bfloat162 r = __floats2bfloat162_rn(__uint_as_float(v[e]), __uint_as_float(v[e + 1]));
+            const uint32_t bits = *reinterpret_cast<const uint32_t*>(&r);
+            asm volatile("st.shared.b16 [%0], %1;" ::"r"(slab_lane + (uint32_t)(e * 64)), "h"(__bfloat16_as_ushort(r.x)) : "memory");
+            asm volatile("st.shared.b16 [%0], %1;" ::"r"(slab_lane + (uint32_t)((e + 1) * 64)), "h"(__bfloat16_as_ushort(r.y)) : "memory");
+            const float f0 = __uint_as_float(bits << 16), f1 = __uint_as_float(bits & 0xffff0000u);
+            sum[e & 3] += f0;
+            sumsq[e & 3] = fmaf(f0, f0, sumsq[e & 3]);
+            sum[(e + 1) & 3] += f1;
+            sumsq[(e + 1) & 3] = fmaf(f1, f1, sumsq[(e + 1) & 3]);
         }
     } else if (in_mask == 0xffffffffu) {
 #pragma unroll
@@ -650,7 +667,7 @@ tc_conv_t_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                 const uint32_t slab = out_stage + (uint32_t)(((warp - 2) * kTSlabs + (chunk_count % kTSlabs)) * 2048);
                 if (lane == 0) tma_store_wait_read<kTSlabs - 1>();    // the store that last read this slab has left it
                 __syncwarp();
-                t_chunk_to_slab(v, in_mask, slab + (uint32_t)(lane * 2), stats, sum, sumsq);
+                t_chunk_to_slab<true>(v, in_mask, slab + (uint32_t)(lane * 2), stats, sum, sumsq);
                 fence_proxy_async();
                 __syncwarp();
                 if (lane == 0 && in_mask != 0u && co_tile * 128 + quarter * 32 < p.c_out) {
@@ -839,7 +856,7 @@ tc_conv_tp_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
                 const uint32_t slab = out_stage + (uint32_t)((warp - 2) * 2048);
                 if (lane == 0) tma_store_wait_read<0>();          // the store that last read this slab has left it
                 __syncwarp();
-                t_chunk_to_slab(v, in_mask, slab + (uint32_t)(lane * 2), stats, sum, sumsq);
+                t_chunk_to_slab<false>(v, in_mask, slab + (uint32_t)(lane * 2), stats, sum, sumsq);
                 fence_proxy_async();
                 __syncwarp();
                 if (lane == 0 && in_mask != 0u && co_tile * 128 + quarter * 32 < p.c_out) {
