@@ -263,9 +263,9 @@ static int block_interiors(StepCtx& c, const Unit& u, const void* x, const Block
     return CKPT_OK;
 }
 
-static int block_forward(StepCtx& c, const Unit& u, const void* x, void* y) {
+static int block_forward(StepCtx& c, const Unit& u, const void* x, void* y, bool have_stats = false) {
     const BlockBuffers B = block_buffers(c, u);
-    int rc = block_interiors(c, u, x, B);
+    int rc = block_interiors(c, u, x, B, have_stats);
     if (rc) return rc;
     const bool project = (u.desc.flags & 2) != 0;
     return bn_add_relu(c.ch->dtype, c.ch->batch * u.out.h * u.out.w, u.out.c, B.z3, B.s3, project ? (const void*)B.zp : x,
@@ -308,7 +308,10 @@ static int block_backward(StepCtx& c, const Unit& u, const void* x, const void* 
 }
 
 // d_i = f_i(d_{i-1}, w_i)  (Eq. (1)); i is 1-based.
-static int unit_forward(StepCtx& c, int64_t i, const void* x_raw, void* y) {
+// recompute: the unit ran before in this step (segment recomputation of Algorithms 2 and 4).  Its output is a function of
+// the same inputs and parameters, so the batch statistics saved by its first run are the ones a second pass over the
+// output would find: the convolutions skip the sums in their epilogues and no finalize kernel runs.
+static int unit_forward(StepCtx& c, int64_t i, const void* x_raw, void* y, bool recompute = false) {
     if (c.dry) return CKPT_OK;
     const Unit& u = c.ch->units[i - 1];
     const int dt = c.ch->dtype;
@@ -319,14 +322,15 @@ static int unit_forward(StepCtx& c, int64_t i, const void* x_raw, void* y) {
     switch (u.desc.kind) {
         case CKPT_UNIT_CONV_BN_RELU:
             if ((rc = activated(c, i - 1, x_raw, &x))) return rc;
+            if (recompute) return conv_forward_any(c, u.geom, x, p[0], y, nullptr, 0);
             return conv_with_statistics(c, u.geom, x, p[0], y, (const float*)p[1], (const float*)p[2], stats_of(c, i));
         case CKPT_UNIT_CONV:
             if ((rc = activated(c, i - 1, x_raw, &x))) return rc;
             return conv_forward_any(c, u.geom, x, p[0], y, nullptr, 0);
         case CKPT_UNIT_BN:
             if ((rc = activated(c, i - 1, x_raw, &x))) return rc;
-            if ((rc = bn_statistics(dt, rows_of(c.ch, i), u.out.c, x, (const float*)p[0], (const float*)p[1], stats_of(c, i),
-                                    ws + c.ch->off_scr, c.stream))) return rc;
+            if (!recompute && (rc = bn_statistics(dt, rows_of(c.ch, i), u.out.c, x, (const float*)p[0], (const float*)p[1], stats_of(c, i),
+                                                  ws + c.ch->off_scr, c.stream))) return rc;
             return bn_apply(dt, rows_of(c.ch, i), u.out.c, x, stats_of(c, i), 0, y, c.stream);
         case CKPT_UNIT_RELU:
             if ((rc = activated(c, i - 1, x_raw, &x))) return rc;
@@ -348,7 +352,7 @@ static int unit_forward(StepCtx& c, int64_t i, const void* x_raw, void* y) {
             return conv_forward_any(c, u.geom, x, p[0], y, (const float*)p[1], u.desc.flags & 1);
         case CKPT_UNIT_BOTTLENECK:
             if ((rc = activated(c, i - 1, x_raw, &x))) return rc;
-            return block_forward(c, u, x, y);
+            return block_forward(c, u, x, y, recompute);
     }
     set_error("unit kind %d has no forward kernel", u.desc.kind);
     return CKPT_E_UNSUPPORTED;
@@ -550,7 +554,7 @@ static int run_step(StepCtx& c, double* loss_out) {
             }
             for (int64_t k = h + 1; k < i; ++k) {
                 if ((rc = A.alloc_stack(k, d[k], &off))) return rc;
-                if ((rc = unit_forward(c, k, ptr(k - 1), ptr(k)))) return rc;
+                if ((rc = unit_forward(c, k, ptr(k - 1), ptr(k), true))) return rc;
                 ++c.recomputed;
                 if (c.policy == CKPT_POLICY_STATIC) live_segment.push_back(k);
             }
