@@ -484,3 +484,43 @@ def sqrt_n_plan(n):
         step += 1
     C = [0] + [k for k in range(step, n, step)] + [n]
     return sorted(set(C))
+
+
+# --------------------------------------------------------------------------------------------
+# Least recomputation under a memory budget
+# --------------------------------------------------------------------------------------------
+# Section 3.1 minimises the peak alone, and many sets reach the optimum of Eq. (memory) (the 24-unit VGG-19 chain of
+# Section 5 has hundreds of thousands).  Which of them runs fastest is a second question: the backward pass of
+# Algorithm 4 recomputes every tensor that is not a checkpoint once, so the recomputation time of a set C is the sum of
+# cost[i] over the units i outside C (cost[i] = time of the forward of unit i).  The definition, by enumeration:
+
+def recompute_cost(cost, C):
+    """Sum of cost[i] over the units i = 1..n-1 that are not in C (d_0 and d_n are never recomputed)."""
+    n = len(cost) - 1
+    _check_set(n, C)
+    members = set(C)
+    return sum(cost[i] for i in range(1, n) if i not in members)
+
+
+def brute_force_min_recompute(d, cost, budget):
+    """Among all feasible sets whose Eq. (memory) value is at most `budget`, the least recomputation cost; returns
+    dict(cost, set, peak, feasible_sets) with one set that attains it (the first in enumeration order: fewer
+    checkpoints first, then lexicographic), or None when no set fits the budget."""
+    n = _check_sizes(d)
+    if len(cost) != n + 1 or any(c < 0 for c in cost):
+        raise ValueError("cost needs n + 1 non-negative entries")
+    best = None
+    feasible = 0
+    for inner in _all_sets(0, n):
+        C = (0,) + inner + (n,)
+        peak = eval_dynamic(d, C)
+        if peak > budget:
+            continue
+        feasible += 1
+        c = recompute_cost(cost, C)
+        if best is None or c < best["cost"]:
+            best = {"cost": c, "set": list(C), "peak": peak}
+    if best is None:
+        return None
+    best["feasible_sets"] = feasible
+    return best
