@@ -114,6 +114,20 @@ CKPT_API int ckpt_plan_sizes(int algo, int64_t n, const int64_t* kept, const int
 CKPT_API int ckpt_eval_sizes(int64_t n, const int64_t* kept, const int64_t* live, const int64_t* grad, int incoming,
                     const uint8_t* is_ckpt, int64_t* peak_bytes);
 
+/* Least recomputation under a memory budget (plan(layer sizes, layer costs) -> checkpoint set).  Section 3.1 asks for
+ * the smallest peak only, and many sets reach the optimum of Eq. (memory); the backward pass of Algorithm 4 runs the
+ * forward of every unit whose output is not a checkpoint a second time, so among the sets whose Eq. (memory) value is
+ * at most budget_bytes this call returns one with the smallest sum of cost[i] over the non-checkpoint units
+ * i = 1..n-1.  budget_bytes = 0 stands for the optimum of Algorithms 5/6 (same peak as ckpt_plan, fewer or cheaper
+ * recomputed units); a larger budget buys less recomputation.  Exact: a search over suffix plans that keeps, per
+ * checkpoint, the plans no other plan beats in both cost and tolerated prefix.
+ * d, cost: host, n+1 entries (cost[0] and cost[n] are not read; entries >= 0, any unit: ckpt_chain_unit_costs gives
+ * nanoseconds).  is_ckpt: host, n+1 entries written; *peak_bytes = Eq. (memory) of the returned set (<= budget);
+ * *recompute_cost = its recomputation cost.  Errors: as ckpt_plan, CKPT_E_BAD_ARG when a cost is negative or no set
+ * fits the budget. */
+CKPT_API int ckpt_plan_min_recompute(int64_t n, const int64_t* d, const int64_t* cost, int64_t budget_bytes, uint8_t* is_ckpt,
+                            int64_t* peak_bytes, int64_t* recompute_cost);
+
 /* ---------------------------------------------------------------- launch log (host only)
  *
  * Which kernels ran.  ckpt_launch_log(1) clears the log and starts counting every kernel the library launches, by
@@ -212,6 +226,9 @@ CKPT_API void ckpt_chain_destroy(ckpt_chain* chain);
 /* d: host, n+1 entries written (bytes, 256-aligned).  shapes (host, may be null): 3*(n+1) int32
  * {H, W, C} of d_0..d_n. */
 CKPT_API int ckpt_chain_sizes(const ckpt_chain* chain, int64_t* d, int32_t* shapes);
+/* cost_ns: host, n+1 entries written: a model of the time of each unit's forward pass (nanoseconds, from its
+ * arithmetic and memory traffic at nominal rates; entry 0 is 0), the layer costs ckpt_plan_min_recompute takes. */
+CKPT_API int ckpt_chain_unit_costs(const ckpt_chain* chain, int64_t* cost_ns);
 CKPT_API int ckpt_chain_num_params(const ckpt_chain* chain, int64_t* count);
 /* unit (1-based index of the owning unit), elems (element count), dtype (CKPT_DTYPE_* of the
  * parameter's storage; its gradient is always f32): host, written. */

@@ -123,6 +123,21 @@ def eval(model, d, is_ckpt):  # noqa: A001 - named after ckpt_eval
     return peak.value
 
 
+def plan_min_recompute(d, cost, budget=0):
+    """ckpt_plan_min_recompute: (is_ckpt mask, peak bytes, recomputation cost) of a set with the least recomputation
+    cost among those whose Eq. (memory) value is at most ``budget`` (0: the optimum of Algorithms 5/6)."""
+    d = np.ascontiguousarray(d, dtype=np.int64)
+    cost = np.ascontiguousarray(cost, dtype=np.int64)
+    if cost.shape != d.shape:
+        raise ValueError("cost needs one entry per tensor d_0..d_n")
+    n = d.size - 1
+    mask = np.zeros(n + 1, dtype=np.uint8)
+    peak, rec = C.c_int64(0), C.c_int64(0)
+    _check(lib().ckpt_plan_min_recompute(C.c_int64(n), _ptr(d, C.c_int64), _ptr(cost, C.c_int64), C.c_int64(int(budget)),
+                                         _ptr(mask, C.c_uint8), C.byref(peak), C.byref(rec)))
+    return mask, peak.value, rec.value
+
+
 def plan_sizes(algo, kept, live, grad, incoming=False):
     """ckpt_plan_sizes: returns (is_ckpt uint8[n+1], peak_bytes)."""
     kept, live, grad = _i64(kept), _i64(live), _i64(grad)
@@ -253,6 +268,12 @@ class Chain:
     def set_graph(self, enable):
         """ckpt_chain_set_graph: record the launch sequence of a repeated step once and replay it."""
         _check(lib().ckpt_chain_set_graph(self._h, C.c_int(1 if enable else 0)))
+
+    def unit_costs(self):
+        """ckpt_chain_unit_costs: modelled forward time of every unit in nanoseconds (entry 0 is 0)."""
+        out = np.zeros(self.n + 1, dtype=np.int64)
+        _check(lib().ckpt_chain_unit_costs(self._h, _ptr(out, C.c_int64)))
+        return out
 
     def staging_bytes(self):
         """ckpt_chain_staging_bytes: size of the two-slot staging buffer of ckpt_chain_stage_batch."""

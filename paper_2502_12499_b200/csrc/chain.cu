@@ -933,6 +933,41 @@ int ckpt_chain_sizes(const ckpt_chain* chain, int64_t* d, int32_t* shapes) {
     return CKPT_OK;
 }
 
+// Forward cost of every unit in nanoseconds from its arithmetic and its memory traffic at nominal rates (1.1 PFLOP/s
+// for the contractions, 5.5 TB/s for everything that streams a tensor): what a recomputation of the unit costs, for
+// ckpt_plan_min_recompute.  A model, not a measurement: only the order of magnitude between units matters.
+int ckpt_chain_unit_costs(const ckpt_chain* chain, int64_t* cost_ns) {
+    if (!chain || !cost_ns) { set_error("null pointer"); return CKPT_E_NULL; }
+    const double flop_per_ns = 1.1e6, byte_per_ns = 5.5e3;
+    auto conv_flops = [](const ConvGeom& g) { return 2.0 * g.n * g.ho * g.wo * g.cout * g.k * g.k * g.cin; };
+    cost_ns[0] = 0;
+    for (size_t i = 1; i < chain->d.size(); ++i) {
+        const Unit& u = chain->units[i - 1];
+        const double in_b = (double)chain->d[i - 1], out_b = (double)chain->d[i];
+        const bool pending = pending_act(chain, (int64_t)i - 1);       // the producer's normalisation is applied on the way in
+        double ns = 0;
+        switch (u.desc.kind) {
+            case CKPT_UNIT_CONV_BN_RELU:
+            case CKPT_UNIT_CONV:
+            case CKPT_UNIT_FC: {
+                const double w_b = (double)u.geom.cout * u.geom.k * u.geom.k * u.geom.cin * dtype_size(chain->dtype);
+                ns = conv_flops(u.geom) / flop_per_ns + ((pending ? 3.0 : 1.0) * in_b + out_b + w_b) / byte_per_ns;
+                break;
+            }
+            case CKPT_UNIT_BOTTLENECK: {
+                double fl = conv_flops(u.g1) + conv_flops(u.g2) + conv_flops(u.g3) + ((u.desc.flags & 2) ? conv_flops(u.gp) : 0.0);
+                // the 1x1 layers stream their tensors: input, three interior pairs, output and the residual join
+                ns = fl / flop_per_ns + (2.0 * in_b + 6.0 * out_b) / byte_per_ns;
+                break;
+            }
+            default:
+                ns = ((pending ? 1.0 : 1.0) * in_b + out_b) / byte_per_ns;
+        }
+        cost_ns[i] = (int64_t)(ns + 0.5) + 1000;        // plus a launch or two
+    }
+    return CKPT_OK;
+}
+
 int ckpt_chain_num_params(const ckpt_chain* chain, int64_t* count) {
     if (!chain || !count) { set_error("null pointer"); return CKPT_E_NULL; }
     *count = (int64_t)chain->params.size();

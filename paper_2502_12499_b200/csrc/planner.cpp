@@ -300,6 +300,64 @@ int plan_dynamic_n(int64_t n, const int64_t* d, uint8_t* is_ckpt, int64_t* peak,
     return plan_dynamic_n_sizes(n, z, is_ckpt, peak, work);
 }
 
+// ------------------------------------------------------------------------------------------------
+// Least recomputation under a memory budget.  Eq. (memory) of a set is the largest, over consecutive
+// checkpoints (i, j), of P_i + d_i + U(i,j) with P_i the sum of the checkpoints left of i (and P_n + d_n
+// at the end), so a suffix plan that starts at checkpoint i is described by two numbers: the cost of the
+// units it recomputes and the largest prefix sum R it tolerates.  G(i) keeps the plans no other plan
+// beats in both (cost up, R up along the list); a segment (i, j) maps a plan of G(j) to
+// (cost + sum of cost over i < k < j, min(budget - d_i - U(i,j), R - d_i)).  U(i,j) grows with j
+// (Lemma 1), so the scan over j stops at the first segment the budget cannot hold.  The answer is the
+// cheapest plan of G(0) (the prefix of d_0 is empty: R >= 0).
+// ------------------------------------------------------------------------------------------------
+static int64_t eval_sizes(int64_t n, const Sizes3& z, const uint8_t* is_ckpt);
+static inline int64_t eval_sizes_fwd(int64_t n, const Sizes3& z, const uint8_t* is_ckpt) { return eval_sizes(n, z, is_ckpt); }
+struct SuffixPlan { int64_t cost, room; int64_t next; int32_t next_plan; };
+
+int plan_min_recompute(int64_t n, const int64_t* d, const int64_t* cost, int64_t budget, uint8_t* is_ckpt, int64_t* peak,
+                       int64_t* recompute) {
+    std::vector<std::vector<SuffixPlan>> G(n + 1);
+    if (budget - d[n] >= 0) G[n].push_back({0, budget - d[n], -1, -1});
+    std::vector<SuffixPlan> cand;
+    for (int64_t i = n - 1; i >= 0; --i) {
+        cand.clear();
+        int64_t seg = 0, out_max = d[i], seg_cost = 0;
+        for (int64_t j = i + 1; j <= n; ++j) {
+            const int64_t cap = budget - d[i] - (seg + out_max + d[j]);
+            if (cap < 0) break;
+            for (size_t k = 0; k < G[j].size(); ++k) {
+                const int64_t room = std::min(cap, G[j][k].room - d[i]);
+                if (room >= 0) cand.push_back({G[j][k].cost + seg_cost, room, j, (int32_t)k});
+            }
+            seg += d[j];
+            out_max = std::max(out_max, d[j]);
+            seg_cost += cost[j];
+        }
+        // cheapest first; among equal costs the roomiest, then the nearest next checkpoint
+        std::sort(cand.begin(), cand.end(), [](const SuffixPlan& a, const SuffixPlan& b) {
+            if (a.cost != b.cost) return a.cost < b.cost;
+            if (a.room != b.room) return a.room > b.room;
+            return a.next < b.next;
+        });
+        int64_t best_room = -1;
+        for (const SuffixPlan& c : cand)
+            if (c.room > best_room) { G[i].push_back(c); best_room = c.room; }
+    }
+    if (G[0].empty()) { set_error("no checkpoint set fits a budget of %lld bytes", (long long)budget); return CKPT_E_BAD_ARG; }
+    for (int64_t i = 0; i <= n; ++i) is_ckpt[i] = 0;
+    int64_t i = 0;
+    int32_t k = 0;
+    while (i >= 0) {
+        is_ckpt[i] = 1;
+        const SuffixPlan& sp = G[i][k];
+        i = sp.next; k = sp.next_plan;
+    }
+    *recompute = G[0][0].cost;
+    const Sizes3 z{d, d, d, 0};
+    *peak = eval_sizes_fwd(n, z, is_ckpt);
+    return CKPT_OK;
+}
+
 // Generalised Eq. (memory) of a given set.
 static int64_t eval_sizes(int64_t n, const Sizes3& z, const uint8_t* is_ckpt) {
     int64_t worst = 0, kept_sum = z.kept[0], h = 0;
@@ -373,6 +431,25 @@ int ckpt_plan(int algo, int64_t n, const int64_t* d, uint8_t* is_ckpt, int64_t* 
 
 int ckpt_eval(int model, int64_t n, const int64_t* d, const uint8_t* is_ckpt, int64_t* peak_bytes) {
     return ckpt::eval_model(model, n, d, is_ckpt, peak_bytes);
+}
+
+int ckpt_plan_min_recompute(int64_t n, const int64_t* d, const int64_t* cost, int64_t budget_bytes, uint8_t* is_ckpt,
+                            int64_t* peak_bytes, int64_t* recompute_cost) {
+    int rc = ckpt::validate_sizes(n, d);
+    if (rc) return rc;
+    if (!cost || !is_ckpt || !peak_bytes || !recompute_cost) { ckpt::set_error("null pointer"); return CKPT_E_NULL; }
+    int64_t total = 0;
+    for (int64_t i = 1; i < n; ++i) {
+        if (cost[i] < 0) { ckpt::set_error("cost[%lld] is negative", (long long)i); return CKPT_E_BAD_ARG; }
+        if (cost[i] > std::numeric_limits<int64_t>::max() / 2 - total) { ckpt::set_error("sum of costs overflows int64"); return CKPT_E_OVERFLOW; }
+        total += cost[i];
+    }
+    if (budget_bytes < 0) { ckpt::set_error("negative budget"); return CKPT_E_BAD_ARG; }
+    if (budget_bytes == 0) {                 // the optimum of Eq. (memory)
+        std::vector<uint8_t> tmp(n + 1);
+        if ((rc = ckpt::plan_dynamic_n(n, d, tmp.data(), &budget_bytes, nullptr))) return rc;
+    }
+    return ckpt::plan_min_recompute(n, d, cost, budget_bytes, is_ckpt, peak_bytes, recompute_cost);
 }
 
 }  // extern "C"

@@ -247,6 +247,15 @@ def step_properties(spec, seed=0, finite_last_units=None):
         if finite_last_units is None or ui >= runner.n - finite_last_units:
             assert np.all(np.isfinite(a)), (ui, name)
         assert np.array_equal(a, b, equal_nan=True)     # checkpointed == store-all, bit for bit
+    # the set bench.py runs: same peak, least recomputation (the canonical set above when nothing is cheaper)
+    mask_mr, peak_mr, _ = ck.plan_min_recompute(d, runner.chain.unit_costs())
+    assert peak_mr == peak and int(mask_mr.sum()) >= int(mask.sum())
+    if not np.array_equal(mask_mr, mask):
+        rep_mr, g_mr = runner.run(ck.POLICY_DYNAMIC, mask_mr, x, labels)
+        assert rep_mr["peak_bytes"] == rep_mr["extent_bytes"] == rep_mr["predicted_bytes"] == peak
+        assert rep_mr["recomputed_units"] == runner.n + 1 - int(mask_mr.sum()) and rep_mr["loss"] == rep0["loss"]
+        for a, b in zip(g_mr, g0):
+            assert np.array_equal(a, b, equal_nan=True)
     mask3, peak3 = ck.plan(ck.ALGO_STATIC_N3, d)
     rep3, g3 = runner.run(ck.POLICY_STATIC, mask3, x, labels)
     assert rep3["peak_bytes"] == rep3["extent_bytes"] == peak3

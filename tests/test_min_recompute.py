@@ -68,3 +68,61 @@ def test_monotone_in_the_budget_and_consistent_with_the_optimum():
             c = po.brute_force_min_recompute(d, cost, budget)["cost"]
             assert last is None or c <= last
             last = c
+
+
+# ------------------------------------------------------------------------------------------------ library vs oracle
+
+def test_library_equals_enumeration():
+    rng = random.Random(12)
+    for trial in range(200):
+        n = rng.randint(1, 10)
+        d = [rng.randint(1, 40) for _ in range(n + 1)]
+        cost = [0] + [rng.randint(0, 25) for _ in range(n)]
+        optimum = po.brute_force_dynamic(d)["value"]
+        everything = po.eval_dynamic(d, list(range(n + 1)))
+        for budget in {0, optimum, optimum + rng.randint(0, 30), (optimum + everything) // 2, everything}:
+            want = po.brute_force_min_recompute(d, cost, optimum if budget == 0 else budget)
+            mask, peak, rec = ck.plan_min_recompute(d, cost, budget)
+            C = [int(i) for i in np.nonzero(mask)[0]]
+            assert rec == want["cost"], (d, cost, budget)
+            assert po.recompute_cost(cost, C) == rec
+            assert peak == po.eval_dynamic(d, C) <= (optimum if budget == 0 else budget)
+        if n >= 2:
+            with pytest.raises(ck.CkptError) as e:
+                ck.plan_min_recompute(d, cost, optimum - 1)
+            assert e.value.code == -6 and "budget" in str(e.value)
+
+
+def test_library_on_long_chains():
+    rng = random.Random(13)
+    for n in (60, 400):
+        d = [rng.randint(1, 1 << 20) for _ in range(n + 1)]
+        cost = [0] + [rng.randint(1, 1000) for _ in range(n)]
+        mask6, peak6 = ck.plan(ck.ALGO_DYNAMIC_N, d)
+        mask, peak, rec = ck.plan_min_recompute(d, cost)
+        assert peak <= peak6 and ck.eval(ck.MODEL_DYNAMIC, d, mask) == peak
+        assert rec == int(np.asarray(cost)[1:-1][mask[1:-1] == 0].sum())
+        assert rec <= int(np.asarray(cost)[1:-1][mask6[1:-1] == 0].sum())
+        # more room, less recomputation; the whole chain fits at the store-all-like peak of "every tensor a checkpoint"
+        looser = ck.plan_min_recompute(d, cost, int(peak6 * 1.3))[2]
+        assert looser <= rec
+        assert ck.plan_min_recompute(d, cost, ck.eval(ck.MODEL_DYNAMIC, d, np.ones(n + 1, dtype=np.uint8)))[2] == 0
+
+
+def test_library_errors_and_chain_costs():
+    with pytest.raises(ck.CkptError) as e:
+        ck.plan_min_recompute([1, 2, 3], [0, -1, 0])
+    assert e.value.code == -6
+    with pytest.raises(ck.CkptError) as e:
+        ck.plan_min_recompute([1, 0, 3], [0, 1, 0])
+    assert e.value.code == -3
+    from paper_2502_12499_b200 import workloads as wl
+    chain = ck.Chain(wl.config(2))
+    cost = chain.unit_costs()
+    assert cost[0] == 0 and np.all(cost[1:] > 0)
+    # the second 3x3 layer at 224 x 224 is the most expensive unit of the VGG-16 chain, the pools are cheap
+    assert int(np.argmax(cost)) == 2 and cost[3] < cost[2] / 3
+    d = chain.sizes()
+    mask6, peak6 = ck.plan(ck.ALGO_DYNAMIC_N, d)
+    mask, peak, rec = ck.plan_min_recompute(d, cost)
+    assert peak == peak6 and int(mask.sum()) > int(mask6.sum())
