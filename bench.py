@@ -216,6 +216,7 @@ def measure_config(spec, args, rank, world, steps, regions, with_roofline, peaks
     labels_pinned = torch.from_numpy(labels_h).pin_memory()
     x_dev, labels_dev = x_pinned.cuda(), labels_pinned.cuda()
     ws_bytes = chain.workspace_bytes()
+    ws_plan = chain.workspace_bytes_for(ck.POLICY_DYNAMIC)       # Algorithm 4 needs no buffer for activated copies
     workspace = torch.empty(ws_bytes, dtype=torch.uint8, device="cuda")
     stream = torch.cuda.current_stream()
 
@@ -302,8 +303,8 @@ def measure_config(spec, args, rank, world, steps, regions, with_roofline, peaks
                                "recompute_overhead_pct": 100.0 * (ms_canon / ms_all - 1.0)},
            "launches_per_step": int(rep["launches"]), "store_all_launches_per_step": int(rep_all["launches"]),
            "memory_gib": {"arena_plan": peak / gib, "arena_store_all": store_all / gib, "arena_measured": rep["peak_bytes"] / gib,
-                          "workspace": ws_bytes / gib, "parameters_and_gradients": param_bytes / gib,
-                          "total_plan": (peak + ws_bytes + param_bytes) / gib, "total_store_all": (store_all + ws_bytes + param_bytes) / gib},
+                          "workspace": ws_plan / gib, "workspace_store_all": ws_bytes / gib, "parameters_and_gradients": param_bytes / gib,
+                          "total_plan": (peak + ws_plan + param_bytes) / gib, "total_store_all": (store_all + ws_bytes + param_bytes) / gib},
            "peak_bytes": int(rep["peak_bytes"]), "predicted_bytes": int(peak), "store_all_bytes": int(store_all),
            "planner_us": planner_us, "loss": rep["loss"],
            "step_tflops": flops / (ms * 1e-3) / 1e12, "step_tensor_frac_of_sustained": flops / (ms * 1e-3) / 1e12 / peaks["tflops_sustained"],

@@ -238,6 +238,11 @@ CKPT_API int ckpt_chain_param_info(const ckpt_chain* chain, int64_t p, int64_t* 
  * pre-normalisation buffer that each unit's backward re-derives, split-K partial sums, saved
  * batch statistics.  bytes: host, written. */
 CKPT_API int ckpt_chain_workspace_bytes(const ckpt_chain* chain, int64_t* bytes);
+/* The same for one schedule (policy as in ckpt_train_step).  Algorithm 4's schedule (CKPT_POLICY_DYNAMIC) places the
+ * activated copy of a unit's input in whichever of its gradient buffers is idle at that moment and needs no buffer
+ * of its own for it: its workspace is a prefix of the full one, shorter by the largest such copy.  ckpt_train_step
+ * accepts a workspace of this size for that policy.  Errors: CKPT_E_NULL, CKPT_E_BAD_ARG (policy). */
+CKPT_API int ckpt_chain_workspace_bytes_for(const ckpt_chain* chain, int policy, int64_t* bytes);
 /* Kernel selection for dense contractions: 0 = automatic (tensor cores where a kernel exists),
  * 1 = plain CUDA-core kernels only. */
 CKPT_API int ckpt_chain_set_impl(ckpt_chain* chain, int impl);
@@ -306,7 +311,7 @@ CKPT_API int ckpt_chain_set_selftest(ckpt_chain* chain, int wait_runs_out);
  * grads:   host array of device pointers (float32), written.
  * arena:   device, arena_bytes >= ckpt_eval(model of policy) or CKPT_E_ARENA_OOM is returned before
  *          anything is launched.  Contents on return are unspecified.
- * workspace: device, ws_bytes >= ckpt_chain_workspace_bytes().
+ * workspace: device, ws_bytes >= ckpt_chain_workspace_bytes_for(policy) (ckpt_chain_workspace_bytes() fits every policy).
  * stream:  a cudaStream_t (null = default stream).  The call returns after the stream has drained.
  * report:  host, written.
  * Determinism: every reduction has a fixed order, so gradients are bit-identical across policies

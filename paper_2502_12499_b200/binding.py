@@ -250,6 +250,12 @@ class Chain:
         _check(lib().ckpt_chain_workspace_bytes(self._h, C.byref(b)))
         return b.value
 
+    def workspace_bytes_for(self, policy):
+        """ckpt_chain_workspace_bytes_for: the workspace one schedule needs (Algorithm 4's is shorter)."""
+        b = C.c_int64(0)
+        _check(lib().ckpt_chain_workspace_bytes_for(self._h, C.c_int(policy), C.byref(b)))
+        return b.value
+
     def set_impl(self, impl):
         _check(lib().ckpt_chain_set_impl(self._h, C.c_int(impl)))
 

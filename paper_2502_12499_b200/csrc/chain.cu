@@ -104,6 +104,7 @@ struct StepCtx {
     int64_t recomputed = 0;
     int64_t* stage_trace = nullptr;     // optional: live arena bytes at the end of each of the 2n+2 stages
     void* host_result = nullptr;        // capture: pinned destination of the loss and the status word (no wait)
+    char* act_buf = nullptr;            // where the activated copy of a unit's input goes (null: the workspace's own buffer)
     int* status() const { return (int*)(ws + ch->off_misc + 64); }
 };
 
@@ -203,7 +204,7 @@ static int64_t rows_of(const ckpt_chain* ch, int64_t j) { return ch->batch * ch-
 static int activated(StepCtx& c, int64_t j, const void* raw, const void** out) {
     *out = raw;
     if (!pending_act(c.ch, j)) return CKPT_OK;
-    void* xbuf = c.ws + c.ch->off_z;
+    void* xbuf = c.act_buf ? c.act_buf : c.ws + c.ch->off_z;
     *out = xbuf;
     return bn_apply(c.ch->dtype, rows_of(c.ch, j), c.ch->shapes[j].c, raw, stats_of(c, j), 1, xbuf, c.stream);
 }
@@ -478,6 +479,20 @@ static int run_step(StepCtx& c, double* loss_out) {
     int rc;
     int64_t off;
 
+    // Activated copies under Algorithm 4: a backward hop has its gradient in one of {segment buffer, carry 0, carry 1}
+    // and writes the next one into another, so the third is idle and takes the activated copy of the unit's input
+    // (the segment's buffer is at least as large as every tensor of the segment, the carry buffers as the largest
+    // tensor of the chain); forward and recomputation have at most one gradient alive.  The workspace's own buffer
+    // for that copy is then never touched.
+    const bool lean = c.policy == CKPT_POLICY_DYNAMIC && !c.dry;
+    char* const carry[2] = {c.dry ? nullptr : c.ws + ch->off_g0, c.dry ? nullptr : c.ws + ch->off_g1};
+    auto idle_buffer = [&](const void* busy_a, const void* busy_b, char* segment_buffer) -> char* {
+        for (char* cand : {carry[1], carry[0]})
+            if (cand != busy_a && cand != busy_b) return cand;
+        return segment_buffer;
+    };
+    if (lean) c.act_buf = carry[1];
+
     // ---------------- forward phase
     if ((rc = A.alloc_stack(0, d[0], &off))) return rc;
     if (c.stage_trace) c.stage_trace[0] = A.live_bytes();
@@ -552,6 +567,7 @@ static int run_step(StepCtx& c, double* loss_out) {
                 for (int64_t k : live_segment) if ((rc = A.release(k))) return rc;
                 live_segment.clear();
             }
+            if (lean) c.act_buf = idle_buffer(g_cur, nullptr, nullptr);
             for (int64_t k = h + 1; k < i; ++k) {
                 if ((rc = A.alloc_stack(k, d[k], &off))) return rc;
                 if ((rc = unit_forward(c, k, ptr(k - 1), ptr(k), true))) return rc;
@@ -577,6 +593,7 @@ static int run_step(StepCtx& c, double* loss_out) {
         else g_next = (g_cur == gbuf[0]) ? gbuf[1] : gbuf[0];
         bypass_r_once = false;
         const bool need_dx = i > 1;   // the gradient w.r.t. the input batch is never used
+        if (lean) c.act_buf = idle_buffer(g_cur, need_dx ? g_next : nullptr, have_r ? (char*)ptr(kGradId) : nullptr);
         if ((rc = unit_backward(c, i, ptr(i - 1), ptr(i), g_cur, need_dx ? g_next : nullptr))) return rc;
         if (need_dx) {
             g_cur = g_next; g_in_r = next_in_r;
@@ -912,11 +929,13 @@ int ckpt_chain_create(const ckpt_unit_desc* units, int64_t n, int64_t batch, int
     int64_t o = 0;
     ch->off_g0 = o; o += ch->max_d;
     ch->off_g1 = o; o += ch->max_d;
-    ch->off_z = o; o += std::max<int64_t>(max_z, 256);
     ch->off_scr = o; ch->scr_bytes = align_up(scr, 256); o += ch->scr_bytes;
     ch->off_stats = o; o += align_up(std::max<int64_t>(stats_floats, 1) * 4, 256);
     ch->off_misc = o; o += align_up(128 + 256 + batch * 4, 256);
     ch->off_blk = o; o += ch->blk_bytes;
+    // last: the buffer of the activated copy.  Algorithm 4's schedule never needs it (see run_step) and takes a
+    // workspace that ends here
+    ch->off_z = o; o += std::max<int64_t>(max_z, 256);
     ch->ws_bytes = o;
     *out = ch;
     return CKPT_OK;
@@ -983,6 +1002,13 @@ int ckpt_chain_param_info(const ckpt_chain* chain, int64_t p, int64_t* unit, int
     return CKPT_OK;
 }
 
+int ckpt_chain_workspace_bytes_for(const ckpt_chain* chain, int policy, int64_t* bytes) {
+    if (!chain || !bytes) { set_error("null pointer"); return CKPT_E_NULL; }
+    if (policy < 0 || policy > 2) { set_error("unknown policy %d", policy); return CKPT_E_BAD_ARG; }
+    *bytes = policy == CKPT_POLICY_DYNAMIC ? chain->off_z : chain->ws_bytes;
+    return CKPT_OK;
+}
+
 int ckpt_chain_workspace_bytes(const ckpt_chain* chain, int64_t* bytes) {
     if (!chain || !bytes) { set_error("null pointer"); return CKPT_E_NULL; }
     *bytes = chain->ws_bytes;
@@ -1017,8 +1043,10 @@ int ckpt_train_step(ckpt_chain* chain, const uint8_t* is_ckpt, int policy, const
         set_error("arena of %lld bytes is smaller than the plan's peak of %lld bytes", (long long)arena_bytes, (long long)predicted);
         return CKPT_E_ARENA_OOM;
     }
-    if (ws_bytes < chain->ws_bytes) {
-        set_error("workspace of %lld bytes, %lld needed", (long long)ws_bytes, (long long)chain->ws_bytes);
+    const int64_t ws_need = policy == CKPT_POLICY_DYNAMIC ? chain->off_z : chain->ws_bytes;
+    report->workspace_bytes = ws_need;
+    if (ws_bytes < ws_need) {
+        set_error("workspace of %lld bytes, %lld needed", (long long)ws_bytes, (long long)ws_need);
         return CKPT_E_WORKSPACE;
     }
     int ndev = 0;

@@ -256,6 +256,21 @@ def step_properties(spec, seed=0, finite_last_units=None):
         assert rep_mr["recomputed_units"] == runner.n + 1 - int(mask_mr.sum()) and rep_mr["loss"] == rep0["loss"]
         for a, b in zip(g_mr, g0):
             assert np.array_equal(a, b, equal_nan=True)
+    # Algorithm 4's schedule in the shorter workspace it asks for (no buffer for activated copies), filled with NaN patterns
+    full_ws = runner.workspace
+    lean_bytes = runner.chain.workspace_bytes_for(ck.POLICY_DYNAMIC)
+    assert lean_bytes <= runner.chain.workspace_bytes_for(ck.POLICY_STORE_ALL) == runner.chain.workspace_bytes()
+    runner.workspace = torch.empty(lean_bytes, dtype=torch.uint8, device="cuda")
+    runner.workspace.fill_(0xFF)
+    rep_lean, g_lean = runner.run(ck.POLICY_DYNAMIC, mask_mr, x, labels)
+    assert rep_lean["peak_bytes"] == peak and rep_lean["workspace_bytes"] == lean_bytes and rep_lean["loss"] == rep0["loss"]
+    for a, b in zip(g_lean, g0):
+        assert np.array_equal(a, b, equal_nan=True)
+    if lean_bytes < runner.chain.workspace_bytes():
+        with pytest.raises(ck.CkptError) as e:
+            runner.run(ck.POLICY_STORE_ALL, None, x, labels)
+        assert e.value.code == -8
+    runner.workspace = full_ws
     mask3, peak3 = ck.plan(ck.ALGO_STATIC_N3, d)
     rep3, g3 = runner.run(ck.POLICY_STATIC, mask3, x, labels)
     assert rep3["peak_bytes"] == rep3["extent_bytes"] == peak3

@@ -317,3 +317,9 @@ def test_chain_option_errors_need_no_device():
                                       C.byref(out_l)) == -1 and "labels" in lib.ckpt_last_error().decode()
     assert args(1, fake, fake, need_stage - 1) == -8 and "staging" in lib.ckpt_last_error().decode()
     assert lib.ckpt_chain_staging_bytes(chain._h, None) == -1
+    # workspace per schedule: Algorithm 4's is a prefix of the full one
+    assert chain.workspace_bytes_for(ck.POLICY_STORE_ALL) == chain.workspace_bytes_for(ck.POLICY_STATIC) == chain.workspace_bytes()
+    assert 0 < chain.workspace_bytes_for(ck.POLICY_DYNAMIC) < chain.workspace_bytes()
+    out_bytes = C.c_int64(0)
+    assert lib.ckpt_chain_workspace_bytes_for(chain._h, C.c_int(3), C.byref(out_bytes)) == -6
+    assert lib.ckpt_chain_workspace_bytes_for(chain._h, C.c_int(2), None) == -1
