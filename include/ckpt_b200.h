@@ -239,8 +239,9 @@ CKPT_API int ckpt_chain_param_info(const ckpt_chain* chain, int64_t p, int64_t* 
  * batch statistics.  bytes: host, written. */
 CKPT_API int ckpt_chain_workspace_bytes(const ckpt_chain* chain, int64_t* bytes);
 /* The same for one schedule (policy as in ckpt_train_step).  Algorithm 4's schedule (CKPT_POLICY_DYNAMIC) places the
- * activated copy of a unit's input in whichever of its gradient buffers is idle at that moment and needs no buffer
- * of its own for it: its workspace is a prefix of the full one, shorter by the largest such copy.  ckpt_train_step
+ * activated copy of a unit's input, and the last pre-normalisation tensor of a residual block, in whichever of its
+ * gradient buffers is idle at that moment and needs no buffer of its own for them: its workspace is a prefix of the
+ * full one.  ckpt_train_step
  * accepts a workspace of this size for that policy.  Errors: CKPT_E_NULL, CKPT_E_BAD_ARG (policy). */
 CKPT_API int ckpt_chain_workspace_bytes_for(const ckpt_chain* chain, int policy, int64_t* bytes);
 /* Kernel selection for dense contractions: 0 = automatic (tensor cores where a kernel exists),

@@ -19,6 +19,7 @@ struct Unit {
     Shape in, out;
     int param_first = 0, n_params = 0;
     int64_t stats_off = 0;       // float offset of this unit's saved batch statistics
+    bool in_pending = false;     // the unit's input is a conv+BN+ReLU unit's stored output (normalisation applied on the way in)
     ConvGeom geom;               // conv / fc as a convolution
     // bottleneck block: its four convolutions (1x1, 3x3 with the stride, 1x1, projection 1x1 with the stride)
     ConvGeom g1, g2, g3, gp;
@@ -47,7 +48,7 @@ struct ckpt_chain {
     int dtype = 0, loss = 0, impl = 0;
     // workspace layout (byte offsets)
     int64_t max_d = 0, off_g0 = 0, off_g1 = 0, off_z = 0, off_scr = 0, scr_bytes = 0, off_stats = 0,
-            off_misc = 0, off_blk = 0, blk_bytes = 0, ws_bytes = 0;
+            off_misc = 0, off_blk = 0, blk_bytes = 0, blk_lean_bytes = 0, ws_bytes = 0;
     // graph replay: steps captured once per distinct argument set (pointers, plan, policy)
     int use_graph = 0;
     std::vector<ckpt::StepGraph> graphs;
@@ -105,6 +106,7 @@ struct StepCtx {
     int64_t* stage_trace = nullptr;     // optional: live arena bytes at the end of each of the 2n+2 stages
     void* host_result = nullptr;        // capture: pinned destination of the loss and the status word (no wait)
     char* act_buf = nullptr;            // where the activated copy of a unit's input goes (null: the workspace's own buffer)
+    int64_t act_cap = 0;                // its capacity in bytes
     int* status() const { return (int*)(ws + ch->off_misc + 64); }
 };
 
@@ -226,13 +228,19 @@ static BlockBuffers block_buffers(StepCtx& c, const Unit& u) {
     const int64_t c_out = align_up(out_px * u.out.c * es, 256);
     BlockBuffers B;
     char* p = c.ws + c.ch->off_blk;
+    const bool project = (u.desc.flags & 2) != 0;
     B.z1 = p; p += m_in; B.a = p; p += m_in; B.da = p; p += m_in;
     B.z2 = p; p += m_out; B.b = p; p += m_out; B.db = p; p += m_out;
-    B.z3 = p; p += c_out; B.zp = p; p += c_out;
+    // projection branch: its pre-normalisation output and the gradient with respect to the block's input through it
+    B.zp = project ? p : nullptr; if (project) p += c_out;
+    B.dxs = project ? p : nullptr; if (project) p += align_up(in_px * u.in.c * es, 256);
+    // z3 last: where an idle gradient buffer is at hand (Algorithm 4's schedule, see run_step) z3 lives there and
+    // the block region ends here
+    if (c.act_buf && !u.in_pending && c.act_cap >= c_out) B.z3 = c.act_buf;
+    else B.z3 = p;
     // the gradients with respect to z3 and zp are written over z3 and zp themselves (the batch-norm backward reads an
     // element of z and of the incoming gradient and writes the same element; nothing reads z3 or zp afterwards)
     B.t1 = B.z3; B.t0 = B.zp;
-    B.dxs = p;
     float* st = (float*)(c.ws + c.ch->off_stats) + u.stats_off;
     B.s1 = st; B.s2 = st + 4 * u.desc.mid; B.s3 = st + 8 * u.desc.mid; B.sp = B.s3 + 4 * u.out.c;
     return B;
@@ -491,7 +499,7 @@ static int run_step(StepCtx& c, double* loss_out) {
             if (cand != busy_a && cand != busy_b) return cand;
         return segment_buffer;
     };
-    if (lean) c.act_buf = carry[1];
+    if (lean) { c.act_buf = carry[1]; c.act_cap = ch->max_d; }
 
     // ---------------- forward phase
     if ((rc = A.alloc_stack(0, d[0], &off))) return rc;
@@ -546,6 +554,7 @@ static int run_step(StepCtx& c, double* loss_out) {
 
     // ---------------- backward phase
     bool have_r = false;            // Algorithm 4: a per-segment gradient buffer is live in the arena
+    int64_t r_bytes = 0;            // its size
     bool g_in_r = false;            // the current gradient lives in that buffer
     bool bypass_r_once = false;     // first hop of a segment with an odd number of hops goes carry -> carry
     std::vector<int64_t> live_segment;
@@ -567,7 +576,7 @@ static int run_step(StepCtx& c, double* loss_out) {
                 for (int64_t k : live_segment) if ((rc = A.release(k))) return rc;
                 live_segment.clear();
             }
-            if (lean) c.act_buf = idle_buffer(g_cur, nullptr, nullptr);
+            if (lean) { c.act_buf = idle_buffer(g_cur, nullptr, nullptr); c.act_cap = ch->max_d; }
             for (int64_t k = h + 1; k < i; ++k) {
                 if ((rc = A.alloc_stack(k, d[k], &off))) return rc;
                 if ((rc = unit_forward(c, k, ptr(k - 1), ptr(k), true))) return rc;
@@ -579,10 +588,15 @@ static int run_step(StepCtx& c, double* loss_out) {
                 for (int64_t k = h; k < i; ++k) r = std::max(r, d[k]);
                 if ((rc = A.alloc_stack(kGradId, r, &off))) return rc;
                 have_r = true;
+                r_bytes = r;
                 // The gradient alternates between the segment's buffer and a carry buffer, one hop per
                 // unit.  It has to sit in a carry buffer when the segment ends (its buffer is released
                 // then), so a segment with an odd number of hops starts with one carry -> carry hop.
                 bypass_r_once = h > 0 && ((i - h) % 2 == 1);
+                // a carry -> carry hop leaves only the segment's buffer idle; a residual block keeps a tensor of its
+                // output's size there, so the hop is taken only when that fits (otherwise the gradient is copied out
+                // of the segment's buffer when the segment ends)
+                if (bypass_r_once && ch->units[i - 1].desc.kind == CKPT_UNIT_BOTTLENECK && r < d[i]) bypass_r_once = false;
             }
         }
         // where the outgoing gradient goes: the segment's buffer (Algorithm 4) or the other carry buffer
@@ -593,7 +607,10 @@ static int run_step(StepCtx& c, double* loss_out) {
         else g_next = (g_cur == gbuf[0]) ? gbuf[1] : gbuf[0];
         bypass_r_once = false;
         const bool need_dx = i > 1;   // the gradient w.r.t. the input batch is never used
-        if (lean) c.act_buf = idle_buffer(g_cur, need_dx ? g_next : nullptr, have_r ? (char*)ptr(kGradId) : nullptr);
+        if (lean) {
+            c.act_buf = idle_buffer(g_cur, need_dx ? g_next : nullptr, have_r ? (char*)ptr(kGradId) : nullptr);
+            c.act_cap = (c.act_buf == carry[0] || c.act_buf == carry[1]) ? ch->max_d : r_bytes;
+        }
         if ((rc = unit_backward(c, i, ptr(i - 1), ptr(i), g_cur, need_dx ? g_next : nullptr))) return rc;
         if (need_dx) {
             g_cur = g_next; g_in_r = next_in_r;
@@ -908,9 +925,12 @@ int ckpt_chain_create(const ckpt_unit_desc* units, int64_t n, int64_t batch, int
                 stats_floats += 4 * (int64_t)(2 * mid + 2 * co);
                 // interiors and gradient temporaries of one block (see block_buffers)
                 const int64_t in_px = batch * cur.h * cur.w, out_px = batch * ho * wo;
-                const int64_t blk = 3 * align_up(in_px * mid * es, 256) + 3 * align_up(out_px * mid * es, 256) +
-                                    2 * align_up(out_px * co * es, 256) + align_up(in_px * cur.c * es, 256);
+                const int64_t z3_bytes = align_up(out_px * co * es, 256);
+                const int64_t blk = 3 * align_up(in_px * mid * es, 256) + 3 * align_up(out_px * mid * es, 256) + z3_bytes +
+                                    (project ? z3_bytes + align_up(in_px * cur.c * es, 256) : 0);
+                u.in_pending = i >= 2 && units[i - 2].kind == CKPT_UNIT_CONV_BN_RELU;
                 ch->blk_bytes = std::max(ch->blk_bytes, blk);
+                ch->blk_lean_bytes = std::max(ch->blk_lean_bytes, u.in_pending ? blk : blk - z3_bytes);
                 break;
             }
             default:
@@ -1005,7 +1025,7 @@ int ckpt_chain_param_info(const ckpt_chain* chain, int64_t p, int64_t* unit, int
 int ckpt_chain_workspace_bytes_for(const ckpt_chain* chain, int policy, int64_t* bytes) {
     if (!chain || !bytes) { set_error("null pointer"); return CKPT_E_NULL; }
     if (policy < 0 || policy > 2) { set_error("unknown policy %d", policy); return CKPT_E_BAD_ARG; }
-    *bytes = policy == CKPT_POLICY_DYNAMIC ? chain->off_z : chain->ws_bytes;
+    *bytes = policy == CKPT_POLICY_DYNAMIC ? chain->off_blk + chain->blk_lean_bytes : chain->ws_bytes;
     return CKPT_OK;
 }
 
@@ -1043,7 +1063,7 @@ int ckpt_train_step(ckpt_chain* chain, const uint8_t* is_ckpt, int policy, const
         set_error("arena of %lld bytes is smaller than the plan's peak of %lld bytes", (long long)arena_bytes, (long long)predicted);
         return CKPT_E_ARENA_OOM;
     }
-    const int64_t ws_need = policy == CKPT_POLICY_DYNAMIC ? chain->off_z : chain->ws_bytes;
+    const int64_t ws_need = policy == CKPT_POLICY_DYNAMIC ? chain->off_blk + chain->blk_lean_bytes : chain->ws_bytes;
     report->workspace_bytes = ws_need;
     if (ws_bytes < ws_need) {
         set_error("workspace of %lld bytes, %lld needed", (long long)ws_bytes, (long long)ws_need);
