@@ -279,12 +279,24 @@ def measure_config(spec, args, rank, world, steps, regions, with_roofline, peaks
     del arena
     arena_all = torch.empty(store_all, dtype=torch.uint8, device="cuda")
     all_ms, rep_all = timed_regions(ck.POLICY_STORE_ALL, None, arena_all, x_dev, labels_dev, warm)
+    # Algorithm 1 literally: residual blocks keep their interior tensors as well (a region per block in the workspace)
+    kept_ms, ws_kept = None, ws_bytes
+    if any(u["kind"] == "bottleneck" for u in spec["units"]):
+        chain.set_keep_interiors(True)
+        ws_kept = chain.workspace_bytes()
+        workspace = None
+        torch.cuda.empty_cache()
+        workspace = torch.empty(ws_kept, dtype=torch.uint8, device="cuda")
+        kept_ms, rep_kept = timed_regions(ck.POLICY_STORE_ALL, None, arena_all, x_dev, labels_dev, warm)
+        assert rep_kept["loss"] == rep_all["loss"]
+        chain.set_keep_interiors(False)
     del arena_all
 
     med = lambda v: float(sorted(v)[len(v) // 2])  # noqa: E731
     ms, ms_e2e, ms_all = med(ckpt_ms) / steps, med(e2e_ms) / steps, med(all_ms) / steps
     ms_e2e_sync = med(e2e_sync_ms) / steps
     ms_canon = med(canon_ms) / steps
+    ms_kept = med(kept_ms) / steps if kept_ms else None
     flops, _ = conv_flops(spec, mask, shapes)
     gib = 2.0 ** 30
     out = {"workload": workload_name(spec), "n_units": len(spec["units"]), "batch": spec["batch"], "steps": steps,
@@ -296,7 +308,12 @@ def measure_config(spec, args, rank, world, steps, regions, with_roofline, peaks
            "h2d_bytes_per_step": int(x_pinned.numel() * x_pinned.element_size() + labels_pinned.numel() * 4), "d2h_bytes_per_step": 12,
            "store_all_ms_per_step": ms_all, "store_all_images_per_s": whole_job_images_per_s(spec["batch"], world, 1, ms_all),
            "recompute_overhead_pct": 100.0 * (ms / ms_all - 1.0),
-           "store_all_note": "residual blocks re-derive their interior tensors in the backward under every schedule, store-all included",
+           "store_all_note": "residual blocks re-derive their interior tensors in the backward under every schedule, store-all included; "
+                             "store_all_keeping_interiors is Algorithm 1 taken literally (every block keeps its interiors in the workspace)",
+           "store_all_keeping_interiors": None if ms_kept is None else {
+               "ms_per_step": ms_kept, "images_per_s": whole_job_images_per_s(spec["batch"], world, 1, ms_kept),
+               "recompute_overhead_pct": 100.0 * (ms / ms_kept - 1.0), "workspace_gib": ws_kept / 2.0 ** 30,
+               "total_gib": (store_all + ws_kept + param_bytes) / 2.0 ** 30},
            "recomputed_units": int(rep["recomputed_units"]), "checkpoints": int(mask.sum()),
            "algorithm_6_set": {"ms_per_step": ms_canon, "recomputed_units": int(rep_canon["recomputed_units"]),
                                "checkpoints": int(mask_canonical.sum()), "peak_bytes": int(rep_canon["peak_bytes"]),
@@ -437,6 +454,7 @@ def main():
                 "peak_gib": head["memory_gib"]["arena_measured"], "workspace_gib": head["memory_gib"]["workspace"],
                 "memory_gib": head["memory_gib"], "store_all_ms_per_step": head["store_all_ms_per_step"],
                 "recompute_overhead_pct": head["recompute_overhead_pct"], "recomputed_units": head["recomputed_units"],
+                "store_all_keeping_interiors": head["store_all_keeping_interiors"], "algorithm_6_set": head["algorithm_6_set"],
                 "planner_us": head["planner_us"], "loss": head["loss"], "step_tflops": head["step_tflops"],
                 "step_tensor_frac_of_sustained": head["step_tensor_frac_of_sustained"], "peaks": peaks}
         if "roofline" in head:

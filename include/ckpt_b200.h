@@ -244,6 +244,15 @@ CKPT_API int ckpt_chain_workspace_bytes(const ckpt_chain* chain, int64_t* bytes)
  * full one.  ckpt_train_step
  * accepts a workspace of this size for that policy.  Errors: CKPT_E_NULL, CKPT_E_BAD_ARG (policy). */
 CKPT_API int ckpt_chain_workspace_bytes_for(const ckpt_chain* chain, int policy, int64_t* bytes);
+/* Algorithm 1 taken literally for residual blocks (off by default).  A block's output is the only chain tensor of the
+ * block, and by default every schedule re-derives the block's interior tensors from its input at the start of the
+ * block's backward - store-all included, which therefore already pays one extra forward of every block.  With
+ * enable = 1 a CKPT_POLICY_STORE_ALL step gives every block a region of its own in the workspace, keeps the interiors
+ * from the forward pass and re-derives nothing: the step time of a schedule that stores everything, against which the
+ * recomputation overhead of the checkpointed schedules is measured.  The other policies are unaffected.  The
+ * workspace of the store-all policy grows by the sum of all blocks' regions (ckpt_chain_workspace_bytes and
+ * ckpt_chain_workspace_bytes_for report it); gradients are bit-identical either way.  Drops recorded graphs. */
+CKPT_API int ckpt_chain_set_keep_interiors(ckpt_chain* chain, int enable);
 /* Kernel selection for dense contractions: 0 = automatic (tensor cores where a kernel exists),
  * 1 = plain CUDA-core kernels only. */
 CKPT_API int ckpt_chain_set_impl(ckpt_chain* chain, int impl);

@@ -256,6 +256,10 @@ class Chain:
         _check(lib().ckpt_chain_workspace_bytes_for(self._h, C.c_int(policy), C.byref(b)))
         return b.value
 
+    def set_keep_interiors(self, enable):
+        """ckpt_chain_set_keep_interiors: store-all steps keep every residual block's interior tensors."""
+        _check(lib().ckpt_chain_set_keep_interiors(self._h, C.c_int(1 if enable else 0)))
+
     def set_impl(self, impl):
         _check(lib().ckpt_chain_set_impl(self._h, C.c_int(impl)))
 

@@ -20,6 +20,7 @@ struct Unit {
     int param_first = 0, n_params = 0;
     int64_t stats_off = 0;       // float offset of this unit's saved batch statistics
     bool in_pending = false;     // the unit's input is a conv+BN+ReLU unit's stored output (normalisation applied on the way in)
+    int64_t blk_off = 0;         // residual block: offset of a region of its own when every block keeps its interiors
     ConvGeom geom;               // conv / fc as a convolution
     // bottleneck block: its four convolutions (1x1, 3x3 with the stride, 1x1, projection 1x1 with the stride)
     ConvGeom g1, g2, g3, gp;
@@ -49,6 +50,10 @@ struct ckpt_chain {
     // workspace layout (byte offsets)
     int64_t max_d = 0, off_g0 = 0, off_g1 = 0, off_z = 0, off_scr = 0, scr_bytes = 0, off_stats = 0,
             off_misc = 0, off_blk = 0, blk_bytes = 0, blk_lean_bytes = 0, ws_bytes = 0;
+    // Algorithm 1 taken literally (ckpt_chain_set_keep_interiors): every residual block keeps its interior tensors
+    // from the forward to the backward pass in a region of its own, blk_sum bytes in all
+    int keep_interiors = 0;
+    int64_t blk_sum = 0, z_bytes = 0;
     // graph replay: steps captured once per distinct argument set (pointers, plan, policy)
     int use_graph = 0;
     std::vector<ckpt::StepGraph> graphs;
@@ -111,6 +116,15 @@ struct StepCtx {
 };
 
 static const int64_t kGradId = 1000000007;   // arena id of the per-segment gradient buffer
+
+// Workspace layout per schedule: Algorithm 4's schedule stops before the tail of the block region and the buffer of
+// the activated copy; a store-all step that keeps block interiors has one block region per residual block.
+static bool keeps_interiors(const ckpt_chain* ch, int policy) { return ch->keep_interiors && policy == CKPT_POLICY_STORE_ALL; }
+static int64_t z_offset(const ckpt_chain* ch, int policy) { return keeps_interiors(ch, policy) ? ch->off_blk + ch->blk_sum : ch->off_z; }
+static int64_t workspace_need(const ckpt_chain* ch, int policy) {
+    if (policy == CKPT_POLICY_DYNAMIC) return ch->off_blk + ch->blk_lean_bytes;
+    return z_offset(ch, policy) + ch->z_bytes;
+}
 
 static int conv_forward_any(StepCtx& c, const ConvGeom& g, const void* x, const void* w, void* z,
                             const float* bias, int relu) {
@@ -206,7 +220,7 @@ static int64_t rows_of(const ckpt_chain* ch, int64_t j) { return ch->batch * ch-
 static int activated(StepCtx& c, int64_t j, const void* raw, const void** out) {
     *out = raw;
     if (!pending_act(c.ch, j)) return CKPT_OK;
-    void* xbuf = c.act_buf ? c.act_buf : c.ws + c.ch->off_z;
+    void* xbuf = c.act_buf ? c.act_buf : c.ws + z_offset(c.ch, c.policy);
     *out = xbuf;
     return bn_apply(c.ch->dtype, rows_of(c.ch, j), c.ch->shapes[j].c, raw, stats_of(c, j), 1, xbuf, c.stream);
 }
@@ -227,7 +241,7 @@ static BlockBuffers block_buffers(StepCtx& c, const Unit& u) {
     const int64_t m_in = align_up(in_px * u.desc.mid * es, 256), m_out = align_up(out_px * u.desc.mid * es, 256);
     const int64_t c_out = align_up(out_px * u.out.c * es, 256);
     BlockBuffers B;
-    char* p = c.ws + c.ch->off_blk;
+    char* p = c.ws + c.ch->off_blk + (keeps_interiors(c.ch, c.policy) ? u.blk_off : 0);
     const bool project = (u.desc.flags & 2) != 0;
     B.z1 = p; p += m_in; B.a = p; p += m_in; B.da = p; p += m_in;
     B.z2 = p; p += m_out; B.b = p; p += m_out; B.db = p; p += m_out;
@@ -293,7 +307,8 @@ static int block_backward(StepCtx& c, const Unit& u, const void* x, const void* 
     const int mid = u.desc.mid, co = u.out.c;
     const bool project = (u.desc.flags & 2) != 0;
     int rc;
-    if ((rc = block_interiors(c, u, x, B, true))) return rc;
+    // the interiors are re-derived from x, unless every block kept its own since the forward pass (store-all, literally)
+    if (!keeps_interiors(c.ch, c.policy) && (rc = block_interiors(c, u, x, B, true))) return rc;
     // through the final ReLU: g_in <- dL/d(bn3 + shortcut)
     if ((rc = relu_mask_inplace(dt, out_px * co, g_in, y, c.stream))) return rc;
     const void* dx_shortcut = g_in;                       // identity shortcut: the same gradient flows to x
@@ -666,6 +681,7 @@ static uint64_t step_key(const ckpt_chain* ch, const uint8_t* is_ckpt, int polic
     args->push_back((uint64_t)(uintptr_t)arena); args->push_back((uint64_t)(uintptr_t)ws);
     args->push_back((uint64_t)ch->impl);
     args->push_back((uint64_t)(uintptr_t)ch->tap); args->push_back((uint64_t)ch->selftest_wait);
+    args->push_back((uint64_t)ch->keep_interiors);
     { uint32_t bits; memcpy(&bits, &ch->sgd_lr, sizeof(bits)); args->push_back((uint64_t)bits); }
     for (size_t p = 0; p < ch->params.size(); ++p) { args->push_back((uint64_t)(uintptr_t)params[p]); args->push_back((uint64_t)(uintptr_t)grads[p]); }
     if (policy != CKPT_POLICY_STORE_ALL)
@@ -929,6 +945,8 @@ int ckpt_chain_create(const ckpt_unit_desc* units, int64_t n, int64_t batch, int
                 const int64_t blk = 3 * align_up(in_px * mid * es, 256) + 3 * align_up(out_px * mid * es, 256) + z3_bytes +
                                     (project ? z3_bytes + align_up(in_px * cur.c * es, 256) : 0);
                 u.in_pending = i >= 2 && units[i - 2].kind == CKPT_UNIT_CONV_BN_RELU;
+                u.blk_off = ch->blk_sum;
+                ch->blk_sum += blk;
                 ch->blk_bytes = std::max(ch->blk_bytes, blk);
                 ch->blk_lean_bytes = std::max(ch->blk_lean_bytes, u.in_pending ? blk : blk - z3_bytes);
                 break;
@@ -955,7 +973,8 @@ int ckpt_chain_create(const ckpt_unit_desc* units, int64_t n, int64_t batch, int
     ch->off_blk = o; o += ch->blk_bytes;
     // last: the buffer of the activated copy.  Algorithm 4's schedule never needs it (see run_step) and takes a
     // workspace that ends here
-    ch->off_z = o; o += std::max<int64_t>(max_z, 256);
+    ch->z_bytes = std::max<int64_t>(max_z, 256);
+    ch->off_z = o; o += ch->z_bytes;
     ch->ws_bytes = o;
     *out = ch;
     return CKPT_OK;
@@ -1025,13 +1044,13 @@ int ckpt_chain_param_info(const ckpt_chain* chain, int64_t p, int64_t* unit, int
 int ckpt_chain_workspace_bytes_for(const ckpt_chain* chain, int policy, int64_t* bytes) {
     if (!chain || !bytes) { set_error("null pointer"); return CKPT_E_NULL; }
     if (policy < 0 || policy > 2) { set_error("unknown policy %d", policy); return CKPT_E_BAD_ARG; }
-    *bytes = policy == CKPT_POLICY_DYNAMIC ? chain->off_blk + chain->blk_lean_bytes : chain->ws_bytes;
+    *bytes = workspace_need(chain, policy);
     return CKPT_OK;
 }
 
 int ckpt_chain_workspace_bytes(const ckpt_chain* chain, int64_t* bytes) {
     if (!chain || !bytes) { set_error("null pointer"); return CKPT_E_NULL; }
-    *bytes = chain->ws_bytes;
+    *bytes = std::max(workspace_need(chain, CKPT_POLICY_STORE_ALL), workspace_need(chain, CKPT_POLICY_STATIC));
     return CKPT_OK;
 }
 
@@ -1063,7 +1082,7 @@ int ckpt_train_step(ckpt_chain* chain, const uint8_t* is_ckpt, int policy, const
         set_error("arena of %lld bytes is smaller than the plan's peak of %lld bytes", (long long)arena_bytes, (long long)predicted);
         return CKPT_E_ARENA_OOM;
     }
-    const int64_t ws_need = policy == CKPT_POLICY_DYNAMIC ? chain->off_blk + chain->blk_lean_bytes : chain->ws_bytes;
+    const int64_t ws_need = workspace_need(chain, policy);
     report->workspace_bytes = ws_need;
     if (ws_bytes < ws_need) {
         set_error("workspace of %lld bytes, %lld needed", (long long)ws_bytes, (long long)ws_need);
@@ -1193,6 +1212,13 @@ int ckpt_chain_set_sgd(ckpt_chain* chain, double learning_rate) {
     if (!chain) { set_error("null pointer"); return CKPT_E_NULL; }
     if (!(learning_rate == learning_rate) || learning_rate < 0) { set_error("learning rate must be >= 0"); return CKPT_E_BAD_ARG; }
     chain->sgd_lr = (float)learning_rate;
+    return CKPT_OK;
+}
+
+int ckpt_chain_set_keep_interiors(ckpt_chain* chain, int enable) {
+    if (!chain) { set_error("null pointer"); return CKPT_E_NULL; }
+    chain->keep_interiors = enable ? 1 : 0;
+    drop_graphs(chain);
     return CKPT_OK;
 }
 

@@ -394,3 +394,43 @@ def test_staged_batches_equal_direct_steps(graph):
     with pytest.raises(ck.CkptError) as e:
         staged.chain.stage_batch(0, batches[0][0], batches[0][1], staging[:-256])
     assert e.value.code == -8
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_store_all_that_keeps_block_interiors(dtype):
+    """ckpt_chain_set_keep_interiors: a store-all step in which every residual block keeps its interior tensors from the
+    forward pass (a region of its own per block) instead of re-deriving them in its backward gives the same loss and
+    bit-identical gradients, launches fewer kernels, and leaves the checkpointed schedules as they were."""
+    import torch
+    if dtype == "f32":
+        spec = mini_resnet("f32")
+    else:
+        units = [{"kind": "bottleneck", "cin": 64, "mid": 64, "cout": 256, "stride": 1, "project": True},
+                 {"kind": "bottleneck", "cin": 256, "mid": 64, "cout": 256, "stride": 1, "project": False},
+                 {"kind": "bottleneck", "cin": 256, "mid": 128, "cout": 512, "stride": 2, "project": True},
+                 {"kind": "avgpool"}, {"kind": "fc", "cin": 512, "cout": 10, "relu": False}]
+        spec = dict(units=units, input_hwc=(12, 12, 64), batch=8, dtype="bf16", loss="softmax_ce", name="blocks_keep")
+    params = wl.make_params(spec, seed=51, bn_affine="random")
+    x, labels = wl.make_batch(spec, seed=52)
+    plain, keeping = StepRunner(spec, params), StepRunner(spec, params)
+    base_ws = keeping.chain.workspace_bytes()
+    keeping.chain.set_keep_interiors(True)
+    assert keeping.chain.workspace_bytes() > base_ws
+    assert keeping.chain.workspace_bytes_for(ck.POLICY_DYNAMIC) == plain.chain.workspace_bytes_for(ck.POLICY_DYNAMIC)
+    with pytest.raises(ck.CkptError) as e:                   # the old workspace is too small for the store-all policy now
+        keeping.run(ck.POLICY_STORE_ALL, None, x, labels)
+    assert e.value.code == -8
+    keeping.workspace = torch.empty(keeping.chain.workspace_bytes(), dtype=torch.uint8, device="cuda")
+    keeping.workspace.fill_(0xFF)
+    rep_a, g_a = plain.run(ck.POLICY_STORE_ALL, None, x, labels)
+    rep_b, g_b = keeping.run(ck.POLICY_STORE_ALL, None, x, labels)
+    assert rep_a["loss"] == rep_b["loss"] and rep_b["device_status"] == 0
+    assert rep_b["launches"] < rep_a["launches"]
+    for a, b in zip(g_a, g_b):
+        assert np.array_equal(a, b)
+    mask = ck.plan(ck.ALGO_DYNAMIC_N, plain.d)[0]
+    rep_c, g_c = keeping.run(ck.POLICY_DYNAMIC, mask, x, labels)
+    rep_d, _ = plain.run(ck.POLICY_DYNAMIC, mask, x, labels)
+    assert rep_c["launches"] == rep_d["launches"] and rep_c["peak_bytes"] == rep_d["peak_bytes"]
+    for a, b in zip(g_a, g_c):
+        assert np.array_equal(a, b)
